@@ -1,0 +1,177 @@
+/*
+ * fsharp.h -- C ABI of the FAVOR# hot path on one NVIDIA B200 (sm_100a).
+ *
+ * FAVOR# approximates softmax attention with dense exponential random
+ * features (DERFs, Section 4 of the paper):
+ *
+ *   f^(k)(w, x) = D exp(w^T A w + w^T B^(k) x + x^T C^(k) x),  k = 1 (queries), 2 (keys)
+ *   P_i = M^-1/2 (f^(1)(w_m, x_i))_m,   S_j = M^-1/2 (f^(2)(w_m, y_j))_m       (Section 2.1)
+ *   Y   = diag(P S^T 1)^-1 P S^T V                                              (Section 2.2)
+ *
+ * The calls follow the paper's statement of the problem:
+ *   fsharp_stats          set statistics M1, M2, mu4, mu5 of Theorems 4.2 / 4.3
+ *   fsharp_fit_params     closed-form optimal A, B, C, D per parameter group
+ *   fsharp_featurize      P or S for given parameters
+ *   fsharp_attend         Y, bidirectional or causal (lower-triangular mask)
+ *   fsharp_pair_estimate  Khat(x, y) for pairs, with Theorem 4.1's variance
+ *
+ * Conventions common to every call
+ *   - All data pointers are DEVICE pointers owned by the caller unless the
+ *     parameter is documented as host memory.  The library neither frees them
+ *     nor keeps them after the call's work has finished on the stream.
+ *   - Work is enqueued on the context's stream and the call returns without
+ *     waiting, except where stated.
+ *   - Tensors are addressed through element strides (batch, head, token); the
+ *     innermost dimension (d, dv or M) is contiguous.  A stride triple of
+ *     zeros means dense [B, H, L, inner].
+ *   - Every function returns 0 on success or a negative FSHARP_E_* code.
+ *     Nothing aborts, throws or traps.  Conditions found on the device
+ *     (non-finite input, singular M1/M2, 8A not below I, a bounded wait that
+ *     ran out) are latched in a device status word read by fsharp_status().
+ *   - x = qk_scale * Q_i and y = qk_scale * K_j.  Section 2.2 uses
+ *     qk_scale = d^-1/4; pass 1 if the tensors already hold x and y.
+ *   - Supported shapes: d, dv in {16, 32, 64, 128}; M a multiple of 16, at
+ *     most 1024; causal needs Lq == Lk and chunk in {64, 128, 256} dividing L.
+ */
+#ifndef FSHARP_H
+#define FSHARP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fsharp_ctx fsharp_ctx;
+
+enum {
+  FSHARP_OK = 0,
+  FSHARP_E_BADARG = -1,     /* null pointer, unknown enum value */
+  FSHARP_E_SHAPE = -2,      /* unsupported or inconsistent sizes */
+  FSHARP_E_ALIGN = -3,      /* base pointer or stride not 16-byte aligned */
+  FSHARP_E_DTYPE = -4,
+  FSHARP_E_NOMEM = -5,      /* workspace allocation failed */
+  FSHARP_E_CONSTRAINT = -6, /* Theorem 4.1 / 4.2 preconditions violated (device-detected) */
+  FSHARP_E_NONFINITE = -7,  /* NaN or Inf met on the device */
+  FSHARP_E_TIMEOUT = -8,    /* a bounded device-side wait expired */
+  FSHARP_E_CUDA = -9        /* a CUDA runtime or driver call failed */
+};
+
+enum { FSHARP_F32 = 0, FSHARP_BF16 = 1 };
+enum { FSHARP_POSRF = 0, FSHARP_GERF = 1, FSHARP_SADERF = 2, FSHARP_ADERF = 3, FSHARP_SDERF = 4 };
+enum { FSHARP_POOL_PER_BH = 0, FSHARP_POOL_PER_HEAD = 1 };
+enum { FSHARP_STAB_NONE = 0, FSHARP_STAB_ROW = 1, FSHARP_STAB_GROUP = 2 };
+enum { FSHARP_IMPL_AUTO = 0, FSHARP_IMPL_SIMT = 1, FSHARP_IMPL_TENSOR = 2 };
+
+/* Problem sizes and addressing.  G, the number of parameter groups, is B*H for
+ * pool == FSHARP_POOL_PER_BH (one operator instance per group, as Theorems 4.2
+ * and 4.3 define the statistics) and H for FSHARP_POOL_PER_HEAD (statistics
+ * pooled over the batch).  Group of (b, h): b*H + h, respectively h. */
+typedef struct {
+  int32_t B, H, Lq, Lk, d, dv, M;
+  int32_t pool;
+  int64_t q_stride[3];        /* element strides of Q: batch, head, token */
+  int64_t k_stride[3];
+  int64_t v_stride[3];
+  int64_t y_stride[3];
+  int64_t omega_head_stride;  /* elements between the Omegas of two heads; 0 = one shared Omega */
+} fsharp_dims;
+
+/* ---- context ------------------------------------------------------------ */
+
+/* Creates a context on CUDA device `device` that enqueues on `stream`
+ * (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ * The context owns a scratch workspace in device memory that grows on demand
+ * (growing synchronises the stream) and a device status word. */
+int fsharp_create(fsharp_ctx** out, int device, void* stream);
+int fsharp_destroy(fsharp_ctx* ctx);
+int fsharp_set_stream(fsharp_ctx* ctx, void* stream);
+/* Forces a kernel family for fsharp_attend (FSHARP_IMPL_*).  AUTO picks the
+ * tensor-core path when the shape allows it (bf16, d = dv in {64, 128}). */
+int fsharp_set_impl(fsharp_ctx* ctx, int impl);
+/* Synchronises the stream, then returns the latched device status in *code
+ * (0 or a negative FSHARP_E_*), and clears it. */
+int fsharp_status(fsharp_ctx* ctx, int* code);
+/* Number of kernels this context has launched since creation. */
+int64_t fsharp_launch_count(const fsharp_ctx* ctx);
+/* Bytes of scratch the context currently holds. */
+size_t fsharp_workspace_bytes(const fsharp_ctx* ctx);
+const char* fsharp_strerror(int code);
+
+/* ---- layouts of the two fp64 blobs ---------------------------------------- */
+
+/* Doubles per group in the statistics blob:
+ *   [M1 (d*d, row-major)] [M2 (d*d)] [mu4 (d)] [mu5 (d)] [max_i |x_i|^2] [max_j |y_j|^2]
+ * = 2 d^2 + 2 d + 2. */
+size_t fsharp_stats_doubles(int d);
+/* Doubles per group in the parameter blob:
+ *   [A (d*d, symmetric)] [B1 (d*d)] [B2 (d*d)] [C1 (d*d)] [C2 (d*d)]
+ *   [logD] [objective] [phi] [kappa1] [kappa2] [rho2max_x] [rho2max_y] [reserved]
+ * = 5 d^2 + 8.  objective is the shifted log-variance of Section 3.1 at the
+ * optimum (Theorems 4.2 / 4.3); phi is the argument of Lemma A.1 (ADERF, GERF,
+ * SADERF; for SDERF the largest eigenvalue of N).  kappa_k >= 0 is a lower bound on
+ * the smallest eigenvalue of -C^(k) and rho2max the largest squared norm in the
+ * set; they only steer the overflow guard (any per-row factor on queries and any
+ * per-group factor on keys cancels in Section 2.2's normalisation), never the
+ * mathematical result.  A caller who writes a blob by hand may set kappa = 0 and
+ * rho2max to the largest squared norm it expects. */
+size_t fsharp_params_doubles(int d);
+
+/* ---- the path -------------------------------------------------------------- */
+
+/* Statistics of Theorem 4.2 (M1 = L^-1 sum x x^T, M2 likewise for y) and Theorem
+ * 4.3 (mu4 = mean x, mu5 = mean y) for every group, from Q [B,H,Lq,d] and
+ * K [B,H,Lk,d] of type `dtype`.  stats: device, G * fsharp_stats_doubles(d). */
+int fsharp_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dims* dims,
+                 int dtype, float qk_scale, double* stats);
+
+/* Closed-form minimisers of the shifted log-variance objective (Section 3.1):
+ * PosRF and GERF (Section 2.3 / 3.1), SADERF (Section 4.3), ADERF (Theorem 4.2),
+ * SDERF (Theorem 4.3), all through Lemma A.1's scalar map.  The symmetric
+ * eigenproblems are solved on the device by a cyclic Jacobi method in fp64, one
+ * thread block per group.  ADERF uses eig(M1) and eig(L1^1/2 Q1^T M2 Q1 L1^1/2),
+ * whose eigenvectors and eigenvalues are U and Sigma^2 of the theorem's SVD.
+ * ridge >= 0 adds ridge * tr(M)/d * I to M1 and M2 first (0 = the paper's formulas).
+ * stats: device, G groups.  params: device, G * fsharp_params_doubles(d). */
+int fsharp_fit_params(fsharp_ctx* ctx, const double* stats, int G, int d, int variant,
+                      double ridge, double* params);
+
+/* P (side = 1, parameters B1, C1) or S (side = 2, B2, C2) of Section 2.1 for the
+ * DERF of Section 4: phi[b,h,i,m] * exp(logscale) = M^-1/2 D exp(w_m^T A w_m +
+ * w_m^T B x_i + x_i^T C x_i).  X is addressed with (Lq, q_stride) for side 1 and
+ * (Lk, k_stride) for side 2.  Omega: float32 [M, d] (or [H, M, d]).
+ * phi: float32, dense [B,H,L,M].  logscale: float32, [B,H,L] for FSHARP_STAB_ROW,
+ * [B,H] for FSHARP_STAB_GROUP, ignored (may be NULL) for FSHARP_STAB_NONE. */
+int fsharp_featurize(fsharp_ctx* ctx, const void* X, const float* Omega, const double* params,
+                     int side, const fsharp_dims* dims, int dtype, float qk_scale, int stab,
+                     float* phi, float* logscale);
+
+/* Y [B,H,Lq,dv] (type `dtype`) of Section 2.2 with Khat = P S^T in place of the
+ * exact kernel matrix, evaluated as P (S^T [V | 1]) (Section 2.1's O(L M n) order).
+ * causal != 0 restricts key j to j <= i and evaluates chunk by chunk with a running
+ * prefix of S^T [V | 1]; chunk is ignored when causal == 0. */
+int fsharp_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V,
+                  const float* Omega, const double* params, const fsharp_dims* dims,
+                  int dtype, int causal, int chunk, float qk_scale, void* Y);
+
+/* The whole path on HOST buffers: copies Q, K, V (dense [B,H,L,*], type `dtype`)
+ * to the device, runs stats -> fit -> attend, copies Y back and waits for it.
+ * Q, K, V, Y: host memory (pinned memory makes the copies asynchronous).
+ * Omega: host float32 [M, d].  dims' strides are ignored (dense). */
+int fsharp_forward_host(fsharp_ctx* ctx, const void* Q, const void* K, const void* V,
+                        const float* Omega, const fsharp_dims* dims, int dtype, int variant,
+                        int causal, int chunk, float qk_scale, void* Y);
+
+/* Kernel estimates for npairs (x_p, y_p) pairs (Section 2.1: Khat = sum_m P_pm S_pm)
+ * with R independent feature draws: X, Y float32 [npairs, d]; Omega float32
+ * [R, M, d]; params: one group; est: float32 [R, npairs].  If var_cf is not NULL it
+ * receives, per pair, Theorem 4.1's variance divided by M (needs a diagonal A). */
+int fsharp_pair_estimate(fsharp_ctx* ctx, const float* X, const float* Y, const float* Omega,
+                         const double* params, int64_t npairs, int d, int M, int R,
+                         float* est, double* var_cf);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FSHARP_H */

@@ -1,0 +1,151 @@
+// Shared declarations of the FAVOR# library: context, blob layouts, launch helpers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/fsharp.h"
+
+#define FS_LOG2E 1.4426950408889634f
+
+// Layout of the per-group parameter blob (doubles); see fsharp_params_doubles().
+struct ParamsLayout {
+  int d;
+  __host__ __device__ size_t dd() const { return (size_t)d * d; }
+  __host__ __device__ size_t A() const { return 0; }
+  __host__ __device__ size_t B(int k) const { return dd() * (size_t)k; }        // k = 1, 2
+  __host__ __device__ size_t C(int k) const { return dd() * (size_t)(2 + k); }  // k = 1, 2
+  __host__ __device__ size_t tail() const { return 5 * dd(); }
+  __host__ __device__ size_t total() const { return 5 * dd() + 8; }
+};
+enum { PT_LOGD = 0, PT_OBJ = 1, PT_PHI = 2, PT_KAPPA1 = 3, PT_KAPPA2 = 4, PT_RHO2X = 5, PT_RHO2Y = 6, PT_RES = 7 };
+
+struct StatsLayout {
+  int d;
+  __host__ __device__ size_t M(int k) const { return (size_t)d * d * (size_t)(k - 1); }               // k = 1, 2
+  __host__ __device__ size_t mu(int k) const { return 2 * (size_t)d * d + (size_t)d * (k - 4); }      // k = 4, 5
+  __host__ __device__ size_t rho2(int k) const { return 2 * (size_t)d * d + 2 * (size_t)d + (k - 1); }  // k = 1, 2
+  __host__ __device__ size_t total() const { return 2 * (size_t)d * d + 2 * (size_t)d + 2; }
+};
+
+// What prep produces per (group, side): everything the feature kernels need (fp32).
+//   W      [M, d]  row m = (B^T w_m)^T
+//   a      [M]     w_m^T A w_m
+//   scal   [8]     see PS_* below
+//   Cmat   [d, d]  copy of C (row-major)
+struct PrepLayout {
+  int d, M;
+  __host__ __device__ size_t W() const { return 0; }
+  __host__ __device__ size_t a() const { return (size_t)M * d; }
+  __host__ __device__ size_t scal() const { return (size_t)M * d + M; }
+  __host__ __device__ size_t Cmat() const { return (size_t)M * d + M + 8; }
+  __host__ __device__ size_t total() const { return (size_t)M * d + M + 8 + (size_t)d * d; }
+};
+// PS_BIAS logD - 1/2 log M; PS_AMAX max_m a_m; PS_WMAX max_m |W_m|; PS_CSCALAR 1 if C = gamma I;
+// PS_CGAMMA gamma; PS_GSHIFT the per-group shift used for keys; PS_KAPPA, PS_RHO2 copied from the blob.
+enum { PS_BIAS = 0, PS_AMAX = 1, PS_WMAX = 2, PS_CSCALAR = 3, PS_CGAMMA = 4, PS_GSHIFT = 5, PS_KAPPA = 6, PS_RHO2 = 7 };
+
+// Headroom (natural-log units) left above the guaranteed upper bound of a key
+// exponent when the per-group shift is chosen: key features are at most
+// exp(FS_MARGIN); sums of up to 2^17 of them times |V| stay far below exp(88).
+#define FS_MARGIN 40.0f
+
+struct fsharp_ctx {
+  int device;
+  cudaStream_t stream;
+  int impl;
+  char* ws;
+  size_t ws_bytes;
+  int* d_status;      // device status word
+  int64_t launches;
+  int sm_count;
+};
+
+// Bump allocator over the context workspace.
+struct WsAlloc {
+  char* base;
+  size_t off;
+  template <typename T>
+  T* take(size_t n) {
+    size_t bytes = (n * sizeof(T) + 255) & ~(size_t)255;
+    T* p = reinterpret_cast<T*>(base + off);
+    off += bytes;
+    return p;
+  }
+};
+static inline size_t ws_round(size_t bytes) { return (bytes + 255) & ~(size_t)255; }
+
+int fs_ws_reserve(fsharp_ctx* ctx, size_t bytes);   // grows the workspace; FSHARP_OK or error
+
+#define FS_CUDA_OK(expr)                         \
+  do {                                           \
+    cudaError_t _e = (expr);                     \
+    if (_e != cudaSuccess) {                     \
+      (void)cudaGetLastError();                  \
+      return FSHARP_E_CUDA;                      \
+    }                                            \
+  } while (0)
+
+#define FS_LAUNCH_CHECK(ctx)                                   \
+  do {                                                         \
+    (ctx)->launches++;                                         \
+    if (cudaPeekAtLastError() != cudaSuccess) {                \
+      (void)cudaGetLastError();                                \
+      return FSHARP_E_CUDA;                                    \
+    }                                                          \
+  } while (0)
+
+#define FS_TRY(expr)                 \
+  do {                               \
+    int _rc = (expr);                \
+    if (_rc != FSHARP_OK) return _rc; \
+  } while (0)
+
+// Resolved addressing of one [B,H,L,inner] tensor.
+struct TensorAddr {
+  int64_t sb, sh, sl;
+};
+static inline TensorAddr fs_addr(const int64_t s[3], int H, int L, int inner) {
+  TensorAddr t;
+  if (s[0] == 0 && s[1] == 0 && s[2] == 0) {
+    t.sl = inner;
+    t.sh = (int64_t)L * inner;
+    t.sb = (int64_t)H * L * inner;
+  } else {
+    t.sb = s[0];
+    t.sh = s[1];
+    t.sl = s[2];
+  }
+  return t;
+}
+
+__device__ __forceinline__ float fs_load(const float* p) { return *p; }
+__device__ __forceinline__ float fs_load(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+__device__ __forceinline__ void fs_store(float* p, float v) { *p = v; }
+__device__ __forceinline__ void fs_store(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+static inline int fs_groups(const fsharp_dims* dm) {
+  return dm->pool == FSHARP_POOL_PER_BH ? dm->B * dm->H : dm->H;
+}
+
+// ---- stage entry points (host side, defined in the .cu files) -------------
+int fs_run_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dims* dm, int dtype,
+                 float qk_scale, double* stats);
+int fs_run_fit(fsharp_ctx* ctx, const double* stats, int G, int d, int variant, double ridge,
+               double* params, double* scratch);
+size_t fs_fit_scratch_doubles(int G, int d);
+int fs_run_prep(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_stride, const double* params,
+                int G, int H, int pool, int d, int M, float* prep /* [G][2][PrepLayout] */);
+// rowc: scratch [B*H*L] floats.  phi: [B,H,L,M] floats.
+int fs_simt_featurize(fsharp_ctx* ctx, const void* X, int dtype, TensorAddr ax, int B, int H, int L, int d,
+                      int M, int pool, const float* prep, int side, float qk_scale, int stab,
+                      float* rowc, float* phi, float* logscale);
+int fs_simt_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm,
+                   int dtype, int causal, int chunk, float qk_scale, const float* prep, void* Y,
+                   WsAlloc* ws);
+size_t fs_simt_attend_scratch_bytes(const fsharp_dims* dm, int causal, int chunk);
+int fs_run_pairs(fsharp_ctx* ctx, const float* X, const float* Y, const float* Omega, const double* params,
+                 int64_t npairs, int d, int M, int R, float* est, double* var_cf, WsAlloc* ws);
+size_t fs_pairs_scratch_bytes(int d, int M, int R);

@@ -1,0 +1,123 @@
+// Context, workspace and status handling of the FAVOR# library.
+#include <new>
+
+#include "common.cuh"
+
+extern "C" {
+
+int fsharp_create(fsharp_ctx** out, int device, void* stream) {
+  if (!out) return FSHARP_E_BADARG;
+  *out = nullptr;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) {
+    (void)cudaGetLastError();
+    return FSHARP_E_CUDA;
+  }
+  FS_CUDA_OK(cudaSetDevice(device));
+  fsharp_ctx* c = new (std::nothrow) fsharp_ctx();
+  if (!c) return FSHARP_E_NOMEM;
+  c->device = device;
+  c->stream = reinterpret_cast<cudaStream_t>(stream);
+  c->impl = FSHARP_IMPL_AUTO;
+  c->ws = nullptr;
+  c->ws_bytes = 0;
+  c->launches = 0;
+  c->d_status = nullptr;
+  c->sm_count = 148;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) == cudaSuccess) c->sm_count = prop.multiProcessorCount;
+  if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess) {
+    (void)cudaGetLastError();
+    delete c;
+    return FSHARP_E_NOMEM;
+  }
+  if (cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess) {
+    (void)cudaGetLastError();
+    cudaFree(c->d_status);
+    delete c;
+    return FSHARP_E_CUDA;
+  }
+  *out = c;
+  return FSHARP_OK;
+}
+
+int fsharp_destroy(fsharp_ctx* ctx) {
+  if (!ctx) return FSHARP_E_BADARG;
+  cudaSetDevice(ctx->device);
+  cudaStreamSynchronize(ctx->stream);
+  if (ctx->ws) cudaFree(ctx->ws);
+  if (ctx->d_status) cudaFree(ctx->d_status);
+  delete ctx;
+  return FSHARP_OK;
+}
+
+int fsharp_set_stream(fsharp_ctx* ctx, void* stream) {
+  if (!ctx) return FSHARP_E_BADARG;
+  ctx->stream = reinterpret_cast<cudaStream_t>(stream);
+  return FSHARP_OK;
+}
+
+int fsharp_set_impl(fsharp_ctx* ctx, int impl) {
+  if (!ctx || impl < FSHARP_IMPL_AUTO || impl > FSHARP_IMPL_TENSOR) return FSHARP_E_BADARG;
+  ctx->impl = impl;
+  return FSHARP_OK;
+}
+
+int fsharp_status(fsharp_ctx* ctx, int* code) {
+  if (!ctx || !code) return FSHARP_E_BADARG;
+  FS_CUDA_OK(cudaStreamSynchronize(ctx->stream));
+  int h = 0;
+  FS_CUDA_OK(cudaMemcpy(&h, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (h != 0) FS_CUDA_OK(cudaMemset(ctx->d_status, 0, sizeof(int)));
+  *code = h;
+  return FSHARP_OK;
+}
+
+int64_t fsharp_launch_count(const fsharp_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+size_t fsharp_workspace_bytes(const fsharp_ctx* ctx) { return ctx ? ctx->ws_bytes : 0; }
+
+const char* fsharp_strerror(int code) {
+  switch (code) {
+    case FSHARP_OK: return "ok";
+    case FSHARP_E_BADARG: return "bad argument";
+    case FSHARP_E_SHAPE: return "unsupported or inconsistent shape";
+    case FSHARP_E_ALIGN: return "pointer or stride not 16-byte aligned";
+    case FSHARP_E_DTYPE: return "unsupported dtype";
+    case FSHARP_E_NOMEM: return "out of memory";
+    case FSHARP_E_CONSTRAINT: return "parameter constraint violated (singular M or 8A not below I)";
+    case FSHARP_E_NONFINITE: return "non-finite value met on the device";
+    case FSHARP_E_TIMEOUT: return "bounded device-side wait expired";
+    case FSHARP_E_CUDA: return "CUDA call failed";
+    default: return "unknown error";
+  }
+}
+
+size_t fsharp_stats_doubles(int d) { return StatsLayout{d}.total(); }
+size_t fsharp_params_doubles(int d) { return ParamsLayout{d}.total(); }
+
+}  // extern "C"
+
+int fs_ws_reserve(fsharp_ctx* ctx, size_t bytes) {
+  if (bytes <= ctx->ws_bytes) return FSHARP_OK;
+  // Growing: wait for work that may still use the old block, then replace it.
+  FS_CUDA_OK(cudaStreamSynchronize(ctx->stream));
+  if (ctx->ws) {
+    cudaFree(ctx->ws);
+    ctx->ws = nullptr;
+    ctx->ws_bytes = 0;
+  }
+  size_t want = bytes + (bytes >> 3);
+  void* p = nullptr;
+  if (cudaMalloc(&p, want) != cudaSuccess) {
+    (void)cudaGetLastError();
+    want = bytes;
+    if (cudaMalloc(&p, want) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return FSHARP_E_NOMEM;
+    }
+  }
+  ctx->ws = static_cast<char*>(p);
+  ctx->ws_bytes = want;
+  return FSHARP_OK;
+}
