@@ -1,0 +1,363 @@
+// Closed-form parameter fits (Section 3.1, Section 4.3, Theorems 4.2 and 4.3, Lemma A.1)
+// with an fp64 cyclic Jacobi eigensolver, one thread block per parameter group.
+#include "common.cuh"
+
+namespace {
+
+constexpr int FIT_THREADS = 256;
+constexpr int JACOBI_MAX_SWEEPS = 40;
+
+__device__ __forceinline__ double block_reduce(double v, double* red, int op /*0 sum, 1 max, 2 min*/) {
+  const int tid = threadIdx.x;
+  __syncthreads();
+  red[tid] = v;
+  __syncthreads();
+  for (int s = FIT_THREADS / 2; s > 0; s >>= 1) {
+    if (tid < s) {
+      double a = red[tid], b = red[tid + s];
+      red[tid] = op == 0 ? a + b : (op == 1 ? fmax(a, b) : fmin(a, b));
+    }
+    __syncthreads();
+  }
+  double r = red[0];
+  __syncthreads();
+  return r;
+}
+
+// Lemma A.1 in the cancellation-free form that follows from its proof:
+// 1 - 8A = (2 phi + 1 + s)/2 with s = sqrt((2 phi + 1)^2 + 8 phi).
+__device__ __forceinline__ double lemma_a1(double phi) {
+  double s = sqrt((2.0 * phi + 1.0) * (2.0 * phi + 1.0) + 8.0 * phi);
+  return -(2.0 * phi + (12.0 * phi + 4.0 * phi * phi) / (1.0 + s)) / 16.0;
+}
+
+// Two-sided cyclic Jacobi with the round-robin ("tournament") ordering: every round
+// rotates d/2 disjoint index pairs at once.  On exit the diagonal of A holds the
+// eigenvalues and the columns of V the eigenvectors.  A: d x d, leading dimension
+// lda; V likewise.  cs: 2*d doubles, pq: 2*d ints, red: FIT_THREADS doubles (shared).
+__device__ void jacobi_eig(double* A, int lda, double* V, int ldv, int d, double* cs, int* pq, double* red) {
+  const int tid = threadIdx.x;
+  const int half = d / 2;
+  for (int e = tid; e < d * d; e += FIT_THREADS) V[(e / d) * ldv + (e % d)] = (e / d == e % d) ? 1.0 : 0.0;
+  __syncthreads();
+  for (int sweep = 0; sweep < JACOBI_MAX_SWEEPS; sweep++) {
+    double off = 0.0, tot = 0.0;
+    for (int e = tid; e < d * d; e += FIT_THREADS) {
+      int i = e / d, j = e % d;
+      double v = A[i * lda + j];
+      tot += v * v;
+      if (i != j) off += v * v;
+    }
+    off = block_reduce(off, red, 0);
+    tot = block_reduce(tot, red, 0);
+    if (off <= 1e-26 * tot || tot == 0.0) break;
+    for (int r = 0; r < d - 1; r++) {
+      if (tid < half) {
+        int p, q;
+        if (tid == 0) { p = r; q = d - 1; }
+        else { p = (r + tid) % (d - 1); q = (r - tid + (d - 1)) % (d - 1); }
+        if (p > q) { int t = p; p = q; q = t; }
+        double app = A[p * lda + p], aqq = A[q * lda + q], apq = A[p * lda + q];
+        double c = 1.0, s = 0.0;
+        if (fabs(apq) > 1e-300) {
+          double tau = (aqq - app) / (2.0 * apq);
+          double t = copysign(1.0, tau) / (fabs(tau) + sqrt(1.0 + tau * tau));
+          c = 1.0 / sqrt(1.0 + t * t);
+          s = t * c;
+        }
+        cs[2 * tid] = c; cs[2 * tid + 1] = s;
+        pq[2 * tid] = p; pq[2 * tid + 1] = q;
+      }
+      __syncthreads();
+      for (int e = tid; e < half * d; e += FIT_THREADS) {        // A <- A J, V <- V J
+        int k = e / d, row = e % d;
+        int p = pq[2 * k], q = pq[2 * k + 1];
+        double c = cs[2 * k], s = cs[2 * k + 1];
+        double x = A[row * lda + p], y = A[row * lda + q];
+        A[row * lda + p] = c * x - s * y;
+        A[row * lda + q] = s * x + c * y;
+        x = V[row * ldv + p]; y = V[row * ldv + q];
+        V[row * ldv + p] = c * x - s * y;
+        V[row * ldv + q] = s * x + c * y;
+      }
+      __syncthreads();
+      for (int e = tid; e < half * d; e += FIT_THREADS) {        // A <- J^T A
+        int k = e / d, col = e % d;
+        int p = pq[2 * k], q = pq[2 * k + 1];
+        double c = cs[2 * k], s = cs[2 * k + 1];
+        double x = A[p * lda + col], y = A[q * lda + col];
+        A[p * lda + col] = c * x - s * y;
+        A[q * lda + col] = s * x + c * y;
+      }
+      __syncthreads();
+    }
+  }
+  __syncthreads();
+}
+
+struct FitArgs {
+  const double* stats;
+  double* params;
+  double* scratch;   // per group 4*d*d doubles
+  int d, variant;
+  double ridge;
+  int v_in_smem;
+  int* status;
+};
+
+__global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
+  extern __shared__ double sm[];
+  const int d = a.d, tid = threadIdx.x, g = blockIdx.x;
+  const int lda = d + 1;
+  StatsLayout sl{d};
+  ParamsLayout pl{d};
+  const double* st = a.stats + (size_t)g * sl.total();
+  double* out = a.params + (size_t)g * pl.total();
+  double* gs = a.scratch + (size_t)g * 4 * d * d;
+
+  double* As = sm;                                   // d*(d+1)
+  double* Vs = a.v_in_smem ? As + d * lda : gs;      // eigenvectors
+  const int ldv = a.v_in_smem ? lda : d;
+  double* vec = As + d * lda + (a.v_in_smem ? d * lda : 0);
+  double* lam = vec;             // [d]
+  double* aux = vec + d;         // [d]
+  double* cs = vec + 2 * d;      // [2d]
+  double* red = vec + 4 * d;     // [FIT_THREADS]
+  int* pq = reinterpret_cast<int*>(red + FIT_THREADS);   // [2d]
+  int* perm = pq + 2 * d;                                 // [d]
+
+  const double* M1 = st + sl.M(1);
+  const double* M2 = st + sl.M(2);
+  const double* mu4 = st + sl.mu(4);
+  const double* mu5 = st + sl.mu(5);
+
+  // traces, mu4.mu5, finiteness
+  double t1 = 0.0, t2 = 0.0, mm = 0.0, badv = 0.0;
+  for (int i = tid; i < d; i += FIT_THREADS) {
+    t1 += M1[i * d + i];
+    t2 += M2[i * d + i];
+    mm += mu4[i] * mu5[i];
+  }
+  for (int e = tid; e < (int)sl.total(); e += FIT_THREADS)
+    if (!isfinite(st[e])) badv = 1.0;
+  t1 = block_reduce(t1, red, 0);
+  t2 = block_reduce(t2, red, 0);
+  mm = block_reduce(mm, red, 0);
+  badv = block_reduce(badv, red, 1);
+  if (badv > 0.0 && tid == 0) atomicExch(a.status, FSHARP_E_NONFINITE);
+  const double rg1 = a.ridge * t1 / d, rg2 = a.ridge * t2 / d;
+  t1 += d * rg1;
+  t2 += d * rg2;
+
+  double* oA = out + pl.A();
+  double* oB1 = out + pl.B(1);
+  double* oB2 = out + pl.B(2);
+  double* oC1 = out + pl.C(1);
+  double* oC2 = out + pl.C(2);
+  double* tail = out + pl.tail();
+  double logD = 0.0, obj = 0.0, phi = 0.0, kap1 = 0.5, kap2 = 0.5;
+  bool violated = false;
+
+  if (a.variant == FSHARP_POSRF || a.variant == FSHARP_GERF) {
+    const double S = t1 + t2 + 2.0 * mm;
+    double A = 0.0;
+    if (a.variant == FSHARP_GERF) { phi = S / d; A = lemma_a1(phi); }
+    const double b = sqrt(1.0 - 4.0 * A);
+    for (int e = tid; e < d * d; e += FIT_THREADS) {
+      double dg = (e / d == e % d) ? 1.0 : 0.0;
+      oA[e] = A * dg; oB1[e] = b * dg; oB2[e] = b * dg; oC1[e] = -0.5 * dg; oC2[e] = -0.5 * dg;
+    }
+    logD = 0.25 * d * log(1.0 - 4.0 * A);
+    obj = d * (log(1.0 - 4.0 * A) - 0.5 * log(1.0 - 8.0 * A)) + (2.0 - 8.0 * A) / (1.0 - 8.0 * A) * S - t1 - t2;
+  } else if (a.variant == FSHARP_SADERF) {
+    // Section 4.3: Psi_ll = (M2_ll / M1_ll)^(1/4), then the GERF fit on {Psi x}, {Psi^-1 y}.
+    double sq = 0.0, kmin1 = 1e300, kmin2 = 1e300;
+    for (int i = tid; i < d; i += FIT_THREADS) {
+      double m1 = M1[i * d + i] + rg1, m2 = M2[i * d + i] + rg2;
+      if (!(m1 > 0.0) || !(m2 > 0.0)) { violated = true; m1 = fmax(m1, 1e-300); m2 = fmax(m2, 1e-300); }
+      double psi2 = sqrt(m2 / m1);
+      lam[i] = sqrt(psi2);
+      sq += sqrt(m1 * m2);
+      kmin1 = fmin(kmin1, psi2);
+      kmin2 = fmin(kmin2, 1.0 / psi2);
+    }
+    sq = block_reduce(sq, red, 0);
+    kap1 = 0.5 * block_reduce(kmin1, red, 2);
+    kap2 = 0.5 * block_reduce(kmin2, red, 2);
+    const double S = 2.0 * sq + 2.0 * mm;
+    phi = S / d;
+    const double A = lemma_a1(phi);
+    const double b = sqrt(1.0 - 4.0 * A);
+    for (int e = tid; e < d * d; e += FIT_THREADS) {
+      int i = e / d;
+      double dg = (i == e % d) ? 1.0 : 0.0, psi = lam[i];
+      oA[e] = A * dg; oB1[e] = b * psi * dg; oB2[e] = b / psi * dg;
+      oC1[e] = -0.5 * psi * psi * dg; oC2[e] = -0.5 / (psi * psi) * dg;
+    }
+    logD = 0.25 * d * log(1.0 - 4.0 * A);
+    obj = d * (log(1.0 - 4.0 * A) - 0.5 * log(1.0 - 8.0 * A)) + (2.0 - 8.0 * A) / (1.0 - 8.0 * A) * S - 2.0 * sq;
+  } else if (a.variant == FSHARP_SDERF) {
+    // Theorem 4.3: N = M1 + mu4 mu5^T + mu5 mu4^T + M2, eigenvalues non-ascending.
+    for (int e = tid; e < d * d; e += FIT_THREADS) {
+      int i = e / d, j = e % d;
+      As[i * lda + j] = M1[e] + M2[e] + mu4[i] * mu5[j] + mu5[i] * mu4[j] + (i == j ? rg1 + rg2 : 0.0);
+    }
+    __syncthreads();
+    jacobi_eig(As, lda, Vs, ldv, d, cs, pq, red);
+    for (int i = tid; i < d; i += FIT_THREADS) {
+      double li = As[i * lda + i];
+      int rank = 0;
+      for (int j = 0; j < d; j++) {
+        double lj = As[j * lda + j];
+        rank += (lj > li) || (lj == li && j < i);
+      }
+      perm[rank] = i;
+    }
+    __syncthreads();
+    double sl_log = 0.0, so = 0.0;
+    for (int l = tid; l < d; l += FIT_THREADS) {
+      double lv = fmax(As[perm[l] * lda + perm[l]], 0.0);   // N is PSD; rounding may give -1e-17
+      double al = lemma_a1(lv);
+      lam[l] = lv;
+      aux[l] = al;
+      sl_log += log(1.0 - 4.0 * al);
+      so += log(1.0 - 4.0 * al) - 0.5 * log(1.0 - 8.0 * al) + (1.0 + 1.0 / (1.0 - 8.0 * al)) * lv;
+    }
+    sl_log = block_reduce(sl_log, red, 0);
+    so = block_reduce(so, red, 0);
+    for (int e = tid; e < d * d; e += FIT_THREADS) {
+      int l = e / d, j = e % d;
+      double dg = (l == j) ? 1.0 : 0.0;
+      double b = sqrt(1.0 - 4.0 * aux[l]) * Vs[j * ldv + perm[l]];     // B = (I-4A)^1/2 Q3^T
+      oA[e] = aux[l] * dg; oB1[e] = b; oB2[e] = b; oC1[e] = -0.5 * dg; oC2[e] = -0.5 * dg;
+    }
+    logD = 0.25 * sl_log;
+    obj = so - t1 - t2;
+    phi = lam[0];
+  } else {  // FSHARP_ADERF, Theorem 4.2
+    double* Q1g = gs + (size_t)d * d;
+    double* T1g = gs + (size_t)2 * d * d;
+    double* Ug = gs + (size_t)3 * d * d;
+    for (int e = tid; e < d * d; e += FIT_THREADS) {
+      int i = e / d, j = e % d;
+      As[i * lda + j] = M1[e] + (i == j ? rg1 : 0.0);
+    }
+    __syncthreads();
+    jacobi_eig(As, lda, Vs, ldv, d, cs, pq, red);
+    double lmin = 1e300, lmax = 0.0;
+    for (int i = tid; i < d; i += FIT_THREADS) {
+      double li = As[i * lda + i];
+      lmin = fmin(lmin, li); lmax = fmax(lmax, li);
+    }
+    lmin = block_reduce(lmin, red, 2);
+    lmax = block_reduce(lmax, red, 1);
+    if (!(lmin > 1e-12 * lmax)) violated = true;
+    for (int i = tid; i < d; i += FIT_THREADS) lam[i] = fmax(As[i * lda + i], 1e-300 + 1e-12 * lmax);
+    for (int e = tid; e < d * d; e += FIT_THREADS) Q1g[e] = Vs[(e / d) * ldv + (e % d)];
+    __syncthreads();
+    // T1 = M2 Q1 L1^1/2
+    for (int e = tid; e < d * d; e += FIT_THREADS) {
+      int i = e / d, l = e % d;
+      double s = 0.0;
+      for (int j = 0; j < d; j++) s = fma(M2[i * d + j] + (i == j ? rg2 : 0.0), Q1g[j * d + l], s);
+      T1g[e] = s * sqrt(lam[l]);
+    }
+    __syncthreads();
+    // Z Z^T = L1^1/2 Q1^T M2 Q1 L1^1/2  (symmetric; both triangles written from the same sum)
+    for (int e = tid; e < d * d; e += FIT_THREADS) {
+      int r = e / d, c = e % d;
+      if (r > c) continue;
+      double s = 0.0;
+      for (int i = 0; i < d; i++) s = fma(Q1g[i * d + r] * sqrt(lam[r]), T1g[i * d + c], s);
+      double s2 = 0.0;
+      for (int i = 0; i < d; i++) s2 = fma(Q1g[i * d + c] * sqrt(lam[c]), T1g[i * d + r], s2);
+      double v = 0.5 * (s + s2);
+      As[r * lda + c] = v;
+      As[c * lda + r] = v;
+    }
+    __syncthreads();
+    jacobi_eig(As, lda, Vs, ldv, d, cs, pq, red);     // eigenvalues Sigma^2, eigenvectors U
+    double smin = 1e300, smax = 0.0, ssum = 0.0;
+    for (int l = tid; l < d; l += FIT_THREADS) {
+      double sg = sqrt(fmax(As[l * lda + l], 0.0));
+      aux[l] = sg;
+      smin = fmin(smin, sg); smax = fmax(smax, sg); ssum += sg;
+    }
+    smin = block_reduce(smin, red, 2);
+    smax = block_reduce(smax, red, 1);
+    ssum = block_reduce(ssum, red, 0);
+    if (!(smin > 1e-12 * smax)) violated = true;
+    for (int l = tid; l < d; l += FIT_THREADS) aux[l] = fmax(aux[l], 1e-300 + 1e-12 * smax);
+    for (int e = tid; e < d * d; e += FIT_THREADS) Ug[e] = Vs[(e / d) * ldv + (e % d)];
+    __syncthreads();
+    const double mu3 = mm / d;
+    phi = 2.0 * ssum / d + 2.0 * mu3;
+    const double A = lemma_a1(phi);
+    const double r = sqrt(1.0 - 4.0 * A);
+    // B1 = r Sigma^1/2 U^T L1^-1/2 Q1^T,  B2 = r Sigma^-1/2 U^T L1^1/2 Q1^T
+    for (int e = tid; e < d * d; e += FIT_THREADS) {
+      int l = e / d, j = e % d;
+      double s1 = 0.0, s2 = 0.0;
+      for (int i = 0; i < d; i++) {
+        double u = Ug[i * d + l], q = Q1g[j * d + i], sq = sqrt(lam[i]);
+        s1 = fma(u / sq, q, s1);
+        s2 = fma(u * sq, q, s2);
+      }
+      double sg = sqrt(aux[l]);
+      oB1[e] = r * sg * s1;
+      oB2[e] = r / sg * s2;
+      oA[e] = (l == j) ? A : 0.0;
+    }
+    __syncthreads();
+    for (int e = tid; e < d * d; e += FIT_THREADS) {
+      int i = e / d, j = e % d;
+      double s1 = 0.0, s2 = 0.0;
+      for (int l = 0; l < d; l++) {
+        s1 = fma(oB1[l * d + i], oB1[l * d + j], s1);
+        s2 = fma(oB2[l * d + i], oB2[l * d + j], s2);
+      }
+      oC1[e] = -s1 / (2.0 * (1.0 - 4.0 * A));
+      oC2[e] = -s2 / (2.0 * (1.0 - 4.0 * A));
+    }
+    logD = 0.25 * d * log(1.0 - 4.0 * A);
+    obj = d * (log(1.0 - 4.0 * A) - 0.5 * log(1.0 - 8.0 * A) + 2.0 / (1.0 - 8.0 * A) * (ssum / d + mu3) + 2.0 * mu3);
+    // -C1 = F/2 and -C2 = F^-1/2 with F = Q1 L1^-1/2 U Sigma U^T L1^-1/2 Q1^T:
+    // lambda_min(F) >= sigma_min / lambda1_max, lambda_min(F^-1) >= lambda1_min / sigma_max.
+    kap1 = 0.5 * smin / lmax;
+    kap2 = 0.5 * lmin / smax;
+  }
+  if (tid == 0) {
+    tail[PT_LOGD] = logD;
+    tail[PT_OBJ] = obj;
+    tail[PT_PHI] = phi;
+    tail[PT_KAPPA1] = kap1;
+    tail[PT_KAPPA2] = kap2;
+    tail[PT_RHO2X] = st[sl.rho2(1)];
+    tail[PT_RHO2Y] = st[sl.rho2(2)];
+    tail[PT_RES] = 0.0;
+  }
+  if (violated) atomicExch(a.status, FSHARP_E_CONSTRAINT);
+}
+
+size_t fit_smem_bytes(int d, int v_in_smem) {
+  size_t dbl = (size_t)d * (d + 1) * (v_in_smem ? 2 : 1) + 4 * (size_t)d + FIT_THREADS;
+  return dbl * sizeof(double) + 3 * (size_t)d * sizeof(int);
+}
+
+}  // namespace
+
+size_t fs_fit_scratch_doubles(int G, int d) { return (size_t)G * 4 * d * d; }
+
+int fs_run_fit(fsharp_ctx* ctx, const double* stats, int G, int d, int variant, double ridge,
+               double* params, double* scratch) {
+  if (G == 0) return FSHARP_OK;
+  FitArgs a;
+  a.stats = stats; a.params = params; a.scratch = scratch; a.d = d; a.variant = variant; a.ridge = ridge;
+  a.v_in_smem = d <= 64 ? 1 : 0;
+  a.status = ctx->d_status;
+  size_t smem = fit_smem_bytes(d, a.v_in_smem);
+  FS_CUDA_OK(cudaFuncSetAttribute(fit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  fit_kernel<<<G, FIT_THREADS, smem, ctx->stream>>>(a);
+  FS_LAUNCH_CHECK(ctx);
+  return FSHARP_OK;
+}
