@@ -1,0 +1,270 @@
+"""Thin ctypes binding of libfsharp.so: the same names as include/fsharp.h, argument
+marshalling only.  torch is used for device memory and streams; every step of the path
+runs in the library's CUDA kernels.  There is no CPU fallback: if the library is missing
+or a call fails, an exception is raised."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "lib", "libfsharp.so")
+
+FSHARP_F32, FSHARP_BF16 = 0, 1
+VARIANTS = {"posrf": 0, "gerf": 1, "saderf": 2, "aderf": 3, "sderf": 4}
+POOL_PER_BH, POOL_PER_HEAD = 0, 1
+STAB_NONE, STAB_ROW, STAB_GROUP = 0, 1, 2
+IMPL_AUTO, IMPL_SIMT, IMPL_TENSOR = 0, 1, 2
+
+EXPORTS = [
+    "fsharp_create", "fsharp_destroy", "fsharp_set_stream", "fsharp_set_impl", "fsharp_status",
+    "fsharp_launch_count", "fsharp_workspace_bytes", "fsharp_strerror", "fsharp_stats_doubles",
+    "fsharp_params_doubles", "fsharp_stats", "fsharp_fit_params", "fsharp_featurize", "fsharp_attend",
+    "fsharp_forward_host", "fsharp_pair_estimate",
+]
+
+
+class FsharpError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+class fsharp_dims(C.Structure):
+    _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("Lq", C.c_int32), ("Lk", C.c_int32),
+                ("d", C.c_int32), ("dv", C.c_int32), ("M", C.c_int32), ("pool", C.c_int32),
+                ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 3),
+                ("v_stride", C.c_int64 * 3), ("y_stride", C.c_int64 * 3),
+                ("omega_head_stride", C.c_int64)]
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Loads lib/libfsharp.so (built by build.py); raises if it is not there."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2302_00787_b200.build` "
+            "(there is no fallback implementation)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, f32, f64 = C.c_void_p, C.c_int, C.c_int64, C.c_float, C.c_double
+    dims_p = C.POINTER(fsharp_dims)
+    sig = {
+        "fsharp_create": (i32, [C.POINTER(vp), i32, vp]),
+        "fsharp_destroy": (i32, [vp]),
+        "fsharp_set_stream": (i32, [vp, vp]),
+        "fsharp_set_impl": (i32, [vp, i32]),
+        "fsharp_status": (i32, [vp, C.POINTER(i32)]),
+        "fsharp_launch_count": (i64, [vp]),
+        "fsharp_workspace_bytes": (C.c_size_t, [vp]),
+        "fsharp_strerror": (C.c_char_p, [i32]),
+        "fsharp_stats_doubles": (C.c_size_t, [i32]),
+        "fsharp_params_doubles": (C.c_size_t, [i32]),
+        "fsharp_stats": (i32, [vp, vp, vp, dims_p, i32, f32, vp]),
+        "fsharp_fit_params": (i32, [vp, vp, i32, i32, i32, f64, vp]),
+        "fsharp_featurize": (i32, [vp, vp, vp, vp, i32, dims_p, i32, f32, i32, vp, vp]),
+        "fsharp_attend": (i32, [vp, vp, vp, vp, vp, vp, dims_p, i32, i32, i32, f32, vp]),
+        "fsharp_forward_host": (i32, [vp, vp, vp, vp, vp, dims_p, i32, i32, i32, i32, f32, vp]),
+        "fsharp_pair_estimate": (i32, [vp, vp, vp, vp, vp, i64, i32, i32, i32, vp, vp]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load_library().fsharp_strerror(code).decode()
+
+
+def stats_doubles(d: int) -> int:
+    return load_library().fsharp_stats_doubles(d)
+
+
+def params_doubles(d: int) -> int:
+    return load_library().fsharp_params_doubles(d)
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != 0:
+        raise FsharpError(rc, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return FSHARP_F32
+    if t.dtype == torch.bfloat16:
+        return FSHARP_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _strides(t: torch.Tensor):
+    """Element strides (batch, head, token) of a [B,H,L,inner] tensor, innermost contiguous."""
+    if t.dim() != 4 or (t.shape[3] > 1 and t.stride(3) != 1):
+        raise ValueError("expected a [B, H, L, inner] tensor whose last dimension is contiguous")
+    return (C.c_int64 * 3)(t.stride(0), t.stride(1), t.stride(2))
+
+
+def make_dims(B, H, Lq, Lk, d, dv, M, pool=POOL_PER_BH, q=None, k=None, v=None, y=None,
+              omega_head_stride=0) -> fsharp_dims:
+    dm = fsharp_dims()
+    dm.B, dm.H, dm.Lq, dm.Lk, dm.d, dm.dv, dm.M, dm.pool = B, H, Lq, Lk, d, dv, M, pool
+    for name, t in (("q_stride", q), ("k_stride", k), ("v_stride", v), ("y_stride", y)):
+        if t is not None:
+            setattr(dm, name, _strides(t))
+    dm.omega_head_stride = omega_head_stride
+    return dm
+
+
+class Context:
+    """Owns one fsharp_ctx bound to a CUDA device and stream."""
+
+    def __init__(self, device: int = 0, stream: torch.cuda.Stream | None = None):
+        self.lib = load_library()
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required (no CPU implementation exists)")
+        self.device = device
+        self._h = C.c_void_p()
+        sp = stream.cuda_stream if stream is not None else torch.cuda.current_stream(device).cuda_stream
+        _check(self.lib.fsharp_create(C.byref(self._h), device, C.c_void_p(sp)), "fsharp_create")
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self.lib.fsharp_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- plumbing
+    def set_stream(self, stream: torch.cuda.Stream):
+        _check(self.lib.fsharp_set_stream(self._h, C.c_void_p(stream.cuda_stream)), "fsharp_set_stream")
+
+    def set_impl(self, impl: int):
+        _check(self.lib.fsharp_set_impl(self._h, impl), "fsharp_set_impl")
+
+    def status(self) -> int:
+        code = C.c_int(0)
+        _check(self.lib.fsharp_status(self._h, C.byref(code)), "fsharp_status")
+        return code.value
+
+    def launch_count(self) -> int:
+        return self.lib.fsharp_launch_count(self._h)
+
+    def workspace_bytes(self) -> int:
+        return self.lib.fsharp_workspace_bytes(self._h)
+
+    # -- the path
+    def fsharp_stats(self, Q, K, pool=POOL_PER_BH, qk_scale=1.0, out=None):
+        B, H, Lq, d = Q.shape
+        Lk = K.shape[2]
+        dm = make_dims(B, H, Lq, Lk, d, d, 16, pool, q=Q, k=K)
+        G = B * H if pool == POOL_PER_BH else H
+        if out is None:
+            out = torch.empty(G, stats_doubles(d), dtype=torch.float64, device=Q.device)
+        _check(self.lib.fsharp_stats(self._h, Q.data_ptr(), K.data_ptr(), C.byref(dm), _dtype_code(Q),
+                                     qk_scale, out.data_ptr()), "fsharp_stats")
+        return out
+
+    def fsharp_fit_params(self, stats, d, variant, ridge=0.0, out=None):
+        G = stats.shape[0]
+        v = VARIANTS[variant] if isinstance(variant, str) else variant
+        if out is None:
+            out = torch.empty(G, params_doubles(d), dtype=torch.float64, device=stats.device)
+        _check(self.lib.fsharp_fit_params(self._h, stats.data_ptr(), G, d, v, ridge, out.data_ptr()),
+               "fsharp_fit_params")
+        return out
+
+    def fsharp_featurize(self, X, Omega, params, side, pool=POOL_PER_BH, qk_scale=1.0, stab=STAB_ROW):
+        B, H, L, d = X.shape
+        M = Omega.shape[-2]
+        ohs = Omega.stride(0) if Omega.dim() == 3 else 0
+        dm = make_dims(B, H, L, L, d, d, M, pool, q=X, k=X, omega_head_stride=ohs)
+        phi = torch.empty(B, H, L, M, dtype=torch.float32, device=X.device)
+        ls = None
+        if stab == STAB_ROW:
+            ls = torch.empty(B, H, L, dtype=torch.float32, device=X.device)
+        elif stab == STAB_GROUP:
+            ls = torch.empty(B, H, dtype=torch.float32, device=X.device)
+        _check(self.lib.fsharp_featurize(self._h, X.data_ptr(), Omega.data_ptr(), params.data_ptr(), side,
+                                         C.byref(dm), _dtype_code(X), qk_scale, stab, phi.data_ptr(),
+                                         ls.data_ptr() if ls is not None else None), "fsharp_featurize")
+        return phi, ls
+
+    def fsharp_attend(self, Q, K, V, Omega, params, causal=False, chunk=0, pool=POOL_PER_BH, qk_scale=1.0,
+                      out=None):
+        B, H, Lq, d = Q.shape
+        Lk, dv = K.shape[2], V.shape[3]
+        M = Omega.shape[-2]
+        ohs = Omega.stride(0) if Omega.dim() == 3 else 0
+        if out is None:
+            out = torch.empty(B, H, Lq, dv, dtype=Q.dtype, device=Q.device)
+        dm = make_dims(B, H, Lq, Lk, d, dv, M, pool, q=Q, k=K, v=V, y=out, omega_head_stride=ohs)
+        _check(self.lib.fsharp_attend(self._h, Q.data_ptr(), K.data_ptr(), V.data_ptr(), Omega.data_ptr(),
+                                      params.data_ptr(), C.byref(dm), _dtype_code(Q), int(bool(causal)), chunk,
+                                      qk_scale, out.data_ptr()), "fsharp_attend")
+        return out
+
+    def fsharp_forward_host(self, Q, K, V, Omega, variant, causal=False, chunk=0, pool=POOL_PER_BH,
+                            qk_scale=1.0, out=None):
+        """Q, K, V, Omega, out: HOST tensors (dense; pinned memory recommended)."""
+        for t in (Q, K, V, Omega):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError("fsharp_forward_host takes dense host tensors")
+        B, H, Lq, d = Q.shape
+        Lk, dv = K.shape[2], V.shape[3]
+        M = Omega.shape[0]
+        if out is None:
+            out = torch.empty(B, H, Lq, dv, dtype=Q.dtype).pin_memory()
+        dm = make_dims(B, H, Lq, Lk, d, dv, M, pool)
+        v = VARIANTS[variant] if isinstance(variant, str) else variant
+        _check(self.lib.fsharp_forward_host(self._h, Q.data_ptr(), K.data_ptr(), V.data_ptr(), Omega.data_ptr(),
+                                            C.byref(dm), _dtype_code(Q), v, int(bool(causal)), chunk, qk_scale,
+                                            out.data_ptr()), "fsharp_forward_host")
+        return out
+
+    def fsharp_pair_estimate(self, X, Y, Omega, params, want_variance=True):
+        npairs, d = X.shape
+        R, M = Omega.shape[0], Omega.shape[1]
+        est = torch.empty(R, npairs, dtype=torch.float32, device=X.device)
+        var = torch.empty(npairs, dtype=torch.float64, device=X.device) if want_variance else None
+        _check(self.lib.fsharp_pair_estimate(self._h, X.data_ptr(), Y.data_ptr(), Omega.data_ptr(),
+                                             params.data_ptr(), npairs, d, M, R, est.data_ptr(),
+                                             var.data_ptr() if var is not None else None), "fsharp_pair_estimate")
+        return est, var
+
+
+def unpack_params(blob: torch.Tensor, d: int):
+    """Splits one group's parameter blob (a 1-D float64 tensor or array) into named pieces."""
+    b = blob.detach().cpu().numpy() if isinstance(blob, torch.Tensor) else blob
+    dd = d * d
+    t = b[5 * dd:]
+    return {"A": b[0:dd].reshape(d, d), "B1": b[dd:2 * dd].reshape(d, d), "B2": b[2 * dd:3 * dd].reshape(d, d),
+            "C1": b[3 * dd:4 * dd].reshape(d, d), "C2": b[4 * dd:5 * dd].reshape(d, d),
+            "logD": float(t[0]), "objective": float(t[1]), "phi": float(t[2]),
+            "kappa1": float(t[3]), "kappa2": float(t[4]), "rho2max_x": float(t[5]), "rho2max_y": float(t[6])}
+
+
+def pack_params(p: dict, d: int, kappa=(0.0, 0.0), rho2max=(0.0, 0.0)):
+    """Builds a parameter blob (numpy float64) from matrices A, B1, B2, C1, C2 and logD."""
+    import numpy as np
+    out = np.zeros(5 * d * d + 8, dtype=np.float64)
+    for i, k in enumerate(("A", "B1", "B2", "C1", "C2")):
+        out[i * d * d:(i + 1) * d * d] = np.asarray(p[k], dtype=np.float64).reshape(-1)
+    t = out[5 * d * d:]
+    t[0] = p["logD"]
+    t[1] = p.get("objective", 0.0)
+    t[3], t[4] = kappa
+    t[5], t[6] = rho2max
+    return out

@@ -1,0 +1,192 @@
+// C-ABI entry points: argument checks, workspace sizing and dispatch to the kernel families.
+#include <math.h>
+
+#include "common.cuh"
+
+// tensor-core path (tc_*.cu)
+int fs_tc_supported(const fsharp_dims* dm, int dtype, int causal, int chunk, float qk_scale);
+size_t fs_tc_attend_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm, int causal, int chunk);
+int fs_tc_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, int causal,
+                 int chunk, const float* prep, void* Y, WsAlloc* ws);
+
+namespace {
+
+bool dim_ok(int d) { return d == 16 || d == 32 || d == 64 || d == 128; }
+
+int check_dims(const fsharp_dims* dm, bool need_v) {
+  if (!dm) return FSHARP_E_BADARG;
+  if (dm->B < 0 || dm->H < 0 || dm->Lq < 0 || dm->Lk < 0) return FSHARP_E_SHAPE;
+  if (!dim_ok(dm->d)) return FSHARP_E_SHAPE;
+  if (need_v && !dim_ok(dm->dv)) return FSHARP_E_SHAPE;
+  if (dm->M <= 0 || dm->M % 16 != 0 || dm->M > 1024) return FSHARP_E_SHAPE;
+  if (dm->pool != FSHARP_POOL_PER_BH && dm->pool != FSHARP_POOL_PER_HEAD) return FSHARP_E_BADARG;
+  if ((int64_t)dm->B * dm->H > 65535) return FSHARP_E_SHAPE;
+  return FSHARP_OK;
+}
+
+int check_ptr(const void* p, int dtype, const int64_t s[3]) {
+  if (!p) return FSHARP_E_BADARG;
+  const size_t es = dtype == FSHARP_F32 ? 4 : 2;
+  if (reinterpret_cast<uintptr_t>(p) % 16 != 0) return FSHARP_E_ALIGN;
+  for (int i = 0; i < 3; i++)
+    if (s[i] < 0 || (s[i] * es) % 16 != 0) return FSHARP_E_ALIGN;
+  return FSHARP_OK;
+}
+
+bool dtype_ok(int dtype) { return dtype == FSHARP_F32 || dtype == FSHARP_BF16; }
+
+}  // namespace
+
+extern "C" {
+
+int fsharp_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dims* dims, int dtype,
+                 float qk_scale, double* stats) {
+  if (!ctx || !stats) return FSHARP_E_BADARG;
+  FS_TRY(check_dims(dims, false));
+  if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
+  if (dims->B * dims->H == 0) return FSHARP_OK;
+  FS_TRY(check_ptr(Q, dtype, dims->q_stride));
+  FS_TRY(check_ptr(K, dtype, dims->k_stride));
+  FS_CUDA_OK(cudaSetDevice(ctx->device));
+  return fs_run_stats(ctx, Q, K, dims, dtype, qk_scale, stats);
+}
+
+int fsharp_fit_params(fsharp_ctx* ctx, const double* stats, int G, int d, int variant, double ridge,
+                      double* params) {
+  if (!ctx || !stats || !params) return FSHARP_E_BADARG;
+  if (G < 0 || !dim_ok(d)) return FSHARP_E_SHAPE;
+  if (variant < FSHARP_POSRF || variant > FSHARP_SDERF) return FSHARP_E_BADARG;
+  if (!(ridge >= 0.0)) return FSHARP_E_BADARG;
+  if (G == 0) return FSHARP_OK;
+  FS_CUDA_OK(cudaSetDevice(ctx->device));
+  size_t need = ws_round(fs_fit_scratch_doubles(G, d) * sizeof(double));
+  FS_TRY(fs_ws_reserve(ctx, need));
+  return fs_run_fit(ctx, stats, G, d, variant, ridge, params, reinterpret_cast<double*>(ctx->ws));
+}
+
+int fsharp_featurize(fsharp_ctx* ctx, const void* X, const float* Omega, const double* params, int side,
+                     const fsharp_dims* dims, int dtype, float qk_scale, int stab, float* phi, float* logscale) {
+  if (!ctx || !Omega || !params || !phi) return FSHARP_E_BADARG;
+  FS_TRY(check_dims(dims, false));
+  if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
+  if (side != 1 && side != 2) return FSHARP_E_BADARG;
+  if (stab < FSHARP_STAB_NONE || stab > FSHARP_STAB_GROUP) return FSHARP_E_BADARG;
+  if (stab != FSHARP_STAB_NONE && !logscale) return FSHARP_E_BADARG;
+  const int L = side == 1 ? dims->Lq : dims->Lk;
+  const int64_t* st = side == 1 ? dims->q_stride : dims->k_stride;
+  if (dims->B * dims->H == 0 || L == 0) return FSHARP_OK;
+  FS_TRY(check_ptr(X, dtype, st));
+  FS_CUDA_OK(cudaSetDevice(ctx->device));
+  const int G = fs_groups(dims);
+  const size_t prep_f = (size_t)G * 2 * PrepLayout{dims->d, dims->M}.total();
+  const size_t need = ws_round(prep_f * 4) + ws_round((size_t)dims->B * dims->H * L * 4);
+  FS_TRY(fs_ws_reserve(ctx, need));
+  WsAlloc ws{ctx->ws, 0};
+  float* prep = ws.take<float>(prep_f);
+  float* rowc = ws.take<float>((size_t)dims->B * dims->H * L);
+  FS_TRY(fs_run_prep(ctx, Omega, dims->omega_head_stride, params, (int64_t)ParamsLayout{dims->d}.total(), G,
+                     dims->H, dims->pool, dims->d, dims->M, prep));
+  return fs_simt_featurize(ctx, X, dtype, fs_addr(st, dims->H, L, dims->d), dims->B, dims->H, L, dims->d, dims->M,
+                           dims->pool, prep, side, qk_scale, stab, rowc, phi, logscale);
+}
+
+int fsharp_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const float* Omega,
+                  const double* params, const fsharp_dims* dims, int dtype, int causal, int chunk, float qk_scale,
+                  void* Y) {
+  if (!ctx || !Omega || !params) return FSHARP_E_BADARG;
+  FS_TRY(check_dims(dims, true));
+  if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
+  if (causal) {
+    if (dims->Lq != dims->Lk) return FSHARP_E_SHAPE;
+    if (chunk != 64 && chunk != 128 && chunk != 256) return FSHARP_E_SHAPE;
+    if (dims->Lq % chunk != 0) return FSHARP_E_SHAPE;
+  }
+  if (dims->B * dims->H == 0 || dims->Lq == 0) return FSHARP_OK;
+  if (dims->Lk == 0) return FSHARP_E_SHAPE;   // no key: the normaliser of Section 2.2 is zero
+  FS_TRY(check_ptr(Q, dtype, dims->q_stride));
+  FS_TRY(check_ptr(K, dtype, dims->k_stride));
+  FS_TRY(check_ptr(V, dtype, dims->v_stride));
+  FS_TRY(check_ptr(Y, dtype, dims->y_stride));
+  FS_CUDA_OK(cudaSetDevice(ctx->device));
+  const int G = fs_groups(dims);
+  const size_t prep_f = (size_t)G * 2 * PrepLayout{dims->d, dims->M}.total();
+  bool use_tc = false;
+  if (ctx->impl != FSHARP_IMPL_SIMT) {
+    use_tc = fs_tc_supported(dims, dtype, causal, chunk, qk_scale) != 0;
+    if (!use_tc && ctx->impl == FSHARP_IMPL_TENSOR) return FSHARP_E_SHAPE;
+  }
+  const size_t need = ws_round(prep_f * 4) + (use_tc ? fs_tc_attend_scratch_bytes(ctx, dims, causal, chunk)
+                                                     : fs_simt_attend_scratch_bytes(dims, causal, chunk));
+  FS_TRY(fs_ws_reserve(ctx, need));
+  WsAlloc ws{ctx->ws, 0};
+  float* prep = ws.take<float>(prep_f);
+  FS_TRY(fs_run_prep(ctx, Omega, dims->omega_head_stride, params, (int64_t)ParamsLayout{dims->d}.total(), G,
+                     dims->H, dims->pool, dims->d, dims->M, prep));
+  if (use_tc) return fs_tc_attend(ctx, Q, K, V, dims, causal, chunk, prep, Y, &ws);
+  return fs_simt_attend(ctx, Q, K, V, dims, dtype, causal, chunk, qk_scale, prep, Y, &ws);
+}
+
+int fsharp_forward_host(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const float* Omega,
+                        const fsharp_dims* dims, int dtype, int variant, int causal, int chunk, float qk_scale,
+                        void* Y) {
+  if (!ctx || !Q || !K || !V || !Omega || !Y) return FSHARP_E_BADARG;
+  FS_TRY(check_dims(dims, true));
+  if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
+  if (variant < FSHARP_POSRF || variant > FSHARP_SDERF) return FSHARP_E_BADARG;
+  if (dims->omega_head_stride != 0) return FSHARP_E_BADARG;
+  FS_CUDA_OK(cudaSetDevice(ctx->device));
+  fsharp_dims dd = *dims;
+  for (int i = 0; i < 3; i++) dd.q_stride[i] = dd.k_stride[i] = dd.v_stride[i] = dd.y_stride[i] = 0;
+  const size_t es = dtype == FSHARP_F32 ? 4 : 2;
+  const size_t BH = (size_t)dd.B * dd.H;
+  const size_t nq = BH * dd.Lq * dd.d * es, nk = BH * dd.Lk * dd.d * es, nv = BH * dd.Lk * dd.dv * es;
+  const size_t ny = BH * dd.Lq * dd.dv * es, no = (size_t)dd.M * dd.d * 4;
+  if (ny == 0) return FSHARP_OK;
+  const int G = fs_groups(&dd);
+  const size_t nstats = (size_t)G * StatsLayout{dd.d}.total() * 8, nparams = (size_t)G * ParamsLayout{dd.d}.total() * 8;
+  // The staging buffers live at the END of the workspace so that the nested calls, which
+  // carve their scratch from the start, do not overlap them.
+  const size_t stage = ws_round(nq) + ws_round(nk) + ws_round(nv) + ws_round(ny) + ws_round(no) + ws_round(nstats) +
+                       ws_round(nparams);
+  const int G2 = G;
+  size_t inner = ws_round((size_t)G2 * 2 * PrepLayout{dd.d, dd.M}.total() * 4);
+  {
+    size_t a = fs_simt_attend_scratch_bytes(&dd, causal, chunk);
+    size_t b = fs_tc_supported(&dd, dtype, causal, chunk, qk_scale) ? fs_tc_attend_scratch_bytes(ctx, &dd, causal, chunk) : 0;
+    size_t c = ws_round(fs_fit_scratch_doubles(G, dd.d) * 8);
+    size_t use = ctx->impl == FSHARP_IMPL_SIMT ? a : (b ? b : a);
+    inner += use > c ? use : c;
+  }
+  FS_TRY(fs_ws_reserve(ctx, inner + stage + 256));
+  WsAlloc ws{ctx->ws, (ctx->ws_bytes - stage) & ~(size_t)255};
+  char* dQ = ws.take<char>(nq);
+  char* dK = ws.take<char>(nk);
+  char* dV = ws.take<char>(nv);
+  char* dY = ws.take<char>(ny);
+  float* dO = ws.take<float>((size_t)dd.M * dd.d);
+  double* dS = ws.take<double>(nstats / 8);
+  double* dP = ws.take<double>(nparams / 8);
+  FS_CUDA_OK(cudaMemcpyAsync(dQ, Q, nq, cudaMemcpyHostToDevice, ctx->stream));
+  FS_CUDA_OK(cudaMemcpyAsync(dK, K, nk, cudaMemcpyHostToDevice, ctx->stream));
+  FS_CUDA_OK(cudaMemcpyAsync(dV, V, nv, cudaMemcpyHostToDevice, ctx->stream));
+  FS_CUDA_OK(cudaMemcpyAsync(dO, Omega, no, cudaMemcpyHostToDevice, ctx->stream));
+  FS_TRY(fsharp_stats(ctx, dQ, dK, &dd, dtype, qk_scale, dS));
+  FS_TRY(fsharp_fit_params(ctx, dS, G, dd.d, variant, 0.0, dP));
+  FS_TRY(fsharp_attend(ctx, dQ, dK, dV, dO, dP, &dd, dtype, causal, chunk, qk_scale, dY));
+  FS_CUDA_OK(cudaMemcpyAsync(Y, dY, ny, cudaMemcpyDeviceToHost, ctx->stream));
+  FS_CUDA_OK(cudaStreamSynchronize(ctx->stream));
+  return FSHARP_OK;
+}
+
+int fsharp_pair_estimate(fsharp_ctx* ctx, const float* X, const float* Y, const float* Omega, const double* params,
+                         int64_t npairs, int d, int M, int R, float* est, double* var_cf) {
+  if (!ctx || !Omega || !params) return FSHARP_E_BADARG;
+  if (npairs < 0 || !dim_ok(d) || M <= 0 || M % 16 != 0 || M > 1024 || R <= 0 || R > 65535) return FSHARP_E_SHAPE;
+  if (npairs > 0 && (!X || !Y || !est)) return FSHARP_E_BADARG;
+  FS_CUDA_OK(cudaSetDevice(ctx->device));
+  FS_TRY(fs_ws_reserve(ctx, fs_pairs_scratch_bytes(d, M, R)));
+  WsAlloc ws{ctx->ws, 0};
+  return fs_run_pairs(ctx, X, Y, Omega, params, npairs, d, M, R, est, var_cf, &ws);
+}
+
+}  // extern "C"

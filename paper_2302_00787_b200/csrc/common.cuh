@@ -136,8 +136,9 @@ int fs_run_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dim
 int fs_run_fit(fsharp_ctx* ctx, const double* stats, int G, int d, int variant, double ridge,
                double* params, double* scratch);
 size_t fs_fit_scratch_doubles(int G, int d);
+// params_stride: doubles between the blobs of two groups (0 = every group reads the same blob)
 int fs_run_prep(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_stride, const double* params,
-                int G, int H, int pool, int d, int M, float* prep /* [G][2][PrepLayout] */);
+                int64_t params_stride, int G, int H, int pool, int d, int M, float* prep /* [G][2][PrepLayout] */);
 // rowc: scratch [B*H*L] floats.  phi: [B,H,L,M] floats.
 int fs_simt_featurize(fsharp_ctx* ctx, const void* X, int dtype, TensorAddr ax, int B, int H, int L, int d,
                       int M, int pool, const float* prep, int side, float qk_scale, int stab,

@@ -9,7 +9,7 @@ constexpr int PREP_THREADS = 256;
 
 __global__ void __launch_bounds__(PREP_THREADS)
 prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const double* __restrict__ params,
-            int H, int pool, int d, int M, float* __restrict__ prep) {
+            int64_t params_stride, int H, int pool, int d, int M, float* __restrict__ prep) {
   __shared__ float red[PREP_THREADS];
   __shared__ float red2[PREP_THREADS];
   __shared__ int redi[PREP_THREADS];
@@ -18,7 +18,7 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
   const float* Om = Omega + (int64_t)h * omega_head_stride;
   ParamsLayout pl{d};
   PrepLayout pr{d, M};
-  const double* P = params + (size_t)g * pl.total();
+  const double* P = params + (size_t)g * params_stride;
   const double* A = P + pl.A();
   const double* Bm = P + pl.B(side);
   const double* Cm = P + pl.C(side);
@@ -101,9 +101,10 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
 }  // namespace
 
 int fs_run_prep(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_stride, const double* params,
-                int G, int H, int pool, int d, int M, float* prep) {
+                int64_t params_stride, int G, int H, int pool, int d, int M, float* prep) {
   if (G == 0) return FSHARP_OK;
-  prep_kernel<<<dim3(G, 2), PREP_THREADS, 0, ctx->stream>>>(Omega, omega_head_stride, params, H, pool, d, M, prep);
+  prep_kernel<<<dim3(G, 2), PREP_THREADS, 0, ctx->stream>>>(Omega, omega_head_stride, params, params_stride, H, pool, d, M,
+                                                                 prep);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;
 }

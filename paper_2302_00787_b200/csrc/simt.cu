@@ -1,0 +1,378 @@
+// fp32 CUDA-core path: features (Section 4 definition with Section 2.1's M^-1/2) and the
+// linear-attention contraction (Sections 2.1 / 2.2), bidirectional and causal-chunked.
+// Used for fp32 inputs, for shapes the tensor-core path does not take, and on request.
+//
+// Scratch (from the context workspace): the two feature matrices, the per-token
+// quadratic term, S^T [V | 1] (per (batch, head); per chunk when causal) and, when
+// causal, the masked in-chunk score blocks.
+#include "common.cuh"
+#include "simt_tile.cuh"
+
+namespace {
+
+__device__ __forceinline__ int group_of(int bh, int H, int pool) { return pool == FSHARP_POOL_PER_BH ? bh : bh % H; }
+
+// ---- per-token quadratic term c_i = x_i^T C x_i --------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(NTH)
+rowterm_kernel(const T* __restrict__ X, TensorAddr ax, int H, int L, int d, int M, int pool, int side,
+               const float* __restrict__ prep, float qk_scale, float* __restrict__ rowc) {
+  extern __shared__ float smf[];
+  const int bh = blockIdx.y, b = bh / H, h = bh % H;
+  PrepLayout pr{d, M};
+  const float* pp = prep + ((size_t)group_of(bh, H, pool) * 2 + (side - 1)) * pr.total();
+  const float* scal = pp + pr.scal();
+  const bool cscalar = scal[PS_CSCALAR] != 0.f;
+  const float gamma = scal[PS_CGAMMA];
+  float* Cs = smf;                   // d*d (only when C is dense)
+  float* xs = smf + (cscalar ? 0 : d * d);   // 8 warps * d
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (!cscalar) {
+    const float* Cm = pp + pr.Cmat();
+    for (int e = tid; e < d * d; e += NTH) Cs[e] = Cm[e];
+  }
+  __syncthreads();
+  const T* Xb = X + b * ax.sb + h * ax.sh;
+  float* xw = xs + warp * d;
+  for (int i = blockIdx.x * 8 + warp; i < L; i += gridDim.x * 8) {
+    for (int j = lane; j < d; j += 32) xw[j] = qk_scale * fs_load(Xb + (int64_t)i * ax.sl + j);
+    __syncwarp();
+    float s = 0.f;
+    if (cscalar) {
+      for (int j = lane; j < d; j += 32) s = fmaf(xw[j], xw[j], s);
+      s *= gamma;
+    } else {
+      for (int j = lane; j < d; j += 32) {
+        float t = 0.f;
+        for (int k = 0; k < d; k++) t = fmaf(xw[k], Cs[k * d + j], t);
+        s = fmaf(t, xw[j], s);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) rowc[(int64_t)bh * L + i] = s;
+    __syncwarp();
+  }
+}
+
+// ---- exponents e_im = bias + a_m + w_m . x_i + c_i -----------------------------------
+template <typename T>
+__global__ void __launch_bounds__(NTH)
+logits_kernel(const T* __restrict__ X, TensorAddr ax, int H, int L, int d, int M, int pool, int side,
+              const float* __restrict__ prep, float qk_scale, const float* __restrict__ rowc,
+              float* __restrict__ phi) {
+  __shared__ Tiles sm;
+  const int bh = blockIdx.z, b = bh / H, h = bh % H;
+  const int i0 = blockIdx.x * TM, m0 = blockIdx.y * TN;
+  PrepLayout pr{d, M};
+  const float* pp = prep + ((size_t)group_of(bh, H, pool) * 2 + (side - 1)) * pr.total();
+  const float* W = pp + pr.W();
+  const float* av = pp + pr.a();
+  const float bias = pp[pr.scal() + PS_BIAS];
+  const T* Xb = X + b * ax.sb + h * ax.sh;
+  float acc[4][4] = {};
+  tile_gemm<true, true>(
+      acc, d,
+      [&](int r, int k) { return (i0 + r < L) ? qk_scale * fs_load(Xb + (int64_t)(i0 + r) * ax.sl + k) : 0.f; },
+      [&](int k, int c) { return (m0 + c < M) ? W[(size_t)(m0 + c) * d + k] : 0.f; }, sm);
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+#pragma unroll
+  for (int i = 0; i < 4; i++) {
+    int row = i0 + ty + 16 * i;
+    if (row >= L) continue;
+    float ci = rowc[(int64_t)bh * L + row] + bias;
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+      int m = m0 + tx + 16 * j;
+      if (m < M) phi[((int64_t)bh * L + row) * M + m] = acc[i][j] + av[m] + ci;
+    }
+  }
+}
+
+// ---- phi = exp(e - shift), one warp per row ------------------------------------------
+__global__ void __launch_bounds__(NTH)
+expshift_kernel(float* __restrict__ phi, int H, int L, int d, int M, int pool, int side, int stab,
+                const float* __restrict__ prep, float* __restrict__ logscale, int* __restrict__ status) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int bh = blockIdx.y;
+  PrepLayout pr{d, M};
+  const float gshift = prep[((size_t)group_of(bh, H, pool) * 2 + (side - 1)) * pr.total() + pr.scal() + PS_GSHIFT];
+  for (int i = blockIdx.x * 8 + warp; i < L; i += gridDim.x * 8) {
+    float* row = phi + ((int64_t)bh * L + i) * M;
+    float s = 0.f;
+    if (stab == FSHARP_STAB_ROW) {
+      float mx = -3.0e38f;
+      for (int m = lane; m < M; m += 32) mx = fmaxf(mx, row[m]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      s = mx;
+    } else if (stab == FSHARP_STAB_GROUP) {
+      s = gshift;
+    }
+    bool bad = false;
+    for (int m = lane; m < M; m += 32) {
+      float e = row[m];
+      if (!isfinite(e)) bad = true;
+      row[m] = expf(e - s);
+    }
+    if (bad) atomicExch(status, FSHARP_E_NONFINITE);
+    if (logscale && lane == 0) {
+      if (stab == FSHARP_STAB_ROW) logscale[(int64_t)bh * L + i] = s;
+      else if (stab == FSHARP_STAB_GROUP && i == 0) logscale[bh] = s;
+    }
+  }
+}
+
+// ---- S^T [V | 1]: out[slot][m][n] += sum_{j in slice} phiK[j][m] * V1[j][n] -------------
+template <typename T>
+__global__ void __launch_bounds__(NTH)
+kv_kernel(const float* __restrict__ phiK, const T* __restrict__ V, TensorAddr av, int H, int L, int M, int dv,
+          int slice_len, int nslices, int per_slice_out, float* __restrict__ out) {
+  __shared__ Tiles sm;
+  const int bh = blockIdx.z / nslices, sl = blockIdx.z % nslices;
+  const int b = bh / H, h = bh % H;
+  const int m0 = blockIdx.x * TM, n0 = blockIdx.y * TN;
+  const int j0 = sl * slice_len, j1 = min(L, j0 + slice_len);
+  if (j0 >= j1) return;
+  const int N = dv + 1;
+  const float* P = phiK + (int64_t)bh * L * M;
+  const T* Vb = V + b * av.sb + h * av.sh;
+  float acc[4][4] = {};
+  tile_gemm<false, false>(
+      acc, j1 - j0,
+      [&](int r, int k) { return (m0 + r < M) ? P[(int64_t)(j0 + k) * M + m0 + r] : 0.f; },
+      [&](int k, int c) {
+        int n = n0 + c;
+        return n < dv ? fs_load(Vb + (int64_t)(j0 + k) * av.sl + n) : (n == dv ? 1.f : 0.f);
+      },
+      sm);
+  float* O = out + (int64_t)(per_slice_out ? blockIdx.z : bh) * M * N;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+#pragma unroll
+  for (int i = 0; i < 4; i++) {
+    int m = m0 + ty + 16 * i;
+    if (m >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+      int n = n0 + tx + 16 * j;
+      if (n < N) {
+        if (per_slice_out) O[(int64_t)m * N + n] = acc[i][j];
+        else atomicAdd(&O[(int64_t)m * N + n], acc[i][j]);
+      }
+    }
+  }
+}
+
+// ---- exclusive prefix over chunks of the per-chunk S^T [V | 1] ---------------------------
+__global__ void __launch_bounds__(NTH)
+prefix_kernel(float* __restrict__ st, int nchunks, int64_t elems) {
+  const int bh = blockIdx.y;
+  float* base = st + (int64_t)bh * nchunks * elems;
+  for (int64_t e = blockIdx.x * (int64_t)NTH + threadIdx.x; e < elems; e += (int64_t)gridDim.x * NTH) {
+    float run = 0.f;
+    for (int c = 0; c < nchunks; c++) {
+      float v = base[c * elems + e];
+      base[c * elems + e] = run;
+      run += v;
+    }
+  }
+}
+
+// ---- masked in-chunk scores: sc[bh, c][i][j] = (j <= i) phiQ_i . phiK_j -------------------
+__global__ void __launch_bounds__(NTH)
+scores_kernel(const float* __restrict__ phiQ, const float* __restrict__ phiK, int L, int M, int C, int nchunks,
+              float* __restrict__ sc) {
+  __shared__ Tiles sm;
+  const int bh = blockIdx.z / nchunks, c = blockIdx.z % nchunks;
+  const int i0 = blockIdx.x * TM, j0 = blockIdx.y * TN;
+  float* S = sc + (int64_t)blockIdx.z * C * C;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  float acc[4][4] = {};
+  if (j0 <= i0) {
+    const float* PQ = phiQ + ((int64_t)bh * L + (int64_t)c * C) * M;
+    const float* PK = phiK + ((int64_t)bh * L + (int64_t)c * C) * M;
+    tile_gemm<true, true>(
+        acc, M, [&](int r, int k) { return PQ[(int64_t)(i0 + r) * M + k]; },
+        [&](int k, int cc) { return PK[(int64_t)(j0 + cc) * M + k]; }, sm);
+  }
+#pragma unroll
+  for (int i = 0; i < 4; i++)
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+      int r = i0 + ty + 16 * i, cc = j0 + tx + 16 * j;
+      S[(int64_t)r * C + cc] = (cc <= r) ? acc[i][j] : 0.f;
+    }
+}
+
+// ---- Y = num / den -------------------------------------------------------------------
+// Bidirectional: [num | den] = phiQ (S^T [V | 1]).  Causal: per chunk, phiQ_c times the
+// prefix state plus the masked scores times [V_c | 1].
+template <typename T>
+__global__ void __launch_bounds__(NTH)
+out_kernel(const float* __restrict__ phiQ, const float* __restrict__ KV, const float* __restrict__ sc,
+           const T* __restrict__ V, TensorAddr av, T* __restrict__ Y, TensorAddr ay, int H, int L, int M, int dv,
+           int causal, int C, int nchunks, int* __restrict__ status) {
+  __shared__ Tiles sm;
+  __shared__ float den[TM];
+  const int bh = blockIdx.z, b = bh / H, h = bh % H;
+  const int i0 = blockIdx.x * TM, n0 = blockIdx.y * TN;
+  const int N = dv + 1;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const float* PQ = phiQ + (int64_t)bh * L * M;
+  const int chunk = causal ? i0 / C : 0;
+  const float* S = KV + (int64_t)(causal ? bh * nchunks + chunk : bh) * M * N;
+  const float* SC = causal ? sc + ((int64_t)bh * nchunks + chunk) * C * C : nullptr;
+  const int ic = causal ? i0 - chunk * C : 0;   // row offset inside the chunk
+  const T* Vb = V + b * av.sb + h * av.sh;
+
+  // denominators: 4 threads per row
+  {
+    int r = tid >> 2, part = tid & 3;
+    float s = 0.f;
+    if (i0 + r < L) {
+      for (int m = part; m < M; m += 4) s = fmaf(PQ[(int64_t)(i0 + r) * M + m], S[(int64_t)m * N + dv], s);
+      if (causal)
+        for (int j = part; j < C; j += 4) s += SC[(int64_t)(ic + r) * C + j];
+    }
+    s += __shfl_xor_sync(0xffffffffu, s, 1);
+    s += __shfl_xor_sync(0xffffffffu, s, 2);
+    if (part == 0) den[r] = s;
+  }
+  __syncthreads();
+  float acc[4][4] = {};
+  tile_gemm<true, false>(
+      acc, M, [&](int r, int k) { return (i0 + r < L) ? PQ[(int64_t)(i0 + r) * M + k] : 0.f; },
+      [&](int k, int c) { return (n0 + c < dv) ? S[(int64_t)k * N + n0 + c] : 0.f; }, sm);
+  if (causal) {
+    const int jmax = min(C, ic + TM);   // columns beyond the tile's last row are masked to zero
+    tile_gemm<true, false>(
+        acc, jmax, [&](int r, int k) { return SC[(int64_t)(ic + r) * C + k]; },
+        [&](int k, int c) {
+          return (n0 + c < dv) ? fs_load(Vb + (int64_t)(chunk * C + k) * av.sl + n0 + c) : 0.f;
+        },
+        sm);
+  }
+  T* Yb = Y + b * ay.sb + h * ay.sh;
+  bool bad = false;
+#pragma unroll
+  for (int i = 0; i < 4; i++) {
+    int r = ty + 16 * i;
+    if (i0 + r >= L) continue;
+    float dn = den[r];
+    if (!(dn > 0.f) || !isfinite(dn)) bad = true;
+    float inv = 1.f / dn;
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+      int n = n0 + tx + 16 * j;
+      if (n < dv) fs_store(Yb + (int64_t)(i0 + r) * ay.sl + n, acc[i][j] * inv);
+    }
+  }
+  if (bad) atomicExch(status, FSHARP_E_NONFINITE);
+}
+
+template <typename T>
+int featurize_t(fsharp_ctx* ctx, const void* X, TensorAddr ax, int B, int H, int L, int d, int M, int pool,
+                const float* prep, int side, float qk_scale, int stab, float* rowc, float* phi, float* logscale) {
+  const int BH = B * H;
+  if (BH == 0 || L == 0) return FSHARP_OK;
+  {
+    int gx = (L + 7) / 8;
+    if (gx > 4 * ctx->sm_count) gx = 4 * ctx->sm_count;
+    // shared memory: dense C (d*d) + one x per warp; sized for the dense case
+    size_t smem = ((size_t)d * d + 8 * (size_t)d) * sizeof(float);
+    FS_CUDA_OK(cudaFuncSetAttribute(rowterm_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    rowterm_kernel<T><<<dim3(gx, BH), NTH, smem, ctx->stream>>>((const T*)X, ax, H, L, d, M, pool, side, prep,
+                                                               qk_scale, rowc);
+    FS_LAUNCH_CHECK(ctx);
+  }
+  logits_kernel<T><<<dim3((L + TM - 1) / TM, (M + TN - 1) / TN, BH), NTH, 0, ctx->stream>>>(
+      (const T*)X, ax, H, L, d, M, pool, side, prep, qk_scale, rowc, phi);
+  FS_LAUNCH_CHECK(ctx);
+  {
+    int gx = (L + 7) / 8;
+    if (gx > 4 * ctx->sm_count) gx = 4 * ctx->sm_count;
+    expshift_kernel<<<dim3(gx, BH), NTH, 0, ctx->stream>>>(phi, H, L, d, M, pool, side, stab, prep, logscale,
+                                                          ctx->d_status);
+    FS_LAUNCH_CHECK(ctx);
+  }
+  return FSHARP_OK;
+}
+
+template <typename T>
+int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, int causal,
+             int chunk, float qk_scale, const float* prep, void* Y, WsAlloc* ws) {
+  const int B = dm->B, H = dm->H, BH = B * H, Lq = dm->Lq, Lk = dm->Lk, d = dm->d, dv = dm->dv, M = dm->M;
+  const int N = dv + 1;
+  TensorAddr aq = fs_addr(dm->q_stride, H, Lq, d), ak = fs_addr(dm->k_stride, H, Lk, d);
+  TensorAddr av = fs_addr(dm->v_stride, H, Lk, dv), ay = fs_addr(dm->y_stride, H, Lq, dv);
+  float* phiQ = ws->take<float>((size_t)BH * Lq * M);
+  float* phiK = ws->take<float>((size_t)BH * Lk * M);
+  float* rowc = ws->take<float>((size_t)BH * (Lq > Lk ? Lq : Lk));
+  FS_TRY(featurize_t<T>(ctx, K, ak, B, H, Lk, d, M, dm->pool, prep, 2, qk_scale, FSHARP_STAB_GROUP, rowc, phiK,
+                        nullptr));
+  FS_TRY(featurize_t<T>(ctx, Q, aq, B, H, Lq, d, M, dm->pool, prep, 1, qk_scale, FSHARP_STAB_ROW, rowc, phiQ,
+                        nullptr));
+  dim3 gout((Lq + TM - 1) / TM, (dv + TN - 1) / TN, BH);
+  if (!causal) {
+    float* KV = ws->take<float>((size_t)BH * M * N);
+    FS_CUDA_OK(cudaMemsetAsync(KV, 0, (size_t)BH * M * N * sizeof(float), ctx->stream));
+    int nsl = (4 * ctx->sm_count + BH - 1) / BH;
+    int maxsl = (Lk + 255) / 256;
+    if (nsl > maxsl) nsl = maxsl;
+    if (nsl < 1) nsl = 1;
+    int slen = (Lk + nsl - 1) / nsl;
+    nsl = (Lk + slen - 1) / slen;
+    kv_kernel<T><<<dim3((M + TM - 1) / TM, (N + TN - 1) / TN, BH * nsl), NTH, 0, ctx->stream>>>(
+        phiK, (const T*)V, av, H, Lk, M, dv, slen, nsl, 0, KV);
+    FS_LAUNCH_CHECK(ctx);
+    out_kernel<T><<<gout, NTH, 0, ctx->stream>>>(phiQ, KV, nullptr, (const T*)V, av, (T*)Y, ay, H, Lq, M, dv, 0, 0,
+                                                1, ctx->d_status);
+    FS_LAUNCH_CHECK(ctx);
+  } else {
+    const int C = chunk, nch = Lq / C;
+    float* st = ws->take<float>((size_t)BH * nch * M * N);
+    float* sc = ws->take<float>((size_t)BH * nch * C * C);
+    kv_kernel<T><<<dim3((M + TM - 1) / TM, (N + TN - 1) / TN, BH * nch), NTH, 0, ctx->stream>>>(
+        phiK, (const T*)V, av, H, Lk, M, dv, C, nch, 1, st);
+    FS_LAUNCH_CHECK(ctx);
+    int64_t elems = (int64_t)M * N;
+    prefix_kernel<<<dim3((unsigned)((elems + NTH - 1) / NTH), BH), NTH, 0, ctx->stream>>>(st, nch, elems);
+    FS_LAUNCH_CHECK(ctx);
+    scores_kernel<<<dim3(C / TM, C / TN, BH * nch), NTH, 0, ctx->stream>>>(phiQ, phiK, Lq, M, C, nch, sc);
+    FS_LAUNCH_CHECK(ctx);
+    out_kernel<T><<<gout, NTH, 0, ctx->stream>>>(phiQ, st, sc, (const T*)V, av, (T*)Y, ay, H, Lq, M, dv, 1, C, nch,
+                                                ctx->d_status);
+    FS_LAUNCH_CHECK(ctx);
+  }
+  return FSHARP_OK;
+}
+
+}  // namespace
+
+int fs_simt_featurize(fsharp_ctx* ctx, const void* X, int dtype, TensorAddr ax, int B, int H, int L, int d,
+                      int M, int pool, const float* prep, int side, float qk_scale, int stab,
+                      float* rowc, float* phi, float* logscale) {
+  if (dtype == FSHARP_F32)
+    return featurize_t<float>(ctx, X, ax, B, H, L, d, M, pool, prep, side, qk_scale, stab, rowc, phi, logscale);
+  return featurize_t<__nv_bfloat16>(ctx, X, ax, B, H, L, d, M, pool, prep, side, qk_scale, stab, rowc, phi,
+                                    logscale);
+}
+
+size_t fs_simt_attend_scratch_bytes(const fsharp_dims* dm, int causal, int chunk) {
+  const size_t BH = (size_t)dm->B * dm->H, N = dm->dv + 1;
+  const size_t Lmax = dm->Lq > dm->Lk ? dm->Lq : dm->Lk;
+  size_t b = ws_round(BH * dm->Lq * dm->M * 4) + ws_round(BH * dm->Lk * dm->M * 4) + ws_round(BH * Lmax * 4);
+  if (!causal) {
+    b += ws_round(BH * dm->M * N * 4);
+  } else {
+    size_t nch = chunk > 0 ? dm->Lq / chunk : 0;
+    b += ws_round(BH * nch * dm->M * N * 4) + ws_round(BH * nch * (size_t)chunk * chunk * 4);
+  }
+  return b;
+}
+
+int fs_simt_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm,
+                   int dtype, int causal, int chunk, float qk_scale, const float* prep, void* Y, WsAlloc* ws) {
+  if (dtype == FSHARP_F32) return attend_t<float>(ctx, Q, K, V, dm, causal, chunk, qk_scale, prep, Y, ws);
+  return attend_t<__nv_bfloat16>(ctx, Q, K, V, dm, causal, chunk, qk_scale, prep, Y, ws);
+}

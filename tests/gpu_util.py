@@ -1,0 +1,42 @@
+"""Helpers shared by the GPU parity tests: device upload, the checker run per (batch, head),
+and the error metric max|Y_gpu - Y_ref| / max|Y_ref| per (batch, head)."""
+import numpy as np
+import torch
+
+from oracle import favor_sharp as fs
+from paper_2302_00787_b200 import binding as fb
+from paper_2302_00787_b200 import workloads as wl
+
+TOL = {"f32": 1e-4, "bf16": 1e-2}      # attention outputs, max relative error per (batch, head)
+FIT_TOL = 1e-5                          # parameter fits, relative
+
+
+def dev(a, dtype="f32"):
+    t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    return t.to(torch.bfloat16) if dtype == "bf16" else t
+
+
+def host(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def rel_err(got, ref):
+    return float(np.max(np.abs(got - ref)) / np.max(np.abs(ref)))
+
+
+def upload(w):
+    Q, K, V = wl.make_qkv(w)
+    Om = wl.make_omega(w)
+    return (Q, K, V, Om), (dev(Q, w.dtype), dev(K, w.dtype), dev(V, w.dtype), dev(Om))
+
+
+def gpu_fit(ctx, dQ, dK, d, variant, pool=fb.POOL_PER_BH):
+    st = ctx.fsharp_stats(dQ, dK, pool=pool)
+    pr = ctx.fsharp_fit_params(st, d, variant)
+    assert ctx.status() == 0
+    return st, pr
+
+
+def oracle_unit(Q, K, V, Om, blob, d, b, h, causal, rows=None):
+    p = fb.unpack_params(blob, d)
+    return fs.favor_sharp_attention(Q[b, h], K[b, h], V[b, h], Om, p, causal=causal, rows=rows)

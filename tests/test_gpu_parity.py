@@ -1,0 +1,347 @@
+"""GPU parity: every stage of the CUDA path, called through the C ABI, against the fp64
+checker on the same seeded inputs and the same Omega.  Tolerances: attention outputs 1e-4
+(fp32) / 1e-2 (bf16) max relative error per (batch, head); fits 1e-5 relative on the
+rotation-invariant quantities (the literal B of Theorems 4.2/4.3 is one of many solutions)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import favor_sharp as fs
+from paper_2302_00787_b200 import binding as fb
+from paper_2302_00787_b200 import workloads as wl
+from tests.gpu_util import FIT_TOL, TOL, dev, gpu_fit, host, oracle_unit, rel_err, upload
+
+pytestmark = pytest.mark.gpu
+
+W = wl.WORKLOADS
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = fb.Context(0)
+    yield c
+    c.close()
+
+
+def small_cases():
+    return [
+        W["cfg1"],
+        W["cfg2"].scaled(B=2, H=2, L=300),                       # ragged tail: 300 = 2*128 + 44
+        W["cfg3"].scaled(B=1, H=2, L=512),
+        W["cfg3b"].scaled(B=1, H=2, L=200),
+        W["cfg5"].scaled(B=1, H=2, L=1024, outlier_frac=0.1),
+        W["cfg1"].scaled(L=64, causal=True, chunk=64, variant="gerf"),
+        W["cfg1"].scaled(L=17, variant="posrf", d=32, dv=16, M=48),
+    ]
+
+
+# ------------------------------------------------------------------ stats
+@pytest.mark.parametrize("w", small_cases()[:5], ids=lambda w: w.name)
+def test_stats_match_definition(ctx, w):
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    st = host(ctx.fsharp_stats(dQ, dK))
+    d = w.d
+    for b in range(w.B):
+        for h in range(w.H):
+            ref = fs.set_statistics(Q[b, h], K[b, h])
+            g = st[b * w.H + h]
+            M1, M2 = g[: d * d].reshape(d, d), g[d * d: 2 * d * d].reshape(d, d)
+            scale = np.abs(ref["M1"]).max()
+            assert np.abs(M1 - ref["M1"]).max() < 2e-6 * scale
+            assert np.abs(M2 - ref["M2"]).max() < 2e-6 * scale
+            assert np.abs(g[2 * d * d: 2 * d * d + d] - ref["mu4"]).max() < 2e-6
+            assert np.abs(g[2 * d * d + d: 2 * d * d + 2 * d] - ref["mu5"]).max() < 2e-6
+            assert abs(g[-2] / np.max(np.sum(Q[b, h].astype(np.float64) ** 2, axis=1)) - 1) < 1e-5
+            assert abs(g[-1] / np.max(np.sum(K[b, h].astype(np.float64) ** 2, axis=1)) - 1) < 1e-5
+
+
+def test_stats_pooled_over_batch_and_strided(ctx):
+    w = W["cfg2"].scaled(B=3, H=2, L=160)
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    st = host(ctx.fsharp_stats(dQ, dK, pool=fb.POOL_PER_HEAD))
+    assert st.shape[0] == w.H
+    for h in range(w.H):
+        ref = fs.set_statistics(Q[:, h].reshape(-1, w.d), K[:, h].reshape(-1, w.d))
+        assert np.abs(st[h][: w.d * w.d].reshape(w.d, w.d) - ref["M1"]).max() < 2e-6 * np.abs(ref["M1"]).max()
+    # [B, L, H, d] storage viewed as [B, H, L, d]
+    dQs = dQ.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    dKs = dK.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    assert not dQs.is_contiguous()
+    st2 = host(ctx.fsharp_stats(dQs, dKs, pool=fb.POOL_PER_HEAD))
+    assert np.abs(st2 - st).max() < 1e-12
+
+
+# ------------------------------------------------------------------ fits
+def invariants(p, d):
+    """Quantities that do not depend on eigenvector signs or rotations in equal eigenvalues."""
+    return {
+        "eigA": np.sort(np.linalg.eigvalsh(p["A"])),
+        "logD": np.array([p["logD"]]),
+        "objective": np.array([p["objective"]]),
+        "B1tB1": p["B1"].T @ p["B1"], "B2tB2": p["B2"].T @ p["B2"], "B1tB2": p["B1"].T @ p["B2"],
+        "C1": p["C1"], "C2": p["C2"],
+        "B1tAB1": p["B1"].T @ p["A"] @ p["B1"],
+    }
+
+
+def assert_fit_close(got, ref, d, tol):
+    gi, ri = invariants(got, d), invariants(ref, d)
+    for k in ri:
+        scale = max(np.abs(ri[k]).max(), 1e-30)
+        assert np.abs(gi[k] - ri[k]).max() <= tol * scale, (k, np.abs(gi[k] - ri[k]).max() / scale)
+
+
+@pytest.mark.parametrize("variant", ["posrf", "gerf", "saderf", "aderf", "sderf"])
+@pytest.mark.parametrize("d", [16, 64, 128])
+def test_fit_from_exact_statistics(ctx, variant, d):
+    """The fit kernel alone: statistics computed by the checker in fp64, uploaded, fitted on
+    the GPU; invariants agree to 1e-9 and the blob satisfies Theorem 4.1's conditions."""
+    rng = np.random.default_rng(100 + d)
+    G, L = 3, 4 * d
+    sl = fb.stats_doubles(d)
+    blob = np.zeros((G, sl))
+    refs = []
+    for g in range(G):
+        X = rng.standard_normal((L, d)) * rng.uniform(0.5, 1.5, d) / d ** 0.25 + 0.05 * g
+        Y = rng.standard_normal((L, d)) * rng.uniform(0.5, 1.5, d) / d ** 0.25 - 0.03
+        st = fs.set_statistics(X, Y)
+        blob[g, : d * d] = st["M1"].ravel()
+        blob[g, d * d: 2 * d * d] = st["M2"].ravel()
+        blob[g, 2 * d * d: 2 * d * d + d] = st["mu4"]
+        blob[g, 2 * d * d + d: 2 * d * d + 2 * d] = st["mu5"]
+        blob[g, -2:] = [np.max(np.sum(X * X, 1)), np.max(np.sum(Y * Y, 1))]
+        refs.append(fs.FITS[variant](st))
+    pr = ctx.fsharp_fit_params(torch.from_numpy(blob).cuda(), d, variant)
+    assert ctx.status() == 0
+    pr = pr.cpu().numpy()
+    I = np.eye(d)
+    for g in range(G):
+        p = fb.unpack_params(pr[g], d)
+        assert_fit_close(p, refs[g], d, 1e-9)
+        Sinv = np.linalg.inv(I - 4 * p["A"])
+        assert np.abs(p["B1"].T @ Sinv @ p["B2"] - I).max() < 1e-9
+        assert np.abs(p["C1"] + 0.5 * p["B1"].T @ Sinv @ p["B1"]).max() < 1e-9 * max(1, np.abs(p["C1"]).max())
+        if variant == "sderf":
+            a = np.diag(p["A"])
+            assert np.all(np.diff(a) >= -1e-15)          # eigenvalues of N non-ascending
+        # the guard constants are true lower bounds
+        for k in (1, 2):
+            lam_min = np.linalg.eigvalsh(-p[f"C{k}"]).min()
+            assert p[f"kappa{k}"] <= lam_min * (1 + 1e-9) + 1e-15
+
+
+@pytest.mark.parametrize("w", small_cases()[:5], ids=lambda w: w.name)
+def test_stats_then_fit_end_to_end(ctx, w):
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    for variant in ("sderf", "aderf", "gerf", "saderf"):
+        _, pr = gpu_fit(ctx, dQ, dK, w.d, variant)
+        pr = pr.cpu().numpy()
+        for b in range(w.B):
+            for h in range(w.H):
+                ref = fs.fit_params(Q[b, h], K[b, h], variant)
+                assert_fit_close(fb.unpack_params(pr[b * w.H + h], w.d), ref, w.d, FIT_TOL)
+
+
+# ------------------------------------------------------------------ featurize
+@pytest.mark.parametrize("w", [small_cases()[0], small_cases()[2], small_cases()[4]], ids=lambda w: w.name)
+@pytest.mark.parametrize("stab", [fb.STAB_NONE, fb.STAB_ROW, fb.STAB_GROUP])
+def test_featurize_matches_definition(ctx, w, stab):
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    _, pr = gpu_fit(ctx, dQ, dK, w.d, w.variant)
+    prh = pr.cpu().numpy()
+    for side, X, dX in ((1, Q, dQ), (2, K, dK)):
+        phi, ls = ctx.fsharp_featurize(dX, dOm, pr, side, stab=stab)
+        assert ctx.status() == 0
+        phi = host(phi)
+        for b in range(w.B):
+            for h in range(w.H):
+                p = fb.unpack_params(prh[b * w.H + h], w.d)
+                ref = fs.derf_log_features(X[b, h], Om, p["A"], p[f"B{side}"], p[f"C{side}"], p["logD"])
+                if stab == fb.STAB_ROW:
+                    shift = host(ls)[b, h][:, None]
+                    assert phi[b, h].max() <= 1.0 + 1e-6
+                elif stab == fb.STAB_GROUP:
+                    shift = host(ls)[b, h]
+                    assert np.all(ref - shift <= 40.0 + 1e-3)   # the bound holds with its headroom
+                else:
+                    shift = 0.0
+                got = phi[b, h]
+                expect = np.exp(ref - shift)
+                big = expect > 1e-30                                # below that fp32 has flushed
+                tol = 2e-4 if w.dtype == "f32" else 2e-4
+                assert np.max(np.abs(got[big] / expect[big] - 1)) < tol
+
+
+# ------------------------------------------------------------------ attend
+@pytest.mark.parametrize("w", small_cases(), ids=lambda w: f"{w.name}-L{w.L}-{w.variant}")
+@pytest.mark.parametrize("impl", [fb.IMPL_SIMT, fb.IMPL_AUTO])
+def test_attend_small_full_parity(ctx, w, impl):
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    _, pr = gpu_fit(ctx, dQ, dK, w.d, w.variant)
+    ctx.set_impl(impl)
+    try:
+        Y = ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=w.causal, chunk=w.chunk)
+        assert ctx.status() == 0
+    finally:
+        ctx.set_impl(fb.IMPL_AUTO)
+    Y = host(Y)
+    prh = pr.cpu().numpy()
+    for b in range(w.B):
+        for h in range(w.H):
+            ref = oracle_unit(Q, K, V, Om, prh[b * w.H + h], w.d, b, h, w.causal)
+            assert rel_err(Y[b, h], ref) < TOL[w.dtype], (b, h)
+    if w.causal:
+        assert np.abs(Y[:, :, 0] - V[:, :, 0]).max() < (1e-5 if w.dtype == "f32" else 1e-2)
+
+
+def test_attend_properties(ctx):
+    w = W["cfg2"].scaled(B=1, H=3, L=384)
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    _, pr = gpu_fit(ctx, dQ, dK, w.d, w.variant)
+    ones = torch.ones_like(dV)
+    Y1 = host(ctx.fsharp_attend(dQ, dK, ones, dOm, pr))
+    assert np.abs(Y1 - 1).max() < 1e-2                      # right stochastic: V = 1 gives Y = 1
+    Y = host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr))
+    perm = torch.randperm(w.L, generator=torch.Generator().manual_seed(1)).cuda()
+    Yp = host(ctx.fsharp_attend(dQ, dK[:, :, perm].contiguous(), dV[:, :, perm].contiguous(), dOm, pr))
+    assert np.abs(Y - Yp).max() < 2e-2                      # key order does not matter
+    # causal: outputs before position t do not depend on tokens from t on; chunk size is immaterial
+    wc = W["cfg3"].scaled(B=1, H=2, L=512)
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(wc)
+    _, pr = gpu_fit(ctx, dQ, dK, wc.d, wc.variant)
+    Ya = host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=True, chunk=128))
+    dK2, dV2 = dK.clone(), dV.clone()
+    dK2[:, :, 300:] *= 1.5
+    dV2[:, :, 300:] += 1.0
+    Yb = host(ctx.fsharp_attend(dQ, dK2, dV2, dOm, pr, causal=True, chunk=128))
+    assert np.abs(Ya[:, :, :300] - Yb[:, :, :300]).max() == 0.0
+    for ch in (64, 256):
+        Yc = host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=True, chunk=ch))
+        assert rel_err(Yc, Ya) < 1e-2
+    assert ctx.status() == 0
+
+
+def test_attend_strided_layout_per_head_omega_and_pooling(ctx):
+    w = W["cfg2"].scaled(B=2, H=3, L=256)
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    OmH = np.stack([wl.orthogonal_omega(w.M, w.d, 77 + h) for h in range(w.H)])
+    dOmH = dev(OmH)
+    st = ctx.fsharp_stats(dQ, dK, pool=fb.POOL_PER_HEAD)
+    pr = ctx.fsharp_fit_params(st, w.d, "sderf")
+    tr = lambda t: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    out = torch.empty(w.B, w.L, w.H, w.dv, dtype=dQ.dtype, device="cuda").permute(0, 2, 1, 3)
+    Y = ctx.fsharp_attend(tr(dQ), tr(dK), tr(dV), dOmH, pr, pool=fb.POOL_PER_HEAD, out=out)
+    assert ctx.status() == 0
+    Y = host(Y)
+    prh = pr.cpu().numpy()
+    for b in range(w.B):
+        for h in range(w.H):
+            p = fb.unpack_params(prh[h], w.d)
+            ref = fs.favor_sharp_attention(Q[b, h], K[b, h], V[b, h], OmH[h], p)
+            assert rel_err(Y[b, h], ref) < TOL["bf16"]
+
+
+def test_qk_scale_is_applied(ctx):
+    w = W["cfg1"]
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    s = w.d ** -0.25
+    st = ctx.fsharp_stats(dQ, dK, qk_scale=s)
+    pr = ctx.fsharp_fit_params(st, w.d, "sderf")
+    Y = host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr, qk_scale=s))
+    p = fb.unpack_params(pr.cpu().numpy()[0], w.d)
+    ref = fs.favor_sharp_attention(Q[0, 0], K[0, 0], V[0, 0], Om, p, qk_scale=s)
+    assert rel_err(Y[0, 0], ref) < TOL["f32"]
+    refp = fs.fit_params(s * Q[0, 0].astype(np.float64), s * K[0, 0].astype(np.float64), "sderf")
+    assert abs(p["objective"] - refp["objective"]) < FIT_TOL * abs(refp["objective"])
+
+
+def test_forward_host_matches_device_path(ctx):
+    w = W["cfg3"].scaled(B=1, H=2, L=256)
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    _, pr = gpu_fit(ctx, dQ, dK, w.d, w.variant)
+    Yd = host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=True, chunk=128))
+    pin = lambda t: t.cpu().contiguous().pin_memory()
+    Yh = ctx.fsharp_forward_host(pin(dQ), pin(dK), pin(dV), pin(dOm), w.variant, causal=True, chunk=128)
+    assert np.abs(host(Yh) - Yd).max() < 2e-2
+    assert rel_err(host(Yh)[0, 0], oracle_unit(Q, K, V, Om, pr.cpu().numpy()[0], w.d, 0, 0, True)) < TOL["bf16"]
+
+
+# ------------------------------------------------------------------ edge cases and errors
+def test_empty_and_degenerate_inputs(ctx):
+    d, M = 16, 32
+    Om = dev(wl.iid_omega(M, d, 1))
+    pr = torch.zeros(1, fb.params_doubles(d), dtype=torch.float64, device="cuda")
+    e = torch.empty(1, 1, 0, d, device="cuda")
+    assert ctx.fsharp_attend(e, e, e, Om, pr).shape == (1, 1, 0, d)            # no query: nothing to do
+    e0 = torch.empty(0, 1, 8, d, device="cuda")
+    assert ctx.fsharp_stats(e0, e0).shape[0] == 0
+    # single token: Y = V exactly (one key carries all the weight)
+    w = W["cfg1"].scaled(L=1)
+    (Q, K, V, Om1), (dQ, dK, dV, dOm) = upload(w)
+    st = ctx.fsharp_stats(dQ, dK)
+    prg = ctx.fsharp_fit_params(st, w.d, "gerf")
+    Y = host(ctx.fsharp_attend(dQ, dK, dV, dOm, prg))
+    assert np.abs(Y - V).max() < 1e-5
+    assert ctx.status() == 0
+
+
+def test_error_codes(ctx):
+    w = W["cfg1"].scaled(L=64)
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    _, pr = gpu_fit(ctx, dQ, dK, w.d, "sderf")
+
+    def code(fn):
+        with pytest.raises(fb.FsharpError) as ei:
+            fn()
+        return ei.value.code
+
+    assert code(lambda: ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=True, chunk=48)) == -2     # chunk size
+    assert code(lambda: ctx.fsharp_attend(dQ[:, :, :40].contiguous(), dK[:, :, :40].contiguous(),
+                                          dV[:, :, :40].contiguous(), dOm, pr, causal=True, chunk=64)) == -2
+    bad = torch.empty(1, 1, 64, 24, device="cuda")
+    assert code(lambda: ctx.fsharp_stats(bad, bad)) == -2                                         # d = 24
+    flat = torch.empty(64 * 16 + 1, device="cuda")[1:].view(1, 1, 64, 16)
+    assert code(lambda: ctx.fsharp_stats(flat, flat)) == -3                                       # misaligned
+    assert code(lambda: ctx.fsharp_attend(dQ, dK[:, :, :0], dV[:, :, :0], dOm, pr)) == -2         # no keys
+    lib = fb.load_library()
+    assert lib.fsharp_fit_params(ctx._h, None, 1, 16, 4, 0.0, pr.data_ptr()) == -1
+    assert lib.fsharp_fit_params(ctx._h, pr.data_ptr(), 1, 16, 9, 0.0, pr.data_ptr()) == -1
+    assert ctx.status() == 0
+
+
+def test_device_detected_conditions(ctx):
+    w = W["cfg1"].scaled(L=64)
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    dQn = dQ.clone()
+    dQn[0, 0, 3, 5] = float("nan")
+    ctx.fsharp_stats(dQn, dK)
+    assert ctx.status() == -7                      # non-finite input
+    assert ctx.status() == 0                       # reading clears it
+    dQz = dQ.clone()
+    dQz[..., 2] = 0.0                              # a zero column makes M1 singular
+    st = ctx.fsharp_stats(dQz, dK)
+    ctx.fsharp_fit_params(st, w.d, "aderf")
+    assert ctx.status() == -6
+    pr = ctx.fsharp_fit_params(st, w.d, "aderf", ridge=1e-3)     # the ridge repairs it
+    assert ctx.status() == 0
+    assert torch.isfinite(pr).all()
+
+
+# ------------------------------------------------------------------ pairs
+@pytest.mark.parametrize("variant", ["aderf", "sderf", "gerf", "posrf"])
+def test_pair_estimates_and_closed_form_variance(ctx, variant):
+    npairs, d, M, R = 1000, 64, 64, 3
+    X, Y = wl.make_pairs(npairs, d)
+    Om = np.stack([wl.orthogonal_omega(M, d, 4000 + r) for r in range(R)])
+    dX, dY = dev(X), dev(Y)
+    st = ctx.fsharp_stats(dX.view(1, 1, npairs, d), dY.view(1, 1, npairs, d))
+    pr = ctx.fsharp_fit_params(st, d, variant)
+    est, var = ctx.fsharp_pair_estimate(dX, dY, dev(Om), pr)
+    assert ctx.status() == 0
+    p = fb.unpack_params(pr.cpu().numpy()[0], d)
+    for r in range(R):
+        ref = fs.pair_estimate(X, Y, Om[r], p)
+        assert np.max(np.abs(host(est[r]) / ref - 1)) < 1e-4
+    sel = np.arange(0, npairs, 37)
+    refv = fs.pair_closed_form_variance(X[sel], Y[sel], p, M)
+    assert np.max(np.abs(var.cpu().numpy()[sel] / refv - 1)) < 1e-8
