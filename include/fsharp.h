@@ -102,20 +102,15 @@ const char* fsharp_strerror(int code);
 /* ---- layouts of the two fp64 blobs ---------------------------------------- */
 
 /* Doubles per group in the statistics blob:
- *   [M1 (d*d, row-major)] [M2 (d*d)] [mu4 (d)] [mu5 (d)] [max_i |x_i|^2] [max_j |y_j|^2]
- * = 2 d^2 + 2 d + 2. */
+ *   [M1 (d*d, row-major)] [M2 (d*d)] [mu4 (d)] [mu5 (d)]  = 2 d^2 + 2 d. */
 size_t fsharp_stats_doubles(int d);
 /* Doubles per group in the parameter blob:
  *   [A (d*d, symmetric)] [B1 (d*d)] [B2 (d*d)] [C1 (d*d)] [C2 (d*d)]
- *   [logD] [objective] [phi] [kappa1] [kappa2] [rho2max_x] [rho2max_y] [reserved]
+ *   [logD] [objective] [phi] [5 reserved, zero]
  * = 5 d^2 + 8.  objective is the shifted log-variance of Section 3.1 at the
  * optimum (Theorems 4.2 / 4.3); phi is the argument of Lemma A.1 (ADERF, GERF,
- * SADERF; for SDERF the largest eigenvalue of N).  kappa_k >= 0 is a lower bound on
- * the smallest eigenvalue of -C^(k) and rho2max the largest squared norm in the
- * set; they only steer the overflow guard (any per-row factor on queries and any
- * per-group factor on keys cancels in Section 2.2's normalisation), never the
- * mathematical result.  A caller who writes a blob by hand may set kappa = 0 and
- * rho2max to the largest squared norm it expects. */
+ * SADERF; for SDERF the largest eigenvalue of N).  Only A, B, C and logD enter the
+ * features; a caller may write a blob by hand (e.g. PosRF: A = 0, B = I, C = -I/2). */
 size_t fsharp_params_doubles(int d);
 
 /* ---- the path -------------------------------------------------------------- */
@@ -142,7 +137,10 @@ int fsharp_fit_params(fsharp_ctx* ctx, const double* stats, int G, int d, int va
  * w_m^T B x_i + x_i^T C x_i).  X is addressed with (Lq, q_stride) for side 1 and
  * (Lk, k_stride) for side 2.  Omega: float32 [M, d] (or [H, M, d]).
  * phi: float32, dense [B,H,L,M].  logscale: float32, [B,H,L] for FSHARP_STAB_ROW,
- * [B,H] for FSHARP_STAB_GROUP, ignored (may be NULL) for FSHARP_STAB_NONE. */
+ * [B,H] for FSHARP_STAB_GROUP, ignored (may be NULL) for FSHARP_STAB_NONE.
+ * ROW shifts by the row's largest exponent, GROUP by the largest exponent of the whole
+ * (batch, head), so phi <= 1 in both; any per-row factor on queries and any per-(batch,
+ * head) factor on keys cancels in Section 2.2's normalisation. */
 int fsharp_featurize(fsharp_ctx* ctx, const void* X, const float* Omega, const double* params,
                      int side, const fsharp_dims* dims, int dtype, float qk_scale, int stab,
                      float* phi, float* logscale);

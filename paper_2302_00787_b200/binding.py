@@ -252,11 +252,10 @@ def unpack_params(blob: torch.Tensor, d: int):
     t = b[5 * dd:]
     return {"A": b[0:dd].reshape(d, d), "B1": b[dd:2 * dd].reshape(d, d), "B2": b[2 * dd:3 * dd].reshape(d, d),
             "C1": b[3 * dd:4 * dd].reshape(d, d), "C2": b[4 * dd:5 * dd].reshape(d, d),
-            "logD": float(t[0]), "objective": float(t[1]), "phi": float(t[2]),
-            "kappa1": float(t[3]), "kappa2": float(t[4]), "rho2max_x": float(t[5]), "rho2max_y": float(t[6])}
+            "logD": float(t[0]), "objective": float(t[1]), "phi": float(t[2])}
 
 
-def pack_params(p: dict, d: int, kappa=(0.0, 0.0), rho2max=(0.0, 0.0)):
+def pack_params(p: dict, d: int):
     """Builds a parameter blob (numpy float64) from matrices A, B1, B2, C1, C2 and logD."""
     import numpy as np
     out = np.zeros(5 * d * d + 8, dtype=np.float64)
@@ -265,6 +264,4 @@ def pack_params(p: dict, d: int, kappa=(0.0, 0.0), rho2max=(0.0, 0.0)):
     t = out[5 * d * d:]
     t[0] = p["logD"]
     t[1] = p.get("objective", 0.0)
-    t[3], t[4] = kappa
-    t[5], t[6] = rho2max
     return out

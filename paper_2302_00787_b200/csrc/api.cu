@@ -41,10 +41,11 @@ extern "C" {
 
 int fsharp_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dims* dims, int dtype,
                  float qk_scale, double* stats) {
-  if (!ctx || !stats) return FSHARP_E_BADARG;
+  if (!ctx) return FSHARP_E_BADARG;
   FS_TRY(check_dims(dims, false));
   if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
   if (dims->B * dims->H == 0) return FSHARP_OK;
+  if (!stats) return FSHARP_E_BADARG;
   FS_TRY(check_ptr(Q, dtype, dims->q_stride));
   FS_TRY(check_ptr(K, dtype, dims->k_stride));
   FS_CUDA_OK(cudaSetDevice(ctx->device));
@@ -79,15 +80,17 @@ int fsharp_featurize(fsharp_ctx* ctx, const void* X, const float* Omega, const d
   FS_CUDA_OK(cudaSetDevice(ctx->device));
   const int G = fs_groups(dims);
   const size_t prep_f = (size_t)G * 2 * PrepLayout{dims->d, dims->M}.total();
-  const size_t need = ws_round(prep_f * 4) + ws_round((size_t)dims->B * dims->H * L * 4);
+  const size_t need = ws_round(prep_f * 4) + ws_round((size_t)dims->B * dims->H * L * 4) +
+                      ws_round((size_t)dims->B * dims->H * 4);
   FS_TRY(fs_ws_reserve(ctx, need));
   WsAlloc ws{ctx->ws, 0};
   float* prep = ws.take<float>(prep_f);
   float* rowc = ws.take<float>((size_t)dims->B * dims->H * L);
+  unsigned* gmax = ws.take<unsigned>((size_t)dims->B * dims->H);
   FS_TRY(fs_run_prep(ctx, Omega, dims->omega_head_stride, params, (int64_t)ParamsLayout{dims->d}.total(), G,
                      dims->H, dims->pool, dims->d, dims->M, prep));
   return fs_simt_featurize(ctx, X, dtype, fs_addr(st, dims->H, L, dims->d), dims->B, dims->H, L, dims->d, dims->M,
-                           dims->pool, prep, side, qk_scale, stab, rowc, phi, logscale);
+                           dims->pool, prep, side, qk_scale, stab, rowc, gmax, phi, logscale);
 }
 
 int fsharp_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const float* Omega,

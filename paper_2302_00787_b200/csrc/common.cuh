@@ -20,14 +20,13 @@ struct ParamsLayout {
   __host__ __device__ size_t tail() const { return 5 * dd(); }
   __host__ __device__ size_t total() const { return 5 * dd() + 8; }
 };
-enum { PT_LOGD = 0, PT_OBJ = 1, PT_PHI = 2, PT_KAPPA1 = 3, PT_KAPPA2 = 4, PT_RHO2X = 5, PT_RHO2Y = 6, PT_RES = 7 };
+enum { PT_LOGD = 0, PT_OBJ = 1, PT_PHI = 2 };   // tail[3..7] reserved (zero)
 
 struct StatsLayout {
   int d;
   __host__ __device__ size_t M(int k) const { return (size_t)d * d * (size_t)(k - 1); }               // k = 1, 2
   __host__ __device__ size_t mu(int k) const { return 2 * (size_t)d * d + (size_t)d * (k - 4); }      // k = 4, 5
-  __host__ __device__ size_t rho2(int k) const { return 2 * (size_t)d * d + 2 * (size_t)d + (k - 1); }  // k = 1, 2
-  __host__ __device__ size_t total() const { return 2 * (size_t)d * d + 2 * (size_t)d + 2; }
+  __host__ __device__ size_t total() const { return 2 * (size_t)d * d + 2 * (size_t)d; }
 };
 
 // What prep produces per (group, side): everything the feature kernels need (fp32).
@@ -43,14 +42,8 @@ struct PrepLayout {
   __host__ __device__ size_t Cmat() const { return (size_t)M * d + M + 8; }
   __host__ __device__ size_t total() const { return (size_t)M * d + M + 8 + (size_t)d * d; }
 };
-// PS_BIAS logD - 1/2 log M; PS_AMAX max_m a_m; PS_WMAX max_m |W_m|; PS_CSCALAR 1 if C = gamma I;
-// PS_CGAMMA gamma; PS_GSHIFT the per-group shift used for keys; PS_KAPPA, PS_RHO2 copied from the blob.
-enum { PS_BIAS = 0, PS_AMAX = 1, PS_WMAX = 2, PS_CSCALAR = 3, PS_CGAMMA = 4, PS_GSHIFT = 5, PS_KAPPA = 6, PS_RHO2 = 7 };
-
-// Headroom (natural-log units) left above the guaranteed upper bound of a key
-// exponent when the per-group shift is chosen: key features are at most
-// exp(FS_MARGIN); sums of up to 2^17 of them times |V| stay far below exp(88).
-#define FS_MARGIN 40.0f
+// PS_BIAS logD - 1/2 log M; PS_AMAX max_m a_m; PS_CSCALAR 1 if C = gamma I; PS_CGAMMA gamma.
+enum { PS_BIAS = 0, PS_AMAX = 1, PS_CSCALAR = 3, PS_CGAMMA = 4 };
 
 struct fsharp_ctx {
   int device;
@@ -139,10 +132,10 @@ size_t fs_fit_scratch_doubles(int G, int d);
 // params_stride: doubles between the blobs of two groups (0 = every group reads the same blob)
 int fs_run_prep(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_stride, const double* params,
                 int64_t params_stride, int G, int H, int pool, int d, int M, float* prep /* [G][2][PrepLayout] */);
-// rowc: scratch [B*H*L] floats.  phi: [B,H,L,M] floats.
+// rowc: scratch [B*H*L] floats.  gmax: scratch [B*H] words.  phi: [B,H,L,M] floats.
 int fs_simt_featurize(fsharp_ctx* ctx, const void* X, int dtype, TensorAddr ax, int B, int H, int L, int d,
                       int M, int pool, const float* prep, int side, float qk_scale, int stab,
-                      float* rowc, float* phi, float* logscale);
+                      float* rowc, unsigned* gmax, float* phi, float* logscale);
 int fs_simt_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm,
                    int dtype, int causal, int chunk, float qk_scale, const float* prep, void* Y,
                    WsAlloc* ws);

@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
   double* oC1 = out + pl.C(1);
   double* oC2 = out + pl.C(2);
   double* tail = out + pl.tail();
-  double logD = 0.0, obj = 0.0, phi = 0.0, kap1 = 0.5, kap2 = 0.5;
+  double logD = 0.0, obj = 0.0, phi = 0.0;
   bool violated = false;
 
   if (a.variant == FSHARP_POSRF || a.variant == FSHARP_GERF) {
@@ -171,19 +171,15 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
     obj = d * (log(1.0 - 4.0 * A) - 0.5 * log(1.0 - 8.0 * A)) + (2.0 - 8.0 * A) / (1.0 - 8.0 * A) * S - t1 - t2;
   } else if (a.variant == FSHARP_SADERF) {
     // Section 4.3: Psi_ll = (M2_ll / M1_ll)^(1/4), then the GERF fit on {Psi x}, {Psi^-1 y}.
-    double sq = 0.0, kmin1 = 1e300, kmin2 = 1e300;
+    double sq = 0.0;
     for (int i = tid; i < d; i += FIT_THREADS) {
       double m1 = M1[i * d + i] + rg1, m2 = M2[i * d + i] + rg2;
       if (!(m1 > 0.0) || !(m2 > 0.0)) { violated = true; m1 = fmax(m1, 1e-300); m2 = fmax(m2, 1e-300); }
       double psi2 = sqrt(m2 / m1);
       lam[i] = sqrt(psi2);
       sq += sqrt(m1 * m2);
-      kmin1 = fmin(kmin1, psi2);
-      kmin2 = fmin(kmin2, 1.0 / psi2);
     }
     sq = block_reduce(sq, red, 0);
-    kap1 = 0.5 * block_reduce(kmin1, red, 2);
-    kap2 = 0.5 * block_reduce(kmin2, red, 2);
     const double S = 2.0 * sq + 2.0 * mm;
     phi = S / d;
     const double A = lemma_a1(phi);
@@ -321,20 +317,12 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
     }
     logD = 0.25 * d * log(1.0 - 4.0 * A);
     obj = d * (log(1.0 - 4.0 * A) - 0.5 * log(1.0 - 8.0 * A) + 2.0 / (1.0 - 8.0 * A) * (ssum / d + mu3) + 2.0 * mu3);
-    // -C1 = F/2 and -C2 = F^-1/2 with F = Q1 L1^-1/2 U Sigma U^T L1^-1/2 Q1^T:
-    // lambda_min(F) >= sigma_min / lambda1_max, lambda_min(F^-1) >= lambda1_min / sigma_max.
-    kap1 = 0.5 * smin / lmax;
-    kap2 = 0.5 * lmin / smax;
   }
   if (tid == 0) {
     tail[PT_LOGD] = logD;
     tail[PT_OBJ] = obj;
     tail[PT_PHI] = phi;
-    tail[PT_KAPPA1] = kap1;
-    tail[PT_KAPPA2] = kap2;
-    tail[PT_RHO2X] = st[sl.rho2(1)];
-    tail[PT_RHO2Y] = st[sl.rho2(2)];
-    tail[PT_RES] = 0.0;
+    for (int i = 3; i < 8; i++) tail[i] = 0.0;
   }
   if (violated) atomicExch(a.status, FSHARP_E_CONSTRAINT);
 }

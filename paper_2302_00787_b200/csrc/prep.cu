@@ -1,6 +1,6 @@
 // Per-group precomputation for the feature kernels (Section 4, cost paragraph):
 // W^(k) = Omega B^(k) (row m = (B^(k)T w_m)^T), a_m = w_m^T A w_m, the constant
-// log D - 1/2 log M, and the bound that fixes the per-group shift of the keys.
+// log D - 1/2 log M.
 #include "common.cuh"
 
 namespace {
@@ -11,7 +11,6 @@ __global__ void __launch_bounds__(PREP_THREADS)
 prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const double* __restrict__ params,
             int64_t params_stride, int H, int pool, int d, int M, float* __restrict__ prep) {
   __shared__ float red[PREP_THREADS];
-  __shared__ float red2[PREP_THREADS];
   __shared__ int redi[PREP_THREADS];
   const int g = blockIdx.x, side = blockIdx.y + 1, tid = threadIdx.x;
   const int h = pool == FSHARP_POOL_PER_BH ? g % H : g;
@@ -54,47 +53,21 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
     Cf[e] = (float)Cm[e];
     if (i == j ? (Cm[e] != gamma) : (Cm[e] != 0.0)) cscalar = 0;
   }
-  __syncthreads();   // W complete
-  float wmax = 0.f;
-  for (int m = tid; m < M; m += PREP_THREADS) {
-    float s = 0.f;
-    for (int j = 0; j < d; j++) s = fmaf(W[m * d + j], W[m * d + j], s);
-    wmax = fmaxf(wmax, sqrtf(s));
-  }
-  red[tid] = amax; red2[tid] = wmax; redi[tid] = cscalar;
+  red[tid] = amax; redi[tid] = cscalar;
   __syncthreads();
   for (int s = PREP_THREADS / 2; s > 0; s >>= 1) {
     if (tid < s) {
       red[tid] = fmaxf(red[tid], red[tid + s]);
-      red2[tid] = fmaxf(red2[tid], red2[tid + s]);
       redi[tid] = redi[tid] & redi[tid + s];
     }
     __syncthreads();
   }
   if (tid == 0) {
-    amax = red[0];
-    wmax = red2[0] * 1.0001f;   // round the norm bound upwards
-    const float bias = (float)(tail[PT_LOGD] - 0.5 * log((double)M));
-    const float kappa = (float)fmax(tail[side == 1 ? PT_KAPPA1 : PT_KAPPA2], 0.0);
-    const double rho2 = tail[side == 1 ? PT_RHO2X : PT_RHO2Y];
-    // exponent <= bias + a_max + max_{0 <= rho <= rho_max} (w_max rho - kappa rho^2)   (Cauchy-Schwarz)
-    float lin;
-    const bool rho_ok = isfinite(rho2) && rho2 >= 0.0;
-    const float rhomax = rho_ok ? (float)sqrt(rho2) * 1.0001f : 0.f;
-    if (kappa > 0.f) {
-      float rstar = wmax / (2.f * kappa);
-      lin = (!rho_ok || rhomax >= rstar) ? wmax * wmax / (4.f * kappa) : wmax * rhomax - kappa * rhomax * rhomax;
-    } else {
-      lin = wmax * rhomax;
-    }
-    scal[PS_BIAS] = bias;
-    scal[PS_AMAX] = amax;
-    scal[PS_WMAX] = wmax;
+    for (int i = 0; i < 8; i++) scal[i] = 0.f;
+    scal[PS_BIAS] = (float)(tail[PT_LOGD] - 0.5 * log((double)M));
+    scal[PS_AMAX] = red[0];
     scal[PS_CSCALAR] = redi[0] ? 1.f : 0.f;
     scal[PS_CGAMMA] = (float)gamma;
-    scal[PS_GSHIFT] = bias + amax + lin - FS_MARGIN;
-    scal[PS_KAPPA] = kappa;
-    scal[PS_RHO2] = (float)rho2;
   }
 }
 

@@ -89,14 +89,42 @@ logits_kernel(const T* __restrict__ X, TensorAddr ax, int H, int L, int d, int M
   }
 }
 
-// ---- phi = exp(e - shift), one warp per row ------------------------------------------
+// Order-preserving map float -> unsigned, so that atomicMax on words gives the float maximum.
+__device__ __forceinline__ unsigned f2ord(float f) {
+  unsigned u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float ord2f(unsigned u) {
+  return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
+}
+
+// ---- largest exponent of each (batch, head) --------------------------------------------
 __global__ void __launch_bounds__(NTH)
-expshift_kernel(float* __restrict__ phi, int H, int L, int d, int M, int pool, int side, int stab,
-                const float* __restrict__ prep, float* __restrict__ logscale, int* __restrict__ status) {
+groupmax_kernel(const float* __restrict__ phi, int64_t per_bh, unsigned* __restrict__ gmax) {
+  __shared__ float red[NTH / 32];
+  const int bh = blockIdx.y;
+  const float* p = phi + (int64_t)bh * per_bh;
+  float mx = -3.0e38f;
+  for (int64_t e = blockIdx.x * (int64_t)NTH + threadIdx.x; e < per_bh; e += (int64_t)gridDim.x * NTH)
+    mx = fmaxf(mx, p[e]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int i = 1; i < NTH / 32; i++) mx = fmaxf(mx, red[i]);
+    atomicMax(&gmax[bh], f2ord(mx));
+  }
+}
+
+// ---- phi = exp(e - shift), one warp per row ------------------------------------------
+// shift: the row's largest exponent (ROW), the (batch, head)'s largest exponent (GROUP), or 0.
+__global__ void __launch_bounds__(NTH)
+expshift_kernel(float* __restrict__ phi, int L, int M, int stab, const unsigned* __restrict__ gmax,
+                float* __restrict__ logscale, int* __restrict__ status) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int bh = blockIdx.y;
-  PrepLayout pr{d, M};
-  const float gshift = prep[((size_t)group_of(bh, H, pool) * 2 + (side - 1)) * pr.total() + pr.scal() + PS_GSHIFT];
+  const float gshift = stab == FSHARP_STAB_GROUP ? ord2f(gmax[bh]) : 0.f;
   for (int i = blockIdx.x * 8 + warp; i < L; i += gridDim.x * 8) {
     float* row = phi + ((int64_t)bh * L + i) * M;
     float s = 0.f;
@@ -272,7 +300,8 @@ out_kernel(const float* __restrict__ phiQ, const float* __restrict__ KV, const f
 
 template <typename T>
 int featurize_t(fsharp_ctx* ctx, const void* X, TensorAddr ax, int B, int H, int L, int d, int M, int pool,
-                const float* prep, int side, float qk_scale, int stab, float* rowc, float* phi, float* logscale) {
+                const float* prep, int side, float qk_scale, int stab, float* rowc, unsigned* gmax, float* phi,
+                float* logscale) {
   const int BH = B * H;
   if (BH == 0 || L == 0) return FSHARP_OK;
   {
@@ -291,8 +320,15 @@ int featurize_t(fsharp_ctx* ctx, const void* X, TensorAddr ax, int B, int H, int
   {
     int gx = (L + 7) / 8;
     if (gx > 4 * ctx->sm_count) gx = 4 * ctx->sm_count;
-    expshift_kernel<<<dim3(gx, BH), NTH, 0, ctx->stream>>>(phi, H, L, d, M, pool, side, stab, prep, logscale,
-                                                          ctx->d_status);
+    if (stab == FSHARP_STAB_GROUP) {
+      FS_CUDA_OK(cudaMemsetAsync(gmax, 0, (size_t)BH * sizeof(unsigned), ctx->stream));
+      int64_t per_bh = (int64_t)L * M;
+      int gm = (int)((per_bh + 16 * NTH - 1) / (16 * NTH));
+      if (gm > 64) gm = 64;
+      groupmax_kernel<<<dim3(gm, BH), NTH, 0, ctx->stream>>>(phi, per_bh, gmax);
+      FS_LAUNCH_CHECK(ctx);
+    }
+    expshift_kernel<<<dim3(gx, BH), NTH, 0, ctx->stream>>>(phi, L, M, stab, gmax, logscale, ctx->d_status);
     FS_LAUNCH_CHECK(ctx);
   }
   return FSHARP_OK;
@@ -308,10 +344,11 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
   float* phiQ = ws->take<float>((size_t)BH * Lq * M);
   float* phiK = ws->take<float>((size_t)BH * Lk * M);
   float* rowc = ws->take<float>((size_t)BH * (Lq > Lk ? Lq : Lk));
-  FS_TRY(featurize_t<T>(ctx, K, ak, B, H, Lk, d, M, dm->pool, prep, 2, qk_scale, FSHARP_STAB_GROUP, rowc, phiK,
-                        nullptr));
-  FS_TRY(featurize_t<T>(ctx, Q, aq, B, H, Lq, d, M, dm->pool, prep, 1, qk_scale, FSHARP_STAB_ROW, rowc, phiQ,
-                        nullptr));
+  unsigned* gmax = ws->take<unsigned>((size_t)BH);
+  FS_TRY(featurize_t<T>(ctx, K, ak, B, H, Lk, d, M, dm->pool, prep, 2, qk_scale, FSHARP_STAB_GROUP, rowc, gmax,
+                        phiK, nullptr));
+  FS_TRY(featurize_t<T>(ctx, Q, aq, B, H, Lq, d, M, dm->pool, prep, 1, qk_scale, FSHARP_STAB_ROW, rowc, gmax,
+                        phiQ, nullptr));
   dim3 gout((Lq + TM - 1) / TM, (dv + TN - 1) / TN, BH);
   if (!causal) {
     float* KV = ws->take<float>((size_t)BH * M * N);
@@ -351,17 +388,19 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
 
 int fs_simt_featurize(fsharp_ctx* ctx, const void* X, int dtype, TensorAddr ax, int B, int H, int L, int d,
                       int M, int pool, const float* prep, int side, float qk_scale, int stab,
-                      float* rowc, float* phi, float* logscale) {
+                      float* rowc, unsigned* gmax, float* phi, float* logscale) {
   if (dtype == FSHARP_F32)
-    return featurize_t<float>(ctx, X, ax, B, H, L, d, M, pool, prep, side, qk_scale, stab, rowc, phi, logscale);
-  return featurize_t<__nv_bfloat16>(ctx, X, ax, B, H, L, d, M, pool, prep, side, qk_scale, stab, rowc, phi,
+    return featurize_t<float>(ctx, X, ax, B, H, L, d, M, pool, prep, side, qk_scale, stab, rowc, gmax, phi,
+                              logscale);
+  return featurize_t<__nv_bfloat16>(ctx, X, ax, B, H, L, d, M, pool, prep, side, qk_scale, stab, rowc, gmax, phi,
                                     logscale);
 }
 
 size_t fs_simt_attend_scratch_bytes(const fsharp_dims* dm, int causal, int chunk) {
   const size_t BH = (size_t)dm->B * dm->H, N = dm->dv + 1;
   const size_t Lmax = dm->Lq > dm->Lk ? dm->Lq : dm->Lk;
-  size_t b = ws_round(BH * dm->Lq * dm->M * 4) + ws_round(BH * dm->Lk * dm->M * 4) + ws_round(BH * Lmax * 4);
+  size_t b = ws_round(BH * dm->Lq * dm->M * 4) + ws_round(BH * dm->Lk * dm->M * 4) + ws_round(BH * Lmax * 4) +
+             ws_round(BH * 4);
   if (!causal) {
     b += ws_round(BH * dm->M * N * 4);
   } else {

@@ -1,5 +1,5 @@
 // Set statistics of Theorems 4.2 and 4.3: M1 = L^-1 sum x x^T, M2 = L^-1 sum y y^T,
-// mu4 = mean x, mu5 = mean y, plus the largest squared norms (overflow guard only).
+// mu4 = mean x, mu5 = mean y.
 //
 // One thread block accumulates the Gram matrix of a slice of tokens of one
 // (batch, head, side): products in fp32 over 128 tokens, then folded into fp64
@@ -39,7 +39,6 @@ stats_kernel(const T* __restrict__ Q, const T* __restrict__ K, TensorAddr aq, Te
     for (int j = 0; j < RB; j++) { acc[i][j] = 0.f; accd[i][j] = 0.0; }
   float colacc = 0.f;
   double colaccd = 0.0;
-  float rho2 = 0.f;
   bool bad = false;
   int since = 0;
 
@@ -67,12 +66,6 @@ stats_kernel(const T* __restrict__ Q, const T* __restrict__ K, TensorAddr aq, Te
       for (int t = 0; t < ST_TT; t++) s += xs[t][tid];
       colacc += s;
     }
-    if (tid >= ST_THREADS - ST_TT) {
-      int t = tid - (ST_THREADS - ST_TT);
-      float s = 0.f;
-      for (int c = 0; c < D; c++) s = fmaf(xs[t][c], xs[t][c], s);
-      rho2 = fmaxf(rho2, s);
-    }
     __syncthreads();
     if (++since == ST_FLUSH) {
       since = 0;
@@ -94,11 +87,6 @@ stats_kernel(const T* __restrict__ Q, const T* __restrict__ K, TensorAddr aq, Te
     for (int j = 0; j < RB; j++)
       atomicAdd(&Mo[(size_t)(ty + 16 * i) * D + (tx + 16 * j)], (accd[i][j] + (double)acc[i][j]) * inv);
   if (tid < D) atomicAdd(&out[sl.mu(side + 4) + tid], (colaccd + (double)colacc) * inv);
-  if (tid >= ST_THREADS - ST_TT) {
-    // non-negative doubles order like their bit patterns
-    atomicMax(reinterpret_cast<unsigned long long*>(&out[sl.rho2(side + 1)]),
-              (unsigned long long)__double_as_longlong((double)rho2));
-  }
   if (bad) atomicExch(status, FSHARP_E_NONFINITE);
 }
 

@@ -17,7 +17,10 @@ def dev(a, dtype="f32"):
 
 
 def host(t):
-    return t.detach().float().cpu().numpy().astype(np.float64)
+    t = t.detach()
+    if t.dtype != torch.float64:
+        t = t.float()
+    return t.cpu().numpy().astype(np.float64)
 
 
 def rel_err(got, ref):

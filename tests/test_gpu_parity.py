@@ -51,8 +51,6 @@ def test_stats_match_definition(ctx, w):
             assert np.abs(M2 - ref["M2"]).max() < 2e-6 * scale
             assert np.abs(g[2 * d * d: 2 * d * d + d] - ref["mu4"]).max() < 2e-6
             assert np.abs(g[2 * d * d + d: 2 * d * d + 2 * d] - ref["mu5"]).max() < 2e-6
-            assert abs(g[-2] / np.max(np.sum(Q[b, h].astype(np.float64) ** 2, axis=1)) - 1) < 1e-5
-            assert abs(g[-1] / np.max(np.sum(K[b, h].astype(np.float64) ** 2, axis=1)) - 1) < 1e-5
 
 
 def test_stats_pooled_over_batch_and_strided(ctx):
@@ -109,7 +107,6 @@ def test_fit_from_exact_statistics(ctx, variant, d):
         blob[g, d * d: 2 * d * d] = st["M2"].ravel()
         blob[g, 2 * d * d: 2 * d * d + d] = st["mu4"]
         blob[g, 2 * d * d + d: 2 * d * d + 2 * d] = st["mu5"]
-        blob[g, -2:] = [np.max(np.sum(X * X, 1)), np.max(np.sum(Y * Y, 1))]
         refs.append(fs.FITS[variant](st))
     pr = ctx.fsharp_fit_params(torch.from_numpy(blob).cuda(), d, variant)
     assert ctx.status() == 0
@@ -124,10 +121,6 @@ def test_fit_from_exact_statistics(ctx, variant, d):
         if variant == "sderf":
             a = np.diag(p["A"])
             assert np.all(np.diff(a) >= -1e-15)          # eigenvalues of N non-ascending
-        # the guard constants are true lower bounds
-        for k in (1, 2):
-            lam_min = np.linalg.eigvalsh(-p[f"C{k}"]).min()
-            assert p[f"kappa{k}"] <= lam_min * (1 + 1e-9) + 1e-15
 
 
 @pytest.mark.parametrize("w", small_cases()[:5], ids=lambda w: w.name)
@@ -162,7 +155,7 @@ def test_featurize_matches_definition(ctx, w, stab):
                     assert phi[b, h].max() <= 1.0 + 1e-6
                 elif stab == fb.STAB_GROUP:
                     shift = host(ls)[b, h]
-                    assert np.all(ref - shift <= 40.0 + 1e-3)   # the bound holds with its headroom
+                    assert abs(shift - ref.max()) < 1e-4 * max(1.0, abs(ref.max()))   # the exact maximum
                 else:
                     shift = 0.0
                 got = phi[b, h]
@@ -214,7 +207,9 @@ def test_attend_properties(ctx):
     dK2[:, :, 300:] *= 1.5
     dV2[:, :, 300:] += 1.0
     Yb = host(ctx.fsharp_attend(dQ, dK2, dV2, dOm, pr, causal=True, chunk=128))
-    assert np.abs(Ya[:, :, :300] - Yb[:, :, :300]).max() == 0.0
+    # (the keys' common shift is taken over the whole sequence, so only rounding may differ)
+    assert np.abs(Ya[:, :, :300] - Yb[:, :, :300]).max() <= 2.0 ** -7
+    assert np.abs(Ya[:, :, 300:] - Yb[:, :, 300:]).max() > 0.1
     for ch in (64, 256):
         Yc = host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=True, chunk=ch))
         assert rel_err(Yc, Ya) < 1e-2
