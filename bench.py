@@ -1,0 +1,345 @@
+"""Benchmark of the FAVOR# hot path: one step = statistics -> fit -> prep -> featurize ->
+contraction over one batch of synthetic input.  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg3b|cfg5]
+  python bench.py --impl reference ...     times the fp64 CPU checker instead (bounded sample)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "FAVOR# attention tokens/sec/GPU and % of roofline (fwd, bidirectional + causal)"
+UNIT = "tokens/s"
+
+
+def algorithmic_work(w):
+    """Per step, over all (batch, head) units: flops and HBM bytes of the attend stage counted on
+    the method's own sizes (no padding, no L^2 work), and the exponentials."""
+    units = w.B * w.H
+    L, d, dv, M = w.L, w.d, w.dv, w.M
+    feat = 2 * 2 * L * d * M                       # X W^T for queries and keys
+    if w.variant == "aderf":
+        feat += 2 * 2 * L * d * d                  # dense x^T C x per token
+    contr = 2 * 2 * L * M * (dv + 1)               # S^T [V|1] and P (S^T [V|1])
+    if w.causal:
+        contr += L * w.chunk * M + L * w.chunk * (dv + 1)   # triangular halves of the in-chunk products
+    es = 2 if w.dtype == "bf16" else 4
+    bytes_ = (2 * L * d + 2 * L * dv) * es
+    return {"flops": units * (feat + contr), "bytes": units * bytes_, "exps": units * 2 * L * M}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) during the timed region."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.stop_flag = index, [], set(), False
+        self.max_mhz = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {"hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown if hasattr(nv, "nvmlClocksEventReasonHwSlowdown") else 0x8,
+                 "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
+        while not self.stop_flag:
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def result(self):
+        s = sorted(self.samples)
+        return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def physical_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def oracle_units(w, Q, K, V, Om, units):
+    """The checker's whole path for the given (b, h) units; returns seconds."""
+    from oracle import favor_sharp as fs
+    t0 = time.perf_counter()
+    for u in units:
+        b, h = divmod(u, w.H)
+        p = fs.fit_params(Q[b, h], K[b, h], w.variant)
+        fs.favor_sharp_attention(Q[b, h], K[b, h], V[b, h], Om, p, causal=False) if not w.causal else \
+            fs.attend_causal_recurrent(*fs.features_pair(Q[b, h].astype(np.float64), K[b, h].astype(np.float64), Om, p), V[b, h])
+    return time.perf_counter() - t0
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info()]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, w):
+    """The fp64 CPU checker as it stands, on host cores; each step is a bounded sample."""
+    from paper_2302_00787_b200 import workloads as wl
+    from paper_2302_00787_b200.sharding import env_rank_world
+    rank, _, world = env_rank_world()
+    if rank != 0:
+        return
+    n_units = max(1, min(w.B * w.H, args.ref_units))
+    ws = w.scaled(B=1, H=n_units)
+    Q, K, V = wl.make_qkv(ws)
+    Om = wl.make_omega(ws)
+    for _ in range(args.warmup):
+        oracle_units(ws, Q, K, V, Om, range(1))
+    t = 0.0
+    for _ in range(args.steps):
+        t += oracle_units(ws, Q, K, V, Om, range(n_units))
+    head_tokens = args.steps * n_units * w.L
+    value = head_tokens / w.H / t
+    cores = cpu_threads()
+    sample = f"{n_units} of {w.B * w.H} (batch, head) units of {w.name} per step (statistics, fit, features, contraction)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "L": w.L, "d": w.d, "dv": w.dv, "M": w.M,
+                   "variant": w.variant, "causal": w.causal, "chunk": w.chunk},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--ref-units", type=int, default=2)
+    ap.add_argument("--buffers", type=int, default=3, help="input sets rotated so that a step's inputs are cold in L2")
+    ap.add_argument("--cpu-baseline-seconds", type=float, default=12.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel-impl", default="auto", choices=["auto", "simt", "tensor"])
+    args = ap.parse_args()
+
+    from paper_2302_00787_b200 import workloads as wl
+    w = wl.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2302_00787_b200 import binding as fb
+    from paper_2302_00787_b200.sharding import env_rank_world, max_over_ranks, rank_seed
+
+    rank, local_rank, world = env_rank_world()
+    if args.warmup < 3:
+        args.warmup = 3
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    w_rank = w.scaled(seed=rank_seed(w.seed, rank))
+    td = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+
+    # inputs: `buffers` independent draws resident in HBM, rotated step by step
+    sets = []
+    host_set = None
+    for i in range(args.buffers):
+        wi = w_rank.scaled(seed=w_rank.seed + i)
+        Q, K, V = wl.make_qkv(wi)
+        if i == 0:
+            host_set = (Q, K, V)
+        sets.append(tuple(torch.from_numpy(a).to(dev).to(td) for a in (Q, K, V)))
+    Om = wl.make_omega(w_rank)
+    dOm = torch.from_numpy(Om).to(dev)
+    G = w.B * w.H
+    ctx = fb.Context(local_rank)
+    ctx.set_impl({"auto": fb.IMPL_AUTO, "simt": fb.IMPL_SIMT, "tensor": fb.IMPL_TENSOR}[args.kernel_impl])
+    st = torch.empty(G, fb.stats_doubles(w.d), dtype=torch.float64, device=dev)
+    pr = torch.empty(G, fb.params_doubles(w.d), dtype=torch.float64, device=dev)
+    Y = torch.empty(w.B, w.H, w.L, w.dv, dtype=td, device=dev)
+
+    def step(i):
+        dQ, dK, dV = sets[i % len(sets)]
+        ctx.fsharp_stats(dQ, dK, out=st)
+        ctx.fsharp_fit_params(st, w.d, w.variant, out=pr)
+        ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=w.causal, chunk=w.chunk, out=Y)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    assert ctx.status() == 0, "device status after warm-up"
+    sampler = ClockSampler(physical_index(local_rank))
+    barrier()
+    sampler.start()
+    n0 = ctx.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = ctx.launch_count() - n0
+    # same loop once more with an event pair around every launch: per-kernel device time
+    ctx.set_timing(True)
+    ksteps = max(1, min(args.steps, 4096 // max(1, launches // args.steps)))
+    for i in range(ksteps):
+        step(i)
+    per_kernel = ctx.read_timing()
+    ctx.set_timing(False)
+    sampler.stop_flag = True
+    sampler.join(timeout=2)
+    assert ctx.status() == 0, "device status after the timed region"
+    ms = max_over_ranks(ms, dev)
+
+    # end to end through the host-buffer entry point (pinned host memory; copies inside the timing)
+    hQ, hK, hV = (torch.from_numpy(a).to(td).pin_memory() for a in host_set)
+    hOm = torch.from_numpy(Om).pin_memory()
+    hY = torch.empty(w.B, w.H, w.L, w.dv, dtype=td).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(3):
+        ctx.fsharp_forward_host(hQ, hK, hV, hOm, w.variant, causal=w.causal, chunk=w.chunk, out=hY)
+    barrier()
+    t0 = time.perf_counter()
+    e0.record()
+    for _ in range(e2e_steps):
+        ctx.fsharp_forward_host(hQ, hK, hV, hOm, w.variant, causal=w.causal, chunk=w.chunk, out=hY)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0))
+    e2e_ms = max_over_ranks(e2e_ms, dev)
+    es = 2 if w.dtype == "bf16" else 4
+    h2d = (hQ.numel() + hK.numel() + hV.numel()) * es + hOm.numel() * 4
+    d2h = hY.numel() * es
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    tokens_per_step = world * w.B * w.L
+    value = tokens_per_step * args.steps / (ms * 1e-3)
+    work = algorithmic_work(w)
+    peaks = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+    pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pk):
+        j = json.load(open(pk))
+        peaks = {"hbm_gbs": j["hbm_gbs"], "bf16_tflops": j["bf16_tflops_sustained"], "source": "measured (sustained)"}
+    # dominant kernel of the step and its roofline
+    tot = sum(v[0] for v in per_kernel.values()) or 1.0
+    kernels = {k: {"ms_per_launch": v[0] / v[1], "launches_per_step": v[1] / ksteps, "share": v[0] / tot}
+               for k, v in sorted(per_kernel.items(), key=lambda kv: -kv[1][0])}
+    dom = next(iter(kernels))
+    roof = roofline_for(dom, kernels[dom], w, work, peaks)
+    attend_ms = sum(v[0] for k, v in per_kernel.items() if k not in ("stats_kernel", "fit_kernel")) / ksteps
+    t_roof = max(work["flops"] / (peaks["bf16_tflops"] * 1e12), work["bytes"] / (peaks["hbm_gbs"] * 1e9))
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "L": w.L, "d": w.d, "dv": w.dv, "M": w.M,
+                   "variant": w.variant, "causal": w.causal, "chunk": w.chunk, "kernel_impl": args.kernel_impl,
+                   "l2": f"inputs rotate over {len(sets)} resident sets ({len(sets) * work['bytes'] / 1e6:.0f} MB > 126 MB L2)",
+                   "step": "stats + fit + prep + featurize + contraction"},
+        "clocks": sampler.result(),
+        "e2e": {"value": tokens_per_step * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches,
+        "roofline": roof,
+        "attend": {"ms": attend_ms, "tokens_per_s": w.B * w.L / (attend_ms * 1e-3),
+                   "algorithmic_tflops": work["flops"] / (attend_ms * 1e-3) / 1e12,
+                   "algorithmic_gbs": work["bytes"] / (attend_ms * 1e-3) / 1e9,
+                   "gexp_per_s": work["exps"] / (attend_ms * 1e-3) / 1e9,
+                   "roofline_frac": t_roof * 1e3 / attend_ms, "peaks": peaks},
+        "kernels": kernels,
+    }
+    if not args.no_cpu_baseline:
+        Q, K, V = host_set
+        n, t = 0, 0.0
+        while t < args.cpu_baseline_seconds and n < G:
+            t += oracle_units(w, Q, K, V, Om, [n])
+            n += 1
+        out["cpu_baseline"] = {"value": n * w.L / w.H / t, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                               "sample": f"{n} of {G} (batch, head) units of {w.name}: statistics, fit, features, contraction"}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def roofline_for(name, k, w, work, peaks):
+    """Roofline entry for the step's dominant kernel.  Algorithmic work per launch:
+    tensor-bound kernels carry their share of the attend flops; the rest are judged on bytes."""
+    units = w.B * w.H
+    L, d, dv, M = w.L, w.d, w.dv, w.M
+    es = 2 if w.dtype == "bf16" else 4
+    per_launch = 1.0 / max(k["launches_per_step"], 1e-9)
+    t = k["ms_per_launch"] * 1e-3
+    flops_of = {
+        "logits_kernel": 2 * L * d * M * units, "kv_kernel": 2 * L * M * (dv + 1) * units,
+        "out_kernel": 2 * L * M * (dv + 1) * units, "scores_kernel": L * w.chunk * M * units if w.causal else 0,
+        "tc_kv_kernel": (2 * L * d * M + 2 * L * M * (dv + 1)) * units,
+        "tc_out_kernel": (2 * L * d * M + 2 * L * M * (dv + 1)) * units,
+        "tc_causal_out_kernel": work["flops"], "tc_causal_state_kernel": (2 * L * d * M + 2 * L * M * (dv + 1)) * units,
+    }
+    bytes_of = {"stats_kernel": 2 * L * d * es * units, "expshift_kernel": 2 * L * M * 4 * units,
+                "rowterm_kernel": L * d * es * units, "groupmax_kernel": L * M * 4 * units}
+    if name in flops_of and flops_of[name]:
+        fl = flops_of[name] * (per_launch if name in ("logits_kernel", "kv_kernel", "out_kernel", "scores_kernel") and
+                               k["launches_per_step"] > 1 else 1.0)
+        ach = fl / t / 1e12
+        return {"kernel": name, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": ach / peaks["bf16_tflops"], "traffic": None, "peak_source": peaks["source"]}
+    if name == "fit_kernel":
+        return {"kernel": name, "bound": "alu", "achieved": None, "peak": None, "unit": "TFLOP/s", "frac": None,
+                "traffic": None, "note": "latency-bound fp64 Jacobi sweeps, one block per group"}
+    by = bytes_of.get(name, work["bytes"]) * (per_launch if k["launches_per_step"] > 1 else 1.0)
+    ach = by / t / 1e9
+    return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
+
+
+if __name__ == "__main__":
+    main()

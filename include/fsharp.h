@@ -95,6 +95,15 @@ int fsharp_set_impl(fsharp_ctx* ctx, int impl);
 int fsharp_status(fsharp_ctx* ctx, int* code);
 /* Number of kernels this context has launched since creation. */
 int64_t fsharp_launch_count(const fsharp_ctx* ctx);
+/* Per-kernel device times.  While timing is on, every launch of this context is
+ * bracketed by a pair of CUDA events on the context's stream (up to 4096 launches
+ * between two reads).  fsharp_read_timing synchronises the stream and returns, for
+ * kernel ids 0..cap-1, the summed milliseconds and the launch count since the last
+ * read (host arrays of `cap` entries); fsharp_kernel_name maps an id to the kernel's
+ * name ("" for unused ids).  Ids are below 32. */
+int fsharp_set_timing(fsharp_ctx* ctx, int on);
+int fsharp_read_timing(fsharp_ctx* ctx, int cap, float* total_ms, int* launches);
+const char* fsharp_kernel_name(int id);
 /* Bytes of scratch the context currently holds. */
 size_t fsharp_workspace_bytes(const fsharp_ctx* ctx);
 const char* fsharp_strerror(int code);

@@ -22,7 +22,8 @@ EXPORTS = [
     "fsharp_create", "fsharp_destroy", "fsharp_set_stream", "fsharp_set_impl", "fsharp_status",
     "fsharp_launch_count", "fsharp_workspace_bytes", "fsharp_strerror", "fsharp_stats_doubles",
     "fsharp_params_doubles", "fsharp_stats", "fsharp_fit_params", "fsharp_featurize", "fsharp_attend",
-    "fsharp_forward_host", "fsharp_pair_estimate",
+    "fsharp_forward_host", "fsharp_pair_estimate", "fsharp_set_timing", "fsharp_read_timing",
+    "fsharp_kernel_name",
 ]
 
 
@@ -72,6 +73,9 @@ def load_library() -> C.CDLL:
         "fsharp_attend": (i32, [vp, vp, vp, vp, vp, vp, dims_p, i32, i32, i32, f32, vp]),
         "fsharp_forward_host": (i32, [vp, vp, vp, vp, vp, dims_p, i32, i32, i32, i32, f32, vp]),
         "fsharp_pair_estimate": (i32, [vp, vp, vp, vp, vp, i64, i32, i32, i32, vp, vp]),
+        "fsharp_set_timing": (i32, [vp, i32]),
+        "fsharp_read_timing": (i32, [vp, i32, C.POINTER(C.c_float), C.POINTER(i32)]),
+        "fsharp_kernel_name": (C.c_char_p, [i32]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -164,6 +168,21 @@ class Context:
 
     def workspace_bytes(self) -> int:
         return self.lib.fsharp_workspace_bytes(self._h)
+
+    def set_timing(self, on: bool):
+        _check(self.lib.fsharp_set_timing(self._h, int(on)), "fsharp_set_timing")
+
+    def read_timing(self) -> dict:
+        """{kernel name: (total milliseconds, launches)} since the last read."""
+        cap = 32
+        ms = (C.c_float * cap)()
+        n = (C.c_int * cap)()
+        _check(self.lib.fsharp_read_timing(self._h, cap, ms, n), "fsharp_read_timing")
+        out = {}
+        for i in range(cap):
+            if n[i]:
+                out[self.lib.fsharp_kernel_name(i).decode()] = (float(ms[i]), int(n[i]))
+        return out
 
     # -- the path
     def fsharp_stats(self, Q, K, pool=POOL_PER_BH, qk_scale=1.0, out=None):

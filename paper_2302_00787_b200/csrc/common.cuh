@@ -45,6 +45,15 @@ struct PrepLayout {
 // PS_BIAS logD - 1/2 log M; PS_AMAX max_m a_m; PS_CSCALAR 1 if C = gamma I; PS_CGAMMA gamma.
 enum { PS_BIAS = 0, PS_AMAX = 1, PS_CSCALAR = 3, PS_CGAMMA = 4 };
 
+// Kernel ids for the optional per-kernel timing (fsharp_set_timing / fsharp_read_timing).
+enum {
+  FS_K_STATS = 1, FS_K_FIT, FS_K_PREP, FS_K_ROWTERM, FS_K_LOGITS, FS_K_GROUPMAX, FS_K_EXPSHIFT, FS_K_KV,
+  FS_K_PREFIX, FS_K_SCORES, FS_K_OUT, FS_K_PAIRS, FS_K_PAIRVAR_PREP, FS_K_PAIRVAR,
+  FS_K_TC_KV, FS_K_TC_MERGE, FS_K_TC_OUT, FS_K_TC_CAUSAL_STATE, FS_K_TC_CAUSAL_PREFIX, FS_K_TC_CAUSAL_OUT,
+  FS_K_COUNT
+};
+constexpr int FS_TIMING_SLOTS = 4096;
+
 struct fsharp_ctx {
   int device;
   cudaStream_t stream;
@@ -54,7 +63,17 @@ struct fsharp_ctx {
   int* d_status;      // device status word
   int64_t launches;
   int sm_count;
+  // timing: pairs of events around each launch while enabled
+  int timing;
+  int t_used;
+  cudaEvent_t* t_ev;  // 2 * FS_TIMING_SLOTS, created on first use
+  int* t_tag;
 };
+
+void fs_time_begin(fsharp_ctx* ctx, int tag);
+void fs_time_end(fsharp_ctx* ctx);
+#define FS_TIME_BEGIN(ctx, tag) do { if ((ctx)->timing) fs_time_begin((ctx), (tag)); } while (0)
+#define FS_TIME_END(ctx) do { if ((ctx)->timing) fs_time_end((ctx)); } while (0)
 
 // Bump allocator over the context workspace.
 struct WsAlloc {

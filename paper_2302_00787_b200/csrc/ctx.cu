@@ -24,6 +24,10 @@ int fsharp_create(fsharp_ctx** out, int device, void* stream) {
   c->launches = 0;
   c->d_status = nullptr;
   c->sm_count = 148;
+  c->timing = 0;
+  c->t_used = 0;
+  c->t_ev = nullptr;
+  c->t_tag = nullptr;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) == cudaSuccess) c->sm_count = prop.multiProcessorCount;
   if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess) {
@@ -47,6 +51,11 @@ int fsharp_destroy(fsharp_ctx* ctx) {
   cudaStreamSynchronize(ctx->stream);
   if (ctx->ws) cudaFree(ctx->ws);
   if (ctx->d_status) cudaFree(ctx->d_status);
+  if (ctx->t_ev) {
+    for (int i = 0; i < 2 * FS_TIMING_SLOTS; i++) cudaEventDestroy(ctx->t_ev[i]);
+    delete[] ctx->t_ev;
+    delete[] ctx->t_tag;
+  }
   delete ctx;
   return FSHARP_OK;
 }
@@ -93,10 +102,77 @@ const char* fsharp_strerror(int code) {
   }
 }
 
+int fsharp_set_timing(fsharp_ctx* ctx, int on) {
+  if (!ctx) return FSHARP_E_BADARG;
+  if (on && !ctx->t_ev) {
+    FS_CUDA_OK(cudaSetDevice(ctx->device));
+    ctx->t_ev = new (std::nothrow) cudaEvent_t[2 * FS_TIMING_SLOTS];
+    ctx->t_tag = new (std::nothrow) int[FS_TIMING_SLOTS];
+    if (!ctx->t_ev || !ctx->t_tag) return FSHARP_E_NOMEM;
+    for (int i = 0; i < 2 * FS_TIMING_SLOTS; i++) FS_CUDA_OK(cudaEventCreate(&ctx->t_ev[i]));
+  }
+  ctx->timing = on ? 1 : 0;
+  ctx->t_used = 0;
+  return FSHARP_OK;
+}
+
+int fsharp_read_timing(fsharp_ctx* ctx, int cap, float* total_ms, int* launches) {
+  if (!ctx || !total_ms || !launches || cap <= 0) return FSHARP_E_BADARG;
+  for (int i = 0; i < cap; i++) { total_ms[i] = 0.f; launches[i] = 0; }
+  if (!ctx->t_ev) return FSHARP_OK;
+  FS_CUDA_OK(cudaStreamSynchronize(ctx->stream));
+  for (int i = 0; i < ctx->t_used; i++) {
+    float ms = 0.f;
+    FS_CUDA_OK(cudaEventElapsedTime(&ms, ctx->t_ev[2 * i], ctx->t_ev[2 * i + 1]));
+    int tag = ctx->t_tag[i];
+    if (tag >= 0 && tag < cap) { total_ms[tag] += ms; launches[tag]++; }
+  }
+  ctx->t_used = 0;
+  return FSHARP_OK;
+}
+
+const char* fsharp_kernel_name(int id) {
+  switch (id) {
+    case FS_K_STATS: return "stats_kernel";
+    case FS_K_FIT: return "fit_kernel";
+    case FS_K_PREP: return "prep_kernel";
+    case FS_K_ROWTERM: return "rowterm_kernel";
+    case FS_K_LOGITS: return "logits_kernel";
+    case FS_K_GROUPMAX: return "groupmax_kernel";
+    case FS_K_EXPSHIFT: return "expshift_kernel";
+    case FS_K_KV: return "kv_kernel";
+    case FS_K_PREFIX: return "prefix_kernel";
+    case FS_K_SCORES: return "scores_kernel";
+    case FS_K_OUT: return "out_kernel";
+    case FS_K_PAIRS: return "pairs_kernel";
+    case FS_K_PAIRVAR_PREP: return "pairvar_prep_kernel";
+    case FS_K_PAIRVAR: return "pairvar_kernel";
+    case FS_K_TC_KV: return "tc_kv_kernel";
+    case FS_K_TC_MERGE: return "tc_merge_kernel";
+    case FS_K_TC_OUT: return "tc_out_kernel";
+    case FS_K_TC_CAUSAL_STATE: return "tc_causal_state_kernel";
+    case FS_K_TC_CAUSAL_PREFIX: return "tc_causal_prefix_kernel";
+    case FS_K_TC_CAUSAL_OUT: return "tc_causal_out_kernel";
+    default: return "";
+  }
+}
+
 size_t fsharp_stats_doubles(int d) { return StatsLayout{d}.total(); }
 size_t fsharp_params_doubles(int d) { return ParamsLayout{d}.total(); }
 
 }  // extern "C"
+
+void fs_time_begin(fsharp_ctx* ctx, int tag) {
+  if (ctx->t_used >= FS_TIMING_SLOTS) return;
+  ctx->t_tag[ctx->t_used] = tag;
+  cudaEventRecord(ctx->t_ev[2 * ctx->t_used], ctx->stream);
+}
+
+void fs_time_end(fsharp_ctx* ctx) {
+  if (ctx->t_used >= FS_TIMING_SLOTS) return;
+  cudaEventRecord(ctx->t_ev[2 * ctx->t_used + 1], ctx->stream);
+  ctx->t_used++;
+}
 
 int fs_ws_reserve(fsharp_ctx* ctx, size_t bytes) {
   if (bytes <= ctx->ws_bytes) return FSHARP_OK;

@@ -345,7 +345,9 @@ int fs_run_fit(fsharp_ctx* ctx, const double* stats, int G, int d, int variant, 
   a.status = ctx->d_status;
   size_t smem = fit_smem_bytes(d, a.v_in_smem);
   FS_CUDA_OK(cudaFuncSetAttribute(fit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  FS_TIME_BEGIN(ctx, FS_K_FIT);
   fit_kernel<<<G, FIT_THREADS, smem, ctx->stream>>>(a);
+  FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;
 }

@@ -162,14 +162,20 @@ int fs_run_pairs(fsharp_ctx* ctx, const float* X, const float* Y, const float* O
   if (npairs == 0) return FSHARP_OK;
   int64_t tiles = (npairs + TM - 1) / TM;
   if (tiles > 2147483647LL) return FSHARP_E_SHAPE;
+  FS_TIME_BEGIN(ctx, FS_K_PAIRS);
   pairs_kernel<<<dim3((unsigned)tiles, R), NTH, 0, ctx->stream>>>(X, Y, npairs, d, M, prep, est);
+  FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   if (var_cf) {
+    FS_TIME_BEGIN(ctx, FS_K_PAIRVAR_PREP);
     pairvar_prep_kernel<<<1, NTH, 0, ctx->stream>>>(params, d, ev, ctx->d_status);
+    FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
     int64_t blocks = (npairs + 7) / 8;
     if (blocks > 8 * ctx->sm_count) blocks = 8 * ctx->sm_count;
+    FS_TIME_BEGIN(ctx, FS_K_PAIRVAR);
     pairvar_kernel<<<(unsigned)blocks, NTH, 0, ctx->stream>>>(X, Y, npairs, d, M, ev, var_cf);
+    FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
   }
   return FSHARP_OK;

@@ -76,8 +76,10 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
 int fs_run_prep(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_stride, const double* params,
                 int64_t params_stride, int G, int H, int pool, int d, int M, float* prep) {
   if (G == 0) return FSHARP_OK;
+  FS_TIME_BEGIN(ctx, FS_K_PREP);
   prep_kernel<<<dim3(G, 2), PREP_THREADS, 0, ctx->stream>>>(Omega, omega_head_stride, params, params_stride, H, pool, d, M,
                                                                  prep);
+  FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;
 }

@@ -310,12 +310,16 @@ int featurize_t(fsharp_ctx* ctx, const void* X, TensorAddr ax, int B, int H, int
     // shared memory: dense C (d*d) + one x per warp; sized for the dense case
     size_t smem = ((size_t)d * d + 8 * (size_t)d) * sizeof(float);
     FS_CUDA_OK(cudaFuncSetAttribute(rowterm_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    FS_TIME_BEGIN(ctx, FS_K_ROWTERM);
     rowterm_kernel<T><<<dim3(gx, BH), NTH, smem, ctx->stream>>>((const T*)X, ax, H, L, d, M, pool, side, prep,
                                                                qk_scale, rowc);
+    FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
   }
+  FS_TIME_BEGIN(ctx, FS_K_LOGITS);
   logits_kernel<T><<<dim3((L + TM - 1) / TM, (M + TN - 1) / TN, BH), NTH, 0, ctx->stream>>>(
       (const T*)X, ax, H, L, d, M, pool, side, prep, qk_scale, rowc, phi);
+  FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   {
     int gx = (L + 7) / 8;
@@ -325,10 +329,14 @@ int featurize_t(fsharp_ctx* ctx, const void* X, TensorAddr ax, int B, int H, int
       int64_t per_bh = (int64_t)L * M;
       int gm = (int)((per_bh + 16 * NTH - 1) / (16 * NTH));
       if (gm > 64) gm = 64;
+      FS_TIME_BEGIN(ctx, FS_K_GROUPMAX);
       groupmax_kernel<<<dim3(gm, BH), NTH, 0, ctx->stream>>>(phi, per_bh, gmax);
+      FS_TIME_END(ctx);
       FS_LAUNCH_CHECK(ctx);
     }
+    FS_TIME_BEGIN(ctx, FS_K_EXPSHIFT);
     expshift_kernel<<<dim3(gx, BH), NTH, 0, ctx->stream>>>(phi, L, M, stab, gmax, logscale, ctx->d_status);
+    FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
   }
   return FSHARP_OK;
@@ -359,26 +367,38 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
     if (nsl < 1) nsl = 1;
     int slen = (Lk + nsl - 1) / nsl;
     nsl = (Lk + slen - 1) / slen;
+    FS_TIME_BEGIN(ctx, FS_K_KV);
     kv_kernel<T><<<dim3((M + TM - 1) / TM, (N + TN - 1) / TN, BH * nsl), NTH, 0, ctx->stream>>>(
         phiK, (const T*)V, av, H, Lk, M, dv, slen, nsl, 0, KV);
+    FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
+    FS_TIME_BEGIN(ctx, FS_K_OUT);
     out_kernel<T><<<gout, NTH, 0, ctx->stream>>>(phiQ, KV, nullptr, (const T*)V, av, (T*)Y, ay, H, Lq, M, dv, 0, 0,
                                                 1, ctx->d_status);
+    FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
   } else {
     const int C = chunk, nch = Lq / C;
     float* st = ws->take<float>((size_t)BH * nch * M * N);
     float* sc = ws->take<float>((size_t)BH * nch * C * C);
+    FS_TIME_BEGIN(ctx, FS_K_KV);
     kv_kernel<T><<<dim3((M + TM - 1) / TM, (N + TN - 1) / TN, BH * nch), NTH, 0, ctx->stream>>>(
         phiK, (const T*)V, av, H, Lk, M, dv, C, nch, 1, st);
+    FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
     int64_t elems = (int64_t)M * N;
+    FS_TIME_BEGIN(ctx, FS_K_PREFIX);
     prefix_kernel<<<dim3((unsigned)((elems + NTH - 1) / NTH), BH), NTH, 0, ctx->stream>>>(st, nch, elems);
+    FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
+    FS_TIME_BEGIN(ctx, FS_K_SCORES);
     scores_kernel<<<dim3(C / TM, C / TN, BH * nch), NTH, 0, ctx->stream>>>(phiQ, phiK, Lq, M, C, nch, sc);
+    FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
+    FS_TIME_BEGIN(ctx, FS_K_OUT);
     out_kernel<T><<<gout, NTH, 0, ctx->stream>>>(phiQ, st, sc, (const T*)V, av, (T*)Y, ay, H, Lq, M, dv, 1, C, nch,
                                                 ctx->d_status);
+    FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
   }
   return FSHARP_OK;

@@ -110,6 +110,7 @@ int launch_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dim
   stats_kernel<T, DD><<<grid, ST_THREADS, 0, ctx->stream>>>((const T*)Q, (const T*)K, aq, ak, dm->H, dm->Lq, \
                                                             dm->Lk, dm->pool, Bpool, qk_scale, tps, stats,   \
                                                             ctx->d_status)
+  FS_TIME_BEGIN(ctx, FS_K_STATS);
   switch (dm->d) {
     case 16: FS_ST(16); break;
     case 32: FS_ST(32); break;
@@ -118,6 +119,7 @@ int launch_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dim
     default: return FSHARP_E_SHAPE;
   }
 #undef FS_ST
+  FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;
 }
