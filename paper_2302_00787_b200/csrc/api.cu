@@ -7,7 +7,7 @@
 int fs_tc_supported(const fsharp_dims* dm, int dtype, int causal, int chunk, float qk_scale);
 size_t fs_tc_attend_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm, int causal, int chunk);
 int fs_tc_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, int causal,
-                 int chunk, const float* prep, void* Y, WsAlloc* ws);
+                 int chunk, float qk_scale, const float* prep, void* Y, WsAlloc* ws);
 
 namespace {
 
@@ -125,7 +125,7 @@ int fsharp_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, 
   float* prep = ws.take<float>(prep_f);
   FS_TRY(fs_run_prep(ctx, Omega, dims->omega_head_stride, params, (int64_t)ParamsLayout{dims->d}.total(), G,
                      dims->H, dims->pool, dims->d, dims->M, prep));
-  if (use_tc) return fs_tc_attend(ctx, Q, K, V, dims, causal, chunk, prep, Y, &ws);
+  if (use_tc) return fs_tc_attend(ctx, Q, K, V, dims, causal, chunk, qk_scale, prep, Y, &ws);
   return fs_simt_attend(ctx, Q, K, V, dims, dtype, causal, chunk, qk_scale, prep, Y, &ws);
 }
 

@@ -1,0 +1,615 @@
+// Tensor-core path, bidirectional attention (Sections 2.1 / 2.2) for bf16, d = dv = 64, M = 256.
+//
+//   key side   (tc_kv_kernel):  per 128-key tile   logits = Y W2^T + a      (tcgen05, TMEM)
+//                               phi = 2^(logits + c_j - s)  -> bf16 tile in shared memory
+//                               KV += phi^T [V | 1]                          (tcgen05, TMEM)
+//   merge      (tc_merge_kernel): partial KV of the splits of one (batch, head), brought to a
+//                               common shift, summed, written transposed in bf16
+//   query side (tc_out_kernel): logits, phi = 2^(logits - rowmax), [num | den] = phi KV,
+//                               Y = num / den
+//
+// The feature tiles never leave the SM.  One block = 8 epilogue warps (exponentials), one
+// TMA producer warp and one MMA issuing warp; all exponents are kept in log2 units
+// (W, a and C are pre-multiplied by log2 e), so the feature is one ex2 per element.
+#include "common.cuh"
+#include "tc_common.cuh"
+#include "tc_layout.cuh"
+
+using namespace tc;
+using namespace tcl;
+
+namespace {
+
+// ------------------------------------------------------------------------------------------
+// key side
+// ------------------------------------------------------------------------------------------
+struct KvSmem {
+  static constexpr uint32_t X0 = 0, V0 = 2 * TILE_BYTES, ONES = 4 * TILE_BYTES, W = ONES + TILE_BYTES,
+                            CHI = W + IMG_W_BYTES, CLO = CHI + IMG_C_BYTES, BAUG = CLO + IMG_C_BYTES,
+                            AAUG = BAUG + IMG_BAUG_BYTES, PHI = AAUG + 4096, MISC = PHI + 4 * TILE_BYTES,
+                            TOTAL = MISC + 256;
+};
+static_assert(KvSmem::PHI % 1024 == 0 && KvSmem::W % 1024 == 0, "swizzled tiles need 1024-byte alignment");
+
+struct KvMisc {
+  uint64_t full[2], empty[2], logits_full, logits_free, phi_full, phi_free, const_bar;
+  uint32_t tmem_base;
+  int abort_flag;
+  int tile_max[3];
+};
+
+constexpr uint32_t KV_COL_LOGITS = 0, KV_COL_T = 256, KV_COL_ACC = 320;   // TMEM columns
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+             const uint8_t* __restrict__ images, const int* __restrict__ img_flags, int H, int pool, int L,
+             int tiles_per_split, int nsplit, float* __restrict__ partial, float* __restrict__ shifts,
+             int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  KvMisc* misc = reinterpret_cast<KvMisc*>(sm + KvSmem::MISC);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
+  const int g = pool == FSHARP_POOL_PER_BH ? bh : h;
+  const int total_tiles = (L + TILE - 1) / TILE;
+  const int tile0 = split * tiles_per_split;
+  const int ntiles = min(tiles_per_split, total_tiles - tile0);
+  const uint8_t* img = images + ((size_t)g * 2 + 1) * IMG_BYTES;        // side 2 (keys)
+  const int* fl = img_flags + ((size_t)g * 2 + 1) * FLAG_WORDS;
+  const bool cdense = (fl[0] & FLAG_C_DENSE) != 0, clo = (fl[0] & FLAG_C_LO) != 0;
+  const float gamma2 = __int_as_float(fl[1]);          // C = gamma I: c_j = gamma2 |x_j|^2 (log2 units)
+  volatile int* abortp = &misc->abort_flag;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], 1); }
+    mbar_init(&misc->logits_full, 1);
+    mbar_init(&misc->logits_free, EPI_THREADS);
+    mbar_init(&misc->phi_full, EPI_THREADS);
+    mbar_init(&misc->phi_free, 1);
+    mbar_init(&misc->const_bar, 1);
+    misc->abort_flag = 0;
+    misc->tile_max[0] = misc->tile_max[1] = misc->tile_max[2] = f2ord(-INFINITY);
+    fence_barrier_init();
+  }
+  // constant tiles written by the block itself: the ones column of [V | 1] and the rows (1, 1, 0, ...)
+  // that pick a_hi + a_lo out of the augmented feature operand
+  for (int i = threadIdx.x; i < TILE_BYTES / 16; i += TC_THREADS) reinterpret_cast<uint4*>(sm + KvSmem::ONES)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = threadIdx.x; i < 4096 / 16; i += TC_THREADS) reinterpret_cast<uint4*>(sm + KvSmem::AAUG)[i] = make_uint4(0, 0, 0, 0);
+  __syncthreads();
+  if (threadIdx.x < TILE) {
+    const uint32_t r = threadIdx.x;
+    *reinterpret_cast<__nv_bfloat16*>(sm + KvSmem::ONES + sw128_offset(r, 0)) = __float2bfloat16(1.f);
+    *reinterpret_cast<__nv_bfloat16*>(sm + KvSmem::AAUG + core16_offset(r, 0)) = __float2bfloat16(1.f);
+    *reinterpret_cast<__nv_bfloat16*>(sm + KvSmem::AAUG + core16_offset(r, 1)) = __float2bfloat16(1.f);
+  }
+  fence_proxy_async_smem();
+  if (warp == WARP_MMA) {
+    tmem_alloc(&misc->tmem_base, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem = misc->tmem_base;
+
+  if (warp == WARP_TMA) {
+    if (lane == 0) {
+      prefetch_tmap(&tmK);
+      prefetch_tmap(&tmV);
+      mbar_expect_tx(&misc->const_bar, IMG_BYTES);
+      bulk_load(sm + KvSmem::W, img + IMG_W, IMG_W_BYTES, &misc->const_bar);
+      bulk_load(sm + KvSmem::CHI, img + IMG_CHI, IMG_C_BYTES, &misc->const_bar);
+      bulk_load(sm + KvSmem::CLO, img + IMG_CLO, IMG_C_BYTES, &misc->const_bar);
+      bulk_load(sm + KvSmem::BAUG, img + IMG_BAUG, IMG_BAUG_BYTES, &misc->const_bar);
+      int issued = 0;
+      for (int it = 0; it < ntiles; it++) {
+        const int st = it & 1;
+        if (!mbar_wait(&misc->empty[st], ((it >> 1) & 1) ^ 1, abortp, status)) break;
+        mbar_expect_tx(&misc->full[st], 2 * TILE_BYTES);
+        tma_load_4d(sm + KvSmem::X0 + st * TILE_BYTES, &tmK, &misc->full[st], 0, (tile0 + it) * TILE, h, b);
+        tma_load_4d(sm + KvSmem::V0 + st * TILE_BYTES, &tmV, &misc->full[st], 0, (tile0 + it) * TILE, h, b);
+        issued = it + 1;
+      }
+      // no copy of this block may still be in flight when it exits
+      mbar_wait(&misc->const_bar, 0, abortp, status, false);
+      for (int it = max(0, issued - 2); it < issued; it++) mbar_wait(&misc->full[it & 1], (it >> 1) & 1, abortp, status, false);
+    }
+  } else if (warp == WARP_MMA) {
+    if (lane == 0) {
+      constexpr uint32_t ID_LOGITS = idesc_bf16(128, TC_M, 0, 0);
+      constexpr uint32_t ID_T = idesc_bf16(128, TC_D, 0, 0);
+      constexpr uint32_t ID_KV = idesc_bf16(128, TC_NV, 1, 1);
+      const uint32_t sW = smem_u32(sm + KvSmem::W), sChi = smem_u32(sm + KvSmem::CHI), sClo = smem_u32(sm + KvSmem::CLO);
+      const uint32_t sBaug = smem_u32(sm + KvSmem::BAUG), sAaug = smem_u32(sm + KvSmem::AAUG);
+      const uint32_t sPhi = smem_u32(sm + KvSmem::PHI), sOnes = smem_u32(sm + KvSmem::ONES);
+      auto issue_logits = [&](int st) {
+        const uint32_t sX = smem_u32(sm + KvSmem::X0 + st * TILE_BYTES);
+#pragma unroll
+        for (int k = 0; k < TC_D / 16; k++)
+          mma_bf16(tmem + KV_COL_LOGITS, smem_desc(sX + 32 * k, 16, 1024, SWZ_128B), smem_desc(sW + 32 * k, 16, 1024, SWZ_128B),
+                   ID_LOGITS, k > 0);
+        mma_bf16(tmem + KV_COL_LOGITS, smem_desc(sAaug, 128, 256, SWZ_NONE), smem_desc(sBaug, 128, 256, SWZ_NONE),
+                 ID_LOGITS, 1);
+        if (cdense) {
+#pragma unroll
+          for (int k = 0; k < TC_D / 16; k++)
+            mma_bf16(tmem + KV_COL_T, smem_desc(sX + 32 * k, 16, 1024, SWZ_128B), smem_desc(sChi + 32 * k, 16, 1024, SWZ_128B),
+                     ID_T, k > 0);
+          if (clo) {
+#pragma unroll
+            for (int k = 0; k < TC_D / 16; k++)
+              mma_bf16(tmem + KV_COL_T, smem_desc(sX + 32 * k, 16, 1024, SWZ_128B),
+                       smem_desc(sClo + 32 * k, 16, 1024, SWZ_128B), ID_T, 1);
+          }
+        }
+        mma_commit(&misc->logits_full);
+      };
+      bool ok = mbar_wait(&misc->const_bar, 0, abortp, status);
+      if (ok && ntiles > 0) ok = mbar_wait(&misc->full[0], 0, abortp, status);
+      if (ok && ntiles > 0) {
+        tcgen05_fence_after();
+        issue_logits(0);
+      }
+      for (int it = 0; ok && it < ntiles; it++) {
+        const int st = it & 1;
+        if (it + 1 < ntiles) {
+          if (!mbar_wait(&misc->full[st ^ 1], ((it + 1) >> 1) & 1, abortp, status)) break;
+          if (!mbar_wait(&misc->logits_free, it & 1, abortp, status)) break;
+          tcgen05_fence_after();
+          issue_logits(st ^ 1);
+        }
+        if (!mbar_wait(&misc->phi_full, it & 1, abortp, status)) break;
+        tcgen05_fence_after();
+        const uint32_t sV = smem_u32(sm + KvSmem::V0 + st * TILE_BYTES);
+#pragma unroll
+        for (int hh = 0; hh < 2; hh++)
+#pragma unroll
+          for (int k = 0; k < TILE / 16; k++)
+            mma_bf16(tmem + KV_COL_ACC + hh * TC_NV,
+                     smem_desc(sPhi + hh * 2 * TILE_BYTES + k * 2048, TILE_BYTES, 1024, SWZ_128B),
+                     smem_desc(sV + k * 2048, sOnes - sV, 1024, SWZ_128B), ID_KV, (it > 0 || k > 0) ? 1u : 0u);
+        mma_commit(&misc->phi_free);
+        mma_commit(&misc->empty[st]);
+      }
+    }
+  } else {
+    // ---------------- epilogue warps: one key row per thread, 128 of the 256 features
+    const int q = warp & 3, hf = warp >> 2;
+    const int row = q * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+    float s = 0.f;
+    bool have = false, alive = true;
+    for (int it = 0; it < ntiles && alive; it++) {
+      const int st = it & 1;
+      if (!mbar_wait(&misc->full[st], (it >> 1) & 1, abortp, status, false)) { alive = false; break; }
+      if (!mbar_wait(&misc->logits_full, it & 1, abortp, status, false)) { alive = false; break; }
+      __syncwarp();
+      tcgen05_fence_after();
+      // c_j = x_j^T C x_j in log2 units
+      float cj = 0.f;
+      {
+        const uint8_t* xrow = sm + KvSmem::X0 + st * TILE_BYTES + row * 128;
+        float xv[TC_D];
+#pragma unroll
+        for (int c = 0; c < 8; c++) {
+          uint4 u = *reinterpret_cast<const uint4*>(xrow + ((c ^ (row & 7)) << 4));
+          const uint32_t w4[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+          for (int j = 0; j < 4; j++) {
+            xv[c * 8 + 2 * j] = __uint_as_float(w4[j] << 16);
+            xv[c * 8 + 2 * j + 1] = __uint_as_float(w4[j] & 0xffff0000u);
+          }
+        }
+        if (cdense) {
+#pragma unroll
+          for (int c = 0; c < TC_D / 16; c++) {
+            uint32_t t[16];
+            tmem_ld16(lane_addr + KV_COL_T + c * 16, t);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 16; j++) cj = fmaf(__uint_as_float(t[j]), xv[c * 16 + j], cj);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < TC_D; j++) cj = fmaf(xv[j], xv[j], cj);
+          cj *= gamma2;
+        }
+      }
+      uint32_t v[128];
+#pragma unroll
+      for (int c = 0; c < 8; c++) {
+        uint32_t t[16];
+        tmem_ld16(lane_addr + KV_COL_LOGITS + hf * 128 + c * 16, t);
+#pragma unroll
+        for (int j = 0; j < 16; j++) v[c * 16 + j] = t[j];
+      }
+      tmem_wait_ld();
+      tcgen05_fence_before();
+      mbar_arrive(&misc->logits_free);
+      const bool valid = (tile0 + it) * TILE + row < L;
+      float mx = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 128; i++) {
+        float f = __uint_as_float(v[i]) + cj;
+        v[i] = __float_as_uint(f);
+        mx = fmaxf(mx, f);
+      }
+      if (!valid) mx = -INFINITY;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      if (lane == 0) atomicMax(&misc->tile_max[it % 3], f2ord(mx));
+      if (threadIdx.x == 0) misc->tile_max[(it + 1) % 3] = f2ord(-INFINITY);   // next tile's slot; idle since tile it-2
+      named_bar_sync(1, EPI_THREADS);
+      const float t = ord2f(misc->tile_max[it % 3]);
+      const float s_old = s;
+      bool rescale = false;
+      if (!have || t > s + SHIFT_HEADROOM_LOG2) {
+        rescale = have;
+        s = t;
+        have = true;
+      }
+      if (it > 0) {
+        if (!mbar_wait(&misc->phi_free, (it - 1) & 1, abortp, status, false)) { alive = false; break; }
+      }
+      __syncwarp();
+      if (rescale) {
+        // the running shift moved: bring the accumulated S^T [V | 1] to the new one
+        tcgen05_fence_after();
+        const float f = ex2(s_old - s);
+#pragma unroll
+        for (int c = 0; c < TC_NV / 16; c++) {
+          uint32_t a[16];
+          tmem_ld16(lane_addr + KV_COL_ACC + hf * TC_NV + c * 16, a);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 16; j++) a[j] = __float_as_uint(__uint_as_float(a[j]) * f);
+          tmem_st16(lane_addr + KV_COL_ACC + hf * TC_NV + c * 16, a);
+        }
+        tmem_wait_st();
+      }
+      uint8_t* prow = sm + KvSmem::PHI + hf * 2 * TILE_BYTES + row * 128;
+#pragma unroll
+      for (int c = 0; c < 16; c++) {
+        uint32_t p[4];
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+          float e0 = ex2(__uint_as_float(v[c * 8 + 2 * j]) - s), e1 = ex2(__uint_as_float(v[c * 8 + 2 * j + 1]) - s);
+          p[j] = valid ? pack_bf16(e0, e1) : 0u;
+        }
+        *reinterpret_cast<uint4*>(prow + (c >> 3) * TILE_BYTES + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
+      }
+      fence_proxy_async_smem();
+      tcgen05_fence_before();
+      mbar_arrive(&misc->phi_full);
+    }
+    // write this split's partial S^T [V | 1] (fp32) and its shift
+    if (alive && ntiles > 0 && mbar_wait(&misc->phi_free, (ntiles - 1) & 1, abortp, status, false)) {
+      __syncwarp();
+      tcgen05_fence_after();
+      float* out = partial + (((size_t)bh * nsplit + split) * TC_M + hf * 128 + row) * TC_NV;
+#pragma unroll
+      for (int c = 0; c < TC_NV / 16; c++) {
+        uint32_t a[16];
+        tmem_ld16(lane_addr + KV_COL_ACC + hf * TC_NV + c * 16, a);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 4; j++)
+          reinterpret_cast<uint4*>(out + c * 16)[j] = make_uint4(a[4 * j], a[4 * j + 1], a[4 * j + 2], a[4 * j + 3]);
+      }
+      if (threadIdx.x == 0) shifts[(size_t)bh * nsplit + split] = s;
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == WARP_MMA) {
+    tcgen05_fence_after();
+    tmem_dealloc(tmem, TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// merge of the key-side partials of one (batch, head): common shift, sum, transpose, bf16
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+tc_merge_kernel(const float* __restrict__ partial, const float* __restrict__ shifts, int nsplit,
+                __nv_bfloat16* __restrict__ kvt) {
+  const int bh = blockIdx.x;
+  float smax = -INFINITY;
+  for (int p = 0; p < nsplit; p++) smax = fmaxf(smax, shifts[(size_t)bh * nsplit + p]);
+  const float* base = partial + (size_t)bh * nsplit * TC_M * TC_NV;
+  __nv_bfloat16* out = kvt + (size_t)bh * TC_NV * TC_M;
+  for (int e = threadIdx.x; e < TC_M * TC_NV; e += 256) {
+    const int m = e / TC_NV, n = e % TC_NV;
+    float acc = 0.f;
+    if (n <= TC_DV)
+      for (int p = 0; p < nsplit; p++)
+        acc = fmaf(base[(size_t)p * TC_M * TC_NV + e], exp2f(shifts[(size_t)bh * nsplit + p] - smax), acc);
+    out[(size_t)n * TC_M + m] = __float2bfloat16_rn(acc);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// query side
+// ------------------------------------------------------------------------------------------
+constexpr int OUT_STAGES = 3;
+struct OutSmem {
+  static constexpr uint32_t X0 = 0, W = OUT_STAGES * TILE_BYTES, BAUG = W + IMG_W_BYTES, AAUG = BAUG + IMG_BAUG_BYTES,
+                            PHI = AAUG + 4096, KVT = PHI + 4 * TILE_BYTES, ROWMAX = KVT + KVT_BYTES,
+                            MISC = ROWMAX + 2 * 2 * TILE * 4, TOTAL = MISC + 256;
+};
+static_assert(OutSmem::PHI % 1024 == 0 && OutSmem::KVT % 1024 == 0 && OutSmem::W % 1024 == 0, "alignment");
+
+struct OutMisc {
+  uint64_t full[OUT_STAGES], empty[OUT_STAGES], logits_full, logits_free, phi_full, phi_free, out_full[2], const_bar;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+constexpr uint32_t OUT_COL_LOGITS = 0, OUT_COL_OUT = 256;
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKVt,
+              const uint8_t* __restrict__ images, int H, int pool, int L, int tiles_per_split,
+              __nv_bfloat16* __restrict__ Y, TensorAddr ay, int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  OutMisc* misc = reinterpret_cast<OutMisc*>(sm + OutSmem::MISC);
+  float* rowmax = reinterpret_cast<float*>(sm + OutSmem::ROWMAX);   // [parity][half][row]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
+  const int g = pool == FSHARP_POOL_PER_BH ? bh : h;
+  const int total_tiles = (L + TILE - 1) / TILE;
+  const int tile0 = split * tiles_per_split;
+  const int ntiles = min(tiles_per_split, total_tiles - tile0);
+  const uint8_t* img = images + ((size_t)g * 2 + 0) * IMG_BYTES;        // side 1 (queries)
+  volatile int* abortp = &misc->abort_flag;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < OUT_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], 1); }
+    mbar_init(&misc->logits_full, 1);
+    mbar_init(&misc->logits_free, EPI_THREADS);
+    mbar_init(&misc->phi_full, EPI_THREADS);
+    mbar_init(&misc->phi_free, 1);
+    mbar_init(&misc->out_full[0], 1);
+    mbar_init(&misc->out_full[1], 1);
+    mbar_init(&misc->const_bar, 1);
+    misc->abort_flag = 0;
+    fence_barrier_init();
+  }
+  for (int i = threadIdx.x; i < 4096 / 16; i += TC_THREADS) reinterpret_cast<uint4*>(sm + OutSmem::AAUG)[i] = make_uint4(0, 0, 0, 0);
+  __syncthreads();
+  if (threadIdx.x < TILE) {
+    const uint32_t r = threadIdx.x;
+    *reinterpret_cast<__nv_bfloat16*>(sm + OutSmem::AAUG + core16_offset(r, 0)) = __float2bfloat16(1.f);
+    *reinterpret_cast<__nv_bfloat16*>(sm + OutSmem::AAUG + core16_offset(r, 1)) = __float2bfloat16(1.f);
+  }
+  fence_proxy_async_smem();
+  if (warp == WARP_MMA) {
+    tmem_alloc(&misc->tmem_base, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem = misc->tmem_base;
+
+  if (warp == WARP_TMA) {
+    if (lane == 0) {
+      prefetch_tmap(&tmQ);
+      prefetch_tmap(&tmKVt);
+      mbar_expect_tx(&misc->const_bar, IMG_W_BYTES + IMG_BAUG_BYTES + KVT_BYTES);
+      bulk_load(sm + OutSmem::W, img + IMG_W, IMG_W_BYTES, &misc->const_bar);
+      bulk_load(sm + OutSmem::BAUG, img + IMG_BAUG, IMG_BAUG_BYTES, &misc->const_bar);
+#pragma unroll
+      for (int fb = 0; fb < TC_M / 64; fb++)
+        tma_load_3d(sm + OutSmem::KVT + fb * KVT_BLOCK_BYTES, &tmKVt, &misc->const_bar, fb * 64, 0, bh);
+      int issued = 0;
+      for (int it = 0; it < ntiles; it++) {
+        const int st = it % OUT_STAGES;
+        if (!mbar_wait(&misc->empty[st], ((it / OUT_STAGES) & 1) ^ 1, abortp, status)) break;
+        mbar_expect_tx(&misc->full[st], TILE_BYTES);
+        tma_load_4d(sm + OutSmem::X0 + st * TILE_BYTES, &tmQ, &misc->full[st], 0, (tile0 + it) * TILE, h, b);
+        issued = it + 1;
+      }
+      mbar_wait(&misc->const_bar, 0, abortp, status, false);
+      for (int it = max(0, issued - OUT_STAGES); it < issued; it++)
+        mbar_wait(&misc->full[it % OUT_STAGES], (it / OUT_STAGES) & 1, abortp, status, false);
+    }
+  } else if (warp == WARP_MMA) {
+    if (lane == 0) {
+      constexpr uint32_t ID_LOGITS = idesc_bf16(128, TC_M, 0, 0);
+      constexpr uint32_t ID_OUT = idesc_bf16(128, TC_NV, 0, 0);
+      const uint32_t sW = smem_u32(sm + OutSmem::W), sBaug = smem_u32(sm + OutSmem::BAUG), sAaug = smem_u32(sm + OutSmem::AAUG);
+      const uint32_t sPhi = smem_u32(sm + OutSmem::PHI), sKvt = smem_u32(sm + OutSmem::KVT);
+      auto issue_logits = [&](int st) {
+        const uint32_t sX = smem_u32(sm + OutSmem::X0 + st * TILE_BYTES);
+#pragma unroll
+        for (int k = 0; k < TC_D / 16; k++)
+          mma_bf16(tmem + OUT_COL_LOGITS, smem_desc(sX + 32 * k, 16, 1024, SWZ_128B), smem_desc(sW + 32 * k, 16, 1024, SWZ_128B),
+                   ID_LOGITS, k > 0);
+        mma_bf16(tmem + OUT_COL_LOGITS, smem_desc(sAaug, 128, 256, SWZ_NONE), smem_desc(sBaug, 128, 256, SWZ_NONE),
+                 ID_LOGITS, 1);
+        mma_commit(&misc->logits_full);
+        mma_commit(&misc->empty[st]);
+      };
+      bool ok = mbar_wait(&misc->const_bar, 0, abortp, status);
+      if (ok && ntiles > 0) ok = mbar_wait(&misc->full[0], 0, abortp, status);
+      if (ok && ntiles > 0) {
+        tcgen05_fence_after();
+        issue_logits(0);
+      }
+      for (int it = 0; ok && it < ntiles; it++) {
+        if (it + 1 < ntiles) {
+          const int sn = (it + 1) % OUT_STAGES;
+          if (!mbar_wait(&misc->full[sn], ((it + 1) / OUT_STAGES) & 1, abortp, status)) break;
+          if (!mbar_wait(&misc->logits_free, it & 1, abortp, status)) break;
+          tcgen05_fence_after();
+          issue_logits(sn);
+        }
+        if (!mbar_wait(&misc->phi_full, it & 1, abortp, status)) break;
+        tcgen05_fence_after();
+#pragma unroll
+        for (int fb = 0; fb < TC_M / 64; fb++)
+#pragma unroll
+          for (int k = 0; k < 4; k++)
+            mma_bf16(tmem + OUT_COL_OUT + (it & 1) * TC_NV, smem_desc(sPhi + fb * TILE_BYTES + 32 * k, 16, 1024, SWZ_128B),
+                     smem_desc(sKvt + fb * KVT_BLOCK_BYTES + 32 * k, 16, 1024, SWZ_128B), ID_OUT, (fb > 0 || k > 0) ? 1u : 0u);
+        mma_commit(&misc->phi_free);
+        mma_commit(&misc->out_full[it & 1]);
+      }
+    }
+  } else {
+    const int q = warp & 3, hf = warp >> 2;
+    const int row = q * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+    __nv_bfloat16* Yb = Y + b * ay.sb + h * ay.sh;
+    bool alive = true;
+    // Y rows of tile j: [num | den] from TMEM, one divide per row, 32 of the 64 columns per thread
+    auto write_out = [&](int j) -> bool {
+      if (!mbar_wait(&misc->out_full[j & 1], (j >> 1) & 1, abortp, status, false)) return false;
+      __syncwarp();
+      tcgen05_fence_after();
+      uint32_t n0[16], n1[16], dn[16];
+      const uint32_t base = lane_addr + OUT_COL_OUT + (j & 1) * TC_NV;
+      tmem_ld16(base + hf * 32, n0);
+      tmem_ld16(base + hf * 32 + 16, n1);
+      tmem_ld16(base + TC_DV, dn);
+      tmem_wait_ld();
+      const int64_t r = (int64_t)(tile0 + j) * TILE + row;
+      if (r < L) {
+        const float den = __uint_as_float(dn[0]);
+        if (!(den > 0.f) || !isfinite(den)) atomicExch(status, FSHARP_E_NONFINITE);
+        const float inv = 1.f / den;
+        uint32_t o[16];
+#pragma unroll
+        for (int i = 0; i < 8; i++) {
+          o[i] = pack_bf16(__uint_as_float(n0[2 * i]) * inv, __uint_as_float(n0[2 * i + 1]) * inv);
+          o[8 + i] = pack_bf16(__uint_as_float(n1[2 * i]) * inv, __uint_as_float(n1[2 * i + 1]) * inv);
+        }
+        uint4* dst = reinterpret_cast<uint4*>(Yb + r * ay.sl + hf * 32);
+#pragma unroll
+        for (int i = 0; i < 4; i++) dst[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+      }
+      return true;
+    };
+    for (int it = 0; it < ntiles && alive; it++) {
+      if (!mbar_wait(&misc->logits_full, it & 1, abortp, status, false)) { alive = false; break; }
+      __syncwarp();
+      tcgen05_fence_after();
+      uint32_t v[128];
+#pragma unroll
+      for (int c = 0; c < 8; c++) {
+        uint32_t t[16];
+        tmem_ld16(lane_addr + OUT_COL_LOGITS + hf * 128 + c * 16, t);
+#pragma unroll
+        for (int j = 0; j < 16; j++) v[c * 16 + j] = t[j];
+      }
+      tmem_wait_ld();
+      tcgen05_fence_before();
+      mbar_arrive(&misc->logits_free);
+      float mx = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 128; i++) mx = fmaxf(mx, __uint_as_float(v[i]));
+      float* rm = rowmax + (it & 1) * 2 * TILE;
+      rm[hf * TILE + row] = mx;
+      named_bar_sync(1, EPI_THREADS);
+      mx = fmaxf(mx, rm[(hf ^ 1) * TILE + row]);
+      if (it > 0) {
+        if (!mbar_wait(&misc->phi_free, (it - 1) & 1, abortp, status, false)) { alive = false; break; }
+      }
+      uint8_t* prow = sm + OutSmem::PHI + hf * 2 * TILE_BYTES + row * 128;
+#pragma unroll
+      for (int c = 0; c < 16; c++) {
+        uint32_t p[4];
+#pragma unroll
+        for (int j = 0; j < 4; j++)
+          p[j] = pack_bf16(ex2(__uint_as_float(v[c * 8 + 2 * j]) - mx), ex2(__uint_as_float(v[c * 8 + 2 * j + 1]) - mx));
+        *reinterpret_cast<uint4*>(prow + (c >> 3) * TILE_BYTES + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
+      }
+      fence_proxy_async_smem();
+      tcgen05_fence_before();
+      mbar_arrive(&misc->phi_full);
+      if (it > 0) alive = write_out(it - 1);
+    }
+    if (alive && ntiles > 0) write_out(ntiles - 1);
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == WARP_MMA) {
+    tcgen05_fence_after();
+    tmem_dealloc(tmem, TMEM_COLS);
+  }
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------
+namespace tchost {
+int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int H, int L, int inner);
+int make_map_kvt(CUtensorMap* map, const void* base, int BH);
+}  // namespace tchost
+int fs_tc_prep(fsharp_ctx* ctx, const float* prep, int G, float qk_scale, uint8_t* images, int* flags);
+size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
+int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
+                const float* prep, void* Y, WsAlloc* ws);
+
+size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
+  const size_t BH = (size_t)dm->B * dm->H;
+  const size_t G = fs_groups(dm);
+  const size_t max_split = 64;
+  return ws_round(G * 2 * IMG_BYTES) + ws_round(G * 2 * FLAG_WORDS * 4 + 64) +
+         ws_round(BH * max_split * TC_M * TC_NV * 4) + ws_round(BH * max_split * 4) + ws_round(BH * TC_NV * TC_M * 2);
+}
+
+int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
+                const float* prep, void* Y, WsAlloc* ws) {
+  const int B = dm->B, H = dm->H, BH = B * H, Lq = dm->Lq, Lk = dm->Lk;
+  const int G = fs_groups(dm);
+  uint8_t* images = ws->take<uint8_t>((size_t)G * 2 * IMG_BYTES);
+  int* flags = ws->take<int>((size_t)G * 2 * FLAG_WORDS + 16);
+  FS_TRY(fs_tc_prep(ctx, prep, G, qk_scale, images, flags));
+
+  // key side: splits of the key range so that about one block per SM is busy
+  const int ktiles = (Lk + TILE - 1) / TILE;
+  int nsplit = (ctx->sm_count + BH - 1) / BH;
+  if (nsplit > ktiles) nsplit = ktiles;
+  if (nsplit > 64) nsplit = 64;
+  if (nsplit < 1) nsplit = 1;
+  int tps = (ktiles + nsplit - 1) / nsplit;
+  nsplit = (ktiles + tps - 1) / tps;
+  float* partial = ws->take<float>((size_t)BH * 64 * TC_M * TC_NV);
+  float* shifts = ws->take<float>((size_t)BH * 64);
+  __nv_bfloat16* kvt = ws->take<__nv_bfloat16>((size_t)BH * TC_NV * TC_M);
+
+  CUtensorMap tmK, tmV, tmQ, tmKVt;
+  FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, Lk, dm->d), B, H, Lk, dm->d));
+  FS_TRY(tchost::make_map_tokens(&tmV, V, fs_addr(dm->v_stride, H, Lk, dm->dv), B, H, Lk, dm->dv));
+  FS_TRY(tchost::make_map_tokens(&tmQ, Q, fs_addr(dm->q_stride, H, Lq, dm->d), B, H, Lq, dm->d));
+  FS_TRY(tchost::make_map_kvt(&tmKVt, kvt, BH));
+
+  FS_CUDA_OK(cudaFuncSetAttribute(tc_kv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KvSmem::TOTAL + 1024));
+  FS_CUDA_OK(cudaFuncSetAttribute(tc_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OutSmem::TOTAL + 1024));
+  FS_TIME_BEGIN(ctx, FS_K_TC_KV);
+  tc_kv_kernel<<<dim3(nsplit, BH), TC_THREADS, KvSmem::TOTAL + 1024, ctx->stream>>>(
+      tmK, tmV, images, flags, H, dm->pool, Lk, tps, nsplit, partial, shifts, ctx->d_status);
+  FS_TIME_END(ctx);
+  FS_LAUNCH_CHECK(ctx);
+  FS_TIME_BEGIN(ctx, FS_K_TC_MERGE);
+  tc_merge_kernel<<<BH, 256, 0, ctx->stream>>>(partial, shifts, nsplit, kvt);
+  FS_TIME_END(ctx);
+  FS_LAUNCH_CHECK(ctx);
+
+  const int qtiles = (Lq + TILE - 1) / TILE;
+  int qsplit = (ctx->sm_count + BH - 1) / BH;
+  if (qsplit > qtiles) qsplit = qtiles;
+  if (qsplit < 1) qsplit = 1;
+  int qtps = (qtiles + qsplit - 1) / qsplit;
+  qsplit = (qtiles + qtps - 1) / qtps;
+  FS_TIME_BEGIN(ctx, FS_K_TC_OUT);
+  tc_out_kernel<<<dim3(qsplit, BH), TC_THREADS, OutSmem::TOTAL + 1024, ctx->stream>>>(
+      tmQ, tmKVt, images, H, dm->pool, Lq, qtps, (__nv_bfloat16*)Y, fs_addr(dm->y_stride, H, Lq, dm->dv), ctx->d_status);
+  FS_TIME_END(ctx);
+  FS_LAUNCH_CHECK(ctx);
+  return FSHARP_OK;
+}
