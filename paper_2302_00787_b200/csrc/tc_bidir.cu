@@ -4,13 +4,15 @@
 //                               phi = 2^(logits + c_j - s)  -> bf16 tile in shared memory
 //                               KV += phi^T [V | 1]                          (tcgen05, TMEM)
 //   merge      (tc_merge_kernel): partial KV of the splits of one (batch, head), brought to a
-//                               common shift, summed, written transposed in bf16
+//                               common shift, summed, written transposed in fp16
 //   query side (tc_out_kernel): logits, phi = 2^(logits - rowmax), [num | den] = phi KV,
 //                               Y = num / den
 //
 // The feature tiles never leave the SM.  One block = 8 epilogue warps (exponentials), one
 // TMA producer warp and one MMA issuing warp; all exponents are kept in log2 units
 // (W, a and C are pre-multiplied by log2 e), so the feature is one ex2 per element.
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 #include "tc_common.cuh"
 #include "tc_layout.cuh"
@@ -24,12 +26,13 @@ namespace {
 // key side
 // ------------------------------------------------------------------------------------------
 struct KvSmem {
-  static constexpr uint32_t X0 = 0, V0 = 2 * TILE_BYTES, ONES = 4 * TILE_BYTES, W = ONES + TILE_BYTES,
-                            CHI = W + IMG_W_BYTES, CLO = CHI + IMG_C_BYTES, BAUG = CLO + IMG_C_BYTES,
-                            AAUG = BAUG + IMG_BAUG_BYTES, PHI = AAUG + 4096, MISC = PHI + 4 * TILE_BYTES,
-                            TOTAL = MISC + 256;
+  static constexpr uint32_t X0 = 0, V0 = 2 * TILE_BYTES, W = 4 * TILE_BYTES, WLO = W + IMG_W_BYTES,
+                            CHI = WLO + IMG_W_BYTES, CLO = CHI + IMG_C_BYTES, BAUG = CLO + IMG_C_BYTES,
+                            AAUG = BAUG + IMG_BAUG_BYTES, ONEST = AAUG + 4096, PHI = ONEST + ONEST_BYTES,
+                            MISC = PHI + 4 * TILE_BYTES, TOTAL = MISC + 256;
 };
-static_assert(KvSmem::PHI % 1024 == 0 && KvSmem::W % 1024 == 0, "swizzled tiles need 1024-byte alignment");
+static_assert(KvSmem::TOTAL + 1024 <= 232448, "shared memory budget");
+static_assert(KvSmem::PHI % 1024 == 0 && KvSmem::W % 1024 == 0 && KvSmem::ONEST % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 
 struct KvMisc {
   uint64_t full[2], empty[2], logits_full, logits_free, phi_full, phi_free, const_bar;
@@ -73,12 +76,13 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   }
   // constant tiles written by the block itself: the ones column of [V | 1] and the rows (1, 1, 0, ...)
   // that pick a_hi + a_lo out of the augmented feature operand
-  for (int i = threadIdx.x; i < TILE_BYTES / 16; i += TC_THREADS) reinterpret_cast<uint4*>(sm + KvSmem::ONES)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = threadIdx.x; i < ONEST_BYTES / 16; i += TC_THREADS) reinterpret_cast<uint4*>(sm + KvSmem::ONEST)[i] = make_uint4(0, 0, 0, 0);
   for (int i = threadIdx.x; i < 4096 / 16; i += TC_THREADS) reinterpret_cast<uint4*>(sm + KvSmem::AAUG)[i] = make_uint4(0, 0, 0, 0);
   __syncthreads();
   if (threadIdx.x < TILE) {
     const uint32_t r = threadIdx.x;
-    *reinterpret_cast<__nv_bfloat16*>(sm + KvSmem::ONES + sw128_offset(r, 0)) = __float2bfloat16(1.f);
+    // transposed ones operand: row 0 of a [16 x 128 tokens] K-major matrix, two 64-token blocks of 2 KB
+    *reinterpret_cast<__nv_bfloat16*>(sm + KvSmem::ONEST + (r >> 6) * 2048 + sw128_offset(0, r & 63)) = __float2bfloat16(1.f);
     *reinterpret_cast<__nv_bfloat16*>(sm + KvSmem::AAUG + core16_offset(r, 0)) = __float2bfloat16(1.f);
     *reinterpret_cast<__nv_bfloat16*>(sm + KvSmem::AAUG + core16_offset(r, 1)) = __float2bfloat16(1.f);
   }
@@ -98,6 +102,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       prefetch_tmap(&tmV);
       mbar_expect_tx(&misc->const_bar, IMG_BYTES);
       bulk_load(sm + KvSmem::W, img + IMG_W, IMG_W_BYTES, &misc->const_bar);
+      bulk_load(sm + KvSmem::WLO, img + IMG_WLO, IMG_W_BYTES, &misc->const_bar);
       bulk_load(sm + KvSmem::CHI, img + IMG_CHI, IMG_C_BYTES, &misc->const_bar);
       bulk_load(sm + KvSmem::CLO, img + IMG_CLO, IMG_C_BYTES, &misc->const_bar);
       bulk_load(sm + KvSmem::BAUG, img + IMG_BAUG, IMG_BAUG_BYTES, &misc->const_bar);
@@ -118,16 +123,22 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     if (lane == 0) {
       constexpr uint32_t ID_LOGITS = idesc_bf16(128, TC_M, 0, 0);
       constexpr uint32_t ID_T = idesc_bf16(128, TC_D, 0, 0);
-      constexpr uint32_t ID_KV = idesc_bf16(128, TC_NV, 1, 1);
+      constexpr uint32_t ID_KV = idesc_bf16(128, TC_DV, 1, 1);     // phi^T V
+      constexpr uint32_t ID_KV1 = idesc_bf16(128, 16, 1, 0);       // phi^T 1 (column dv of [V | 1])
+      const uint32_t sWlo = smem_u32(sm + KvSmem::WLO);
       const uint32_t sW = smem_u32(sm + KvSmem::W), sChi = smem_u32(sm + KvSmem::CHI), sClo = smem_u32(sm + KvSmem::CLO);
       const uint32_t sBaug = smem_u32(sm + KvSmem::BAUG), sAaug = smem_u32(sm + KvSmem::AAUG);
-      const uint32_t sPhi = smem_u32(sm + KvSmem::PHI), sOnes = smem_u32(sm + KvSmem::ONES);
+      const uint32_t sPhi = smem_u32(sm + KvSmem::PHI), sOnesT = smem_u32(sm + KvSmem::ONEST);
       auto issue_logits = [&](int st) {
         const uint32_t sX = smem_u32(sm + KvSmem::X0 + st * TILE_BYTES);
 #pragma unroll
         for (int k = 0; k < TC_D / 16; k++)
           mma_bf16(tmem + KV_COL_LOGITS, smem_desc(sX + 32 * k, 16, 1024, SWZ_128B), smem_desc(sW + 32 * k, 16, 1024, SWZ_128B),
                    ID_LOGITS, k > 0);
+#pragma unroll
+        for (int k = 0; k < TC_D / 16; k++)
+          mma_bf16(tmem + KV_COL_LOGITS, smem_desc(sX + 32 * k, 16, 1024, SWZ_128B), smem_desc(sWlo + 32 * k, 16, 1024, SWZ_128B),
+                   ID_LOGITS, 1);
         mma_bf16(tmem + KV_COL_LOGITS, smem_desc(sAaug, 128, 256, SWZ_NONE), smem_desc(sBaug, 128, 256, SWZ_NONE),
                  ID_LOGITS, 1);
         if (cdense) {
@@ -164,10 +175,13 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 #pragma unroll
         for (int hh = 0; hh < 2; hh++)
 #pragma unroll
-          for (int k = 0; k < TILE / 16; k++)
-            mma_bf16(tmem + KV_COL_ACC + hh * TC_NV,
-                     smem_desc(sPhi + hh * 2 * TILE_BYTES + k * 2048, TILE_BYTES, 1024, SWZ_128B),
-                     smem_desc(sV + k * 2048, sOnes - sV, 1024, SWZ_128B), ID_KV, (it > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < TILE / 16; k++) {
+            const uint64_t da = smem_desc(sPhi + hh * 2 * TILE_BYTES + k * 2048, TILE_BYTES, 1024, SWZ_128B);
+            const uint32_t acc = (it > 0 || k > 0) ? 1u : 0u;
+            mma_bf16(tmem + KV_COL_ACC + hh * TC_NV, da, smem_desc(sV + k * 2048, 16, 1024, SWZ_128B), ID_KV, acc);
+            mma_bf16(tmem + KV_COL_ACC + hh * TC_NV + TC_DV, da,
+                     smem_desc(sOnesT + (k >> 2) * 2048 + (k & 3) * 32, 16, 1024, SWZ_128B), ID_KV1, acc);
+          }
         mma_commit(&misc->phi_free);
         mma_commit(&misc->empty[st]);
       }
@@ -312,32 +326,52 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 tc_merge_kernel(const float* __restrict__ partial, const float* __restrict__ shifts, int nsplit,
-                __nv_bfloat16* __restrict__ kvt) {
+                __half* __restrict__ kvt) {
+  __shared__ float red[256];
   const int bh = blockIdx.x;
   float smax = -INFINITY;
   for (int p = 0; p < nsplit; p++) smax = fmaxf(smax, shifts[(size_t)bh * nsplit + p]);
   const float* base = partial + (size_t)bh * nsplit * TC_M * TC_NV;
-  __nv_bfloat16* out = kvt + (size_t)bh * TC_NV * TC_M;
+  __half* out = kvt + (size_t)bh * TC_NV * TC_M;
+  auto merged = [&](int e) {
+    float acc = 0.f;
+    for (int p = 0; p < nsplit; p++)
+      acc = fmaf(base[(size_t)p * TC_M * TC_NV + e], exp2f(shifts[(size_t)bh * nsplit + p] - smax), acc);
+    return acc;
+  };
+  // fp16 has a narrow range: scale the whole (batch, head) by a power of two (it cancels in
+  // num / den) so that the largest magnitude lands near 2^14
+  float mx = 0.f;
+  for (int e = threadIdx.x; e < TC_M * TC_NV; e += 256)
+    if (e % TC_NV <= TC_DV) mx = fmaxf(mx, fabsf(merged(e)));
+  red[threadIdx.x] = mx;
+  __syncthreads();
+  for (int s = 128; s > 0; s >>= 1) {
+    if (threadIdx.x < s) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + s]);
+    __syncthreads();
+  }
+  mx = red[0];
+  int ex = 0;
+  if (mx > 0.f && isfinite(mx)) frexpf(mx, &ex);
+  const float scale = exp2f((float)(14 - ex));
   for (int e = threadIdx.x; e < TC_M * TC_NV; e += 256) {
     const int m = e / TC_NV, n = e % TC_NV;
-    float acc = 0.f;
-    if (n <= TC_DV)
-      for (int p = 0; p < nsplit; p++)
-        acc = fmaf(base[(size_t)p * TC_M * TC_NV + e], exp2f(shifts[(size_t)bh * nsplit + p] - smax), acc);
-    out[(size_t)n * TC_M + m] = __float2bfloat16_rn(acc);
+    out[(size_t)n * TC_M + m] = __float2half_rn(n <= TC_DV ? merged(e) * scale : 0.f);
   }
 }
 
 // ------------------------------------------------------------------------------------------
 // query side
 // ------------------------------------------------------------------------------------------
-constexpr int OUT_STAGES = 3;
+constexpr int OUT_STAGES = 2;
 struct OutSmem {
-  static constexpr uint32_t X0 = 0, W = OUT_STAGES * TILE_BYTES, BAUG = W + IMG_W_BYTES, AAUG = BAUG + IMG_BAUG_BYTES,
+  static constexpr uint32_t X0 = 0, W = OUT_STAGES * TILE_BYTES, WLO = W + IMG_W_BYTES, BAUG = WLO + IMG_W_BYTES,
+                            AAUG = BAUG + IMG_BAUG_BYTES,
                             PHI = AAUG + 4096, KVT = PHI + 4 * TILE_BYTES, ROWMAX = KVT + KVT_BYTES,
                             MISC = ROWMAX + 2 * 2 * TILE * 4, TOTAL = MISC + 256;
 };
 static_assert(OutSmem::PHI % 1024 == 0 && OutSmem::KVT % 1024 == 0 && OutSmem::W % 1024 == 0, "alignment");
+static_assert(OutSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 
 struct OutMisc {
   uint64_t full[OUT_STAGES], empty[OUT_STAGES], logits_full, logits_free, phi_full, phi_free, out_full[2], const_bar;
@@ -396,8 +430,9 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
     if (lane == 0) {
       prefetch_tmap(&tmQ);
       prefetch_tmap(&tmKVt);
-      mbar_expect_tx(&misc->const_bar, IMG_W_BYTES + IMG_BAUG_BYTES + KVT_BYTES);
+      mbar_expect_tx(&misc->const_bar, 2 * IMG_W_BYTES + IMG_BAUG_BYTES + KVT_BYTES);
       bulk_load(sm + OutSmem::W, img + IMG_W, IMG_W_BYTES, &misc->const_bar);
+      bulk_load(sm + OutSmem::WLO, img + IMG_WLO, IMG_W_BYTES, &misc->const_bar);
       bulk_load(sm + OutSmem::BAUG, img + IMG_BAUG, IMG_BAUG_BYTES, &misc->const_bar);
 #pragma unroll
       for (int fb = 0; fb < TC_M / 64; fb++)
@@ -417,8 +452,9 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
   } else if (warp == WARP_MMA) {
     if (lane == 0) {
       constexpr uint32_t ID_LOGITS = idesc_bf16(128, TC_M, 0, 0);
-      constexpr uint32_t ID_OUT = idesc_bf16(128, TC_NV, 0, 0);
+      constexpr uint32_t ID_OUT = idesc_f16(128, TC_NV, 0, 0);      // fp16: phi(Q) <= 1 and the scaled S^T [V | 1]
       const uint32_t sW = smem_u32(sm + OutSmem::W), sBaug = smem_u32(sm + OutSmem::BAUG), sAaug = smem_u32(sm + OutSmem::AAUG);
+      const uint32_t sWlo = smem_u32(sm + OutSmem::WLO);
       const uint32_t sPhi = smem_u32(sm + OutSmem::PHI), sKvt = smem_u32(sm + OutSmem::KVT);
       auto issue_logits = [&](int st) {
         const uint32_t sX = smem_u32(sm + OutSmem::X0 + st * TILE_BYTES);
@@ -426,6 +462,10 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         for (int k = 0; k < TC_D / 16; k++)
           mma_bf16(tmem + OUT_COL_LOGITS, smem_desc(sX + 32 * k, 16, 1024, SWZ_128B), smem_desc(sW + 32 * k, 16, 1024, SWZ_128B),
                    ID_LOGITS, k > 0);
+#pragma unroll
+        for (int k = 0; k < TC_D / 16; k++)
+          mma_bf16(tmem + OUT_COL_LOGITS, smem_desc(sX + 32 * k, 16, 1024, SWZ_128B), smem_desc(sWlo + 32 * k, 16, 1024, SWZ_128B),
+                   ID_LOGITS, 1);
         mma_bf16(tmem + OUT_COL_LOGITS, smem_desc(sAaug, 128, 256, SWZ_NONE), smem_desc(sBaug, 128, 256, SWZ_NONE),
                  ID_LOGITS, 1);
         mma_commit(&misc->logits_full);
@@ -522,7 +562,7 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         uint32_t p[4];
 #pragma unroll
         for (int j = 0; j < 4; j++)
-          p[j] = pack_bf16(ex2(__uint_as_float(v[c * 8 + 2 * j]) - mx), ex2(__uint_as_float(v[c * 8 + 2 * j + 1]) - mx));
+          p[j] = pack_f16(ex2(__uint_as_float(v[c * 8 + 2 * j]) - mx), ex2(__uint_as_float(v[c * 8 + 2 * j + 1]) - mx));
         *reinterpret_cast<uint4*>(prow + (c >> 3) * TILE_BYTES + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
       }
       fence_proxy_async_smem();
@@ -580,7 +620,7 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   nsplit = (ktiles + tps - 1) / tps;
   float* partial = ws->take<float>((size_t)BH * 64 * TC_M * TC_NV);
   float* shifts = ws->take<float>((size_t)BH * 64);
-  __nv_bfloat16* kvt = ws->take<__nv_bfloat16>((size_t)BH * TC_NV * TC_M);
+  __half* kvt = ws->take<__half>((size_t)BH * TC_NV * TC_M);
 
   CUtensorMap tmK, tmV, tmQ, tmKVt;
   FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, Lk, dm->d), B, H, Lk, dm->d));

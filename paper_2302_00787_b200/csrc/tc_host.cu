@@ -28,7 +28,10 @@ tc_prep_kernel(const float* __restrict__ prep, float qk_scale, uint8_t* __restri
   const float sw = FS_LOG2E * qk_scale, sc = FS_LOG2E * qk_scale * qk_scale;
   for (int e = tid; e < TC_M * TC_D; e += 256) {
     int m = e / TC_D, k = e % TC_D;
-    *reinterpret_cast<__nv_bfloat16*>(img + IMG_W + tc::sw128_offset(m, k)) = __float2bfloat16_rn(W[e] * sw);
+    const float v = W[e] * sw;
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    *reinterpret_cast<__nv_bfloat16*>(img + IMG_W + tc::sw128_offset(m, k)) = hi;
+    *reinterpret_cast<__nv_bfloat16*>(img + IMG_WLO + tc::sw128_offset(m, k)) = __float2bfloat16_rn(v - __bfloat162float(hi));
   }
   int lo_nonzero = 0;
   for (int e = tid; e < TC_D * TC_D; e += 256) {
@@ -99,7 +102,7 @@ int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int
   return r == CUDA_SUCCESS ? FSHARP_OK : FSHARP_E_CUDA;
 }
 
-// kvt [BH, 80, 256] bf16 -> 3-D map (feature, row, bh), box 64 x 80 x 1, 128-byte swizzle.
+// kvt [BH, 80, 256] fp16 -> 3-D map (feature, row, bh), box 64 x 80 x 1, 128-byte swizzle.
 int make_map_kvt(CUtensorMap* map, const void* base, int BH) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return FSHARP_E_CUDA;
@@ -107,7 +110,7 @@ int make_map_kvt(CUtensorMap* map, const void* base, int BH) {
   cuuint64_t strides[2] = {(cuuint64_t)TC_M * 2, (cuuint64_t)TC_M * TC_NV * 2};
   cuuint32_t box[3] = {64, (cuuint32_t)TC_NV, 1};
   cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? FSHARP_OK : FSHARP_E_CUDA;
