@@ -115,7 +115,7 @@ const char* fsharp_strerror(int code);
 size_t fsharp_stats_doubles(int d);
 /* Doubles per group in the parameter blob:
  *   [A (d*d, symmetric)] [B1 (d*d)] [B2 (d*d)] [C1 (d*d)] [C2 (d*d)]
- *   [logD] [objective] [phi] [5 reserved, zero]
+ *   [logD] [objective] [phi] [Jacobi sweeps spent by the fit] [4 reserved, zero]
  * = 5 d^2 + 8.  objective is the shifted log-variance of Section 3.1 at the
  * optimum (Theorems 4.2 / 4.3); phi is the argument of Lemma A.1 (ADERF, GERF,
  * SADERF; for SDERF the largest eigenvalue of N).  Only A, B, C and logD enter the

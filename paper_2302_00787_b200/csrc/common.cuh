@@ -42,8 +42,8 @@ struct PrepLayout {
   __host__ __device__ size_t Cmat() const { return (size_t)M * d + M + 8; }
   __host__ __device__ size_t total() const { return (size_t)M * d + M + 8 + (size_t)d * d; }
 };
-// PS_BIAS logD - 1/2 log M; PS_AMAX max_m a_m; PS_CSCALAR 1 if C = gamma I; PS_CGAMMA gamma.
-enum { PS_BIAS = 0, PS_AMAX = 1, PS_CSCALAR = 3, PS_CGAMMA = 4 };
+// PS_BIAS logD - 1/2 log M; PS_CSCALAR 1 if C = gamma I; PS_CGAMMA gamma.
+enum { PS_BIAS = 0, PS_CSCALAR = 3, PS_CGAMMA = 4 };
 
 // Kernel ids for the optional per-kernel timing (fsharp_set_timing / fsharp_read_timing).
 enum {

@@ -4,7 +4,7 @@
 
 namespace {
 
-constexpr int FIT_THREADS = 256;
+constexpr int FIT_THREADS = 512;
 constexpr int JACOBI_MAX_SWEEPS = 40;
 
 __device__ __forceinline__ double block_reduce(double v, double* red, int op /*0 sum, 1 max, 2 min*/) {
@@ -31,68 +31,125 @@ __device__ __forceinline__ double lemma_a1(double phi) {
   return -(2.0 * phi + (12.0 * phi + 4.0 * phi * phi) / (1.0 + s)) / 16.0;
 }
 
-// Two-sided cyclic Jacobi with the round-robin ("tournament") ordering: every round
-// rotates d/2 disjoint index pairs at once.  On exit the diagonal of A holds the
-// eigenvalues and the columns of V the eigenvectors.  A: d x d, leading dimension
-// lda; V likewise.  cs: 2*d doubles, pq: 2*d ints, red: FIT_THREADS doubles (shared).
-__device__ void jacobi_eig(double* A, int lda, double* V, int ldv, int d, double* cs, int* pq, double* red) {
-  const int tid = threadIdx.x;
-  const int half = d / 2;
-  for (int e = tid; e < d * d; e += FIT_THREADS) V[(e / d) * ldv + (e % d)] = (e / d == e % d) ? 1.0 : 0.0;
+// Two-sided cyclic Jacobi with the round-robin ("tournament") ordering: every round rotates
+// d/2 disjoint index pairs at once.  On exit the diagonal of A holds the eigenvalues and ROW k
+// of VT the k-th eigenvector.  A: d x d, leading dimension lda; VT likewise (ldvt).
+// d is a power of two (log2d).  sched: the (d-1) x d/2 pairs of all rounds, filled once per
+// block by jacobi_schedule.  cs: 2*d doubles, red: FIT_THREADS doubles (all shared memory).
+//
+// The rotation angle is computed in fp32 (fast divide and square root) and then (c, s) is made
+// orthonormal in fp64: c = rsqrt(1 + t^2), s = t c.  An angle that is only accurate to 1e-7
+// still annihilates a_pq to that relative level and keeps V exactly orthogonal; the sweeps
+// repeat until the off-diagonal mass is below 1e-24 of the total.
+__device__ void jacobi_schedule(ushort2* sched, int d) {
+  const int half = d >> 1;
+  for (int e = threadIdx.x; e < (d - 1) * half; e += FIT_THREADS) {
+    int r = e / half, k = e % half, p, q;
+    if (k == 0) { p = r; q = d - 1; }
+    else { p = (r + k) % (d - 1); q = (r - k + (d - 1)) % (d - 1); }
+    if (p > q) { int t = p; p = q; q = t; }
+    sched[e] = make_ushort2((unsigned short)p, (unsigned short)q);
+  }
   __syncthreads();
+}
+
+__device__ __forceinline__ int jacobi_eig(double* __restrict__ A, int lda, double* __restrict__ VT, int ldvt, int d,
+                                          int log2d, const ushort2* __restrict__ sched, double* __restrict__ cs,
+                                          double* red) {
+  const int tid = threadIdx.x;
+  const int half = d >> 1, items = half << log2d, dm1 = d - 1;
+  for (int e = tid; e < d * d; e += FIT_THREADS) VT[(e >> log2d) * ldvt + (e & dm1)] = ((e >> log2d) == (e & dm1)) ? 1.0 : 0.0;
+  __syncthreads();
+  int sweeps = 0;
   for (int sweep = 0; sweep < JACOBI_MAX_SWEEPS; sweep++) {
     double off = 0.0, tot = 0.0;
     for (int e = tid; e < d * d; e += FIT_THREADS) {
-      int i = e / d, j = e % d;
+      int i = e >> log2d, j = e & dm1;
       double v = A[i * lda + j];
       tot += v * v;
       if (i != j) off += v * v;
     }
     off = block_reduce(off, red, 0);
     tot = block_reduce(tot, red, 0);
-    if (off <= 1e-26 * tot || tot == 0.0) break;
+    if (off <= 1e-24 * tot || tot == 0.0) break;
+    sweeps++;
     for (int r = 0; r < d - 1; r++) {
+      const ushort2* sr = sched + r * half;
       if (tid < half) {
-        int p, q;
-        if (tid == 0) { p = r; q = d - 1; }
-        else { p = (r + tid) % (d - 1); q = (r - tid + (d - 1)) % (d - 1); }
-        if (p > q) { int t = p; p = q; q = t; }
-        double app = A[p * lda + p], aqq = A[q * lda + q], apq = A[p * lda + q];
+        const int p = sr[tid].x, q = sr[tid].y;
+        const double app = A[p * lda + p], aqq = A[q * lda + q], apq = A[p * lda + q];
         double c = 1.0, s = 0.0;
-        if (fabs(apq) > 1e-300) {
-          double tau = (aqq - app) / (2.0 * apq);
-          double t = copysign(1.0, tau) / (fabs(tau) + sqrt(1.0 + tau * tau));
-          c = 1.0 / sqrt(1.0 + t * t);
-          s = t * c;
+        const float num = (float)(aqq - app), den = (float)(2.0 * apq);
+        if (den != 0.f) {
+          const float zeta = __fdividef(num, den);
+          const float tf = __fdividef(copysignf(1.f, zeta), fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f)));
+          if (isfinite(tf)) {
+            const double t = (double)tf;
+            c = rsqrt(fma(t, t, 1.0));
+            s = t * c;
+          }
         }
         cs[2 * tid] = c; cs[2 * tid + 1] = s;
-        pq[2 * tid] = p; pq[2 * tid + 1] = q;
       }
       __syncthreads();
-      for (int e = tid; e < half * d; e += FIT_THREADS) {        // A <- A J, V <- V J
-        int k = e / d, row = e % d;
-        int p = pq[2 * k], q = pq[2 * k + 1];
-        double c = cs[2 * k], s = cs[2 * k + 1];
-        double x = A[row * lda + p], y = A[row * lda + q];
-        A[row * lda + p] = c * x - s * y;
-        A[row * lda + q] = s * x + c * y;
-        x = V[row * ldv + p]; y = V[row * ldv + q];
-        V[row * ldv + p] = c * x - s * y;
-        V[row * ldv + q] = s * x + c * y;
+      // A <- A J (columns p, q of every row) and VT <- J^T VT (rows p, q): the rotations of a
+      // round touch disjoint elements, so each thread loads a batch first and stores afterwards
+      for (int e0 = tid; e0 < items; e0 += 4 * FIT_THREADS) {
+        double xa[4], ya[4], xv[4], yv[4], cc[4], ss[4];
+        int ia[4], ja[4], iv[4], jv[4];
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+          const int e = e0 + u * FIT_THREADS;
+          if (e < items) {
+            const int k = e >> log2d, row = e & dm1;
+            const int p = sr[k].x, q = sr[k].y;
+            cc[u] = cs[2 * k]; ss[u] = cs[2 * k + 1];
+            ia[u] = row * lda + p; ja[u] = row * lda + q;
+            iv[u] = p * ldvt + row; jv[u] = q * ldvt + row;
+            xa[u] = A[ia[u]]; ya[u] = A[ja[u]];
+            xv[u] = VT[iv[u]]; yv[u] = VT[jv[u]];
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+          const int e = e0 + u * FIT_THREADS;
+          if (e < items) {
+            A[ia[u]] = cc[u] * xa[u] - ss[u] * ya[u];
+            A[ja[u]] = ss[u] * xa[u] + cc[u] * ya[u];
+            VT[iv[u]] = cc[u] * xv[u] - ss[u] * yv[u];
+            VT[jv[u]] = ss[u] * xv[u] + cc[u] * yv[u];
+          }
+        }
       }
       __syncthreads();
-      for (int e = tid; e < half * d; e += FIT_THREADS) {        // A <- J^T A
-        int k = e / d, col = e % d;
-        int p = pq[2 * k], q = pq[2 * k + 1];
-        double c = cs[2 * k], s = cs[2 * k + 1];
-        double x = A[p * lda + col], y = A[q * lda + col];
-        A[p * lda + col] = c * x - s * y;
-        A[q * lda + col] = s * x + c * y;
+      for (int e0 = tid; e0 < items; e0 += 4 * FIT_THREADS) {   // A <- J^T A (rows p, q of every column)
+        double xa[4], ya[4], cc[4], ss[4];
+        int ia[4], ja[4];
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+          const int e = e0 + u * FIT_THREADS;
+          if (e < items) {
+            const int k = e >> log2d, col = e & dm1;
+            const int p = sr[k].x, q = sr[k].y;
+            cc[u] = cs[2 * k]; ss[u] = cs[2 * k + 1];
+            ia[u] = p * lda + col; ja[u] = q * lda + col;
+            xa[u] = A[ia[u]]; ya[u] = A[ja[u]];
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+          const int e = e0 + u * FIT_THREADS;
+          if (e < items) {
+            A[ia[u]] = cc[u] * xa[u] - ss[u] * ya[u];
+            A[ja[u]] = ss[u] * xa[u] + cc[u] * ya[u];
+          }
+        }
       }
       __syncthreads();
     }
   }
   __syncthreads();
+  return sweeps;
 }
 
 struct FitArgs {
@@ -105,6 +162,7 @@ struct FitArgs {
   int* status;
 };
 
+template <bool V_IN_SMEM>
 __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
   extern __shared__ double sm[];
   const int d = a.d, tid = threadIdx.x, g = blockIdx.x;
@@ -116,15 +174,18 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
   double* gs = a.scratch + (size_t)g * 4 * d * d;
 
   double* As = sm;                                   // d*(d+1)
-  double* Vs = a.v_in_smem ? As + d * lda : gs;      // eigenvectors
-  const int ldv = a.v_in_smem ? lda : d;
-  double* vec = As + d * lda + (a.v_in_smem ? d * lda : 0);
+  double* Vs = V_IN_SMEM ? As + d * lda : gs;        // eigenvectors, one per ROW
+  const int ldv = V_IN_SMEM ? lda : d;
+  double* vec = As + d * lda + (V_IN_SMEM ? d * lda : 0);
   double* lam = vec;             // [d]
   double* aux = vec + d;         // [d]
   double* cs = vec + 2 * d;      // [2d]
   double* red = vec + 4 * d;     // [FIT_THREADS]
-  int* pq = reinterpret_cast<int*>(red + FIT_THREADS);   // [2d]
-  int* perm = pq + 2 * d;                                 // [d]
+  int* perm = reinterpret_cast<int*>(red + FIT_THREADS);          // [d]
+  ushort2* sched = reinterpret_cast<ushort2*>(perm + d);          // [(d-1) * d/2]
+  int log2d = 0;
+  while ((1 << log2d) < d) log2d++;
+  if (a.variant == FSHARP_SDERF || a.variant == FSHARP_ADERF) jacobi_schedule(sched, d);
 
   const double* M1 = st + sl.M(1);
   const double* M2 = st + sl.M(2);
@@ -157,6 +218,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
   double* tail = out + pl.tail();
   double logD = 0.0, obj = 0.0, phi = 0.0;
   bool violated = false;
+  int nsweeps = 0;
 
   if (a.variant == FSHARP_POSRF || a.variant == FSHARP_GERF) {
     const double S = t1 + t2 + 2.0 * mm;
@@ -199,7 +261,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
       As[i * lda + j] = M1[e] + M2[e] + mu4[i] * mu5[j] + mu5[i] * mu4[j] + (i == j ? rg1 + rg2 : 0.0);
     }
     __syncthreads();
-    jacobi_eig(As, lda, Vs, ldv, d, cs, pq, red);
+    nsweeps += jacobi_eig(As, lda, Vs, ldv, d, log2d, sched, cs, red);
     for (int i = tid; i < d; i += FIT_THREADS) {
       double li = As[i * lda + i];
       int rank = 0;
@@ -224,7 +286,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
     for (int e = tid; e < d * d; e += FIT_THREADS) {
       int l = e / d, j = e % d;
       double dg = (l == j) ? 1.0 : 0.0;
-      double b = sqrt(1.0 - 4.0 * aux[l]) * Vs[j * ldv + perm[l]];     // B = (I-4A)^1/2 Q3^T
+      double b = sqrt(1.0 - 4.0 * aux[l]) * Vs[perm[l] * ldv + j];     // B = (I-4A)^1/2 Q3^T
       oA[e] = aux[l] * dg; oB1[e] = b; oB2[e] = b; oC1[e] = -0.5 * dg; oC2[e] = -0.5 * dg;
     }
     logD = 0.25 * sl_log;
@@ -239,7 +301,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
       As[i * lda + j] = M1[e] + (i == j ? rg1 : 0.0);
     }
     __syncthreads();
-    jacobi_eig(As, lda, Vs, ldv, d, cs, pq, red);
+    nsweeps += jacobi_eig(As, lda, Vs, ldv, d, log2d, sched, cs, red);
     double lmin = 1e300, lmax = 0.0;
     for (int i = tid; i < d; i += FIT_THREADS) {
       double li = As[i * lda + i];
@@ -249,7 +311,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
     lmax = block_reduce(lmax, red, 1);
     if (!(lmin > 1e-12 * lmax)) violated = true;
     for (int i = tid; i < d; i += FIT_THREADS) lam[i] = fmax(As[i * lda + i], 1e-300 + 1e-12 * lmax);
-    for (int e = tid; e < d * d; e += FIT_THREADS) Q1g[e] = Vs[(e / d) * ldv + (e % d)];
+    for (int e = tid; e < d * d; e += FIT_THREADS) Q1g[e] = Vs[(e % d) * ldv + (e / d)];   // Q1[i][l]
     __syncthreads();
     // T1 = M2 Q1 L1^1/2
     for (int e = tid; e < d * d; e += FIT_THREADS) {
@@ -272,7 +334,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
       As[c * lda + r] = v;
     }
     __syncthreads();
-    jacobi_eig(As, lda, Vs, ldv, d, cs, pq, red);     // eigenvalues Sigma^2, eigenvectors U
+    nsweeps += jacobi_eig(As, lda, Vs, ldv, d, log2d, sched, cs, red);     // eigenvalues Sigma^2, eigenvectors U
     double smin = 1e300, smax = 0.0, ssum = 0.0;
     for (int l = tid; l < d; l += FIT_THREADS) {
       double sg = sqrt(fmax(As[l * lda + l], 0.0));
@@ -284,7 +346,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
     ssum = block_reduce(ssum, red, 0);
     if (!(smin > 1e-12 * smax)) violated = true;
     for (int l = tid; l < d; l += FIT_THREADS) aux[l] = fmax(aux[l], 1e-300 + 1e-12 * smax);
-    for (int e = tid; e < d * d; e += FIT_THREADS) Ug[e] = Vs[(e / d) * ldv + (e % d)];
+    for (int e = tid; e < d * d; e += FIT_THREADS) Ug[e] = Vs[(e % d) * ldv + (e / d)];     // U[i][l]
     __syncthreads();
     const double mu3 = mm / d;
     phi = 2.0 * ssum / d + 2.0 * mu3;
@@ -322,14 +384,15 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
     tail[PT_LOGD] = logD;
     tail[PT_OBJ] = obj;
     tail[PT_PHI] = phi;
-    for (int i = 3; i < 8; i++) tail[i] = 0.0;
+    tail[3] = (double)nsweeps;     // Jacobi sweeps spent (diagnostic)
+    for (int i = 4; i < 8; i++) tail[i] = 0.0;
   }
   if (violated) atomicExch(a.status, FSHARP_E_CONSTRAINT);
 }
 
 size_t fit_smem_bytes(int d, int v_in_smem) {
   size_t dbl = (size_t)d * (d + 1) * (v_in_smem ? 2 : 1) + 4 * (size_t)d + FIT_THREADS;
-  return dbl * sizeof(double) + 3 * (size_t)d * sizeof(int);
+  return dbl * sizeof(double) + (size_t)d * sizeof(int) + (size_t)(d - 1) * (d / 2) * sizeof(ushort2);
 }
 
 }  // namespace
@@ -344,9 +407,11 @@ int fs_run_fit(fsharp_ctx* ctx, const double* stats, int G, int d, int variant, 
   a.v_in_smem = d <= 64 ? 1 : 0;
   a.status = ctx->d_status;
   size_t smem = fit_smem_bytes(d, a.v_in_smem);
-  FS_CUDA_OK(cudaFuncSetAttribute(fit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  if (a.v_in_smem) FS_CUDA_OK(cudaFuncSetAttribute(fit_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  else FS_CUDA_OK(cudaFuncSetAttribute(fit_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   FS_TIME_BEGIN(ctx, FS_K_FIT);
-  fit_kernel<<<G, FIT_THREADS, smem, ctx->stream>>>(a);
+  if (a.v_in_smem) fit_kernel<true><<<G, FIT_THREADS, smem, ctx->stream>>>(a);
+  else fit_kernel<false><<<G, FIT_THREADS, smem, ctx->stream>>>(a);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;

@@ -20,6 +20,30 @@
 using namespace tc;
 using namespace tcl;
 
+#ifdef FS_TRACE
+__device__ long long fs_trace_buf[8192];
+__device__ int fs_trace_n;
+#define TRACE(tag)                                                        \
+  do {                                                                    \
+    if (blockIdx.x == 0 && blockIdx.y == 0) {                             \
+      int _i = atomicAdd(&fs_trace_n, 1);                                 \
+      if (_i < 4096) { fs_trace_buf[2 * _i] = (tag); fs_trace_buf[2 * _i + 1] = clock64(); } \
+    }                                                                     \
+  } while (0)
+extern "C" int fsharp_debug_read_trace(long long* out, int cap) {
+  int n = 0;
+  cudaMemcpyFromSymbol(&n, fs_trace_n, sizeof(int));
+  if (n > cap) n = cap;
+  if (n > 4096) n = 4096;
+  cudaMemcpyFromSymbol(out, fs_trace_buf, (size_t)n * 2 * sizeof(long long));
+  int zero = 0;
+  cudaMemcpyToSymbol(fs_trace_n, &zero, sizeof(int));
+  return n;
+}
+#else
+#define TRACE(tag) do { } while (0)
+#endif
+
 namespace {
 
 // ------------------------------------------------------------------------------------------
@@ -47,7 +71,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
              const uint8_t* __restrict__ images, const int* __restrict__ img_flags, int H, int pool, int L,
              int tiles_per_split, int nsplit, float* __restrict__ partial, float* __restrict__ shifts,
-             int* __restrict__ status) {
+             int* __restrict__ pmax, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   KvMisc* misc = reinterpret_cast<KvMisc*>(sm + KvSmem::MISC);
@@ -110,6 +134,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       for (int it = 0; it < ntiles; it++) {
         const int st = it & 1;
         if (!mbar_wait(&misc->empty[st], ((it >> 1) & 1) ^ 1, abortp, status)) break;
+        TRACE(100 + it * 1000);
         mbar_expect_tx(&misc->full[st], 2 * TILE_BYTES);
         tma_load_4d(sm + KvSmem::X0 + st * TILE_BYTES, &tmK, &misc->full[st], 0, (tile0 + it) * TILE, h, b);
         tma_load_4d(sm + KvSmem::V0 + st * TILE_BYTES, &tmV, &misc->full[st], 0, (tile0 + it) * TILE, h, b);
@@ -129,28 +154,31 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       const uint32_t sW = smem_u32(sm + KvSmem::W), sChi = smem_u32(sm + KvSmem::CHI), sClo = smem_u32(sm + KvSmem::CLO);
       const uint32_t sBaug = smem_u32(sm + KvSmem::BAUG), sAaug = smem_u32(sm + KvSmem::AAUG);
       const uint32_t sPhi = smem_u32(sm + KvSmem::PHI), sOnesT = smem_u32(sm + KvSmem::ONEST);
+      // descriptors are built once; inside the loops each MMA costs one add per operand
+      const uint64_t dX0 = smem_desc(smem_u32(sm + KvSmem::X0), 16, 1024, SWZ_128B);
+      const uint64_t dV0 = smem_desc(smem_u32(sm + KvSmem::V0), 16, 1024, SWZ_128B);
+      const uint64_t dW = smem_desc(sW, 16, 1024, SWZ_128B), dWlo = smem_desc(sWlo, 16, 1024, SWZ_128B);
+      const uint64_t dChi = smem_desc(sChi, 16, 1024, SWZ_128B), dClo = smem_desc(sClo, 16, 1024, SWZ_128B);
+      const uint64_t dAaug = smem_desc(sAaug, 128, 256, SWZ_NONE), dBaug = smem_desc(sBaug, 128, 256, SWZ_NONE);
+      const uint64_t dPhi = smem_desc(sPhi, TILE_BYTES, 1024, SWZ_128B);
+      const uint64_t dOnesT = smem_desc(sOnesT, 16, 1024, SWZ_128B);
       auto issue_logits = [&](int st) {
-        const uint32_t sX = smem_u32(sm + KvSmem::X0 + st * TILE_BYTES);
+        const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
 #pragma unroll
         for (int k = 0; k < TC_D / 16; k++)
-          mma_bf16(tmem + KV_COL_LOGITS, smem_desc(sX + 32 * k, 16, 1024, SWZ_128B), smem_desc(sW + 32 * k, 16, 1024, SWZ_128B),
-                   ID_LOGITS, k > 0);
+          mma_bf16(tmem + KV_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dW, 32 * k), ID_LOGITS, k > 0);
 #pragma unroll
         for (int k = 0; k < TC_D / 16; k++)
-          mma_bf16(tmem + KV_COL_LOGITS, smem_desc(sX + 32 * k, 16, 1024, SWZ_128B), smem_desc(sWlo + 32 * k, 16, 1024, SWZ_128B),
-                   ID_LOGITS, 1);
-        mma_bf16(tmem + KV_COL_LOGITS, smem_desc(sAaug, 128, 256, SWZ_NONE), smem_desc(sBaug, 128, 256, SWZ_NONE),
-                 ID_LOGITS, 1);
+          mma_bf16(tmem + KV_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dWlo, 32 * k), ID_LOGITS, 1);
+        mma_bf16(tmem + KV_COL_LOGITS, dAaug, dBaug, ID_LOGITS, 1);
         if (cdense) {
 #pragma unroll
           for (int k = 0; k < TC_D / 16; k++)
-            mma_bf16(tmem + KV_COL_T, smem_desc(sX + 32 * k, 16, 1024, SWZ_128B), smem_desc(sChi + 32 * k, 16, 1024, SWZ_128B),
-                     ID_T, k > 0);
+            mma_bf16(tmem + KV_COL_T, desc_advance(dX, 32 * k), desc_advance(dChi, 32 * k), ID_T, k > 0);
           if (clo) {
 #pragma unroll
             for (int k = 0; k < TC_D / 16; k++)
-              mma_bf16(tmem + KV_COL_T, smem_desc(sX + 32 * k, 16, 1024, SWZ_128B),
-                       smem_desc(sClo + 32 * k, 16, 1024, SWZ_128B), ID_T, 1);
+              mma_bf16(tmem + KV_COL_T, desc_advance(dX, 32 * k), desc_advance(dClo, 32 * k), ID_T, 1);
           }
         }
         mma_commit(&misc->logits_full);
@@ -165,25 +193,31 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         const int st = it & 1;
         if (it + 1 < ntiles) {
           if (!mbar_wait(&misc->full[st ^ 1], ((it + 1) >> 1) & 1, abortp, status)) break;
+          TRACE(200 + it * 1000);
           if (!mbar_wait(&misc->logits_free, it & 1, abortp, status)) break;
+          TRACE(201 + it * 1000);
           tcgen05_fence_after();
           issue_logits(st ^ 1);
+          TRACE(202 + it * 1000);
         }
         if (!mbar_wait(&misc->phi_full, it & 1, abortp, status)) break;
+        TRACE(203 + it * 1000);
         tcgen05_fence_after();
-        const uint32_t sV = smem_u32(sm + KvSmem::V0 + st * TILE_BYTES);
+        const uint64_t dV = desc_advance(dV0, st * TILE_BYTES);
+        const uint32_t acc0 = it > 0 ? 1u : 0u;
 #pragma unroll
         for (int hh = 0; hh < 2; hh++)
 #pragma unroll
           for (int k = 0; k < TILE / 16; k++) {
-            const uint64_t da = smem_desc(sPhi + hh * 2 * TILE_BYTES + k * 2048, TILE_BYTES, 1024, SWZ_128B);
-            const uint32_t acc = (it > 0 || k > 0) ? 1u : 0u;
-            mma_bf16(tmem + KV_COL_ACC + hh * TC_NV, da, smem_desc(sV + k * 2048, 16, 1024, SWZ_128B), ID_KV, acc);
-            mma_bf16(tmem + KV_COL_ACC + hh * TC_NV + TC_DV, da,
-                     smem_desc(sOnesT + (k >> 2) * 2048 + (k & 3) * 32, 16, 1024, SWZ_128B), ID_KV1, acc);
+            const uint64_t da = desc_advance(dPhi, hh * 2 * TILE_BYTES + k * 2048);
+            const uint32_t acc = k > 0 ? 1u : acc0;
+            mma_bf16(tmem + KV_COL_ACC + hh * TC_NV, da, desc_advance(dV, k * 2048), ID_KV, acc);
+            mma_bf16(tmem + KV_COL_ACC + hh * TC_NV + TC_DV, da, desc_advance(dOnesT, (k >> 2) * 2048 + (k & 3) * 32),
+                     ID_KV1, acc);
           }
         mma_commit(&misc->phi_free);
         mma_commit(&misc->empty[st]);
+        TRACE(204 + it * 1000);
       }
     }
   } else {
@@ -196,7 +230,9 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     for (int it = 0; it < ntiles && alive; it++) {
       const int st = it & 1;
       if (!mbar_wait(&misc->full[st], (it >> 1) & 1, abortp, status, false)) { alive = false; break; }
+      if (threadIdx.x == 0) TRACE(300 + it * 1000);
       if (!mbar_wait(&misc->logits_full, it & 1, abortp, status, false)) { alive = false; break; }
+      if (threadIdx.x == 0) TRACE(301 + it * 1000);
       __syncwarp();
       tcgen05_fence_after();
       // c_j = x_j^T C x_j in log2 units
@@ -216,17 +252,21 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         }
         if (cdense) {
 #pragma unroll
+          float part[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
           for (int c = 0; c < TC_D / 16; c++) {
             uint32_t t[16];
             tmem_ld16(lane_addr + KV_COL_T + c * 16, t);
             tmem_wait_ld();
 #pragma unroll
-            for (int j = 0; j < 16; j++) cj = fmaf(__uint_as_float(t[j]), xv[c * 16 + j], cj);
+            for (int j = 0; j < 16; j++) part[j & 3] = fmaf(__uint_as_float(t[j]), xv[c * 16 + j], part[j & 3]);
           }
+          cj = (part[0] + part[1]) + (part[2] + part[3]);
         } else {
+          float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-          for (int j = 0; j < TC_D; j++) cj = fmaf(xv[j], xv[j], cj);
-          cj *= gamma2;
+          for (int j = 0; j < TC_D; j++) part[j & 3] = fmaf(xv[j], xv[j], part[j & 3]);
+          cj = ((part[0] + part[1]) + (part[2] + part[3])) * gamma2;
         }
       }
       uint32_t v[128];
@@ -240,14 +280,16 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       tmem_wait_ld();
       tcgen05_fence_before();
       mbar_arrive(&misc->logits_free);
+      if (threadIdx.x == 0) TRACE(302 + it * 1000);
       const bool valid = (tile0 + it) * TILE + row < L;
-      float mx = -INFINITY;
+      float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
       for (int i = 0; i < 128; i++) {
         float f = __uint_as_float(v[i]) + cj;
         v[i] = __float_as_uint(f);
-        mx = fmaxf(mx, f);
+        mxp[i & 3] = fmaxf(mxp[i & 3], f);
       }
+      float mx = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
       if (!valid) mx = -INFINITY;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
@@ -255,6 +297,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       if (threadIdx.x == 0) misc->tile_max[(it + 1) % 3] = f2ord(-INFINITY);   // next tile's slot; idle since tile it-2
       named_bar_sync(1, EPI_THREADS);
       const float t = ord2f(misc->tile_max[it % 3]);
+      if (threadIdx.x == 0) TRACE(303 + it * 1000);
       const float s_old = s;
       bool rescale = false;
       if (!have || t > s + SHIFT_HEADROOM_LOG2) {
@@ -265,6 +308,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       if (it > 0) {
         if (!mbar_wait(&misc->phi_free, (it - 1) & 1, abortp, status, false)) { alive = false; break; }
       }
+      if (threadIdx.x == 0) TRACE(304 + it * 1000);
       __syncwarp();
       if (rescale) {
         // the running shift moved: bring the accumulated S^T [V | 1] to the new one
@@ -295,21 +339,30 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       fence_proxy_async_smem();
       tcgen05_fence_before();
       mbar_arrive(&misc->phi_full);
+      if (threadIdx.x == 0) TRACE(305 + it * 1000);
     }
     // write this split's partial S^T [V | 1] (fp32) and its shift
     if (alive && ntiles > 0 && mbar_wait(&misc->phi_free, (ntiles - 1) & 1, abortp, status, false)) {
       __syncwarp();
       tcgen05_fence_after();
       float* out = partial + (((size_t)bh * nsplit + split) * TC_M + hf * 128 + row) * TC_NV;
+      float amax = 0.f;
 #pragma unroll
       for (int c = 0; c < TC_NV / 16; c++) {
         uint32_t a[16];
         tmem_ld16(lane_addr + KV_COL_ACC + hf * TC_NV + c * 16, a);
         tmem_wait_ld();
 #pragma unroll
+        for (int j = 0; j < 16; j++)
+          if (c * 16 + j <= TC_DV) amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
+#pragma unroll
         for (int j = 0; j < 4; j++)
           reinterpret_cast<uint4*>(out + c * 16)[j] = make_uint4(a[4 * j], a[4 * j + 1], a[4 * j + 2], a[4 * j + 3]);
       }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+      // largest magnitude of this partial (non-negative floats order like their bit patterns)
+      if (lane == 0) atomicMax(&pmax[(size_t)bh * nsplit + split], __float_as_int(amax));
       if (threadIdx.x == 0) shifts[(size_t)bh * nsplit + split] = s;
     }
   }
@@ -324,39 +377,38 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 // ------------------------------------------------------------------------------------------
 // merge of the key-side partials of one (batch, head): common shift, sum, transpose, bf16
 // ------------------------------------------------------------------------------------------
+constexpr int MERGE_SLICES = 8;
 __global__ void __launch_bounds__(256)
-tc_merge_kernel(const float* __restrict__ partial, const float* __restrict__ shifts, int nsplit,
-                __half* __restrict__ kvt) {
-  __shared__ float red[256];
-  const int bh = blockIdx.x;
-  float smax = -INFINITY;
-  for (int p = 0; p < nsplit; p++) smax = fmaxf(smax, shifts[(size_t)bh * nsplit + p]);
+tc_merge_kernel(const float* __restrict__ partial, const float* __restrict__ shifts, const int* __restrict__ pmax,
+                int nsplit, __half* __restrict__ kvt) {
+  __shared__ float fac[64];
+  __shared__ float scale_s;
+  const int bh = blockIdx.y;
+  if (threadIdx.x == 0) {
+    float smax = -INFINITY;
+    for (int p = 0; p < nsplit; p++) smax = fmaxf(smax, shifts[(size_t)bh * nsplit + p]);
+    // fp16 has a narrow range: scale the whole (batch, head) by a power of two (it cancels in
+    // num / den) so that the bound sum_p 2^(s_p - smax) max|partial_p| lands near 2^14
+    float bound = 0.f;
+    for (int p = 0; p < nsplit; p++) {
+      fac[p] = exp2f(shifts[(size_t)bh * nsplit + p] - smax);
+      bound = fmaf(fac[p], __int_as_float(pmax[(size_t)bh * nsplit + p]), bound);
+    }
+    int ex = 0;
+    if (bound > 0.f && isfinite(bound)) frexpf(bound, &ex);
+    scale_s = exp2f((float)(14 - ex));
+  }
+  __syncthreads();
+  const float scale = scale_s;
   const float* base = partial + (size_t)bh * nsplit * TC_M * TC_NV;
   __half* out = kvt + (size_t)bh * TC_NV * TC_M;
-  auto merged = [&](int e) {
-    float acc = 0.f;
-    for (int p = 0; p < nsplit; p++)
-      acc = fmaf(base[(size_t)p * TC_M * TC_NV + e], exp2f(shifts[(size_t)bh * nsplit + p] - smax), acc);
-    return acc;
-  };
-  // fp16 has a narrow range: scale the whole (batch, head) by a power of two (it cancels in
-  // num / den) so that the largest magnitude lands near 2^14
-  float mx = 0.f;
-  for (int e = threadIdx.x; e < TC_M * TC_NV; e += 256)
-    if (e % TC_NV <= TC_DV) mx = fmaxf(mx, fabsf(merged(e)));
-  red[threadIdx.x] = mx;
-  __syncthreads();
-  for (int s = 128; s > 0; s >>= 1) {
-    if (threadIdx.x < s) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + s]);
-    __syncthreads();
-  }
-  mx = red[0];
-  int ex = 0;
-  if (mx > 0.f && isfinite(mx)) frexpf(mx, &ex);
-  const float scale = exp2f((float)(14 - ex));
-  for (int e = threadIdx.x; e < TC_M * TC_NV; e += 256) {
+  constexpr int PER = TC_M * TC_NV / MERGE_SLICES;
+  for (int e = blockIdx.x * PER + threadIdx.x; e < (blockIdx.x + 1) * PER; e += 256) {
     const int m = e / TC_NV, n = e % TC_NV;
-    out[(size_t)n * TC_M + m] = __float2half_rn(n <= TC_DV ? merged(e) * scale : 0.f);
+    float acc = 0.f;
+    if (n <= TC_DV)
+      for (int p = 0; p < nsplit; p++) acc = fmaf(base[(size_t)p * TC_M * TC_NV + e], fac[p], acc);
+    out[(size_t)n * TC_M + m] = __float2half_rn(acc * scale);
   }
 }
 
@@ -456,18 +508,19 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       const uint32_t sW = smem_u32(sm + OutSmem::W), sBaug = smem_u32(sm + OutSmem::BAUG), sAaug = smem_u32(sm + OutSmem::AAUG);
       const uint32_t sWlo = smem_u32(sm + OutSmem::WLO);
       const uint32_t sPhi = smem_u32(sm + OutSmem::PHI), sKvt = smem_u32(sm + OutSmem::KVT);
+      const uint64_t dX0 = smem_desc(smem_u32(sm + OutSmem::X0), 16, 1024, SWZ_128B);
+      const uint64_t dW = smem_desc(sW, 16, 1024, SWZ_128B), dWlo = smem_desc(sWlo, 16, 1024, SWZ_128B);
+      const uint64_t dAaug = smem_desc(sAaug, 128, 256, SWZ_NONE), dBaug = smem_desc(sBaug, 128, 256, SWZ_NONE);
+      const uint64_t dPhi = smem_desc(sPhi, 16, 1024, SWZ_128B), dKvt = smem_desc(sKvt, 16, 1024, SWZ_128B);
       auto issue_logits = [&](int st) {
-        const uint32_t sX = smem_u32(sm + OutSmem::X0 + st * TILE_BYTES);
+        const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
 #pragma unroll
         for (int k = 0; k < TC_D / 16; k++)
-          mma_bf16(tmem + OUT_COL_LOGITS, smem_desc(sX + 32 * k, 16, 1024, SWZ_128B), smem_desc(sW + 32 * k, 16, 1024, SWZ_128B),
-                   ID_LOGITS, k > 0);
+          mma_bf16(tmem + OUT_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dW, 32 * k), ID_LOGITS, k > 0);
 #pragma unroll
         for (int k = 0; k < TC_D / 16; k++)
-          mma_bf16(tmem + OUT_COL_LOGITS, smem_desc(sX + 32 * k, 16, 1024, SWZ_128B), smem_desc(sWlo + 32 * k, 16, 1024, SWZ_128B),
-                   ID_LOGITS, 1);
-        mma_bf16(tmem + OUT_COL_LOGITS, smem_desc(sAaug, 128, 256, SWZ_NONE), smem_desc(sBaug, 128, 256, SWZ_NONE),
-                 ID_LOGITS, 1);
+          mma_bf16(tmem + OUT_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dWlo, 32 * k), ID_LOGITS, 1);
+        mma_bf16(tmem + OUT_COL_LOGITS, dAaug, dBaug, ID_LOGITS, 1);
         mma_commit(&misc->logits_full);
         mma_commit(&misc->empty[st]);
       };
@@ -491,8 +544,8 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         for (int fb = 0; fb < TC_M / 64; fb++)
 #pragma unroll
           for (int k = 0; k < 4; k++)
-            mma_bf16(tmem + OUT_COL_OUT + (it & 1) * TC_NV, smem_desc(sPhi + fb * TILE_BYTES + 32 * k, 16, 1024, SWZ_128B),
-                     smem_desc(sKvt + fb * KVT_BLOCK_BYTES + 32 * k, 16, 1024, SWZ_128B), ID_OUT, (fb > 0 || k > 0) ? 1u : 0u);
+            mma_bf16(tmem + OUT_COL_OUT + (it & 1) * TC_NV, desc_advance(dPhi, fb * TILE_BYTES + 32 * k),
+                     desc_advance(dKvt, fb * KVT_BLOCK_BYTES + 32 * k), ID_OUT, (fb > 0 || k > 0) ? 1u : 0u);
         mma_commit(&misc->phi_free);
         mma_commit(&misc->out_full[it & 1]);
       }
@@ -546,9 +599,10 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       tmem_wait_ld();
       tcgen05_fence_before();
       mbar_arrive(&misc->logits_free);
-      float mx = -INFINITY;
+      float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int i = 0; i < 128; i++) mx = fmaxf(mx, __uint_as_float(v[i]));
+      for (int i = 0; i < 128; i++) mxp[i & 3] = fmaxf(mxp[i & 3], __uint_as_float(v[i]));
+      float mx = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
       float* rm = rowmax + (it & 1) * 2 * TILE;
       rm[hf * TILE + row] = mx;
       named_bar_sync(1, EPI_THREADS);
@@ -594,12 +648,29 @@ size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
 int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
                 const float* prep, void* Y, WsAlloc* ws);
 
+// Splits `tiles` tiles of each of `units` independent units into blocks of equal tile count so that
+// (waves of blocks on `sms` SMs) x (tiles per block + fixed overhead) is smallest; ties go to fewer blocks.
+static int pick_split(int units, int tiles, int sms, int max_split, int* tiles_per_split) {
+  int best = 1, best_cost = 0x7fffffff, best_tps = tiles;
+  for (int ns = 1; ns <= tiles && ns <= max_split; ns++) {
+    int tps = (tiles + ns - 1) / ns;
+    int real = (tiles + tps - 1) / tps;
+    if (real != ns) continue;
+    long long blocks = (long long)units * ns;
+    int waves = (int)((blocks + sms - 1) / sms);
+    int cost = waves * (tps + 4);    // a block's fill and drain cost about as much as four tiles
+    if (cost < best_cost) { best_cost = cost; best = ns; best_tps = tps; }
+  }
+  *tiles_per_split = best_tps;
+  return best;
+}
+
 size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
   const size_t BH = (size_t)dm->B * dm->H;
   const size_t G = fs_groups(dm);
   const size_t max_split = 64;
   return ws_round(G * 2 * IMG_BYTES) + ws_round(G * 2 * FLAG_WORDS * 4 + 64) +
-         ws_round(BH * max_split * TC_M * TC_NV * 4) + ws_round(BH * max_split * 4) + ws_round(BH * TC_NV * TC_M * 2);
+         ws_round(BH * max_split * TC_M * TC_NV * 4) + 2 * ws_round(BH * max_split * 4) + ws_round(BH * TC_NV * TC_M * 2);
 }
 
 int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
@@ -610,16 +681,14 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   int* flags = ws->take<int>((size_t)G * 2 * FLAG_WORDS + 16);
   FS_TRY(fs_tc_prep(ctx, prep, G, qk_scale, images, flags));
 
-  // key side: splits of the key range so that about one block per SM is busy
+  // key side: the split of the key range that minimises (waves of blocks) x (tiles per block)
   const int ktiles = (Lk + TILE - 1) / TILE;
-  int nsplit = (ctx->sm_count + BH - 1) / BH;
-  if (nsplit > ktiles) nsplit = ktiles;
-  if (nsplit > 64) nsplit = 64;
-  if (nsplit < 1) nsplit = 1;
-  int tps = (ktiles + nsplit - 1) / nsplit;
-  nsplit = (ktiles + tps - 1) / tps;
+  int tps = 0;
+  int nsplit = pick_split(BH, ktiles, ctx->sm_count, 64, &tps);
   float* partial = ws->take<float>((size_t)BH * 64 * TC_M * TC_NV);
   float* shifts = ws->take<float>((size_t)BH * 64);
+  int* pmax = ws->take<int>((size_t)BH * 64);
+  FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * 64 * sizeof(int), ctx->stream));
   __half* kvt = ws->take<__half>((size_t)BH * TC_NV * TC_M);
 
   CUtensorMap tmK, tmV, tmQ, tmKVt;
@@ -632,20 +701,17 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   FS_CUDA_OK(cudaFuncSetAttribute(tc_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OutSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_KV);
   tc_kv_kernel<<<dim3(nsplit, BH), TC_THREADS, KvSmem::TOTAL + 1024, ctx->stream>>>(
-      tmK, tmV, images, flags, H, dm->pool, Lk, tps, nsplit, partial, shifts, ctx->d_status);
+      tmK, tmV, images, flags, H, dm->pool, Lk, tps, nsplit, partial, shifts, pmax, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   FS_TIME_BEGIN(ctx, FS_K_TC_MERGE);
-  tc_merge_kernel<<<BH, 256, 0, ctx->stream>>>(partial, shifts, nsplit, kvt);
+  tc_merge_kernel<<<dim3(MERGE_SLICES, BH), 256, 0, ctx->stream>>>(partial, shifts, pmax, nsplit, kvt);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
 
   const int qtiles = (Lq + TILE - 1) / TILE;
-  int qsplit = (ctx->sm_count + BH - 1) / BH;
-  if (qsplit > qtiles) qsplit = qtiles;
-  if (qsplit < 1) qsplit = 1;
-  int qtps = (qtiles + qsplit - 1) / qsplit;
-  qsplit = (qtiles + qtps - 1) / qtps;
+  int qtps = 0;
+  int qsplit = pick_split(BH, qtiles, ctx->sm_count, 1 << 20, &qtps);
   FS_TIME_BEGIN(ctx, FS_K_TC_OUT);
   tc_out_kernel<<<dim3(qsplit, BH), TC_THREADS, OutSmem::TOTAL + 1024, ctx->stream>>>(
       tmQ, tmKVt, images, H, dm->pool, Lq, qtps, (__nv_bfloat16*)Y, fs_addr(dm->y_stride, H, Lq, dm->dv), ctx->d_status);
