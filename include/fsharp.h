@@ -55,7 +55,8 @@ enum {
   FSHARP_E_CONSTRAINT = -6, /* Theorem 4.1 / 4.2 preconditions violated (device-detected) */
   FSHARP_E_NONFINITE = -7,  /* NaN or Inf met on the device */
   FSHARP_E_TIMEOUT = -8,    /* a bounded device-side wait expired */
-  FSHARP_E_CUDA = -9        /* a CUDA runtime or driver call failed */
+  FSHARP_E_CUDA = -9,       /* a CUDA runtime or driver call failed */
+  FSHARP_E_LIMIT = -10      /* problem needs more than the fixed scratch of fsharp_featurize_static */
 };
 
 enum { FSHARP_F32 = 0, FSHARP_BF16 = 1 };
@@ -153,6 +154,28 @@ int fsharp_fit_params(fsharp_ctx* ctx, const double* stats, int G, int d, int va
 int fsharp_featurize(fsharp_ctx* ctx, const void* X, const float* Omega, const double* params,
                      int side, const fsharp_dims* dims, int dtype, float qk_scale, int stab,
                      float* phi, float* logscale);
+
+/* (No counterpart in the paper: an integration aid.)  fsharp_featurize for callers that
+ * cannot allocate device memory when they need features -- code running under a memory
+ * pool that forbids foreign allocations, latency-critical loops that must not enter the
+ * allocator (its locks, its implicit synchronisation), processes whose HBM is already fully
+ * committed.  It takes no context and calls no cudaMalloc / cudaFree or any other allocating
+ * routine: its scratch is a fixed array of fsharp_static_scratch_bytes() (8 MiB) inside the
+ * loaded module, which every GPU that loads the library holds until the process exits.
+ * Arguments as fsharp_featurize, plus the stream (cudaStream_t as void*) and an optional
+ * device status word (device int*, may be NULL) that receives FSHARP_E_NONFINITE.
+ * The scratch must hold G*2*(M*d + M + 8 + d*d) + B*H*L + B*H 4-byte words (each block
+ * rounded up to 256 bytes); larger problems are refused with FSHARP_E_LIMIT and nothing runs.
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress)
+ * and, under lazy module loading, is also when the driver materialises the array; make
+ * that first call before any stream capture begins.  All calls share the one array and
+ * it keeps whatever the last call left in it; each call writes every word it later reads,
+ * so stale contents are harmless, but two calls whose kernels may overlap on the GPU
+ * (different streams, or different host threads) race on it: serialise them. */
+size_t fsharp_static_scratch_bytes(void);
+int fsharp_featurize_static(void* stream, const void* X, const float* Omega, const double* params,
+                            int side, const fsharp_dims* dims, int dtype, float qk_scale, int stab,
+                            float* phi, float* logscale, int* device_status);
 
 /* Y [B,H,Lq,dv] (type `dtype`) of Section 2.2 with Khat = P S^T in place of the
  * exact kernel matrix, evaluated as P (S^T [V | 1]) (Section 2.1's O(L M n) order).

@@ -23,7 +23,7 @@ EXPORTS = [
     "fsharp_launch_count", "fsharp_workspace_bytes", "fsharp_strerror", "fsharp_stats_doubles",
     "fsharp_params_doubles", "fsharp_stats", "fsharp_fit_params", "fsharp_featurize", "fsharp_attend",
     "fsharp_forward_host", "fsharp_pair_estimate", "fsharp_set_timing", "fsharp_read_timing",
-    "fsharp_kernel_name",
+    "fsharp_kernel_name", "fsharp_static_scratch_bytes", "fsharp_featurize_static",
 ]
 
 
@@ -76,6 +76,8 @@ def load_library() -> C.CDLL:
         "fsharp_set_timing": (i32, [vp, i32]),
         "fsharp_read_timing": (i32, [vp, i32, C.POINTER(C.c_float), C.POINTER(i32)]),
         "fsharp_kernel_name": (C.c_char_p, [i32]),
+        "fsharp_static_scratch_bytes": (C.c_size_t, []),
+        "fsharp_featurize_static": (i32, [vp, vp, vp, vp, i32, dims_p, i32, f32, i32, vp, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -262,6 +264,28 @@ class Context:
                                              params.data_ptr(), npairs, d, M, R, est.data_ptr(),
                                              var.data_ptr() if var is not None else None), "fsharp_pair_estimate")
         return est, var
+
+
+def static_scratch_bytes() -> int:
+    return load_library().fsharp_static_scratch_bytes()
+
+
+def fsharp_featurize_static(X, Omega, params, side, phi, logscale=None, pool=POOL_PER_BH, qk_scale=1.0,
+                            stab=STAB_ROW, stream=None, device_status=None) -> int:
+    """The feature map without any device allocation by the library: the caller supplies the
+    outputs (phi [B,H,L,M] float32, logscale as for fsharp_featurize) and the library's fixed
+    in-module scratch is used.  Returns the C return code instead of raising, so a caller can
+    test for the size limit (-10)."""
+    lib = load_library()
+    B, H, L, d = X.shape
+    M = Omega.shape[-2]
+    ohs = Omega.stride(0) if Omega.dim() == 3 else 0
+    dm = make_dims(B, H, L, L, d, d, M, pool, q=X, k=X, omega_head_stride=ohs)
+    sp = stream.cuda_stream if stream is not None else torch.cuda.current_stream(X.device).cuda_stream
+    return lib.fsharp_featurize_static(
+        C.c_void_p(sp), X.data_ptr(), Omega.data_ptr(), params.data_ptr(), side, C.byref(dm), _dtype_code(X),
+        qk_scale, stab, phi.data_ptr(), logscale.data_ptr() if logscale is not None else None,
+        device_status.data_ptr() if device_status is not None else None)
 
 
 def unpack_params(blob: torch.Tensor, d: int):

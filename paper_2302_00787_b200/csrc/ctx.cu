@@ -98,6 +98,7 @@ const char* fsharp_strerror(int code) {
     case FSHARP_E_NONFINITE: return "non-finite value met on the device";
     case FSHARP_E_TIMEOUT: return "bounded device-side wait expired";
     case FSHARP_E_CUDA: return "CUDA call failed";
+    case FSHARP_E_LIMIT: return "problem exceeds the fixed scratch of the no-allocation entry point";
     default: return "unknown error";
   }
 }
