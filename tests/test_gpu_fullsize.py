@@ -1,0 +1,77 @@
+"""Parity at the full benchmark sizes, in the launch configuration bench.py times: the CUDA
+path runs the whole workload; the fp64 checker recomputes sampled (batch, head) units on sampled
+query rows (it can compute any output row by itself: features of the row, features of all keys,
+the masked or full weighted average).  Plus properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import favor_sharp as fs
+from paper_2302_00787_b200 import binding as fb
+from paper_2302_00787_b200 import workloads as wl
+from tests.gpu_util import TOL, FIT_TOL, host
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = fb.Context(0)
+    yield c
+    c.close()
+
+
+def run_full(ctx, w):
+    Q, K, V = wl.make_qkv(w)
+    Om = wl.make_omega(w)
+    dQ, dK, dV = (torch.from_numpy(a).cuda().to(torch.bfloat16) for a in (Q, K, V))
+    dOm = torch.from_numpy(Om).cuda()
+    st = ctx.fsharp_stats(dQ, dK)
+    pr = ctx.fsharp_fit_params(st, w.d, w.variant)
+    Y = ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=w.causal, chunk=w.chunk)
+    assert ctx.status() == 0
+    return (Q, K, V, Om), (dQ, dK, dV, dOm), pr, Y
+
+
+def check_sampled(w, host_in, pr, Y, units, nrows, seed):
+    Q, K, V, Om = host_in
+    rng = np.random.default_rng(seed)
+    prh = pr.cpu().numpy()
+    for (b, h) in units:
+        rows = np.sort(np.concatenate([[0, 1, w.L - 1], rng.integers(0, w.L, nrows)]))
+        if w.causal:
+            rows = np.unique(np.concatenate([rows, [w.chunk - 1, w.chunk, w.L - w.chunk]]))
+        p = fb.unpack_params(prh[b * w.H + h], w.d)
+        ref = fs.favor_sharp_attention(Q[b, h], K[b, h], V[b, h], Om, p, causal=w.causal, rows=rows)
+        got = host(Y[b, h])[rows]
+        scale = np.abs(host(Y[b, h])).max()            # max |Y| of the unit (the checker has only sampled rows)
+        assert np.abs(got - ref).max() / scale < TOL["bf16"], (b, h)
+        # the fit of this unit against the checker's, on an invariant
+        refp = fs.fit_params(Q[b, h], K[b, h], w.variant)
+        assert abs(p["objective"] - refp["objective"]) <= FIT_TOL * abs(refp["objective"])
+        assert abs(p["logD"] - refp["logD"]) <= FIT_TOL * max(1e-3, abs(refp["logD"]))
+
+
+@pytest.mark.parametrize("name,units", [("cfg2", [(0, 0), (3, 5), (7, 7)]), ("cfg3b", [(0, 0), (3, 11)]),
+                                        ("cfg3", [(0, 0), (2, 7), (3, 11)])])
+def test_full_size_sampled_parity(ctx, name, units):
+    w = wl.WORKLOADS[name]
+    host_in, dev_in, pr, Y = run_full(ctx, w)
+    assert torch.isfinite(Y.float()).all()
+    check_sampled(w, host_in, pr, Y, units, 24, 11)
+    # right-stochastic at any size: V = 1 gives Y = 1 (bf16 output rounding aside)
+    dQ, dK, dV, dOm = dev_in
+    Y1 = ctx.fsharp_attend(dQ, dK, torch.ones_like(dV), dOm, pr, causal=w.causal, chunk=w.chunk)
+    assert (Y1.float() - 1).abs().max().item() < 1e-2
+    if w.causal:                                      # the first token attends to itself only
+        assert (Y[:, :, 0].float() - dV[:, :, 0].float()).abs().max().item() < 1e-2
+    assert ctx.status() == 0
+
+
+def test_long_sequence_causal_sampled_parity(ctx):
+    """The L = 65536, d = 128, M = 512 workload with x3 outlier tokens (4 of its 16 heads are
+    checked; the other heads run the same launch)."""
+    w = wl.WORKLOADS["cfg5"]
+    host_in, dev_in, pr, Y = run_full(ctx, w)
+    assert torch.isfinite(Y.float()).all()
+    check_sampled(w, host_in, pr, Y, [(0, 0), (0, 9)], 12, 5)
