@@ -54,7 +54,7 @@ __device__ void jacobi_schedule(ushort2* sched, int d) {
 }
 
 __device__ __forceinline__ int jacobi_eig(double* __restrict__ A, int lda, double* __restrict__ VT, int ldvt, int d,
-                                          int log2d, const ushort2* __restrict__ sched, double* __restrict__ cs,
+                                          int log2d, const ushort2* __restrict__ sched, double* __restrict__ cs_base,
                                           double* red) {
   const int tid = threadIdx.x;
   const int half = d >> 1, items = half << log2d, dm1 = d - 1;
@@ -73,40 +73,81 @@ __device__ __forceinline__ int jacobi_eig(double* __restrict__ A, int lda, doubl
     tot = block_reduce(tot, red, 0);
     if (off <= 1e-24 * tot || tot == 0.0) break;
     sweeps++;
+    // Rotation parameters of round r live in cs[(r & 1) * d ...]; those of round r + 1 are
+    // computed by the first d/2 threads while everybody applies round r to VT (VT does not feed
+    // the parameters), so their latency is hidden.
+    auto rotation_params = [&](int r) {
+      const ushort2* sr = sched + r * half;
+      double* csr = cs_base + (r & 1) * d;
+      const int p = sr[tid].x, q = sr[tid].y;
+      const double app = A[p * lda + p], aqq = A[q * lda + q], apq = A[p * lda + q];
+      double c = 1.0, s = 0.0;
+      const float num = (float)(aqq - app), den = (float)(2.0 * apq);
+      if (den != 0.f) {
+        const float zeta = __fdividef(num, den);
+        const float tf = __fdividef(copysignf(1.f, zeta), fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f)));
+        if (isfinite(tf)) {
+          const double t = (double)tf;
+          const double x = fma(t, t, 1.0);
+          const double c0 = (double)rsqrtf(fmaf(tf, tf, 1.f));
+          c = c0 * fma(-0.5 * x, c0 * c0, 1.5);       // one Newton step: |c^2 x - 1| ~ 1e-14
+          s = t * c;
+        }
+      }
+      csr[2 * tid] = c; csr[2 * tid + 1] = s;
+    };
+    if (tid < half) rotation_params(0);
+    __syncthreads();
     for (int r = 0; r < d - 1; r++) {
       const ushort2* sr = sched + r * half;
-      if (tid < half) {
-        const int p = sr[tid].x, q = sr[tid].y;
-        const double app = A[p * lda + p], aqq = A[q * lda + q], apq = A[p * lda + q];
-        double c = 1.0, s = 0.0;
-        const float num = (float)(aqq - app), den = (float)(2.0 * apq);
-        if (den != 0.f) {
-          const float zeta = __fdividef(num, den);
-          const float tf = __fdividef(copysignf(1.f, zeta), fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f)));
-          if (isfinite(tf)) {
-            const double t = (double)tf;
-            c = rsqrt(fma(t, t, 1.0));
-            s = t * c;
+      const double* cs = cs_base + (r & 1) * d;
+      // A <- J^T A J, one 2 x 2 block per item: block (k, l) holds rows {p_k, q_k} and columns
+      // {p_l, q_l}; it is rotated by J_k from the left and J_l from the right in registers, so A
+      // is read and written once per round and no barrier separates the two sides.  Blocks of a
+      // round are disjoint.  VT <- J^T VT (rows p, q) rides along as further disjoint items.
+      const int log2h = log2d - 1;
+      const int nblk = half << log2h;                 // (d/2)^2 blocks
+      for (int e0 = tid; e0 < nblk; e0 += 2 * FIT_THREADS) {
+        double a00[2], a01[2], a10[2], a11[2], ck[2], sk[2], cl[2], sl[2];
+        int i00[2], i01[2], i10[2], i11[2];
+#pragma unroll
+        for (int u = 0; u < 2; u++) {
+          const int e = e0 + u * FIT_THREADS;
+          if (e < nblk) {
+            const int k = e >> log2h, l = e & (half - 1);
+            const int pk = sr[k].x, qk = sr[k].y, pl = sr[l].x, ql = sr[l].y;
+            ck[u] = cs[2 * k]; sk[u] = cs[2 * k + 1]; cl[u] = cs[2 * l]; sl[u] = cs[2 * l + 1];
+            i00[u] = pk * lda + pl; i01[u] = pk * lda + ql; i10[u] = qk * lda + pl; i11[u] = qk * lda + ql;
+            a00[u] = A[i00[u]]; a01[u] = A[i01[u]]; a10[u] = A[i10[u]]; a11[u] = A[i11[u]];
           }
         }
-        cs[2 * tid] = c; cs[2 * tid + 1] = s;
+#pragma unroll
+        for (int u = 0; u < 2; u++) {
+          const int e = e0 + u * FIT_THREADS;
+          if (e < nblk) {
+            // left: rows (p_k, q_k) <- (c x - s y, s x + c y)
+            const double r00 = ck[u] * a00[u] - sk[u] * a10[u], r01 = ck[u] * a01[u] - sk[u] * a11[u];
+            const double r10 = sk[u] * a00[u] + ck[u] * a10[u], r11 = sk[u] * a01[u] + ck[u] * a11[u];
+            // right: columns (p_l, q_l) <- (c x - s y, s x + c y)
+            A[i00[u]] = cl[u] * r00 - sl[u] * r01;
+            A[i01[u]] = sl[u] * r00 + cl[u] * r01;
+            A[i10[u]] = cl[u] * r10 - sl[u] * r11;
+            A[i11[u]] = sl[u] * r10 + cl[u] * r11;
+          }
+        }
       }
       __syncthreads();
-      // A <- A J (columns p, q of every row) and VT <- J^T VT (rows p, q): the rotations of a
-      // round touch disjoint elements, so each thread loads a batch first and stores afterwards
+      if (tid < half && r + 1 < d - 1) rotation_params(r + 1);
       for (int e0 = tid; e0 < items; e0 += 4 * FIT_THREADS) {
-        double xa[4], ya[4], xv[4], yv[4], cc[4], ss[4];
-        int ia[4], ja[4], iv[4], jv[4];
+        double xv[4], yv[4], cc[4], ss[4];
+        int iv[4], jv[4];
 #pragma unroll
         for (int u = 0; u < 4; u++) {
           const int e = e0 + u * FIT_THREADS;
           if (e < items) {
             const int k = e >> log2d, row = e & dm1;
-            const int p = sr[k].x, q = sr[k].y;
             cc[u] = cs[2 * k]; ss[u] = cs[2 * k + 1];
-            ia[u] = row * lda + p; ja[u] = row * lda + q;
-            iv[u] = p * ldvt + row; jv[u] = q * ldvt + row;
-            xa[u] = A[ia[u]]; ya[u] = A[ja[u]];
+            iv[u] = sr[k].x * ldvt + row; jv[u] = sr[k].y * ldvt + row;
             xv[u] = VT[iv[u]]; yv[u] = VT[jv[u]];
           }
         }
@@ -114,34 +155,8 @@ __device__ __forceinline__ int jacobi_eig(double* __restrict__ A, int lda, doubl
         for (int u = 0; u < 4; u++) {
           const int e = e0 + u * FIT_THREADS;
           if (e < items) {
-            A[ia[u]] = cc[u] * xa[u] - ss[u] * ya[u];
-            A[ja[u]] = ss[u] * xa[u] + cc[u] * ya[u];
             VT[iv[u]] = cc[u] * xv[u] - ss[u] * yv[u];
             VT[jv[u]] = ss[u] * xv[u] + cc[u] * yv[u];
-          }
-        }
-      }
-      __syncthreads();
-      for (int e0 = tid; e0 < items; e0 += 4 * FIT_THREADS) {   // A <- J^T A (rows p, q of every column)
-        double xa[4], ya[4], cc[4], ss[4];
-        int ia[4], ja[4];
-#pragma unroll
-        for (int u = 0; u < 4; u++) {
-          const int e = e0 + u * FIT_THREADS;
-          if (e < items) {
-            const int k = e >> log2d, col = e & dm1;
-            const int p = sr[k].x, q = sr[k].y;
-            cc[u] = cs[2 * k]; ss[u] = cs[2 * k + 1];
-            ia[u] = p * lda + col; ja[u] = q * lda + col;
-            xa[u] = A[ia[u]]; ya[u] = A[ja[u]];
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 4; u++) {
-          const int e = e0 + u * FIT_THREADS;
-          if (e < items) {
-            A[ia[u]] = cc[u] * xa[u] - ss[u] * ya[u];
-            A[ja[u]] = ss[u] * xa[u] + cc[u] * ya[u];
           }
         }
       }
