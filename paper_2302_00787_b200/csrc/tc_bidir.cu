@@ -1,16 +1,19 @@
 // Tensor-core path, bidirectional attention (Sections 2.1 / 2.2) for bf16, d = dv = 64, M = 256.
 //
-//   key side   (tc_kv_kernel):  per 128-key tile   logits = Y W2^T + a      (tcgen05, TMEM)
+//   key side   (tc_kv_kernel):  per 128-key tile   logits = Y W2^T           (tcgen05, TMEM)
 //                               phi = 2^(logits + c_j - s)  -> bf16 tile in shared memory
 //                               KV += phi^T [V | 1]                          (tcgen05, TMEM)
 //   merge      (tc_merge_kernel): partial KV of the splits of one (batch, head), brought to a
-//                               common shift, summed, written transposed in fp16
-//   query side (tc_out_kernel): logits, phi = 2^(logits - rowmax), [num | den] = phi KV,
-//                               Y = num / den
+//                               common shift, summed, scaled by 2^a2 per feature, written
+//                               transposed in fp16
+//   query side (tc_out_kernel): logits, phi = 2^(logits - max of the half row) in fp16,
+//                               [num | den] = phi KV per feature half, halves combined, Y = num / den
 //
 // The feature tiles never leave the SM.  One block = 8 epilogue warps (exponentials), one
 // TMA producer warp and one MMA issuing warp; all exponents are kept in log2 units
-// (W, a and C are pre-multiplied by log2 e), so the feature is one ex2 per element.
+// (W and C are pre-multiplied by log2 e), so a feature is one ex2 per element.  The per-feature
+// term w^T A w is the same on the query and the key side, so it is not added to the logits at
+// all: the merge multiplies row m of S^T [V | 1] by 2^(2 log2e w_m^T A w_m).
 #include <cuda_fp16.h>
 
 #include "common.cuh"
@@ -20,49 +23,26 @@
 using namespace tc;
 using namespace tcl;
 
-#ifdef FS_TRACE
-__device__ long long fs_trace_buf[8192];
-__device__ int fs_trace_n;
-#define TRACE(tag)                                                        \
-  do {                                                                    \
-    if (blockIdx.x == 0 && blockIdx.y == 0) {                             \
-      int _i = atomicAdd(&fs_trace_n, 1);                                 \
-      if (_i < 4096) { fs_trace_buf[2 * _i] = (tag); fs_trace_buf[2 * _i + 1] = clock64(); } \
-    }                                                                     \
-  } while (0)
-extern "C" int fsharp_debug_read_trace(long long* out, int cap) {
-  int n = 0;
-  cudaMemcpyFromSymbol(&n, fs_trace_n, sizeof(int));
-  if (n > cap) n = cap;
-  if (n > 4096) n = 4096;
-  cudaMemcpyFromSymbol(out, fs_trace_buf, (size_t)n * 2 * sizeof(long long));
-  int zero = 0;
-  cudaMemcpyToSymbol(fs_trace_n, &zero, sizeof(int));
-  return n;
-}
-#else
-#define TRACE(tag) do { } while (0)
-#endif
-
 namespace {
+
+constexpr int PREFETCH_TILES = 4;   // tiles pulled into L2 ahead of the shared-memory ring
 
 // ------------------------------------------------------------------------------------------
 // key side
 // ------------------------------------------------------------------------------------------
 struct KvSmem {
-  static constexpr uint32_t X0 = 0, V0 = 2 * TILE_BYTES, W = 4 * TILE_BYTES, WLO = W + IMG_W_BYTES,
-                            CHI = WLO + IMG_W_BYTES, CLO = CHI + IMG_C_BYTES, BAUG = CLO + IMG_C_BYTES,
-                            AAUG = BAUG + IMG_BAUG_BYTES, ONEST = AAUG + 4096, PHI = ONEST + ONEST_BYTES,
-                            MISC = PHI + 4 * TILE_BYTES, TOTAL = MISC + 256;
+  static constexpr uint32_t X0 = 0, V0 = 2 * TILE_BYTES, ONES = 4 * TILE_BYTES, W = ONES + TILE_BYTES,
+                            WLO = W + IMG_W_BYTES, CHI = WLO + IMG_W_BYTES, CLO = CHI + IMG_C_BYTES,
+                            PHI = CLO + IMG_C_BYTES, MISC = PHI + 4 * TILE_BYTES, TOTAL = MISC + 256;
 };
 static_assert(KvSmem::TOTAL + 1024 <= 232448, "shared memory budget");
-static_assert(KvSmem::PHI % 1024 == 0 && KvSmem::W % 1024 == 0 && KvSmem::ONEST % 1024 == 0, "swizzled tiles need 1024-byte alignment");
+static_assert(KvSmem::PHI % 1024 == 0 && KvSmem::W % 1024 == 0 && KvSmem::ONES % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 
 struct KvMisc {
   uint64_t full[2], empty[2], logits_full, logits_free, phi_full, phi_free, const_bar;
   uint32_t tmem_base;
   int abort_flag;
-  int tile_max[3];
+  int tile_max[4];     // [0..2] rotating slots of the per-tile maximum, [3] the first tile's
 };
 
 constexpr uint32_t KV_COL_LOGITS = 0, KV_COL_T = 256, KV_COL_ACC = 320;   // TMEM columns
@@ -95,21 +75,15 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     mbar_init(&misc->phi_free, 1);
     mbar_init(&misc->const_bar, 1);
     misc->abort_flag = 0;
-    misc->tile_max[0] = misc->tile_max[1] = misc->tile_max[2] = f2ord(-INFINITY);
+    for (int i = 0; i < 4; i++) misc->tile_max[i] = f2ord(-INFINITY);
     fence_barrier_init();
   }
-  // constant tiles written by the block itself: the ones column of [V | 1] and the rows (1, 1, 0, ...)
-  // that pick a_hi + a_lo out of the augmented feature operand
-  for (int i = threadIdx.x; i < ONEST_BYTES / 16; i += TC_THREADS) reinterpret_cast<uint4*>(sm + KvSmem::ONEST)[i] = make_uint4(0, 0, 0, 0);
-  for (int i = threadIdx.x; i < 4096 / 16; i += TC_THREADS) reinterpret_cast<uint4*>(sm + KvSmem::AAUG)[i] = make_uint4(0, 0, 0, 0);
+  // constant tile written by the block itself: the second 64-column block of [V | 1], whose
+  // first column is the 1 and whose other columns are zero (only 16 of them are read)
+  for (int i = threadIdx.x; i < TILE_BYTES / 16; i += TC_THREADS) reinterpret_cast<uint4*>(sm + KvSmem::ONES)[i] = make_uint4(0, 0, 0, 0);
   __syncthreads();
-  if (threadIdx.x < TILE) {
-    const uint32_t r = threadIdx.x;
-    // transposed ones operand: row 0 of a [16 x 128 tokens] K-major matrix, two 64-token blocks of 2 KB
-    *reinterpret_cast<__nv_bfloat16*>(sm + KvSmem::ONEST + (r >> 6) * 2048 + sw128_offset(0, r & 63)) = __float2bfloat16(1.f);
-    *reinterpret_cast<__nv_bfloat16*>(sm + KvSmem::AAUG + core16_offset(r, 0)) = __float2bfloat16(1.f);
-    *reinterpret_cast<__nv_bfloat16*>(sm + KvSmem::AAUG + core16_offset(r, 1)) = __float2bfloat16(1.f);
-  }
+  if (threadIdx.x < TILE)
+    *reinterpret_cast<__nv_bfloat16*>(sm + KvSmem::ONES + sw128_offset(threadIdx.x, 0)) = __float2bfloat16(1.f);
   fence_proxy_async_smem();
   if (warp == WARP_MMA) {
     tmem_alloc(&misc->tmem_base, TMEM_COLS);
@@ -124,17 +98,24 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     if (lane == 0) {
       prefetch_tmap(&tmK);
       prefetch_tmap(&tmV);
-      mbar_expect_tx(&misc->const_bar, IMG_BYTES);
+      mbar_expect_tx(&misc->const_bar, 2 * IMG_W_BYTES + 2 * IMG_C_BYTES);
       bulk_load(sm + KvSmem::W, img + IMG_W, IMG_W_BYTES, &misc->const_bar);
       bulk_load(sm + KvSmem::WLO, img + IMG_WLO, IMG_W_BYTES, &misc->const_bar);
       bulk_load(sm + KvSmem::CHI, img + IMG_CHI, IMG_C_BYTES, &misc->const_bar);
       bulk_load(sm + KvSmem::CLO, img + IMG_CLO, IMG_C_BYTES, &misc->const_bar);
-      bulk_load(sm + KvSmem::BAUG, img + IMG_BAUG, IMG_BAUG_BYTES, &misc->const_bar);
+      // the shared-memory ring is only two tiles deep; tiles further ahead are pulled into L2
+      for (int it = 0; it < min(ntiles, PREFETCH_TILES); it++) {
+        tma_prefetch_4d(&tmK, 0, (tile0 + it) * TILE, h, b);
+        tma_prefetch_4d(&tmV, 0, (tile0 + it) * TILE, h, b);
+      }
       int issued = 0;
       for (int it = 0; it < ntiles; it++) {
         const int st = it & 1;
+        if (it + PREFETCH_TILES < ntiles) {
+          tma_prefetch_4d(&tmK, 0, (tile0 + it + PREFETCH_TILES) * TILE, h, b);
+          tma_prefetch_4d(&tmV, 0, (tile0 + it + PREFETCH_TILES) * TILE, h, b);
+        }
         if (!mbar_wait(&misc->empty[st], ((it >> 1) & 1) ^ 1, abortp, status)) break;
-        TRACE(100 + it * 1000);
         mbar_expect_tx(&misc->full[st], 2 * TILE_BYTES);
         tma_load_4d(sm + KvSmem::X0 + st * TILE_BYTES, &tmK, &misc->full[st], 0, (tile0 + it) * TILE, h, b);
         tma_load_4d(sm + KvSmem::V0 + st * TILE_BYTES, &tmV, &misc->full[st], 0, (tile0 + it) * TILE, h, b);
@@ -148,20 +129,18 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     if (lane == 0) {
       constexpr uint32_t ID_LOGITS = idesc_bf16(128, TC_M, 0, 0);
       constexpr uint32_t ID_T = idesc_bf16(128, TC_D, 0, 0);
-      constexpr uint32_t ID_KV = idesc_bf16(128, TC_DV, 1, 1);     // phi^T V
-      constexpr uint32_t ID_KV1 = idesc_bf16(128, 16, 1, 0);       // phi^T 1 (column dv of [V | 1])
-      const uint32_t sWlo = smem_u32(sm + KvSmem::WLO);
-      const uint32_t sW = smem_u32(sm + KvSmem::W), sChi = smem_u32(sm + KvSmem::CHI), sClo = smem_u32(sm + KvSmem::CLO);
-      const uint32_t sBaug = smem_u32(sm + KvSmem::BAUG), sAaug = smem_u32(sm + KvSmem::AAUG);
-      const uint32_t sPhi = smem_u32(sm + KvSmem::PHI), sOnesT = smem_u32(sm + KvSmem::ONEST);
+      constexpr uint32_t ID_KV = idesc_bf16(128, TC_NV, 1, 1);     // phi^T [V | 1]
+      const uint32_t sV0 = smem_u32(sm + KvSmem::V0), sOnes = smem_u32(sm + KvSmem::ONES);
       // descriptors are built once; inside the loops each MMA costs one add per operand
       const uint64_t dX0 = smem_desc(smem_u32(sm + KvSmem::X0), 16, 1024, SWZ_128B);
-      const uint64_t dV0 = smem_desc(smem_u32(sm + KvSmem::V0), 16, 1024, SWZ_128B);
-      const uint64_t dW = smem_desc(sW, 16, 1024, SWZ_128B), dWlo = smem_desc(sWlo, 16, 1024, SWZ_128B);
-      const uint64_t dChi = smem_desc(sChi, 16, 1024, SWZ_128B), dClo = smem_desc(sClo, 16, 1024, SWZ_128B);
-      const uint64_t dAaug = smem_desc(sAaug, 128, 256, SWZ_NONE), dBaug = smem_desc(sBaug, 128, 256, SWZ_NONE);
-      const uint64_t dPhi = smem_desc(sPhi, TILE_BYTES, 1024, SWZ_128B);
-      const uint64_t dOnesT = smem_desc(sOnesT, 16, 1024, SWZ_128B);
+      const uint64_t dW = smem_desc(smem_u32(sm + KvSmem::W), 16, 1024, SWZ_128B);
+      const uint64_t dWlo = smem_desc(smem_u32(sm + KvSmem::WLO), 16, 1024, SWZ_128B);
+      const uint64_t dChi = smem_desc(smem_u32(sm + KvSmem::CHI), 16, 1024, SWZ_128B);
+      const uint64_t dClo = smem_desc(smem_u32(sm + KvSmem::CLO), 16, 1024, SWZ_128B);
+      const uint64_t dPhi = smem_desc(smem_u32(sm + KvSmem::PHI), TILE_BYTES, 1024, SWZ_128B);
+      // [V | 1] as one MN-major operand: block 0 = the V tile of the stage, block 1 = the ones tile
+      const uint64_t dVst0 = smem_desc(sV0, sOnes - sV0, 1024, SWZ_128B);
+      const uint64_t dVst1 = smem_desc(sV0 + TILE_BYTES, sOnes - sV0 - TILE_BYTES, 1024, SWZ_128B);
       auto issue_logits = [&](int st) {
         const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
 #pragma unroll
@@ -170,7 +149,6 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 #pragma unroll
         for (int k = 0; k < TC_D / 16; k++)
           mma_bf16(tmem + KV_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dWlo, 32 * k), ID_LOGITS, 1);
-        mma_bf16(tmem + KV_COL_LOGITS, dAaug, dBaug, ID_LOGITS, 1);
         if (cdense) {
 #pragma unroll
           for (int k = 0; k < TC_D / 16; k++)
@@ -193,46 +171,39 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         const int st = it & 1;
         if (it + 1 < ntiles) {
           if (!mbar_wait(&misc->full[st ^ 1], ((it + 1) >> 1) & 1, abortp, status)) break;
-          TRACE(200 + it * 1000);
           if (!mbar_wait(&misc->logits_free, it & 1, abortp, status)) break;
-          TRACE(201 + it * 1000);
           tcgen05_fence_after();
           issue_logits(st ^ 1);
-          TRACE(202 + it * 1000);
         }
         if (!mbar_wait(&misc->phi_full, it & 1, abortp, status)) break;
-        TRACE(203 + it * 1000);
         tcgen05_fence_after();
-        const uint64_t dV = desc_advance(dV0, st * TILE_BYTES);
+        const uint64_t dV = st ? dVst1 : dVst0;
         const uint32_t acc0 = it > 0 ? 1u : 0u;
 #pragma unroll
         for (int hh = 0; hh < 2; hh++)
 #pragma unroll
-          for (int k = 0; k < TILE / 16; k++) {
-            const uint64_t da = desc_advance(dPhi, hh * 2 * TILE_BYTES + k * 2048);
-            const uint32_t acc = k > 0 ? 1u : acc0;
-            mma_bf16(tmem + KV_COL_ACC + hh * TC_NV, da, desc_advance(dV, k * 2048), ID_KV, acc);
-            mma_bf16(tmem + KV_COL_ACC + hh * TC_NV + TC_DV, da, desc_advance(dOnesT, (k >> 2) * 2048 + (k & 3) * 32),
-                     ID_KV1, acc);
-          }
+          for (int k = 0; k < TILE / 16; k++)
+            mma_bf16(tmem + KV_COL_ACC + hh * TC_NV, desc_advance(dPhi, hh * 2 * TILE_BYTES + k * 2048),
+                     desc_advance(dV, k * 2048), ID_KV, k > 0 ? 1u : acc0);
         mma_commit(&misc->phi_free);
         mma_commit(&misc->empty[st]);
-        TRACE(204 + it * 1000);
       }
     }
   } else {
-    // ---------------- epilogue warps: one key row per thread, 128 of the 256 features
+    // ---------------- epilogue warps: one key row per thread, 128 of the 256 features.
+    // The running shift s is taken on trust while the exponentials are computed; the tile's
+    // largest exponent is tracked on the side and checked afterwards.  Only if it exceeds the
+    // headroom (rare: the running maximum grows a handful of times per sequence) is the
+    // accumulated state rescaled and the tile redone from the logits still held in registers.
     const int q = warp & 3, hf = warp >> 2;
     const int row = q * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
     float s = 0.f;
-    bool have = false, alive = true;
+    bool alive = true;
     for (int it = 0; it < ntiles && alive; it++) {
       const int st = it & 1;
       if (!mbar_wait(&misc->full[st], (it >> 1) & 1, abortp, status, false)) { alive = false; break; }
-      if (threadIdx.x == 0) TRACE(300 + it * 1000);
       if (!mbar_wait(&misc->logits_full, it & 1, abortp, status, false)) { alive = false; break; }
-      if (threadIdx.x == 0) TRACE(301 + it * 1000);
       __syncwarp();
       tcgen05_fence_after();
       // c_j = x_j^T C x_j in log2 units
@@ -250,9 +221,8 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
             xv[c * 8 + 2 * j + 1] = __uint_as_float(w4[j] & 0xffff0000u);
           }
         }
+        float part[4] = {0.f, 0.f, 0.f, 0.f};
         if (cdense) {
-#pragma unroll
-          float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
           for (int c = 0; c < TC_D / 16; c++) {
             uint32_t t[16];
@@ -263,7 +233,6 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           }
           cj = (part[0] + part[1]) + (part[2] + part[3]);
         } else {
-          float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
           for (int j = 0; j < TC_D; j++) part[j & 3] = fmaf(xv[j], xv[j], part[j & 3]);
           cj = ((part[0] + part[1]) + (part[2] + part[3])) * gamma2;
@@ -280,40 +249,51 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       tmem_wait_ld();
       tcgen05_fence_before();
       mbar_arrive(&misc->logits_free);
-      if (threadIdx.x == 0) TRACE(302 + it * 1000);
       const bool valid = (tile0 + it) * TILE + row < L;
-      float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      if (it == 0) {
+        // first tile: no shift yet, take the tile's exact maximum
+        float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int i = 0; i < 128; i++) {
-        float f = __uint_as_float(v[i]) + cj;
-        v[i] = __float_as_uint(f);
-        mxp[i & 3] = fmaxf(mxp[i & 3], f);
-      }
-      float mx = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
-      if (!valid) mx = -INFINITY;
+        for (int i = 0; i < 128; i++) mxp[i & 3] = fmaxf(mxp[i & 3], __uint_as_float(v[i]));
+        float mx = valid ? fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])) + cj : -INFINITY;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      if (lane == 0) atomicMax(&misc->tile_max[it % 3], f2ord(mx));
-      if (threadIdx.x == 0) misc->tile_max[(it + 1) % 3] = f2ord(-INFINITY);   // next tile's slot; idle since tile it-2
-      named_bar_sync(1, EPI_THREADS);
-      const float t = ord2f(misc->tile_max[it % 3]);
-      if (threadIdx.x == 0) TRACE(303 + it * 1000);
-      const float s_old = s;
-      bool rescale = false;
-      if (!have || t > s + SHIFT_HEADROOM_LOG2) {
-        rescale = have;
-        s = t;
-        have = true;
-      }
-      if (it > 0) {
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (lane == 0) atomicMax(&misc->tile_max[3], f2ord(mx));
+        named_bar_sync(1, EPI_THREADS);
+        s = ord2f(misc->tile_max[3]);
+      } else {
         if (!mbar_wait(&misc->phi_free, (it - 1) & 1, abortp, status, false)) { alive = false; break; }
       }
-      if (threadIdx.x == 0) TRACE(304 + it * 1000);
-      __syncwarp();
-      if (rescale) {
-        // the running shift moved: bring the accumulated S^T [V | 1] to the new one
+      uint8_t* prow = sm + KvSmem::PHI + hf * 2 * TILE_BYTES + row * 128;
+      float rc = cj - s;
+      float rel = -INFINITY;      // largest exponent of this thread's elements, relative to s
+      for (int pass = 0; pass < 2; pass++) {
+        float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int c = 0; c < 16; c++) {
+          uint32_t p[4];
+#pragma unroll
+          for (int j = 0; j < 4; j++) {
+            const float f0 = __uint_as_float(v[c * 8 + 2 * j]) + rc, f1 = __uint_as_float(v[c * 8 + 2 * j + 1]) + rc;
+            mxp[j] = fmaxf(mxp[j], fmaxf(f0, f1));
+            p[j] = pack_bf16(ex2(f0), ex2(f1));
+          }
+          if (!valid) p[0] = p[1] = p[2] = p[3] = 0u;
+          *reinterpret_cast<uint4*>(prow + (c >> 3) * TILE_BYTES + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
+        }
+        if (pass == 1) break;
+        rel = valid ? fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])) : -INFINITY;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) rel = fmaxf(rel, __shfl_xor_sync(0xffffffffu, rel, o));
+        if (lane == 0) atomicMax(&misc->tile_max[it % 3], f2ord(rel));
+        if (threadIdx.x == 0) misc->tile_max[(it + 1) % 3] = f2ord(-INFINITY);   // next tile's slot; idle since tile it-2
+        named_bar_sync(1, EPI_THREADS);
+        rel = ord2f(misc->tile_max[it % 3]);
+        if (!(rel > SHIFT_HEADROOM_LOG2)) break;       // the common case: nothing to redo
+        // the running shift moves up by rel: bring the accumulated S^T [V | 1] along, redo the tile
+        __syncwarp();
         tcgen05_fence_after();
-        const float f = ex2(s_old - s);
+        const float f = ex2(-rel);
 #pragma unroll
         for (int c = 0; c < TC_NV / 16; c++) {
           uint32_t a[16];
@@ -324,24 +304,14 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           tmem_st16(lane_addr + KV_COL_ACC + hf * TC_NV + c * 16, a);
         }
         tmem_wait_st();
-      }
-      uint8_t* prow = sm + KvSmem::PHI + hf * 2 * TILE_BYTES + row * 128;
-#pragma unroll
-      for (int c = 0; c < 16; c++) {
-        uint32_t p[4];
-#pragma unroll
-        for (int j = 0; j < 4; j++) {
-          float e0 = ex2(__uint_as_float(v[c * 8 + 2 * j]) - s), e1 = ex2(__uint_as_float(v[c * 8 + 2 * j + 1]) - s);
-          p[j] = valid ? pack_bf16(e0, e1) : 0u;
-        }
-        *reinterpret_cast<uint4*>(prow + (c >> 3) * TILE_BYTES + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
+        s += rel;
+        rc = cj - s;
       }
       fence_proxy_async_smem();
       tcgen05_fence_before();
       mbar_arrive(&misc->phi_full);
-      if (threadIdx.x == 0) TRACE(305 + it * 1000);
     }
-    // write this split's partial S^T [V | 1] (fp32) and its shift
+    // write this split's partial S^T [V | 1] (fp32), its shift and its largest magnitude
     if (alive && ntiles > 0 && mbar_wait(&misc->phi_free, (ntiles - 1) & 1, abortp, status, false)) {
       __syncwarp();
       tcgen05_fence_after();
@@ -361,7 +331,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-      // largest magnitude of this partial (non-negative floats order like their bit patterns)
+      // non-negative floats order like their bit patterns
       if (lane == 0) atomicMax(&pmax[(size_t)bh * nsplit + split], __float_as_int(amax));
       if (threadIdx.x == 0) shifts[(size_t)bh * nsplit + split] = s;
     }
@@ -375,20 +345,34 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 }
 
 // ------------------------------------------------------------------------------------------
-// merge of the key-side partials of one (batch, head): common shift, sum, transpose, bf16
+// merge of the key-side partials of one (batch, head): common shift, sum, per-feature factor
+// 2^a2, transpose, fp16
 // ------------------------------------------------------------------------------------------
 constexpr int MERGE_SLICES = 8;
 __global__ void __launch_bounds__(256)
 tc_merge_kernel(const float* __restrict__ partial, const float* __restrict__ shifts, const int* __restrict__ pmax,
-                int nsplit, __half* __restrict__ kvt) {
+                int nsplit, const uint8_t* __restrict__ images, int H, int pool, __half* __restrict__ kvt) {
   __shared__ float fac[64];
+  __shared__ float a2s[TC_M];
+  __shared__ float red[256];
   __shared__ float scale_s;
   const int bh = blockIdx.y;
+  const int g = pool == FSHARP_POOL_PER_BH ? bh : bh % H;
+  const float* a2 = reinterpret_cast<const float*>(images + (size_t)g * 2 * IMG_BYTES + IMG_A2);
+  float amax = -INFINITY;
+  for (int m = threadIdx.x; m < TC_M; m += 256) { a2s[m] = a2[m]; amax = fmaxf(amax, a2[m]); }
+  red[threadIdx.x] = amax;
+  __syncthreads();
+  for (int s = 128; s > 0; s >>= 1) {
+    if (threadIdx.x < s) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + s]);
+    __syncthreads();
+  }
   if (threadIdx.x == 0) {
     float smax = -INFINITY;
     for (int p = 0; p < nsplit; p++) smax = fmaxf(smax, shifts[(size_t)bh * nsplit + p]);
     // fp16 has a narrow range: scale the whole (batch, head) by a power of two (it cancels in
-    // num / den) so that the bound sum_p 2^(s_p - smax) max|partial_p| lands near 2^14
+    // num / den) so that the bound sum_p 2^(s_p - smax) max|partial_p| lands near 2^14; the
+    // per-feature factors are applied relative to their maximum, so none exceeds 1
     float bound = 0.f;
     for (int p = 0; p < nsplit; p++) {
       fac[p] = exp2f(shifts[(size_t)bh * nsplit + p] - smax);
@@ -399,7 +383,7 @@ tc_merge_kernel(const float* __restrict__ partial, const float* __restrict__ shi
     scale_s = exp2f((float)(14 - ex));
   }
   __syncthreads();
-  const float scale = scale_s;
+  const float scale = scale_s, a2max = red[0];
   const float* base = partial + (size_t)bh * nsplit * TC_M * TC_NV;
   __half* out = kvt + (size_t)bh * TC_NV * TC_M;
   constexpr int PER = TC_M * TC_NV / MERGE_SLICES;
@@ -408,28 +392,28 @@ tc_merge_kernel(const float* __restrict__ partial, const float* __restrict__ shi
     float acc = 0.f;
     if (n <= TC_DV)
       for (int p = 0; p < nsplit; p++) acc = fmaf(base[(size_t)p * TC_M * TC_NV + e], fac[p], acc);
-    out[(size_t)n * TC_M + m] = __float2half_rn(acc * scale);
+    out[(size_t)n * TC_M + m] = __float2half_rn(acc * scale * exp2f(a2s[m] - a2max));
   }
 }
 
 // ------------------------------------------------------------------------------------------
 // query side
 // ------------------------------------------------------------------------------------------
-constexpr int OUT_STAGES = 2;
+constexpr int OUT_STAGES = 3;
 struct OutSmem {
-  static constexpr uint32_t X0 = 0, W = OUT_STAGES * TILE_BYTES, WLO = W + IMG_W_BYTES, BAUG = WLO + IMG_W_BYTES,
-                            AAUG = BAUG + IMG_BAUG_BYTES,
-                            PHI = AAUG + 4096, KVT = PHI + 4 * TILE_BYTES, ROWMAX = KVT + KVT_BYTES,
-                            MISC = ROWMAX + 2 * 2 * TILE * 4, TOTAL = MISC + 256;
+  static constexpr uint32_t X0 = 0, W = OUT_STAGES * TILE_BYTES, WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES,
+                            KVT = PHI + 4 * TILE_BYTES, ROWMAX = KVT + KVT_BYTES,
+                            MISC = ROWMAX + 3 * 2 * TILE * 4, TOTAL = MISC + 256;
 };
 static_assert(OutSmem::PHI % 1024 == 0 && OutSmem::KVT % 1024 == 0 && OutSmem::W % 1024 == 0, "alignment");
 static_assert(OutSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 
 struct OutMisc {
-  uint64_t full[OUT_STAGES], empty[OUT_STAGES], logits_full, logits_free, phi_full, phi_free, out_full[2], const_bar;
+  uint64_t full[OUT_STAGES], empty[OUT_STAGES], logits_full, logits_free, phi_full, phi_free, const_bar;
   uint32_t tmem_base;
   int abort_flag;
 };
+// TMEM columns: logits, then [num | den] of feature half 0 and of feature half 1
 constexpr uint32_t OUT_COL_LOGITS = 0, OUT_COL_OUT = 256;
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -439,7 +423,7 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   OutMisc* misc = reinterpret_cast<OutMisc*>(sm + OutSmem::MISC);
-  float* rowmax = reinterpret_cast<float*>(sm + OutSmem::ROWMAX);   // [parity][half][row]
+  float* rowmax = reinterpret_cast<float*>(sm + OutSmem::ROWMAX);   // [tile % 3][half][row]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
   const int g = pool == FSHARP_POOL_PER_BH ? bh : h;
@@ -455,20 +439,10 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
     mbar_init(&misc->logits_free, EPI_THREADS);
     mbar_init(&misc->phi_full, EPI_THREADS);
     mbar_init(&misc->phi_free, 1);
-    mbar_init(&misc->out_full[0], 1);
-    mbar_init(&misc->out_full[1], 1);
     mbar_init(&misc->const_bar, 1);
     misc->abort_flag = 0;
     fence_barrier_init();
   }
-  for (int i = threadIdx.x; i < 4096 / 16; i += TC_THREADS) reinterpret_cast<uint4*>(sm + OutSmem::AAUG)[i] = make_uint4(0, 0, 0, 0);
-  __syncthreads();
-  if (threadIdx.x < TILE) {
-    const uint32_t r = threadIdx.x;
-    *reinterpret_cast<__nv_bfloat16*>(sm + OutSmem::AAUG + core16_offset(r, 0)) = __float2bfloat16(1.f);
-    *reinterpret_cast<__nv_bfloat16*>(sm + OutSmem::AAUG + core16_offset(r, 1)) = __float2bfloat16(1.f);
-  }
-  fence_proxy_async_smem();
   if (warp == WARP_MMA) {
     tmem_alloc(&misc->tmem_base, TMEM_COLS);
     tmem_relinquish();
@@ -482,16 +456,17 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
     if (lane == 0) {
       prefetch_tmap(&tmQ);
       prefetch_tmap(&tmKVt);
-      mbar_expect_tx(&misc->const_bar, 2 * IMG_W_BYTES + IMG_BAUG_BYTES + KVT_BYTES);
+      mbar_expect_tx(&misc->const_bar, 2 * IMG_W_BYTES + KVT_BYTES);
       bulk_load(sm + OutSmem::W, img + IMG_W, IMG_W_BYTES, &misc->const_bar);
       bulk_load(sm + OutSmem::WLO, img + IMG_WLO, IMG_W_BYTES, &misc->const_bar);
-      bulk_load(sm + OutSmem::BAUG, img + IMG_BAUG, IMG_BAUG_BYTES, &misc->const_bar);
 #pragma unroll
       for (int fb = 0; fb < TC_M / 64; fb++)
         tma_load_3d(sm + OutSmem::KVT + fb * KVT_BLOCK_BYTES, &tmKVt, &misc->const_bar, fb * 64, 0, bh);
+      for (int it = 0; it < min(ntiles, PREFETCH_TILES); it++) tma_prefetch_4d(&tmQ, 0, (tile0 + it) * TILE, h, b);
       int issued = 0;
       for (int it = 0; it < ntiles; it++) {
         const int st = it % OUT_STAGES;
+        if (it + PREFETCH_TILES < ntiles) tma_prefetch_4d(&tmQ, 0, (tile0 + it + PREFETCH_TILES) * TILE, h, b);
         if (!mbar_wait(&misc->empty[st], ((it / OUT_STAGES) & 1) ^ 1, abortp, status)) break;
         mbar_expect_tx(&misc->full[st], TILE_BYTES);
         tma_load_4d(sm + OutSmem::X0 + st * TILE_BYTES, &tmQ, &misc->full[st], 0, (tile0 + it) * TILE, h, b);
@@ -505,13 +480,11 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
     if (lane == 0) {
       constexpr uint32_t ID_LOGITS = idesc_bf16(128, TC_M, 0, 0);
       constexpr uint32_t ID_OUT = idesc_f16(128, TC_NV, 0, 0);      // fp16: phi(Q) <= 1 and the scaled S^T [V | 1]
-      const uint32_t sW = smem_u32(sm + OutSmem::W), sBaug = smem_u32(sm + OutSmem::BAUG), sAaug = smem_u32(sm + OutSmem::AAUG);
-      const uint32_t sWlo = smem_u32(sm + OutSmem::WLO);
-      const uint32_t sPhi = smem_u32(sm + OutSmem::PHI), sKvt = smem_u32(sm + OutSmem::KVT);
       const uint64_t dX0 = smem_desc(smem_u32(sm + OutSmem::X0), 16, 1024, SWZ_128B);
-      const uint64_t dW = smem_desc(sW, 16, 1024, SWZ_128B), dWlo = smem_desc(sWlo, 16, 1024, SWZ_128B);
-      const uint64_t dAaug = smem_desc(sAaug, 128, 256, SWZ_NONE), dBaug = smem_desc(sBaug, 128, 256, SWZ_NONE);
-      const uint64_t dPhi = smem_desc(sPhi, 16, 1024, SWZ_128B), dKvt = smem_desc(sKvt, 16, 1024, SWZ_128B);
+      const uint64_t dW = smem_desc(smem_u32(sm + OutSmem::W), 16, 1024, SWZ_128B);
+      const uint64_t dWlo = smem_desc(smem_u32(sm + OutSmem::WLO), 16, 1024, SWZ_128B);
+      const uint64_t dPhi = smem_desc(smem_u32(sm + OutSmem::PHI), 16, 1024, SWZ_128B);
+      const uint64_t dKvt = smem_desc(smem_u32(sm + OutSmem::KVT), 16, 1024, SWZ_128B);
       auto issue_logits = [&](int st) {
         const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
 #pragma unroll
@@ -520,7 +493,6 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
 #pragma unroll
         for (int k = 0; k < TC_D / 16; k++)
           mma_bf16(tmem + OUT_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dWlo, 32 * k), ID_LOGITS, 1);
-        mma_bf16(tmem + OUT_COL_LOGITS, dAaug, dBaug, ID_LOGITS, 1);
         mma_commit(&misc->logits_full);
         mma_commit(&misc->empty[st]);
       };
@@ -538,51 +510,59 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           tcgen05_fence_after();
           issue_logits(sn);
         }
+        // the epilogue arrives on phi_full only after it has read the previous tile's outputs
         if (!mbar_wait(&misc->phi_full, it & 1, abortp, status)) break;
         tcgen05_fence_after();
 #pragma unroll
-        for (int fb = 0; fb < TC_M / 64; fb++)
+        for (int fb = 0; fb < TC_M / 64; fb++)          // feature halves 0 (fb 0, 1) and 1 (fb 2, 3)
 #pragma unroll
           for (int k = 0; k < 4; k++)
-            mma_bf16(tmem + OUT_COL_OUT + (it & 1) * TC_NV, desc_advance(dPhi, fb * TILE_BYTES + 32 * k),
-                     desc_advance(dKvt, fb * KVT_BLOCK_BYTES + 32 * k), ID_OUT, (fb > 0 || k > 0) ? 1u : 0u);
+            mma_bf16(tmem + OUT_COL_OUT + (fb >> 1) * TC_NV, desc_advance(dPhi, fb * TILE_BYTES + 32 * k),
+                     desc_advance(dKvt, fb * KVT_BLOCK_BYTES + 32 * k), ID_OUT, ((fb & 1) || k > 0) ? 1u : 0u);
         mma_commit(&misc->phi_free);
-        mma_commit(&misc->out_full[it & 1]);
       }
     }
   } else {
+    // ---------------- epilogue warps: one query row per thread, 128 of the 256 features.
+    // Each half row is shifted by its own maximum, so no exchange between the two threads of a
+    // row precedes the exponentials; the two halves are contracted into separate accumulators and
+    // brought to the common shift when the tile's output is read (one tile later).
     const int q = warp & 3, hf = warp >> 2;
     const int row = q * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
     __nv_bfloat16* Yb = Y + b * ay.sb + h * ay.sh;
     bool alive = true;
-    // Y rows of tile j: [num | den] from TMEM, one divide per row, 32 of the 64 columns per thread
-    auto write_out = [&](int j) -> bool {
-      if (!mbar_wait(&misc->out_full[j & 1], (j >> 1) & 1, abortp, status, false)) return false;
+    // Y rows of tile j (its contraction has completed): 32 of the 64 columns per thread
+    auto write_out = [&](int j) {
       __syncwarp();
       tcgen05_fence_after();
-      uint32_t n0[16], n1[16], dn[16];
-      const uint32_t base = lane_addr + OUT_COL_OUT + (j & 1) * TC_NV;
-      tmem_ld16(base + hf * 32, n0);
-      tmem_ld16(base + hf * 32 + 16, n1);
-      tmem_ld16(base + TC_DV, dn);
+      uint32_t n0[32], n1[32], d0[16], d1[16];
+      const uint32_t base = lane_addr + OUT_COL_OUT;
+      tmem_ld16(base + hf * 32, reinterpret_cast<uint32_t(&)[16]>(n0[0]));
+      tmem_ld16(base + hf * 32 + 16, reinterpret_cast<uint32_t(&)[16]>(n0[16]));
+      tmem_ld16(base + TC_DV, d0);
+      tmem_ld16(base + TC_NV + hf * 32, reinterpret_cast<uint32_t(&)[16]>(n1[0]));
+      tmem_ld16(base + TC_NV + hf * 32 + 16, reinterpret_cast<uint32_t(&)[16]>(n1[16]));
+      tmem_ld16(base + TC_NV + TC_DV, d1);
       tmem_wait_ld();
+      const float* rm = rowmax + (j % 3) * 2 * TILE;
+      const float m0 = rm[row], m1 = rm[TILE + row];
+      const float m = fmaxf(m0, m1);
+      const float f0 = ex2(m0 - m), f1 = ex2(m1 - m);
       const int64_t r = (int64_t)(tile0 + j) * TILE + row;
       if (r < L) {
-        const float den = __uint_as_float(dn[0]);
+        const float den = fmaf(f0, __uint_as_float(d0[0]), f1 * __uint_as_float(d1[0]));
         if (!(den > 0.f) || !isfinite(den)) atomicExch(status, FSHARP_E_NONFINITE);
-        const float inv = 1.f / den;
+        const float i0 = f0 / den, i1 = f1 / den;
         uint32_t o[16];
 #pragma unroll
-        for (int i = 0; i < 8; i++) {
-          o[i] = pack_bf16(__uint_as_float(n0[2 * i]) * inv, __uint_as_float(n0[2 * i + 1]) * inv);
-          o[8 + i] = pack_bf16(__uint_as_float(n1[2 * i]) * inv, __uint_as_float(n1[2 * i + 1]) * inv);
-        }
+        for (int i = 0; i < 16; i++)
+          o[i] = pack_bf16(fmaf(i0, __uint_as_float(n0[2 * i]), i1 * __uint_as_float(n1[2 * i])),
+                           fmaf(i0, __uint_as_float(n0[2 * i + 1]), i1 * __uint_as_float(n1[2 * i + 1])));
         uint4* dst = reinterpret_cast<uint4*>(Yb + r * ay.sl + hf * 32);
 #pragma unroll
         for (int i = 0; i < 4; i++) dst[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
       }
-      return true;
     };
     for (int it = 0; it < ntiles && alive; it++) {
       if (!mbar_wait(&misc->logits_full, it & 1, abortp, status, false)) { alive = false; break; }
@@ -602,13 +582,12 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
       for (int i = 0; i < 128; i++) mxp[i & 3] = fmaxf(mxp[i & 3], __uint_as_float(v[i]));
-      float mx = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
-      float* rm = rowmax + (it & 1) * 2 * TILE;
-      rm[hf * TILE + row] = mx;
-      named_bar_sync(1, EPI_THREADS);
-      mx = fmaxf(mx, rm[(hf ^ 1) * TILE + row]);
+      const float mx = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
+      rowmax[(it % 3) * 2 * TILE + hf * TILE + row] = mx;
       if (it > 0) {
+        // contraction of the previous tile done: its phi tile and its outputs are ours again
         if (!mbar_wait(&misc->phi_free, (it - 1) & 1, abortp, status, false)) { alive = false; break; }
+        write_out(it - 1);
       }
       uint8_t* prow = sm + OutSmem::PHI + hf * 2 * TILE_BYTES + row * 128;
 #pragma unroll
@@ -622,9 +601,8 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       fence_proxy_async_smem();
       tcgen05_fence_before();
       mbar_arrive(&misc->phi_full);
-      if (it > 0) alive = write_out(it - 1);
     }
-    if (alive && ntiles > 0) write_out(ntiles - 1);
+    if (alive && ntiles > 0 && mbar_wait(&misc->phi_free, (ntiles - 1) & 1, abortp, status, false)) write_out(ntiles - 1);
   }
   tcgen05_fence_before();
   __syncthreads();
@@ -632,6 +610,23 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
     tcgen05_fence_after();
     tmem_dealloc(tmem, TMEM_COLS);
   }
+}
+
+// Splits `tiles` tiles of each of `units` independent units into blocks of equal tile count so that
+// (waves of blocks on `sms` SMs) x (tiles per block + fixed overhead) is smallest; ties go to fewer blocks.
+int pick_split(int units, int tiles, int sms, int max_split, int* tiles_per_split) {
+  int best = 1, best_cost = 0x7fffffff, best_tps = tiles;
+  for (int ns = 1; ns <= tiles && ns <= max_split; ns++) {
+    int tps = (tiles + ns - 1) / ns;
+    int real = (tiles + tps - 1) / tps;
+    if (real != ns) continue;
+    long long blocks = (long long)units * ns;
+    int waves = (int)((blocks + sms - 1) / sms);
+    int cost = waves * (tps + 4);    // a block's fill and drain cost about as much as four tiles
+    if (cost < best_cost) { best_cost = cost; best = ns; best_tps = tps; }
+  }
+  *tiles_per_split = best_tps;
+  return best;
 }
 
 }  // namespace
@@ -648,29 +643,14 @@ size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
 int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
                 const float* prep, void* Y, WsAlloc* ws);
 
-// Splits `tiles` tiles of each of `units` independent units into blocks of equal tile count so that
-// (waves of blocks on `sms` SMs) x (tiles per block + fixed overhead) is smallest; ties go to fewer blocks.
-static int pick_split(int units, int tiles, int sms, int max_split, int* tiles_per_split) {
-  int best = 1, best_cost = 0x7fffffff, best_tps = tiles;
-  for (int ns = 1; ns <= tiles && ns <= max_split; ns++) {
-    int tps = (tiles + ns - 1) / ns;
-    int real = (tiles + tps - 1) / tps;
-    if (real != ns) continue;
-    long long blocks = (long long)units * ns;
-    int waves = (int)((blocks + sms - 1) / sms);
-    int cost = waves * (tps + 4);    // a block's fill and drain cost about as much as four tiles
-    if (cost < best_cost) { best_cost = cost; best = ns; best_tps = tps; }
-  }
-  *tiles_per_split = best_tps;
-  return best;
-}
+constexpr int MAX_KEY_SPLIT = 64;
 
 size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
   const size_t BH = (size_t)dm->B * dm->H;
   const size_t G = fs_groups(dm);
-  const size_t max_split = 64;
   return ws_round(G * 2 * IMG_BYTES) + ws_round(G * 2 * FLAG_WORDS * 4 + 64) +
-         ws_round(BH * max_split * TC_M * TC_NV * 4) + 2 * ws_round(BH * max_split * 4) + ws_round(BH * TC_NV * TC_M * 2);
+         ws_round(BH * MAX_KEY_SPLIT * TC_M * TC_NV * 4) + 2 * ws_round(BH * MAX_KEY_SPLIT * 4) +
+         ws_round(BH * TC_NV * TC_M * 2);
 }
 
 int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
@@ -684,11 +664,11 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   // key side: the split of the key range that minimises (waves of blocks) x (tiles per block)
   const int ktiles = (Lk + TILE - 1) / TILE;
   int tps = 0;
-  int nsplit = pick_split(BH, ktiles, ctx->sm_count, 64, &tps);
-  float* partial = ws->take<float>((size_t)BH * 64 * TC_M * TC_NV);
-  float* shifts = ws->take<float>((size_t)BH * 64);
-  int* pmax = ws->take<int>((size_t)BH * 64);
-  FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * 64 * sizeof(int), ctx->stream));
+  int nsplit = pick_split(BH, ktiles, ctx->sm_count, MAX_KEY_SPLIT, &tps);
+  float* partial = ws->take<float>((size_t)BH * MAX_KEY_SPLIT * TC_M * TC_NV);
+  float* shifts = ws->take<float>((size_t)BH * MAX_KEY_SPLIT);
+  int* pmax = ws->take<int>((size_t)BH * MAX_KEY_SPLIT);
+  FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * MAX_KEY_SPLIT * sizeof(int), ctx->stream));
   __half* kvt = ws->take<__half>((size_t)BH * TC_NV * TC_M);
 
   CUtensorMap tmK, tmV, tmQ, tmKVt;
@@ -705,7 +685,7 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   FS_TIME_BEGIN(ctx, FS_K_TC_MERGE);
-  tc_merge_kernel<<<dim3(MERGE_SLICES, BH), 256, 0, ctx->stream>>>(partial, shifts, pmax, nsplit, kvt);
+  tc_merge_kernel<<<dim3(MERGE_SLICES, BH), 256, 0, ctx->stream>>>(partial, shifts, pmax, nsplit, images, H, dm->pool, kvt);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
 

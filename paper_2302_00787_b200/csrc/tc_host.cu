@@ -43,14 +43,7 @@ tc_prep_kernel(const float* __restrict__ prep, float qk_scale, uint8_t* __restri
     *reinterpret_cast<__nv_bfloat16*>(img + IMG_CHI + tc::sw128_offset(n, k)) = hi;
     *reinterpret_cast<__nv_bfloat16*>(img + IMG_CLO + tc::sw128_offset(n, k)) = lo;
   }
-  for (int e = tid; e < TC_M * 16; e += 256) {
-    int m = e / 16, k = e % 16;
-    float a = av[m] * FS_LOG2E;
-    __nv_bfloat16 hi = __float2bfloat16_rn(a);
-    __nv_bfloat16 lo = __float2bfloat16_rn(a - __bfloat162float(hi));
-    __nv_bfloat16 v = k == 0 ? hi : (k == 1 ? lo : __float2bfloat16_rn(0.f));
-    *reinterpret_cast<__nv_bfloat16*>(img + IMG_BAUG + tc::core16_offset(m, k)) = v;
-  }
+  for (int m = tid; m < TC_M; m += 256) reinterpret_cast<float*>(img + IMG_A2)[m] = 2.f * FS_LOG2E * av[m];
   if (lo_nonzero) atomicOr(&any_lo, 1);
   __syncthreads();
   if (tid == 0) {

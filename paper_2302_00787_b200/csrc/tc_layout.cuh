@@ -10,7 +10,6 @@ constexpr int TILE = 128;          // tokens per tile
 constexpr int EPI_THREADS = 256, WARP_TMA = 8, WARP_MMA = 9, TC_THREADS = 320;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t TILE_BYTES = 16384;          // 128 rows x 128 bytes
-constexpr uint32_t ONEST_BYTES = 4096;          // [16 rows x 128 tokens] K-major: row 0 = ones (the 1 of [V | 1])
 
 // Per (group, side) operand image, already in the shared-memory layouts the MMAs read:
 //   W     [256 features x 64]  K-major, 128-byte swizzle, bf16(log2e * qk_scale * W)
@@ -18,9 +17,10 @@ constexpr uint32_t ONEST_BYTES = 4096;          // [16 rows x 128 tokens] K-majo
 //                              bf16 rounding of W alone costs ~0.4% per feature)
 //   Chi   [64 x 64]            K-major, 128-byte swizzle, bf16 of log2e * qk_scale^2 * C (row n, col k = C[k][n])
 //   Clo   [64 x 64]            the bf16 remainder of the same matrix
-//   Baug  [256 features x 16]  8x16-byte core matrices: (a_hi, a_lo, 0, ...) with a = log2e * w^T A w
+//   a2    [256] fp32           2 log2e w_m^T A w_m: the factor 2^a2 of feature m (it appears once in
+//                              phi(Q) and once in phi(K)) is applied to row m of S^T [V | 1] by the merge
 constexpr uint32_t IMG_W = 0, IMG_W_BYTES = 32768, IMG_WLO = 32768, IMG_CHI = 65536, IMG_C_BYTES = 8192, IMG_CLO = 73728,
-                   IMG_BAUG = 81920, IMG_BAUG_BYTES = 8192, IMG_BYTES = 90112;
+                   IMG_A2 = 81920, IMG_A2_BYTES = 1024, IMG_BYTES = 82944;
 // S^T [V | 1] transposed, fp16: 4 blocks of [80 rows x 64 features], 128-byte swizzle
 constexpr uint32_t KVT_BLOCK_BYTES = 10240, KVT_BYTES = 40960;
 
