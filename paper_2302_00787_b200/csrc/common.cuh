@@ -50,6 +50,7 @@ enum {
   FS_K_STATS = 1, FS_K_FIT, FS_K_PREP, FS_K_ROWTERM, FS_K_LOGITS, FS_K_GROUPMAX, FS_K_EXPSHIFT, FS_K_KV,
   FS_K_PREFIX, FS_K_SCORES, FS_K_OUT, FS_K_PAIRS, FS_K_PAIRVAR_PREP, FS_K_PAIRVAR,
   FS_K_TC_PREP, FS_K_TC_KV, FS_K_TC_MERGE, FS_K_TC_OUT, FS_K_TC_CAUSAL_STATE, FS_K_TC_CAUSAL_PREFIX, FS_K_TC_CAUSAL_OUT,
+  FS_K_TC_STATS, FS_K_TC_ROWTERM,
   FS_K_COUNT
 };
 constexpr int FS_TIMING_SLOTS = 4096;
@@ -145,6 +146,9 @@ static inline int fs_groups(const fsharp_dims* dm) {
 // ---- stage entry points (host side, defined in the .cu files) -------------
 int fs_run_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dims* dm, int dtype,
                  float qk_scale, double* stats);
+// Tensor-core statistics (bf16, d = 64, 16-byte aligned rows); `stats` must already be zero.
+int fs_tc_stats_supported(const void* Q, const void* K, const fsharp_dims* dm, int dtype);
+int fs_tc_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dims* dm, float qk_scale, double* stats);
 int fs_run_fit(fsharp_ctx* ctx, const double* stats, int G, int d, int variant, double ridge,
                double* params, double* scratch);
 size_t fs_fit_scratch_doubles(int G, int d);

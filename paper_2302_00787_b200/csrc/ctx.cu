@@ -155,6 +155,8 @@ const char* fsharp_kernel_name(int id) {
     case FS_K_TC_CAUSAL_STATE: return "tc_causal_state_kernel";
     case FS_K_TC_CAUSAL_PREFIX: return "tc_causal_prefix_kernel";
     case FS_K_TC_CAUSAL_OUT: return "tc_causal_out_kernel";
+    case FS_K_TC_STATS: return "tc_stats_kernel";
+    case FS_K_TC_ROWTERM: return "tc_rowterm_kernel";
     default: return "";
   }
 }

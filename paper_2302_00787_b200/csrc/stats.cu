@@ -131,6 +131,7 @@ int fs_run_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dim
   const int G = fs_groups(dm);
   FS_CUDA_OK(cudaMemsetAsync(stats, 0, (size_t)G * StatsLayout{dm->d}.total() * sizeof(double), ctx->stream));
   if (dm->Lq == 0 && dm->Lk == 0) return FSHARP_OK;
+  if (ctx->impl != FSHARP_IMPL_SIMT && fs_tc_stats_supported(Q, K, dm, dtype)) return fs_tc_stats(ctx, Q, K, dm, qk_scale, stats);
   if (dtype == FSHARP_F32) return launch_stats<float>(ctx, Q, K, dm, qk_scale, stats);
   return launch_stats<__nv_bfloat16>(ctx, Q, K, dm, qk_scale, stats);
 }

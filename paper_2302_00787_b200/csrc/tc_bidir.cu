@@ -94,6 +94,8 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   tcgen05_fence_after();
   const uint32_t tmem = misc->tmem_base;
 
+  if (warp >= WARP_TMA) {
+  regs_release<REGS_PRODUCER>();
   if (warp == WARP_TMA) {
     if (lane == 0) {
       prefetch_tmap(&tmK);
@@ -143,18 +145,18 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       const uint64_t dVst1 = smem_desc(sV0 + TILE_BYTES, sOnes - sV0 - TILE_BYTES, 1024, SWZ_128B);
       auto issue_logits = [&](int st) {
         const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
-#pragma unroll
+#pragma unroll 1
         for (int k = 0; k < TC_D / 16; k++)
           mma_bf16(tmem + KV_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dW, 32 * k), ID_LOGITS, k > 0);
-#pragma unroll
+#pragma unroll 1
         for (int k = 0; k < TC_D / 16; k++)
           mma_bf16(tmem + KV_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dWlo, 32 * k), ID_LOGITS, 1);
         if (cdense) {
-#pragma unroll
+#pragma unroll 1
           for (int k = 0; k < TC_D / 16; k++)
             mma_bf16(tmem + KV_COL_T, desc_advance(dX, 32 * k), desc_advance(dChi, 32 * k), ID_T, k > 0);
           if (clo) {
-#pragma unroll
+#pragma unroll 1
             for (int k = 0; k < TC_D / 16; k++)
               mma_bf16(tmem + KV_COL_T, desc_advance(dX, 32 * k), desc_advance(dClo, 32 * k), ID_T, 1);
           }
@@ -179,9 +181,9 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         tcgen05_fence_after();
         const uint64_t dV = st ? dVst1 : dVst0;
         const uint32_t acc0 = it > 0 ? 1u : 0u;
-#pragma unroll
+#pragma unroll 1
         for (int hh = 0; hh < 2; hh++)
-#pragma unroll
+#pragma unroll 1
           for (int k = 0; k < TILE / 16; k++)
             mma_bf16(tmem + KV_COL_ACC + hh * TC_NV, desc_advance(dPhi, hh * 2 * TILE_BYTES + k * 2048),
                      desc_advance(dV, k * 2048), ID_KV, k > 0 ? 1u : acc0);
@@ -189,7 +191,9 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         mma_commit(&misc->empty[st]);
       }
     }
+  }
   } else {
+    regs_acquire<REGS_EPILOGUE>();
     // ---------------- epilogue warps: one key row per thread, 128 of the 256 features.
     // The running shift s is taken on trust while the exponentials are computed; the tile's
     // largest exponent is tracked on the side and checked afterwards.  Only if it exceeds the
@@ -452,6 +456,8 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
   tcgen05_fence_after();
   const uint32_t tmem = misc->tmem_base;
 
+  if (warp >= WARP_TMA) {
+  regs_release<REGS_PRODUCER>();
   if (warp == WARP_TMA) {
     if (lane == 0) {
       prefetch_tmap(&tmQ);
@@ -487,10 +493,10 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       const uint64_t dKvt = smem_desc(smem_u32(sm + OutSmem::KVT), 16, 1024, SWZ_128B);
       auto issue_logits = [&](int st) {
         const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
-#pragma unroll
+#pragma unroll 1
         for (int k = 0; k < TC_D / 16; k++)
           mma_bf16(tmem + OUT_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dW, 32 * k), ID_LOGITS, k > 0);
-#pragma unroll
+#pragma unroll 1
         for (int k = 0; k < TC_D / 16; k++)
           mma_bf16(tmem + OUT_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dWlo, 32 * k), ID_LOGITS, 1);
         mma_commit(&misc->logits_full);
@@ -513,16 +519,18 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         // the epilogue arrives on phi_full only after it has read the previous tile's outputs
         if (!mbar_wait(&misc->phi_full, it & 1, abortp, status)) break;
         tcgen05_fence_after();
-#pragma unroll
+#pragma unroll 1
         for (int fb = 0; fb < TC_M / 64; fb++)          // feature halves 0 (fb 0, 1) and 1 (fb 2, 3)
-#pragma unroll
+#pragma unroll 1
           for (int k = 0; k < 4; k++)
             mma_bf16(tmem + OUT_COL_OUT + (fb >> 1) * TC_NV, desc_advance(dPhi, fb * TILE_BYTES + 32 * k),
                      desc_advance(dKvt, fb * KVT_BLOCK_BYTES + 32 * k), ID_OUT, ((fb & 1) || k > 0) ? 1u : 0u);
         mma_commit(&misc->phi_free);
       }
     }
+  }
   } else {
+    regs_acquire<REGS_EPILOGUE>();
     // ---------------- epilogue warps: one query row per thread, 128 of the 256 features.
     // Each half row is shifted by its own maximum, so no exchange between the two threads of a
     // row precedes the exponentials; the two halves are contracted into separate accumulators and

@@ -69,6 +69,34 @@ def test_stats_pooled_over_batch_and_strided(ctx):
     assert np.abs(st2 - st).max() < 1e-12
 
 
+def test_stats_tensor_core_path_matches_simt_and_definition(ctx):
+    """bf16, d = 64 takes the tensor-core Gram kernel: several tiles, a ragged tail, unequal
+    query and key lengths, pooled and per-(batch, head) groups, and a query/key scale."""
+    w = W["cfg2"].scaled(B=2, H=3, L=1000)
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    dKs, Ks = dK[:, :, :333], K[:, :, :333]
+    for pool in (fb.POOL_PER_BH, fb.POOL_PER_HEAD):
+        st = host(ctx.fsharp_stats(dQ, dKs, pool=pool, qk_scale=0.75))
+        ctx.set_impl(fb.IMPL_SIMT)
+        try:
+            st_simt = host(ctx.fsharp_stats(dQ, dKs, pool=pool, qk_scale=0.75))
+        finally:
+            ctx.set_impl(fb.IMPL_AUTO)
+        assert ctx.status() == 0
+        assert np.abs(st - st_simt).max() < 2e-6 * np.abs(st_simt).max()
+        d = w.d
+        for g in range(st.shape[0]):
+            if pool == fb.POOL_PER_BH:
+                b, h = divmod(g, w.H)
+                ref = fs.set_statistics(0.75 * Q[b, h], 0.75 * Ks[b, h])
+            else:
+                ref = fs.set_statistics(0.75 * Q[:, g].reshape(-1, d), 0.75 * Ks[:, g].reshape(-1, d))
+            for name, lo in (("M1", 0), ("M2", d * d)):
+                assert np.abs(st[g][lo: lo + d * d].reshape(d, d) - ref[name]).max() < 2e-6 * np.abs(ref[name]).max()
+            assert np.abs(st[g][2 * d * d: 2 * d * d + d] - ref["mu4"]).max() < 2e-6
+            assert np.abs(st[g][2 * d * d + d: 2 * d * d + 2 * d] - ref["mu5"]).max() < 2e-6
+
+
 # ------------------------------------------------------------------ fits
 def invariants(p, d):
     """Quantities that do not depend on eigenvector signs or rotations in equal eigenvalues."""
