@@ -47,7 +47,6 @@ __device__ void jacobi_schedule(ushort2* sched, int d) {
     int r = e / half, k = e % half, p, q;
     if (k == 0) { p = r; q = d - 1; }
     else { p = (r + k) % (d - 1); q = (r - k + (d - 1)) % (d - 1); }
-    if (p > q) { int t = p; p = q; q = t; }
     sched[e] = make_ushort2((unsigned short)p, (unsigned short)q);
   }
   __syncthreads();
@@ -167,6 +166,190 @@ __device__ __forceinline__ int jacobi_eig(double* __restrict__ A, int lda, doubl
   return sweeps;
 }
 
+// The same iteration for matrices small enough that two copies of A fit in shared memory
+// (d <= 64), with three kinds of warps working on a round at the same time:
+//   warp 0            looks ahead: it evaluates, straight from the old copy of A, the three entries
+//                     (a_pp, a_qq, a_pq after round r) of every pair of round r + 1 and turns them
+//                     into that round's rotations;
+//   2 D threads       keep V^T in registers, half a column each, stored in "seat" order (seat 2k
+//                     holds row p_k of the current round, seat 2k + 1 row q_k), so the rotations
+//                     touch fixed registers; between rounds the tournament moves every index one
+//                     seat along, which is a fixed register permutation plus one exchange between
+//                     the two halves of a column;
+//   the other warps   apply round r to A, reading one copy and writing the other, so nothing is
+//                     updated in place.  A is symmetric: only the blocks on and above the block
+//                     diagonal are computed, each is stored twice.
+// One block barrier per round remains.
+//   pos : [(d-1) x d] for round r and index x, (pair number of x, 1 if x is the pair's q)
+//   tri : the (k, l), k <= l, block list
+// Returns the number of sweeps; *final_buf tells which copy (0: A0, 1: A1) holds the result.
+template <int D>
+__device__ __noinline__ int jacobi_eig_lookahead(double* __restrict__ A0, double* __restrict__ A1, int lda,
+                                                 double* __restrict__ VT, int ldvt, const ushort2* __restrict__ sched,
+                                                 const uchar2* __restrict__ pos, const uchar2* __restrict__ tri,
+                                                 double* __restrict__ cs_base, double* red, int* final_buf) {
+  constexpr int d = D, half = D / 2, nrounds = D - 1, N2 = D / 2;
+  constexpr int ntri = half * (half + 1) / 2;
+  constexpr int VT_THREADS = 2 * D;
+  constexpr int NW = FIT_THREADS - 32 - VT_THREADS;      // threads that apply the rotations to A
+  const int tid = threadIdx.x;
+  const bool vt_thread = tid >= 32 && tid < 32 + VT_THREADS;
+  const int vcol = (tid - 32) >> 1, vh = (tid - 32) & 1;  // column of V^T and which half of its seats
+  // index sitting at `seat` in round r
+  auto seat_index = [](int r, int seat) {
+    const int k = seat >> 1;
+    if (k == 0) return (seat & 1) ? d - 1 : r;
+    return (seat & 1) ? (r - k + nrounds) % nrounds : (r + k) % nrounds;
+  };
+  double x[N2];
+#pragma unroll
+  for (int j = 0; j < N2; j++) x[j] = (vt_thread && seat_index(0, vh * N2 + j) == vcol) ? 1.0 : 0.0;
+  auto angle = [](double app, double aqq, double apq, double& c, double& s) {
+    c = 1.0; s = 0.0;
+    const float num = (float)(aqq - app), den = (float)(2.0 * apq);
+    if (den != 0.f) {
+      const float zeta = __fdividef(num, den);
+      const float tf = __fdividef(copysignf(1.f, zeta), fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f)));
+      if (isfinite(tf)) {
+        const double t = (double)tf;
+        const double xx = fma(t, t, 1.0);
+        const double c0 = (double)rsqrtf(fmaf(tf, tf, 1.f));
+        c = c0 * fma(-0.5 * xx, c0 * c0, 1.5);      // one Newton step: |c^2 x - 1| ~ 1e-14
+        s = t * c;
+      }
+    }
+  };
+  int sweeps = 0, rr = 0;                           // rr: rounds done so far; A lives in copy rr & 1
+  for (int sweep = 0; sweep < JACOBI_MAX_SWEEPS; sweep++) {
+    const double* Ac = (rr & 1) ? A1 : A0;
+    double off = 0.0, tot = 0.0;
+    for (int e = tid; e < d * d; e += FIT_THREADS) {
+      int i = e / d, j = e % d;
+      double v = Ac[i * lda + j];
+      tot += v * v;
+      if (i != j) off += v * v;
+    }
+    off = block_reduce(off, red, 0);
+    tot = block_reduce(tot, red, 0);
+    if (off <= 1e-24 * tot || tot == 0.0) break;
+    sweeps++;
+    if (sweep == 0) {                               // later sweeps inherit round 0's rotations from the look-ahead
+      if (tid < half) {
+        const int p = sched[tid].x, q = sched[tid].y;
+        double c, s;
+        angle(Ac[p * lda + p], Ac[q * lda + q], Ac[p * lda + q], c, s);
+        cs_base[2 * tid] = c; cs_base[2 * tid + 1] = s;
+      }
+      __syncthreads();
+    }
+    for (int r = 0; r < nrounds; r++, rr++) {
+      const double* __restrict__ Ao = (rr & 1) ? A1 : A0;
+      double* __restrict__ An = (rr & 1) ? A0 : A1;
+      const ushort2* sr = sched + r * half;
+      const double* cs = cs_base + (rr & 1) * d;
+      if (tid < 32) {
+        // look-ahead: rotations of the next round from entries of J^T A J evaluated directly
+        if (tid < half) {
+          const int rn = (r + 1 == nrounds) ? 0 : r + 1;
+          const uchar2* pr = pos + r * d;
+          const ushort2 nx = sched[rn * half + tid];
+          auto coef = [&](int xi, int& ip, int& iq, double& fp, double& fq) {
+            const uchar2 px = pr[xi];
+            const ushort2 pq = sr[px.x];
+            const double c = cs[2 * px.x], s = cs[2 * px.x + 1];
+            ip = pq.x; iq = pq.y;
+            fp = px.y ? s : c;                     // new row/column x = fp * old p + fq * old q
+            fq = px.y ? c : -s;
+          };
+          int pp, pq_, qp, qq_;
+          double fpp, fpq, fqp, fqq;
+          coef(nx.x, pp, pq_, fpp, fpq);           // the next pair's p
+          coef(nx.y, qp, qq_, fqp, fqq);           // the next pair's q
+          const double a_pp_pp = Ao[pp * lda + pp], a_pp_pq = Ao[pp * lda + pq_], a_pq_pq = Ao[pq_ * lda + pq_];
+          const double a_qp_qp = Ao[qp * lda + qp], a_qp_qq = Ao[qp * lda + qq_], a_qq_qq = Ao[qq_ * lda + qq_];
+          const double b00 = Ao[pp * lda + qp], b01 = Ao[pp * lda + qq_], b10 = Ao[pq_ * lda + qp], b11 = Ao[pq_ * lda + qq_];
+          const double napp = fpp * (fpp * a_pp_pp + fpq * a_pp_pq) + fpq * (fpp * a_pp_pq + fpq * a_pq_pq);
+          const double naqq = fqp * (fqp * a_qp_qp + fqq * a_qp_qq) + fqq * (fqp * a_qp_qq + fqq * a_qq_qq);
+          const double napq = fqp * (fpp * b00 + fpq * b10) + fqq * (fpp * b01 + fpq * b11);
+          double c, s;
+          angle(napp, naqq, napq, c, s);
+          double* csn = cs_base + ((rr + 1) & 1) * d;
+          csn[2 * tid] = c; csn[2 * tid + 1] = s;
+        }
+      } else if (tid < 32 + VT_THREADS) {
+        // V^T <- J^T V^T on this thread's half column, then every index moves one seat along
+        const double2* cs2 = reinterpret_cast<const double2*>(cs) + vh * (N2 / 2);
+#pragma unroll
+        for (int jj = 0; jj < N2 / 2; jj++) {
+          const double2 r2 = cs2[jj];
+          const double a = x[2 * jj], b = x[2 * jj + 1];
+          x[2 * jj] = r2.x * a - r2.y * b;
+          x[2 * jj + 1] = r2.y * a + r2.x * b;
+        }
+        // Even seats move down by two, odd seats up by two; seat 1 is fixed, seat 0 goes to seat 3,
+        // the last odd seat to the last even one.  Two values cross between the halves of a column.
+        const double send = vh ? x[0] : x[N2 - 1];
+        const double recv = __shfl_xor_sync(0xffffffffu, send, 1);
+        const double t0 = x[0];
+#pragma unroll
+        for (int j = 0; j <= N2 - 4; j += 2) x[j] = x[j + 2];
+        x[N2 - 2] = vh ? x[N2 - 1] : recv;
+#pragma unroll
+        for (int j = N2 - 1; j >= 5; j -= 2) x[j] = x[j - 2];
+        x[3] = vh ? x[1] : t0;
+        x[1] = vh ? recv : x[1];
+      } else {
+        const int wid = tid - 32 - VT_THREADS;
+        for (int e = wid; e < ntri; e += NW) {
+          const uchar2 kl = tri[e];
+          const int k = kl.x, l = kl.y;
+          const int pk = sr[k].x, qk = sr[k].y, pl = sr[l].x, ql = sr[l].y;
+          const double2 rk = reinterpret_cast<const double2*>(cs)[k], rl = reinterpret_cast<const double2*>(cs)[l];
+          const double ck = rk.x, sk = rk.y, cl = rl.x, sl = rl.y;
+          const double a00 = Ao[pk * lda + pl], a01 = Ao[pk * lda + ql], a10 = Ao[qk * lda + pl], a11 = Ao[qk * lda + ql];
+          // left: rows (p_k, q_k) <- (c x - s y, s x + c y); right: the same on columns (p_l, q_l)
+          const double r00 = ck * a00 - sk * a10, r01 = ck * a01 - sk * a11;
+          const double r10 = sk * a00 + ck * a10, r11 = sk * a01 + ck * a11;
+          const double n00 = cl * r00 - sl * r01, n01 = sl * r00 + cl * r01;
+          const double n10 = cl * r10 - sl * r11, n11 = sl * r10 + cl * r11;
+          if (k == l) {
+            const double o = 0.5 * (n01 + n10);
+            An[pk * lda + pk] = n00; An[qk * lda + qk] = n11; An[pk * lda + qk] = o; An[qk * lda + pk] = o;
+          } else {
+            An[pk * lda + pl] = n00; An[pk * lda + ql] = n01; An[qk * lda + pl] = n10; An[qk * lda + ql] = n11;
+            An[pl * lda + pk] = n00; An[ql * lda + pk] = n01; An[pl * lda + qk] = n10; An[ql * lda + qk] = n11;
+          }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  // the seats now hold the order of round rr mod (d - 1): put the rows of V^T back
+  if (vt_thread) {
+    const int rf = rr % nrounds;
+#pragma unroll
+    for (int j = 0; j < N2; j++) VT[seat_index(rf, vh * N2 + j) * ldvt + vcol] = x[j];
+  }
+  __syncthreads();
+  *final_buf = rr & 1;
+  return sweeps;
+}
+
+// Tables of jacobi_eig_lookahead: where every index sits in every round, and the block list.
+__device__ void jacobi_tables(const ushort2* sched, uchar2* pos, uchar2* tri, int d) {
+  const int half = d >> 1;
+  for (int e = threadIdx.x; e < (d - 1) * half; e += FIT_THREADS) {
+    const int r = e / half, k = e % half;
+    pos[r * d + sched[e].x] = make_uchar2((unsigned char)k, 0);
+    pos[r * d + sched[e].y] = make_uchar2((unsigned char)k, 1);
+  }
+  for (int e = threadIdx.x; e < half * half; e += FIT_THREADS) {
+    const int k = e / half, l = e % half;
+    if (k <= l) tri[k * half - k * (k - 1) / 2 + (l - k)] = make_uchar2((unsigned char)k, (unsigned char)l);
+  }
+  __syncthreads();
+}
+
 struct FitArgs {
   const double* stats;
   double* params;
@@ -179,7 +362,7 @@ struct FitArgs {
 
 template <bool V_IN_SMEM>
 __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
-  extern __shared__ double sm[];
+  extern __shared__ __align__(16) double sm[];
   const int d = a.d, tid = threadIdx.x, g = blockIdx.x;
   const int lda = d + 1;
   StatsLayout sl{d};
@@ -189,18 +372,37 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
   double* gs = a.scratch + (size_t)g * 4 * d * d;
 
   double* As = sm;                                   // d*(d+1)
-  double* Vs = V_IN_SMEM ? As + d * lda : gs;        // eigenvectors, one per ROW
+  double* A1 = As + d * lda;                         // second copy of A (look-ahead solver only)
+  double* Vs = V_IN_SMEM ? A1 + d * lda : gs;        // eigenvectors, one per ROW
   const int ldv = V_IN_SMEM ? lda : d;
-  double* vec = As + d * lda + (V_IN_SMEM ? d * lda : 0);
+  double* vec = As + d * lda + (V_IN_SMEM ? 2 * d * lda : 0);
   double* lam = vec;             // [d]
   double* aux = vec + d;         // [d]
   double* cs = vec + 2 * d;      // [2d]
   double* red = vec + 4 * d;     // [FIT_THREADS]
   int* perm = reinterpret_cast<int*>(red + FIT_THREADS);          // [d]
   ushort2* sched = reinterpret_cast<ushort2*>(perm + d);          // [(d-1) * d/2]
+  uchar2* pos = reinterpret_cast<uchar2*>(sched + (d - 1) * (d / 2));   // [(d-1) * d]      (look-ahead solver only)
+  uchar2* tri = pos + (d - 1) * d;                                      // [d/2 (d/2 + 1) / 2]
   int log2d = 0;
   while ((1 << log2d) < d) log2d++;
-  if (a.variant == FSHARP_SDERF || a.variant == FSHARP_ADERF) jacobi_schedule(sched, d);
+  if (a.variant == FSHARP_SDERF || a.variant == FSHARP_ADERF) {
+    jacobi_schedule(sched, d);
+    if (V_IN_SMEM) jacobi_tables(sched, pos, tri, d);
+  }
+  // eigen-decomposition of the matrix in As: eigenvalues on its diagonal, eigenvectors in the rows of Vs
+  auto eig = [&]() -> int {
+    if (!V_IN_SMEM) return jacobi_eig(As, lda, Vs, ldv, d, log2d, sched, cs, red);
+    int buf = 0, n = 0;
+    if (d == 64) n = jacobi_eig_lookahead<64>(As, A1, lda, Vs, ldv, sched, pos, tri, cs, red, &buf);
+    else if (d == 32) n = jacobi_eig_lookahead<32>(As, A1, lda, Vs, ldv, sched, pos, tri, cs, red, &buf);
+    else n = jacobi_eig_lookahead<16>(As, A1, lda, Vs, ldv, sched, pos, tri, cs, red, &buf);
+    if (buf) {
+      for (int e = tid; e < d * lda; e += FIT_THREADS) As[e] = A1[e];
+      __syncthreads();
+    }
+    return n;
+  };
 
   const double* M1 = st + sl.M(1);
   const double* M2 = st + sl.M(2);
@@ -276,7 +478,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
       As[i * lda + j] = M1[e] + M2[e] + mu4[i] * mu5[j] + mu5[i] * mu4[j] + (i == j ? rg1 + rg2 : 0.0);
     }
     __syncthreads();
-    nsweeps += jacobi_eig(As, lda, Vs, ldv, d, log2d, sched, cs, red);
+    nsweeps += eig();
     for (int i = tid; i < d; i += FIT_THREADS) {
       double li = As[i * lda + i];
       int rank = 0;
@@ -316,7 +518,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
       As[i * lda + j] = M1[e] + (i == j ? rg1 : 0.0);
     }
     __syncthreads();
-    nsweeps += jacobi_eig(As, lda, Vs, ldv, d, log2d, sched, cs, red);
+    nsweeps += eig();
     double lmin = 1e300, lmax = 0.0;
     for (int i = tid; i < d; i += FIT_THREADS) {
       double li = As[i * lda + i];
@@ -349,7 +551,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
       As[c * lda + r] = v;
     }
     __syncthreads();
-    nsweeps += jacobi_eig(As, lda, Vs, ldv, d, log2d, sched, cs, red);     // eigenvalues Sigma^2, eigenvectors U
+    nsweeps += eig();     // eigenvalues Sigma^2, eigenvectors U
     double smin = 1e300, smax = 0.0, ssum = 0.0;
     for (int l = tid; l < d; l += FIT_THREADS) {
       double sg = sqrt(fmax(As[l * lda + l], 0.0));
@@ -406,8 +608,9 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
 }
 
 size_t fit_smem_bytes(int d, int v_in_smem) {
-  size_t dbl = (size_t)d * (d + 1) * (v_in_smem ? 2 : 1) + 4 * (size_t)d + FIT_THREADS;
-  return dbl * sizeof(double) + (size_t)d * sizeof(int) + (size_t)(d - 1) * (d / 2) * sizeof(ushort2);
+  size_t dbl = (size_t)d * (d + 1) * (v_in_smem ? 3 : 1) + 4 * (size_t)d + FIT_THREADS;
+  size_t tables = v_in_smem ? ((size_t)(d - 1) * d + (size_t)(d / 2) * (d / 2 + 1) / 2) * sizeof(uchar2) : 0;
+  return dbl * sizeof(double) + (size_t)d * sizeof(int) + (size_t)(d - 1) * (d / 2) * sizeof(ushort2) + tables;
 }
 
 }  // namespace
