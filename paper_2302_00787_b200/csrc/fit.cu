@@ -167,116 +167,156 @@ __device__ __forceinline__ int jacobi_eig(double* __restrict__ A, int lda, doubl
 }
 
 // The same iteration for matrices small enough that two copies of A fit in shared memory
-// (d <= 64), with three kinds of warps working on a round at the same time:
-//   warp 0            looks ahead: it evaluates, straight from the old copy of A, the three entries
-//                     (a_pp, a_qq, a_pq after round r) of every pair of round r + 1 and turns them
-//                     into that round's rotations;
-//   2 D threads       keep V^T in registers, half a column each, stored in "seat" order (seat 2k
-//                     holds row p_k of the current round, seat 2k + 1 row q_k), so the rotations
-//                     touch fixed registers; between rounds the tournament moves every index one
-//                     seat along, which is a fixed register permutation plus one exchange between
-//                     the two halves of a column;
-//   the other warps   apply round r to A, reading one copy and writing the other, so nothing is
-//                     updated in place.  A is symmetric: only the blocks on and above the block
-//                     diagonal are computed, each is stored twice.
-// One block barrier per round remains.
-//   pos : [(d-1) x d] for round r and index x, (pair number of x, 1 if x is the pair's q)
+// (d <= 64), with three kinds of warps working on a round at the same time, each in a loop of
+// its own (jacobi_role) so that the register needs of one do not constrain the others:
+//   JR_AHEAD  warp 0 looks ahead: it evaluates, straight from the old copy of A, the three
+//             entries (a_pp, a_qq, a_pq after round r) of every pair of round r + 1 and turns
+//             them into that round's rotations;
+//   JR_VT     2 D threads keep V^T in registers, half a column each, stored in "seat" order
+//             (seat 2k holds row p_k of the current round, seat 2k + 1 row q_k), so the rotations
+//             touch fixed registers; between rounds the tournament moves every index one seat
+//             along, which is a fixed register permutation plus one exchange between the two
+//             halves of a column.  Afterwards they help with A;
+//   JR_A      the other warps apply round r to A, reading one copy and writing the other, so
+//             nothing is updated in place.  A is symmetric: only the blocks on and above the
+//             block diagonal are computed, and element (i, j) lives at [min(i, j)][max(i, j)]
+//             only; the block list pairs block row k with block row d/2 - k, which keeps the
+//             shared-memory bank conflicts of a warp's accesses low.
+// One block barrier per round remains; the three loops meet at the same barriers.
+//   la  : [(d-1) x d/2] for round r and pair j of round r + 1, where that pair's two indices sit in
+//         round r: x = rows (p, q) of both current pairs, y = the two pair numbers and two flags
+//         (bit 16: the next p is its current pair's q; bit 17: the same for the next q)
 //   tri : the (k, l), k <= l, block list
-// Returns the number of sweeps; *final_buf tells which copy (0: A0, 1: A1) holds the result.
+struct JacobiCtx {
+  double* A0; double* A1; double* VT; double* cs_base; double* red;
+  const ushort2* sched; const uint2* la; const uchar2* tri;
+  int lda, ldvt;
+};
+enum { JR_AHEAD = 0, JR_VT = 1, JR_A = 2 };
+
+// (c, s) that annihilates a_pq, from fp32 arithmetic with two special-function calls, then made
+// orthonormal in fp64 (one Newton step on c^2 + s^2 = 1).  An angle accurate to 1e-7 still
+// removes a_pq to that relative level and keeps V exactly orthogonal.  scale brings the entries
+// to order one so that the fp32 squares neither overflow nor vanish.
+__device__ __forceinline__ void jacobi_angle(double app, double aqq, double apq, double scale, double& c, double& s) {
+  c = 1.0; s = 0.0;
+  const float num = (float)((aqq - app) * scale), den = (float)((apq + apq) * scale);
+  const float h2 = fmaf(num, num, den * den);
+  const float u = fabsf(num) + h2 * rsqrtf(h2);            // |num| + hypot(num, den)
+  const float rw = rsqrtf(fmaf(u, u, den * den));
+  const float c0 = u * rw, s0 = copysignf(1.f, num) * den * rw;
+  if (den != 0.f && isfinite(c0) && isfinite(s0)) {        // zero or non-finite: no rotation
+    const double cd = (double)c0, sd = (double)s0;
+    const double f = fma(-0.5, fma(cd, cd, sd * sd), 1.5);
+    c = cd * f; s = sd * f;
+  }
+}
+
+// where element (i, j) of the symmetric matrix is kept
+__device__ __forceinline__ int jacobi_upper(int i, int j, int lda) { return i < j ? i * lda + j : j * lda + i; }
+
 template <int D>
-__device__ __noinline__ int jacobi_eig_lookahead(double* __restrict__ A0, double* __restrict__ A1, int lda,
-                                                 double* __restrict__ VT, int ldvt, const ushort2* __restrict__ sched,
-                                                 const uchar2* __restrict__ pos, const uchar2* __restrict__ tri,
-                                                 double* __restrict__ cs_base, double* red, int* final_buf) {
+__device__ __forceinline__ void jacobi_a_items(const JacobiCtx& jc, const double* __restrict__ Ao, double* __restrict__ An,
+                                               const ushort2* sr, const double* cs, int wid, int nw) {
+  constexpr int half = D / 2, ntri = half * (half + 1) / 2;
+  const int lda = jc.lda;
+  for (int e = wid; e < ntri; e += nw) {
+    const uchar2 kl = jc.tri[e];
+    const int k = kl.x, l = kl.y;
+    const int pk = sr[k].x, qk = sr[k].y, pl = sr[l].x, ql = sr[l].y;
+    const double2 rk = reinterpret_cast<const double2*>(cs)[k], rl = reinterpret_cast<const double2*>(cs)[l];
+    const double ck = rk.x, sk = rk.y, cl = rl.x, sl = rl.y;
+    const int i00 = jacobi_upper(pk, pl, lda), i01 = jacobi_upper(pk, ql, lda), i10 = jacobi_upper(qk, pl, lda), i11 = jacobi_upper(qk, ql, lda);
+    const double a00 = Ao[i00], a01 = Ao[i01], a10 = Ao[i10], a11 = Ao[i11];
+    // left: rows (p_k, q_k) <- (c x - s y, s x + c y); right: the same on columns (p_l, q_l)
+    const double r00 = ck * a00 - sk * a10, r01 = ck * a01 - sk * a11;
+    const double r10 = sk * a00 + ck * a10, r11 = sk * a01 + ck * a11;
+    const double n00 = cl * r00 - sl * r01, n01 = sl * r00 + cl * r01;
+    const double n10 = cl * r10 - sl * r11, n11 = sl * r10 + cl * r11;
+    if (k == l) {
+      An[i00] = n00; An[i11] = n11; An[i01] = 0.5 * (n01 + n10);       // i01 == i10
+    } else {
+      An[i00] = n00; An[i01] = n01; An[i10] = n10; An[i11] = n11;
+    }
+  }
+}
+
+// Returns the number of sweeps; *final_buf tells which copy (0: A0, 1: A1) holds the result.
+template <int D, int ROLE>
+__device__ __forceinline__ int jacobi_role(const JacobiCtx& jc_in, int* final_buf) {
+  const JacobiCtx jc = jc_in;                            // by value: the fields stay in registers
   constexpr int d = D, half = D / 2, nrounds = D - 1, N2 = D / 2;
-  constexpr int ntri = half * (half + 1) / 2;
   constexpr int VT_THREADS = 2 * D;
-  constexpr int NW = FIT_THREADS - 32 - VT_THREADS;      // threads that apply the rotations to A
-  const int tid = threadIdx.x;
-  const bool vt_thread = tid >= 32 && tid < 32 + VT_THREADS;
-  const int vcol = (tid - 32) >> 1, vh = (tid - 32) & 1;  // column of V^T and which half of its seats
+  constexpr int NW = FIT_THREADS - 32;                   // threads that work on A (the V^T threads after their own work)
+  const int tid = threadIdx.x, lda = jc.lda;
+  const int vcol = (tid - 32) >> 1, vh = (tid - 32) & 1;  // JR_VT: column of V^T and which half of its seats
+  // JR_A threads come first in the item order, so the V^T threads only pick up what is left
+  // when the others have one item each
+  const int wid = ROLE == JR_A ? tid - 32 - VT_THREADS : tid - 32 + (FIT_THREADS - 32 - VT_THREADS);
   // index sitting at `seat` in round r
   auto seat_index = [](int r, int seat) {
     const int k = seat >> 1;
     if (k == 0) return (seat & 1) ? d - 1 : r;
     return (seat & 1) ? (r - k + nrounds) % nrounds : (r + k) % nrounds;
   };
-  double x[N2];
+  double x[ROLE == JR_VT ? N2 : 1];
+  if (ROLE == JR_VT) {
 #pragma unroll
-  for (int j = 0; j < N2; j++) x[j] = (vt_thread && seat_index(0, vh * N2 + j) == vcol) ? 1.0 : 0.0;
-  auto angle = [](double app, double aqq, double apq, double& c, double& s) {
-    c = 1.0; s = 0.0;
-    const float num = (float)(aqq - app), den = (float)(2.0 * apq);
-    if (den != 0.f) {
-      const float zeta = __fdividef(num, den);
-      const float tf = __fdividef(copysignf(1.f, zeta), fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.f)));
-      if (isfinite(tf)) {
-        const double t = (double)tf;
-        const double xx = fma(t, t, 1.0);
-        const double c0 = (double)rsqrtf(fmaf(tf, tf, 1.f));
-        c = c0 * fma(-0.5 * xx, c0 * c0, 1.5);      // one Newton step: |c^2 x - 1| ~ 1e-14
-        s = t * c;
-      }
-    }
-  };
+    for (int j = 0; j < N2; j++) x[j] = seat_index(0, vh * N2 + j) == vcol ? 1.0 : 0.0;
+  }
   int sweeps = 0, rr = 0;                           // rr: rounds done so far; A lives in copy rr & 1
   for (int sweep = 0; sweep < JACOBI_MAX_SWEEPS; sweep++) {
-    const double* Ac = (rr & 1) ? A1 : A0;
+    const double* Ac = (rr & 1) ? jc.A1 : jc.A0;
     double off = 0.0, tot = 0.0;
     for (int e = tid; e < d * d; e += FIT_THREADS) {
       int i = e / d, j = e % d;
+      if (i > j) continue;
       double v = Ac[i * lda + j];
-      tot += v * v;
-      if (i != j) off += v * v;
+      tot += i == j ? v * v : 2.0 * v * v;
+      if (i != j) off += 2.0 * v * v;
     }
-    off = block_reduce(off, red, 0);
-    tot = block_reduce(tot, red, 0);
+    off = block_reduce(off, jc.red, 0);
+    tot = block_reduce(tot, jc.red, 0);
     if (off <= 1e-24 * tot || tot == 0.0) break;
     sweeps++;
+    const double scale = ROLE == JR_AHEAD ? rsqrt(tot * (1.0 / d)) : 0.0;      // entries of A -> order one
     if (sweep == 0) {                               // later sweeps inherit round 0's rotations from the look-ahead
-      if (tid < half) {
-        const int p = sched[tid].x, q = sched[tid].y;
+      if (ROLE == JR_AHEAD && tid < half) {
+        const int p = jc.sched[tid].x, q = jc.sched[tid].y;
         double c, s;
-        angle(Ac[p * lda + p], Ac[q * lda + q], Ac[p * lda + q], c, s);
-        cs_base[2 * tid] = c; cs_base[2 * tid + 1] = s;
+        jacobi_angle(Ac[p * lda + p], Ac[q * lda + q], Ac[jacobi_upper(p, q, lda)], scale, c, s);
+        jc.cs_base[2 * tid] = c; jc.cs_base[2 * tid + 1] = s;
       }
       __syncthreads();
     }
     for (int r = 0; r < nrounds; r++, rr++) {
-      const double* __restrict__ Ao = (rr & 1) ? A1 : A0;
-      double* __restrict__ An = (rr & 1) ? A0 : A1;
-      const ushort2* sr = sched + r * half;
-      const double* cs = cs_base + (rr & 1) * d;
-      if (tid < 32) {
-        // look-ahead: rotations of the next round from entries of J^T A J evaluated directly
+      const double* __restrict__ Ao = (rr & 1) ? jc.A1 : jc.A0;
+      double* __restrict__ An = (rr & 1) ? jc.A0 : jc.A1;
+      const ushort2* sr = jc.sched + r * half;
+      const double* cs = jc.cs_base + (rr & 1) * d;
+      if (ROLE == JR_AHEAD) {
+        // rotations of the next round from entries of J^T A J evaluated directly
         if (tid < half) {
-          const int rn = (r + 1 == nrounds) ? 0 : r + 1;
-          const uchar2* pr = pos + r * d;
-          const ushort2 nx = sched[rn * half + tid];
-          auto coef = [&](int xi, int& ip, int& iq, double& fp, double& fq) {
-            const uchar2 px = pr[xi];
-            const ushort2 pq = sr[px.x];
-            const double c = cs[2 * px.x], s = cs[2 * px.x + 1];
-            ip = pq.x; iq = pq.y;
-            fp = px.y ? s : c;                     // new row/column x = fp * old p + fq * old q
-            fq = px.y ? c : -s;
-          };
-          int pp, pq_, qp, qq_;
-          double fpp, fpq, fqp, fqq;
-          coef(nx.x, pp, pq_, fpp, fpq);           // the next pair's p
-          coef(nx.y, qp, qq_, fqp, fqq);           // the next pair's q
-          const double a_pp_pp = Ao[pp * lda + pp], a_pp_pq = Ao[pp * lda + pq_], a_pq_pq = Ao[pq_ * lda + pq_];
-          const double a_qp_qp = Ao[qp * lda + qp], a_qp_qq = Ao[qp * lda + qq_], a_qq_qq = Ao[qq_ * lda + qq_];
-          const double b00 = Ao[pp * lda + qp], b01 = Ao[pp * lda + qq_], b10 = Ao[pq_ * lda + qp], b11 = Ao[pq_ * lda + qq_];
+          const uint2 t = jc.la[r * half + tid];
+          const int pp = t.x & 255, pq_ = (t.x >> 8) & 255, qp = (t.x >> 16) & 255, qq_ = t.x >> 24;
+          const double2 rx = reinterpret_cast<const double2*>(cs)[t.y & 255], ry = reinterpret_cast<const double2*>(cs)[(t.y >> 8) & 255];
+          const double a_pp_pp = Ao[pp * lda + pp], a_pp_pq = Ao[jacobi_upper(pp, pq_, lda)], a_pq_pq = Ao[pq_ * lda + pq_];
+          const double a_qp_qp = Ao[qp * lda + qp], a_qp_qq = Ao[jacobi_upper(qp, qq_, lda)], a_qq_qq = Ao[qq_ * lda + qq_];
+          const double b00 = Ao[jacobi_upper(pp, qp, lda)], b01 = Ao[jacobi_upper(pp, qq_, lda)];
+          const double b10 = Ao[jacobi_upper(pq_, qp, lda)], b11 = Ao[jacobi_upper(pq_, qq_, lda)];
+          // new row/column x = f.p * old p + f.q * old q of x's current pair
+          const bool xq = (t.y >> 16) & 1, yq = (t.y >> 17) & 1;
+          const double fpp = xq ? rx.y : rx.x, fpq = xq ? rx.x : -rx.y;
+          const double fqp = yq ? ry.y : ry.x, fqq = yq ? ry.x : -ry.y;
           const double napp = fpp * (fpp * a_pp_pp + fpq * a_pp_pq) + fpq * (fpp * a_pp_pq + fpq * a_pq_pq);
           const double naqq = fqp * (fqp * a_qp_qp + fqq * a_qp_qq) + fqq * (fqp * a_qp_qq + fqq * a_qq_qq);
           const double napq = fqp * (fpp * b00 + fpq * b10) + fqq * (fpp * b01 + fpq * b11);
           double c, s;
-          angle(napp, naqq, napq, c, s);
-          double* csn = cs_base + ((rr + 1) & 1) * d;
+          jacobi_angle(napp, naqq, napq, scale, c, s);
+          double* csn = jc.cs_base + ((rr + 1) & 1) * d;
           csn[2 * tid] = c; csn[2 * tid + 1] = s;
         }
-      } else if (tid < 32 + VT_THREADS) {
+      } else if (ROLE == JR_VT) {
         // V^T <- J^T V^T on this thread's half column, then every index moves one seat along
         const double2* cs2 = reinterpret_cast<const double2*>(cs) + vh * (N2 / 2);
 #pragma unroll
@@ -298,45 +338,34 @@ __device__ __noinline__ int jacobi_eig_lookahead(double* __restrict__ A0, double
         for (int j = N2 - 1; j >= 5; j -= 2) x[j] = x[j - 2];
         x[3] = vh ? x[1] : t0;
         x[1] = vh ? recv : x[1];
+        jacobi_a_items<D>(jc, Ao, An, sr, cs, wid, NW);
       } else {
-        const int wid = tid - 32 - VT_THREADS;
-        for (int e = wid; e < ntri; e += NW) {
-          const uchar2 kl = tri[e];
-          const int k = kl.x, l = kl.y;
-          const int pk = sr[k].x, qk = sr[k].y, pl = sr[l].x, ql = sr[l].y;
-          const double2 rk = reinterpret_cast<const double2*>(cs)[k], rl = reinterpret_cast<const double2*>(cs)[l];
-          const double ck = rk.x, sk = rk.y, cl = rl.x, sl = rl.y;
-          const double a00 = Ao[pk * lda + pl], a01 = Ao[pk * lda + ql], a10 = Ao[qk * lda + pl], a11 = Ao[qk * lda + ql];
-          // left: rows (p_k, q_k) <- (c x - s y, s x + c y); right: the same on columns (p_l, q_l)
-          const double r00 = ck * a00 - sk * a10, r01 = ck * a01 - sk * a11;
-          const double r10 = sk * a00 + ck * a10, r11 = sk * a01 + ck * a11;
-          const double n00 = cl * r00 - sl * r01, n01 = sl * r00 + cl * r01;
-          const double n10 = cl * r10 - sl * r11, n11 = sl * r10 + cl * r11;
-          if (k == l) {
-            const double o = 0.5 * (n01 + n10);
-            An[pk * lda + pk] = n00; An[qk * lda + qk] = n11; An[pk * lda + qk] = o; An[qk * lda + pk] = o;
-          } else {
-            An[pk * lda + pl] = n00; An[pk * lda + ql] = n01; An[qk * lda + pl] = n10; An[qk * lda + ql] = n11;
-            An[pl * lda + pk] = n00; An[ql * lda + pk] = n01; An[pl * lda + qk] = n10; An[ql * lda + qk] = n11;
-          }
-        }
+        jacobi_a_items<D>(jc, Ao, An, sr, cs, wid, NW);
       }
       __syncthreads();
     }
   }
   // the seats now hold the order of round rr mod (d - 1): put the rows of V^T back
-  if (vt_thread) {
+  if (ROLE == JR_VT) {
     const int rf = rr % nrounds;
 #pragma unroll
-    for (int j = 0; j < N2; j++) VT[seat_index(rf, vh * N2 + j) * ldvt + vcol] = x[j];
+    for (int j = 0; j < N2; j++) jc.VT[seat_index(rf, vh * N2 + j) * jc.ldvt + vcol] = x[j];
   }
   __syncthreads();
   *final_buf = rr & 1;
   return sweeps;
 }
 
-// Tables of jacobi_eig_lookahead: where every index sits in every round, and the block list.
-__device__ void jacobi_tables(const ushort2* sched, uchar2* pos, uchar2* tri, int d) {
+template <int D>
+__device__ __forceinline__ int jacobi_eig_lookahead(const JacobiCtx& jc, int* final_buf) {
+  const int tid = threadIdx.x;
+  if (tid < 32) return jacobi_role<D, JR_AHEAD>(jc, final_buf);
+  if (tid < 32 + 2 * D) return jacobi_role<D, JR_VT>(jc, final_buf);
+  return jacobi_role<D, JR_A>(jc, final_buf);
+}
+
+// Tables of jacobi_eig_lookahead (pos is scratch: where every index sits in every round).
+__device__ void jacobi_tables(const ushort2* sched, uchar2* pos, uint2* la, uchar2* tri, int d) {
   const int half = d >> 1;
   for (int e = threadIdx.x; e < (d - 1) * half; e += FIT_THREADS) {
     const int r = e / half, k = e % half;
@@ -345,7 +374,20 @@ __device__ void jacobi_tables(const ushort2* sched, uchar2* pos, uchar2* tri, in
   }
   for (int e = threadIdx.x; e < half * half; e += FIT_THREADS) {
     const int k = e / half, l = e % half;
-    if (k <= l) tri[k * half - k * (k - 1) / 2 + (l - k)] = make_uchar2((unsigned char)k, (unsigned char)l);
+    if (k > l) continue;
+    // block row k <= half/2 is followed by block row half - k: together they fill `half` slots
+    const int slot = k <= half / 2 ? half * k + (l - k) : half * (half - k) + k + (l - k);
+    tri[slot] = make_uchar2((unsigned char)k, (unsigned char)l);
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < (d - 1) * half; e += FIT_THREADS) {
+    const int r = e / half, j = e % half;
+    const int rn = (r + 1 == d - 1) ? 0 : r + 1;
+    const ushort2 nx = sched[rn * half + j];
+    const uchar2 px = pos[r * d + nx.x], py = pos[r * d + nx.y];
+    const ushort2 cx = sched[r * half + px.x], cy = sched[r * half + py.x];
+    la[e] = make_uint2((unsigned)cx.x | ((unsigned)cx.y << 8) | ((unsigned)cy.x << 16) | ((unsigned)cy.y << 24),
+                       (unsigned)px.x | ((unsigned)py.x << 8) | ((unsigned)px.y << 16) | ((unsigned)py.y << 17));
   }
   __syncthreads();
 }
@@ -382,21 +424,23 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
   double* red = vec + 4 * d;     // [FIT_THREADS]
   int* perm = reinterpret_cast<int*>(red + FIT_THREADS);          // [d]
   ushort2* sched = reinterpret_cast<ushort2*>(perm + d);          // [(d-1) * d/2]
-  uchar2* pos = reinterpret_cast<uchar2*>(sched + (d - 1) * (d / 2));   // [(d-1) * d]      (look-ahead solver only)
+  uint2* la = reinterpret_cast<uint2*>(sched + (d - 1) * (d / 2) + ((d - 1) * (d / 2) & 1));   // 8-byte aligned; look-ahead solver only
+  uchar2* pos = reinterpret_cast<uchar2*>(la + (d - 1) * (d / 2));      // [(d-1) * d]
   uchar2* tri = pos + (d - 1) * d;                                      // [d/2 (d/2 + 1) / 2]
   int log2d = 0;
   while ((1 << log2d) < d) log2d++;
   if (a.variant == FSHARP_SDERF || a.variant == FSHARP_ADERF) {
     jacobi_schedule(sched, d);
-    if (V_IN_SMEM) jacobi_tables(sched, pos, tri, d);
+    if (V_IN_SMEM) jacobi_tables(sched, pos, la, tri, d);
   }
   // eigen-decomposition of the matrix in As: eigenvalues on its diagonal, eigenvectors in the rows of Vs
   auto eig = [&]() -> int {
     if (!V_IN_SMEM) return jacobi_eig(As, lda, Vs, ldv, d, log2d, sched, cs, red);
     int buf = 0, n = 0;
-    if (d == 64) n = jacobi_eig_lookahead<64>(As, A1, lda, Vs, ldv, sched, pos, tri, cs, red, &buf);
-    else if (d == 32) n = jacobi_eig_lookahead<32>(As, A1, lda, Vs, ldv, sched, pos, tri, cs, red, &buf);
-    else n = jacobi_eig_lookahead<16>(As, A1, lda, Vs, ldv, sched, pos, tri, cs, red, &buf);
+    JacobiCtx jc{As, A1, Vs, cs, red, sched, la, tri, lda, ldv};
+    if (d == 64) n = jacobi_eig_lookahead<64>(jc, &buf);
+    else if (d == 32) n = jacobi_eig_lookahead<32>(jc, &buf);
+    else n = jacobi_eig_lookahead<16>(jc, &buf);
     if (buf) {
       for (int e = tid; e < d * lda; e += FIT_THREADS) As[e] = A1[e];
       __syncthreads();
@@ -609,7 +653,8 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
 
 size_t fit_smem_bytes(int d, int v_in_smem) {
   size_t dbl = (size_t)d * (d + 1) * (v_in_smem ? 3 : 1) + 4 * (size_t)d + FIT_THREADS;
-  size_t tables = v_in_smem ? ((size_t)(d - 1) * d + (size_t)(d / 2) * (d / 2 + 1) / 2) * sizeof(uchar2) : 0;
+  size_t tables = v_in_smem ? ((size_t)(d - 1) * d + (size_t)(d / 2) * (d / 2 + 1) / 2) * sizeof(uchar2) +
+                                  ((size_t)(d - 1) * (d / 2) + 1) * sizeof(uint2) : 0;
   return dbl * sizeof(double) + (size_t)d * sizeof(int) + (size_t)(d - 1) * (d / 2) * sizeof(ushort2) + tables;
 }
 
