@@ -6,11 +6,21 @@
 namespace {
 
 constexpr int PREP_THREADS = 256;
+constexpr int PREP_MB = 64;                   // features per block
+constexpr int PREP_LDO = PREP_MB + 4;         // row stride of the transposed Omega chunk (keeps 16-byte alignment)
 
+// One block = one (group, side, chunk of 64 features).  Omega's chunk (transposed) and the d x d
+// matrix (B, then A) sit in shared memory in fp32; every thread owns a 4 x d/16 tile of the
+// 64 x d product and walks the inner index with vector loads.
+template <int D>
 __global__ void __launch_bounds__(PREP_THREADS)
 prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const double* __restrict__ params,
-            int64_t params_stride, int H, int pool, int d, int M, float* __restrict__ prep) {
+            int64_t params_stride, int H, int pool, int M, float* __restrict__ prep) {
+  constexpr int d = D, NC = D / 16;
   __shared__ int redi[PREP_THREADS];
+  extern __shared__ __align__(16) float stage[];
+  float* Ot = stage;                          // [d][PREP_LDO]: Ot[i][m] = Omega[m0 + m][i]
+  float* Ms = stage + d * PREP_LDO;           // [d][d]
   const int g = blockIdx.x, side = blockIdx.y + 1, tid = threadIdx.x;
   const int h = pool == FSHARP_POOL_PER_BH ? g % H : g;
   const float* Om = Omega + (int64_t)h * omega_head_stride;
@@ -27,58 +37,58 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
   float* scal = out + pr.scal();
   float* Cf = out + pr.Cmat();
 
-  // W = Omega B and a = diag(Omega A Omega^T) in fp32 (both end up in fp32 / bf16 operands);
-  // B and A are staged through shared memory 32 rows at a time.
-  extern __shared__ float stage[];            // [32][d] slice of B or A, then Omega rows per warp
-  float* slice = stage;                       // 32 * d
-  const int lane = tid & 31, warp = tid >> 5;
-  for (int pass = 0; pass < 2; pass++) {      // pass 0: W (matrix B), pass 1: a (matrix A)
+  const int m0 = blockIdx.z * PREP_MB;
+  const int ty = tid >> 4, tx = tid & 15;     // rows m0 + 4 ty + u, columns NC tx + v
+  for (int e = tid; e < PREP_MB * d; e += PREP_THREADS) {
+    const int m = e % PREP_MB, i = e / PREP_MB;
+    Ot[i * PREP_LDO + m] = (m0 + m < M) ? Om[(size_t)(m0 + m) * d + i] : 0.f;
+  }
+  for (int pass = 0; pass < 2; pass++) {      // pass 0: W = Omega B, pass 1: a = diag(Omega A Omega^T)
     const double* Mat = pass == 0 ? Bm : A;
-    {
-      const int m0 = blockIdx.z * 64;          // one block per chunk of 64 features
-      // each thread owns outputs (m, j): m = m0 + warp + 8 * u, j = lane + 32 * v
-      float acc[8][4];
+    __syncthreads();
+    for (int e = tid; e < d * d; e += PREP_THREADS) Ms[e] = (float)Mat[e];
+    __syncthreads();
+    float acc[4][NC];
 #pragma unroll
-      for (int u = 0; u < 8; u++)
+    for (int u = 0; u < 4; u++)
 #pragma unroll
-        for (int v = 0; v < 4; v++) acc[u][v] = 0.f;
-      for (int i0 = 0; i0 < d; i0 += 32) {
-        __syncthreads();
-        for (int e = tid; e < 32 * d; e += PREP_THREADS)
-          slice[e] = (i0 + e / d < d) ? (float)Mat[(size_t)(i0 + e / d) * d + (e % d)] : 0.f;
-        __syncthreads();
+      for (int v = 0; v < NC; v++) acc[u][v] = 0.f;
+#pragma unroll 4
+    for (int i = 0; i < d; i++) {
+      const float4 a4 = *reinterpret_cast<const float4*>(Ot + i * PREP_LDO + 4 * ty);
+      const float a[4] = {a4.x, a4.y, a4.z, a4.w};
+      float b[NC];
+      if (NC >= 4) {
 #pragma unroll
-        for (int u = 0; u < 8; u++) {
-          const int m = m0 + warp + 8 * u;
-          const float om = (m < M && i0 + lane < d) ? Om[(size_t)m * d + i0 + lane] : 0.f;   // Omega[m][i0 + lane]
-#pragma unroll 8
-          for (int ii = 0; ii < 32; ii++) {
-            const float o = __shfl_sync(0xffffffffu, om, ii);
-#pragma unroll
-            for (int v = 0; v < 4; v++)
-              if (lane + 32 * v < d) acc[u][v] = fmaf(o, slice[ii * d + lane + 32 * v], acc[u][v]);
-          }
+        for (int v4 = 0; v4 < NC / 4; v4++) {
+          const float4 b4 = *reinterpret_cast<const float4*>(Ms + i * d + NC * tx + 4 * v4);
+          b[4 * v4] = b4.x; b[4 * v4 + 1] = b4.y; b[4 * v4 + 2] = b4.z; b[4 * v4 + 3] = b4.w;
         }
+      } else {
+#pragma unroll
+        for (int v = 0; v < NC; v++) b[v] = Ms[i * d + NC * tx + v];
       }
 #pragma unroll
-      for (int u = 0; u < 8; u++) {
-        const int m = m0 + warp + 8 * u;
+      for (int u = 0; u < 4; u++)
+#pragma unroll
+        for (int v = 0; v < NC; v++) acc[u][v] = fmaf(a[u], b[v], acc[u][v]);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; u++) {
+      const int m = m0 + 4 * ty + u;
+      if (pass == 0) {
         if (m < M) {
-          if (pass == 0) {
 #pragma unroll
-            for (int v = 0; v < 4; v++)
-              if (lane + 32 * v < d) W[(size_t)m * d + lane + 32 * v] = acc[u][v];
-          } else {
-            // a_m = sum_j (Omega A)_mj Omega_mj
-            float sacc = 0.f;
-#pragma unroll
-            for (int v = 0; v < 4; v++)
-              if (lane + 32 * v < d) sacc = fmaf(acc[u][v], Om[(size_t)m * d + lane + 32 * v], sacc);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, o);
-            if (lane == 0) av[m] = sacc;
-          }
+          for (int v = 0; v < NC; v++) W[(size_t)m * d + NC * tx + v] = acc[u][v];
         }
+      } else {
+        // a_m = sum_j (Omega A)_mj Omega_mj, summed over the 16 threads that share row m
+        float sacc = 0.f;
+#pragma unroll
+        for (int v = 0; v < NC; v++) sacc = fmaf(acc[u][v], Ot[(NC * tx + v) * PREP_LDO + 4 * ty + u], sacc);
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, o);
+        if (tx == 0 && m < M) av[m] = sacc;
       }
     }
   }
@@ -110,9 +120,23 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
 int fs_run_prep(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_stride, const double* params,
                 int64_t params_stride, int G, int H, int pool, int d, int M, float* prep) {
   if (G == 0) return FSHARP_OK;
-  FS_TIME_BEGIN(ctx, FS_K_PREP);
-  prep_kernel<<<dim3(G, 2, (M + 63) / 64), PREP_THREADS, 32 * (size_t)d * sizeof(float), ctx->stream>>>(Omega, omega_head_stride, params, params_stride, H, pool, d, M,
-                                                                 prep);
+  const dim3 grid(G, 2, (M + PREP_MB - 1) / PREP_MB);
+  const size_t smem = ((size_t)d * PREP_LDO + (size_t)d * d) * sizeof(float);
+#define FS_PREP(DD)                                                                                                  \
+  do {                                                                                                               \
+    FS_CUDA_OK(cudaFuncSetAttribute(prep_kernel<DD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));        \
+    FS_TIME_BEGIN(ctx, FS_K_PREP);                                                                                    \
+    prep_kernel<DD><<<grid, PREP_THREADS, smem, ctx->stream>>>(Omega, omega_head_stride, params, params_stride, H,   \
+                                                               pool, M, prep);                                       \
+  } while (0)
+  switch (d) {
+    case 16: FS_PREP(16); break;
+    case 32: FS_PREP(32); break;
+    case 64: FS_PREP(64); break;
+    case 128: FS_PREP(128); break;
+    default: return FSHARP_E_SHAPE;
+  }
+#undef FS_PREP
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;

@@ -11,11 +11,12 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
 
 namespace {
 
-// Builds the per-(group, side) operand images from the fp32 prep block.
+// Builds the per-(group, side) operand images from the fp32 prep block; block z converts a
+// quarter of every array.  The flag words must be zero on entry (blocks OR their bits in).
+constexpr int TCP_SPLIT = 4;
 __global__ void __launch_bounds__(256)
 tc_prep_kernel(const float* __restrict__ prep, float qk_scale, uint8_t* __restrict__ images, int* __restrict__ flags) {
-  __shared__ int any_lo;
-  const int g = blockIdx.x, side = blockIdx.y, tid = threadIdx.x;
+  const int g = blockIdx.x, side = blockIdx.y, z = blockIdx.z, tid = threadIdx.x;
   PrepLayout pr{TC_D, TC_M};
   const float* pp = prep + ((size_t)g * 2 + side) * pr.total();
   const float* W = pp + pr.W();
@@ -23,18 +24,21 @@ tc_prep_kernel(const float* __restrict__ prep, float qk_scale, uint8_t* __restri
   const float* Cm = pp + pr.Cmat();
   const float* scal = pp + pr.scal();
   uint8_t* img = images + ((size_t)g * 2 + side) * IMG_BYTES;
-  if (tid == 0) any_lo = 0;
-  __syncthreads();
+  int* fl = flags + ((size_t)g * 2 + side) * FLAG_WORDS;
   const float sw = FS_LOG2E * qk_scale, sc = FS_LOG2E * qk_scale * qk_scale;
-  for (int e = tid; e < TC_M * TC_D; e += 256) {
-    int m = e / TC_D, k = e % TC_D;
-    const float v = W[e] * sw;
-    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-    *reinterpret_cast<__nv_bfloat16*>(img + IMG_W + tc::sw128_offset(m, k)) = hi;
-    *reinterpret_cast<__nv_bfloat16*>(img + IMG_WLO + tc::sw128_offset(m, k)) = __float2bfloat16_rn(v - __bfloat162float(hi));
+  constexpr int WQ = TC_M * TC_D / TCP_SPLIT, CQ = TC_D * TC_D / TCP_SPLIT, AQ = TC_M / TCP_SPLIT;
+  // two neighbouring elements per thread: one 4-byte store into each image
+  for (int e2 = tid; e2 < WQ / 2; e2 += 256) {
+    const int e = z * WQ + 2 * e2, m = e / TC_D, k = e % TC_D;
+    const float2 w2 = *reinterpret_cast<const float2*>(W + e);
+    const float v0 = w2.x * sw, v1 = w2.y * sw;
+    const __nv_bfloat16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
+    *reinterpret_cast<__nv_bfloat162*>(img + IMG_W + tc::sw128_offset(m, k)) = __nv_bfloat162(h0, h1);
+    *reinterpret_cast<__nv_bfloat162*>(img + IMG_WLO + tc::sw128_offset(m, k)) =
+        __nv_bfloat162(__float2bfloat16_rn(v0 - __bfloat162float(h0)), __float2bfloat16_rn(v1 - __bfloat162float(h1)));
   }
   int lo_nonzero = 0;
-  for (int e = tid; e < TC_D * TC_D; e += 256) {
+  for (int e = z * CQ + tid; e < (z + 1) * CQ; e += 256) {
     int k = e / TC_D, n = e % TC_D;          // C[k][n] goes to row n, column k of the B operand
     float v = Cm[e] * sc;
     __nv_bfloat16 hi = __float2bfloat16_rn(v);
@@ -43,13 +47,10 @@ tc_prep_kernel(const float* __restrict__ prep, float qk_scale, uint8_t* __restri
     *reinterpret_cast<__nv_bfloat16*>(img + IMG_CHI + tc::sw128_offset(n, k)) = hi;
     *reinterpret_cast<__nv_bfloat16*>(img + IMG_CLO + tc::sw128_offset(n, k)) = lo;
   }
-  for (int m = tid; m < TC_M; m += 256) reinterpret_cast<float*>(img + IMG_A2)[m] = 2.f * FS_LOG2E * av[m];
-  if (lo_nonzero) atomicOr(&any_lo, 1);
-  __syncthreads();
-  if (tid == 0) {
-    int* fl = flags + ((size_t)g * 2 + side) * FLAG_WORDS;
-    const bool cscalar = scal[PS_CSCALAR] != 0.f;
-    fl[0] = (cscalar ? 0 : FLAG_C_DENSE) | (any_lo ? FLAG_C_LO : 0);
+  if (tid < AQ) reinterpret_cast<float*>(img + IMG_A2)[z * AQ + tid] = 2.f * FS_LOG2E * av[z * AQ + tid];
+  if (__syncthreads_or(lo_nonzero) && tid == 0) atomicOr(&fl[0], FLAG_C_LO);
+  if (z == 0 && tid == 0) {
+    if (scal[PS_CSCALAR] == 0.f) atomicOr(&fl[0], FLAG_C_DENSE);
     fl[1] = __float_as_int(scal[PS_CGAMMA] * sc);
   }
 }
@@ -112,8 +113,9 @@ int make_map_kvt(CUtensorMap* map, const void* base, int BH) {
 }  // namespace tchost
 
 int fs_tc_prep(fsharp_ctx* ctx, const float* prep, int G, float qk_scale, uint8_t* images, int* flags) {
+  FS_CUDA_OK(cudaMemsetAsync(flags, 0, (size_t)G * 2 * FLAG_WORDS * sizeof(int), ctx->stream));
   FS_TIME_BEGIN(ctx, FS_K_TC_PREP);
-  tc_prep_kernel<<<dim3(G, 2), 256, 0, ctx->stream>>>(prep, qk_scale, images, flags);
+  tc_prep_kernel<<<dim3(G, 2, TCP_SPLIT), 256, 0, ctx->stream>>>(prep, qk_scale, images, flags);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;
