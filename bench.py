@@ -267,14 +267,17 @@ def main():
     pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(pk):
         j = json.load(open(pk))
-        peaks = {"hbm_gbs": j["hbm_gbs"], "bf16_tflops": j["bf16_tflops_sustained"], "source": "measured (sustained)"}
+        peaks = {"hbm_gbs": j["hbm_gbs"], "bf16_tflops": j["bf16_tflops_sustained"], "source": "measured (sustained)",
+                 "sm_max_mhz": j.get("sm_max_mhz", 1965.0)}
     # dominant kernel of the step and its roofline
     tot = sum(v[0] for v in per_kernel.values()) or 1.0
     kernels = {k: {"ms_per_launch": v[0] / v[1], "launches_per_step": v[1] / ksteps, "share": v[0] / tot}
                for k, v in sorted(per_kernel.items(), key=lambda kv: -kv[1][0])}
     dom = next(iter(kernels))
+    work["fit_sweeps"] = float(pr[:, 5 * w.d * w.d + 3].mean().item())
+    peaks["sm_count"] = torch.cuda.get_device_properties(dev).multi_processor_count
     roof = roofline_for(dom, kernels[dom], w, work, peaks)
-    attend_ms = sum(v[0] for k, v in per_kernel.items() if k not in ("stats_kernel", "fit_kernel")) / ksteps
+    attend_ms = sum(v[0] for k, v in per_kernel.items() if k not in ("stats_kernel", "tc_stats_kernel", "fit_kernel")) / ksteps
     t_roof = max(work["flops"] / (peaks["bf16_tflops"] * 1e12), work["bytes"] / (peaks["hbm_gbs"] * 1e9))
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -324,7 +327,7 @@ def roofline_for(name, k, w, work, peaks):
         "tc_out_kernel": (2 * L * d * M + 2 * L * M * (dv + 1)) * units,
         "tc_causal_out_kernel": work["flops"], "tc_causal_state_kernel": (2 * L * d * M + 2 * L * M * (dv + 1)) * units,
     }
-    bytes_of = {"stats_kernel": 2 * L * d * es * units, "expshift_kernel": 2 * L * M * 4 * units,
+    bytes_of = {"stats_kernel": 2 * L * d * es * units, "tc_stats_kernel": 2 * L * d * es * units, "expshift_kernel": 2 * L * M * 4 * units,
                 "rowterm_kernel": L * d * es * units, "groupmax_kernel": L * M * 4 * units}
     if name in flops_of and flops_of[name]:
         fl = flops_of[name] * (per_launch if name in ("logits_kernel", "kv_kernel", "out_kernel", "scores_kernel") and
@@ -333,8 +336,18 @@ def roofline_for(name, k, w, work, peaks):
         return {"kernel": name, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": ach / peaks["bf16_tflops"], "traffic": None, "peak_source": peaks["source"]}
     if name == "fit_kernel":
-        return {"kernel": name, "bound": "alu", "achieved": None, "peak": None, "unit": "TFLOP/s", "frac": None,
-                "traffic": None, "note": "latency-bound fp64 Jacobi sweeps, one block per group"}
+        # fp64 arithmetic of the Jacobi sweeps (the rest of the fit is negligible): per round and group the
+        # 2 x 2 blocks of A (8 multiplies + 8 multiply-adds each) and d/2 * d row-pair entries of V^T
+        # (2 multiplies + 2 multiply-adds each); peak = 64 fp64 FMA per clock and SM.
+        h = d // 2
+        blocks = h * (h + 1) // 2 if d <= 64 else h * h
+        flops = work.get("fit_sweeps", 0.0) * (d - 1) * (blocks * 24 + h * d * 6) * units
+        peak = 64 * 2 * peaks.get("sm_count", 148) * peaks.get("sm_max_mhz", 1965.0) * 1e6 / 1e12
+        ach = flops / t / 1e12
+        return {"kernel": name, "bound": "alu", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
+                "traffic": None, "peak_source": "64 fp64 FMA/clk/SM x SMs x max SM clock",
+                "note": f"one block per group ({units} of {peaks.get('sm_count', 148)} SMs busy), "
+                        f"{work.get('fit_sweeps', 0.0):.1f} Jacobi sweeps per group; bound by shared-memory wavefronts and barrier latency"}
     by = bytes_of.get(name, work["bytes"]) * (per_launch if k["launches_per_step"] > 1 else 1.0)
     ach = by / t / 1e9
     return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",

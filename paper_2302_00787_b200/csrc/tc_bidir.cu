@@ -2,10 +2,10 @@
 //
 //   key side   (tc_kv_kernel):  per 128-key tile   logits = Y W2^T           (tcgen05, TMEM)
 //                               phi = 2^(logits + c_j - s)  -> bf16 tile in shared memory
-//                               KV += phi^T [V | 1]                          (tcgen05, TMEM)
-//   merge      (tc_merge_kernel): partial KV of the splits of one (batch, head), brought to a
-//                               common shift, summed, scaled by 2^a2 per feature, written
-//                               transposed in fp16
+//                               KV^T += [V | 1]^T phi                        (tcgen05, TMEM)
+//                               (c_j, the key's quadratic term, comes from tc_rowterm_kernel)
+//   merge      (tc_merge_kernel): partial KV^T of the splits of one (batch, head), brought to a
+//                               common shift, summed, scaled by 2^a2 per feature, written in fp16
 //   query side (tc_out_kernel): logits, phi = 2^(logits - max of the half row) in fp16,
 //                               [num | den] = phi KV per feature half, halves combined, Y = num / den
 //
@@ -13,7 +13,7 @@
 // TMA producer warp and one MMA issuing warp; all exponents are kept in log2 units
 // (W and C are pre-multiplied by log2 e), so a feature is one ex2 per element.  The per-feature
 // term w^T A w is the same on the query and the key side, so it is not added to the logits at
-// all: the merge multiplies row m of S^T [V | 1] by 2^(2 log2e w_m^T A w_m).
+// all: the merge multiplies feature m of S^T [V | 1] by 2^(2 log2e w_m^T A w_m).
 #include <cuda_fp16.h>
 
 #include "common.cuh"
@@ -30,26 +30,34 @@ constexpr int PREFETCH_TILES = 4;   // tiles pulled into L2 ahead of the shared-
 // ------------------------------------------------------------------------------------------
 // key side
 // ------------------------------------------------------------------------------------------
+// The two halves of the feature range (128 features each) run as two pipelines of their own:
+// four epilogue warps, a phi half tile, a pair of barriers, a running shift and a TMEM
+// accumulator per half.  They only share the key / value tiles, the logits MMA and the MMA
+// pipe itself, so while the tensor cores contract one half the other half's exponentials run.
+// The accumulator is kept transposed, acc_h = [V | 1]^T phi_h ([80 used of 128 lanes] x 128
+// columns): one MMA covers N = 128 features instead of 80 value columns.
 struct KvSmem {
   static constexpr uint32_t X0 = 0, V0 = 2 * TILE_BYTES, ONES = 4 * TILE_BYTES, W = ONES + TILE_BYTES,
-                            WLO = W + IMG_W_BYTES, CHI = WLO + IMG_W_BYTES, CLO = CHI + IMG_C_BYTES,
-                            PHI = CLO + IMG_C_BYTES, MISC = PHI + 4 * TILE_BYTES, TOTAL = MISC + 256;
+                            WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES, MISC = PHI + 4 * TILE_BYTES,
+                            TOTAL = MISC + 256;
 };
 static_assert(KvSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 static_assert(KvSmem::PHI % 1024 == 0 && KvSmem::W % 1024 == 0 && KvSmem::ONES % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 
 struct KvMisc {
-  uint64_t full[2], empty[2], logits_full, logits_free, phi_full, phi_free, const_bar;
+  uint64_t full[2], empty[2], logits_full, logits_free, phi_full[2], phi_free[2], const_bar;
   uint32_t tmem_base;
   int abort_flag;
-  int tile_max[4];     // [0..2] rotating slots of the per-tile maximum, [3] the first tile's
+  int tile_max[2][4];     // per half: [0..2] rotating slots of the per-tile maximum, [3] the first tile's
 };
+static_assert(sizeof(KvMisc) <= 256, "misc block");
 
-constexpr uint32_t KV_COL_LOGITS = 0, KV_COL_T = 256, KV_COL_ACC = 320;   // TMEM columns
+constexpr uint32_t KV_COL_LOGITS = 0, KV_COL_ACC = 256;   // TMEM columns; half h accumulates at KV_COL_ACC + 128 h
+constexpr int HALF_THREADS = EPI_THREADS / 2;
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-             const uint8_t* __restrict__ images, const int* __restrict__ img_flags, int H, int pool, int L,
+             const uint8_t* __restrict__ images, const float* __restrict__ crow, int H, int pool, int L, int Lpad,
              int tiles_per_split, int nsplit, float* __restrict__ partial, float* __restrict__ shifts,
              int* __restrict__ pmax, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
@@ -62,24 +70,24 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   const int tile0 = split * tiles_per_split;
   const int ntiles = min(tiles_per_split, total_tiles - tile0);
   const uint8_t* img = images + ((size_t)g * 2 + 1) * IMG_BYTES;        // side 2 (keys)
-  const int* fl = img_flags + ((size_t)g * 2 + 1) * FLAG_WORDS;
-  const bool cdense = (fl[0] & FLAG_C_DENSE) != 0, clo = (fl[0] & FLAG_C_LO) != 0;
-  const float gamma2 = __int_as_float(fl[1]);          // C = gamma I: c_j = gamma2 |x_j|^2 (log2 units)
   volatile int* abortp = &misc->abort_flag;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 2; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], 1); }
+    for (int i = 0; i < 2; i++) {
+      mbar_init(&misc->full[i], 1);
+      mbar_init(&misc->empty[i], 1);
+      mbar_init(&misc->phi_full[i], HALF_THREADS);
+      mbar_init(&misc->phi_free[i], 1);
+      for (int j = 0; j < 4; j++) misc->tile_max[i][j] = f2ord(-INFINITY);
+    }
     mbar_init(&misc->logits_full, 1);
     mbar_init(&misc->logits_free, EPI_THREADS);
-    mbar_init(&misc->phi_full, EPI_THREADS);
-    mbar_init(&misc->phi_free, 1);
     mbar_init(&misc->const_bar, 1);
     misc->abort_flag = 0;
-    for (int i = 0; i < 4; i++) misc->tile_max[i] = f2ord(-INFINITY);
     fence_barrier_init();
   }
-  // constant tile written by the block itself: the second 64-column block of [V | 1], whose
-  // first column is the 1 and whose other columns are zero (only 16 of them are read)
+  // constant tile written by the block itself: the second 64-row block of [V | 1]^T, whose
+  // first row is the 1 and whose other rows are zero
   for (int i = threadIdx.x; i < TILE_BYTES / 16; i += TC_THREADS) reinterpret_cast<uint4*>(sm + KvSmem::ONES)[i] = make_uint4(0, 0, 0, 0);
   __syncthreads();
   if (threadIdx.x < TILE)
@@ -100,11 +108,9 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     if (lane == 0) {
       prefetch_tmap(&tmK);
       prefetch_tmap(&tmV);
-      mbar_expect_tx(&misc->const_bar, 2 * IMG_W_BYTES + 2 * IMG_C_BYTES);
+      mbar_expect_tx(&misc->const_bar, 2 * IMG_W_BYTES);
       bulk_load(sm + KvSmem::W, img + IMG_W, IMG_W_BYTES, &misc->const_bar);
       bulk_load(sm + KvSmem::WLO, img + IMG_WLO, IMG_W_BYTES, &misc->const_bar);
-      bulk_load(sm + KvSmem::CHI, img + IMG_CHI, IMG_C_BYTES, &misc->const_bar);
-      bulk_load(sm + KvSmem::CLO, img + IMG_CLO, IMG_C_BYTES, &misc->const_bar);
       // the shared-memory ring is only two tiles deep; tiles further ahead are pulled into L2
       for (int it = 0; it < min(ntiles, PREFETCH_TILES); it++) {
         tma_prefetch_4d(&tmK, 0, (tile0 + it) * TILE, h, b);
@@ -130,37 +136,25 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   } else if (warp == WARP_MMA) {
     if (lane == 0) {
       constexpr uint32_t ID_LOGITS = idesc_bf16(128, TC_M, 0, 0);
-      constexpr uint32_t ID_T = idesc_bf16(128, TC_D, 0, 0);
-      constexpr uint32_t ID_KV = idesc_bf16(128, TC_NV, 1, 1);     // phi^T [V | 1]
+      constexpr uint32_t ID_KV = idesc_bf16(128, 128, 1, 1);       // [V | 1]^T phi_h
       const uint32_t sV0 = smem_u32(sm + KvSmem::V0), sOnes = smem_u32(sm + KvSmem::ONES);
       // descriptors are built once; inside the loops each MMA costs one add per operand
       const uint64_t dX0 = smem_desc(smem_u32(sm + KvSmem::X0), 16, 1024, SWZ_128B);
       const uint64_t dW = smem_desc(smem_u32(sm + KvSmem::W), 16, 1024, SWZ_128B);
       const uint64_t dWlo = smem_desc(smem_u32(sm + KvSmem::WLO), 16, 1024, SWZ_128B);
-      const uint64_t dChi = smem_desc(smem_u32(sm + KvSmem::CHI), 16, 1024, SWZ_128B);
-      const uint64_t dClo = smem_desc(smem_u32(sm + KvSmem::CLO), 16, 1024, SWZ_128B);
+      // phi half h as an operand whose 128 features are the contiguous index: two 64-feature blocks
       const uint64_t dPhi = smem_desc(smem_u32(sm + KvSmem::PHI), TILE_BYTES, 1024, SWZ_128B);
-      // [V | 1] as one MN-major operand: block 0 = the V tile of the stage, block 1 = the ones tile
+      // [V | 1] with the value index contiguous: block 0 = the V tile of the stage, block 1 = the ones tile
       const uint64_t dVst0 = smem_desc(sV0, sOnes - sV0, 1024, SWZ_128B);
       const uint64_t dVst1 = smem_desc(sV0 + TILE_BYTES, sOnes - sV0 - TILE_BYTES, 1024, SWZ_128B);
       auto issue_logits = [&](int st) {
         const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
-#pragma unroll 1
+#pragma unroll
         for (int k = 0; k < TC_D / 16; k++)
           mma_bf16(tmem + KV_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dW, 32 * k), ID_LOGITS, k > 0);
-#pragma unroll 1
+#pragma unroll
         for (int k = 0; k < TC_D / 16; k++)
           mma_bf16(tmem + KV_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dWlo, 32 * k), ID_LOGITS, 1);
-        if (cdense) {
-#pragma unroll 1
-          for (int k = 0; k < TC_D / 16; k++)
-            mma_bf16(tmem + KV_COL_T, desc_advance(dX, 32 * k), desc_advance(dChi, 32 * k), ID_T, k > 0);
-          if (clo) {
-#pragma unroll 1
-            for (int k = 0; k < TC_D / 16; k++)
-              mma_bf16(tmem + KV_COL_T, desc_advance(dX, 32 * k), desc_advance(dClo, 32 * k), ID_T, 1);
-          }
-        }
         mma_commit(&misc->logits_full);
       };
       bool ok = mbar_wait(&misc->const_bar, 0, abortp, status);
@@ -177,71 +171,43 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           tcgen05_fence_after();
           issue_logits(st ^ 1);
         }
-        if (!mbar_wait(&misc->phi_full, it & 1, abortp, status)) break;
-        tcgen05_fence_after();
         const uint64_t dV = st ? dVst1 : dVst0;
         const uint32_t acc0 = it > 0 ? 1u : 0u;
 #pragma unroll 1
-        for (int hh = 0; hh < 2; hh++)
-#pragma unroll 1
+        for (int hh = 0; hh < 2 && ok; hh++) {
+          if (!mbar_wait(&misc->phi_full[hh], it & 1, abortp, status)) { ok = false; break; }
+          tcgen05_fence_after();
+#pragma unroll 2
           for (int k = 0; k < TILE / 16; k++)
-            mma_bf16(tmem + KV_COL_ACC + hh * TC_NV, desc_advance(dPhi, hh * 2 * TILE_BYTES + k * 2048),
-                     desc_advance(dV, k * 2048), ID_KV, k > 0 ? 1u : acc0);
-        mma_commit(&misc->phi_free);
+            mma_bf16(tmem + KV_COL_ACC + hh * 128, desc_advance(dV, k * 2048),
+                     desc_advance(dPhi, hh * 2 * TILE_BYTES + k * 2048), ID_KV, k > 0 ? 1u : acc0);
+          mma_commit(&misc->phi_free[hh]);
+        }
         mma_commit(&misc->empty[st]);
       }
     }
   }
   } else {
     regs_acquire<REGS_EPILOGUE>();
-    // ---------------- epilogue warps: one key row per thread, 128 of the 256 features.
-    // The running shift s is taken on trust while the exponentials are computed; the tile's
-    // largest exponent is tracked on the side and checked afterwards.  Only if it exceeds the
-    // headroom (rare: the running maximum grows a handful of times per sequence) is the
+    // ---------------- epilogue warps: one key row per thread, the 128 features of its half.
+    // The running shift s of the half is taken on trust while the exponentials are computed; the
+    // tile's largest exponent is tracked on the side and checked afterwards.  Only if it exceeds
+    // the headroom (rare: the running maximum grows a handful of times per sequence) is the
     // accumulated state rescaled and the tile redone from the logits still held in registers.
     const int q = warp & 3, hf = warp >> 2;
     const int row = q * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+    const uint32_t acc_addr = lane_addr + KV_COL_ACC + hf * 128;
+    int* tmax = misc->tile_max[hf];
+    const float* cptr = crow + (size_t)bh * Lpad + (size_t)tile0 * TILE + row;
     float s = 0.f;
+    float cj = ntiles > 0 ? cptr[0] : 0.f;
     bool alive = true;
     for (int it = 0; it < ntiles && alive; it++) {
-      const int st = it & 1;
-      if (!mbar_wait(&misc->full[st], (it >> 1) & 1, abortp, status, false)) { alive = false; break; }
+      const float cnext = it + 1 < ntiles ? cptr[(size_t)(it + 1) * TILE] : 0.f;     // in flight during this tile
       if (!mbar_wait(&misc->logits_full, it & 1, abortp, status, false)) { alive = false; break; }
       __syncwarp();
       tcgen05_fence_after();
-      // c_j = x_j^T C x_j in log2 units
-      float cj = 0.f;
-      {
-        const uint8_t* xrow = sm + KvSmem::X0 + st * TILE_BYTES + row * 128;
-        float xv[TC_D];
-#pragma unroll
-        for (int c = 0; c < 8; c++) {
-          uint4 u = *reinterpret_cast<const uint4*>(xrow + ((c ^ (row & 7)) << 4));
-          const uint32_t w4[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-          for (int j = 0; j < 4; j++) {
-            xv[c * 8 + 2 * j] = __uint_as_float(w4[j] << 16);
-            xv[c * 8 + 2 * j + 1] = __uint_as_float(w4[j] & 0xffff0000u);
-          }
-        }
-        float part[4] = {0.f, 0.f, 0.f, 0.f};
-        if (cdense) {
-#pragma unroll
-          for (int c = 0; c < TC_D / 16; c++) {
-            uint32_t t[16];
-            tmem_ld16(lane_addr + KV_COL_T + c * 16, t);
-            tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 16; j++) part[j & 3] = fmaf(__uint_as_float(t[j]), xv[c * 16 + j], part[j & 3]);
-          }
-          cj = (part[0] + part[1]) + (part[2] + part[3]);
-        } else {
-#pragma unroll
-          for (int j = 0; j < TC_D; j++) part[j & 3] = fmaf(xv[j], xv[j], part[j & 3]);
-          cj = ((part[0] + part[1]) + (part[2] + part[3])) * gamma2;
-        }
-      }
       uint32_t v[128];
 #pragma unroll
       for (int c = 0; c < 8; c++) {
@@ -255,18 +221,18 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       mbar_arrive(&misc->logits_free);
       const bool valid = (tile0 + it) * TILE + row < L;
       if (it == 0) {
-        // first tile: no shift yet, take the tile's exact maximum
+        // first tile: no shift yet, take the exact maximum of this half of the tile
         float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
         for (int i = 0; i < 128; i++) mxp[i & 3] = fmaxf(mxp[i & 3], __uint_as_float(v[i]));
         float mx = valid ? fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])) + cj : -INFINITY;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        if (lane == 0) atomicMax(&misc->tile_max[3], f2ord(mx));
-        named_bar_sync(1, EPI_THREADS);
-        s = ord2f(misc->tile_max[3]);
+        if (lane == 0) atomicMax(&tmax[3], f2ord(mx));
+        named_bar_sync(1 + hf, HALF_THREADS);
+        s = ord2f(tmax[3]);
       } else {
-        if (!mbar_wait(&misc->phi_free, (it - 1) & 1, abortp, status, false)) { alive = false; break; }
+        if (!mbar_wait(&misc->phi_free[hf], (it - 1) & 1, abortp, status, false)) { alive = false; break; }
       }
       uint8_t* prow = sm + KvSmem::PHI + hf * 2 * TILE_BYTES + row * 128;
       float rc = cj - s;
@@ -289,23 +255,23 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         rel = valid ? fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])) : -INFINITY;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) rel = fmaxf(rel, __shfl_xor_sync(0xffffffffu, rel, o));
-        if (lane == 0) atomicMax(&misc->tile_max[it % 3], f2ord(rel));
-        if (threadIdx.x == 0) misc->tile_max[(it + 1) % 3] = f2ord(-INFINITY);   // next tile's slot; idle since tile it-2
-        named_bar_sync(1, EPI_THREADS);
-        rel = ord2f(misc->tile_max[it % 3]);
+        if (lane == 0) atomicMax(&tmax[it % 3], f2ord(rel));
+        if (q == 0 && lane == 0) tmax[(it + 1) % 3] = f2ord(-INFINITY);   // next tile's slot; idle since tile it-2
+        named_bar_sync(1 + hf, HALF_THREADS);
+        rel = ord2f(tmax[it % 3]);
         if (!(rel > SHIFT_HEADROOM_LOG2)) break;       // the common case: nothing to redo
-        // the running shift moves up by rel: bring the accumulated S^T [V | 1] along, redo the tile
+        // the running shift moves up by rel: bring the accumulated [V | 1]^T phi_h along, redo the tile
         __syncwarp();
         tcgen05_fence_after();
         const float f = ex2(-rel);
 #pragma unroll
-        for (int c = 0; c < TC_NV / 16; c++) {
+        for (int c = 0; c < 8; c++) {
           uint32_t a[16];
-          tmem_ld16(lane_addr + KV_COL_ACC + hf * TC_NV + c * 16, a);
+          tmem_ld16(acc_addr + c * 16, a);
           tmem_wait_ld();
 #pragma unroll
           for (int j = 0; j < 16; j++) a[j] = __float_as_uint(__uint_as_float(a[j]) * f);
-          tmem_st16(lane_addr + KV_COL_ACC + hf * TC_NV + c * 16, a);
+          tmem_st16(acc_addr + c * 16, a);
         }
         tmem_wait_st();
         s += rel;
@@ -313,31 +279,36 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       }
       fence_proxy_async_smem();
       tcgen05_fence_before();
-      mbar_arrive(&misc->phi_full);
+      mbar_arrive(&misc->phi_full[hf]);
+      cj = cnext;
     }
-    // write this split's partial S^T [V | 1] (fp32), its shift and its largest magnitude
-    if (alive && ntiles > 0 && mbar_wait(&misc->phi_free, (ntiles - 1) & 1, abortp, status, false)) {
+    // write this split's partial [V | 1]^T phi_h (fp32, rows 0..79), its shift and its largest magnitude
+    if (alive && ntiles > 0 && mbar_wait(&misc->phi_free[hf], (ntiles - 1) & 1, abortp, status, false)) {
       __syncwarp();
       tcgen05_fence_after();
-      float* out = partial + (((size_t)bh * nsplit + split) * TC_M + hf * 128 + row) * TC_NV;
+      float* out = partial + (((size_t)bh * nsplit + split) * TC_NV + row) * TC_M + hf * 128;
       float amax = 0.f;
+      if (q * 32 < TC_NV) {                 // warp-uniform: lanes 0..79 carry data
 #pragma unroll
-      for (int c = 0; c < TC_NV / 16; c++) {
-        uint32_t a[16];
-        tmem_ld16(lane_addr + KV_COL_ACC + hf * TC_NV + c * 16, a);
-        tmem_wait_ld();
+        for (int c = 0; c < 8; c++) {
+          uint32_t a[16];
+          tmem_ld16(acc_addr + c * 16, a);
+          tmem_wait_ld();
+          if (row < TC_NV) {
 #pragma unroll
-        for (int j = 0; j < 16; j++)
-          if (c * 16 + j <= TC_DV) amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
+            for (int j = 0; j < 16; j++)
+              if (row <= TC_DV) amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
 #pragma unroll
-        for (int j = 0; j < 4; j++)
-          reinterpret_cast<uint4*>(out + c * 16)[j] = make_uint4(a[4 * j], a[4 * j + 1], a[4 * j + 2], a[4 * j + 3]);
+            for (int j = 0; j < 4; j++)
+              reinterpret_cast<uint4*>(out + c * 16)[j] = make_uint4(a[4 * j], a[4 * j + 1], a[4 * j + 2], a[4 * j + 3]);
+          }
+        }
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
       // non-negative floats order like their bit patterns
-      if (lane == 0) atomicMax(&pmax[(size_t)bh * nsplit + split], __float_as_int(amax));
-      if (threadIdx.x == 0) shifts[(size_t)bh * nsplit + split] = s;
+      if (lane == 0) atomicMax(&pmax[((size_t)bh * nsplit + split) * 2 + hf], __float_as_int(amax));
+      if (q == 0 && lane == 0) shifts[((size_t)bh * nsplit + split) * 2 + hf] = s;
     }
   }
   tcgen05_fence_before();
@@ -350,70 +321,69 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 
 // ------------------------------------------------------------------------------------------
 // merge of the key-side partials of one (batch, head): common shift, sum, per-feature factor
-// 2^a2, transpose, fp16
+// 2^a2, fp16.  Partials and result are both [80 rows][256 features].
 // ------------------------------------------------------------------------------------------
 constexpr int MERGE_SLICES = 8;
 __global__ void __launch_bounds__(256)
 tc_merge_kernel(const float* __restrict__ partial, const float* __restrict__ shifts, const int* __restrict__ pmax,
                 int nsplit, const uint8_t* __restrict__ images, int H, int pool, __half* __restrict__ kvt) {
-  __shared__ float fac[64];
-  __shared__ float a2s[TC_M];
+  __shared__ float fac[2 * 64];
+  __shared__ float rowfac[TC_M];
   __shared__ float red[256];
-  __shared__ float scale_s;
   const int bh = blockIdx.y;
   const int g = pool == FSHARP_POOL_PER_BH ? bh : bh % H;
   const float* a2 = reinterpret_cast<const float*>(images + (size_t)g * 2 * IMG_BYTES + IMG_A2);
-  float amax = -INFINITY;
-  for (int m = threadIdx.x; m < TC_M; m += 256) { a2s[m] = a2[m]; amax = fmaxf(amax, a2[m]); }
-  red[threadIdx.x] = amax;
+  const float a2m = a2[threadIdx.x];          // 256 threads, 256 features
+  red[threadIdx.x] = a2m;
+  if (threadIdx.x < 2 * nsplit) fac[threadIdx.x] = shifts[(size_t)bh * nsplit * 2 + threadIdx.x];
   __syncthreads();
   for (int s = 128; s > 0; s >>= 1) {
     if (threadIdx.x < s) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + s]);
     __syncthreads();
   }
-  if (threadIdx.x == 0) {
-    float smax = -INFINITY;
-    for (int p = 0; p < nsplit; p++) smax = fmaxf(smax, shifts[(size_t)bh * nsplit + p]);
-    // fp16 has a narrow range: scale the whole (batch, head) by a power of two (it cancels in
-    // num / den) so that the bound sum_p 2^(s_p - smax) max|partial_p| lands near 2^14; the
-    // per-feature factors are applied relative to their maximum, so none exceeds 1
-    float bound = 0.f;
-    for (int p = 0; p < nsplit; p++) {
-      fac[p] = exp2f(shifts[(size_t)bh * nsplit + p] - smax);
-      bound = fmaf(fac[p], __int_as_float(pmax[(size_t)bh * nsplit + p]), bound);
-    }
-    int ex = 0;
-    if (bound > 0.f && isfinite(bound)) frexpf(bound, &ex);
-    scale_s = exp2f((float)(14 - ex));
-  }
+  const float a2max = red[0];
+  float smax = -INFINITY;
+  for (int p = 0; p < 2 * nsplit; p++) smax = fmaxf(smax, fac[p]);
+  // fp16 has a narrow range: scale the whole (batch, head) by a power of two (it cancels in
+  // num / den) so that the bound sum_p 2^(s_p - smax) max|partial_p| lands near 2^14; the
+  // per-feature factors are applied relative to their maximum, so none exceeds 1
+  float bound = 0.f;
+  for (int p = 0; p < 2 * nsplit; p++) bound = fmaf(exp2f(fac[p] - smax), __int_as_float(pmax[(size_t)bh * nsplit * 2 + p]), bound);
+  int ex = 0;
+  if (bound > 0.f && isfinite(bound)) frexpf(bound, &ex);
+  const float scale = exp2f((float)(14 - ex));
   __syncthreads();
-  const float scale = scale_s, a2max = red[0];
-  const float* base = partial + (size_t)bh * nsplit * TC_M * TC_NV;
+  if (threadIdx.x < 2 * nsplit) fac[threadIdx.x] = exp2f(fac[threadIdx.x] - smax);
+  rowfac[threadIdx.x] = scale * exp2f(a2m - a2max);
+  __syncthreads();
+  const float* base = partial + (size_t)bh * nsplit * TC_NV * TC_M;
   __half* out = kvt + (size_t)bh * TC_NV * TC_M;
   constexpr int PER = TC_M * TC_NV / MERGE_SLICES;
   for (int e = blockIdx.x * PER + threadIdx.x; e < (blockIdx.x + 1) * PER; e += 256) {
-    const int m = e / TC_NV, n = e % TC_NV;
+    const int n = e / TC_M, m = e % TC_M, hh = m >> 7;
     float acc = 0.f;
     if (n <= TC_DV)
-      for (int p = 0; p < nsplit; p++) acc = fmaf(base[(size_t)p * TC_M * TC_NV + e], fac[p], acc);
-    out[(size_t)n * TC_M + m] = __float2half_rn(acc * scale * exp2f(a2s[m] - a2max));
+      for (int p = 0; p < nsplit; p++) acc = fmaf(base[(size_t)p * TC_NV * TC_M + e], fac[2 * p + hh], acc);
+    out[e] = __float2half_rn(acc * rowfac[m]);
   }
 }
 
 // ------------------------------------------------------------------------------------------
 // query side
 // ------------------------------------------------------------------------------------------
-constexpr int OUT_STAGES = 3;
+constexpr int OUT_STAGES = 2;
 struct OutSmem {
   static constexpr uint32_t X0 = 0, W = OUT_STAGES * TILE_BYTES, WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES,
                             KVT = PHI + 4 * TILE_BYTES, ROWMAX = KVT + KVT_BYTES,
-                            MISC = ROWMAX + 3 * 2 * TILE * 4, TOTAL = MISC + 256;
+                            STAGE = ROWMAX + 3 * 2 * TILE * 4,          // 2 KB per epilogue warp: output rows on their way out
+                            MISC = STAGE + (EPI_THREADS / 32) * 2048, TOTAL = MISC + 256;
 };
 static_assert(OutSmem::PHI % 1024 == 0 && OutSmem::KVT % 1024 == 0 && OutSmem::W % 1024 == 0, "alignment");
 static_assert(OutSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 
 struct OutMisc {
-  uint64_t full[OUT_STAGES], empty[OUT_STAGES], logits_full, logits_free, phi_full, phi_free, const_bar;
+  // phi_full[f]: the 64-feature block f of the phi tile is written (the 128 threads of its half arrive)
+  uint64_t full[OUT_STAGES], empty[OUT_STAGES], logits_full, logits_free, phi_full[TC_M / 64], phi_free, const_bar;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -441,7 +411,7 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
     for (int i = 0; i < OUT_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], 1); }
     mbar_init(&misc->logits_full, 1);
     mbar_init(&misc->logits_free, EPI_THREADS);
-    mbar_init(&misc->phi_full, EPI_THREADS);
+    for (int i = 0; i < TC_M / 64; i++) mbar_init(&misc->phi_full[i], EPI_THREADS / 2);
     mbar_init(&misc->phi_free, 1);
     mbar_init(&misc->const_bar, 1);
     misc->abort_flag = 0;
@@ -493,10 +463,10 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       const uint64_t dKvt = smem_desc(smem_u32(sm + OutSmem::KVT), 16, 1024, SWZ_128B);
       auto issue_logits = [&](int st) {
         const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
-#pragma unroll 1
+#pragma unroll
         for (int k = 0; k < TC_D / 16; k++)
           mma_bf16(tmem + OUT_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dW, 32 * k), ID_LOGITS, k > 0);
-#pragma unroll 1
+#pragma unroll
         for (int k = 0; k < TC_D / 16; k++)
           mma_bf16(tmem + OUT_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dWlo, 32 * k), ID_LOGITS, 1);
         mma_commit(&misc->logits_full);
@@ -516,15 +486,19 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           tcgen05_fence_after();
           issue_logits(sn);
         }
-        // the epilogue arrives on phi_full only after it has read the previous tile's outputs
-        if (!mbar_wait(&misc->phi_full, it & 1, abortp, status)) break;
-        tcgen05_fence_after();
+        // Every 64-feature block of phi is contracted as soon as it is written, first blocks of both
+        // halves first, so only the last block's MMAs are left when the exponentials end.  The
+        // epilogue arrives on a tile's first block only after it has read the previous tile's outputs.
 #pragma unroll 1
-        for (int fb = 0; fb < TC_M / 64; fb++)          // feature halves 0 (fb 0, 1) and 1 (fb 2, 3)
-#pragma unroll 1
+        for (int o = 0; o < TC_M / 64 && ok; o++) {
+          const int fb = ((o & 1) << 1) | (o >> 1);      // 0, 2, 1, 3: feature halves 0 (fb 0, 1) and 1 (fb 2, 3)
+          if (!mbar_wait(&misc->phi_full[fb], it & 1, abortp, status)) { ok = false; break; }
+          tcgen05_fence_after();
+#pragma unroll
           for (int k = 0; k < 4; k++)
             mma_bf16(tmem + OUT_COL_OUT + (fb >> 1) * TC_NV, desc_advance(dPhi, fb * TILE_BYTES + 32 * k),
                      desc_advance(dKvt, fb * KVT_BLOCK_BYTES + 32 * k), ID_OUT, ((fb & 1) || k > 0) ? 1u : 0u);
+        }
         mma_commit(&misc->phi_free);
       }
     }
@@ -557,19 +531,28 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       const float m0 = rm[row], m1 = rm[TILE + row];
       const float m = fmaxf(m0, m1);
       const float f0 = ex2(m0 - m), f1 = ex2(m1 - m);
-      const int64_t r = (int64_t)(tile0 + j) * TILE + row;
-      if (r < L) {
-        const float den = fmaf(f0, __uint_as_float(d0[0]), f1 * __uint_as_float(d1[0]));
-        if (!(den > 0.f) || !isfinite(den)) atomicExch(status, FSHARP_E_NONFINITE);
-        const float i0 = f0 / den, i1 = f1 / den;
-        uint32_t o[16];
+      const int64_t r0 = (int64_t)(tile0 + j) * TILE + q * 32;       // first row of this warp
+      const float den = fmaf(f0, __uint_as_float(d0[0]), f1 * __uint_as_float(d1[0]));
+      if (r0 + lane < L && (!(den > 0.f) || !isfinite(den))) atomicExch(status, FSHARP_E_NONFINITE);
+      const float i0 = f0 / den, i1 = f1 / den;
+      // The thread's 64 bytes go through shared memory so that a store instruction of the warp
+      // covers 8 rows x 64 contiguous bytes instead of 32 rows x 16 bytes.
+      uint8_t* stg = sm + OutSmem::STAGE + warp * 2048;
 #pragma unroll
-        for (int i = 0; i < 16; i++)
-          o[i] = pack_bf16(fmaf(i0, __uint_as_float(n0[2 * i]), i1 * __uint_as_float(n1[2 * i])),
-                           fmaf(i0, __uint_as_float(n0[2 * i + 1]), i1 * __uint_as_float(n1[2 * i + 1])));
-        uint4* dst = reinterpret_cast<uint4*>(Yb + r * ay.sl + hf * 32);
+      for (int i = 0; i < 4; i++) {
+        uint32_t o[4];
 #pragma unroll
-        for (int i = 0; i < 4; i++) dst[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+        for (int e = 0; e < 4; e++)
+          o[e] = pack_bf16(fmaf(i0, __uint_as_float(n0[8 * i + 2 * e]), i1 * __uint_as_float(n1[8 * i + 2 * e])),
+                           fmaf(i0, __uint_as_float(n0[8 * i + 2 * e + 1]), i1 * __uint_as_float(n1[8 * i + 2 * e + 1])));
+        *reinterpret_cast<uint4*>(stg + lane * 64 + ((i ^ ((lane >> 1) & 3)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+      __syncwarp();
+#pragma unroll
+      for (int i = 0; i < 4; i++) {
+        const int rr = (lane >> 2) + 8 * i, c = lane & 3;
+        const uint4 val = *reinterpret_cast<const uint4*>(stg + rr * 64 + ((c ^ ((rr >> 1) & 3)) << 4));
+        if (r0 + rr < L) *reinterpret_cast<uint4*>(Yb + (r0 + rr) * ay.sl + hf * 32 + c * 8) = val;
       }
     };
     for (int it = 0; it < ntiles && alive; it++) {
@@ -605,10 +588,12 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         for (int j = 0; j < 4; j++)
           p[j] = pack_f16(ex2(__uint_as_float(v[c * 8 + 2 * j]) - mx), ex2(__uint_as_float(v[c * 8 + 2 * j + 1]) - mx));
         *reinterpret_cast<uint4*>(prow + (c >> 3) * TILE_BYTES + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
+        if ((c & 7) == 7) {                     // a 64-feature block of this half is complete
+          fence_proxy_async_smem();
+          tcgen05_fence_before();
+          mbar_arrive(&misc->phi_full[hf * 2 + (c >> 3)]);
+        }
       }
-      fence_proxy_async_smem();
-      tcgen05_fence_before();
-      mbar_arrive(&misc->phi_full);
     }
     if (alive && ntiles > 0 && mbar_wait(&misc->phi_free, (ntiles - 1) & 1, abortp, status, false)) write_out(ntiles - 1);
   }
@@ -647,6 +632,8 @@ int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int
 int make_map_kvt(CUtensorMap* map, const void* base, int BH);
 }  // namespace tchost
 int fs_tc_prep(fsharp_ctx* ctx, const float* prep, int G, float qk_scale, uint8_t* images, int* flags);
+int fs_tc_rowterm(fsharp_ctx* ctx, const void* K, const fsharp_dims* dm, const uint8_t* images, const int* flags, int Lpad,
+                  int tiles_per_split, int nsplit, float* crow);
 size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
 int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
                 const float* prep, void* Y, WsAlloc* ws);
@@ -657,7 +644,8 @@ size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
   const size_t BH = (size_t)dm->B * dm->H;
   const size_t G = fs_groups(dm);
   return ws_round(G * 2 * IMG_BYTES) + ws_round(G * 2 * FLAG_WORDS * 4 + 64) +
-         ws_round(BH * MAX_KEY_SPLIT * TC_M * TC_NV * 4) + 2 * ws_round(BH * MAX_KEY_SPLIT * 4) +
+         ws_round(BH * MAX_KEY_SPLIT * TC_M * TC_NV * 4) + 2 * ws_round(BH * MAX_KEY_SPLIT * 2 * 4) +
+         ws_round(BH * (size_t)((dm->Lk + TILE - 1) / TILE) * TILE * 4) +
          ws_round(BH * TC_NV * TC_M * 2);
 }
 
@@ -674,9 +662,12 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   int tps = 0;
   int nsplit = pick_split(BH, ktiles, ctx->sm_count, MAX_KEY_SPLIT, &tps);
   float* partial = ws->take<float>((size_t)BH * MAX_KEY_SPLIT * TC_M * TC_NV);
-  float* shifts = ws->take<float>((size_t)BH * MAX_KEY_SPLIT);
-  int* pmax = ws->take<int>((size_t)BH * MAX_KEY_SPLIT);
-  FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * MAX_KEY_SPLIT * sizeof(int), ctx->stream));
+  float* shifts = ws->take<float>((size_t)BH * MAX_KEY_SPLIT * 2);
+  int* pmax = ws->take<int>((size_t)BH * MAX_KEY_SPLIT * 2);
+  FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * MAX_KEY_SPLIT * 2 * sizeof(int), ctx->stream));
+  const int Lpad = ktiles * TILE;
+  float* crow = ws->take<float>((size_t)BH * Lpad);
+  FS_TRY(fs_tc_rowterm(ctx, K, dm, images, flags, Lpad, tps, nsplit, crow));
   __half* kvt = ws->take<__half>((size_t)BH * TC_NV * TC_M);
 
   CUtensorMap tmK, tmV, tmQ, tmKVt;
@@ -689,7 +680,7 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   FS_CUDA_OK(cudaFuncSetAttribute(tc_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OutSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_KV);
   tc_kv_kernel<<<dim3(nsplit, BH), TC_THREADS, KvSmem::TOTAL + 1024, ctx->stream>>>(
-      tmK, tmV, images, flags, H, dm->pool, Lk, tps, nsplit, partial, shifts, pmax, ctx->d_status);
+      tmK, tmV, images, crow, H, dm->pool, Lk, Lpad, tps, nsplit, partial, shifts, pmax, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   FS_TIME_BEGIN(ctx, FS_K_TC_MERGE);

@@ -157,7 +157,7 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes
 // A descriptor moved by a byte offset inside its matrix: only the 14-bit start-address field
 // (16-byte units) of the low word changes, so one 32-bit add does it.
 __device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t byte_offset) {
-  return desc + (uint64_t)(byte_offset >> 4);
+  return (desc & 0xFFFFFFFF00000000ull) | (uint64_t)((uint32_t)desc + (byte_offset >> 4));
 }
 // Instruction descriptor, kind::f16 with bf16 operands and fp32 accumulation.
 // a_mn / b_mn: 1 if that operand is MN-major (its M or N index is the contiguous one).

@@ -1,0 +1,169 @@
+// Per-key term of the feature exponent (Theorem 4.1: the x^T C^(2) x part of phi) on the tensor
+// cores, for bf16 keys with d = 64:  c_j = log2e * qk_scale^2 * x_j^T C x_j, one fp32 value per key.
+//
+// T = X C (tcgen05, C split into a bf16 value and its bf16 remainder) lands in TMEM; thread j of
+// the epilogue dots row j of T with x_j, which it reads from the same shared-memory tile.
+// Computing c_j ahead of the key-side kernel keeps that kernel's TMEM and shared memory for the
+// feature tiles; the keys read here stay in L2 for it.
+#include "common.cuh"
+#include "tc_common.cuh"
+#include "tc_layout.cuh"
+
+using namespace tc;
+using namespace tcl;
+
+namespace {
+
+constexpr int RT_STAGES = 4;
+constexpr int RT_EPI_THREADS = 128, RT_WARP_TMA = 4, RT_WARP_MMA = 5, RT_THREADS = 192;
+constexpr uint32_t RT_TMEM_COLS = 128;       // two T buffers of 64 columns
+
+struct RtSmem {
+  static constexpr uint32_t X0 = 0, CHI = RT_STAGES * TILE_BYTES, CLO = CHI + IMG_C_BYTES, MISC = CLO + IMG_C_BYTES,
+                            TOTAL = MISC + 256;
+};
+struct RtMisc {
+  uint64_t full[RT_STAGES], empty[RT_STAGES], t_full[2], t_free[2], const_bar;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+static_assert(sizeof(RtMisc) <= 256, "misc block");
+
+__global__ void __launch_bounds__(RT_THREADS)
+tc_rowterm_kernel(const __grid_constant__ CUtensorMap tmK, const uint8_t* __restrict__ images,
+                  const int* __restrict__ img_flags, int H, int pool, int L, int Lpad, int tiles_per_split,
+                  float* __restrict__ crow, int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  RtMisc* misc = reinterpret_cast<RtMisc*>(sm + RtSmem::MISC);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = blockIdx.y, b = bh / H, h = bh % H;
+  const int g = pool == FSHARP_POOL_PER_BH ? bh : h;
+  const int total_tiles = (L + TILE - 1) / TILE;
+  const int tile0 = blockIdx.x * tiles_per_split;
+  const int ntiles = min(tiles_per_split, total_tiles - tile0);
+  if (ntiles <= 0) return;                    // uniform over the block, before anything is allocated
+  const uint8_t* img = images + ((size_t)g * 2 + 1) * IMG_BYTES;        // side 2 (keys)
+  const bool clo = (img_flags[((size_t)g * 2 + 1) * FLAG_WORDS] & FLAG_C_LO) != 0;
+  volatile int* abortp = &misc->abort_flag;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < RT_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], RT_EPI_THREADS); }
+    for (int i = 0; i < 2; i++) { mbar_init(&misc->t_full[i], 1); mbar_init(&misc->t_free[i], RT_EPI_THREADS); }
+    mbar_init(&misc->const_bar, 1);
+    misc->abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == RT_WARP_MMA) {
+    tmem_alloc(&misc->tmem_base, RT_TMEM_COLS);
+    tmem_relinquish();
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem = misc->tmem_base;
+
+  if (warp == RT_WARP_TMA) {
+    if (lane == 0) {
+      prefetch_tmap(&tmK);
+      mbar_expect_tx(&misc->const_bar, 2 * IMG_C_BYTES);
+      bulk_load(sm + RtSmem::CHI, img + IMG_CHI, IMG_C_BYTES, &misc->const_bar);
+      bulk_load(sm + RtSmem::CLO, img + IMG_CLO, IMG_C_BYTES, &misc->const_bar);
+      int issued = 0;
+      for (int it = 0; it < ntiles; it++) {
+        const int st = it % RT_STAGES;
+        if (!mbar_wait(&misc->empty[st], ((it / RT_STAGES) & 1) ^ 1, abortp, status)) break;
+        mbar_expect_tx(&misc->full[st], TILE_BYTES);
+        tma_load_4d(sm + RtSmem::X0 + st * TILE_BYTES, &tmK, &misc->full[st], 0, (tile0 + it) * TILE, h, b);
+        issued = it + 1;
+      }
+      // no copy of this block may still be in flight when it exits
+      mbar_wait(&misc->const_bar, 0, abortp, status, false);
+      for (int it = max(0, issued - RT_STAGES); it < issued; it++)
+        mbar_wait(&misc->full[it % RT_STAGES], (it / RT_STAGES) & 1, abortp, status, false);
+    }
+  } else if (warp == RT_WARP_MMA) {
+    if (lane == 0) {
+      constexpr uint32_t ID_T = idesc_bf16(128, TC_D, 0, 0);
+      const uint64_t dX0 = smem_desc(smem_u32(sm + RtSmem::X0), 16, 1024, SWZ_128B);
+      const uint64_t dChi = smem_desc(smem_u32(sm + RtSmem::CHI), 16, 1024, SWZ_128B);
+      const uint64_t dClo = smem_desc(smem_u32(sm + RtSmem::CLO), 16, 1024, SWZ_128B);
+      bool ok = mbar_wait(&misc->const_bar, 0, abortp, status);
+      for (int it = 0; ok && it < ntiles; it++) {
+        const int st = it % RT_STAGES, buf = it & 1;
+        if (!mbar_wait(&misc->full[st], (it / RT_STAGES) & 1, abortp, status)) break;
+        if (!mbar_wait(&misc->t_free[buf], ((it >> 1) & 1) ^ 1, abortp, status)) break;
+        tcgen05_fence_after();
+        const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
+#pragma unroll 1
+        for (int k = 0; k < TC_D / 16; k++)
+          mma_bf16(tmem + buf * TC_D, desc_advance(dX, 32 * k), desc_advance(dChi, 32 * k), ID_T, k > 0);
+        if (clo) {
+#pragma unroll 1
+          for (int k = 0; k < TC_D / 16; k++)
+            mma_bf16(tmem + buf * TC_D, desc_advance(dX, 32 * k), desc_advance(dClo, 32 * k), ID_T, 1);
+        }
+        mma_commit(&misc->t_full[buf]);
+      }
+    }
+  } else {
+    // epilogue: one key row per thread
+    const int row = warp * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+    float* out = crow + (size_t)bh * Lpad + (size_t)tile0 * TILE + row;
+    for (int it = 0; it < ntiles; it++) {
+      const int st = it % RT_STAGES, buf = it & 1;
+      if (!mbar_wait(&misc->full[st], (it / RT_STAGES) & 1, abortp, status, false)) break;
+      if (!mbar_wait(&misc->t_full[buf], (it >> 1) & 1, abortp, status, false)) break;
+      __syncwarp();
+      tcgen05_fence_after();
+      const uint8_t* xrow = sm + RtSmem::X0 + st * TILE_BYTES + row * 128;
+      float part[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int c = 0; c < TC_D / 16; c++) {
+        uint32_t t[16];
+        tmem_ld16(lane_addr + buf * TC_D + c * 16, t);
+        const uint4 u0 = *reinterpret_cast<const uint4*>(xrow + (((2 * c) ^ (row & 7)) << 4));
+        const uint4 u1 = *reinterpret_cast<const uint4*>(xrow + (((2 * c + 1) ^ (row & 7)) << 4));
+        const uint32_t w8[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+          part[j & 3] = fmaf(__uint_as_float(t[2 * j]), __uint_as_float(w8[j] << 16), part[j & 3]);
+          part[j & 3] = fmaf(__uint_as_float(t[2 * j + 1]), __uint_as_float(w8[j] & 0xffff0000u), part[j & 3]);
+        }
+      }
+      tcgen05_fence_before();
+      mbar_arrive(&misc->t_free[buf]);
+      mbar_arrive(&misc->empty[st]);
+      out[(size_t)it * TILE] = (part[0] + part[1]) + (part[2] + part[3]);
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == RT_WARP_MMA) {
+    tcgen05_fence_after();
+    tmem_dealloc(tmem, RT_TMEM_COLS);
+  }
+}
+
+}  // namespace
+
+namespace tchost {
+int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int H, int L, int inner);
+}
+
+// crow: [B*H][Lpad] floats with Lpad = ceil(Lk / 128) * 128; rows at and beyond Lk come out as zero.
+int fs_tc_rowterm(fsharp_ctx* ctx, const void* K, const fsharp_dims* dm, const uint8_t* images, const int* flags, int Lpad,
+                  int tiles_per_split, int nsplit, float* crow) {
+  const int B = dm->B, H = dm->H, Lk = dm->Lk;
+  CUtensorMap tmK;
+  FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, Lk, dm->d), B, H, Lk, dm->d));
+  FS_CUDA_OK(cudaFuncSetAttribute(tc_rowterm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RtSmem::TOTAL + 1024));
+  FS_TIME_BEGIN(ctx, FS_K_TC_ROWTERM);
+  tc_rowterm_kernel<<<dim3(nsplit, B * H), RT_THREADS, RtSmem::TOTAL + 1024, ctx->stream>>>(
+      tmK, images, flags, H, dm->pool, Lk, Lpad, tiles_per_split, crow, ctx->d_status);
+  FS_TIME_END(ctx);
+  FS_LAUNCH_CHECK(ctx);
+  return FSHARP_OK;
+}
