@@ -395,7 +395,7 @@ __device__ void jacobi_tables(const ushort2* sched, uchar2* pos, uint2* la, ucha
 struct FitArgs {
   const double* stats;
   double* params;
-  double* scratch;   // per group 4*d*d doubles
+  double* scratch;   // per group 5*d*d doubles
   int d, variant;
   double ridge;
   int v_in_smem;
@@ -411,13 +411,14 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
   ParamsLayout pl{d};
   const double* st = a.stats + (size_t)g * sl.total();
   double* out = a.params + (size_t)g * pl.total();
-  double* gs = a.scratch + (size_t)g * 4 * d * d;
+  double* gs = a.scratch + (size_t)g * 5 * d * d;
 
   double* As = sm;                                   // d*(d+1)
   double* A1 = As + d * lda;                         // second copy of A (look-ahead solver only)
   double* Vs = V_IN_SMEM ? A1 + d * lda : gs;        // eigenvectors, one per ROW
   const int ldv = V_IN_SMEM ? lda : d;
-  double* vec = As + d * lda + (V_IN_SMEM ? 2 * d * lda : 0);
+  double* Ws = Vs + d * lda;                         // fourth d x d buffer (ADERF products, d <= 64 only)
+  double* vec = As + d * lda + (V_IN_SMEM ? 3 * d * lda : 0);
   double* lam = vec;             // [d]
   double* aux = vec + d;         // [d]
   double* cs = vec + 2 * d;      // [2d]
@@ -554,48 +555,112 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
     obj = so - t1 - t2;
     phi = lam[0];
   } else {  // FSHARP_ADERF, Theorem 4.2
-    double* Q1g = gs + (size_t)d * d;
+    // The theorem writes M1 = Q1 L1 Q1^T and uses F = L1^1/2 Q1^T only as a factor with F^T F = M1:
+    // with any other such factor F' = O F (O orthogonal), F' M2 F'^T = O (F M2 F^T) O^T has the
+    // eigenvectors U' = O U and the same Sigma^2, so B1 = r Sigma^1/2 U'^T F'^-T and
+    // B2 = r Sigma^-1/2 U'^T F' come out the same.  The Cholesky factor F' = L^T (M1 = L L^T) is
+    // taken: one eigen-solve is left instead of two.
+    double* Lg = gs + (size_t)d * d;        // L     [i][j], lower triangular (upper part zero)
     double* T1g = gs + (size_t)2 * d * d;
     double* Ug = gs + (size_t)3 * d * d;
+    double* Lig = gs + (size_t)4 * d * d;   // L^-1  [i][j], lower triangular
     for (int e = tid; e < d * d; e += FIT_THREADS) {
       int i = e / d, j = e % d;
       As[i * lda + j] = M1[e] + (i == j ? rg1 : 0.0);
     }
     __syncthreads();
-    nsweeps += eig();
-    double lmin = 1e300, lmax = 0.0;
-    for (int i = tid; i < d; i += FIT_THREADS) {
-      double li = As[i * lda + i];
-      lmin = fmin(lmin, li); lmax = fmax(lmax, li);
+    // Cholesky, column by column: `parts` threads share the dot product of a row.
+    const int parts = FIT_THREADS / d, ri = tid / parts, part = tid % parts;
+    const double floor_piv = 1e-12 * t1 / d;
+    for (int j = 0; j < d; j++) {
+      double t = 0.0;
+      if (ri >= j) {
+        for (int k = part; k < j; k += parts) t = fma(As[ri * lda + k], As[j * lda + k], t);
+      }
+      for (int o = parts >> 1; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+      if (ri >= j && part == 0) aux[ri] = As[ri * lda + j] - t;
+      __syncthreads();
+      double piv = aux[j];
+      if (!(piv > floor_piv)) { violated = true; piv = floor_piv + 1e-300; }
+      const double ljj = sqrt(piv);
+      if (part == 0) {
+        if (ri == j) As[j * lda + j] = ljj;
+        else if (ri > j) As[ri * lda + j] = aux[ri] / ljj;
+        else As[ri * lda + j] = 0.0;                 // upper triangle
+      }
+      __syncthreads();
     }
-    lmin = block_reduce(lmin, red, 2);
-    lmax = block_reduce(lmax, red, 1);
-    if (!(lmin > 1e-12 * lmax)) violated = true;
-    for (int i = tid; i < d; i += FIT_THREADS) lam[i] = fmax(As[i * lda + i], 1e-300 + 1e-12 * lmax);
-    for (int e = tid; e < d * d; e += FIT_THREADS) Q1g[e] = Vs[(e % d) * ldv + (e / d)];   // Q1[i][l]
+    // L^-1 by forward substitution, one column per thread group (columns are independent; the
+    // threads of a group sit in one warp).  It is built in shared memory when there is room.
+    double* Li = V_IN_SMEM ? A1 : Lig;
+    const int ldi = V_IN_SMEM ? lda : d;
+    {
+      const int c = ri;
+      for (int i = 0; i < d; i++) {
+        double t = 0.0;
+        if (i > c)
+          for (int k = c + part; k < i; k += parts) t = fma(As[i * lda + k], Li[k * ldi + c], t);
+        for (int o = parts >> 1; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (part == 0) Li[i * ldi + c] = i < c ? 0.0 : (i == c ? 1.0 / As[c * lda + c] : -t / As[i * lda + i]);
+        __syncwarp();
+      }
+    }
     __syncthreads();
-    // T1 = M2 Q1 L1^1/2
     for (int e = tid; e < d * d; e += FIT_THREADS) {
-      int i = e / d, l = e % d;
-      double s = 0.0;
-      for (int j = 0; j < d; j++) s = fma(M2[i * d + j] + (i == j ? rg2 : 0.0), Q1g[j * d + l], s);
-      T1g[e] = s * sqrt(lam[l]);
+      Lg[e] = As[(e / d) * lda + (e % d)];
+      if (V_IN_SMEM) {
+        Lig[e] = Li[(e / d) * ldi + (e % d)];
+        Vs[(e / d) * lda + (e % d)] = M2[e] + ((e / d) == (e % d) ? rg2 : 0.0);      // M2 into shared memory
+      }
     }
     __syncthreads();
-    // Z Z^T = L1^1/2 Q1^T M2 Q1 L1^1/2  (symmetric; both triangles written from the same sum)
-    for (int e = tid; e < d * d; e += FIT_THREADS) {
-      int r = e / d, c = e % d;
-      if (r > c) continue;
-      double s = 0.0;
-      for (int i = 0; i < d; i++) s = fma(Q1g[i * d + r] * sqrt(lam[r]), T1g[i * d + c], s);
-      double s2 = 0.0;
-      for (int i = 0; i < d; i++) s2 = fma(Q1g[i * d + c] * sqrt(lam[c]), T1g[i * d + r], s2);
-      double v = 0.5 * (s + s2);
-      As[r * lda + c] = v;
-      As[c * lda + r] = v;
+    if (V_IN_SMEM) {
+      // T1 = M2 L (M2 in Vs, L in As) -> Ws
+      for (int e = tid; e < d * d; e += FIT_THREADS) {
+        int i = e / d, l = e % d;
+        double s = 0.0;
+        for (int j = l; j < d; j++) s = fma(Vs[i * lda + j], As[j * lda + l], s);
+        Ws[i * lda + l] = s;
+      }
+      __syncthreads();
+      // Z Z^T = L^T T1 (symmetric; both triangles written from the same sum) -> Vs, then As
+      for (int e = tid; e < d * d; e += FIT_THREADS) {
+        int r = e / d, c = e % d;
+        if (r > c) continue;
+        double s = 0.0, s2 = 0.0;
+        for (int i = r; i < d; i++) s = fma(As[i * lda + r], Ws[i * lda + c], s);
+        for (int i = c; i < d; i++) s2 = fma(As[i * lda + c], Ws[i * lda + r], s2);
+        double v = 0.5 * (s + s2);
+        Vs[r * lda + c] = v;
+        Vs[c * lda + r] = v;
+      }
+      __syncthreads();
+      for (int e = tid; e < d * lda; e += FIT_THREADS) As[e] = Vs[e];
+      __syncthreads();
+    } else {
+      // T1 = M2 L
+      for (int e = tid; e < d * d; e += FIT_THREADS) {
+        int i = e / d, l = e % d;
+        double s = 0.0;
+        for (int j = l; j < d; j++) s = fma(M2[i * d + j] + (i == j ? rg2 : 0.0), Lg[j * d + l], s);
+        T1g[e] = s;
+      }
+      __syncthreads();
+      // Z Z^T = L^T M2 L  (symmetric; both triangles written from the same sum)
+      for (int e = tid; e < d * d; e += FIT_THREADS) {
+        int r = e / d, c = e % d;
+        if (r > c) continue;
+        double s = 0.0;
+        for (int i = r; i < d; i++) s = fma(Lg[i * d + r], T1g[i * d + c], s);
+        double s2 = 0.0;
+        for (int i = c; i < d; i++) s2 = fma(Lg[i * d + c], T1g[i * d + r], s2);
+        double v = 0.5 * (s + s2);
+        As[r * lda + c] = v;
+        As[c * lda + r] = v;
+      }
+      __syncthreads();
     }
-    __syncthreads();
-    nsweeps += eig();     // eigenvalues Sigma^2, eigenvectors U
+    nsweeps += eig();     // eigenvalues Sigma^2, eigenvectors U (rows of Vs)
     double smin = 1e300, smax = 0.0, ssum = 0.0;
     for (int l = tid; l < d; l += FIT_THREADS) {
       double sg = sqrt(fmax(As[l * lda + l], 0.0));
@@ -607,36 +672,83 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
     ssum = block_reduce(ssum, red, 0);
     if (!(smin > 1e-12 * smax)) violated = true;
     for (int l = tid; l < d; l += FIT_THREADS) aux[l] = fmax(aux[l], 1e-300 + 1e-12 * smax);
-    for (int e = tid; e < d * d; e += FIT_THREADS) Ug[e] = Vs[(e % d) * ldv + (e / d)];     // U[i][l]
-    __syncthreads();
     const double mu3 = mm / d;
     phi = 2.0 * ssum / d + 2.0 * mu3;
     const double A = lemma_a1(phi);
     const double r = sqrt(1.0 - 4.0 * A);
-    // B1 = r Sigma^1/2 U^T L1^-1/2 Q1^T,  B2 = r Sigma^-1/2 U^T L1^1/2 Q1^T
-    for (int e = tid; e < d * d; e += FIT_THREADS) {
-      int l = e / d, j = e % d;
-      double s1 = 0.0, s2 = 0.0;
-      for (int i = 0; i < d; i++) {
-        double u = Ug[i * d + l], q = Q1g[j * d + i], sq = sqrt(lam[i]);
-        s1 = fma(u / sq, q, s1);
-        s2 = fma(u * sq, q, s2);
+    if (V_IN_SMEM) {
+      // L^-1 -> A1, L -> Ws (shared memory again; the eigen-solve used both buffers)
+      for (int e = tid; e < d * d; e += FIT_THREADS) {
+        A1[(e / d) * lda + (e % d)] = Lig[e];
+        Ws[(e / d) * lda + (e % d)] = Lg[e];
       }
-      double sg = sqrt(aux[l]);
-      oB1[e] = r * sg * s1;
-      oB2[e] = r / sg * s2;
-      oA[e] = (l == j) ? A : 0.0;
-    }
-    __syncthreads();
-    for (int e = tid; e < d * d; e += FIT_THREADS) {
-      int i = e / d, j = e % d;
-      double s1 = 0.0, s2 = 0.0;
-      for (int l = 0; l < d; l++) {
-        s1 = fma(oB1[l * d + i], oB1[l * d + j], s1);
-        s2 = fma(oB2[l * d + i], oB2[l * d + j], s2);
+      __syncthreads();
+      // B1 = r Sigma^1/2 U^T L^-1,  B2 = r Sigma^-1/2 U^T L^T, kept in shared memory (As, then A1) for C
+      constexpr int EPT = 8;                      // d * d / FIT_THREADS for d = 64; fewer elements for smaller d
+      double b1[EPT], b2[EPT];
+#pragma unroll
+      for (int u = 0; u < EPT; u++) {
+        const int e = tid + u * FIT_THREADS;
+        b1[u] = b2[u] = 0.0;
+        if (e < d * d) {
+          int l = e / d, j = e % d;
+          double s1 = 0.0, s2 = 0.0;
+          for (int i = j; i < d; i++) s1 = fma(Vs[l * ldv + i], A1[i * lda + j], s1);
+          for (int i = 0; i <= j; i++) s2 = fma(Vs[l * ldv + i], Ws[j * lda + i], s2);
+          const double sg = sqrt(aux[l]);
+          b1[u] = r * sg * s1;
+          b2[u] = r / sg * s2;
+        }
       }
-      oC1[e] = -s1 / (2.0 * (1.0 - 4.0 * A));
-      oC2[e] = -s2 / (2.0 * (1.0 - 4.0 * A));
+      __syncthreads();
+#pragma unroll
+      for (int u = 0; u < EPT; u++) {
+        const int e = tid + u * FIT_THREADS;
+        if (e < d * d) {
+          int l = e / d, j = e % d;
+          As[l * lda + j] = b1[u];
+          A1[l * lda + j] = b2[u];
+          oB1[e] = b1[u];
+          oB2[e] = b2[u];
+          oA[e] = (l == j) ? A : 0.0;
+        }
+      }
+      __syncthreads();
+      for (int e = tid; e < d * d; e += FIT_THREADS) {
+        int i = e / d, j = e % d;
+        double s1 = 0.0, s2 = 0.0;
+        for (int l = 0; l < d; l++) {
+          s1 = fma(As[l * lda + i], As[l * lda + j], s1);
+          s2 = fma(A1[l * lda + i], A1[l * lda + j], s2);
+        }
+        oC1[e] = -s1 / (2.0 * (1.0 - 4.0 * A));
+        oC2[e] = -s2 / (2.0 * (1.0 - 4.0 * A));
+      }
+    } else {
+      for (int e = tid; e < d * d; e += FIT_THREADS) Ug[e] = Vs[(e % d) * ldv + (e / d)];     // U[i][l]
+      __syncthreads();
+      // B1 = r Sigma^1/2 U^T L^-1,  B2 = r Sigma^-1/2 U^T L^T
+      for (int e = tid; e < d * d; e += FIT_THREADS) {
+        int l = e / d, j = e % d;
+        double s1 = 0.0, s2 = 0.0;
+        for (int i = j; i < d; i++) s1 = fma(Ug[i * d + l], Lig[i * d + j], s1);
+        for (int i = 0; i <= j; i++) s2 = fma(Ug[i * d + l], Lg[j * d + i], s2);
+        double sg = sqrt(aux[l]);
+        oB1[e] = r * sg * s1;
+        oB2[e] = r / sg * s2;
+        oA[e] = (l == j) ? A : 0.0;
+      }
+      __syncthreads();
+      for (int e = tid; e < d * d; e += FIT_THREADS) {
+        int i = e / d, j = e % d;
+        double s1 = 0.0, s2 = 0.0;
+        for (int l = 0; l < d; l++) {
+          s1 = fma(oB1[l * d + i], oB1[l * d + j], s1);
+          s2 = fma(oB2[l * d + i], oB2[l * d + j], s2);
+        }
+        oC1[e] = -s1 / (2.0 * (1.0 - 4.0 * A));
+        oC2[e] = -s2 / (2.0 * (1.0 - 4.0 * A));
+      }
     }
     logD = 0.25 * d * log(1.0 - 4.0 * A);
     obj = d * (log(1.0 - 4.0 * A) - 0.5 * log(1.0 - 8.0 * A) + 2.0 / (1.0 - 8.0 * A) * (ssum / d + mu3) + 2.0 * mu3);
@@ -652,7 +764,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
 }
 
 size_t fit_smem_bytes(int d, int v_in_smem) {
-  size_t dbl = (size_t)d * (d + 1) * (v_in_smem ? 3 : 1) + 4 * (size_t)d + FIT_THREADS;
+  size_t dbl = (size_t)d * (d + 1) * (v_in_smem ? 4 : 1) + 4 * (size_t)d + FIT_THREADS;
   size_t tables = v_in_smem ? ((size_t)(d - 1) * d + (size_t)(d / 2) * (d / 2 + 1) / 2) * sizeof(uchar2) +
                                   ((size_t)(d - 1) * (d / 2) + 1) * sizeof(uint2) : 0;
   return dbl * sizeof(double) + (size_t)d * sizeof(int) + (size_t)(d - 1) * (d / 2) * sizeof(ushort2) + tables;
@@ -660,7 +772,7 @@ size_t fit_smem_bytes(int d, int v_in_smem) {
 
 }  // namespace
 
-size_t fs_fit_scratch_doubles(int G, int d) { return (size_t)G * 4 * d * d; }
+size_t fs_fit_scratch_doubles(int G, int d) { return (size_t)G * 5 * d * d; }
 
 int fs_run_fit(fsharp_ctx* ctx, const double* stats, int G, int d, int variant, double ridge,
                double* params, double* scratch) {
