@@ -198,10 +198,16 @@ prefix_kernel(float* __restrict__ st, int nchunks, int64_t elems) {
   float* base = st + (int64_t)bh * nchunks * elems;
   for (int64_t e = blockIdx.x * (int64_t)NTH + threadIdx.x; e < elems; e += (int64_t)gridDim.x * NTH) {
     float run = 0.f;
-    for (int c = 0; c < nchunks; c++) {
-      float v = base[c * elems + e];
-      base[c * elems + e] = run;
-      run += v;
+    // eight chunks at a time: the loads are issued together, then the running sums are stored
+    for (int c0 = 0; c0 < nchunks; c0 += 8) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; u++) v[u] = c0 + u < nchunks ? base[(c0 + u) * elems + e] : 0.f;
+#pragma unroll
+      for (int u = 0; u < 8; u++) {
+        if (c0 + u < nchunks) base[(c0 + u) * elems + e] = run;
+        run += v[u];
+      }
     }
   }
 }
