@@ -157,6 +157,7 @@ const char* fsharp_kernel_name(int id) {
     case FS_K_TC_CAUSAL_OUT: return "tc_causal_out_kernel";
     case FS_K_TC_STATS: return "tc_stats_kernel";
     case FS_K_TC_ROWTERM: return "tc_rowterm_kernel";
+    case FS_K_TC_FEATQ: return "tc_featq_kernel";
     default: return "";
   }
 }

@@ -38,8 +38,8 @@ constexpr int PREFETCH_TILES = 4;   // tiles pulled into L2 ahead of the shared-
 // columns): one MMA covers N = 128 features instead of 80 value columns.
 struct KvSmem {
   static constexpr uint32_t X0 = 0, V0 = 2 * TILE_BYTES, ONES = 4 * TILE_BYTES, W = ONES + TILE_BYTES,
-                            WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES, MISC = PHI + 4 * TILE_BYTES,
-                            TOTAL = MISC + 256;
+                            WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES, FA2 = PHI + 4 * TILE_BYTES,
+                            MISC = FA2 + TC_M * 4, TOTAL = MISC + 256;
 };
 static_assert(KvSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 static_assert(KvSmem::PHI % 1024 == 0 && KvSmem::W % 1024 == 0 && KvSmem::ONES % 1024 == 0, "swizzled tiles need 1024-byte alignment");
@@ -59,10 +59,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
              const uint8_t* __restrict__ images, const float* __restrict__ crow, int H, int pool, int L, int Lpad,
              int tiles_per_split, int nsplit, float* __restrict__ partial, float* __restrict__ shifts,
-             int* __restrict__ pmax, int* __restrict__ status) {
+             int* __restrict__ pmax, __half* __restrict__ phik16, int* __restrict__ status) {
+  // phik16 != nullptr (causal use: one 128-key chunk per block): the key side's share a2 / 2 of the
+  // per-feature term is added to the logits (the in-chunk scores cannot take it from a merged state,
+  // and with it the features that matter are the ones near 1, where fp16 is precise), the two feature
+  // halves share one shift, and the chunk's features are also written in fp16, [B*H][Lpad][256].
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   KvMisc* misc = reinterpret_cast<KvMisc*>(sm + KvSmem::MISC);
+  float* fa2 = reinterpret_cast<float*>(sm + KvSmem::FA2);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
   const int g = pool == FSHARP_POOL_PER_BH ? bh : h;
@@ -89,6 +94,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   // constant tile written by the block itself: the second 64-row block of [V | 1]^T, whose
   // first row is the 1 and whose other rows are zero
   for (int i = threadIdx.x; i < TILE_BYTES / 16; i += TC_THREADS) reinterpret_cast<uint4*>(sm + KvSmem::ONES)[i] = make_uint4(0, 0, 0, 0);
+  if (phik16 != nullptr && threadIdx.x < TC_M) fa2[threadIdx.x] = 0.5f * reinterpret_cast<const float*>(img + IMG_A2)[threadIdx.x];
   __syncthreads();
   if (threadIdx.x < TILE)
     *reinterpret_cast<__nv_bfloat16*>(sm + KvSmem::ONES + sw128_offset(threadIdx.x, 0)) = __float2bfloat16(1.f);
@@ -219,6 +225,16 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       tmem_wait_ld();
       tcgen05_fence_before();
       mbar_arrive(&misc->logits_free);
+      if (phik16 != nullptr) {
+#pragma unroll
+        for (int i = 0; i < 128; i += 4) {
+          const float4 a4 = *reinterpret_cast<const float4*>(fa2 + hf * 128 + i);
+          v[i] = __float_as_uint(__uint_as_float(v[i]) + a4.x);
+          v[i + 1] = __float_as_uint(__uint_as_float(v[i + 1]) + a4.y);
+          v[i + 2] = __float_as_uint(__uint_as_float(v[i + 2]) + a4.z);
+          v[i + 3] = __float_as_uint(__uint_as_float(v[i + 3]) + a4.w);
+        }
+      }
       const bool valid = (tile0 + it) * TILE + row < L;
       if (it == 0) {
         // first tile: no shift yet, take the exact maximum of this half of the tile
@@ -228,9 +244,15 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         float mx = valid ? fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])) + cj : -INFINITY;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        if (lane == 0) atomicMax(&tmax[3], f2ord(mx));
-        named_bar_sync(1 + hf, HALF_THREADS);
-        s = ord2f(tmax[3]);
+        if (phik16 != nullptr) {              // one shift for both halves
+          if (lane == 0) atomicMax(&misc->tile_max[0][3], f2ord(mx));
+          named_bar_sync(3, EPI_THREADS);
+          s = ord2f(misc->tile_max[0][3]);
+        } else {
+          if (lane == 0) atomicMax(&tmax[3], f2ord(mx));
+          named_bar_sync(1 + hf, HALF_THREADS);
+          s = ord2f(tmax[3]);
+        }
       } else {
         if (!mbar_wait(&misc->phi_free[hf], (it - 1) & 1, abortp, status, false)) { alive = false; break; }
       }
@@ -242,14 +264,22 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 #pragma unroll
         for (int c = 0; c < 16; c++) {
           uint32_t p[4];
+          uint32_t g16[4];
 #pragma unroll
           for (int j = 0; j < 4; j++) {
             const float f0 = __uint_as_float(v[c * 8 + 2 * j]) + rc, f1 = __uint_as_float(v[c * 8 + 2 * j + 1]) + rc;
             mxp[j] = fmaxf(mxp[j], fmaxf(f0, f1));
-            p[j] = pack_bf16(ex2(f0), ex2(f1));
+            const float e0 = ex2(f0), e1 = ex2(f1);
+            p[j] = pack_bf16(e0, e1);
+            if (phik16 != nullptr) g16[j] = pack_f16(e0, e1);
           }
           if (!valid) p[0] = p[1] = p[2] = p[3] = 0u;
           *reinterpret_cast<uint4*>(prow + (c >> 3) * TILE_BYTES + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
+          if (phik16 != nullptr) {
+            if (!valid) g16[0] = g16[1] = g16[2] = g16[3] = 0u;
+            *reinterpret_cast<uint4*>(phik16 + ((size_t)bh * Lpad + (size_t)(tile0 + it) * TILE + row) * TC_M + hf * 128 + c * 8) =
+                make_uint4(g16[0], g16[1], g16[2], g16[3]);
+          }
         }
         if (pass == 1) break;
         rel = valid ? fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])) : -INFINITY;
@@ -637,6 +667,9 @@ int fs_tc_rowterm(fsharp_ctx* ctx, const void* K, const fsharp_dims* dm, const u
 size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
 int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
                 const float* prep, void* Y, WsAlloc* ws);
+int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
+                   const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax,
+                   __half* phik16);
 
 constexpr int MAX_KEY_SPLIT = 64;
 
@@ -647,6 +680,28 @@ size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
          ws_round(BH * MAX_KEY_SPLIT * TC_M * TC_NV * 4) + 2 * ws_round(BH * MAX_KEY_SPLIT * 2 * 4) +
          ws_round(BH * (size_t)((dm->Lk + TILE - 1) / TILE) * TILE * 4) +
          ws_round(BH * TC_NV * TC_M * 2);
+}
+
+// Key side: the per-key quadratic term, then the feature / contraction kernel.  crow: [B*H][Lpad] floats,
+// Lpad = ceil(Lk / 128) * 128; partial: [B*H][nsplit][80][256] floats; shifts, pmax: [B*H][nsplit][2], pmax
+// zeroed by the caller; phik16 (may be null): fp16 [B*H][Lpad][256], written when tiles_per_split == 1.
+int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
+                   const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax,
+                   __half* phik16) {
+  const int B = dm->B, H = dm->H, Lk = dm->Lk;
+  const int Lpad = (Lk + TILE - 1) / TILE * TILE;
+  if (phik16 != nullptr && tiles_per_split != 1) return FSHARP_E_BADARG;
+  FS_TRY(fs_tc_rowterm(ctx, K, dm, images, flags, Lpad, tiles_per_split, nsplit, crow));
+  CUtensorMap tmK, tmV;
+  FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, Lk, dm->d), B, H, Lk, dm->d));
+  FS_TRY(tchost::make_map_tokens(&tmV, V, fs_addr(dm->v_stride, H, Lk, dm->dv), B, H, Lk, dm->dv));
+  FS_CUDA_OK(cudaFuncSetAttribute(tc_kv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KvSmem::TOTAL + 1024));
+  FS_TIME_BEGIN(ctx, FS_K_TC_KV);
+  tc_kv_kernel<<<dim3(nsplit, B * H), TC_THREADS, KvSmem::TOTAL + 1024, ctx->stream>>>(
+      tmK, tmV, images, crow, H, dm->pool, Lk, Lpad, tiles_per_split, nsplit, partial, shifts, pmax, phik16, ctx->d_status);
+  FS_TIME_END(ctx);
+  FS_LAUNCH_CHECK(ctx);
+  return FSHARP_OK;
 }
 
 int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
@@ -667,22 +722,13 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * MAX_KEY_SPLIT * 2 * sizeof(int), ctx->stream));
   const int Lpad = ktiles * TILE;
   float* crow = ws->take<float>((size_t)BH * Lpad);
-  FS_TRY(fs_tc_rowterm(ctx, K, dm, images, flags, Lpad, tps, nsplit, crow));
   __half* kvt = ws->take<__half>((size_t)BH * TC_NV * TC_M);
+  FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, tps, nsplit, crow, partial, shifts, pmax, nullptr));
 
-  CUtensorMap tmK, tmV, tmQ, tmKVt;
-  FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, Lk, dm->d), B, H, Lk, dm->d));
-  FS_TRY(tchost::make_map_tokens(&tmV, V, fs_addr(dm->v_stride, H, Lk, dm->dv), B, H, Lk, dm->dv));
+  CUtensorMap tmQ, tmKVt;
   FS_TRY(tchost::make_map_tokens(&tmQ, Q, fs_addr(dm->q_stride, H, Lq, dm->d), B, H, Lq, dm->d));
   FS_TRY(tchost::make_map_kvt(&tmKVt, kvt, BH));
-
-  FS_CUDA_OK(cudaFuncSetAttribute(tc_kv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KvSmem::TOTAL + 1024));
   FS_CUDA_OK(cudaFuncSetAttribute(tc_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OutSmem::TOTAL + 1024));
-  FS_TIME_BEGIN(ctx, FS_K_TC_KV);
-  tc_kv_kernel<<<dim3(nsplit, BH), TC_THREADS, KvSmem::TOTAL + 1024, ctx->stream>>>(
-      tmK, tmV, images, crow, H, dm->pool, Lk, Lpad, tps, nsplit, partial, shifts, pmax, ctx->d_status);
-  FS_TIME_END(ctx);
-  FS_LAUNCH_CHECK(ctx);
   FS_TIME_BEGIN(ctx, FS_K_TC_MERGE);
   tc_merge_kernel<<<dim3(MERGE_SLICES, BH), 256, 0, ctx->stream>>>(partial, shifts, pmax, nsplit, images, H, dm->pool, kvt);
   FS_TIME_END(ctx);

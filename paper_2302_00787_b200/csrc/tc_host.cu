@@ -6,6 +6,10 @@
 using namespace tcl;
 
 size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
+int fs_tc_causal_supported(const fsharp_dims* dm, int chunk);
+size_t fs_tc_causal_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
+int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
+                 const float* prep, void* Y, WsAlloc* ws);
 int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
                 const float* prep, void* Y, WsAlloc* ws);
 
@@ -110,6 +114,20 @@ int make_map_kvt(CUtensorMap* map, const void* base, int BH) {
   return r == CUDA_SUCCESS ? FSHARP_OK : FSHARP_E_CUDA;
 }
 
+// fp16 features [BH, Lpad, 256] -> 3-D map (feature, token, bh), box 64 x 128 x 1, 128-byte swizzle.
+int make_map_feat(CUtensorMap* map, const void* base, int BH, int Lpad) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return FSHARP_E_CUDA;
+  cuuint64_t dims[3] = {(cuuint64_t)TC_M, (cuuint64_t)Lpad, (cuuint64_t)BH};
+  cuuint64_t strides[2] = {(cuuint64_t)TC_M * 2, (cuuint64_t)TC_M * 2 * (cuuint64_t)Lpad};
+  cuuint32_t box[3] = {64, (cuuint32_t)TILE, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? FSHARP_OK : FSHARP_E_CUDA;
+}
+
 }  // namespace tchost
 
 int fs_tc_prep(fsharp_ctx* ctx, const float* prep, int G, float qk_scale, uint8_t* images, int* flags) {
@@ -126,20 +144,19 @@ int fs_tc_supported(const fsharp_dims* dm, int dtype, int causal, int chunk, flo
   (void)qk_scale;
   if (dtype != FSHARP_BF16) return 0;
   if (dm->d != TC_D || dm->dv != TC_DV || dm->M != TC_M) return 0;
-  if (causal) return 0;
   if (dm->Lq <= 0 || dm->Lk <= 0) return 0;
+  if (causal) return fs_tc_causal_supported(dm, chunk);
   return 1;
 }
 
 size_t fs_tc_attend_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm, int causal, int chunk) {
-  (void)causal;
   (void)chunk;
-  return fs_tc_bidir_scratch_bytes(ctx, dm);
+  return causal ? fs_tc_causal_scratch_bytes(ctx, dm) : fs_tc_bidir_scratch_bytes(ctx, dm);
 }
 
 int fs_tc_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, int causal,
                  int chunk, float qk_scale, const float* prep, void* Y, WsAlloc* ws) {
   (void)chunk;
-  if (causal) return FSHARP_E_SHAPE;
+  if (causal) return fs_tc_causal(ctx, Q, K, V, dm, qk_scale, prep, Y, ws);
   return fs_tc_bidir(ctx, Q, K, V, dm, qk_scale, prep, Y, ws);
 }
