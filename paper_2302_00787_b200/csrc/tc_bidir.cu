@@ -49,6 +49,7 @@ struct KvMisc {
   uint32_t tmem_base;
   int abort_flag;
   int tile_max[2][4];     // per half: [0..2] rotating slots of the per-tile maximum, [3] the first tile's
+  int chunk_max[3];       // causal use: rotating slots of the exact maximum of a whole tile
 };
 static_assert(sizeof(KvMisc) <= 256, "misc block");
 
@@ -57,13 +58,13 @@ constexpr int HALF_THREADS = EPI_THREADS / 2;
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-             const uint8_t* __restrict__ images, const float* __restrict__ crow, int H, int pool, int L, int Lpad,
+             const __grid_constant__ CUtensorMap tmPhi, const uint8_t* __restrict__ images, const float* __restrict__ crow, int H, int pool, int L, int Lpad,
              int tiles_per_split, int nsplit, float* __restrict__ partial, float* __restrict__ shifts,
-             int* __restrict__ pmax, __half* __restrict__ phik16, int* __restrict__ status) {
-  // phik16 != nullptr (causal use: one 128-key chunk per block): the key side's share a2 / 2 of the
-  // per-feature term is added to the logits (the in-chunk scores cannot take it from a merged state,
-  // and with it the features that matter are the ones near 1, where fp16 is precise), the two feature
-  // halves share one shift, and the chunk's features are also written in fp16, [B*H][Lpad][256].
+             int* __restrict__ pmax, int per_tile, int* __restrict__ status) {
+  // per_tile != 0 (causal use: every 128-key tile is a chunk with a state, a shift and a partial of its
+  // own, numbered by its tile index): the key side's share a2 / 2 of the per-feature term is added to the
+  // logits (the in-chunk scores cannot take it from a merged state), the two feature halves share one
+  // shift, and the tile of features, as the MMA reads it, is also stored through tmPhi, bf16 [B*H][Lpad][256].
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   KvMisc* misc = reinterpret_cast<KvMisc*>(sm + KvSmem::MISC);
@@ -85,6 +86,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       mbar_init(&misc->phi_free[i], 1);
       for (int j = 0; j < 4; j++) misc->tile_max[i][j] = f2ord(-INFINITY);
     }
+    for (int j = 0; j < 3; j++) misc->chunk_max[j] = f2ord(-INFINITY);
     mbar_init(&misc->logits_full, 1);
     mbar_init(&misc->logits_free, EPI_THREADS);
     mbar_init(&misc->const_bar, 1);
@@ -94,7 +96,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   // constant tile written by the block itself: the second 64-row block of [V | 1]^T, whose
   // first row is the 1 and whose other rows are zero
   for (int i = threadIdx.x; i < TILE_BYTES / 16; i += TC_THREADS) reinterpret_cast<uint4*>(sm + KvSmem::ONES)[i] = make_uint4(0, 0, 0, 0);
-  if (phik16 != nullptr && threadIdx.x < TC_M) fa2[threadIdx.x] = 0.5f * reinterpret_cast<const float*>(img + IMG_A2)[threadIdx.x];
+  if (per_tile && threadIdx.x < TC_M) fa2[threadIdx.x] = 0.5f * reinterpret_cast<const float*>(img + IMG_A2)[threadIdx.x];
   __syncthreads();
   if (threadIdx.x < TILE)
     *reinterpret_cast<__nv_bfloat16*>(sm + KvSmem::ONES + sw128_offset(threadIdx.x, 0)) = __float2bfloat16(1.f);
@@ -178,19 +180,26 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           issue_logits(st ^ 1);
         }
         const uint64_t dV = st ? dVst1 : dVst0;
-        const uint32_t acc0 = it > 0 ? 1u : 0u;
+        const uint32_t acc0 = (it > 0 && !per_tile) ? 1u : 0u;      // causal use: every tile starts afresh
 #pragma unroll 1
         for (int hh = 0; hh < 2 && ok; hh++) {
           if (!mbar_wait(&misc->phi_full[hh], it & 1, abortp, status)) { ok = false; break; }
           tcgen05_fence_after();
+          if (per_tile) {                 // the half tile also goes out as it is (two 64-feature blocks)
+            tma_store_3d(&tmPhi, sm + KvSmem::PHI + (2 * hh) * TILE_BYTES, (2 * hh) * 64, (tile0 + it) * TILE, bh);
+            tma_store_3d(&tmPhi, sm + KvSmem::PHI + (2 * hh + 1) * TILE_BYTES, (2 * hh + 1) * 64, (tile0 + it) * TILE, bh);
+            bulk_commit();
+          }
 #pragma unroll 2
           for (int k = 0; k < TILE / 16; k++)
             mma_bf16(tmem + KV_COL_ACC + hh * 128, desc_advance(dV, k * 2048),
                      desc_advance(dPhi, hh * 2 * TILE_BYTES + k * 2048), ID_KV, k > 0 ? 1u : acc0);
+          if (per_tile) bulk_wait_read0();       // the store has read the half tile: it may be overwritten
           mma_commit(&misc->phi_free[hh]);
         }
         mma_commit(&misc->empty[st]);
       }
+      if (per_tile) bulk_wait0();
     }
   }
   } else {
@@ -209,6 +218,35 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     float s = 0.f;
     float cj = ntiles > 0 ? cptr[0] : 0.f;
     bool alive = true;
+    // accumulator of this half -> partial `slot` (the contraction that feeds it has completed)
+    auto write_partial = [&](size_t slot) {
+      __syncwarp();
+      tcgen05_fence_after();
+      float* out = partial + (slot * TC_NV + row) * TC_M + hf * 128;
+      float amax = 0.f;
+      if (q * 32 < TC_NV) {                 // warp-uniform: lanes 0..79 carry data
+#pragma unroll
+        for (int c = 0; c < 8; c++) {
+          uint32_t a[16];
+          tmem_ld16(acc_addr + c * 16, a);
+          tmem_wait_ld();
+          if (row < TC_NV) {
+#pragma unroll
+            for (int j = 0; j < 16; j++)
+              if (row <= TC_DV) amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
+#pragma unroll
+            for (int j = 0; j < 4; j++)
+              reinterpret_cast<uint4*>(out + c * 16)[j] = make_uint4(a[4 * j], a[4 * j + 1], a[4 * j + 2], a[4 * j + 3]);
+          }
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+      // non-negative floats order like their bit patterns
+      if (lane == 0) atomicMax(&pmax[slot * 2 + hf], __float_as_int(amax));
+      if (q == 0 && lane == 0) shifts[slot * 2 + hf] = s;
+      tcgen05_fence_before();
+    };
     for (int it = 0; it < ntiles && alive; it++) {
       const float cnext = it + 1 < ntiles ? cptr[(size_t)(it + 1) * TILE] : 0.f;     // in flight during this tile
       if (!mbar_wait(&misc->logits_full, it & 1, abortp, status, false)) { alive = false; break; }
@@ -225,7 +263,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       tmem_wait_ld();
       tcgen05_fence_before();
       mbar_arrive(&misc->logits_free);
-      if (phik16 != nullptr) {
+      if (per_tile) {
 #pragma unroll
         for (int i = 0; i < 128; i += 4) {
           const float4 a4 = *reinterpret_cast<const float4*>(fa2 + hf * 128 + i);
@@ -236,23 +274,26 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         }
       }
       const bool valid = (tile0 + it) * TILE + row < L;
-      if (it == 0) {
-        // first tile: no shift yet, take the exact maximum of this half of the tile
+      if (it == 0 || per_tile) {
+        // first tile (causal use: every tile): no shift yet, take the exact maximum of this half of the tile
         float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
         for (int i = 0; i < 128; i++) mxp[i & 3] = fmaxf(mxp[i & 3], __uint_as_float(v[i]));
-        float mx = valid ? fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])) + cj : -INFINITY;
+        const float hm = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
+        float mx = valid ? hm + cj : -INFINITY;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        if (phik16 != nullptr) {              // one shift for both halves
-          if (lane == 0) atomicMax(&misc->tile_max[0][3], f2ord(mx));
+        if (per_tile) {              // one shift for both halves
+          if (lane == 0) atomicMax(&misc->chunk_max[it % 3], f2ord(mx));
+          if (threadIdx.x == 0) misc->chunk_max[(it + 1) % 3] = f2ord(-INFINITY);   // next tile's slot; idle since tile it-2
           named_bar_sync(3, EPI_THREADS);
-          s = ord2f(misc->tile_max[0][3]);
+          s = ord2f(misc->chunk_max[it % 3]);
         } else {
           if (lane == 0) atomicMax(&tmax[3], f2ord(mx));
           named_bar_sync(1 + hf, HALF_THREADS);
           s = ord2f(tmax[3]);
         }
+        if (it > 0 && !mbar_wait(&misc->phi_free[hf], (it - 1) & 1, abortp, status, false)) { alive = false; break; }
       } else {
         if (!mbar_wait(&misc->phi_free[hf], (it - 1) & 1, abortp, status, false)) { alive = false; break; }
       }
@@ -264,22 +305,15 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 #pragma unroll
         for (int c = 0; c < 16; c++) {
           uint32_t p[4];
-          uint32_t g16[4];
 #pragma unroll
           for (int j = 0; j < 4; j++) {
             const float f0 = __uint_as_float(v[c * 8 + 2 * j]) + rc, f1 = __uint_as_float(v[c * 8 + 2 * j + 1]) + rc;
             mxp[j] = fmaxf(mxp[j], fmaxf(f0, f1));
             const float e0 = ex2(f0), e1 = ex2(f1);
             p[j] = pack_bf16(e0, e1);
-            if (phik16 != nullptr) g16[j] = pack_f16(e0, e1);
           }
           if (!valid) p[0] = p[1] = p[2] = p[3] = 0u;
           *reinterpret_cast<uint4*>(prow + (c >> 3) * TILE_BYTES + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
-          if (phik16 != nullptr) {
-            if (!valid) g16[0] = g16[1] = g16[2] = g16[3] = 0u;
-            *reinterpret_cast<uint4*>(phik16 + ((size_t)bh * Lpad + (size_t)(tile0 + it) * TILE + row) * TC_M + hf * 128 + c * 8) =
-                make_uint4(g16[0], g16[1], g16[2], g16[3]);
-          }
         }
         if (pass == 1) break;
         rel = valid ? fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])) : -INFINITY;
@@ -311,35 +345,14 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       tcgen05_fence_before();
       mbar_arrive(&misc->phi_full[hf]);
       cj = cnext;
+      if (per_tile) {                // causal use: the tile's state leaves now, numbered by its tile index
+        if (!mbar_wait(&misc->phi_free[hf], it & 1, abortp, status, false)) { alive = false; break; }
+        write_partial((size_t)bh * total_tiles + tile0 + it);
+      }
     }
     // write this split's partial [V | 1]^T phi_h (fp32, rows 0..79), its shift and its largest magnitude
-    if (alive && ntiles > 0 && mbar_wait(&misc->phi_free[hf], (ntiles - 1) & 1, abortp, status, false)) {
-      __syncwarp();
-      tcgen05_fence_after();
-      float* out = partial + (((size_t)bh * nsplit + split) * TC_NV + row) * TC_M + hf * 128;
-      float amax = 0.f;
-      if (q * 32 < TC_NV) {                 // warp-uniform: lanes 0..79 carry data
-#pragma unroll
-        for (int c = 0; c < 8; c++) {
-          uint32_t a[16];
-          tmem_ld16(acc_addr + c * 16, a);
-          tmem_wait_ld();
-          if (row < TC_NV) {
-#pragma unroll
-            for (int j = 0; j < 16; j++)
-              if (row <= TC_DV) amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
-#pragma unroll
-            for (int j = 0; j < 4; j++)
-              reinterpret_cast<uint4*>(out + c * 16)[j] = make_uint4(a[4 * j], a[4 * j + 1], a[4 * j + 2], a[4 * j + 3]);
-          }
-        }
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-      // non-negative floats order like their bit patterns
-      if (lane == 0) atomicMax(&pmax[((size_t)bh * nsplit + split) * 2 + hf], __float_as_int(amax));
-      if (q == 0 && lane == 0) shifts[((size_t)bh * nsplit + split) * 2 + hf] = s;
-    }
+    if (alive && ntiles > 0 && !per_tile && mbar_wait(&misc->phi_free[hf], (ntiles - 1) & 1, abortp, status, false))
+      write_partial((size_t)bh * nsplit + split);
   }
   tcgen05_fence_before();
   __syncthreads();
@@ -659,7 +672,8 @@ int pick_split(int units, int tiles, int sms, int max_split, int* tiles_per_spli
 // ------------------------------------------------------------------------------------------
 namespace tchost {
 int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int H, int L, int inner);
-int make_map_kvt(CUtensorMap* map, const void* base, int BH);
+int make_map_kvt(CUtensorMap* map, const void* base, int BH, int bf16);
+int make_map_feat(CUtensorMap* map, const void* base, int BH, int Lpad);
 }  // namespace tchost
 int fs_tc_prep(fsharp_ctx* ctx, const float* prep, int G, float qk_scale, uint8_t* images, int* flags);
 int fs_tc_rowterm(fsharp_ctx* ctx, const void* K, const fsharp_dims* dm, const uint8_t* images, const int* flags, int Lpad,
@@ -669,7 +683,7 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
                 const float* prep, void* Y, WsAlloc* ws);
 int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                    const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax,
-                   __half* phik16);
+                   __nv_bfloat16* phik);
 
 constexpr int MAX_KEY_SPLIT = 64;
 
@@ -684,21 +698,24 @@ size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
 
 // Key side: the per-key quadratic term, then the feature / contraction kernel.  crow: [B*H][Lpad] floats,
 // Lpad = ceil(Lk / 128) * 128; partial: [B*H][nsplit][80][256] floats; shifts, pmax: [B*H][nsplit][2], pmax
-// zeroed by the caller; phik16 (may be null): fp16 [B*H][Lpad][256], written when tiles_per_split == 1.
+// zeroed by the caller.  phik (may be null; causal use): bf16 [B*H][Lpad][256]; with it every 128-key tile
+// is a chunk of its own and partial, shifts, pmax are indexed by tile: [B*H][ceil(Lk / 128)] entries.
 int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                    const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax,
-                   __half* phik16) {
+                   __nv_bfloat16* phik) {
   const int B = dm->B, H = dm->H, Lk = dm->Lk;
   const int Lpad = (Lk + TILE - 1) / TILE * TILE;
-  if (phik16 != nullptr && tiles_per_split != 1) return FSHARP_E_BADARG;
   FS_TRY(fs_tc_rowterm(ctx, K, dm, images, flags, Lpad, tiles_per_split, nsplit, crow));
-  CUtensorMap tmK, tmV;
+  CUtensorMap tmK, tmV, tmPhi;
   FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, Lk, dm->d), B, H, Lk, dm->d));
   FS_TRY(tchost::make_map_tokens(&tmV, V, fs_addr(dm->v_stride, H, Lk, dm->dv), B, H, Lk, dm->dv));
+  if (phik != nullptr) FS_TRY(tchost::make_map_feat(&tmPhi, phik, B * H, Lpad));
+  else tmPhi = tmK;                       // not used
   FS_CUDA_OK(cudaFuncSetAttribute(tc_kv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KvSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_KV);
   tc_kv_kernel<<<dim3(nsplit, B * H), TC_THREADS, KvSmem::TOTAL + 1024, ctx->stream>>>(
-      tmK, tmV, images, crow, H, dm->pool, Lk, Lpad, tiles_per_split, nsplit, partial, shifts, pmax, phik16, ctx->d_status);
+      tmK, tmV, tmPhi, images, crow, H, dm->pool, Lk, Lpad, tiles_per_split, nsplit, partial, shifts, pmax,
+      phik != nullptr ? 1 : 0, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;
@@ -727,7 +744,7 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
 
   CUtensorMap tmQ, tmKVt;
   FS_TRY(tchost::make_map_tokens(&tmQ, Q, fs_addr(dm->q_stride, H, Lq, dm->d), B, H, Lq, dm->d));
-  FS_TRY(tchost::make_map_kvt(&tmKVt, kvt, BH));
+  FS_TRY(tchost::make_map_kvt(&tmKVt, kvt, BH, 0));
   FS_CUDA_OK(cudaFuncSetAttribute(tc_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OutSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_MERGE);
   tc_merge_kernel<<<dim3(MERGE_SLICES, BH), 256, 0, ctx->stream>>>(partial, shifts, pmax, nsplit, images, H, dm->pool, kvt);

@@ -4,13 +4,13 @@
 //   Y_c = [ phiQ_c P_c  +  tril(phiQ_c phiK_c^T) [V_c | 1] ]  (numerator | denominator),
 //   P_c = sum over earlier chunks c' of phiK_c'^T [V_c' | 1].
 //
-//   tc_kv_kernel (tc_bidir.cu), one chunk per block: chunk states and fp16 key features
-//   tc_featq_kernel:          fp16 query features, each row shifted by its own maximum
-//   tc_causal_prefix_kernel:  exclusive scan of the chunk states -> fp16 prefixes P_c, every
+//   tc_kv_kernel (tc_bidir.cu), every tile a chunk: chunk states and the chunk's bf16 key features
+//   tc_featq_kernel:          bf16 query features, each row shifted by its own maximum
+//   tc_causal_prefix_kernel:  exclusive scan of the chunk states -> bf16 prefixes P_c, every
 //                             chunk brought to a scale of its own that also weighs the in-chunk term
-//   tc_causal_out_kernel:     per chunk  D = phiQ P_c^T (fp16 MMA), S = phiQ phiK^T (fp16 MMA, TMEM),
+//   tc_causal_out_kernel:     per chunk  D = phiQ P_c^T, S = phiQ phiK^T (TMEM),
 //                             S masked, scaled, rounded to bf16 into shared memory,
-//                             D += S V (bf16 MMA), denominator += row sums of S, Y = num / den
+//                             D += S V, denominator += row sums of S, Y = num / den
 #include <cuda_fp16.h>
 
 #include "common.cuh"
@@ -27,7 +27,8 @@ namespace {
 // ------------------------------------------------------------------------------------------
 constexpr int FQ_STAGES = 3;
 struct FqSmem {
-  static constexpr uint32_t X0 = 0, W = FQ_STAGES * TILE_BYTES, WLO = W + IMG_W_BYTES, ROWMAX = WLO + IMG_W_BYTES,
+  static constexpr uint32_t X0 = 0, W = FQ_STAGES * TILE_BYTES, WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES,
+                            ROWMAX = PHI + 4 * TILE_BYTES,
                             AH = ROWMAX + 2 * 2 * TILE * 4, MISC = AH + TC_M * 4, TOTAL = MISC + 256;
 };
 struct FqMisc {
@@ -37,8 +38,8 @@ struct FqMisc {
 };
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
-tc_featq_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict__ images, int H, int pool, int L, int Lpad,
-                int tiles_per_split, __half* __restrict__ phiq16, int* __restrict__ status) {
+tc_featq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmPhi,
+                const uint8_t* __restrict__ images, int H, int pool, int L, int tiles_per_split, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   FqMisc* misc = reinterpret_cast<FqMisc*>(sm + FqSmem::MISC);
@@ -154,16 +155,27 @@ tc_featq_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restri
       rm[hf * TILE + row] = mx;
       named_bar_sync(1, EPI_THREADS);
       mx = fmaxf(mx, rm[(hf ^ 1) * TILE + row]);
-      __half* dst = phiq16 + ((size_t)bh * Lpad + (size_t)(tile0 + it) * TILE + row) * TC_M + hf * 128;
+      // the tile goes to shared memory in the layout of an MMA operand and leaves as one TMA store per
+      // 64-feature block; thread 0 waits for the store to have read the tile before the next one is written
+      uint8_t* prow = sm + FqSmem::PHI + hf * 2 * TILE_BYTES + row * 128;
 #pragma unroll
       for (int c = 0; c < 16; c++) {
         uint32_t p[4];
 #pragma unroll
         for (int j = 0; j < 4; j++)
-          p[j] = pack_f16(ex2(__uint_as_float(v[c * 8 + 2 * j]) - mx), ex2(__uint_as_float(v[c * 8 + 2 * j + 1]) - mx));
-        *reinterpret_cast<uint4*>(dst + c * 8) = make_uint4(p[0], p[1], p[2], p[3]);
+          p[j] = pack_bf16(ex2(__uint_as_float(v[c * 8 + 2 * j]) - mx), ex2(__uint_as_float(v[c * 8 + 2 * j + 1]) - mx));
+        *reinterpret_cast<uint4*>(prow + (c >> 3) * TILE_BYTES + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
+      }
+      fence_proxy_async_smem();
+      named_bar_sync(2, EPI_THREADS);
+      if (threadIdx.x == 0) {
+#pragma unroll
+        for (int fb = 0; fb < TC_M / 64; fb++) tma_store_3d(&tmPhi, sm + FqSmem::PHI + fb * TILE_BYTES, fb * 64, (tile0 + it) * TILE, bh);
+        bulk_commit();
+        bulk_wait_read0();
       }
     }
+    if (threadIdx.x == 0) bulk_wait0();
   }
   tcgen05_fence_before();
   __syncthreads();
@@ -178,15 +190,15 @@ tc_featq_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restri
 // ------------------------------------------------------------------------------------------
 // state[bh][c]: [80][256] fp32, chunk c's [V | 1]^T phiK with phiK = 2^(exponent - s_c); pmax its largest
 // magnitude.  For every chunk c the kernel writes
-//   prefix[bh][c] = alpha_c 2^(-e_c) sum_{c' < c} 2^(s_c' - sigma_c) state[c']   (fp16),
+//   prefix[bh][c] = alpha_c 2^(-e_c) sum_{c' < c} 2^(s_c' - sigma_c) state[c']   (bf16),
 //   beta[bh][c],
-// where sigma_c = max_{c' < c} s_c', e_c brings the sum into fp16 range, and (alpha_c, beta_c) <= 1 put the
+// where sigma_c = max_{c' < c} s_c', e_c brings the sum to order 2^14, and (alpha_c, beta_c) <= 1 put the
 // prefix term (true scale 2^(sigma_c + e_c)) and the in-chunk term (true scale 2^(s_c)) on one scale.
 constexpr int PFX_SLICES = 10;               // 80 x 256 elements = 10 x 256 threads x 8
 constexpr int PFX_MAXCH = 1024;
 __global__ void __launch_bounds__(256)
 tc_causal_prefix_kernel(const float* __restrict__ state, const float* __restrict__ shifts, const int* __restrict__ pmax,
-                        int nch, __half* __restrict__ prefix, float* __restrict__ beta) {
+                        int nch, __nv_bfloat16* __restrict__ prefix, float* __restrict__ beta) {
   __shared__ float up[PFX_MAXCH], add[PFX_MAXCH], oscale[PFX_MAXCH];
   const int bh = blockIdx.y;
   if (threadIdx.x == 0) {
@@ -215,7 +227,7 @@ tc_causal_prefix_kernel(const float* __restrict__ state, const float* __restrict
   __syncthreads();
   // thread t of slice x owns rows 8x .. 8x+7 of column t
   const float* sb = state + (size_t)bh * nch * TC_NV * TC_M;
-  __half* pb = prefix + (size_t)bh * nch * TC_NV * TC_M;
+  __nv_bfloat16* pb = prefix + (size_t)bh * nch * TC_NV * TC_M;
   float R[8];
 #pragma unroll
   for (int u = 0; u < 8; u++) R[u] = 0.f;
@@ -230,7 +242,7 @@ tc_causal_prefix_kernel(const float* __restrict__ state, const float* __restrict
 #pragma unroll
     for (int u = 0; u < 8; u++) {
       const int n = blockIdx.x * 8 + u;
-      pb[((size_t)c * TC_NV + n) * TC_M + threadIdx.x] = __float2half_rn(R[u] * os);
+      pb[((size_t)c * TC_NV + n) * TC_M + threadIdx.x] = __float2bfloat16_rn(R[u] * os);
       R[u] = fmaf(R[u], upc, adc * kv[u]);
     }
   }
@@ -315,8 +327,8 @@ tc_causal_out_kernel(const __grid_constant__ CUtensorMap tmPhiQ, const __grid_co
       }
     } else if (warp == WARP_MMA) {
       if (lane == 0) {
-        constexpr uint32_t ID_INTER = idesc_f16(128, TC_NV, 0, 0);      // phiQ P^T
-        constexpr uint32_t ID_SCORE = idesc_f16(128, 128, 0, 0);        // phiQ phiK^T
+        constexpr uint32_t ID_INTER = idesc_bf16(128, TC_NV, 0, 0);      // phiQ P^T
+        constexpr uint32_t ID_SCORE = idesc_bf16(128, 128, 0, 0);        // phiQ phiK^T
         constexpr uint32_t ID_SV = idesc_bf16(128, TC_DV, 0, 1);        // S V (V with the value index contiguous)
         const uint64_t dQ = smem_desc(smem_u32(sm + CoSmem::PHIQ), 16, 1024, SWZ_128B);
         const uint64_t dK = smem_desc(smem_u32(sm + CoSmem::PHIK), 16, 1024, SWZ_128B);
@@ -434,13 +446,13 @@ tc_causal_out_kernel(const __grid_constant__ CUtensorMap tmPhiQ, const __grid_co
 // ------------------------------------------------------------------------------------------
 namespace tchost {
 int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int H, int L, int inner);
-int make_map_kvt(CUtensorMap* map, const void* base, int BH);
+int make_map_kvt(CUtensorMap* map, const void* base, int BH, int bf16);
 int make_map_feat(CUtensorMap* map, const void* base, int BH, int Lpad);
 }  // namespace tchost
 int fs_tc_prep(fsharp_ctx* ctx, const float* prep, int G, float qk_scale, uint8_t* images, int* flags);
 int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                    const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax,
-                   __half* phik16);
+                   __nv_bfloat16* phik);
 int fs_tc_causal_supported(const fsharp_dims* dm, int chunk);
 size_t fs_tc_causal_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
 int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
@@ -472,14 +484,12 @@ int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, c
   float* shifts = ws->take<float>((size_t)BH * nch * 2);
   int* pmax = ws->take<int>((size_t)BH * nch * 2);
   float* crow = ws->take<float>((size_t)BH * Lpad);
-  __half* phik16 = ws->take<__half>((size_t)BH * Lpad * TC_M);
-  __half* phiq16 = ws->take<__half>((size_t)BH * Lpad * TC_M);
-  __half* prefix = ws->take<__half>((size_t)BH * nch * TC_NV * TC_M);
+  __nv_bfloat16* phik16 = ws->take<__nv_bfloat16>((size_t)BH * Lpad * TC_M);
+  __nv_bfloat16* phiq16 = ws->take<__nv_bfloat16>((size_t)BH * Lpad * TC_M);
+  __nv_bfloat16* prefix = ws->take<__nv_bfloat16>((size_t)BH * nch * TC_NV * TC_M);
   float* beta = ws->take<float>((size_t)BH * nch);
   FS_TRY(fs_tc_prep(ctx, prep, G, qk_scale, images, flags));
   FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * nch * 2 * sizeof(int), ctx->stream));
-  // key side, one chunk per block: chunk states and fp16 key features
-  FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, 1, nch, crow, state, shifts, pmax, phik16));
 
   // query features
   CUtensorMap tmQ, tmPhiQ, tmPhiK, tmPfx, tmV;
@@ -487,7 +497,7 @@ int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, c
   FS_TRY(tchost::make_map_tokens(&tmV, V, fs_addr(dm->v_stride, H, L, dm->dv), B, H, L, dm->dv));
   FS_TRY(tchost::make_map_feat(&tmPhiQ, phiq16, BH, Lpad));
   FS_TRY(tchost::make_map_feat(&tmPhiK, phik16, BH, Lpad));
-  FS_TRY(tchost::make_map_kvt(&tmPfx, prefix, BH * nch));
+  FS_TRY(tchost::make_map_kvt(&tmPfx, prefix, BH * nch, 1));
   // blocks of equal tile count: (waves of blocks) x (tiles per block + fill and drain)
   auto split = [&](int overhead, int* per) {
     int best = 1, best_cost = 0x7fffffff, best_per = nch;
@@ -501,12 +511,16 @@ int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, c
     *per = best_per;
     return best;
   };
+  // key side: chunk states and bf16 key features
+  int kper = 0;
+  const int ksplit = split(4, &kper);
+  FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, kper, ksplit, crow, state, shifts, pmax, phik16));
   int qper = 0;
   const int qsplit = split(4, &qper);
   FS_CUDA_OK(cudaFuncSetAttribute(tc_featq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FqSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_FEATQ);
-  tc_featq_kernel<<<dim3(qsplit, BH), TC_THREADS, FqSmem::TOTAL + 1024, ctx->stream>>>(tmQ, images, H, dm->pool, L, Lpad, qper,
-                                                                                       phiq16, ctx->d_status);
+  tc_featq_kernel<<<dim3(qsplit, BH), TC_THREADS, FqSmem::TOTAL + 1024, ctx->stream>>>(tmQ, tmPhiQ, images, H, dm->pool, L, qper,
+                                                                                       ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
 
