@@ -231,19 +231,28 @@ tc_causal_prefix_kernel(const float* __restrict__ state, const float* __restrict
   float R[8];
 #pragma unroll
   for (int u = 0; u < 8; u++) R[u] = 0.f;
-  for (int c = 0; c < nch; c++) {
-    float kv[8];
+  // four chunks per trip: their loads are issued together, then the running sums move on
+  for (int c0 = 0; c0 < nch; c0 += 4) {
+    float kv[4][8];
 #pragma unroll
-    for (int u = 0; u < 8; u++) {
-      const int n = blockIdx.x * 8 + u;
-      kv[u] = n <= TC_DV ? sb[((size_t)c * TC_NV + n) * TC_M + threadIdx.x] : 0.f;
-    }
-    const float os = oscale[c], upc = up[c], adc = add[c];
+    for (int k = 0; k < 4; k++)
 #pragma unroll
-    for (int u = 0; u < 8; u++) {
-      const int n = blockIdx.x * 8 + u;
-      pb[((size_t)c * TC_NV + n) * TC_M + threadIdx.x] = __float2bfloat16_rn(R[u] * os);
-      R[u] = fmaf(R[u], upc, adc * kv[u]);
+      for (int u = 0; u < 8; u++) {
+        const int n = blockIdx.x * 8 + u;
+        kv[k][u] = (c0 + k < nch && n <= TC_DV) ? sb[((size_t)(c0 + k) * TC_NV + n) * TC_M + threadIdx.x] : 0.f;
+      }
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+      const int c = c0 + k;
+      if (c < nch) {
+        const float os = oscale[c], upc = up[c], adc = add[c];
+#pragma unroll
+        for (int u = 0; u < 8; u++) {
+          const int n = blockIdx.x * 8 + u;
+          pb[((size_t)c * TC_NV + n) * TC_M + threadIdx.x] = __float2bfloat16_rn(R[u] * os);
+          R[u] = fmaf(R[u], upc, adc * kv[k][u]);
+        }
+      }
     }
   }
 }
@@ -321,6 +330,15 @@ tc_causal_out_kernel(const __grid_constant__ CUtensorMap tmPhiQ, const __grid_co
           }
           tma_load_4d(sm + CoSmem::V, &tmV, &misc->full, 0, c * TILE, h, b);
           issued = it + 1;
+          if (it + 1 < nmine) {           // the next chunk's operands: into L2 while this one is worked on
+#pragma unroll
+            for (int fb = 0; fb < TC_M / 64; fb++) {
+              tma_prefetch_3d(&tmPhiQ, fb * 64, (c + 1) * TILE, bh);
+              tma_prefetch_3d(&tmPhiK, fb * 64, (c + 1) * TILE, bh);
+              tma_prefetch_3d(&tmPfx, fb * 64, 0, bh * nch + c + 1);
+            }
+            tma_prefetch_4d(&tmV, 0, (c + 1) * TILE, h, b);
+          }
         }
         // no copy of this block may still be in flight when it exits
         if (issued > 0) mbar_wait(&misc->full, (issued - 1) & 1, abortp, status, false);
