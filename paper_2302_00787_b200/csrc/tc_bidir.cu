@@ -39,7 +39,8 @@ constexpr int PREFETCH_TILES = 4;   // tiles pulled into L2 ahead of the shared-
 struct KvSmem {
   static constexpr uint32_t X0 = 0, V0 = 2 * TILE_BYTES, ONES = 4 * TILE_BYTES, W = ONES + TILE_BYTES,
                             WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES, FA2 = PHI + 4 * TILE_BYTES,
-                            MISC = FA2 + TC_M * 4, TOTAL = MISC + 256;
+                            STG = FA2 + TC_M * 4,        // 2 KB per storing epilogue warp: accumulator rows on their way out
+                            MISC = STG + 6 * 2048, TOTAL = MISC + 256;
 };
 static_assert(KvSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 static_assert(KvSmem::PHI % 1024 == 0 && KvSmem::W % 1024 == 0 && KvSmem::ONES % 1024 == 0, "swizzled tiles need 1024-byte alignment");
@@ -222,22 +223,32 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     auto write_partial = [&](size_t slot) {
       __syncwarp();
       tcgen05_fence_after();
-      float* out = partial + (slot * TC_NV + row) * TC_M + hf * 128;
+      float* out = partial + slot * TC_NV * TC_M + hf * 128;            // row n at out + n * TC_M
       float amax = 0.f;
-      if (q * 32 < TC_NV) {                 // warp-uniform: lanes 0..79 carry data
+      if (q * 32 <= TC_DV) {                // warp-uniform: rows 0..64 carry data (65..79 are zero and never read)
+        // 16 columns at a time go through shared memory, so that a store instruction of the warp
+        // covers 8 rows x 64 contiguous bytes instead of 32 rows x 16 bytes
+        uint8_t* stg = sm + KvSmem::STG + (hf * 3 + q) * 2048;
 #pragma unroll
         for (int c = 0; c < 8; c++) {
           uint32_t a[16];
           tmem_ld16(acc_addr + c * 16, a);
           tmem_wait_ld();
-          if (row < TC_NV) {
+          if (row <= TC_DV) {
 #pragma unroll
-            for (int j = 0; j < 16; j++)
-              if (row <= TC_DV) amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
-#pragma unroll
-            for (int j = 0; j < 4; j++)
-              reinterpret_cast<uint4*>(out + c * 16)[j] = make_uint4(a[4 * j], a[4 * j + 1], a[4 * j + 2], a[4 * j + 3]);
+            for (int j = 0; j < 16; j++) amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
           }
+#pragma unroll
+          for (int i = 0; i < 4; i++)
+            *reinterpret_cast<uint4*>(stg + lane * 64 + ((i ^ ((lane >> 1) & 3)) << 4)) = make_uint4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 4; i++) {
+            const int rr = (lane >> 2) + 8 * i, cw = lane & 3, n = q * 32 + rr;
+            const uint4 val = *reinterpret_cast<const uint4*>(stg + rr * 64 + ((cw ^ ((rr >> 1) & 3)) << 4));
+            if (n <= TC_DV) *reinterpret_cast<uint4*>(out + (size_t)n * TC_M + c * 16 + cw * 4) = val;
+          }
+          __syncwarp();
         }
       }
 #pragma unroll
