@@ -325,10 +325,13 @@ def roofline_for(name, k, w, work, peaks):
         "out_kernel": 2 * L * M * (dv + 1) * units, "scores_kernel": L * w.chunk * M * units if w.causal else 0,
         "tc_kv_kernel": (2 * L * d * M + 2 * L * M * (dv + 1)) * units,
         "tc_out_kernel": (2 * L * d * M + 2 * L * M * (dv + 1)) * units,
-        "tc_causal_out_kernel": work["flops"], "tc_causal_state_kernel": (2 * L * d * M + 2 * L * M * (dv + 1)) * units,
+        "tc_featq_kernel": 2 * L * d * M * units,
+        "tc_causal_out_kernel": (2 * L * M * (dv + 1) + 2 * L * 128 * M + 2 * L * 128 * dv) * units,
     }
     bytes_of = {"stats_kernel": 2 * L * d * es * units, "tc_stats_kernel": 2 * L * d * es * units, "expshift_kernel": 2 * L * M * 4 * units,
-                "rowterm_kernel": L * d * es * units, "groupmax_kernel": L * M * 4 * units}
+                "rowterm_kernel": L * d * es * units, "groupmax_kernel": L * M * 4 * units,
+                "tc_rowterm_kernel": L * d * es * units,
+                "tc_causal_prefix_kernel": ((L + 127) // 128) * (65 * M * 4 + 80 * M * 2) * units}
     if name in flops_of and flops_of[name]:
         fl = flops_of[name] * (per_launch if name in ("logits_kernel", "kv_kernel", "out_kernel", "scores_kernel") and
                                k["launches_per_step"] > 1 else 1.0)

@@ -392,6 +392,30 @@ __device__ void jacobi_tables(const ushort2* sched, uchar2* pos, uint2* la, ucha
   __syncthreads();
 }
 
+// d x d product with both operands in shared memory: out(r, c, sum_k a(r, k) b(k, c)).  Thread t owns
+// column c = t % d and up to eight rows t / d + u * (FIT_THREADS / d): eight independent sums per trip.
+template <class FA, class FB, class FO>
+__device__ __forceinline__ void smem_product(int d, FA a, FB b, FO out) {
+  const int c = threadIdx.x % d, r0 = threadIdx.x / d, rstep = FIT_THREADS / d;
+  if (r0 >= d) return;
+  double acc[8];
+#pragma unroll
+  for (int u = 0; u < 8; u++) acc[u] = 0.0;
+  for (int k = 0; k < d; k++) {
+    const double bv = b(k, c);
+#pragma unroll
+    for (int u = 0; u < 8; u++) {
+      const int r = r0 + u * rstep;
+      if (r < d) acc[u] = fma(a(r, k), bv, acc[u]);
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < 8; u++) {
+    const int r = r0 + u * rstep;
+    if (r < d) out(r, c, acc[u]);
+  }
+}
+
 struct FitArgs {
   const double* stats;
   double* params;
@@ -582,10 +606,11 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
       __syncthreads();
       double piv = aux[j];
       if (!(piv > floor_piv)) { violated = true; piv = floor_piv + 1e-300; }
-      const double ljj = sqrt(piv);
+      double rs = rsqrt(piv);
+      rs = rs * fma(-0.5 * piv * rs, rs, 1.5);       // one Newton step on 1 / sqrt(piv)
       if (part == 0) {
-        if (ri == j) As[j * lda + j] = ljj;
-        else if (ri > j) As[ri * lda + j] = aux[ri] / ljj;
+        if (ri == j) { As[j * lda + j] = piv * rs; lam[j] = rs; }     // lam: 1 / l_jj
+        else if (ri > j) As[ri * lda + j] = aux[ri] * rs;
         else As[ri * lda + j] = 0.0;                 // upper triangle
       }
       __syncthreads();
@@ -601,7 +626,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
         if (i > c)
           for (int k = c + part; k < i; k += parts) t = fma(As[i * lda + k], Li[k * ldi + c], t);
         for (int o = parts >> 1; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-        if (part == 0) Li[i * ldi + c] = i < c ? 0.0 : (i == c ? 1.0 / As[c * lda + c] : -t / As[i * lda + i]);
+        if (part == 0) Li[i * ldi + c] = i < c ? 0.0 : (i == c ? lam[c] : -t * lam[i]);
         __syncwarp();
       }
     }
@@ -616,23 +641,16 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
     __syncthreads();
     if (V_IN_SMEM) {
       // T1 = M2 L (M2 in Vs, L in As) -> Ws
-      for (int e = tid; e < d * d; e += FIT_THREADS) {
-        int i = e / d, l = e % d;
-        double s = 0.0;
-        for (int j = l; j < d; j++) s = fma(Vs[i * lda + j], As[j * lda + l], s);
-        Ws[i * lda + l] = s;
-      }
+      smem_product(d, [&](int r, int k) { return Vs[r * lda + k]; }, [&](int k, int c) { return As[k * lda + c]; },
+                   [&](int r, int c, double v) { Ws[r * lda + c] = v; });
       __syncthreads();
-      // Z Z^T = L^T T1 (symmetric; both triangles written from the same sum) -> Vs, then As
+      // L^T T1 -> A1 (its L^-1 is already in global memory), then Z Z^T = its symmetric part -> Vs
+      smem_product(d, [&](int r, int k) { return As[k * lda + r]; }, [&](int k, int c) { return Ws[k * lda + c]; },
+                   [&](int r, int c, double v) { A1[r * lda + c] = v; });
+      __syncthreads();
       for (int e = tid; e < d * d; e += FIT_THREADS) {
         int r = e / d, c = e % d;
-        if (r > c) continue;
-        double s = 0.0, s2 = 0.0;
-        for (int i = r; i < d; i++) s = fma(As[i * lda + r], Ws[i * lda + c], s);
-        for (int i = c; i < d; i++) s2 = fma(As[i * lda + c], Ws[i * lda + r], s2);
-        double v = 0.5 * (s + s2);
-        Vs[r * lda + c] = v;
-        Vs[c * lda + r] = v;
+        Vs[r * lda + c] = 0.5 * (A1[r * lda + c] + A1[c * lda + r]);
       }
       __syncthreads();
       for (int e = tid; e < d * lda; e += FIT_THREADS) As[e] = Vs[e];
@@ -683,47 +701,28 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
         Ws[(e / d) * lda + (e % d)] = Lg[e];
       }
       __syncthreads();
-      // B1 = r Sigma^1/2 U^T L^-1,  B2 = r Sigma^-1/2 U^T L^T, kept in shared memory (As, then A1) for C
-      constexpr int EPT = 8;                      // d * d / FIT_THREADS for d = 64; fewer elements for smaller d
-      double b1[EPT], b2[EPT];
-#pragma unroll
-      for (int u = 0; u < EPT; u++) {
-        const int e = tid + u * FIT_THREADS;
-        b1[u] = b2[u] = 0.0;
-        if (e < d * d) {
-          int l = e / d, j = e % d;
-          double s1 = 0.0, s2 = 0.0;
-          for (int i = j; i < d; i++) s1 = fma(Vs[l * ldv + i], A1[i * lda + j], s1);
-          for (int i = 0; i <= j; i++) s2 = fma(Vs[l * ldv + i], Ws[j * lda + i], s2);
-          const double sg = sqrt(aux[l]);
-          b1[u] = r * sg * s1;
-          b2[u] = r / sg * s2;
-        }
-      }
+      // B1 = r Sigma^1/2 U^T L^-1 -> As,  B2 = r Sigma^-1/2 U^T L^T -> global, then A1 once L^-1 is no longer read
+      smem_product(d, [&](int l, int i) { return Vs[l * ldv + i]; }, [&](int i, int j) { return A1[i * lda + j]; },
+                   [&](int l, int j, double v) {
+                     const double b1 = r * sqrt(aux[l]) * v;
+                     As[l * lda + j] = b1;
+                     oB1[l * d + j] = b1;
+                     oA[l * d + j] = (l == j) ? A : 0.0;
+                   });
       __syncthreads();
-#pragma unroll
-      for (int u = 0; u < EPT; u++) {
-        const int e = tid + u * FIT_THREADS;
-        if (e < d * d) {
-          int l = e / d, j = e % d;
-          As[l * lda + j] = b1[u];
-          A1[l * lda + j] = b2[u];
-          oB1[e] = b1[u];
-          oB2[e] = b2[u];
-          oA[e] = (l == j) ? A : 0.0;
-        }
-      }
+      smem_product(d, [&](int l, int i) { return Vs[l * ldv + i]; }, [&](int i, int j) { return Ws[j * lda + i]; },
+                   [&](int l, int j, double v) {
+                     const double b2 = r / sqrt(aux[l]) * v;
+                     A1[l * lda + j] = b2;
+                     oB2[l * d + j] = b2;
+                   });
       __syncthreads();
-      for (int e = tid; e < d * d; e += FIT_THREADS) {
-        int i = e / d, j = e % d;
-        double s1 = 0.0, s2 = 0.0;
-        for (int l = 0; l < d; l++) {
-          s1 = fma(As[l * lda + i], As[l * lda + j], s1);
-          s2 = fma(A1[l * lda + i], A1[l * lda + j], s2);
-        }
-        oC1[e] = -s1 / (2.0 * (1.0 - 4.0 * A));
-        oC2[e] = -s2 / (2.0 * (1.0 - 4.0 * A));
-      }
+      // C = -B^T B / (2 (1 - 4A))
+      const double cf = -1.0 / (2.0 * (1.0 - 4.0 * A));
+      smem_product(d, [&](int i, int l) { return As[l * lda + i]; }, [&](int l, int j) { return As[l * lda + j]; },
+                   [&](int i, int j, double v) { oC1[i * d + j] = cf * v; });
+      smem_product(d, [&](int i, int l) { return A1[l * lda + i]; }, [&](int l, int j) { return A1[l * lda + j]; },
+                   [&](int i, int j, double v) { oC2[i * d + j] = cf * v; });
     } else {
       for (int e = tid; e < d * d; e += FIT_THREADS) Ug[e] = Vs[(e % d) * ldv + (e / d)];     // U[i][l]
       __syncthreads();
