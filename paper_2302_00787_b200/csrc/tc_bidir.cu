@@ -5,15 +5,16 @@
 //                               KV^T += [V | 1]^T phi                        (tcgen05, TMEM)
 //                               (c_j, the key's quadratic term, comes from tc_rowterm_kernel)
 //   merge      (tc_merge_kernel): partial KV^T of the splits of one (batch, head), brought to a
-//                               common shift, summed, scaled by 2^a2 per feature, written in fp16
-//   query side (tc_out_kernel): logits, phi = 2^(logits - max of the half row) in fp16,
+//                               common shift, summed, every feature's column scaled to order one
+//                               (fp16); the scales' exponents g, with a2, go to the query side
+//   query side (tc_out_kernel): logits + g, phi = 2^(... - max of the half row) in fp16,
 //                               [num | den] = phi KV per feature half, halves combined, Y = num / den
 //
 // The feature tiles never leave the SM.  One block = 8 epilogue warps (exponentials), one
 // TMA producer warp and one MMA issuing warp; all exponents are kept in log2 units
 // (W and C are pre-multiplied by log2 e), so a feature is one ex2 per element.  The per-feature
-// term w^T A w is the same on the query and the key side, so it is not added to the logits at
-// all: the merge multiplies feature m of S^T [V | 1] by 2^(2 log2e w_m^T A w_m).
+// term w^T A w is the same on the query and the key side; the key side leaves it out and the query
+// side adds both shares, 2 log2e w_m^T A w_m, to its logits (inside g).
 #include <cuda_fp16.h>
 
 #include "common.cuh"
@@ -374,20 +375,27 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 }
 
 // ------------------------------------------------------------------------------------------
-// merge of the key-side partials of one (batch, head): common shift, sum, per-feature factor
-// 2^a2, fp16.  Partials and result are both [80 rows][256 features].
+// merge of the key-side partials of one (batch, head): common shift, sum, and a scale of its own
+// for every feature.  Partials and result are both [80 rows][256 features].
+//
+// The query side contracts phi(Q) with this state in fp16, whose exponent range is narrow, and what
+// a feature contributes to an output is phi(Q)_m times the size of column m of the state.  So every
+// column m is brought to order one by a power of two 2^-e_m, and g_m = e_m + a2_m - max a2 (the
+// per-feature term w^T A w of both sides rides along) is handed to the query side, which adds it
+// to its logits BEFORE it takes the row maximum: a query feature near 1 is then one that matters,
+// and what underflows in either operand is negligible by construction.
 // ------------------------------------------------------------------------------------------
-constexpr int MERGE_SLICES = 8;
-__global__ void __launch_bounds__(256)
-tc_merge_kernel(const float* __restrict__ partial, const float* __restrict__ shifts, const int* __restrict__ pmax,
-                int nsplit, const uint8_t* __restrict__ images, int H, int pool, __half* __restrict__ kvt) {
+constexpr int MERGE_THREADS = 1024, MERGE_ROWS = (TC_DV + 4) / 4;       // thread = (feature, one row in four)
+__global__ void __launch_bounds__(MERGE_THREADS)
+tc_merge_kernel(const float* __restrict__ partial, const float* __restrict__ shifts, int nsplit,
+                const uint8_t* __restrict__ images, int H, int pool, __half* __restrict__ kvt, float* __restrict__ gq) {
   __shared__ float fac[2 * 64];
-  __shared__ float rowfac[TC_M];
-  __shared__ float red[256];
-  const int bh = blockIdx.y;
+  __shared__ float red[MERGE_THREADS];
+  const int bh = blockIdx.x;
   const int g = pool == FSHARP_POOL_PER_BH ? bh : bh % H;
+  const int m = threadIdx.x & (TC_M - 1), qt = threadIdx.x >> 8, hh = m >> 7;
   const float* a2 = reinterpret_cast<const float*>(images + (size_t)g * 2 * IMG_BYTES + IMG_A2);
-  const float a2m = a2[threadIdx.x];          // 256 threads, 256 features
+  const float a2m = a2[m];
   red[threadIdx.x] = a2m;
   if (threadIdx.x < 2 * nsplit) fac[threadIdx.x] = shifts[(size_t)bh * nsplit * 2 + threadIdx.x];
   __syncthreads();
@@ -398,28 +406,35 @@ tc_merge_kernel(const float* __restrict__ partial, const float* __restrict__ shi
   const float a2max = red[0];
   float smax = -INFINITY;
   for (int p = 0; p < 2 * nsplit; p++) smax = fmaxf(smax, fac[p]);
-  // fp16 has a narrow range: scale the whole (batch, head) by a power of two (it cancels in
-  // num / den) so that the bound sum_p 2^(s_p - smax) max|partial_p| lands near 2^14; the
-  // per-feature factors are applied relative to their maximum, so none exceeds 1
-  float bound = 0.f;
-  for (int p = 0; p < 2 * nsplit; p++) bound = fmaf(exp2f(fac[p] - smax), __int_as_float(pmax[(size_t)bh * nsplit * 2 + p]), bound);
-  int ex = 0;
-  if (bound > 0.f && isfinite(bound)) frexpf(bound, &ex);
-  const float scale = exp2f((float)(14 - ex));
   __syncthreads();
   if (threadIdx.x < 2 * nsplit) fac[threadIdx.x] = exp2f(fac[threadIdx.x] - smax);
-  rowfac[threadIdx.x] = scale * exp2f(a2m - a2max);
   __syncthreads();
   const float* base = partial + (size_t)bh * nsplit * TC_NV * TC_M;
-  __half* out = kvt + (size_t)bh * TC_NV * TC_M;
-  constexpr int PER = TC_M * TC_NV / MERGE_SLICES;
-  for (int e = blockIdx.x * PER + threadIdx.x; e < (blockIdx.x + 1) * PER; e += 256) {
-    const int n = e / TC_M, m = e % TC_M, hh = m >> 7;
+  float val[MERGE_ROWS];
+  float amax = 0.f;
+#pragma unroll
+  for (int u = 0; u < MERGE_ROWS; u++) {
+    const int n = qt + 4 * u;
     float acc = 0.f;
     if (n <= TC_DV)
-      for (int p = 0; p < nsplit; p++) acc = fmaf(base[(size_t)p * TC_NV * TC_M + e], fac[2 * p + hh], acc);
-    out[e] = __float2half_rn(acc * rowfac[m]);
+      for (int p = 0; p < nsplit; p++) acc = fmaf(base[((size_t)p * TC_NV + n) * TC_M + m], fac[2 * p + hh], acc);
+    val[u] = acc;
+    amax = fmaxf(amax, fabsf(acc));
   }
+  red[threadIdx.x] = amax;
+  __syncthreads();
+  amax = fmaxf(fmaxf(red[m], red[TC_M + m]), fmaxf(red[2 * TC_M + m], red[3 * TC_M + m]));
+  int ex = 0;
+  if (amax > 0.f && isfinite(amax)) frexpf(amax, &ex);          // amax = f 2^ex, f in [1/2, 1)
+  const float sc = exp2f((float)-ex);
+  __half* out = kvt + (size_t)bh * TC_NV * TC_M;
+#pragma unroll
+  for (int u = 0; u < MERGE_ROWS; u++) {
+    const int n = qt + 4 * u;
+    if (n <= TC_DV) out[(size_t)n * TC_M + m] = __float2half_rn(val[u] * sc);
+  }
+  for (int n = TC_DV + 1 + qt; n < TC_NV; n += 4) out[(size_t)n * TC_M + m] = __float2half_rn(0.f);     // padding rows
+  if (qt == 0) gq[(size_t)bh * TC_M + m] = (float)ex + a2m - a2max;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -430,7 +445,8 @@ struct OutSmem {
   static constexpr uint32_t X0 = 0, W = OUT_STAGES * TILE_BYTES, WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES,
                             KVT = PHI + 4 * TILE_BYTES, ROWMAX = KVT + KVT_BYTES,
                             STAGE = ROWMAX + 3 * 2 * TILE * 4,          // 2 KB per epilogue warp: output rows on their way out
-                            MISC = STAGE + (EPI_THREADS / 32) * 2048, TOTAL = MISC + 256;
+                            GQ = STAGE + (EPI_THREADS / 32) * 2048,     // the merge's per-feature exponents g_m
+                            MISC = GQ + TC_M * 4, TOTAL = MISC + 256;
 };
 static_assert(OutSmem::PHI % 1024 == 0 && OutSmem::KVT % 1024 == 0 && OutSmem::W % 1024 == 0, "alignment");
 static_assert(OutSmem::TOTAL + 1024 <= 232448, "shared memory budget");
@@ -446,12 +462,13 @@ constexpr uint32_t OUT_COL_LOGITS = 0, OUT_COL_OUT = 256;
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKVt,
-              const uint8_t* __restrict__ images, int H, int pool, int L, int tiles_per_split,
+              const uint8_t* __restrict__ images, const float* __restrict__ gq, int H, int pool, int L, int tiles_per_split,
               __nv_bfloat16* __restrict__ Y, TensorAddr ay, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   OutMisc* misc = reinterpret_cast<OutMisc*>(sm + OutSmem::MISC);
   float* rowmax = reinterpret_cast<float*>(sm + OutSmem::ROWMAX);   // [tile % 3][half][row]
+  float* gs = reinterpret_cast<float*>(sm + OutSmem::GQ);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
   const int g = pool == FSHARP_POOL_PER_BH ? bh : h;
@@ -461,6 +478,7 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
   const uint8_t* img = images + ((size_t)g * 2 + 0) * IMG_BYTES;        // side 1 (queries)
   volatile int* abortp = &misc->abort_flag;
 
+  if (threadIdx.x < TC_M) gs[threadIdx.x] = gq[(size_t)bh * TC_M + threadIdx.x];
   if (threadIdx.x == 0) {
     for (int i = 0; i < OUT_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], 1); }
     mbar_init(&misc->logits_full, 1);
@@ -509,7 +527,7 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
   } else if (warp == WARP_MMA) {
     if (lane == 0) {
       constexpr uint32_t ID_LOGITS = idesc_bf16(128, TC_M, 0, 0);
-      constexpr uint32_t ID_OUT = idesc_f16(128, TC_NV, 0, 0);      // fp16: phi(Q) <= 1 and the scaled S^T [V | 1]
+      constexpr uint32_t ID_OUT = idesc_f16(128, TC_NV, 0, 0);      // fp16: phi(Q) <= 1 and a state of order one per feature
       const uint64_t dX0 = smem_desc(smem_u32(sm + OutSmem::X0), 16, 1024, SWZ_128B);
       const uint64_t dW = smem_desc(smem_u32(sm + OutSmem::W), 16, 1024, SWZ_128B);
       const uint64_t dWlo = smem_desc(smem_u32(sm + OutSmem::WLO), 16, 1024, SWZ_128B);
@@ -624,6 +642,15 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       tmem_wait_ld();
       tcgen05_fence_before();
       mbar_arrive(&misc->logits_free);
+      // the exponent of feature m's column of the state, and w^T A w of both sides, join the logit
+#pragma unroll
+      for (int i = 0; i < 128; i += 4) {
+        const float4 g4 = *reinterpret_cast<const float4*>(gs + hf * 128 + i);
+        v[i] = __float_as_uint(__uint_as_float(v[i]) + g4.x);
+        v[i + 1] = __float_as_uint(__uint_as_float(v[i + 1]) + g4.y);
+        v[i + 2] = __float_as_uint(__uint_as_float(v[i + 2]) + g4.z);
+        v[i + 3] = __float_as_uint(__uint_as_float(v[i + 3]) + g4.w);
+      }
       float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
       for (int i = 0; i < 128; i++) mxp[i & 3] = fmaxf(mxp[i & 3], __uint_as_float(v[i]));
@@ -704,7 +731,7 @@ size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
   return ws_round(G * 2 * IMG_BYTES) + ws_round(G * 2 * FLAG_WORDS * 4 + 64) +
          ws_round(BH * MAX_KEY_SPLIT * TC_M * TC_NV * 4) + 2 * ws_round(BH * MAX_KEY_SPLIT * 2 * 4) +
          ws_round(BH * (size_t)((dm->Lk + TILE - 1) / TILE) * TILE * 4) +
-         ws_round(BH * TC_NV * TC_M * 2);
+         ws_round(BH * TC_NV * TC_M * 2) + ws_round(BH * TC_M * 4);
 }
 
 // Key side: the per-key quadratic term, then the feature / contraction kernel.  crow: [B*H][Lpad] floats,
@@ -751,6 +778,7 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   const int Lpad = ktiles * TILE;
   float* crow = ws->take<float>((size_t)BH * Lpad);
   __half* kvt = ws->take<__half>((size_t)BH * TC_NV * TC_M);
+  float* gq = ws->take<float>((size_t)BH * TC_M);
   FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, tps, nsplit, crow, partial, shifts, pmax, nullptr));
 
   CUtensorMap tmQ, tmKVt;
@@ -758,7 +786,7 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   FS_TRY(tchost::make_map_kvt(&tmKVt, kvt, BH, 0));
   FS_CUDA_OK(cudaFuncSetAttribute(tc_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OutSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_MERGE);
-  tc_merge_kernel<<<dim3(MERGE_SLICES, BH), 256, 0, ctx->stream>>>(partial, shifts, pmax, nsplit, images, H, dm->pool, kvt);
+  tc_merge_kernel<<<BH, MERGE_THREADS, 0, ctx->stream>>>(partial, shifts, nsplit, images, H, dm->pool, kvt, gq);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
 
@@ -767,7 +795,7 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   int qsplit = pick_split(BH, qtiles, ctx->sm_count, 1 << 20, &qtps);
   FS_TIME_BEGIN(ctx, FS_K_TC_OUT);
   tc_out_kernel<<<dim3(qsplit, BH), TC_THREADS, OutSmem::TOTAL + 1024, ctx->stream>>>(
-      tmQ, tmKVt, images, H, dm->pool, Lq, qtps, (__nv_bfloat16*)Y, fs_addr(dm->y_stride, H, Lq, dm->dv), ctx->d_status);
+      tmQ, tmKVt, images, gq, H, dm->pool, Lq, qtps, (__nv_bfloat16*)Y, fs_addr(dm->y_stride, H, Lq, dm->dv), ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;

@@ -245,6 +245,31 @@ def test_attend_properties(ctx):
     assert ctx.status() == 0
 
 
+@pytest.mark.parametrize("stress", ["keys_ramp_up", "keys_ramp_down", "all_scaled"])
+def test_bidirectional_tensor_core_path_wide_dynamic_range(ctx, stress):
+    """Keys whose size changes threefold along the sequence (or queries and keys scaled 2.5x) spread the
+    feature exponents over far more than fp16's range; the tensor-core kernels must still agree with
+    the checker (per-feature scales of the contracted state, joined to the query logits)."""
+    for variant in ("sderf", "aderf"):
+        w = W["cfg3b"].scaled(B=1, H=2, L=896, variant=variant)
+        Q, K, V = wl.make_qkv(w)
+        Om = wl.make_omega(w)
+        t = np.arange(w.L, dtype=np.float64) / w.L
+        if stress == "all_scaled":
+            Q, K = wl.bf16_round(Q * 2.5), wl.bf16_round(K * 2.5)
+        else:
+            gain = 1.0 + 2.0 * t if stress == "keys_ramp_up" else 3.0 - 2.0 * t
+            K = wl.bf16_round(K * gain[None, None, :, None])
+        dQ, dK, dV, dOm = dev(Q, "bf16"), dev(K, "bf16"), dev(V, "bf16"), dev(Om)
+        _, pr = gpu_fit(ctx, dQ, dK, w.d, w.variant)
+        Y = host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr))
+        assert ctx.status() == 0
+        prh = pr.cpu().numpy()
+        for h in range(w.H):
+            ref = oracle_unit(Q, K, V, Om, prh[h], w.d, 0, h, False)
+            assert rel_err(Y[0, h], ref) < TOL["bf16"], (variant, h)
+
+
 @pytest.mark.parametrize("ramp", ["up", "down", "flat"])
 def test_causal_tensor_core_path_scales_across_chunks(ctx, ramp):
     """bf16, d = dv = 64, M = 256, chunk 128 takes the tensor-core causal kernels.  Keys that grow
