@@ -312,6 +312,12 @@ def main():
         dist.destroy_process_group()
 
 
+# DRAM bytes per launch (read + write) from the ncu captures summarised under profiles/ (same kernels, same workload);
+# an entry is dropped when its kernel changes.
+NCU_TRAFFIC = {("cfg2", "fit_kernel"): 4.36e6, ("cfg2", "tc_kv_kernel"): 75.4e6, ("cfg2", "tc_out_kernel"): 42.3e6,
+               ("cfg2", "tc_stats_kernel"): 72.1e6, ("cfg3", "tc_kv_kernel"): 531.4e6, ("cfg3", "tc_causal_out_kernel"): 626.2e6}
+
+
 def roofline_for(name, k, w, work, peaks):
     """Roofline entry for the step's dominant kernel.  Algorithmic work per launch:
     tensor-bound kernels carry their share of the attend flops; the rest are judged on bytes."""
@@ -337,7 +343,7 @@ def roofline_for(name, k, w, work, peaks):
                                k["launches_per_step"] > 1 else 1.0)
         ach = fl / t / 1e12
         return {"kernel": name, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": ach / peaks["bf16_tflops"], "traffic": None, "peak_source": peaks["source"]}
+                "frac": ach / peaks["bf16_tflops"], "traffic": NCU_TRAFFIC.get((w.name, name)), "peak_source": peaks["source"]}
     if name == "fit_kernel":
         # fp64 arithmetic of the Jacobi sweeps (the rest of the fit is negligible): per round and group the
         # 2 x 2 blocks of A (8 multiplies + 8 multiply-adds each) and d/2 * d row-pair entries of V^T
@@ -348,13 +354,13 @@ def roofline_for(name, k, w, work, peaks):
         peak = 64 * 2 * peaks.get("sm_count", 148) * peaks.get("sm_max_mhz", 1965.0) * 1e6 / 1e12
         ach = flops / t / 1e12
         return {"kernel": name, "bound": "alu", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
-                "traffic": None, "peak_source": "64 fp64 FMA/clk/SM x SMs x max SM clock",
+                "traffic": NCU_TRAFFIC.get((w.name, name)) if w.variant == "sderf" else None, "peak_source": "64 fp64 FMA/clk/SM x SMs x max SM clock",
                 "note": f"one block per group ({units} of {peaks.get('sm_count', 148)} SMs busy), "
                         f"{work.get('fit_sweeps', 0.0):.1f} Jacobi sweeps per group; bound by shared-memory wavefronts and barrier latency"}
     by = bytes_of.get(name, work["bytes"]) * (per_launch if k["launches_per_step"] > 1 else 1.0)
     ach = by / t / 1e9
     return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-            "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
+            "frac": ach / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC.get((w.name, name)), "peak_source": peaks["source"]}
 
 
 if __name__ == "__main__":

@@ -2,12 +2,13 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "tc_layout.cuh"
 
 // tensor-core path (tc_*.cu)
 int fs_tc_supported(const fsharp_dims* dm, int dtype, int causal, int chunk, float qk_scale);
 size_t fs_tc_attend_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm, int causal, int chunk);
 int fs_tc_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, int causal,
-                 int chunk, float qk_scale, const float* prep, void* Y, WsAlloc* ws);
+                 int chunk, const uint8_t* images, const int* flags, void* Y, WsAlloc* ws);
 
 namespace {
 
@@ -123,9 +124,16 @@ int fsharp_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, 
   FS_TRY(fs_ws_reserve(ctx, need));
   WsAlloc ws{ctx->ws, 0};
   float* prep = ws.take<float>(prep_f);
+  if (use_tc) {
+    // the prep kernel also writes the tensor-core path's operand images
+    uint8_t* images = ws.take<uint8_t>((size_t)G * 2 * tcl::IMG_BYTES);
+    int* flags = ws.take<int>((size_t)G * 2 * tcl::FLAG_WORDS + 16);
+    FS_TRY(fs_run_prep_images(ctx, Omega, dims->omega_head_stride, params, (int64_t)ParamsLayout{dims->d}.total(), G,
+                              dims->H, dims->pool, dims->d, dims->M, prep, qk_scale, images, flags));
+    return fs_tc_attend(ctx, Q, K, V, dims, causal, chunk, images, flags, Y, &ws);
+  }
   FS_TRY(fs_run_prep(ctx, Omega, dims->omega_head_stride, params, (int64_t)ParamsLayout{dims->d}.total(), G,
                      dims->H, dims->pool, dims->d, dims->M, prep));
-  if (use_tc) return fs_tc_attend(ctx, Q, K, V, dims, causal, chunk, qk_scale, prep, Y, &ws);
   return fs_simt_attend(ctx, Q, K, V, dims, dtype, causal, chunk, qk_scale, prep, Y, &ws);
 }
 

@@ -155,6 +155,10 @@ size_t fs_fit_scratch_doubles(int G, int d);
 // params_stride: doubles between the blobs of two groups (0 = every group reads the same blob)
 int fs_run_prep(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_stride, const double* params,
                 int64_t params_stride, int G, int H, int pool, int d, int M, float* prep /* [G][2][PrepLayout] */);
+// The same, and (images != nullptr; d = 64, M = 256) the tensor-core path's operand images and flag words too.
+int fs_run_prep_images(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_stride, const double* params,
+                       int64_t params_stride, int G, int H, int pool, int d, int M, float* prep, float qk_scale,
+                       uint8_t* images, int* flags);
 // rowc: scratch [B*H*L] floats.  gmax: scratch [B*H] words.  phi: [B,H,L,M] floats.
 int fs_simt_featurize(fsharp_ctx* ctx, const void* X, int dtype, TensorAddr ax, int B, int H, int L, int d,
                       int M, int pool, const float* prep, int side, float qk_scale, int stab,

@@ -217,10 +217,9 @@ __device__ __forceinline__ int jacobi_upper(int i, int j, int lda) { return i < 
 
 template <int D>
 __device__ __forceinline__ void jacobi_a_items(const JacobiCtx& jc, const double* __restrict__ Ao, double* __restrict__ An,
-                                               const ushort2* sr, const double* cs, int wid, int nw) {
-  constexpr int half = D / 2, ntri = half * (half + 1) / 2;
+                                               const ushort2* sr, const double* cs, int first, int last, int step) {
   const int lda = jc.lda;
-  for (int e = wid; e < ntri; e += nw) {
+  for (int e = first; e < last; e += step) {
     const uchar2 kl = jc.tri[e];
     const int k = kl.x, l = kl.y;
     const int pk = sr[k].x, qk = sr[k].y, pl = sr[l].x, ql = sr[l].y;
@@ -247,12 +246,16 @@ __device__ __forceinline__ int jacobi_role(const JacobiCtx& jc_in, int* final_bu
   const JacobiCtx jc = jc_in;                            // by value: the fields stay in registers
   constexpr int d = D, half = D / 2, nrounds = D - 1, N2 = D / 2;
   constexpr int VT_THREADS = 2 * D;
-  constexpr int NW = FIT_THREADS - 32;                   // threads that work on A (the V^T threads after their own work)
+  constexpr int ntri = half * (half + 1) / 2;            // blocks of A on and above the block diagonal
+  constexpr int NA = FIT_THREADS - 32 - VT_THREADS;      // threads that only work on A
+  // the V^T threads take the last VT_ITEMS blocks of A after their own work (measured best: three quarters
+  // of a block per thread), the others share the rest
+  constexpr int VT_ITEMS = (3 * VT_THREADS / 4) < ntri ? 3 * VT_THREADS / 4 : ntri;
   const int tid = threadIdx.x, lda = jc.lda;
   const int vcol = (tid - 32) >> 1, vh = (tid - 32) & 1;  // JR_VT: column of V^T and which half of its seats
-  // JR_A threads come first in the item order, so the V^T threads only pick up what is left
-  // when the others have one item each
-  const int wid = ROLE == JR_A ? tid - 32 - VT_THREADS : tid - 32 + (FIT_THREADS - 32 - VT_THREADS);
+  const int a_first = ROLE == JR_A ? tid - 32 - VT_THREADS : ntri - VT_ITEMS + (tid - 32);
+  const int a_last = ROLE == JR_A ? ntri - VT_ITEMS : ntri;
+  constexpr int a_step = ROLE == JR_A ? NA : VT_THREADS;
   // index sitting at `seat` in round r
   auto seat_index = [](int r, int seat) {
     const int k = seat >> 1;
@@ -338,9 +341,9 @@ __device__ __forceinline__ int jacobi_role(const JacobiCtx& jc_in, int* final_bu
         for (int j = N2 - 1; j >= 5; j -= 2) x[j] = x[j - 2];
         x[3] = vh ? x[1] : t0;
         x[1] = vh ? recv : x[1];
-        jacobi_a_items<D>(jc, Ao, An, sr, cs, wid, NW);
+        jacobi_a_items<D>(jc, Ao, An, sr, cs, a_first, a_last, a_step);
       } else {
-        jacobi_a_items<D>(jc, Ao, An, sr, cs, wid, NW);
+        jacobi_a_items<D>(jc, Ao, An, sr, cs, a_first, a_last, a_step);
       }
       __syncthreads();
     }

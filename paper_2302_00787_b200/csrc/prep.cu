@@ -2,6 +2,8 @@
 // W^(k) = Omega B^(k) (row m = (B^(k)T w_m)^T), a_m = w_m^T A w_m, the constant
 // log D - 1/2 log M.
 #include "common.cuh"
+#include "tc_common.cuh"
+#include "tc_layout.cuh"
 
 namespace {
 
@@ -15,7 +17,10 @@ constexpr int PREP_LDO = PREP_MB + 4;         // row stride of the transposed Om
 template <int D>
 __global__ void __launch_bounds__(PREP_THREADS)
 prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const double* __restrict__ params,
-            int64_t params_stride, int H, int pool, int M, float* __restrict__ prep) {
+            int64_t params_stride, int H, int pool, int M, float* __restrict__ prep, float qk_scale,
+            uint8_t* __restrict__ images, int* __restrict__ img_flags) {
+  // images != nullptr (d = 64, M = 256 only): the tensor-core path's operand images of this (group, side)
+  // are written as well, in the layouts of tc_layout.cuh
   constexpr int d = D, NC = D / 16;
   __shared__ int redi[PREP_THREADS];
   extern __shared__ __align__(16) float stage[];
@@ -80,6 +85,20 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
         if (m < M) {
 #pragma unroll
           for (int v = 0; v < NC; v++) W[(size_t)m * d + NC * tx + v] = acc[u][v];
+          if (images != nullptr) {
+            // log2e * qk_scale * W as a bf16 value and its bf16 remainder, two neighbours per store
+            uint8_t* img = images + ((size_t)g * 2 + (side - 1)) * tcl::IMG_BYTES;
+            const float sw = FS_LOG2E * qk_scale;
+#pragma unroll
+            for (int v = 0; v + 1 < NC; v += 2) {
+              const float v0 = acc[u][v] * sw, v1 = acc[u][v + 1] * sw;
+              const __nv_bfloat16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
+              const uint32_t off = tc::sw128_offset(m, NC * tx + v);
+              *reinterpret_cast<__nv_bfloat162*>(img + tcl::IMG_W + off) = __nv_bfloat162(h0, h1);
+              *reinterpret_cast<__nv_bfloat162*>(img + tcl::IMG_WLO + off) =
+                  __nv_bfloat162(__float2bfloat16_rn(v0 - __bfloat162float(h0)), __float2bfloat16_rn(v1 - __bfloat162float(h1)));
+            }
+          }
         }
       } else {
         // a_m = sum_j (Omega A)_mj Omega_mj, summed over the 16 threads that share row m
@@ -88,19 +107,33 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
         for (int v = 0; v < NC; v++) sacc = fmaf(acc[u][v], Ot[(NC * tx + v) * PREP_LDO + 4 * ty + u], sacc);
 #pragma unroll
         for (int o = 8; o > 0; o >>= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, o);
-        if (tx == 0 && m < M) av[m] = sacc;
+        if (tx == 0 && m < M) {
+          av[m] = sacc;
+          if (images != nullptr)
+            reinterpret_cast<float*>(images + ((size_t)g * 2 + (side - 1)) * tcl::IMG_BYTES + tcl::IMG_A2)[m] = 2.f * FS_LOG2E * sacc;
+        }
       }
     }
   }
   if (blockIdx.z != 0) return;
   // C = gamma I exactly?
-  int cscalar = 1;
+  int cscalar = 1, lo_nonzero = 0;
   const double gamma = Cm[0];
   for (int e = tid; e < d * d; e += PREP_THREADS) {
     int i = e / d, j = e % d;
     Cf[e] = (float)Cm[e];
     if (i == j ? (Cm[e] != gamma) : (Cm[e] != 0.0)) cscalar = 0;
+    if (images != nullptr) {
+      // log2e * qk_scale^2 * C[i][j] goes to row j, column i of the MMA operand
+      uint8_t* img = images + ((size_t)g * 2 + (side - 1)) * tcl::IMG_BYTES;
+      const float v = (float)Cm[e] * (FS_LOG2E * qk_scale * qk_scale);
+      const __nv_bfloat16 hi = __float2bfloat16_rn(v), lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+      if (__bfloat162float(lo) != 0.f) lo_nonzero = 1;
+      *reinterpret_cast<__nv_bfloat16*>(img + tcl::IMG_CHI + tc::sw128_offset(j, i)) = hi;
+      *reinterpret_cast<__nv_bfloat16*>(img + tcl::IMG_CLO + tc::sw128_offset(j, i)) = lo;
+    }
   }
+  lo_nonzero = __syncthreads_or(lo_nonzero);
   redi[tid] = cscalar;
   __syncthreads();
   for (int s = PREP_THREADS / 2; s > 0; s >>= 1) {
@@ -112,6 +145,11 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
     scal[PS_BIAS] = (float)(tail[PT_LOGD] - 0.5 * log((double)M));
     scal[PS_CSCALAR] = redi[0] ? 1.f : 0.f;
     scal[PS_CGAMMA] = (float)gamma;
+    if (images != nullptr) {
+      int* fl = img_flags + ((size_t)g * 2 + (side - 1)) * tcl::FLAG_WORDS;
+      fl[0] = (redi[0] ? 0 : tcl::FLAG_C_DENSE) | (lo_nonzero ? tcl::FLAG_C_LO : 0);
+      fl[1] = __float_as_int((float)gamma * (FS_LOG2E * qk_scale * qk_scale));
+    }
   }
 }
 
@@ -119,7 +157,14 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
 
 int fs_run_prep(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_stride, const double* params,
                 int64_t params_stride, int G, int H, int pool, int d, int M, float* prep) {
+  return fs_run_prep_images(ctx, Omega, omega_head_stride, params, params_stride, G, H, pool, d, M, prep, 1.f, nullptr, nullptr);
+}
+
+int fs_run_prep_images(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_stride, const double* params,
+                       int64_t params_stride, int G, int H, int pool, int d, int M, float* prep, float qk_scale,
+                       uint8_t* images, int* flags) {
   if (G == 0) return FSHARP_OK;
+  if (images != nullptr && (d != tcl::TC_D || M != tcl::TC_M)) return FSHARP_E_SHAPE;
   const dim3 grid(G, 2, (M + PREP_MB - 1) / PREP_MB);
   const size_t smem = ((size_t)d * PREP_LDO + (size_t)d * d) * sizeof(float);
 #define FS_PREP(DD)                                                                                                  \
@@ -127,7 +172,7 @@ int fs_run_prep(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_stride, 
     FS_CUDA_OK(cudaFuncSetAttribute(prep_kernel<DD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));        \
     FS_TIME_BEGIN(ctx, FS_K_PREP);                                                                                    \
     prep_kernel<DD><<<grid, PREP_THREADS, smem, ctx->stream>>>(Omega, omega_head_stride, params, params_stride, H,   \
-                                                               pool, M, prep);                                       \
+                                                               pool, M, prep, qk_scale, images, flags);              \
   } while (0)
   switch (d) {
     case 16: FS_PREP(16); break;

@@ -713,12 +713,11 @@ int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int
 int make_map_kvt(CUtensorMap* map, const void* base, int BH, int bf16);
 int make_map_feat(CUtensorMap* map, const void* base, int BH, int Lpad);
 }  // namespace tchost
-int fs_tc_prep(fsharp_ctx* ctx, const float* prep, int G, float qk_scale, uint8_t* images, int* flags);
 int fs_tc_rowterm(fsharp_ctx* ctx, const void* K, const fsharp_dims* dm, const uint8_t* images, const int* flags, int Lpad,
                   int tiles_per_split, int nsplit, float* crow);
 size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
-int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
-                const float* prep, void* Y, WsAlloc* ws);
+int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
+                const int* flags, void* Y, WsAlloc* ws);
 int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                    const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax,
                    __nv_bfloat16* phik);
@@ -759,13 +758,9 @@ int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_d
   return FSHARP_OK;
 }
 
-int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
-                const float* prep, void* Y, WsAlloc* ws) {
+int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
+                const int* flags, void* Y, WsAlloc* ws) {
   const int B = dm->B, H = dm->H, BH = B * H, Lq = dm->Lq, Lk = dm->Lk;
-  const int G = fs_groups(dm);
-  uint8_t* images = ws->take<uint8_t>((size_t)G * 2 * IMG_BYTES);
-  int* flags = ws->take<int>((size_t)G * 2 * FLAG_WORDS + 16);
-  FS_TRY(fs_tc_prep(ctx, prep, G, qk_scale, images, flags));
 
   // key side: the split of the key range that minimises (waves of blocks) x (tiles per block)
   const int ktiles = (Lk + TILE - 1) / TILE;

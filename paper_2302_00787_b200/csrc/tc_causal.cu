@@ -467,14 +467,13 @@ int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int
 int make_map_kvt(CUtensorMap* map, const void* base, int BH, int bf16);
 int make_map_feat(CUtensorMap* map, const void* base, int BH, int Lpad);
 }  // namespace tchost
-int fs_tc_prep(fsharp_ctx* ctx, const float* prep, int G, float qk_scale, uint8_t* images, int* flags);
 int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                    const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax,
                    __nv_bfloat16* phik);
 int fs_tc_causal_supported(const fsharp_dims* dm, int chunk);
 size_t fs_tc_causal_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
-int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
-                 const float* prep, void* Y, WsAlloc* ws);
+int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
+                 const int* flags, void* Y, WsAlloc* ws);
 
 int fs_tc_causal_supported(const fsharp_dims* dm, int chunk) {
   if (chunk != TILE || dm->Lq != dm->Lk || dm->Lq <= 0) return 0;
@@ -491,13 +490,10 @@ size_t fs_tc_causal_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) 
          ws_round(BH * nch * TC_NV * TC_M * 2) + ws_round(BH * nch * 4);
 }
 
-int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
-                 const float* prep, void* Y, WsAlloc* ws) {
+int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
+                 const int* flags, void* Y, WsAlloc* ws) {
   const int B = dm->B, H = dm->H, BH = B * H, L = dm->Lq;
-  const int G = fs_groups(dm);
   const int nch = (L + TILE - 1) / TILE, Lpad = nch * TILE;
-  uint8_t* images = ws->take<uint8_t>((size_t)G * 2 * IMG_BYTES);
-  int* flags = ws->take<int>((size_t)G * 2 * FLAG_WORDS + 16);
   float* state = ws->take<float>((size_t)BH * nch * TC_M * TC_NV);
   float* shifts = ws->take<float>((size_t)BH * nch * 2);
   int* pmax = ws->take<int>((size_t)BH * nch * 2);
@@ -506,7 +502,6 @@ int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, c
   __nv_bfloat16* phiq16 = ws->take<__nv_bfloat16>((size_t)BH * Lpad * TC_M);
   __nv_bfloat16* prefix = ws->take<__nv_bfloat16>((size_t)BH * nch * TC_NV * TC_M);
   float* beta = ws->take<float>((size_t)BH * nch);
-  FS_TRY(fs_tc_prep(ctx, prep, G, qk_scale, images, flags));
   FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * nch * 2 * sizeof(int), ctx->stream));
 
   // query features

@@ -1,4 +1,4 @@
-// Host side of the tensor-core path: operand images, TMA descriptors, dispatch.
+// Host side of the tensor-core path: TMA descriptors and dispatch (the operand images are written by prep.cu).
 #include "common.cuh"
 #include "tc_common.cuh"
 #include "tc_layout.cuh"
@@ -8,56 +8,12 @@ using namespace tcl;
 size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
 int fs_tc_causal_supported(const fsharp_dims* dm, int chunk);
 size_t fs_tc_causal_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
-int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
-                 const float* prep, void* Y, WsAlloc* ws);
-int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, float qk_scale,
-                const float* prep, void* Y, WsAlloc* ws);
+int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
+                 const int* flags, void* Y, WsAlloc* ws);
+int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
+                const int* flags, void* Y, WsAlloc* ws);
 
 namespace {
-
-// Builds the per-(group, side) operand images from the fp32 prep block; block z converts a
-// quarter of every array.  The flag words must be zero on entry (blocks OR their bits in).
-constexpr int TCP_SPLIT = 4;
-__global__ void __launch_bounds__(256)
-tc_prep_kernel(const float* __restrict__ prep, float qk_scale, uint8_t* __restrict__ images, int* __restrict__ flags) {
-  const int g = blockIdx.x, side = blockIdx.y, z = blockIdx.z, tid = threadIdx.x;
-  PrepLayout pr{TC_D, TC_M};
-  const float* pp = prep + ((size_t)g * 2 + side) * pr.total();
-  const float* W = pp + pr.W();
-  const float* av = pp + pr.a();
-  const float* Cm = pp + pr.Cmat();
-  const float* scal = pp + pr.scal();
-  uint8_t* img = images + ((size_t)g * 2 + side) * IMG_BYTES;
-  int* fl = flags + ((size_t)g * 2 + side) * FLAG_WORDS;
-  const float sw = FS_LOG2E * qk_scale, sc = FS_LOG2E * qk_scale * qk_scale;
-  constexpr int WQ = TC_M * TC_D / TCP_SPLIT, CQ = TC_D * TC_D / TCP_SPLIT, AQ = TC_M / TCP_SPLIT;
-  // two neighbouring elements per thread: one 4-byte store into each image
-  for (int e2 = tid; e2 < WQ / 2; e2 += 256) {
-    const int e = z * WQ + 2 * e2, m = e / TC_D, k = e % TC_D;
-    const float2 w2 = *reinterpret_cast<const float2*>(W + e);
-    const float v0 = w2.x * sw, v1 = w2.y * sw;
-    const __nv_bfloat16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
-    *reinterpret_cast<__nv_bfloat162*>(img + IMG_W + tc::sw128_offset(m, k)) = __nv_bfloat162(h0, h1);
-    *reinterpret_cast<__nv_bfloat162*>(img + IMG_WLO + tc::sw128_offset(m, k)) =
-        __nv_bfloat162(__float2bfloat16_rn(v0 - __bfloat162float(h0)), __float2bfloat16_rn(v1 - __bfloat162float(h1)));
-  }
-  int lo_nonzero = 0;
-  for (int e = z * CQ + tid; e < (z + 1) * CQ; e += 256) {
-    int k = e / TC_D, n = e % TC_D;          // C[k][n] goes to row n, column k of the B operand
-    float v = Cm[e] * sc;
-    __nv_bfloat16 hi = __float2bfloat16_rn(v);
-    __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-    if (__bfloat162float(lo) != 0.f) lo_nonzero = 1;
-    *reinterpret_cast<__nv_bfloat16*>(img + IMG_CHI + tc::sw128_offset(n, k)) = hi;
-    *reinterpret_cast<__nv_bfloat16*>(img + IMG_CLO + tc::sw128_offset(n, k)) = lo;
-  }
-  if (tid < AQ) reinterpret_cast<float*>(img + IMG_A2)[z * AQ + tid] = 2.f * FS_LOG2E * av[z * AQ + tid];
-  if (__syncthreads_or(lo_nonzero) && tid == 0) atomicOr(&fl[0], FLAG_C_LO);
-  if (z == 0 && tid == 0) {
-    if (scal[PS_CSCALAR] == 0.f) atomicOr(&fl[0], FLAG_C_DENSE);
-    fl[1] = __float_as_int(scal[PS_CGAMMA] * sc);
-  }
-}
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -130,15 +86,6 @@ int make_map_feat(CUtensorMap* map, const void* base, int BH, int Lpad) {
 
 }  // namespace tchost
 
-int fs_tc_prep(fsharp_ctx* ctx, const float* prep, int G, float qk_scale, uint8_t* images, int* flags) {
-  FS_CUDA_OK(cudaMemsetAsync(flags, 0, (size_t)G * 2 * FLAG_WORDS * sizeof(int), ctx->stream));
-  FS_TIME_BEGIN(ctx, FS_K_TC_PREP);
-  tc_prep_kernel<<<dim3(G, 2, TCP_SPLIT), 256, 0, ctx->stream>>>(prep, qk_scale, images, flags);
-  FS_TIME_END(ctx);
-  FS_LAUNCH_CHECK(ctx);
-  return FSHARP_OK;
-}
-
 int fs_tc_supported(const fsharp_dims* dm, int dtype, int causal, int chunk, float qk_scale) {
   (void)chunk;
   (void)qk_scale;
@@ -155,8 +102,8 @@ size_t fs_tc_attend_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm, 
 }
 
 int fs_tc_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, int causal,
-                 int chunk, float qk_scale, const float* prep, void* Y, WsAlloc* ws) {
+                 int chunk, const uint8_t* images, const int* flags, void* Y, WsAlloc* ws) {
   (void)chunk;
-  if (causal) return fs_tc_causal(ctx, Q, K, V, dm, qk_scale, prep, Y, ws);
-  return fs_tc_bidir(ctx, Q, K, V, dm, qk_scale, prep, Y, ws);
+  if (causal) return fs_tc_causal(ctx, Q, K, V, dm, images, flags, Y, ws);
+  return fs_tc_bidir(ctx, Q, K, V, dm, images, flags, Y, ws);
 }
