@@ -48,7 +48,9 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
     const int m = e % PREP_MB, i = e / PREP_MB;
     Ot[i * PREP_LDO + m] = (m0 + m < M) ? Om[(size_t)(m0 + m) * d + i] : 0.f;
   }
-  for (int pass = 0; pass < 2; pass++) {      // pass 0: W = Omega B, pass 1: a = diag(Omega A Omega^T)
+  // pass 0: W = Omega B; pass 1: a = diag(Omega A Omega^T), which is the same for both sides: the
+  // side-1 block computes it and writes it for both
+  for (int pass = 0; pass < (side == 1 ? 2 : 1); pass++) {
     const double* Mat = pass == 0 ? Bm : A;
     __syncthreads();
     for (int e = tid; e < d * d; e += PREP_THREADS) Ms[e] = (float)Mat[e];
@@ -109,8 +111,11 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
         for (int o = 8; o > 0; o >>= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, o);
         if (tx == 0 && m < M) {
           av[m] = sacc;
-          if (images != nullptr)
-            reinterpret_cast<float*>(images + ((size_t)g * 2 + (side - 1)) * tcl::IMG_BYTES + tcl::IMG_A2)[m] = 2.f * FS_LOG2E * sacc;
+          av[pr.total() + m] = sacc;          // side 2's copy
+          if (images != nullptr) {
+            reinterpret_cast<float*>(images + ((size_t)g * 2 + 0) * tcl::IMG_BYTES + tcl::IMG_A2)[m] = 2.f * FS_LOG2E * sacc;
+            reinterpret_cast<float*>(images + ((size_t)g * 2 + 1) * tcl::IMG_BYTES + tcl::IMG_A2)[m] = 2.f * FS_LOG2E * sacc;
+          }
         }
       }
     }

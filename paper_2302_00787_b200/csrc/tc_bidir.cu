@@ -4,10 +4,10 @@
 //                               phi = 2^(logits + c_j - s)  -> bf16 tile in shared memory
 //                               KV^T += [V | 1]^T phi                        (tcgen05, TMEM)
 //                               (c_j, the key's quadratic term, comes from tc_rowterm_kernel)
-//   merge      (tc_merge_kernel): partial KV^T of the splits of one (batch, head), brought to a
-//                               common shift, summed, every feature's column scaled to order one
-//                               (fp16); the scales' exponents g, with a2, go to the query side
-//   query side (tc_out_kernel): logits + g, phi = 2^(... - max of the half row) in fp16,
+//   query side (tc_out_kernel): first the merge of the key-side partials of its (batch, head): common
+//                               shift, sum, every feature's column scaled to order one (fp16), the
+//                               scales' exponents g (with a2) kept for the logits; then per tile
+//                               logits + g, phi = 2^(... - max of the half row) in fp16,
 //                               [num | den] = phi KV per feature half, halves combined, Y = num / den
 //
 // The feature tiles never leave the SM.  One block = 8 epilogue warps (exponentials), one
@@ -26,6 +26,7 @@ using namespace tcl;
 
 namespace {
 
+constexpr int MAX_KEY_SPLIT = 64;    // splits of the key range of one (batch, head)
 constexpr int PREFETCH_TILES = 4;   // tiles pulled into L2 ahead of the shared-memory ring
 
 // ------------------------------------------------------------------------------------------
@@ -375,71 +376,16 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 }
 
 // ------------------------------------------------------------------------------------------
-// merge of the key-side partials of one (batch, head): common shift, sum, and a scale of its own
-// for every feature.  Partials and result are both [80 rows][256 features].
-//
-// The query side contracts phi(Q) with this state in fp16, whose exponent range is narrow, and what
-// a feature contributes to an output is phi(Q)_m times the size of column m of the state.  So every
-// column m is brought to order one by a power of two 2^-e_m, and g_m = e_m + a2_m - max a2 (the
-// per-feature term w^T A w of both sides rides along) is handed to the query side, which adds it
-// to its logits BEFORE it takes the row maximum: a query feature near 1 is then one that matters,
-// and what underflows in either operand is negligible by construction.
-// ------------------------------------------------------------------------------------------
-constexpr int MERGE_THREADS = 1024, MERGE_ROWS = (TC_DV + 4) / 4;       // thread = (feature, one row in four)
-__global__ void __launch_bounds__(MERGE_THREADS)
-tc_merge_kernel(const float* __restrict__ partial, const float* __restrict__ shifts, int nsplit,
-                const uint8_t* __restrict__ images, int H, int pool, __half* __restrict__ kvt, float* __restrict__ gq) {
-  __shared__ float fac[2 * 64];
-  __shared__ float red[MERGE_THREADS];
-  const int bh = blockIdx.x;
-  const int g = pool == FSHARP_POOL_PER_BH ? bh : bh % H;
-  const int m = threadIdx.x & (TC_M - 1), qt = threadIdx.x >> 8, hh = m >> 7;
-  const float* a2 = reinterpret_cast<const float*>(images + (size_t)g * 2 * IMG_BYTES + IMG_A2);
-  const float a2m = a2[m];
-  red[threadIdx.x] = a2m;
-  if (threadIdx.x < 2 * nsplit) fac[threadIdx.x] = shifts[(size_t)bh * nsplit * 2 + threadIdx.x];
-  __syncthreads();
-  for (int s = 128; s > 0; s >>= 1) {
-    if (threadIdx.x < s) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + s]);
-    __syncthreads();
-  }
-  const float a2max = red[0];
-  float smax = -INFINITY;
-  for (int p = 0; p < 2 * nsplit; p++) smax = fmaxf(smax, fac[p]);
-  __syncthreads();
-  if (threadIdx.x < 2 * nsplit) fac[threadIdx.x] = exp2f(fac[threadIdx.x] - smax);
-  __syncthreads();
-  const float* base = partial + (size_t)bh * nsplit * TC_NV * TC_M;
-  float val[MERGE_ROWS];
-  float amax = 0.f;
-#pragma unroll
-  for (int u = 0; u < MERGE_ROWS; u++) {
-    const int n = qt + 4 * u;
-    float acc = 0.f;
-    if (n <= TC_DV)
-      for (int p = 0; p < nsplit; p++) acc = fmaf(base[((size_t)p * TC_NV + n) * TC_M + m], fac[2 * p + hh], acc);
-    val[u] = acc;
-    amax = fmaxf(amax, fabsf(acc));
-  }
-  red[threadIdx.x] = amax;
-  __syncthreads();
-  amax = fmaxf(fmaxf(red[m], red[TC_M + m]), fmaxf(red[2 * TC_M + m], red[3 * TC_M + m]));
-  int ex = 0;
-  if (amax > 0.f && isfinite(amax)) frexpf(amax, &ex);          // amax = f 2^ex, f in [1/2, 1)
-  const float sc = exp2f((float)-ex);
-  __half* out = kvt + (size_t)bh * TC_NV * TC_M;
-#pragma unroll
-  for (int u = 0; u < MERGE_ROWS; u++) {
-    const int n = qt + 4 * u;
-    if (n <= TC_DV) out[(size_t)n * TC_M + m] = __float2half_rn(val[u] * sc);
-  }
-  for (int n = TC_DV + 1 + qt; n < TC_NV; n += 4) out[(size_t)n * TC_M + m] = __float2half_rn(0.f);     // padding rows
-  if (qt == 0) gq[(size_t)bh * TC_M + m] = (float)ex + a2m - a2max;
-}
-
-// ------------------------------------------------------------------------------------------
 // query side
 // ------------------------------------------------------------------------------------------
+// Every block first merges the key-side partials of its (batch, head) into shared memory: common
+// shift, sum over the splits, and a scale of its own for every feature.  The query side contracts
+// phi(Q) with this state in fp16, whose exponent range is narrow, and what a feature contributes to
+// an output is phi(Q)_m times the size of column m of the state.  So every column m is brought to
+// order one by a power of two 2^-e_m, and g_m = e_m + a2_m - max a2 (the per-feature term w^T A w
+// of both sides rides along) is added to the query logits BEFORE the row maximum is taken: a query
+// feature near 1 is then one that matters, and what underflows in either operand is negligible by
+// construction.
 constexpr int OUT_STAGES = 2;
 struct OutSmem {
   static constexpr uint32_t X0 = 0, W = OUT_STAGES * TILE_BYTES, WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES,
@@ -461,8 +407,9 @@ struct OutMisc {
 constexpr uint32_t OUT_COL_LOGITS = 0, OUT_COL_OUT = 256;
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
-tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKVt,
-              const uint8_t* __restrict__ images, const float* __restrict__ gq, int H, int pool, int L, int tiles_per_split,
+tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict__ images,
+              const float* __restrict__ partial, const float* __restrict__ shifts, int nsplit, int H, int pool, int L,
+              int tiles_per_split,
               __nv_bfloat16* __restrict__ Y, TensorAddr ay, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -478,7 +425,6 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
   const uint8_t* img = images + ((size_t)g * 2 + 0) * IMG_BYTES;        // side 1 (queries)
   volatile int* abortp = &misc->abort_flag;
 
-  if (threadIdx.x < TC_M) gs[threadIdx.x] = gq[(size_t)bh * TC_M + threadIdx.x];
   if (threadIdx.x == 0) {
     for (int i = 0; i < OUT_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], 1); }
     mbar_init(&misc->logits_full, 1);
@@ -503,13 +449,9 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
   if (warp == WARP_TMA) {
     if (lane == 0) {
       prefetch_tmap(&tmQ);
-      prefetch_tmap(&tmKVt);
-      mbar_expect_tx(&misc->const_bar, 2 * IMG_W_BYTES + KVT_BYTES);
+      mbar_expect_tx(&misc->const_bar, 2 * IMG_W_BYTES);
       bulk_load(sm + OutSmem::W, img + IMG_W, IMG_W_BYTES, &misc->const_bar);
       bulk_load(sm + OutSmem::WLO, img + IMG_WLO, IMG_W_BYTES, &misc->const_bar);
-#pragma unroll
-      for (int fb = 0; fb < TC_M / 64; fb++)
-        tma_load_3d(sm + OutSmem::KVT + fb * KVT_BLOCK_BYTES, &tmKVt, &misc->const_bar, fb * 64, 0, bh);
       for (int it = 0; it < min(ntiles, PREFETCH_TILES); it++) tma_prefetch_4d(&tmQ, 0, (tile0 + it) * TILE, h, b);
       int issued = 0;
       for (int it = 0; it < ntiles; it++) {
@@ -586,6 +528,49 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
     __nv_bfloat16* Yb = Y + b * ay.sb + h * ay.sh;
     bool alive = true;
+    {
+      // merge (see above); thread = feature m, whose half (m / 128) is also the thread's half below, so the
+      // arrivals that release a 64-feature block to the MMA warp cover the writers of that block of the state
+      const int m = threadIdx.x, hh = m >> 7;
+      float* sft = reinterpret_cast<float*>(sm + OutSmem::STAGE);        // shifts, then their factors (the stage is idle)
+      float* red = sft + 2 * MAX_KEY_SPLIT;
+      const float a2m = reinterpret_cast<const float*>(img + IMG_A2)[m];
+      float wmx = a2m;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) wmx = fmaxf(wmx, __shfl_xor_sync(0xffffffffu, wmx, o));
+      if (lane == 0) red[warp] = wmx;
+      if (m < 2 * nsplit) sft[m] = shifts[(size_t)bh * nsplit * 2 + m];
+      named_bar_sync(1, EPI_THREADS);
+      float a2max = red[0], smax = -INFINITY;
+#pragma unroll
+      for (int i = 1; i < EPI_THREADS / 32; i++) a2max = fmaxf(a2max, red[i]);
+      for (int p = 0; p < 2 * nsplit; p++) smax = fmaxf(smax, sft[p]);
+      named_bar_sync(1, EPI_THREADS);
+      if (m < 2 * nsplit) sft[m] = exp2f(sft[m] - smax);
+      named_bar_sync(1, EPI_THREADS);
+      const float* base = partial + (size_t)bh * nsplit * TC_NV * TC_M + m;
+      float val[TC_DV + 1];
+#pragma unroll
+      for (int n = 0; n <= TC_DV; n++) val[n] = 0.f;
+      for (int p = 0; p < nsplit; p++) {        // 65 independent loads in flight per split
+        const float f = sft[2 * p + hh];
+        const float* bp = base + (size_t)p * TC_NV * TC_M;
+#pragma unroll
+        for (int n = 0; n <= TC_DV; n++) val[n] = fmaf(bp[n * TC_M], f, val[n]);
+      }
+      float amax = 0.f;
+#pragma unroll
+      for (int n = 0; n <= TC_DV; n++) amax = fmaxf(amax, fabsf(val[n]));
+      int ex = 0;
+      if (amax > 0.f && isfinite(amax)) frexpf(amax, &ex);          // amax = f 2^ex, f in [1/2, 1)
+      const float sc = exp2f((float)-ex);
+      uint8_t* kcol = sm + OutSmem::KVT + (m >> 6) * KVT_BLOCK_BYTES;
+#pragma unroll
+      for (int n = 0; n < TC_NV; n++)
+        *reinterpret_cast<__half*>(kcol + sw128_offset(n, m & 63)) = __float2half_rn(n <= TC_DV ? val[n <= TC_DV ? n : 0] * sc : 0.f);
+      gs[m] = (float)ex + a2m - a2max;
+      named_bar_sync(1, EPI_THREADS);
+    }
     // Y rows of tile j (its contraction has completed): 32 of the 64 columns per thread
     auto write_out = [&](int j) {
       __syncwarp();
@@ -722,7 +707,6 @@ int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_d
                    const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax,
                    __nv_bfloat16* phik);
 
-constexpr int MAX_KEY_SPLIT = 64;
 
 size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
   const size_t BH = (size_t)dm->B * dm->H;
@@ -772,25 +756,17 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * MAX_KEY_SPLIT * 2 * sizeof(int), ctx->stream));
   const int Lpad = ktiles * TILE;
   float* crow = ws->take<float>((size_t)BH * Lpad);
-  __half* kvt = ws->take<__half>((size_t)BH * TC_NV * TC_M);
-  float* gq = ws->take<float>((size_t)BH * TC_M);
   FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, tps, nsplit, crow, partial, shifts, pmax, nullptr));
 
-  CUtensorMap tmQ, tmKVt;
+  CUtensorMap tmQ;
   FS_TRY(tchost::make_map_tokens(&tmQ, Q, fs_addr(dm->q_stride, H, Lq, dm->d), B, H, Lq, dm->d));
-  FS_TRY(tchost::make_map_kvt(&tmKVt, kvt, BH, 0));
   FS_CUDA_OK(cudaFuncSetAttribute(tc_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OutSmem::TOTAL + 1024));
-  FS_TIME_BEGIN(ctx, FS_K_TC_MERGE);
-  tc_merge_kernel<<<BH, MERGE_THREADS, 0, ctx->stream>>>(partial, shifts, nsplit, images, H, dm->pool, kvt, gq);
-  FS_TIME_END(ctx);
-  FS_LAUNCH_CHECK(ctx);
-
   const int qtiles = (Lq + TILE - 1) / TILE;
   int qtps = 0;
   int qsplit = pick_split(BH, qtiles, ctx->sm_count, 1 << 20, &qtps);
   FS_TIME_BEGIN(ctx, FS_K_TC_OUT);
   tc_out_kernel<<<dim3(qsplit, BH), TC_THREADS, OutSmem::TOTAL + 1024, ctx->stream>>>(
-      tmQ, tmKVt, images, gq, H, dm->pool, Lq, qtps, (__nv_bfloat16*)Y, fs_addr(dm->y_stride, H, Lq, dm->dv), ctx->d_status);
+      tmQ, images, partial, shifts, nsplit, H, dm->pool, Lq, qtps, (__nv_bfloat16*)Y, fs_addr(dm->y_stride, H, Lq, dm->dv), ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;
