@@ -177,12 +177,22 @@ int fsharp_forward_host(fsharp_ctx* ctx, const void* Q, const void* K, const voi
   float* dO = ws.take<float>((size_t)dd.M * dd.d);
   double* dS = ws.take<double>(nstats / 8);
   double* dP = ws.take<double>(nparams / 8);
+  if (!ctx->copy_stream) {
+    FS_CUDA_OK(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+    FS_CUDA_OK(cudaEventCreateWithFlags(&ctx->ev_inputs, cudaEventDisableTiming));
+    FS_CUDA_OK(cudaEventCreateWithFlags(&ctx->ev_v, cudaEventDisableTiming));
+  }
+  // Q, K and Omega go up first; V follows on a stream of its own while statistics and fit run
   FS_CUDA_OK(cudaMemcpyAsync(dQ, Q, nq, cudaMemcpyHostToDevice, ctx->stream));
   FS_CUDA_OK(cudaMemcpyAsync(dK, K, nk, cudaMemcpyHostToDevice, ctx->stream));
-  FS_CUDA_OK(cudaMemcpyAsync(dV, V, nv, cudaMemcpyHostToDevice, ctx->stream));
   FS_CUDA_OK(cudaMemcpyAsync(dO, Omega, no, cudaMemcpyHostToDevice, ctx->stream));
+  FS_CUDA_OK(cudaEventRecord(ctx->ev_inputs, ctx->stream));
+  FS_CUDA_OK(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_inputs, 0));
+  FS_CUDA_OK(cudaMemcpyAsync(dV, V, nv, cudaMemcpyHostToDevice, ctx->copy_stream));
+  FS_CUDA_OK(cudaEventRecord(ctx->ev_v, ctx->copy_stream));
   FS_TRY(fsharp_stats(ctx, dQ, dK, &dd, dtype, qk_scale, dS));
   FS_TRY(fsharp_fit_params(ctx, dS, G, dd.d, variant, 0.0, dP));
+  FS_CUDA_OK(cudaStreamWaitEvent(ctx->stream, ctx->ev_v, 0));
   FS_TRY(fsharp_attend(ctx, dQ, dK, dV, dO, dP, &dd, dtype, causal, chunk, qk_scale, dY));
   FS_CUDA_OK(cudaMemcpyAsync(Y, dY, ny, cudaMemcpyDeviceToHost, ctx->stream));
   FS_CUDA_OK(cudaStreamSynchronize(ctx->stream));

@@ -69,6 +69,9 @@ struct fsharp_ctx {
   int t_used;
   cudaEvent_t* t_ev;  // 2 * FS_TIMING_SLOTS, created on first use
   int* t_tag;
+  // second stream and two events of fsharp_forward_host (V is uploaded while statistics and fit run); created on first use
+  cudaStream_t copy_stream;
+  cudaEvent_t ev_inputs, ev_v;
 };
 
 void fs_time_begin(fsharp_ctx* ctx, int tag);

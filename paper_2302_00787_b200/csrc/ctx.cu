@@ -28,6 +28,9 @@ int fsharp_create(fsharp_ctx** out, int device, void* stream) {
   c->t_used = 0;
   c->t_ev = nullptr;
   c->t_tag = nullptr;
+  c->copy_stream = nullptr;
+  c->ev_inputs = nullptr;
+  c->ev_v = nullptr;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) == cudaSuccess) c->sm_count = prop.multiProcessorCount;
   if (cudaMalloc(&c->d_status, sizeof(int)) != cudaSuccess) {
@@ -51,6 +54,12 @@ int fsharp_destroy(fsharp_ctx* ctx) {
   cudaStreamSynchronize(ctx->stream);
   if (ctx->ws) cudaFree(ctx->ws);
   if (ctx->d_status) cudaFree(ctx->d_status);
+  if (ctx->copy_stream) {
+    cudaStreamSynchronize(ctx->copy_stream);
+    cudaStreamDestroy(ctx->copy_stream);
+    cudaEventDestroy(ctx->ev_inputs);
+    cudaEventDestroy(ctx->ev_v);
+  }
   if (ctx->t_ev) {
     for (int i = 0; i < 2 * FS_TIMING_SLOTS; i++) cudaEventDestroy(ctx->t_ev[i]);
     delete[] ctx->t_ev;

@@ -98,6 +98,9 @@ extern "C" int fsharp_featurize_static(void* stream, const void* X, const float*
   ctx.t_used = 0;
   ctx.t_ev = nullptr;
   ctx.t_tag = nullptr;
+  ctx.copy_stream = nullptr;
+  ctx.ev_inputs = nullptr;
+  ctx.ev_v = nullptr;
 
   WsAlloc ws{ctx.ws, 0};
   float* prep = ws.take<float>(prep_f);
