@@ -252,7 +252,9 @@ __device__ __forceinline__ int jacobi_role(const JacobiCtx& jc_in, int* final_bu
   // of a block per thread), the others share the rest
   constexpr int VT_ITEMS = (3 * VT_THREADS / 4) < ntri ? 3 * VT_THREADS / 4 : ntri;
   const int tid = threadIdx.x, lda = jc.lda;
-  const int vcol = (tid - 32) >> 1, vh = (tid - 32) & 1;  // JR_VT: column of V^T and which half of its seats
+  // JR_VT: column of V^T and which half of its seats.  The two halves of a column sit 16 lanes apart, so that
+  // the eight lanes that share a shared-memory transaction read the same rotation (one broadcast, no bank conflict).
+  const int vcol = ((tid - 32) >> 5) * 16 + (tid & 15), vh = (tid >> 4) & 1;
   const int a_first = ROLE == JR_A ? tid - 32 - VT_THREADS : ntri - VT_ITEMS + (tid - 32);
   const int a_last = ROLE == JR_A ? ntri - VT_ITEMS : ntri;
   constexpr int a_step = ROLE == JR_A ? NA : VT_THREADS;
@@ -332,7 +334,7 @@ __device__ __forceinline__ int jacobi_role(const JacobiCtx& jc_in, int* final_bu
         // Even seats move down by two, odd seats up by two; seat 1 is fixed, seat 0 goes to seat 3,
         // the last odd seat to the last even one.  Two values cross between the halves of a column.
         const double send = vh ? x[0] : x[N2 - 1];
-        const double recv = __shfl_xor_sync(0xffffffffu, send, 1);
+        const double recv = __shfl_xor_sync(0xffffffffu, send, 16);
         const double t0 = x[0];
 #pragma unroll
         for (int j = 0; j <= N2 - 4; j += 2) x[j] = x[j + 2];
