@@ -421,6 +421,306 @@ __device__ __forceinline__ void smem_product(int d, FA a, FB b, FO out) {
   }
 }
 
+// ---- direct eigensolver for d <= 64 --------------------------------------------------------------
+// Householder tridiagonalisation, eigenvalues of the tridiagonal matrix by multisection on Sturm
+// counts, one eigenvector per eigenvalue from the twisted factorisation of T - sigma I, the
+// reflectors applied back, one first-order symmetric orthogonalisation, and A' = V^T A V.  The
+// Jacobi solver then starts from A', which is diagonal to rounding whenever the eigenvalues are
+// separated, and checks (or completes) the result with its own convergence test: the accuracy is
+// that of the Jacobi solver, the cost that of a few matrix products.  Vectors that fail the
+// orthogonality check (eigenvalues that agree to rounding, a matrix that splits) make the
+// function return false with A restored; the caller then runs the Jacobi solver on A itself.
+//
+// Thread t = (row or vector r = t / P, part = t % P) with P = FIT_THREADS / D lanes of one warp
+// sharing every reduction.
+template <int D>
+__device__ __forceinline__ bool direct_eig(double* __restrict__ As, double* __restrict__ A1, double* __restrict__ Vs,
+                                           double* __restrict__ Ws, int lda, double* __restrict__ dd,
+                                           double* __restrict__ ee, double* __restrict__ beta, double* red) {
+  constexpr int P = FIT_THREADS / D, NU = (D + P - 1) / P;
+  static_assert(P >= 8 && P <= 32, "lanes per vector");
+  const int tid = threadIdx.x, r = tid / P, part = tid % P;
+  auto gsum = [](double v) {
+#pragma unroll
+    for (int o = P >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+  };
+  for (int e = tid; e < D * D; e += FIT_THREADS) Ws[(e / D) * lda + (e % D)] = As[(e / D) * lda + (e % D)];
+
+  // 1. A -> Q^T A Q = T (tridiagonal).  Reflector k, I - beta_k v v^T, acts on indices k+1..D-1; v is kept in
+  //    column k of A below the diagonal.
+  for (int k = 0; k < D - 2; k++) {
+    const int n = D - k - 1;
+    double* xc = As + (k + 1) * lda + k;              // x_i = xc[i * lda]
+    double* A22 = As + (k + 1) * lda + (k + 1);
+    double vj[NU], s2 = 0.0;
+#pragma unroll
+    for (int u = 0; u < NU; u++) {
+      const int j = part + u * P;
+      vj[u] = j < n ? xc[j * lda] : 0.0;
+      if (j >= 1) s2 = fma(vj[u], vj[u], s2);
+    }
+    s2 = gsum(s2);
+    const double x0 = xc[0];
+    double vr = r < n ? xc[r * lda] : 0.0;
+    double b = 0.0, alpha = x0, v0 = x0;
+    if (s2 > 0.0) {
+      alpha = -copysign(sqrt(fma(x0, x0, s2)), x0);
+      v0 = x0 - alpha;
+      b = -1.0 / (alpha * v0);
+      if (part == 0) vj[0] = v0;
+      if (r == 0) vr = v0;
+    }
+    // p = beta A22 v
+    double pr = 0.0;
+    if (r < n) {
+#pragma unroll
+      for (int u = 0; u < NU; u++) {
+        const int j = part + u * P;
+        if (j < n) pr = fma(A22[r * lda + j], vj[u], pr);
+      }
+    }
+    pr = gsum(pr) * b;
+    if (part == 0 && r < n) red[r] = pr;
+    __syncthreads();
+    if (tid == 0) { ee[k] = alpha; beta[k] = b; dd[k] = As[k * lda + k]; xc[0] = v0; }
+    // w = p - (beta/2 v.p) v ;  A22 -= v w^T + w v^T
+    double pj[NU], kk = 0.0;
+#pragma unroll
+    for (int u = 0; u < NU; u++) {
+      const int j = part + u * P;
+      pj[u] = j < n ? red[j] : 0.0;
+      kk = fma(vj[u], pj[u], kk);
+    }
+    kk = gsum(kk) * (0.5 * b);
+    if (r < n && b != 0.0) {
+      const double wr = fma(-kk, vr, pr);
+#pragma unroll
+      for (int u = 0; u < NU; u++) {
+        const int j = part + u * P;
+        if (j < n) {
+          const double wj = fma(-kk, vj[u], pj[u]);
+          A22[r * lda + j] -= fma(vr, wj, wr * vj[u]);
+        }
+      }
+    }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    dd[D - 2] = As[(D - 2) * lda + (D - 2)];
+    dd[D - 1] = As[(D - 1) * lda + (D - 1)];
+    ee[D - 2] = As[(D - 1) * lda + (D - 2)];
+    ee[D - 1] = 0.0;
+  }
+  __syncthreads();
+
+  // 2. Eigenvalues of T.  Gershgorin interval, T scaled by a power of two so that it is of order one (the
+  //    vectors do not change; the final eigenvalues are read from A' later).
+  double lo = 1e300, hi = -1e300;
+#pragma unroll
+  for (int u = 0; u < NU; u++) {
+    const int i = part + u * P;
+    if (i < D) {
+      const double rad = fabs(ee[i]) + (i > 0 ? fabs(ee[i - 1]) : 0.0);
+      lo = fmin(lo, dd[i] - rad);
+      hi = fmax(hi, dd[i] + rad);
+    }
+  }
+#pragma unroll
+  for (int o = P >> 1; o > 0; o >>= 1) {
+    lo = fmin(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+    hi = fmax(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+  }
+  const double nrm = fmax(fabs(lo), fabs(hi));
+  if (!(nrm > 1e-290) || !(nrm < 1e290)) {            // zero, non-finite or absurdly scaled: leave it to the caller
+    __syncthreads();
+    for (int e = tid; e < D * D; e += FIT_THREADS) As[(e / D) * lda + (e % D)] = Ws[(e / D) * lda + (e % D)];
+    __syncthreads();
+    return false;
+  }
+  const int nex = ((__double2hiint(nrm) >> 20) & 0x7ff) - 1023;
+  const double sc = __hiloint2double((1023 - nex) << 20, 0);         // 2^-nex: nrm * sc in [1, 2)
+  __syncthreads();
+  if (tid < D) { dd[tid] *= sc; ee[tid] *= sc; }
+  __syncthreads();
+  lo *= sc; hi *= sc;
+  // number of eigenvalues below x: sign changes of the leading principal minors p_i of T - x I,
+  // p_i = (d_i - x) p_{i-1} - e_{i-1}^2 p_{i-2}; a zero minor takes the sign opposite to its predecessor.
+  auto below = [&](double x) {
+    double pm2 = 1.0, pm1 = dd[0] - x;
+    bool neg_prev = (pm1 < 0.0) || (pm1 == 0.0);
+    int c = neg_prev ? 1 : 0;
+#pragma unroll 8
+    for (int i = 1; i < D; i++) {
+      const double e = ee[i - 1];
+      const double p = fma(dd[i] - x, pm1, -(e * e) * pm2);
+      const bool neg = (p < 0.0) || (p == 0.0 && !neg_prev);
+      c += neg != neg_prev;
+      neg_prev = neg;
+      pm2 = pm1; pm1 = p;
+      if ((i & 7) == 0) {                             // keep the pair of minors of order one
+        const double m = fmax(fabs(pm1), fabs(pm2));
+        const int ex = (__double2hiint(m) >> 20) & 0x7ff;
+        if (ex > 0 && ex < 0x7fe) {
+          const double s = __hiloint2double((2046 - ex) << 20, 0);
+          pm1 *= s; pm2 *= s;
+        }
+      }
+    }
+    return c;
+  };
+  double sigma;
+  {
+    constexpr int NIT = P == 8 ? 18 : (P == 16 ? 14 : 12);             // (P + 1)^NIT > 2^54
+    double a = lo - 0.001 * (hi - lo) - 1e-3, bq = hi + 0.001 * (hi - lo) + 1e-3;
+    const unsigned gshift = (tid & 31) / P * P;
+    for (int it = 0; it < NIT; it++) {
+      const double h = (bq - a) * (1.0 / (P + 1));
+      const double x = fma(h, (double)(part + 1), a);
+      const bool above = below(x) >= r + 1;           // at least r + 1 eigenvalues lie below x
+      unsigned mask = __ballot_sync(0xffffffffu, above) >> gshift;
+      if (P < 32) mask &= (1u << P) - 1u;
+      const int first = mask ? __ffs(mask) - 1 : P;   // first point with the r-th eigenvalue below it
+      const double na = first > 0 ? fma(h, (double)first, a) : a;
+      const double nb = first < P ? fma(h, (double)(first + 1), a) : bq;
+      a = na; bq = nb;
+    }
+    sigma = 0.5 * (a + bq);
+  }
+
+  // 3. Eigenvector of T for sigma from the twisted factorisation: pivots of the elimination from the top
+  //    (D+) and from the bottom (D-), gamma_i = D+_i + D-_i - (d_i - sigma); the vector starts with 1 at the
+  //    index of the smallest |gamma| and runs outwards with the multipliers of the two eliminations.
+  //    Pivots below 2^-64 (T is of order one) are replaced by -2^-64.
+  constexpr double PIVMIN = 5.421010862427522e-20;
+  double* Dp = A1 + r * lda;                          // D+ of this vector, later the vector itself
+  double* Dm = Vs + r * lda;
+  if (part < 2) {
+    if (part == 0) {
+      double t = dd[0] - sigma;
+      for (int i = 0; i < D - 1; i++) {
+        if (fabs(t) < PIVMIN) t = -PIVMIN;
+        Dp[i] = t;
+        const double e = ee[i];
+        t = fma(-e, e / t, dd[i + 1] - sigma);
+      }
+      Dp[D - 1] = t;
+    } else {
+      double t = dd[D - 1] - sigma;
+      for (int i = D - 1; i > 0; i--) {
+        if (fabs(t) < PIVMIN) t = -PIVMIN;
+        Dm[i] = t;
+        const double e = ee[i - 1];
+        t = fma(-e, e / t, dd[i - 1] - sigma);
+      }
+      Dm[0] = t;
+    }
+  }
+  __syncwarp();
+  double gbest = 1e300;
+  int ibest = 0;
+#pragma unroll
+  for (int u = 0; u < NU; u++) {
+    const int i = part + u * P;
+    if (i < D) {
+      const double g = fabs(Dp[i] + Dm[i] - (dd[i] - sigma));
+      if (g < gbest) { gbest = g; ibest = i; }        // NaN never wins
+    }
+  }
+#pragma unroll
+  for (int o = P >> 1; o > 0; o >>= 1) {
+    const double go = __shfl_xor_sync(0xffffffffu, gbest, o);
+    const int io = __shfl_xor_sync(0xffffffffu, ibest, o);
+    if (go < gbest || (go == gbest && io < ibest)) { gbest = go; ibest = io; }
+  }
+  __syncwarp();
+  double zz = 0.0;
+  if (part == 0) {
+    double z = 1.0;
+    zz = 1.0;
+    for (int i = ibest - 1; i >= 0; i--) {
+      z = -(ee[i] / Dp[i]) * z;
+      Dp[i] = z;
+      zz = fma(z, z, zz);
+    }
+  } else if (part == 1) {
+    double z = 1.0;
+    for (int i = ibest; i < D - 1; i++) {
+      z = -(ee[i] / Dm[i + 1]) * z;
+      Dp[i + 1] = z;
+      zz = fma(z, z, zz);
+    }
+  }
+  if (part == 0) Dp[ibest] = 1.0;
+  zz = gsum(zz);
+  __syncwarp();
+  const double zn = rsqrt(zz);
+  double z[NU];
+#pragma unroll
+  for (int u = 0; u < NU; u++) {
+    const int i = part + u * P;
+    z[u] = i < D ? Dp[i] * zn : 0.0;
+  }
+  __syncthreads();                                    // every vector is in registers: A1 and Vs are free
+
+  // 4. Eigenvector of A = Q z: the reflectors in reverse order, each vector within its own lanes.
+  for (int k = D - 3; k >= 0; k--) {
+    const double b = beta[k];
+    if (b == 0.0) continue;
+    const double* vc = As + k;                        // v_i = vc[i * lda], i > k
+    double vi[NU], dot = 0.0;
+#pragma unroll
+    for (int u = 0; u < NU; u++) {
+      const int i = part + u * P;
+      vi[u] = (i > k && i < D) ? vc[i * lda] : 0.0;
+      dot = fma(vi[u], z[u], dot);
+    }
+    dot = gsum(dot) * b;
+#pragma unroll
+    for (int u = 0; u < NU; u++) z[u] = fma(-dot, vi[u], z[u]);
+  }
+#pragma unroll
+  for (int u = 0; u < NU; u++) {
+    const int i = part + u * P;
+    if (i < D) Vs[r * lda + i] = z[u];                // row r of Vs: the r-th vector
+  }
+  __syncthreads();
+
+  // 5. G = V V^T - I (rows are the vectors) -> A1; give up unless the vectors are orthonormal to 1e-6.
+  double gmax = 0.0;
+  smem_product(D, [&](int i, int k) { return Vs[i * lda + k]; }, [&](int k, int j) { return Vs[j * lda + k]; },
+               [&](int i, int j, double v) {
+                 v -= (i == j) ? 1.0 : 0.0;
+                 A1[i * lda + j] = v;
+                 gmax = fmax(gmax, isfinite(v) ? fabs(v) : 1e300);
+               });
+  gmax = block_reduce(gmax, red, 1);
+  if (!(gmax <= 1e-6)) {
+    for (int e = tid; e < D * D; e += FIT_THREADS) As[(e / D) * lda + (e % D)] = Ws[(e / D) * lda + (e % D)];
+    __syncthreads();
+    return false;
+  }
+  // V <- (I - G/2) V -> As: orthonormal to second order in G
+  smem_product(D, [&](int j, int i) { return A1[j * lda + i]; }, [&](int i, int c) { return Vs[i * lda + c]; },
+               [&](int j, int c, double v) { As[j * lda + c] = fma(-0.5, v, Vs[j * lda + c]); });
+  __syncthreads();
+  // V A -> A1, then A' = (V A) V^T -> Vs
+  smem_product(D, [&](int j, int k) { return As[j * lda + k]; }, [&](int k, int m) { return Ws[k * lda + m]; },
+               [&](int j, int m, double v) { A1[j * lda + m] = v; });
+  __syncthreads();
+  smem_product(D, [&](int i, int m) { return A1[i * lda + m]; }, [&](int m, int j) { return As[j * lda + m]; },
+               [&](int i, int j, double v) { Vs[i * lda + j] = v; });
+  __syncthreads();
+  // A' -> As, V -> Ws
+  for (int e = tid; e < D * D; e += FIT_THREADS) {
+    const int o = (e / D) * lda + (e % D);
+    Ws[o] = As[o];
+    As[o] = Vs[o];
+  }
+  __syncthreads();
+  return true;
+}
+
 struct FitArgs {
   const double* stats;
   double* params;
@@ -467,12 +767,29 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
   auto eig = [&]() -> int {
     if (!V_IN_SMEM) return jacobi_eig(As, lda, Vs, ldv, d, log2d, sched, cs, red);
     int buf = 0, n = 0;
+    bool direct;
+    if (d == 64) direct = direct_eig<64>(As, A1, Vs, Ws, lda, lam, aux, cs, red);
+    else if (d == 32) direct = direct_eig<32>(As, A1, Vs, Ws, lda, lam, aux, cs, red);
+    else direct = direct_eig<16>(As, A1, Vs, Ws, lda, lam, aux, cs, red);
+    // As: A' = V A V^T with the rows of V (in Ws) the direct solver's eigenvectors, or A itself
     JacobiCtx jc{As, A1, Vs, cs, red, sched, la, tri, lda, ldv};
     if (d == 64) n = jacobi_eig_lookahead<64>(jc, &buf);
     else if (d == 32) n = jacobi_eig_lookahead<32>(jc, &buf);
     else n = jacobi_eig_lookahead<16>(jc, &buf);
     if (buf) {
       for (int e = tid; e < d * lda; e += FIT_THREADS) As[e] = A1[e];
+      __syncthreads();
+    }
+    if (direct) {
+      if (n == 0) {
+        for (int e = tid; e < d * d; e += FIT_THREADS) Vs[(e / d) * lda + (e % d)] = Ws[(e / d) * lda + (e % d)];
+      } else {
+        // eigenvectors of A: (rows of the Jacobi solver's V^T) x (rows of V)
+        smem_product(d, [&](int j, int i) { return Vs[j * lda + i]; }, [&](int i, int c) { return Ws[i * lda + c]; },
+                     [&](int j, int c, double v) { A1[j * lda + c] = v; });
+        __syncthreads();
+        for (int e = tid; e < d * d; e += FIT_THREADS) Vs[(e / d) * lda + (e % d)] = A1[(e / d) * lda + (e % d)];
+      }
       __syncthreads();
     }
     return n;
