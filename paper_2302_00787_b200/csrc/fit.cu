@@ -397,28 +397,69 @@ __device__ void jacobi_tables(const ushort2* sched, uchar2* pos, uint2* la, ucha
   __syncthreads();
 }
 
-// d x d product with both operands in shared memory: out(r, c, sum_k a(r, k) b(k, c)).  Thread t owns
-// column c = t % d and up to eight rows t / d + u * (FIT_THREADS / d): eight independent sums per trip.
-template <class FA, class FB, class FO>
-__device__ __forceinline__ void smem_product(int d, FA a, FB b, FO out) {
-  const int c = threadIdx.x % d, r0 = threadIdx.x / d, rstep = FIT_THREADS / d;
-  if (r0 >= d) return;
-  double acc[8];
+// 1 / sqrt(t) and 1 / t to rounding: the 20-bit hardware estimate and two Newton steps (t normal and positive,
+// resp. non-zero; no special cases).
+__device__ __forceinline__ double rsqrt_fast(double t) {
+  double q;
+  asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(q) : "d"(t));
+  q = fma(q * 0.5, fma(-t * q, q, 1.0), q);
+  return fma(q * 0.5, fma(-t * q, q, 1.0), q);
+}
+__device__ __forceinline__ double recip_fast(double t) {
+  double q;
+  asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(q) : "d"(t));
+  q = fma(q, fma(-t, q, 1.0), q);
+  return fma(q, fma(-t, q, 1.0), q);
+}
+
+// Row handled by lane group `grp` when `parts` lanes share a row: with eight lanes per row the two rows of a
+// half-warp are eight apart, so that their 8-byte accesses to a matrix with an odd leading dimension fall into
+// different banks.
+__device__ __forceinline__ int group_row(int grp, int parts) {
+  return parts == 8 ? ((grp & ~15) | ((grp & 1) << 3) | ((grp >> 1) & 7)) : grp;
+}
+
+// D x D product with both operands in shared memory (leading dimension D + 1):
+// out(r, c, sum_k a(r, k) b(k, c)) with a(r, k) = A[r][k] (TA: A[k][r]) and b(k, c) = B[k][c] (TB: B[c][k]).
+// Thread t < (D/4)^2 owns the 4 x 4 outputs in rows t / (D/4) + u D/4 and columns t % (D/4) + v D/4: eight loads
+// at fixed offsets from two running pointers feed sixteen fp64 multiply-adds, which keeps the fp64 pipe and not
+// the shared-memory port or the issue slots the limit.
+template <int D, bool TA, bool TB, class FO>
+__device__ __forceinline__ void product_impl(const double* A, const double* B, FO out) {
+  constexpr int q = D / 4, lda = D + 1;
+  if ((int)threadIdx.x >= q * q) return;
+  const int r0 = threadIdx.x / q, c0 = threadIdx.x % q;
+  constexpr int sa_u = TA ? q : q * lda, sa_k = TA ? lda : 1;
+  constexpr int sb_v = TB ? q * lda : q, sb_k = TB ? 1 : lda;
+  const double* pa = A + (TA ? r0 : r0 * lda);
+  const double* pb = B + (TB ? c0 * lda : c0);
+  double acc[4][4];
 #pragma unroll
-  for (int u = 0; u < 8; u++) acc[u] = 0.0;
-  for (int k = 0; k < d; k++) {
-    const double bv = b(k, c);
+  for (int u = 0; u < 4; u++)
 #pragma unroll
-    for (int u = 0; u < 8; u++) {
-      const int r = r0 + u * rstep;
-      if (r < d) acc[u] = fma(a(r, k), bv, acc[u]);
-    }
+    for (int v = 0; v < 4; v++) acc[u][v] = 0.0;
+#pragma unroll 4
+  for (int k = 0; k < D; k++) {
+    double av[4], bv[4];
+#pragma unroll
+    for (int u = 0; u < 4; u++) av[u] = pa[u * sa_u + k * sa_k];
+#pragma unroll
+    for (int v = 0; v < 4; v++) bv[v] = pb[v * sb_v + k * sb_k];
+#pragma unroll
+    for (int u = 0; u < 4; u++)
+#pragma unroll
+      for (int v = 0; v < 4; v++) acc[u][v] = fma(av[u], bv[v], acc[u][v]);
   }
 #pragma unroll
-  for (int u = 0; u < 8; u++) {
-    const int r = r0 + u * rstep;
-    if (r < d) out(r, c, acc[u]);
-  }
+  for (int u = 0; u < 4; u++)
+#pragma unroll
+    for (int v = 0; v < 4; v++) out(r0 + u * q, c0 + v * q, acc[u][v]);
+}
+template <bool TA, bool TB, class FO>
+__device__ __forceinline__ void smem_product(int d, const double* A, const double* B, FO out) {
+  if (d == 64) product_impl<64, TA, TB>(A, B, out);
+  else if (d == 32) product_impl<32, TA, TB>(A, B, out);
+  else product_impl<16, TA, TB>(A, B, out);
 }
 
 // ---- direct eigensolver for d <= 64 --------------------------------------------------------------
@@ -439,7 +480,12 @@ __device__ __forceinline__ bool direct_eig(double* __restrict__ As, double* __re
                                            double* __restrict__ ee, double* __restrict__ beta, double* red) {
   constexpr int P = FIT_THREADS / D, NU = (D + P - 1) / P;
   static_assert(P >= 8 && P <= 32, "lanes per vector");
-  const int tid = threadIdx.x, r = tid / P, part = tid % P;
+  const int tid = threadIdx.x, part = tid % P;
+  // row (or vector) of this group of lanes.  With eight lanes per row the two rows of a half-warp are eight
+  // apart, so that their 8-byte accesses to a padded (odd leading dimension) matrix fall into different banks.
+  const int grp = tid / P;
+  const int r = group_row(grp, P);
+  const int warp_row0 = P == 8 ? (((tid >> 5) * 4) & 48) | (((tid >> 5) * 2) & 6) : (tid & ~31) / P;   // smallest row of this warp
   auto gsum = [](double v) {
 #pragma unroll
     for (int o = P >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -447,60 +493,72 @@ __device__ __forceinline__ bool direct_eig(double* __restrict__ As, double* __re
   };
   for (int e = tid; e < D * D; e += FIT_THREADS) Ws[(e / D) * lda + (e % D)] = As[(e / D) * lda + (e % D)];
 
-  // 1. A -> Q^T A Q = T (tridiagonal).  Reflector k, I - beta_k v v^T, acts on indices k+1..D-1; v is kept in
-  //    column k of A below the diagonal.
+  // 1. A -> Q^T A Q = T (tridiagonal).  Reflector k, I - beta_k v v^T with v = x - alpha e_1, acts on indices
+  //    k+1..D-1 (x: column k below the diagonal); v is kept in column k of A.  Per step, with A22 the trailing
+  //    block: y = A22 x and |x|^2 do not wait for alpha; p = beta A22 v = beta (y - alpha A22 e_1);
+  //    w = p - (beta/2 v.p) v;  A22 -= v w^T + w v^T.  Warps whose rows all lie outside the block only keep the barriers.
   for (int k = 0; k < D - 2; k++) {
     const int n = D - k - 1;
+    const bool active = warp_row0 < n;
     double* xc = As + (k + 1) * lda + k;              // x_i = xc[i * lda]
     double* A22 = As + (k + 1) * lda + (k + 1);
-    double vj[NU], s2 = 0.0;
-#pragma unroll
-    for (int u = 0; u < NU; u++) {
-      const int j = part + u * P;
-      vj[u] = j < n ? xc[j * lda] : 0.0;
-      if (j >= 1) s2 = fma(vj[u], vj[u], s2);
-    }
-    s2 = gsum(s2);
-    const double x0 = xc[0];
-    double vr = r < n ? xc[r * lda] : 0.0;
-    double b = 0.0, alpha = x0, v0 = x0;
-    if (s2 > 0.0) {
-      alpha = -copysign(sqrt(fma(x0, x0, s2)), x0);
-      v0 = x0 - alpha;
-      b = -1.0 / (alpha * v0);
-      if (part == 0) vj[0] = v0;
-      if (r == 0) vr = v0;
-    }
-    // p = beta A22 v
-    double pr = 0.0;
-    if (r < n) {
+    double vj[NU], a22[NU], vr = 0.0, pr = 0.0, b = 0.0, alpha = 0.0, v0 = 0.0;
+    if (active) {
+      double s2a = 0.0, s2b = 0.0, ya = 0.0, yb = 0.0;
 #pragma unroll
       for (int u = 0; u < NU; u++) {
         const int j = part + u * P;
-        if (j < n) pr = fma(A22[r * lda + j], vj[u], pr);
+        vj[u] = j < n ? xc[j * lda] : 0.0;
       }
-    }
-    pr = gsum(pr) * b;
-    if (part == 0 && r < n) red[r] = pr;
-    __syncthreads();
-    if (tid == 0) { ee[k] = alpha; beta[k] = b; dd[k] = As[k * lda + k]; xc[0] = v0; }
-    // w = p - (beta/2 v.p) v ;  A22 -= v w^T + w v^T
-    double pj[NU], kk = 0.0;
-#pragma unroll
-    for (int u = 0; u < NU; u++) {
-      const int j = part + u * P;
-      pj[u] = j < n ? red[j] : 0.0;
-      kk = fma(vj[u], pj[u], kk);
-    }
-    kk = gsum(kk) * (0.5 * b);
-    if (r < n && b != 0.0) {
-      const double wr = fma(-kk, vr, pr);
+      const double x0 = xc[0];
+      const double ar0 = r < n ? A22[r * lda] : 0.0;   // A22[r][0]
+      vr = r < n ? xc[r * lda] : 0.0;
 #pragma unroll
       for (int u = 0; u < NU; u++) {
         const int j = part + u * P;
-        if (j < n) {
-          const double wj = fma(-kk, vj[u], pj[u]);
-          A22[r * lda + j] -= fma(vr, wj, wr * vj[u]);
+        a22[u] = (r < n && j < n) ? A22[r * lda + j] : 0.0;
+        if (u & 1) { yb = fma(a22[u], vj[u], yb); if (j >= 1) s2b = fma(vj[u], vj[u], s2b); }
+        else { ya = fma(a22[u], vj[u], ya); if (j >= 1) s2a = fma(vj[u], vj[u], s2a); }
+      }
+      double y = ya + yb, s2 = s2a + s2b;
+#pragma unroll
+      for (int o = P >> 1; o > 0; o >>= 1) {
+        y += __shfl_xor_sync(0xffffffffu, y, o);
+        s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+      }
+      alpha = x0; v0 = x0;
+      if (s2 > 0.0) {
+        const double nrm2 = fma(x0, x0, s2);
+        const double anorm = nrm2 * rsqrt_fast(nrm2);                 // |x|
+        alpha = -copysign(anorm, x0);
+        v0 = x0 - alpha;
+        b = recip_fast(fma(fabs(x0), anorm, nrm2));                   // 2 / |v|^2 = 1 / (|x|^2 + |x_0| |x|)
+        if (part == 0) vj[0] = v0;
+        if (r == 0) vr = v0;
+      }
+      pr = b * fma(-alpha, ar0, y);
+      if (part == 0 && r < n) red[r] = pr;
+    }
+    __syncthreads();
+    if (active) {
+      if (tid == 0) { ee[k] = alpha; beta[k] = b; dd[k] = As[k * lda + k]; xc[0] = v0; }
+      double pj[NU], ka = 0.0, kb = 0.0;
+#pragma unroll
+      for (int u = 0; u < NU; u++) {
+        const int j = part + u * P;
+        pj[u] = j < n ? red[j] : 0.0;
+        if (u & 1) kb = fma(vj[u], pj[u], kb); else ka = fma(vj[u], pj[u], ka);
+      }
+      const double kk = gsum(ka + kb) * (0.5 * b);
+      if (r < n && b != 0.0) {
+        const double wr = fma(-kk, vr, pr);
+#pragma unroll
+        for (int u = 0; u < NU; u++) {
+          const int j = part + u * P;
+          if (j < n) {
+            const double wj = fma(-kk, vj[u], pj[u]);
+            A22[r * lda + j] = a22[u] - fma(vr, wj, wr * vj[u]);
+          }
         }
       }
     }
@@ -540,27 +598,31 @@ __device__ __forceinline__ bool direct_eig(double* __restrict__ As, double* __re
   }
   const int nex = ((__double2hiint(nrm) >> 20) & 0x7ff) - 1023;
   const double sc = __hiloint2double((1023 - nex) << 20, 0);         // 2^-nex: nrm * sc in [1, 2)
+  double2* de = reinterpret_cast<double2*>(red);      // de[i] = (d_i, e_{i-1}^2), scaled
+  int* cnt = reinterpret_cast<int*>(red + 2 * D);     // counts at the FIT_THREADS points of the first grid
+  __syncthreads();
+  if (tid < D) {
+    const double ep = tid > 0 ? ee[tid - 1] * sc : 0.0;
+    de[tid] = make_double2(dd[tid] * sc, ep * ep);
+  }
   __syncthreads();
   if (tid < D) { dd[tid] *= sc; ee[tid] *= sc; }
   __syncthreads();
   lo *= sc; hi *= sc;
-  // number of eigenvalues below x: sign changes of the leading principal minors p_i of T - x I,
-  // p_i = (d_i - x) p_{i-1} - e_{i-1}^2 p_{i-2}; a zero minor takes the sign opposite to its predecessor.
+  // Number of eigenvalues below x: sign changes along the leading principal minors p_i of T - x I,
+  // p_i = (d_i - x) p_{i-1} - e_{i-1}^2 p_{i-2}, p_{-1} = 1.  The pair of minors is brought back to order one
+  // every eight steps.
   auto below = [&](double x) {
-    double pm2 = 1.0, pm1 = dd[0] - x;
-    bool neg_prev = (pm1 < 0.0) || (pm1 == 0.0);
-    int c = neg_prev ? 1 : 0;
+    double pm2 = 1.0, pm1 = de[0].x - x;
+    int c = (unsigned)__double2hiint(pm1) >> 31;
 #pragma unroll 8
     for (int i = 1; i < D; i++) {
-      const double e = ee[i - 1];
-      const double p = fma(dd[i] - x, pm1, -(e * e) * pm2);
-      const bool neg = (p < 0.0) || (p == 0.0 && !neg_prev);
-      c += neg != neg_prev;
-      neg_prev = neg;
+      const double2 t = de[i];
+      const double p = fma(t.x - x, pm1, -(t.y * pm2));
+      c += (unsigned)(__double2hiint(p) ^ __double2hiint(pm1)) >> 31;
       pm2 = pm1; pm1 = p;
-      if ((i & 7) == 0) {                             // keep the pair of minors of order one
-        const double m = fmax(fabs(pm1), fabs(pm2));
-        const int ex = (__double2hiint(m) >> 20) & 0x7ff;
+      if ((i & 7) == 0) {
+        const int ex = max((__double2hiint(pm1) >> 20) & 0x7ff, (__double2hiint(pm2) >> 20) & 0x7ff);
         if (ex > 0 && ex < 0x7fe) {
           const double s = __hiloint2double((2046 - ex) << 20, 0);
           pm1 *= s; pm2 *= s;
@@ -571,15 +633,30 @@ __device__ __forceinline__ bool direct_eig(double* __restrict__ As, double* __re
   };
   double sigma;
   {
-    constexpr int NIT = P == 8 ? 18 : (P == 16 ? 14 : 12);             // (P + 1)^NIT > 2^54
+    // first a grid of FIT_THREADS points over the whole interval, one count per thread ...
     double a = lo - 0.001 * (hi - lo) - 1e-3, bq = hi + 0.001 * (hi - lo) + 1e-3;
+    {
+      const double h = (bq - a) * (1.0 / (FIT_THREADS + 1));
+      cnt[tid] = below(fma(h, (double)(tid + 1), a));
+      __syncthreads();
+      int lo_i = 0, hi_i = FIT_THREADS;               // first grid point with more than r eigenvalues below it
+      while (lo_i < hi_i) {
+        const int mid = (lo_i + hi_i) >> 1;
+        if (cnt[mid] >= r + 1) hi_i = mid; else lo_i = mid + 1;
+      }
+      const double na = lo_i > 0 ? fma(h, (double)lo_i, a) : a;
+      const double nb = lo_i < FIT_THREADS ? fma(h, (double)(lo_i + 1), a) : bq;
+      a = na; bq = nb;
+    }
+    // ... then P points per step inside the bracket of this group's eigenvalue, to 2^-50 of the first interval
+    constexpr int NIT = P == 8 ? 13 : (P == 16 ? 10 : 8);
     const unsigned gshift = (tid & 31) / P * P;
     for (int it = 0; it < NIT; it++) {
       const double h = (bq - a) * (1.0 / (P + 1));
       const double x = fma(h, (double)(part + 1), a);
       const bool above = below(x) >= r + 1;           // at least r + 1 eigenvalues lie below x
       unsigned mask = __ballot_sync(0xffffffffu, above) >> gshift;
-      if (P < 32) mask &= (1u << P) - 1u;
+      mask &= P < 32 ? (1u << (P & 31)) - 1u : 0xffffffffu;
       const int first = mask ? __ffs(mask) - 1 : P;   // first point with the r-th eigenvalue below it
       const double na = first > 0 ? fma(h, (double)first, a) : a;
       const double nb = first < P ? fma(h, (double)(first + 1), a) : bq;
@@ -588,43 +665,65 @@ __device__ __forceinline__ bool direct_eig(double* __restrict__ As, double* __re
     sigma = 0.5 * (a + bq);
   }
 
-  // 3. Eigenvector of T for sigma from the twisted factorisation: pivots of the elimination from the top
-  //    (D+) and from the bottom (D-), gamma_i = D+_i + D-_i - (d_i - sigma); the vector starts with 1 at the
-  //    index of the smallest |gamma| and runs outwards with the multipliers of the two eliminations.
-  //    Pivots below 2^-64 (T is of order one) are replaced by -2^-64.
-  constexpr double PIVMIN = 5.421010862427522e-20;
-  double* Dp = A1 + r * lda;                          // D+ of this vector, later the vector itself
-  double* Dm = Vs + r * lda;
+  // 3. Eigenvector of T for sigma from the twisted factorisation.  With P+_i the leading and P-_i the trailing
+  //    principal minors of T - sigma I (P+_{-1} = P-_D = 1), the pivots of the elimination from the top and from
+  //    the bottom are D+_i = P+_i / P+_{i-1} and D-_i = P-_i / P-_{i+1}, and
+  //    gamma_i = D+_i + D-_i - (d_i - sigma).  The vector starts with 1 at the index of the smallest |gamma| and
+  //    runs outwards: z_i = -l+_i z_{i+1} with l+_i = e_i / D+_i, z_{i+1} = -l-_{i+1} z_i with l-_i = e_{i-1} / D-_i.
+  //    Two lanes run the two minor recurrences (one multiply-add per step); all lanes then form the quotients.
+  //    A minor that is exactly zero gives a non-finite vector, which the orthogonality check below rejects.
+  double* Lp = A1 + r * lda;                          // P+, then l+, then the vector itself
+  double* Lm = Vs + r * lda;                          // P-, then l-
   if (part < 2) {
-    if (part == 0) {
-      double t = dd[0] - sigma;
-      for (int i = 0; i < D - 1; i++) {
-        if (fabs(t) < PIVMIN) t = -PIVMIN;
-        Dp[i] = t;
-        const double e = ee[i];
-        t = fma(-e, e / t, dd[i + 1] - sigma);
+    // lane 0 runs up from the top, lane 1 down from the bottom, in one instruction stream
+    const bool fwd = part == 0;
+    double* out = fwd ? Lp : Lm;
+    const int i0 = fwd ? 0 : D - 1, di = fwd ? 1 : -1;
+    double pm2 = 1.0, pm1 = de[i0].x - sigma;
+    out[i0] = pm1;
+    for (int s0 = 1; s0 < D; s0 += 8) {               // eight steps' operands are loaded ahead of the chain
+      double dv[8], ev[8], pv[8];
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const int i = i0 + di * (s0 + q);
+        const bool in = s0 + q < D;
+        dv[q] = in ? de[i].x - sigma : 0.0;
+        ev[q] = in ? de[fwd ? i : i + 1].y : 0.0;
       }
-      Dp[D - 1] = t;
-    } else {
-      double t = dd[D - 1] - sigma;
-      for (int i = D - 1; i > 0; i--) {
-        if (fabs(t) < PIVMIN) t = -PIVMIN;
-        Dm[i] = t;
-        const double e = ee[i - 1];
-        t = fma(-e, e / t, dd[i - 1] - sigma);
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        pv[q] = fma(dv[q], pm1, -(ev[q] * pm2));
+        pm2 = pm1; pm1 = pv[q];
       }
-      Dm[0] = t;
+#pragma unroll
+      for (int q = 0; q < 8; q++)
+        if (s0 + q < D) out[i0 + di * (s0 + q)] = pv[q];
     }
   }
   __syncwarp();
   double gbest = 1e300;
   int ibest = 0;
+  {
+    double lp[NU], lm[NU];
 #pragma unroll
-  for (int u = 0; u < NU; u++) {
-    const int i = part + u * P;
-    if (i < D) {
-      const double g = fabs(Dp[i] + Dm[i] - (dd[i] - sigma));
-      if (g < gbest) { gbest = g; ibest = i; }        // NaN never wins
+    for (int u = 0; u < NU; u++) {
+      const int i = part + u * P;
+      lp[u] = lm[u] = 0.0;
+      if (i < D) {
+        const double pp = Lp[i], ppm = i > 0 ? Lp[i - 1] : 1.0;       // P+_i, P+_{i-1}
+        const double pq = Lm[i], pqp = i < D - 1 ? Lm[i + 1] : 1.0;   // P-_i, P-_{i+1}
+        const double rp = recip_fast(pp), rq = recip_fast(pq);
+        lp[u] = ee[i] * ppm * rp;                                     // l+_i (unused for i = D - 1: e = 0)
+        lm[u] = (i > 0 ? ee[i - 1] : 0.0) * pqp * rq;                 // l-_i
+        const double g = fabs(fma(pp, recip_fast(ppm), fma(pq, recip_fast(pqp), -(dd[i] - sigma))));
+        if (g < gbest) { gbest = g; ibest = i; }      // NaN never wins
+      }
+    }
+    __syncwarp();
+#pragma unroll
+    for (int u = 0; u < NU; u++) {
+      const int i = part + u * P;
+      if (i < D) { Lp[i] = lp[u]; Lm[i] = lm[u]; }
     }
   }
 #pragma unroll
@@ -635,23 +734,30 @@ __device__ __forceinline__ bool direct_eig(double* __restrict__ As, double* __re
   }
   __syncwarp();
   double zz = 0.0;
-  if (part == 0) {
+  if (part < 2) {
+    const bool up = part == 0;
+    const double* mul = up ? Lp : Lm;
+    const int di = up ? -1 : 1;
+    const int steps = up ? ibest : D - 1 - ibest;
     double z = 1.0;
-    zz = 1.0;
-    for (int i = ibest - 1; i >= 0; i--) {
-      z = -(ee[i] / Dp[i]) * z;
-      Dp[i] = z;
-      zz = fma(z, z, zz);
-    }
-  } else if (part == 1) {
-    double z = 1.0;
-    for (int i = ibest; i < D - 1; i++) {
-      z = -(ee[i] / Dm[i + 1]) * z;
-      Dp[i + 1] = z;
-      zz = fma(z, z, zz);
+    zz = up ? 1.0 : 0.0;
+    for (int s0 = 1; s0 <= steps; s0 += 8) {
+      double mv[8], zv[8];
+#pragma unroll
+      for (int q = 0; q < 8; q++) mv[q] = s0 + q <= steps ? mul[ibest + di * (s0 + q)] : 0.0;
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        z = -mv[q] * z;
+        zv[q] = z;
+        zz = fma(z, z, zz);
+      }
+#pragma unroll
+      for (int q = 0; q < 8; q++)
+        if (s0 + q <= steps) Lp[ibest + di * (s0 + q)] = zv[q];
     }
   }
-  if (part == 0) Dp[ibest] = 1.0;
+  __syncwarp();
+  if (part == 0) Lp[ibest] = 1.0;
   zz = gsum(zz);
   __syncwarp();
   const double zn = rsqrt(zz);
@@ -659,7 +765,7 @@ __device__ __forceinline__ bool direct_eig(double* __restrict__ As, double* __re
 #pragma unroll
   for (int u = 0; u < NU; u++) {
     const int i = part + u * P;
-    z[u] = i < D ? Dp[i] * zn : 0.0;
+    z[u] = i < D ? Lp[i] * zn : 0.0;
   }
   __syncthreads();                                    // every vector is in registers: A1 and Vs are free
 
@@ -688,7 +794,7 @@ __device__ __forceinline__ bool direct_eig(double* __restrict__ As, double* __re
 
   // 5. G = V V^T - I (rows are the vectors) -> A1; give up unless the vectors are orthonormal to 1e-6.
   double gmax = 0.0;
-  smem_product(D, [&](int i, int k) { return Vs[i * lda + k]; }, [&](int k, int j) { return Vs[j * lda + k]; },
+  product_impl<D, false, true>(Vs, Vs,
                [&](int i, int j, double v) {
                  v -= (i == j) ? 1.0 : 0.0;
                  A1[i * lda + j] = v;
@@ -701,14 +807,14 @@ __device__ __forceinline__ bool direct_eig(double* __restrict__ As, double* __re
     return false;
   }
   // V <- (I - G/2) V -> As: orthonormal to second order in G
-  smem_product(D, [&](int j, int i) { return A1[j * lda + i]; }, [&](int i, int c) { return Vs[i * lda + c]; },
+  product_impl<D, false, false>(A1, Vs,
                [&](int j, int c, double v) { As[j * lda + c] = fma(-0.5, v, Vs[j * lda + c]); });
   __syncthreads();
   // V A -> A1, then A' = (V A) V^T -> Vs
-  smem_product(D, [&](int j, int k) { return As[j * lda + k]; }, [&](int k, int m) { return Ws[k * lda + m]; },
+  product_impl<D, false, false>(As, Ws,
                [&](int j, int m, double v) { A1[j * lda + m] = v; });
   __syncthreads();
-  smem_product(D, [&](int i, int m) { return A1[i * lda + m]; }, [&](int m, int j) { return As[j * lda + m]; },
+  product_impl<D, false, true>(A1, As,
                [&](int i, int j, double v) { Vs[i * lda + j] = v; });
   __syncthreads();
   // A' -> As, V -> Ws
@@ -719,6 +825,78 @@ __device__ __forceinline__ bool direct_eig(double* __restrict__ As, double* __re
   }
   __syncthreads();
   return true;
+}
+
+// Cholesky M1 = L L^T (M1 in As, leading dimension D + 1) by elimination, one column per step, and L^-1 with
+// it: the row operations that reduce M1 to L^T, applied to the identity, leave L^-1.  Step j subtracts
+// f_i = a_ij / a_jj times row j from every row i > j, in the trailing block of M1 (kept symmetric, so that
+// column j is read as row j) and in W, which carries the rows of L^-1 without their final scale 1/l_ii.
+// The matrix lives in registers for the whole factorisation: lane group i holds row i, the slot of column c
+// holding M1[i][c] while c > j and W[i][c] afterwards; only the pivot row of a step goes through shared memory
+// (rowbuf, 2 D doubles), since it is the traffic through shared memory that bounds such a step.
+// On exit As = L and W = L^-1 (both with zeros above the diagonal), rdiag[j] = 1 / l_jj.  Returns true when a
+// pivot had to be raised to `floor_piv`.
+template <int D>
+__device__ __forceinline__ bool cholesky_inverse(double* __restrict__ As, double* __restrict__ W, double* __restrict__ rdiag,
+                                                 double* __restrict__ ldiag, double* __restrict__ rowbuf, double floor_piv) {
+  constexpr int P = FIT_THREADS / D, NU = (D + P - 1) / P, lda = D + 1;
+  const int tid = threadIdx.x, part = tid % P, ri = group_row(tid / P, P);
+  bool raised = false;
+  double a[NU];
+#pragma unroll
+  for (int u = 0; u < NU; u++) {
+    const int c = part + u * P;
+    a[u] = c < D ? As[ri * lda + c] : 0.0;
+    if (ri == 0 && c < D) rowbuf[c] = a[u];
+  }
+  __syncthreads();
+  for (int j = 0; j < D; j++) {
+    const double* rb = rowbuf + (j & 1) * D;
+    double piv = rb[j];
+    if (!(piv > floor_piv)) { raised = true; piv = floor_piv + 1e-300; }
+    if (ri > j) {
+      double rowj[NU];
+#pragma unroll
+      for (int u = 0; u < NU; u++) {
+        const int c = part + u * P;
+        rowj[u] = c < D ? rb[c] : 0.0;
+      }
+      const double arj = rb[ri];                      // M1[i][j] = M1[j][i]
+      const double rs = rsqrt_fast(piv);
+      const double lij = arj * rs, f = lij * rs;
+#pragma unroll
+      for (int u = 0; u < NU; u++) {
+        const int c = part + u * P;
+        a[u] = c == j ? -f : fma(-f, rowj[u], a[u]);  // W[j][j] = 1
+      }
+      if (part == j % P) As[ri * lda + j] = lij;
+      if (ri == j + 1) {
+        double* nb = rowbuf + ((j + 1) & 1) * D;
+#pragma unroll
+        for (int u = 0; u < NU; u++) {
+          const int c = part + u * P;
+          if (c < D) nb[c] = a[u];
+        }
+      }
+    } else if (ri == j && part == 0) {
+      const double rs = rsqrt_fast(piv);
+      ldiag[j] = piv * rs;
+      rdiag[j] = rs;
+    }
+    __syncthreads();
+  }
+  const double rd = rdiag[ri], ld = ldiag[ri];
+#pragma unroll
+  for (int u = 0; u < NU; u++) {
+    const int c = part + u * P;
+    if (c < D) {
+      W[ri * lda + c] = c > ri ? 0.0 : (c == ri ? rd : a[u] * rd);
+      if (c > ri) As[ri * lda + c] = 0.0;
+      else if (c == ri) As[ri * lda + c] = ld;
+    }
+  }
+  __syncthreads();
+  return raised;
 }
 
 struct FitArgs {
@@ -785,7 +963,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
         for (int e = tid; e < d * d; e += FIT_THREADS) Vs[(e / d) * lda + (e % d)] = Ws[(e / d) * lda + (e % d)];
       } else {
         // eigenvectors of A: (rows of the Jacobi solver's V^T) x (rows of V)
-        smem_product(d, [&](int j, int i) { return Vs[j * lda + i]; }, [&](int i, int c) { return Ws[i * lda + c]; },
+        smem_product<false, false>(d, Vs, Ws,
                      [&](int j, int c, double v) { A1[j * lda + c] = v; });
         __syncthreads();
         for (int e = tid; e < d * d; e += FIT_THREADS) Vs[(e / d) * lda + (e % d)] = A1[(e / d) * lda + (e % d)];
@@ -915,44 +1093,55 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
       As[i * lda + j] = M1[e] + (i == j ? rg1 : 0.0);
     }
     __syncthreads();
-    // Cholesky, column by column: `parts` threads share the dot product of a row.
-    const int parts = FIT_THREADS / d, ri = tid / parts, part = tid % parts;
+    const int parts = FIT_THREADS / d, part = tid % parts;
     const double floor_piv = 1e-12 * t1 / d;
-    for (int j = 0; j < d; j++) {
-      double t = 0.0;
-      if (ri >= j) {
-        for (int k = part; k < j; k += parts) t = fma(As[ri * lda + k], As[j * lda + k], t);
-      }
-      for (int o = parts >> 1; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-      if (ri >= j && part == 0) aux[ri] = As[ri * lda + j] - t;
-      __syncthreads();
-      double piv = aux[j];
-      if (!(piv > floor_piv)) { violated = true; piv = floor_piv + 1e-300; }
-      double rs = rsqrt(piv);
-      rs = rs * fma(-0.5 * piv * rs, rs, 1.5);       // one Newton step on 1 / sqrt(piv)
-      if (part == 0) {
-        if (ri == j) { As[j * lda + j] = piv * rs; lam[j] = rs; }     // lam: 1 / l_jj
-        else if (ri > j) As[ri * lda + j] = aux[ri] * rs;
-        else As[ri * lda + j] = 0.0;                 // upper triangle
-      }
-      __syncthreads();
-    }
-    // L^-1 by forward substitution, one column per thread group (columns are independent; the
-    // threads of a group sit in one warp).  It is built in shared memory when there is room.
     double* Li = V_IN_SMEM ? A1 : Lig;
     const int ldi = V_IN_SMEM ? lda : d;
-    {
-      const int c = ri;
-      for (int i = 0; i < d; i++) {
+    if (V_IN_SMEM) {
+      // Cholesky M1 = L L^T by elimination, one column per step, and L^-1 with it: the row operations that reduce
+      // M1 to L^T, applied to the identity, leave L^-1.  Step j scales by 1/l_jj and subtracts multiples of row j
+      // from the rows below; W (in A1) carries the rows of L^-1 without their final scale 1/l_ii.  The trailing
+      // block of M1 is updated in both triangles, so that column j can be read as row j.
+      if (d == 64) violated |= cholesky_inverse<64>(As, A1, lam, aux, red, floor_piv);
+      else if (d == 32) violated |= cholesky_inverse<32>(As, A1, lam, aux, red, floor_piv);
+      else violated |= cholesky_inverse<16>(As, A1, lam, aux, red, floor_piv);
+    } else {
+      // Cholesky, column by column: `parts` threads share the dot product of a row.
+      const int ri = tid / parts;
+      for (int j = 0; j < d; j++) {
         double t = 0.0;
-        if (i > c)
-          for (int k = c + part; k < i; k += parts) t = fma(As[i * lda + k], Li[k * ldi + c], t);
+        if (ri >= j) {
+          for (int k = part; k < j; k += parts) t = fma(As[ri * lda + k], As[j * lda + k], t);
+        }
         for (int o = parts >> 1; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-        if (part == 0) Li[i * ldi + c] = i < c ? 0.0 : (i == c ? lam[c] : -t * lam[i]);
-        __syncwarp();
+        if (ri >= j && part == 0) aux[ri] = As[ri * lda + j] - t;
+        __syncthreads();
+        double piv = aux[j];
+        if (!(piv > floor_piv)) { violated = true; piv = floor_piv + 1e-300; }
+        double rs = rsqrt(piv);
+        rs = rs * fma(-0.5 * piv * rs, rs, 1.5);       // one Newton step on 1 / sqrt(piv)
+        if (part == 0) {
+          if (ri == j) { As[j * lda + j] = piv * rs; lam[j] = rs; }     // lam: 1 / l_jj
+          else if (ri > j) As[ri * lda + j] = aux[ri] * rs;
+          else As[ri * lda + j] = 0.0;                 // upper triangle
+        }
+        __syncthreads();
       }
+      // L^-1 by forward substitution, one column per thread group (columns are independent; the
+      // threads of a group sit in one warp).  It is built in shared memory when there is room.
+      {
+        const int c = ri;
+        for (int i = 0; i < d; i++) {
+          double t = 0.0;
+          if (i > c)
+            for (int k = c + part; k < i; k += parts) t = fma(As[i * lda + k], Li[k * ldi + c], t);
+          for (int o = parts >> 1; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+          if (part == 0) Li[i * ldi + c] = i < c ? 0.0 : (i == c ? lam[c] : -t * lam[i]);
+          __syncwarp();
+        }
+      }
+      __syncthreads();
     }
-    __syncthreads();
     for (int e = tid; e < d * d; e += FIT_THREADS) {
       Lg[e] = As[(e / d) * lda + (e % d)];
       if (V_IN_SMEM) {
@@ -963,11 +1152,11 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
     __syncthreads();
     if (V_IN_SMEM) {
       // T1 = M2 L (M2 in Vs, L in As) -> Ws
-      smem_product(d, [&](int r, int k) { return Vs[r * lda + k]; }, [&](int k, int c) { return As[k * lda + c]; },
+      smem_product<false, false>(d, Vs, As,
                    [&](int r, int c, double v) { Ws[r * lda + c] = v; });
       __syncthreads();
       // L^T T1 -> A1 (its L^-1 is already in global memory), then Z Z^T = its symmetric part -> Vs
-      smem_product(d, [&](int r, int k) { return As[k * lda + r]; }, [&](int k, int c) { return Ws[k * lda + c]; },
+      smem_product<true, false>(d, As, Ws,
                    [&](int r, int c, double v) { A1[r * lda + c] = v; });
       __syncthreads();
       for (int e = tid; e < d * d; e += FIT_THREADS) {
@@ -1024,7 +1213,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
       }
       __syncthreads();
       // B1 = r Sigma^1/2 U^T L^-1 -> As,  B2 = r Sigma^-1/2 U^T L^T -> global, then A1 once L^-1 is no longer read
-      smem_product(d, [&](int l, int i) { return Vs[l * ldv + i]; }, [&](int i, int j) { return A1[i * lda + j]; },
+      smem_product<false, false>(d, Vs, A1,
                    [&](int l, int j, double v) {
                      const double b1 = r * sqrt(aux[l]) * v;
                      As[l * lda + j] = b1;
@@ -1032,7 +1221,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
                      oA[l * d + j] = (l == j) ? A : 0.0;
                    });
       __syncthreads();
-      smem_product(d, [&](int l, int i) { return Vs[l * ldv + i]; }, [&](int i, int j) { return Ws[j * lda + i]; },
+      smem_product<false, true>(d, Vs, Ws,
                    [&](int l, int j, double v) {
                      const double b2 = r / sqrt(aux[l]) * v;
                      A1[l * lda + j] = b2;
@@ -1041,9 +1230,9 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
       __syncthreads();
       // C = -B^T B / (2 (1 - 4A))
       const double cf = -1.0 / (2.0 * (1.0 - 4.0 * A));
-      smem_product(d, [&](int i, int l) { return As[l * lda + i]; }, [&](int l, int j) { return As[l * lda + j]; },
+      smem_product<true, false>(d, As, As,
                    [&](int i, int j, double v) { oC1[i * d + j] = cf * v; });
-      smem_product(d, [&](int i, int l) { return A1[l * lda + i]; }, [&](int l, int j) { return A1[l * lda + j]; },
+      smem_product<true, false>(d, A1, A1,
                    [&](int i, int j, double v) { oC2[i * d + j] = cf * v; });
     } else {
       for (int e = tid; e < d * d; e += FIT_THREADS) Ug[e] = Vs[(e % d) * ldv + (e / d)];     // U[i][l]
