@@ -11,9 +11,11 @@ constexpr int PREP_THREADS = 256;
 constexpr int PREP_MB = 64;                   // features per block
 constexpr int PREP_LDO = PREP_MB + 4;         // row stride of the transposed Omega chunk (keeps 16-byte alignment)
 
-// One block = one (group, side, chunk of 64 features).  Omega's chunk (transposed) and the d x d
-// matrix (B, then A) sit in shared memory in fp32; every thread owns a 4 x d/16 tile of the
-// 64 x d product and walks the inner index with vector loads.
+// One block = one (group, role, chunk of 64 features) with role 0, 1: W of side 1, 2; role 2: a (the same for both
+// sides, written for both); role 3: C, the scalars and the flags of side blockIdx.z + 1.  Omega's chunk
+// (transposed) and the d x d matrix (B or A) sit in shared memory in fp32; every thread owns a 4 x d/16 tile of
+// the 64 x d product and walks the inner index with vector loads.  The roles are separate blocks because a
+// block's time is the latency of its dependent global loads: short blocks side by side finish sooner.
 template <int D>
 __global__ void __launch_bounds__(PREP_THREADS)
 prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const double* __restrict__ params,
@@ -26,7 +28,9 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
   extern __shared__ __align__(16) float stage[];
   float* Ot = stage;                          // [d][PREP_LDO]: Ot[i][m] = Omega[m0 + m][i]
   float* Ms = stage + d * PREP_LDO;           // [d][d]
-  const int g = blockIdx.x, side = blockIdx.y + 1, tid = threadIdx.x;
+  const int g = blockIdx.x, role = blockIdx.y, tid = threadIdx.x;
+  const int side = role == 3 ? (int)blockIdx.z + 1 : (role == 1 ? 2 : 1);
+  if (role == 3 ? blockIdx.z >= 2 : (int)blockIdx.z * PREP_MB >= M) return;
   const int h = pool == FSHARP_POOL_PER_BH ? g % H : g;
   const float* Om = Omega + (int64_t)h * omega_head_stride;
   ParamsLayout pl{d};
@@ -44,15 +48,14 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
 
   const int m0 = blockIdx.z * PREP_MB;
   const int ty = tid >> 4, tx = tid & 15;     // rows m0 + 4 ty + u, columns NC tx + v
-  for (int e = tid; e < PREP_MB * d; e += PREP_THREADS) {
-    const int m = e % PREP_MB, i = e / PREP_MB;
-    Ot[i * PREP_LDO + m] = (m0 + m < M) ? Om[(size_t)(m0 + m) * d + i] : 0.f;
-  }
-  // pass 0: W = Omega B; pass 1: a = diag(Omega A Omega^T), which is the same for both sides: the
-  // side-1 block computes it and writes it for both
-  for (int pass = 0; pass < (side == 1 ? 2 : 1); pass++) {
+  if (role < 3) {
+    // pass 0 (roles 0, 1): W = Omega B; pass 1 (role 2): a = diag(Omega A Omega^T)
+    const int pass = role == 2 ? 1 : 0;
     const double* Mat = pass == 0 ? Bm : A;
-    __syncthreads();
+    for (int e = tid; e < PREP_MB * d; e += PREP_THREADS) {           // coalesced read, transposed store
+      const int m = e / d, i = e % d;
+      Ot[i * PREP_LDO + m] = (m0 + m < M) ? Om[(size_t)(m0 + m) * d + i] : 0.f;
+    }
     for (int e = tid; e < d * d; e += PREP_THREADS) Ms[e] = (float)Mat[e];
     __syncthreads();
     float acc[4][NC];
@@ -119,8 +122,8 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
         }
       }
     }
+    return;
   }
-  if (blockIdx.z != 0) return;
   // C = gamma I exactly?
   int cscalar = 1, lo_nonzero = 0;
   const double gamma = Cm[0];
@@ -170,7 +173,8 @@ int fs_run_prep_images(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_s
                        uint8_t* images, int* flags) {
   if (G == 0) return FSHARP_OK;
   if (images != nullptr && (d != tcl::TC_D || M != tcl::TC_M)) return FSHARP_E_SHAPE;
-  const dim3 grid(G, 2, (M + PREP_MB - 1) / PREP_MB);
+  const int nchunks = (M + PREP_MB - 1) / PREP_MB;
+  const dim3 grid(G, 4, nchunks > 2 ? nchunks : 2);
   const size_t smem = ((size_t)d * PREP_LDO + (size_t)d * d) * sizeof(float);
 #define FS_PREP(DD)                                                                                                  \
   do {                                                                                                               \
