@@ -1042,9 +1042,22 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
     obj = d * (log(1.0 - 4.0 * A) - 0.5 * log(1.0 - 8.0 * A)) + (2.0 - 8.0 * A) / (1.0 - 8.0 * A) * S - 2.0 * sq;
   } else if (a.variant == FSHARP_SDERF) {
     // Theorem 4.3: N = M1 + mu4 mu5^T + mu5 mu4^T + M2, eigenvalues non-ascending.
-    for (int e = tid; e < d * d; e += FIT_THREADS) {
-      int i = e / d, j = e % d;
-      As[i * lda + j] = M1[e] + M2[e] + mu4[i] * mu5[j] + mu5[i] * mu4[j] + (i == j ? rg1 + rg2 : 0.0);
+    for (int e0 = tid; e0 < d * d; e0 += 8 * FIT_THREADS) {          // global loads in batches ahead of the stores
+      double m1[8], m2[8];
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const int e = e0 + q * FIT_THREADS;
+        m1[q] = e < d * d ? M1[e] : 0.0;
+        m2[q] = e < d * d ? M2[e] : 0.0;
+      }
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const int e = e0 + q * FIT_THREADS;
+        if (e < d * d) {
+          const int i = e / d, j = e % d;
+          As[i * lda + j] = m1[q] + m2[q] + mu4[i] * mu5[j] + mu5[i] * mu4[j] + (i == j ? rg1 + rg2 : 0.0);
+        }
+      }
     }
     __syncthreads();
     nsweeps += eig();
@@ -1088,9 +1101,18 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
     double* T1g = gs + (size_t)2 * d * d;
     double* Ug = gs + (size_t)3 * d * d;
     double* Lig = gs + (size_t)4 * d * d;   // L^-1  [i][j], lower triangular
-    for (int e = tid; e < d * d; e += FIT_THREADS) {
-      int i = e / d, j = e % d;
-      As[i * lda + j] = M1[e] + (i == j ? rg1 : 0.0);
+    for (int e0 = tid; e0 < d * d; e0 += 8 * FIT_THREADS) {          // global loads in batches ahead of the stores
+      double m1[8];
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const int e = e0 + q * FIT_THREADS;
+        m1[q] = e < d * d ? M1[e] : 0.0;
+      }
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const int e = e0 + q * FIT_THREADS;
+        if (e < d * d) As[(e / d) * lda + (e % d)] = m1[q] + (e / d == e % d ? rg1 : 0.0);
+      }
     }
     __syncthreads();
     const int parts = FIT_THREADS / d, part = tid % parts;
@@ -1142,11 +1164,22 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
       }
       __syncthreads();
     }
-    for (int e = tid; e < d * d; e += FIT_THREADS) {
-      Lg[e] = As[(e / d) * lda + (e % d)];
-      if (V_IN_SMEM) {
-        Lig[e] = Li[(e / d) * ldi + (e % d)];
-        Vs[(e / d) * lda + (e % d)] = M2[e] + ((e / d) == (e % d) ? rg2 : 0.0);      // M2 into shared memory
+    for (int e0 = tid; e0 < d * d; e0 += 8 * FIT_THREADS) {
+      double m2[8];
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const int e = e0 + q * FIT_THREADS;
+        m2[q] = (V_IN_SMEM && e < d * d) ? M2[e] : 0.0;
+      }
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const int e = e0 + q * FIT_THREADS;
+        if (e >= d * d) continue;
+        Lg[e] = As[(e / d) * lda + (e % d)];
+        if (V_IN_SMEM) {
+          Lig[e] = Li[(e / d) * ldi + (e % d)];
+          Vs[(e / d) * lda + (e % d)] = m2[q] + ((e / d) == (e % d) ? rg2 : 0.0);    // M2 into shared memory
+        }
       }
     }
     __syncthreads();
@@ -1207,9 +1240,19 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
     const double r = sqrt(1.0 - 4.0 * A);
     if (V_IN_SMEM) {
       // L^-1 -> A1, L -> Ws (shared memory again; the eigen-solve used both buffers)
-      for (int e = tid; e < d * d; e += FIT_THREADS) {
-        A1[(e / d) * lda + (e % d)] = Lig[e];
-        Ws[(e / d) * lda + (e % d)] = Lg[e];
+      for (int e0 = tid; e0 < d * d; e0 += 8 * FIT_THREADS) {
+        double li[8], lg[8];
+#pragma unroll
+        for (int q = 0; q < 8; q++) {
+          const int e = e0 + q * FIT_THREADS;
+          li[q] = e < d * d ? Lig[e] : 0.0;
+          lg[q] = e < d * d ? Lg[e] : 0.0;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; q++) {
+          const int e = e0 + q * FIT_THREADS;
+          if (e < d * d) { A1[(e / d) * lda + (e % d)] = li[q]; Ws[(e / d) * lda + (e % d)] = lg[q]; }
+        }
       }
       __syncthreads();
       // B1 = r Sigma^1/2 U^T L^-1 -> As,  B2 = r Sigma^-1/2 U^T L^T -> global, then A1 once L^-1 is no longer read

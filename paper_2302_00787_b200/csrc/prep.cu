@@ -52,11 +52,34 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
     // pass 0 (roles 0, 1): W = Omega B; pass 1 (role 2): a = diag(Omega A Omega^T)
     const int pass = role == 2 ? 1 : 0;
     const double* Mat = pass == 0 ? Bm : A;
-    for (int e = tid; e < PREP_MB * d; e += PREP_THREADS) {           // coalesced read, transposed store
-      const int m = e / d, i = e % d;
-      Ot[i * PREP_LDO + m] = (m0 + m < M) ? Om[(size_t)(m0 + m) * d + i] : 0.f;
+    // global loads in batches of eight ahead of the shared-memory stores (a store between two loads would keep
+    // the second load from being issued early)
+    for (int e0 = tid; e0 < PREP_MB * d; e0 += 8 * PREP_THREADS) {    // coalesced read, transposed store
+      float v[8];
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const int e = e0 + q * PREP_THREADS, m = e / d, i = e % d;
+        v[q] = (e < PREP_MB * d && m0 + m < M) ? Om[(size_t)(m0 + m) * d + i] : 0.f;
+      }
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const int e = e0 + q * PREP_THREADS, m = e / d, i = e % d;
+        if (e < PREP_MB * d) Ot[i * PREP_LDO + m] = v[q];
+      }
     }
-    for (int e = tid; e < d * d; e += PREP_THREADS) Ms[e] = (float)Mat[e];
+    for (int e0 = tid; e0 < d * d; e0 += 8 * PREP_THREADS) {
+      double v[8];
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const int e = e0 + q * PREP_THREADS;
+        v[q] = e < d * d ? Mat[e] : 0.0;
+      }
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const int e = e0 + q * PREP_THREADS;
+        if (e < d * d) Ms[e] = (float)v[q];
+      }
+    }
     __syncthreads();
     float acc[4][NC];
 #pragma unroll
@@ -127,18 +150,29 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
   // C = gamma I exactly?
   int cscalar = 1, lo_nonzero = 0;
   const double gamma = Cm[0];
-  for (int e = tid; e < d * d; e += PREP_THREADS) {
-    int i = e / d, j = e % d;
-    Cf[e] = (float)Cm[e];
-    if (i == j ? (Cm[e] != gamma) : (Cm[e] != 0.0)) cscalar = 0;
-    if (images != nullptr) {
-      // log2e * qk_scale^2 * C[i][j] goes to row j, column i of the MMA operand
-      uint8_t* img = images + ((size_t)g * 2 + (side - 1)) * tcl::IMG_BYTES;
-      const float v = (float)Cm[e] * (FS_LOG2E * qk_scale * qk_scale);
-      const __nv_bfloat16 hi = __float2bfloat16_rn(v), lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-      if (__bfloat162float(lo) != 0.f) lo_nonzero = 1;
-      *reinterpret_cast<__nv_bfloat16*>(img + tcl::IMG_CHI + tc::sw128_offset(j, i)) = hi;
-      *reinterpret_cast<__nv_bfloat16*>(img + tcl::IMG_CLO + tc::sw128_offset(j, i)) = lo;
+  for (int e0 = tid; e0 < d * d; e0 += 8 * PREP_THREADS) {
+    double cv[8];
+#pragma unroll
+    for (int q = 0; q < 8; q++) {
+      const int e = e0 + q * PREP_THREADS;
+      cv[q] = e < d * d ? Cm[e] : 0.0;
+    }
+#pragma unroll
+    for (int q = 0; q < 8; q++) {
+      const int e = e0 + q * PREP_THREADS;
+      if (e >= d * d) continue;
+      const int i = e / d, j = e % d;
+      Cf[e] = (float)cv[q];
+      if (i == j ? (cv[q] != gamma) : (cv[q] != 0.0)) cscalar = 0;
+      if (images != nullptr) {
+        // log2e * qk_scale^2 * C[i][j] goes to row j, column i of the MMA operand
+        uint8_t* img = images + ((size_t)g * 2 + (side - 1)) * tcl::IMG_BYTES;
+        const float v = (float)cv[q] * (FS_LOG2E * qk_scale * qk_scale);
+        const __nv_bfloat16 hi = __float2bfloat16_rn(v), lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+        if (__bfloat162float(lo) != 0.f) lo_nonzero = 1;
+        *reinterpret_cast<__nv_bfloat16*>(img + tcl::IMG_CHI + tc::sw128_offset(j, i)) = hi;
+        *reinterpret_cast<__nv_bfloat16*>(img + tcl::IMG_CLO + tc::sw128_offset(j, i)) = lo;
+      }
     }
   }
   lo_nonzero = __syncthreads_or(lo_nonzero);
