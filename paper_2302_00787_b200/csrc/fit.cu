@@ -937,10 +937,8 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
   uchar2* tri = pos + (d - 1) * d;                                      // [d/2 (d/2 + 1) / 2]
   int log2d = 0;
   while ((1 << log2d) < d) log2d++;
-  if (a.variant == FSHARP_SDERF || a.variant == FSHARP_ADERF) {
-    jacobi_schedule(sched, d);
-    if (V_IN_SMEM) jacobi_tables(sched, pos, la, tri, d);
-  }
+  if (!V_IN_SMEM && (a.variant == FSHARP_SDERF || a.variant == FSHARP_ADERF)) jacobi_schedule(sched, d);
+  bool tables_built = false;            // the look-ahead solver's tables are built when it first has to sweep
   // eigen-decomposition of the matrix in As: eigenvalues on its diagonal, eigenvectors in the rows of Vs
   auto eig = [&]() -> int {
     if (!V_IN_SMEM) return jacobi_eig(As, lda, Vs, ldv, d, log2d, sched, cs, red);
@@ -950,6 +948,29 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
     else if (d == 32) direct = direct_eig<32>(As, A1, Vs, Ws, lda, lam, aux, cs, red);
     else direct = direct_eig<16>(As, A1, Vs, Ws, lda, lam, aux, cs, red);
     // As: A' = V A V^T with the rows of V (in Ws) the direct solver's eigenvectors, or A itself
+    if (direct) {
+      // the Jacobi solver's own convergence test on A': met, the direct solver's vectors stand
+      double off = 0.0, tot = 0.0;
+      for (int e = tid; e < d * d; e += FIT_THREADS) {
+        const int i = e / d, j = e % d;
+        if (i > j) continue;
+        const double v = As[i * lda + j];
+        tot += i == j ? v * v : 2.0 * v * v;
+        if (i != j) off += 2.0 * v * v;
+      }
+      off = block_reduce(off, red, 0);
+      tot = block_reduce(tot, red, 0);
+      if (off <= 1e-24 * tot || tot == 0.0) {
+        for (int e = tid; e < d * d; e += FIT_THREADS) Vs[(e / d) * lda + (e % d)] = Ws[(e / d) * lda + (e % d)];
+        __syncthreads();
+        return 0;
+      }
+    }
+    if (!tables_built) {
+      jacobi_schedule(sched, d);
+      jacobi_tables(sched, pos, la, tri, d);
+      tables_built = true;
+    }
     JacobiCtx jc{As, A1, Vs, cs, red, sched, la, tri, lda, ldv};
     if (d == 64) n = jacobi_eig_lookahead<64>(jc, &buf);
     else if (d == 32) n = jacobi_eig_lookahead<32>(jc, &buf);
