@@ -314,8 +314,8 @@ def main():
 
 # DRAM bytes per launch (read + write) from the ncu captures summarised under profiles/ (same kernels, same workload);
 # an entry is dropped when its kernel changes.
-NCU_TRAFFIC = {("cfg2", "fit_kernel"): 4.36e6, ("cfg2", "tc_kv_kernel"): 75.5e6, ("cfg2", "tc_out_kernel"): 50.3e6,
-               ("cfg2", "tc_stats_kernel"): 72.2e6, ("cfg3", "tc_kv_kernel"): 531.4e6, ("cfg3", "tc_causal_out_kernel"): 626.2e6}
+NCU_TRAFFIC = {("cfg2", "fit_kernel"): 4.39e6, ("cfg2", "tc_kv_kernel"): 75.4e6, ("cfg2", "tc_out_kernel"): 48.4e6,
+               ("cfg2", "tc_stats_kernel"): 71.9e6, ("cfg3", "tc_kv_kernel"): 531.4e6, ("cfg3", "tc_causal_out_kernel"): 626.2e6}
 
 
 def roofline_for(name, k, w, work, peaks):
@@ -345,18 +345,30 @@ def roofline_for(name, k, w, work, peaks):
         return {"kernel": name, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": ach / peaks["bf16_tflops"], "traffic": NCU_TRAFFIC.get((w.name, name)), "peak_source": peaks["source"]}
     if name == "fit_kernel":
-        # fp64 arithmetic of the Jacobi sweeps (the rest of the fit is negligible): per round and group the
-        # 2 x 2 blocks of A (8 multiplies + 8 multiply-adds each) and d/2 * d row-pair entries of V^T
-        # (2 multiplies + 2 multiply-adds each); peak = 64 fp64 FMA per clock and SM.
+        # fp64 arithmetic of the fit.  Direct solver (d <= 64): Householder tridiagonalisation 4/3 d^3, Sturm counts
+        # (one grid of 512 points, then P = 512/d points per eigenvalue and step, 4 flops per recurrence step),
+        # reflectors applied back 2 d^3, four d^3 products (orthogonality check, correction, V A, (V A) V^T) 8 d^3;
+        # ADERF adds the elimination for L and L^-1 (2 d^3) and six more products (12 d^3).  Jacobi sweeps, when the
+        # direct result needs them (always for d = 128): per round and group the 2 x 2 blocks of A (8 multiplies +
+        # 8 multiply-adds each) and d/2 * d row-pair entries of V^T (2 multiplies + 2 multiply-adds each).
+        # Peak = 64 fp64 FMA per clock and SM.
         h = d // 2
         blocks = h * (h + 1) // 2 if d <= 64 else h * h
-        flops = work.get("fit_sweeps", 0.0) * (d - 1) * (blocks * 24 + h * d * 6) * units
+        per_group = work.get("fit_sweeps", 0.0) * (d - 1) * (blocks * 24 + h * d * 6)
+        if d <= 64 and w.variant in ("sderf", "aderf"):
+            lanes = 512 // d
+            steps = {8: 13, 16: 10, 32: 8}[lanes]
+            per_group += (4.0 / 3.0 + 2.0 + 8.0) * d ** 3 + (512 + steps * lanes * d) * d * 4.0
+            if w.variant == "aderf":
+                per_group += 14.0 * d ** 3
+        flops = per_group * units
         peak = 64 * 2 * peaks.get("sm_count", 148) * peaks.get("sm_max_mhz", 1965.0) * 1e6 / 1e12
         ach = flops / t / 1e12
         return {"kernel": name, "bound": "alu", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
                 "traffic": NCU_TRAFFIC.get((w.name, name)) if w.variant == "sderf" else None, "peak_source": "64 fp64 FMA/clk/SM x SMs x max SM clock",
                 "note": f"one block per group ({units} of {peaks.get('sm_count', 148)} SMs busy), "
-                        f"{work.get('fit_sweeps', 0.0):.1f} Jacobi sweeps per group; bound by shared-memory wavefronts and barrier latency"}
+                        f"direct solver + {work.get('fit_sweeps', 0.0):.1f} Jacobi sweeps per group; bound by instruction issue, "
+                        f"shared-memory traffic and barrier latency of one block per matrix"}
     by = bytes_of.get(name, work["bytes"]) * (per_launch if k["launches_per_step"] > 1 else 1.0)
     ach = by / t / 1e9
     return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
