@@ -151,6 +151,46 @@ def test_fit_from_exact_statistics(ctx, variant, d):
             assert np.all(np.diff(a) >= -1e-15)          # eigenvalues of N non-ascending
 
 
+@pytest.mark.parametrize("variant", ["sderf", "aderf"])
+@pytest.mark.parametrize("d", [16, 32, 64])
+@pytest.mark.parametrize("case", ["all_equal", "clusters", "near_clusters", "two_equal_blocks"])
+def test_fit_with_repeated_eigenvalues(ctx, variant, d, case):
+    """Spectra on which an eigenvector-per-eigenvalue solver has no unique answer (eigenvalues equal or equal to
+    rounding, a matrix that splits into blocks with the same spectrum): the fit must still give the invariants
+    of the closed forms, whichever of its eigensolvers ends up doing the work."""
+    rng = np.random.default_rng(7 * d + len(case))
+    Qm, _ = np.linalg.qr(rng.standard_normal((d, d)))
+    if case == "all_equal":
+        M1 = 0.3 * np.eye(d)
+    elif case in ("clusters", "near_clusters"):
+        lam = np.repeat(np.linspace(0.1, 0.5, 8), d // 8)
+        M1 = (Qm * lam) @ Qm.T
+        if case == "near_clusters":
+            E = rng.standard_normal((d, d))
+            M1 = M1 + 1e-11 * (E + E.T)
+    else:
+        h = d // 2
+        Bk = rng.standard_normal((h, h))
+        Bk = Bk @ Bk.T / h + 0.1 * np.eye(h)
+        M1 = np.zeros((d, d))
+        M1[:h, :h] = Bk
+        M1[h:, h:] = Bk
+    M1 = 0.5 * (M1 + M1.T)
+    M2 = 0.5 * M1 + 0.1 * np.eye(d)
+    mu4 = np.zeros(d) if case != "near_clusters" else 1e-3 * rng.standard_normal(d)
+    mu5 = np.zeros(d)
+    st = {"M1": M1, "M2": M2, "mu4": mu4, "mu5": mu5, "mu3": float(mu4 @ mu5) / d, "d": d}
+    ref = fs.FITS[variant](st)
+    blob = np.concatenate([M1.ravel(), M2.ravel(), mu4, mu5])[None, :]
+    pr = ctx.fsharp_fit_params(torch.from_numpy(blob).cuda(), d, variant)
+    assert ctx.status() == 0
+    p = fb.unpack_params(pr.cpu().numpy()[0], d)
+    assert_fit_close(p, ref, d, 1e-8)
+    I = np.eye(d)
+    Sinv = np.linalg.inv(I - 4 * p["A"])
+    assert np.abs(p["B1"].T @ Sinv @ p["B2"] - I).max() < 1e-9
+
+
 @pytest.mark.parametrize("w", small_cases()[:5], ids=lambda w: w.name)
 def test_stats_then_fit_end_to_end(ctx, w):
     (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
