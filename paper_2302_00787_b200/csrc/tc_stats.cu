@@ -4,8 +4,9 @@
 // A 128-token tile X [128 x 64] sits in shared memory once (TMA, 128-byte swizzle) and is read
 // by the MMA as both operands: D = [X | E]^T X with E the constant tile whose first column is 1.
 // Rows 0..63 of D are the tile's Gram matrix, row 64 its column sums.  Products of bf16 values
-// are exact in fp32; each tile's fp32 sums are folded into fp64 registers, and the blocks of one
-// group are combined with fp64 atomics.  The kernel is bound by the HBM read of Q and K.
+// are exact in fp32; the fp32 sums of ST_FOLD tiles at a time are folded into fp64 registers (the fold, 64
+// conversions and additions per thread, is what a tile's arrival rate from HBM has to cover), and the
+// blocks of one group are combined with fp64 atomics.  The kernel is bound by the HBM read of Q and K.
 #include "common.cuh"
 #include "tc_common.cuh"
 #include "tc_layout.cuh"
@@ -16,6 +17,7 @@ using namespace tcl;
 namespace {
 
 constexpr int ST_STAGES = 8;                 // ring of token tiles in flight
+constexpr int ST_FOLD = 2;                   // tiles summed in one fp32 accumulator before it is folded into fp64
 constexpr int ST_EPI_WARPS = 3;              // rows 0..95 of D; only 0..64 carry data
 constexpr int ST_WARP_TMA = 3, ST_WARP_MMA = 4, ST_THREADS = 160;
 constexpr uint32_t ST_TMEM_COLS = 128;       // two accumulators of 64 columns
@@ -87,9 +89,9 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       constexpr uint32_t ID = idesc_bf16(128, TC_D, 1, 1);      // both operands MN-major (feature index contiguous)
       const uint32_t sX0 = smem_u32(sm + StSmem::X0), sOnes = smem_u32(sm + StSmem::ONES);
       for (int it = 0; it < ntiles; it++) {
-        const int st = it % ST_STAGES, buf = it & 1;
+        const int st = it % ST_STAGES, grp = it / ST_FOLD, buf = grp & 1, sub = it % ST_FOLD;
         if (!mbar_wait(&misc->full[st], (it / ST_STAGES) & 1, abortp, status)) break;
-        if (!mbar_wait(&misc->acc_free[buf], ((it >> 1) & 1) ^ 1, abortp, status)) break;
+        if (sub == 0 && !mbar_wait(&misc->acc_free[buf], ((grp >> 1) & 1) ^ 1, abortp, status)) break;
         tcgen05_fence_after();
         const uint32_t sX = sX0 + st * TILE_BYTES;
         // A = [X | E]: block 0 the tile, block 1 the constant tile (leading offset = their distance)
@@ -97,8 +99,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const uint64_t dB = smem_desc(sX, TILE_BYTES, 1024, SWZ_128B);
 #pragma unroll 1
         for (int k = 0; k < TILE / 16; k++)
-          mma_bf16(tmem + buf * TC_D, desc_advance(dA, k * 2048), desc_advance(dB, k * 2048), ID, k > 0);
-        mma_commit(&misc->acc_full[buf]);
+          mma_bf16(tmem + buf * TC_D, desc_advance(dA, k * 2048), desc_advance(dB, k * 2048), ID, (k > 0 || sub > 0) ? 1 : 0);
+        if (sub == ST_FOLD - 1 || it == ntiles - 1) mma_commit(&misc->acc_full[buf]);
         mma_commit(&misc->empty[st]);
       }
     }
@@ -110,7 +112,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
     for (int j = 0; j < TC_D; j++) acc[j] = 0.0;
     bool alive = true;
-    for (int it = 0; it < ntiles && alive; it++) {
+    const int ngroups = (ntiles + ST_FOLD - 1) / ST_FOLD;
+    for (int it = 0; it < ngroups && alive; it++) {
       const int buf = it & 1;
       if (!mbar_wait(&misc->acc_full[buf], (it >> 1) & 1, abortp, status, false)) { alive = false; break; }
       __syncwarp();
