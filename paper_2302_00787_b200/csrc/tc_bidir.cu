@@ -41,8 +41,8 @@ constexpr int PREFETCH_TILES = 4;   // tiles pulled into L2 ahead of the shared-
 struct KvSmem {
   static constexpr uint32_t X0 = 0, V0 = 2 * TILE_BYTES, ONES = 4 * TILE_BYTES, W = ONES + TILE_BYTES,
                             WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES, FA2 = PHI + 4 * TILE_BYTES,
-                            STG = FA2 + TC_M * 4,        // 2 KB per storing epilogue warp: accumulator rows on their way out
-                            MISC = STG + 6 * 2048, TOTAL = MISC + 256;
+                            STG = FA2 + TC_M * 4,        // two 2 KB buffers per storing epilogue warp: accumulator rows on their way out
+                            MISC = STG + 8 * 2048, TOTAL = MISC + 256;
 };
 static_assert(KvSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 static_assert(KvSmem::PHI % 1024 == 0 && KvSmem::W % 1024 == 0 && KvSmem::ONES % 1024 == 0, "swizzled tiles need 1024-byte alignment");
@@ -61,7 +61,8 @@ constexpr int HALF_THREADS = EPI_THREADS / 2;
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-             const __grid_constant__ CUtensorMap tmPhi, const uint8_t* __restrict__ images, const float* __restrict__ crow, int H, int pool, int L, int Lpad,
+             const __grid_constant__ CUtensorMap tmPhi, const __grid_constant__ CUtensorMap tmState,
+             const uint8_t* __restrict__ images, const float* __restrict__ crow, int H, int pool, int L, int Lpad,
              int tiles_per_split, int nsplit, float* __restrict__ partial, float* __restrict__ shifts,
              int* __restrict__ pmax, int per_tile, int* __restrict__ status) {
   // per_tile != 0 (causal use: every 128-key tile is a chunk with a state, a shift and a partial of its
@@ -225,32 +226,47 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     auto write_partial = [&](size_t slot) {
       __syncwarp();
       tcgen05_fence_after();
-      float* out = partial + slot * TC_NV * TC_M + hf * 128;            // row n at out + n * TC_M
       float amax = 0.f;
-      if (q * 32 <= TC_DV) {                // warp-uniform: rows 0..64 carry data (65..79 are zero and never read)
-        // 16 columns at a time go through shared memory, so that a store instruction of the warp
-        // covers 8 rows x 64 contiguous bytes instead of 32 rows x 16 bytes
-        uint8_t* stg = sm + KvSmem::STG + (hf * 3 + q) * 2048;
+      if (q < 2) {
+        // rows 0..63: 16 columns at a time go into a 2 KB shared-memory buffer (32 rows x 64 bytes, 64-byte
+        // swizzle) that a bulk tensor store takes from there; two buffers per warp, so that the warp fills one
+        // while the other is being read.  The stores run on while the warp goes back to the next tile.
+        uint8_t* stg0 = sm + KvSmem::STG + (hf * 2 + q) * 4096;
+#pragma unroll
+        for (int c = 0; c < 8; c++) {
+          uint8_t* stg = stg0 + (c & 1) * 2048;
+          uint32_t a[16];
+          tmem_ld16(acc_addr + c * 16, a);
+          if (lane == 0) bulk_wait_read1();           // the store that last read this buffer (two stores back)
+          __syncwarp();
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 16; j++) amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
+#pragma unroll
+          for (int i = 0; i < 4; i++)
+            *reinterpret_cast<uint4*>(stg + lane * 64 + ((i ^ ((lane >> 1) & 3)) << 4)) = make_uint4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_3d(&tmState, stg, hf * 128 + c * 16, q * 32, (int)slot);
+            bulk_commit();
+          }
+        }
+      } else if (q == 2) {
+        // row 64 (the normaliser's row) is one lane's: it goes out directly
+        float* out = partial + slot * TC_NV * TC_M + hf * 128 + (size_t)TC_DV * TC_M;
 #pragma unroll
         for (int c = 0; c < 8; c++) {
           uint32_t a[16];
           tmem_ld16(acc_addr + c * 16, a);
           tmem_wait_ld();
-          if (row <= TC_DV) {
+          if (lane == 0) {
 #pragma unroll
             for (int j = 0; j < 16; j++) amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
-          }
 #pragma unroll
-          for (int i = 0; i < 4; i++)
-            *reinterpret_cast<uint4*>(stg + lane * 64 + ((i ^ ((lane >> 1) & 3)) << 4)) = make_uint4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
-          __syncwarp();
-#pragma unroll
-          for (int i = 0; i < 4; i++) {
-            const int rr = (lane >> 2) + 8 * i, cw = lane & 3, n = q * 32 + rr;
-            const uint4 val = *reinterpret_cast<const uint4*>(stg + rr * 64 + ((cw ^ ((rr >> 1) & 3)) << 4));
-            if (n <= TC_DV) *reinterpret_cast<uint4*>(out + (size_t)n * TC_M + c * 16 + cw * 4) = val;
+            for (int i = 0; i < 4; i++)
+              *reinterpret_cast<uint4*>(out + c * 16 + i * 4) = make_uint4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
           }
-          __syncwarp();
         }
       }
 #pragma unroll
@@ -366,6 +382,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     // write this split's partial [V | 1]^T phi_h (fp32, rows 0..79), its shift and its largest magnitude
     if (alive && ntiles > 0 && !per_tile && mbar_wait(&misc->phi_free[hf], (ntiles - 1) & 1, abortp, status, false))
       write_partial((size_t)bh * nsplit + split);
+    if (q < 2 && lane == 0) bulk_wait0();              // this thread's state stores have completed before the block ends
   }
   tcgen05_fence_before();
   __syncthreads();
@@ -697,6 +714,7 @@ namespace tchost {
 int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int H, int L, int inner);
 int make_map_kvt(CUtensorMap* map, const void* base, int BH, int bf16);
 int make_map_feat(CUtensorMap* map, const void* base, int BH, int Lpad);
+int make_map_state(CUtensorMap* map, const void* base, size_t slots);
 }  // namespace tchost
 int fs_tc_rowterm(fsharp_ctx* ctx, const void* K, const fsharp_dims* dm, const uint8_t* images, const int* flags, int Lpad,
                   int tiles_per_split, int nsplit, float* crow);
@@ -727,7 +745,8 @@ int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_d
   const int B = dm->B, H = dm->H, Lk = dm->Lk;
   const int Lpad = (Lk + TILE - 1) / TILE * TILE;
   FS_TRY(fs_tc_rowterm(ctx, K, dm, images, flags, Lpad, tiles_per_split, nsplit, crow));
-  CUtensorMap tmK, tmV, tmPhi;
+  CUtensorMap tmK, tmV, tmPhi, tmState;
+  FS_TRY(tchost::make_map_state(&tmState, partial, (size_t)B * H * (phik != nullptr ? (size_t)((Lk + TILE - 1) / TILE) : (size_t)nsplit)));
   FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, Lk, dm->d), B, H, Lk, dm->d));
   FS_TRY(tchost::make_map_tokens(&tmV, V, fs_addr(dm->v_stride, H, Lk, dm->dv), B, H, Lk, dm->dv));
   if (phik != nullptr) FS_TRY(tchost::make_map_feat(&tmPhi, phik, B * H, Lpad));
@@ -735,7 +754,7 @@ int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_d
   FS_CUDA_OK(cudaFuncSetAttribute(tc_kv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KvSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_KV);
   tc_kv_kernel<<<dim3(nsplit, B * H), TC_THREADS, KvSmem::TOTAL + 1024, ctx->stream>>>(
-      tmK, tmV, tmPhi, images, crow, H, dm->pool, Lk, Lpad, tiles_per_split, nsplit, partial, shifts, pmax,
+      tmK, tmV, tmPhi, tmState, images, crow, H, dm->pool, Lk, Lpad, tiles_per_split, nsplit, partial, shifts, pmax,
       phik != nullptr ? 1 : 0, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
