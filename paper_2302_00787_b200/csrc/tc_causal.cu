@@ -26,9 +26,13 @@ namespace {
 // query features
 // ------------------------------------------------------------------------------------------
 constexpr int FQ_STAGES = 3;
+// The feature tile leaves as four 64-feature blocks (16 KB each, one bulk store each) from a ring of six block
+// slots: block j of tile t sits in slot (4 t + j) % 6, so a tile only reuses slots whose stores were issued at least
+// one and a half tiles earlier and the stores of a tile's last two blocks may still be reading when the next is written.
+constexpr int FQ_PHI_SLOTS = 6;
 struct FqSmem {
   static constexpr uint32_t X0 = 0, W = FQ_STAGES * TILE_BYTES, WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES,
-                            ROWMAX = PHI + 4 * TILE_BYTES,
+                            ROWMAX = PHI + FQ_PHI_SLOTS * TILE_BYTES,
                             AH = ROWMAX + 2 * 2 * TILE * 4, MISC = AH + TC_M * 4, TOTAL = MISC + 256;
 };
 struct FqMisc {
@@ -153,26 +157,30 @@ tc_featq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       float mx = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
       float* rm = rowmax + buf * 2 * TILE;
       rm[hf * TILE + row] = mx;
+      if (threadIdx.x == 0 && it > 0) bulk_wait_read2();      // all stores but the previous tile's last two have read their slots
       named_bar_sync(1, EPI_THREADS);
       mx = fmaxf(mx, rm[(hf ^ 1) * TILE + row]);
       // the tile goes to shared memory in the layout of an MMA operand and leaves as one TMA store per
-      // 64-feature block; thread 0 waits for the store to have read the tile before the next one is written
-      uint8_t* prow = sm + FqSmem::PHI + hf * 2 * TILE_BYTES + row * 128;
+      // 64-feature block
+      const int slot0 = (4 * it + 2 * hf) % FQ_PHI_SLOTS, slot1 = (4 * it + 2 * hf + 1) % FQ_PHI_SLOTS;
+      uint8_t* prow0 = sm + FqSmem::PHI + slot0 * TILE_BYTES + row * 128;
+      uint8_t* prow1 = sm + FqSmem::PHI + slot1 * TILE_BYTES + row * 128;
 #pragma unroll
       for (int c = 0; c < 16; c++) {
         uint32_t p[4];
 #pragma unroll
         for (int j = 0; j < 4; j++)
           p[j] = pack_bf16(ex2(__uint_as_float(v[c * 8 + 2 * j]) - mx), ex2(__uint_as_float(v[c * 8 + 2 * j + 1]) - mx));
-        *reinterpret_cast<uint4*>(prow + (c >> 3) * TILE_BYTES + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
+        *reinterpret_cast<uint4*>((c < 8 ? prow0 : prow1) + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
       }
       fence_proxy_async_smem();
       named_bar_sync(2, EPI_THREADS);
       if (threadIdx.x == 0) {
 #pragma unroll
-        for (int fb = 0; fb < TC_M / 64; fb++) tma_store_3d(&tmPhi, sm + FqSmem::PHI + fb * TILE_BYTES, fb * 64, (tile0 + it) * TILE, bh);
-        bulk_commit();
-        bulk_wait_read0();
+        for (int fb = 0; fb < TC_M / 64; fb++) {
+          tma_store_3d(&tmPhi, sm + FqSmem::PHI + ((4 * it + fb) % FQ_PHI_SLOTS) * TILE_BYTES, fb * 64, (tile0 + it) * TILE, bh);
+          bulk_commit();
+        }
       }
     }
     if (threadIdx.x == 0) bulk_wait0();
