@@ -156,6 +156,8 @@ def main():
     ap.add_argument("--cpu-baseline-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernel-impl", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--streams", type=int, default=2,
+                    help="steps in flight: step i runs on context i mod S, each context with a stream, scratch and outputs of its own")
     args = ap.parse_args()
 
     from paper_2302_00787_b200 import workloads as wl
@@ -191,65 +193,116 @@ def main():
     Om = wl.make_omega(w_rank)
     dOm = torch.from_numpy(Om).to(dev)
     G = w.B * w.H
-    ctx = fb.Context(local_rank)
-    ctx.set_impl({"auto": fb.IMPL_AUTO, "simt": fb.IMPL_SIMT, "tensor": fb.IMPL_TENSOR}[args.kernel_impl])
-    st = torch.empty(G, fb.stats_doubles(w.d), dtype=torch.float64, device=dev)
-    pr = torch.empty(G, fb.params_doubles(w.d), dtype=torch.float64, device=dev)
-    Y = torch.empty(w.B, w.H, w.L, w.dv, dtype=td, device=dev)
+    # Steps are independent of one another, and the fit keeps one block per group busy (fewer blocks than SMs),
+    # so S steps are kept in flight: step i runs on context i mod S.  Every context has a stream, a scratch
+    # block, statistics, parameters and an output tensor of its own; nothing is shared but the read-only inputs.
+    S = max(1, args.streams)
+    main_stream = torch.cuda.current_stream(dev)
+    streams = [torch.cuda.Stream(dev) for _ in range(S)] if S > 1 else [main_stream]
+    ctxs = [fb.Context(local_rank, stream=s_) for s_ in streams]
+    for c in ctxs:
+        c.set_impl({"auto": fb.IMPL_AUTO, "simt": fb.IMPL_SIMT, "tensor": fb.IMPL_TENSOR}[args.kernel_impl])
+    ctx = ctxs[0]
+    sts = [torch.empty(G, fb.stats_doubles(w.d), dtype=torch.float64, device=dev) for _ in ctxs]
+    prs = [torch.empty(G, fb.params_doubles(w.d), dtype=torch.float64, device=dev) for _ in ctxs]
+    Ys = [torch.empty(w.B, w.H, w.L, w.dv, dtype=td, device=dev) for _ in ctxs]
+    pr = prs[0]
+    torch.cuda.synchronize()
 
     def step(i):
         dQ, dK, dV = sets[i % len(sets)]
-        ctx.fsharp_stats(dQ, dK, out=st)
-        ctx.fsharp_fit_params(st, w.d, w.variant, out=pr)
-        ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=w.causal, chunk=w.chunk, out=Y)
+        c = i % S
+        ctxs[c].fsharp_stats(dQ, dK, out=sts[c])
+        ctxs[c].fsharp_fit_params(sts[c], w.d, w.variant, out=prs[c])
+        ctxs[c].fsharp_attend(dQ, dK, dV, dOm, prs[c], causal=w.causal, chunk=w.chunk, out=Ys[c])
+
+    def fork():
+        """The contexts' streams start after everything queued on the timing stream."""
+        if S > 1:
+            ev = torch.cuda.Event()
+            ev.record(main_stream)
+            for s_ in streams:
+                s_.wait_event(ev)
+
+    def join():
+        """The timing stream continues after everything queued on the contexts' streams."""
+        if S > 1:
+            for s_ in streams:
+                ev = torch.cuda.Event()
+                ev.record(s_)
+                main_stream.wait_event(ev)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(args.warmup):
+    for i in range(max(args.warmup, S)):
         step(i)
-    assert ctx.status() == 0, "device status after warm-up"
+    torch.cuda.synchronize()
+    assert all(c.status() == 0 for c in ctxs), "device status after warm-up"
     sampler = ClockSampler(physical_index(local_rank))
     barrier()
     sampler.start()
-    n0 = ctx.launch_count()
+    n0 = sum(c.launch_count() for c in ctxs)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
+    e0.record(main_stream)
+    fork()
     for i in range(args.steps):
         step(i)
-    e1.record()
+    join()
+    e1.record(main_stream)
     barrier()
     ms = e0.elapsed_time(e1)
-    launches = ctx.launch_count() - n0
-    # same loop once more with an event pair around every launch: per-kernel device time
+    launches = sum(c.launch_count() for c in ctxs) - n0
+    # the steps once more, one at a time on one context, with an event pair around every launch:
+    # per-kernel device time of a kernel that has the GPU to itself
     ctx.set_timing(True)
     ksteps = max(1, min(args.steps, 4096 // max(1, launches // args.steps)))
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for i in range(ksteps):
-        step(i)
+        step(i * S)
     per_kernel = ctx.read_timing()
     ctx.set_timing(False)
+    # and untimed inside, one step at a time: the latency of a step that has the GPU to itself
+    torch.cuda.synchronize()
+    e2.record(streams[0])
+    for i in range(ksteps):
+        step(i * S)
+    e3.record(streams[0])
+    torch.cuda.synchronize()
+    serial_ms = e2.elapsed_time(e3) / ksteps
     sampler.stop_flag = True
     sampler.join(timeout=2)
-    assert ctx.status() == 0, "device status after the timed region"
+    assert all(c.status() == 0 for c in ctxs), "device status after the timed region"
     ms = max_over_ranks(ms, dev)
 
     # end to end through the host-buffer entry point (pinned host memory; copies inside the timing)
     hQ, hK, hV = (torch.from_numpy(a).to(td).pin_memory() for a in host_set)
     hOm = torch.from_numpy(Om).pin_memory()
-    hY = torch.empty(w.B, w.H, w.L, w.dv, dtype=td).pin_memory()
-    e2e_steps = max(3, min(args.steps, 20))
-    for _ in range(3):
-        ctx.fsharp_forward_host(hQ, hK, hV, hOm, w.variant, causal=w.causal, chunk=w.chunk, out=hY)
+    hYs = [torch.empty(w.B, w.H, w.L, w.dv, dtype=td).pin_memory() for _ in ctxs]
+    hY = hYs[0]
+    per_thread = max(2, min(args.steps, 20) // S)
+    e2e_steps = per_thread * S
+
+    def host_steps(c, n):
+        # the call returns when the step's output is in host memory; ctypes releases the interpreter lock meanwhile
+        torch.cuda.set_device(local_rank)
+        for _ in range(n):
+            ctxs[c].fsharp_forward_host(hQ, hK, hV, hOm, w.variant, causal=w.causal, chunk=w.chunk, out=hYs[c])
+
+    for c in range(S):
+        host_steps(c, 3)
     barrier()
+    # S host threads, one context each: one step's download and compute overlap the next step's upload
+    workers = [threading.Thread(target=host_steps, args=(c, per_thread)) for c in range(S)]
     t0 = time.perf_counter()
-    e0.record()
-    for _ in range(e2e_steps):
-        ctx.fsharp_forward_host(hQ, hK, hV, hOm, w.variant, causal=w.causal, chunk=w.chunk, out=hY)
-    e1.record()
+    for t_ in workers:
+        t_.start()
+    for t_ in workers:
+        t_.join()
     torch.cuda.synchronize()
-    e2e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0))
+    e2e_ms = 1e3 * (time.perf_counter() - t0)
     e2e_ms = max_over_ranks(e2e_ms, dev)
     es = 2 if w.dtype == "bf16" else 4
     h2d = (hQ.numel() + hK.numel() + hV.numel()) * es + hOm.numel() * 4
@@ -286,7 +339,9 @@ def main():
         "config": {"workload": w.name, "B": w.B, "H": w.H, "L": w.L, "d": w.d, "dv": w.dv, "M": w.M,
                    "variant": w.variant, "causal": w.causal, "chunk": w.chunk, "kernel_impl": args.kernel_impl,
                    "l2": f"inputs rotate over {len(sets)} resident sets ({len(sets) * work['bytes'] / 1e6:.0f} MB > 126 MB L2)",
-                   "step": "stats + fit + prep + featurize + contraction"},
+                   "step": "stats + fit + prep + featurize + contraction",
+                   "steps_in_flight": S},
+        "ms_per_step_alone": serial_ms,
         "clocks": sampler.result(),
         "e2e": {"value": tokens_per_step * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
