@@ -48,10 +48,12 @@ static_assert(KvSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 static_assert(KvSmem::PHI % 1024 == 0 && KvSmem::W % 1024 == 0 && KvSmem::ONES % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 
 struct KvMisc {
-  uint64_t full[2], empty[2], logits_full, logits_free, phi_full[2], phi_free[2], const_bar;
+  // key and value tiles have barriers of their own: a key tile is free again once the logits MMA that read it
+  // has completed, long before the contraction that reads the value tile of the same stage
+  uint64_t fullK[2], emptyK[2], fullV[2], emptyV[2], logits_full, logits_free, phi_full[2], phi_free[2], const_bar;
   uint32_t tmem_base;
   int abort_flag;
-  int tile_max[2][4];     // per half: [0..2] rotating slots of the per-tile maximum, [3] the first tile's
+  int tile_max[2][4];     // per half: [0..2] rotating slots of the per-tile maximum
   int chunk_max[3];       // causal use: rotating slots of the exact maximum of a whole tile
 };
 static_assert(sizeof(KvMisc) <= 256, "misc block");
@@ -84,15 +86,17 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; i++) {
-      mbar_init(&misc->full[i], 1);
-      mbar_init(&misc->empty[i], 1);
-      mbar_init(&misc->phi_full[i], HALF_THREADS);
+      mbar_init(&misc->fullK[i], 1);
+      mbar_init(&misc->emptyK[i], 1);
+      mbar_init(&misc->fullV[i], 1);
+      mbar_init(&misc->emptyV[i], 1);
+      mbar_init(&misc->phi_full[i], HALF_THREADS / 32);
       mbar_init(&misc->phi_free[i], 1);
       for (int j = 0; j < 4; j++) misc->tile_max[i][j] = f2ord(-INFINITY);
     }
     for (int j = 0; j < 3; j++) misc->chunk_max[j] = f2ord(-INFINITY);
     mbar_init(&misc->logits_full, 1);
-    mbar_init(&misc->logits_free, EPI_THREADS);
+    mbar_init(&misc->logits_free, EPI_THREADS / 32);
     mbar_init(&misc->const_bar, 1);
     misc->abort_flag = 0;
     fence_barrier_init();
@@ -128,22 +132,36 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         tma_prefetch_4d(&tmK, 0, (tile0 + it) * TILE, h, b);
         tma_prefetch_4d(&tmV, 0, (tile0 + it) * TILE, h, b);
       }
-      int issued = 0;
-      for (int it = 0; it < ntiles; it++) {
+      // Key tile `it` is loaded as soon as the logits MMA of tile it - 2 has completed; the value tile follows one
+      // iteration behind (its stage is held until the contraction of tile it - 2 has completed, which is later
+      // than the logits MMA of tile it - 1).  So the next tile's logits never wait for a value tile.
+      int issuedK = 0, issuedV = 0;
+      auto load_v = [&](int j) {
+        const int sj = j & 1;
+        if (!mbar_wait(&misc->emptyV[sj], ((j >> 1) & 1) ^ 1, abortp, status)) return false;
+        mbar_expect_tx(&misc->fullV[sj], TILE_BYTES);
+        tma_load_4d(sm + KvSmem::V0 + sj * TILE_BYTES, &tmV, &misc->fullV[sj], 0, (tile0 + j) * TILE, h, b);
+        issuedV = j + 1;
+        return true;
+      };
+      bool okp = true;
+      for (int it = 0; it < ntiles && okp; it++) {
         const int st = it & 1;
         if (it + PREFETCH_TILES < ntiles) {
           tma_prefetch_4d(&tmK, 0, (tile0 + it + PREFETCH_TILES) * TILE, h, b);
           tma_prefetch_4d(&tmV, 0, (tile0 + it + PREFETCH_TILES) * TILE, h, b);
         }
-        if (!mbar_wait(&misc->empty[st], ((it >> 1) & 1) ^ 1, abortp, status)) break;
-        mbar_expect_tx(&misc->full[st], 2 * TILE_BYTES);
-        tma_load_4d(sm + KvSmem::X0 + st * TILE_BYTES, &tmK, &misc->full[st], 0, (tile0 + it) * TILE, h, b);
-        tma_load_4d(sm + KvSmem::V0 + st * TILE_BYTES, &tmV, &misc->full[st], 0, (tile0 + it) * TILE, h, b);
-        issued = it + 1;
+        if (!mbar_wait(&misc->emptyK[st], ((it >> 1) & 1) ^ 1, abortp, status)) { okp = false; break; }
+        mbar_expect_tx(&misc->fullK[st], TILE_BYTES);
+        tma_load_4d(sm + KvSmem::X0 + st * TILE_BYTES, &tmK, &misc->fullK[st], 0, (tile0 + it) * TILE, h, b);
+        issuedK = it + 1;
+        if (it >= 1) okp = load_v(it - 1);
       }
+      if (okp && ntiles > 0) load_v(ntiles - 1);
       // no copy of this block may still be in flight when it exits
       mbar_wait(&misc->const_bar, 0, abortp, status, false);
-      for (int it = max(0, issued - 2); it < issued; it++) mbar_wait(&misc->full[it & 1], (it >> 1) & 1, abortp, status, false);
+      for (int it = max(0, issuedK - 2); it < issuedK; it++) mbar_wait(&misc->fullK[it & 1], (it >> 1) & 1, abortp, status, false);
+      for (int it = max(0, issuedV - 2); it < issuedV; it++) mbar_wait(&misc->fullV[it & 1], (it >> 1) & 1, abortp, status, false);
     }
   } else if (warp == WARP_MMA) {
     if (lane == 0) {
@@ -168,9 +186,10 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         for (int k = 0; k < TC_D / 16; k++)
           mma_bf16(tmem + KV_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dWlo, 32 * k), ID_LOGITS, 1);
         mma_commit(&misc->logits_full);
+        mma_commit(&misc->emptyK[st]);
       };
       bool ok = mbar_wait(&misc->const_bar, 0, abortp, status);
-      if (ok && ntiles > 0) ok = mbar_wait(&misc->full[0], 0, abortp, status);
+      if (ok && ntiles > 0) ok = mbar_wait(&misc->fullK[0], 0, abortp, status);
       if (ok && ntiles > 0) {
         tcgen05_fence_after();
         issue_logits(0);
@@ -178,11 +197,12 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       for (int it = 0; ok && it < ntiles; it++) {
         const int st = it & 1;
         if (it + 1 < ntiles) {
-          if (!mbar_wait(&misc->full[st ^ 1], ((it + 1) >> 1) & 1, abortp, status)) break;
+          if (!mbar_wait(&misc->fullK[st ^ 1], ((it + 1) >> 1) & 1, abortp, status)) break;
           if (!mbar_wait(&misc->logits_free, it & 1, abortp, status)) break;
           tcgen05_fence_after();
           issue_logits(st ^ 1);
         }
+        if (!mbar_wait(&misc->fullV[st], (it >> 1) & 1, abortp, status)) break;
         const uint64_t dV = st ? dVst1 : dVst0;
         const uint32_t acc0 = (it > 0 && !per_tile) ? 1u : 0u;      // causal use: every tile starts afresh
 #pragma unroll 1
@@ -201,7 +221,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           if (per_tile) bulk_wait_read0();       // the store has read the half tile: it may be overwritten
           mma_commit(&misc->phi_free[hh]);
         }
-        mma_commit(&misc->empty[st]);
+        mma_commit(&misc->emptyV[st]);
       }
       if (per_tile) bulk_wait0();
     }
@@ -209,10 +229,9 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   } else {
     regs_acquire<REGS_EPILOGUE>();
     // ---------------- epilogue warps: one key row per thread, the 128 features of its half.
-    // The running shift s of the half is taken on trust while the exponentials are computed; the
-    // tile's largest exponent is tracked on the side and checked afterwards.  Only if it exceeds
-    // the headroom (rare: the running maximum grows a handful of times per sequence) is the
-    // accumulated state rescaled and the tile redone from the logits still held in registers.
+    // The half keeps a running shift s.  Every tile's exact maximum is known before its exponentials
+    // start; only when it exceeds s by more than the headroom (rare: the running maximum grows a
+    // handful of times per sequence) does s move up, and the accumulated state with it.
     const int q = warp & 3, hf = warp >> 2;
     const int row = q * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
@@ -291,7 +310,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       }
       tmem_wait_ld();
       tcgen05_fence_before();
-      mbar_arrive(&misc->logits_free);
+      mbar_arrive_warp(&misc->logits_free, lane);
       if (per_tile) {
 #pragma unroll
         for (int i = 0; i < 128; i += 4) {
@@ -303,8 +322,11 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         }
       }
       const bool valid = (tile0 + it) * TILE + row < L;
-      if (it == 0 || per_tile) {
-        // first tile (causal use: every tile): no shift yet, take the exact maximum of this half of the tile
+      // Exact maximum of this half of the tile (causal use: of the whole tile), taken BEFORE the exponentials:
+      // it overlaps the contraction of the previous tile, and nothing stands between the last exponential and
+      // the arrival that starts this tile's contraction.
+      float tm;
+      {
         float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
         for (int i = 0; i < 128; i++) mxp[i & 3] = fmaxf(mxp[i & 3], __uint_as_float(v[i]));
@@ -316,47 +338,24 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           if (lane == 0) atomicMax(&misc->chunk_max[it % 3], f2ord(mx));
           if (threadIdx.x == 0) misc->chunk_max[(it + 1) % 3] = f2ord(-INFINITY);   // next tile's slot; idle since tile it-2
           named_bar_sync(3, EPI_THREADS);
-          s = ord2f(misc->chunk_max[it % 3]);
+          tm = ord2f(misc->chunk_max[it % 3]);
         } else {
-          if (lane == 0) atomicMax(&tmax[3], f2ord(mx));
+          if (lane == 0) atomicMax(&tmax[it % 3], f2ord(mx));
+          if (q == 0 && lane == 0) tmax[(it + 1) % 3] = f2ord(-INFINITY);           // next tile's slot; idle since tile it-2
           named_bar_sync(1 + hf, HALF_THREADS);
-          s = ord2f(tmax[3]);
+          tm = ord2f(tmax[it % 3]);
         }
-        if (it > 0 && !mbar_wait(&misc->phi_free[hf], (it - 1) & 1, abortp, status, false)) { alive = false; break; }
-      } else {
-        if (!mbar_wait(&misc->phi_free[hf], (it - 1) & 1, abortp, status, false)) { alive = false; break; }
       }
-      uint8_t* prow = sm + KvSmem::PHI + hf * 2 * TILE_BYTES + row * 128;
-      float rc = cj - s;
-      float rel = -INFINITY;      // largest exponent of this thread's elements, relative to s
-      for (int pass = 0; pass < 2; pass++) {
-        float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-        for (int c = 0; c < 16; c++) {
-          uint32_t p[4];
-#pragma unroll
-          for (int j = 0; j < 4; j++) {
-            const float f0 = __uint_as_float(v[c * 8 + 2 * j]) + rc, f1 = __uint_as_float(v[c * 8 + 2 * j + 1]) + rc;
-            mxp[j] = fmaxf(mxp[j], fmaxf(f0, f1));
-            const float e0 = ex2(f0), e1 = ex2(f1);
-            p[j] = pack_bf16(e0, e1);
-          }
-          if (!valid) p[0] = p[1] = p[2] = p[3] = 0u;
-          *reinterpret_cast<uint4*>(prow + (c >> 3) * TILE_BYTES + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
-        }
-        if (pass == 1) break;
-        rel = valid ? fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])) : -INFINITY;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) rel = fmaxf(rel, __shfl_xor_sync(0xffffffffu, rel, o));
-        if (lane == 0) atomicMax(&tmax[it % 3], f2ord(rel));
-        if (q == 0 && lane == 0) tmax[(it + 1) % 3] = f2ord(-INFINITY);   // next tile's slot; idle since tile it-2
-        named_bar_sync(1 + hf, HALF_THREADS);
-        rel = ord2f(tmax[it % 3]);
-        if (!(rel > SHIFT_HEADROOM_LOG2)) break;       // the common case: nothing to redo
-        // the running shift moves up by rel: bring the accumulated [V | 1]^T phi_h along, redo the tile
+      // the previous tile's contraction has read the phi half tile and updated the accumulator
+      if (it > 0 && !mbar_wait(&misc->phi_free[hf], (it - 1) & 1, abortp, status, false)) { alive = false; break; }
+      if (it == 0 || per_tile) {
+        s = tm;                      // first tile (causal use: every tile): the shift is the exact maximum
+      } else if (tm - s > SHIFT_HEADROOM_LOG2) {
+        // rare (the running maximum grows a handful of times per sequence): the shift moves up to this tile's
+        // maximum and the accumulated [V | 1]^T phi_h is brought along
         __syncwarp();
         tcgen05_fence_after();
-        const float f = ex2(-rel);
+        const float f = ex2(s - tm);
 #pragma unroll
         for (int c = 0; c < 8; c++) {
           uint32_t a[16];
@@ -367,12 +366,22 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           tmem_st16(acc_addr + c * 16, a);
         }
         tmem_wait_st();
-        s += rel;
-        rc = cj - s;
+        s = tm;
+      }
+      uint8_t* prow = sm + KvSmem::PHI + hf * 2 * TILE_BYTES + row * 128;
+      const float rc = cj - s;
+#pragma unroll
+      for (int c = 0; c < 16; c++) {
+        uint32_t p[4];
+#pragma unroll
+        for (int j = 0; j < 4; j++)
+          p[j] = pack_bf16(ex2(__uint_as_float(v[c * 8 + 2 * j]) + rc), ex2(__uint_as_float(v[c * 8 + 2 * j + 1]) + rc));
+        if (!valid) p[0] = p[1] = p[2] = p[3] = 0u;
+        *reinterpret_cast<uint4*>(prow + (c >> 3) * TILE_BYTES + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
       }
       fence_proxy_async_smem();
       tcgen05_fence_before();
-      mbar_arrive(&misc->phi_full[hf]);
+      mbar_arrive_warp(&misc->phi_full[hf], lane);
       cj = cnext;
       if (per_tile) {                // causal use: the tile's state leaves now, numbered by its tile index
         if (!mbar_wait(&misc->phi_free[hf], it & 1, abortp, status, false)) { alive = false; break; }
@@ -445,8 +454,8 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
   if (threadIdx.x == 0) {
     for (int i = 0; i < OUT_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], 1); }
     mbar_init(&misc->logits_full, 1);
-    mbar_init(&misc->logits_free, EPI_THREADS);
-    for (int i = 0; i < TC_M / 64; i++) mbar_init(&misc->phi_full[i], EPI_THREADS / 2);
+    mbar_init(&misc->logits_free, EPI_THREADS / 32);
+    for (int i = 0; i < TC_M / 64; i++) mbar_init(&misc->phi_full[i], EPI_THREADS / 64);
     mbar_init(&misc->phi_free, 1);
     mbar_init(&misc->const_bar, 1);
     misc->abort_flag = 0;
@@ -643,7 +652,7 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
       }
       tmem_wait_ld();
       tcgen05_fence_before();
-      mbar_arrive(&misc->logits_free);
+      mbar_arrive_warp(&misc->logits_free, lane);
       // the exponent of feature m's column of the state, and w^T A w of both sides, join the logit
 #pragma unroll
       for (int i = 0; i < 128; i += 4) {
@@ -674,7 +683,7 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
         if ((c & 7) == 7) {                     // a 64-feature block of this half is complete
           fence_proxy_async_smem();
           tcgen05_fence_before();
-          mbar_arrive(&misc->phi_full[hf * 2 + (c >> 3)]);
+          mbar_arrive_warp(&misc->phi_full[hf * 2 + (c >> 3)], lane);
         }
       }
     }

@@ -61,7 +61,7 @@ tc_featq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < FQ_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], 1); }
-    for (int i = 0; i < 2; i++) { mbar_init(&misc->logits_full[i], 1); mbar_init(&misc->logits_free[i], EPI_THREADS); }
+    for (int i = 0; i < 2; i++) { mbar_init(&misc->logits_full[i], 1); mbar_init(&misc->logits_free[i], EPI_THREADS / 32); }
     mbar_init(&misc->const_bar, 1);
     misc->abort_flag = 0;
     fence_barrier_init();
@@ -142,7 +142,7 @@ tc_featq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       tmem_wait_ld();
       tcgen05_fence_before();
-      mbar_arrive(&misc->logits_free[buf]);
+      mbar_arrive_warp(&misc->logits_free[buf], lane);
       float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
       for (int i = 0; i < 128; i += 4) {
@@ -302,9 +302,9 @@ tc_causal_out_kernel(const __grid_constant__ CUtensorMap tmPhiQ, const __grid_co
   if (threadIdx.x == 0) {
     mbar_init(&misc->full, 1);
     mbar_init(&misc->s_ready, 1);
-    mbar_init(&misc->s_full, EPI_THREADS);
+    mbar_init(&misc->s_full, EPI_THREADS / 32);
     mbar_init(&misc->out_done, 1);
-    mbar_init(&misc->chunk_free, EPI_THREADS);
+    mbar_init(&misc->chunk_free, EPI_THREADS / 32);
     misc->abort_flag = 0;
     fence_barrier_init();
   }
@@ -423,7 +423,7 @@ tc_causal_out_kernel(const __grid_constant__ CUtensorMap tmPhiQ, const __grid_co
       rsum[hf * TILE + row] = sum;
       fence_proxy_async_smem();
       tcgen05_fence_before();
-      mbar_arrive(&misc->s_full);
+      mbar_arrive_warp(&misc->s_full, lane);
       if (!mbar_wait(&misc->out_done, it & 1, abortp, status, false)) break;
       __syncwarp();
       tcgen05_fence_after();
@@ -454,7 +454,7 @@ tc_causal_out_kernel(const __grid_constant__ CUtensorMap tmPhiQ, const __grid_co
       }
       __syncwarp();
       tcgen05_fence_before();
-      mbar_arrive(&misc->chunk_free);
+      mbar_arrive_warp(&misc->chunk_free, lane);
     }
   }
   tcgen05_fence_before();

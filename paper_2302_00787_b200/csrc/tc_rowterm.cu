@@ -48,8 +48,8 @@ tc_rowterm_kernel(const __grid_constant__ CUtensorMap tmK, const uint8_t* __rest
   volatile int* abortp = &misc->abort_flag;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < RT_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], RT_EPI_THREADS); }
-    for (int i = 0; i < 2; i++) { mbar_init(&misc->t_full[i], 1); mbar_init(&misc->t_free[i], RT_EPI_THREADS); }
+    for (int i = 0; i < RT_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], RT_EPI_THREADS / 32); }
+    for (int i = 0; i < 2; i++) { mbar_init(&misc->t_full[i], 1); mbar_init(&misc->t_free[i], RT_EPI_THREADS / 32); }
     mbar_init(&misc->const_bar, 1);
     misc->abort_flag = 0;
     fence_barrier_init();
@@ -134,8 +134,11 @@ tc_rowterm_kernel(const __grid_constant__ CUtensorMap tmK, const uint8_t* __rest
         }
       }
       tcgen05_fence_before();
-      mbar_arrive(&misc->t_free[buf]);
-      mbar_arrive(&misc->empty[st]);
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&misc->t_free[buf]);
+        mbar_arrive(&misc->empty[st]);
+      }
       out[(size_t)it * TILE] = (part[0] + part[1]) + (part[2] + part[3]);
     }
   }

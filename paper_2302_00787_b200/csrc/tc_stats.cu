@@ -51,7 +51,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < ST_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], 1); }
-    for (int i = 0; i < 2; i++) { mbar_init(&misc->acc_full[i], 1); mbar_init(&misc->acc_free[i], ST_EPI_WARPS * 32); }
+    for (int i = 0; i < 2; i++) { mbar_init(&misc->acc_full[i], 1); mbar_init(&misc->acc_free[i], ST_EPI_WARPS); }
     misc->abort_flag = 0;
     fence_barrier_init();
   }
@@ -127,7 +127,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int j = 0; j < 16; j++) acc[c * 16 + j] += (double)__uint_as_float(t[j]);
       }
       tcgen05_fence_before();
-      mbar_arrive(&misc->acc_free[buf]);
+      mbar_arrive_warp(&misc->acc_free[buf], lane);
     }
     if (alive && row <= TC_D) {
       const int g = pool == FSHARP_POOL_PER_BH ? bh : h;
