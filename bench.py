@@ -156,7 +156,7 @@ def main():
     ap.add_argument("--cpu-baseline-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernel-impl", default="auto", choices=["auto", "simt", "tensor"])
-    ap.add_argument("--streams", type=int, default=2,
+    ap.add_argument("--streams", type=int, default=3,
                     help="steps in flight: step i runs on context i mod S, each context with a stream, scratch and outputs of its own")
     args = ap.parse_args()
 

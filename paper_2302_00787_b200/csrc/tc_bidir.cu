@@ -36,13 +36,13 @@ constexpr int PREFETCH_TILES = 4;   // tiles pulled into L2 ahead of the shared-
 // four epilogue warps, a phi half tile, a pair of barriers, a running shift and a TMEM
 // accumulator per half.  They only share the key / value tiles, the logits MMA and the MMA
 // pipe itself, so while the tensor cores contract one half the other half's exponentials run.
-// The accumulator is kept transposed, acc_h = [V | 1]^T phi_h ([80 used of 128 lanes] x 128
-// columns): one MMA covers N = 128 features instead of 80 value columns.
+// The accumulator of half h is acc_h = phi_h^T [V | 1] (128 feature lanes x 80 columns: the phi half
+// tile is the M-side operand, [V | 1] the N = 80 side), so a contraction step costs 80 columns of the
+// tensor pipe instead of 128, and every epilogue thread (= one feature) takes part when the state leaves.
 struct KvSmem {
   static constexpr uint32_t X0 = 0, V0 = 2 * TILE_BYTES, ONES = 4 * TILE_BYTES, W = ONES + TILE_BYTES,
                             WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES, FA2 = PHI + 4 * TILE_BYTES,
-                            STG = FA2 + TC_M * 4,        // two 2 KB buffers per storing epilogue warp: accumulator rows on their way out
-                            MISC = STG + 8 * 2048, TOTAL = MISC + 256;
+                            MISC = FA2 + TC_M * 4, TOTAL = MISC + 256;
 };
 static_assert(KvSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 static_assert(KvSmem::PHI % 1024 == 0 && KvSmem::W % 1024 == 0 && KvSmem::ONES % 1024 == 0, "swizzled tiles need 1024-byte alignment");
@@ -51,6 +51,10 @@ struct KvMisc {
   // key and value tiles have barriers of their own: a key tile is free again once the logits MMA that read it
   // has completed, long before the contraction that reads the value tile of the same stage
   uint64_t fullK[2], emptyK[2], fullV[2], emptyV[2], logits_full, logits_free, phi_full[2], phi_free[2], const_bar;
+  // turn[h]: half h may run its exponentials.  The halves take turns (each arrives on the other's barrier when its
+  // exponentials are done), so one half has the exponential unit to itself while the other half's contraction
+  // runs on the tensor cores and its warps load and scan the next tile's logits.
+  uint64_t turn[2];
   uint32_t tmem_base;
   int abort_flag;
   int tile_max[2][4];     // per half: [0..2] rotating slots of the per-tile maximum
@@ -58,12 +62,12 @@ struct KvMisc {
 };
 static_assert(sizeof(KvMisc) <= 256, "misc block");
 
-constexpr uint32_t KV_COL_LOGITS = 0, KV_COL_ACC = 256;   // TMEM columns; half h accumulates at KV_COL_ACC + 128 h
+constexpr uint32_t KV_COL_LOGITS = 0, KV_COL_ACC = 256;   // TMEM columns; half h accumulates at KV_COL_ACC + 80 h
 constexpr int HALF_THREADS = EPI_THREADS / 2;
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-             const __grid_constant__ CUtensorMap tmPhi, const __grid_constant__ CUtensorMap tmState,
+             const __grid_constant__ CUtensorMap tmPhi,
              const uint8_t* __restrict__ images, const float* __restrict__ crow, int H, int pool, int L, int Lpad,
              int tiles_per_split, int nsplit, float* __restrict__ partial, float* __restrict__ shifts,
              int* __restrict__ pmax, int per_tile, int* __restrict__ status) {
@@ -89,9 +93,10 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       mbar_init(&misc->fullK[i], 1);
       mbar_init(&misc->emptyK[i], 1);
       mbar_init(&misc->fullV[i], 1);
-      mbar_init(&misc->emptyV[i], 1);
+      mbar_init(&misc->emptyV[i], 2);
       mbar_init(&misc->phi_full[i], HALF_THREADS / 32);
       mbar_init(&misc->phi_free[i], 1);
+      mbar_init(&misc->turn[i], HALF_THREADS / 32);
       for (int j = 0; j < 4; j++) misc->tile_max[i][j] = f2ord(-INFINITY);
     }
     for (int j = 0; j < 3; j++) misc->chunk_max[j] = f2ord(-INFINITY);
@@ -164,19 +169,15 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       for (int it = max(0, issuedV - 2); it < issuedV; it++) mbar_wait(&misc->fullV[it & 1], (it >> 1) & 1, abortp, status, false);
     }
   } else if (warp == WARP_MMA) {
+    // ---------------- logits MMAs.  Issuing an MMA costs its thread about a hundred cycles (descriptor arithmetic
+    // and the moves into uniform registers, on a scheduler shared with two epilogue warps), so the three MMA
+    // streams of a tile have an issuing warp each: this one the logits, the next two a feature half each.
     if (lane == 0) {
       constexpr uint32_t ID_LOGITS = idesc_bf16(128, TC_M, 0, 0);
-      constexpr uint32_t ID_KV = idesc_bf16(128, 128, 1, 1);       // [V | 1]^T phi_h
-      const uint32_t sV0 = smem_u32(sm + KvSmem::V0), sOnes = smem_u32(sm + KvSmem::ONES);
       // descriptors are built once; inside the loops each MMA costs one add per operand
       const uint64_t dX0 = smem_desc(smem_u32(sm + KvSmem::X0), 16, 1024, SWZ_128B);
       const uint64_t dW = smem_desc(smem_u32(sm + KvSmem::W), 16, 1024, SWZ_128B);
       const uint64_t dWlo = smem_desc(smem_u32(sm + KvSmem::WLO), 16, 1024, SWZ_128B);
-      // phi half h as an operand whose 128 features are the contiguous index: two 64-feature blocks
-      const uint64_t dPhi = smem_desc(smem_u32(sm + KvSmem::PHI), TILE_BYTES, 1024, SWZ_128B);
-      // [V | 1] with the value index contiguous: block 0 = the V tile of the stage, block 1 = the ones tile
-      const uint64_t dVst0 = smem_desc(sV0, sOnes - sV0, 1024, SWZ_128B);
-      const uint64_t dVst1 = smem_desc(sV0 + TILE_BYTES, sOnes - sV0 - TILE_BYTES, 1024, SWZ_128B);
       auto issue_logits = [&](int st) {
         const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
 #pragma unroll
@@ -194,34 +195,45 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         tcgen05_fence_after();
         issue_logits(0);
       }
-      for (int it = 0; ok && it < ntiles; it++) {
+      for (int it = 0; ok && it + 1 < ntiles; it++) {
+        const int sn = (it + 1) & 1;
+        if (!mbar_wait(&misc->fullK[sn], ((it + 1) >> 1) & 1, abortp, status)) break;
+        if (!mbar_wait(&misc->logits_free, it & 1, abortp, status)) break;
+        tcgen05_fence_after();
+        issue_logits(sn);
+      }
+    }
+  } else {
+    // ---------------- contraction of feature half hh = warp - (WARP_MMA + 1)
+    if (lane == 0) {
+      const int hh = warp - (WARP_MMA + 1);
+      constexpr uint32_t ID_KV = idesc_bf16(128, TC_NV, 1, 1);     // phi_h^T [V | 1]
+      const uint32_t sV0 = smem_u32(sm + KvSmem::V0), sOnes = smem_u32(sm + KvSmem::ONES);
+      // phi half hh as the operand whose 128 features (M) are the contiguous index: two 64-feature blocks
+      const uint64_t dPhi = smem_desc(smem_u32(sm + KvSmem::PHI) + hh * 2 * TILE_BYTES, TILE_BYTES, 1024, SWZ_128B);
+      // [V | 1] with the value index (N = 80) contiguous: block 0 = the V tile of the stage, block 1 = the ones
+      // tile, of which the first 16 columns are read
+      const uint64_t dVst0 = smem_desc(sV0, sOnes - sV0, 1024, SWZ_128B);
+      const uint64_t dVst1 = smem_desc(sV0 + TILE_BYTES, sOnes - sV0 - TILE_BYTES, 1024, SWZ_128B);
+      for (int it = 0; it < ntiles; it++) {
         const int st = it & 1;
-        if (it + 1 < ntiles) {
-          if (!mbar_wait(&misc->fullK[st ^ 1], ((it + 1) >> 1) & 1, abortp, status)) break;
-          if (!mbar_wait(&misc->logits_free, it & 1, abortp, status)) break;
-          tcgen05_fence_after();
-          issue_logits(st ^ 1);
-        }
         if (!mbar_wait(&misc->fullV[st], (it >> 1) & 1, abortp, status)) break;
         const uint64_t dV = st ? dVst1 : dVst0;
         const uint32_t acc0 = (it > 0 && !per_tile) ? 1u : 0u;      // causal use: every tile starts afresh
-#pragma unroll 1
-        for (int hh = 0; hh < 2 && ok; hh++) {
-          if (!mbar_wait(&misc->phi_full[hh], it & 1, abortp, status)) { ok = false; break; }
-          tcgen05_fence_after();
-          if (per_tile) {                 // the half tile also goes out as it is (two 64-feature blocks)
-            tma_store_3d(&tmPhi, sm + KvSmem::PHI + (2 * hh) * TILE_BYTES, (2 * hh) * 64, (tile0 + it) * TILE, bh);
-            tma_store_3d(&tmPhi, sm + KvSmem::PHI + (2 * hh + 1) * TILE_BYTES, (2 * hh + 1) * 64, (tile0 + it) * TILE, bh);
-            bulk_commit();
-          }
-#pragma unroll 2
-          for (int k = 0; k < TILE / 16; k++)
-            mma_bf16(tmem + KV_COL_ACC + hh * 128, desc_advance(dV, k * 2048),
-                     desc_advance(dPhi, hh * 2 * TILE_BYTES + k * 2048), ID_KV, k > 0 ? 1u : acc0);
-          if (per_tile) bulk_wait_read0();       // the store has read the half tile: it may be overwritten
-          mma_commit(&misc->phi_free[hh]);
+        if (!mbar_wait(&misc->phi_full[hh], it & 1, abortp, status)) break;
+        tcgen05_fence_after();
+        if (per_tile) {                 // the half tile also goes out as it is (two 64-feature blocks)
+          tma_store_3d(&tmPhi, sm + KvSmem::PHI + (2 * hh) * TILE_BYTES, (2 * hh) * 64, (tile0 + it) * TILE, bh);
+          tma_store_3d(&tmPhi, sm + KvSmem::PHI + (2 * hh + 1) * TILE_BYTES, (2 * hh + 1) * 64, (tile0 + it) * TILE, bh);
+          bulk_commit();
         }
-        mma_commit(&misc->emptyV[st]);
+#pragma unroll
+        for (int k = 0; k < TILE / 16; k++)
+          mma_bf16(tmem + KV_COL_ACC + hh * TC_NV, desc_advance(dPhi, k * 2048), desc_advance(dV, k * 2048), ID_KV,
+                   k > 0 ? 1u : acc0);
+        if (per_tile) bulk_wait_read0();         // the store has read the half tile: it may be overwritten
+        mma_commit(&misc->phi_free[hh]);
+        mma_commit(&misc->emptyV[st]);           // the value tile is free once both halves' contractions have completed
       }
       if (per_tile) bulk_wait0();
     }
@@ -235,56 +247,31 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     const int q = warp & 3, hf = warp >> 2;
     const int row = q * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
-    const uint32_t acc_addr = lane_addr + KV_COL_ACC + hf * 128;
+    const uint32_t acc_addr = lane_addr + KV_COL_ACC + hf * TC_NV;      // this thread's lane: feature hf * 128 + row
     int* tmax = misc->tile_max[hf];
     const float* cptr = crow + (size_t)bh * Lpad + (size_t)tile0 * TILE + row;
     float s = 0.f;
     float cj = ntiles > 0 ? cptr[0] : 0.f;
     bool alive = true;
+    if (hf == 1) mbar_arrive_warp(&misc->turn[0], lane);     // half 0 goes first
     // accumulator of this half -> partial `slot` (the contraction that feeds it has completed)
     auto write_partial = [&](size_t slot) {
       __syncwarp();
       tcgen05_fence_after();
+      // thread = feature m: its row of the accumulator is column m of the state [80][256]; a store instruction of
+      // the warp covers 32 consecutive features of one state row (128 contiguous bytes).  Rows 65..79 are not written.
+      float* out = partial + slot * TC_NV * TC_M + hf * 128 + row;
       float amax = 0.f;
-      if (q < 2) {
-        // rows 0..63: 16 columns at a time go into a 2 KB shared-memory buffer (32 rows x 64 bytes, 64-byte
-        // swizzle) that a bulk tensor store takes from there; two buffers per warp, so that the warp fills one
-        // while the other is being read.  The stores run on while the warp goes back to the next tile.
-        uint8_t* stg0 = sm + KvSmem::STG + (hf * 2 + q) * 4096;
 #pragma unroll
-        for (int c = 0; c < 8; c++) {
-          uint8_t* stg = stg0 + (c & 1) * 2048;
-          uint32_t a[16];
-          tmem_ld16(acc_addr + c * 16, a);
-          if (lane == 0) bulk_wait_read1();           // the store that last read this buffer (two stores back)
-          __syncwarp();
-          tmem_wait_ld();
+      for (int c = 0; c < 5; c++) {
+        uint32_t a[16];
+        tmem_ld16(acc_addr + c * 16, a);
+        tmem_wait_ld();
 #pragma unroll
-          for (int j = 0; j < 16; j++) amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
-#pragma unroll
-          for (int i = 0; i < 4; i++)
-            *reinterpret_cast<uint4*>(stg + lane * 64 + ((i ^ ((lane >> 1) & 3)) << 4)) = make_uint4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) {
-            tma_store_3d(&tmState, stg, hf * 128 + c * 16, q * 32, (int)slot);
-            bulk_commit();
-          }
-        }
-      } else if (q == 2) {
-        // row 64 (the normaliser's row) is one lane's: it goes out directly
-        float* out = partial + slot * TC_NV * TC_M + hf * 128 + (size_t)TC_DV * TC_M;
-#pragma unroll
-        for (int c = 0; c < 8; c++) {
-          uint32_t a[16];
-          tmem_ld16(acc_addr + c * 16, a);
-          tmem_wait_ld();
-          if (lane == 0) {
-#pragma unroll
-            for (int j = 0; j < 16; j++) amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
-#pragma unroll
-            for (int i = 0; i < 4; i++)
-              *reinterpret_cast<uint4*>(out + c * 16 + i * 4) = make_uint4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
+        for (int j = 0; j < 16; j++) {
+          if (c * 16 + j <= TC_DV) {
+            amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
+            out[(size_t)(c * 16 + j) * TC_M] = __uint_as_float(a[j]);
           }
         }
       }
@@ -357,7 +344,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         tcgen05_fence_after();
         const float f = ex2(s - tm);
 #pragma unroll
-        for (int c = 0; c < 8; c++) {
+        for (int c = 0; c < 5; c++) {
           uint32_t a[16];
           tmem_ld16(acc_addr + c * 16, a);
           tmem_wait_ld();
@@ -370,6 +357,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       }
       uint8_t* prow = sm + KvSmem::PHI + hf * 2 * TILE_BYTES + row * 128;
       const float rc = cj - s;
+      if (!mbar_wait(&misc->turn[hf], it & 1, abortp, status, false)) { alive = false; break; }
 #pragma unroll
       for (int c = 0; c < 16; c++) {
         uint32_t p[4];
@@ -382,6 +370,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       fence_proxy_async_smem();
       tcgen05_fence_before();
       mbar_arrive_warp(&misc->phi_full[hf], lane);
+      mbar_arrive_warp(&misc->turn[hf ^ 1], lane);
       cj = cnext;
       if (per_tile) {                // causal use: the tile's state leaves now, numbered by its tile index
         if (!mbar_wait(&misc->phi_free[hf], it & 1, abortp, status, false)) { alive = false; break; }
@@ -391,7 +380,6 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     // write this split's partial [V | 1]^T phi_h (fp32, rows 0..79), its shift and its largest magnitude
     if (alive && ntiles > 0 && !per_tile && mbar_wait(&misc->phi_free[hf], (ntiles - 1) & 1, abortp, status, false))
       write_partial((size_t)bh * nsplit + split);
-    if (q < 2 && lane == 0) bulk_wait0();              // this thread's state stores have completed before the block ends
   }
   tcgen05_fence_before();
   __syncthreads();
@@ -426,10 +414,11 @@ static_assert(OutSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 struct OutMisc {
   // phi_full[f]: the 64-feature block f of the phi tile is written (the 128 threads of its half arrive)
   uint64_t full[OUT_STAGES], empty[OUT_STAGES], logits_full, logits_free, phi_full[TC_M / 64], phi_free, const_bar;
+
   uint32_t tmem_base;
   int abort_flag;
 };
-// TMEM columns: logits, then [num | den] of feature half 0 and of feature half 1
+// TMEM columns: logits, then [num | den]
 constexpr uint32_t OUT_COL_LOGITS = 0, OUT_COL_OUT = 256;
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -493,14 +482,12 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
         mbar_wait(&misc->full[it % OUT_STAGES], (it / OUT_STAGES) & 1, abortp, status, false);
     }
   } else if (warp == WARP_MMA) {
+    // ---------------- logits MMAs (the two warps after this one issue the contractions, a feature half each)
     if (lane == 0) {
       constexpr uint32_t ID_LOGITS = idesc_bf16(128, TC_M, 0, 0);
-      constexpr uint32_t ID_OUT = idesc_f16(128, TC_NV, 0, 0);      // fp16: phi(Q) <= 1 and a state of order one per feature
       const uint64_t dX0 = smem_desc(smem_u32(sm + OutSmem::X0), 16, 1024, SWZ_128B);
       const uint64_t dW = smem_desc(smem_u32(sm + OutSmem::W), 16, 1024, SWZ_128B);
       const uint64_t dWlo = smem_desc(smem_u32(sm + OutSmem::WLO), 16, 1024, SWZ_128B);
-      const uint64_t dPhi = smem_desc(smem_u32(sm + OutSmem::PHI), 16, 1024, SWZ_128B);
-      const uint64_t dKvt = smem_desc(smem_u32(sm + OutSmem::KVT), 16, 1024, SWZ_128B);
       auto issue_logits = [&](int st) {
         const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
 #pragma unroll
@@ -518,37 +505,51 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
         tcgen05_fence_after();
         issue_logits(0);
       }
+      for (int it = 0; ok && it + 1 < ntiles; it++) {
+        const int sn = (it + 1) % OUT_STAGES;
+        if (!mbar_wait(&misc->full[sn], ((it + 1) / OUT_STAGES) & 1, abortp, status)) break;
+        if (!mbar_wait(&misc->logits_free, it & 1, abortp, status)) break;
+        // The tensor pipe runs MMAs in the order they were issued: the last contraction steps of tile it - 1, which
+        // the epilogue is about to wait for, go before the next tile's logits, which nobody needs for a whole tile.
+        if (it > 0 && !mbar_wait(&misc->phi_free, (it - 1) & 1, abortp, status)) break;
+        tcgen05_fence_after();
+        issue_logits(sn);
+      }
+    }
+  } else if (warp == WARP_MMA + 1) {
+    // ---------------- contraction: every 64-feature block of phi is contracted as soon as it is written, first
+    // blocks of both halves first, so only the last block's MMAs are left when the exponentials end.  One
+    // accumulator [num | den] for all 256 features (the two threads of a row agree on the row's shift).
+    if (lane == 0) {
+      constexpr uint32_t ID_OUT = idesc_f16(128, TC_NV, 0, 0);      // fp16: phi(Q) <= 1 and a state of order one per feature
+      const uint64_t dPhi = smem_desc(smem_u32(sm + OutSmem::PHI), 16, 1024, SWZ_128B);
+      const uint64_t dKvt = smem_desc(smem_u32(sm + OutSmem::KVT), 16, 1024, SWZ_128B);
+      bool ok = true;
       for (int it = 0; ok && it < ntiles; it++) {
-        if (it + 1 < ntiles) {
-          const int sn = (it + 1) % OUT_STAGES;
-          if (!mbar_wait(&misc->full[sn], ((it + 1) / OUT_STAGES) & 1, abortp, status)) break;
-          if (!mbar_wait(&misc->logits_free, it & 1, abortp, status)) break;
-          tcgen05_fence_after();
-          issue_logits(sn);
-        }
-        // Every 64-feature block of phi is contracted as soon as it is written, first blocks of both
-        // halves first, so only the last block's MMAs are left when the exponentials end.  The
-        // epilogue arrives on a tile's first block only after it has read the previous tile's outputs.
-#pragma unroll 1
-        for (int o = 0; o < TC_M / 64 && ok; o++) {
-          const int fb = ((o & 1) << 1) | (o >> 1);      // 0, 2, 1, 3: feature halves 0 (fb 0, 1) and 1 (fb 2, 3)
-          if (!mbar_wait(&misc->phi_full[fb], it & 1, abortp, status)) { ok = false; break; }
+        // An epilogue thread arrives on its half's first block only after it has read the previous tile's output
+        // row, so the accumulator may be overwritten once the first blocks of BOTH halves are in.
+        if (!mbar_wait(&misc->phi_full[0], it & 1, abortp, status)) break;
+        if (!mbar_wait(&misc->phi_full[2], it & 1, abortp, status)) break;
+#pragma unroll
+        for (int o = 0; o < TC_M / 64; o++) {
+          const int fb = ((o & 1) << 1) | (o >> 1);      // 0, 2, 1, 3
+          if (o >= 2 && !mbar_wait(&misc->phi_full[fb], it & 1, abortp, status)) { ok = false; break; }
           tcgen05_fence_after();
 #pragma unroll
           for (int k = 0; k < 4; k++)
-            mma_bf16(tmem + OUT_COL_OUT + (fb >> 1) * TC_NV, desc_advance(dPhi, fb * TILE_BYTES + 32 * k),
-                     desc_advance(dKvt, fb * KVT_BLOCK_BYTES + 32 * k), ID_OUT, ((fb & 1) || k > 0) ? 1u : 0u);
+            mma_bf16(tmem + OUT_COL_OUT, desc_advance(dPhi, fb * TILE_BYTES + 32 * k),
+                     desc_advance(dKvt, fb * KVT_BLOCK_BYTES + 32 * k), ID_OUT, (o > 0 || k > 0) ? 1u : 0u);
         }
-        mma_commit(&misc->phi_free);
+        if (ok) mma_commit(&misc->phi_free);
       }
     }
   }
   } else {
     regs_acquire<REGS_EPILOGUE>();
     // ---------------- epilogue warps: one query row per thread, 128 of the 256 features.
-    // Each half row is shifted by its own maximum, so no exchange between the two threads of a
-    // row precedes the exponentials; the two halves are contracted into separate accumulators and
-    // brought to the common shift when the tile's output is read (one tile later).
+    // The two threads of a row exchange the maxima of their half rows (through shared memory, the
+    // two warps of a row quarter meeting at a barrier of their own), so the row has one shift and
+    // both halves are contracted into one accumulator, read when the next tile's maxima are known.
     const int q = warp & 3, hf = warp >> 2;
     const int row = q * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
@@ -601,23 +602,17 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
     auto write_out = [&](int j) {
       __syncwarp();
       tcgen05_fence_after();
-      uint32_t n0[32], n1[32], d0[16], d1[16];
+      uint32_t n0[32], d0[16];
       const uint32_t base = lane_addr + OUT_COL_OUT;
       tmem_ld16(base + hf * 32, reinterpret_cast<uint32_t(&)[16]>(n0[0]));
       tmem_ld16(base + hf * 32 + 16, reinterpret_cast<uint32_t(&)[16]>(n0[16]));
       tmem_ld16(base + TC_DV, d0);
-      tmem_ld16(base + TC_NV + hf * 32, reinterpret_cast<uint32_t(&)[16]>(n1[0]));
-      tmem_ld16(base + TC_NV + hf * 32 + 16, reinterpret_cast<uint32_t(&)[16]>(n1[16]));
-      tmem_ld16(base + TC_NV + TC_DV, d1);
       tmem_wait_ld();
-      const float* rm = rowmax + (j % 3) * 2 * TILE;
-      const float m0 = rm[row], m1 = rm[TILE + row];
-      const float m = fmaxf(m0, m1);
-      const float f0 = ex2(m0 - m), f1 = ex2(m1 - m);
       const int64_t r0 = (int64_t)(tile0 + j) * TILE + q * 32;       // first row of this warp
-      const float den = fmaf(f0, __uint_as_float(d0[0]), f1 * __uint_as_float(d1[0]));
+      const float den = __uint_as_float(d0[0]);
       if (r0 + lane < L && (!(den > 0.f) || !isfinite(den))) atomicExch(status, FSHARP_E_NONFINITE);
-      const float i0 = f0 / den, i1 = f1 / den;
+      float inv;                       // outputs are rounded to bf16: the approximate reciprocal (1 ulp) is exact enough
+      asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(den));
       // The thread's 64 bytes go through shared memory so that a store instruction of the warp
       // covers 8 rows x 64 contiguous bytes instead of 32 rows x 16 bytes.
       uint8_t* stg = sm + OutSmem::STAGE + warp * 2048;
@@ -626,8 +621,7 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
         uint32_t o[4];
 #pragma unroll
         for (int e = 0; e < 4; e++)
-          o[e] = pack_bf16(fmaf(i0, __uint_as_float(n0[8 * i + 2 * e]), i1 * __uint_as_float(n1[8 * i + 2 * e])),
-                           fmaf(i0, __uint_as_float(n0[8 * i + 2 * e + 1]), i1 * __uint_as_float(n1[8 * i + 2 * e + 1])));
+          o[e] = pack_bf16(inv * __uint_as_float(n0[8 * i + 2 * e]), inv * __uint_as_float(n0[8 * i + 2 * e + 1]));
         *reinterpret_cast<uint4*>(stg + lane * 64 + ((i ^ ((lane >> 1) & 3)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
       }
       __syncwarp();
@@ -665,8 +659,12 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
       float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
       for (int i = 0; i < 128; i++) mxp[i & 3] = fmaxf(mxp[i & 3], __uint_as_float(v[i]));
-      const float mx = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
-      rowmax[(it % 3) * 2 * TILE + hf * TILE + row] = mx;
+      float mx = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
+      // the other half of the row: its thread sits in warp q of the other warpgroup (slots rotate over two tiles:
+      // a slot is rewritten only after both warps have passed the next tile's barrier)
+      rowmax[(it & 1) * 2 * TILE + hf * TILE + row] = mx;
+      named_bar_sync(2 + q, 64);
+      mx = fmaxf(mx, rowmax[(it & 1) * 2 * TILE + (hf ^ 1) * TILE + row]);
       if (it > 0) {
         // contraction of the previous tile done: its phi tile and its outputs are ours again
         if (!mbar_wait(&misc->phi_free, (it - 1) & 1, abortp, status, false)) { alive = false; break; }
@@ -723,7 +721,6 @@ namespace tchost {
 int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int H, int L, int inner);
 int make_map_kvt(CUtensorMap* map, const void* base, int BH, int bf16);
 int make_map_feat(CUtensorMap* map, const void* base, int BH, int Lpad);
-int make_map_state(CUtensorMap* map, const void* base, size_t slots);
 }  // namespace tchost
 int fs_tc_rowterm(fsharp_ctx* ctx, const void* K, const fsharp_dims* dm, const uint8_t* images, const int* flags, int Lpad,
                   int tiles_per_split, int nsplit, float* crow);
@@ -754,8 +751,7 @@ int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_d
   const int B = dm->B, H = dm->H, Lk = dm->Lk;
   const int Lpad = (Lk + TILE - 1) / TILE * TILE;
   FS_TRY(fs_tc_rowterm(ctx, K, dm, images, flags, Lpad, tiles_per_split, nsplit, crow));
-  CUtensorMap tmK, tmV, tmPhi, tmState;
-  FS_TRY(tchost::make_map_state(&tmState, partial, (size_t)B * H * (phik != nullptr ? (size_t)((Lk + TILE - 1) / TILE) : (size_t)nsplit)));
+  CUtensorMap tmK, tmV, tmPhi;
   FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, Lk, dm->d), B, H, Lk, dm->d));
   FS_TRY(tchost::make_map_tokens(&tmV, V, fs_addr(dm->v_stride, H, Lk, dm->dv), B, H, Lk, dm->dv));
   if (phik != nullptr) FS_TRY(tchost::make_map_feat(&tmPhi, phik, B * H, Lpad));
@@ -763,7 +759,7 @@ int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_d
   FS_CUDA_OK(cudaFuncSetAttribute(tc_kv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KvSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_KV);
   tc_kv_kernel<<<dim3(nsplit, B * H), TC_THREADS, KvSmem::TOTAL + 1024, ctx->stream>>>(
-      tmK, tmV, tmPhi, tmState, images, crow, H, dm->pool, Lk, Lpad, tiles_per_split, nsplit, partial, shifts, pmax,
+      tmK, tmV, tmPhi, images, crow, H, dm->pool, Lk, Lpad, tiles_per_split, nsplit, partial, shifts, pmax,
       phik != nullptr ? 1 : 0, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);

@@ -70,21 +70,6 @@ int make_map_kvt(CUtensorMap* map, const void* base, int BH, int bf16) {
   return r == CUDA_SUCCESS ? FSHARP_OK : FSHARP_E_CUDA;
 }
 
-// key-side states [slots, 80, 256] fp32 -> 3-D map (feature, row, slot), box 16 x 32 x 1 (2 KB), 64-byte swizzle:
-// the stores of the key-side kernel's accumulator rows.
-int make_map_state(CUtensorMap* map, const void* base, size_t slots) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return FSHARP_E_CUDA;
-  cuuint64_t dims[3] = {(cuuint64_t)TC_M, (cuuint64_t)TC_NV, (cuuint64_t)slots};
-  cuuint64_t strides[2] = {(cuuint64_t)TC_M * 4, (cuuint64_t)TC_M * TC_NV * 4};
-  cuuint32_t box[3] = {16, 32, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? FSHARP_OK : FSHARP_E_CUDA;
-}
-
 // bf16 features [BH, Lpad, 256] -> 3-D map (feature, token, bh), box 64 x 128 x 1, 128-byte swizzle.
 int make_map_feat(CUtensorMap* map, const void* base, int BH, int Lpad) {
   EncodeTiledFn fn = encode_fn();

@@ -7,9 +7,10 @@ namespace tcl {
 constexpr int TC_D = 64, TC_M = 256, TC_DV = 64;
 constexpr int TC_NV = 80;          // dv + 1 (the ones column of [V | 1]) padded to a multiple of 16
 constexpr int TILE = 128;          // tokens per tile
-// Warps 0-7 are the epilogue (two warpgroups); warps 8-11 form the producer warpgroup, of which
-// warp 8 issues the TMA copies, warp 9 the MMAs, and 10-11 only take part in the register hand-over:
-// the producer warpgroup shrinks to REGS_PRODUCER registers per thread so that the epilogue
+// Warps 0-7 are the epilogue (two warpgroups); warps 8-11 form the producer warpgroup: warp 8 issues the TMA
+// copies, warp 9 the MMAs (in the bidirectional kernels: the logits MMAs, while warps 10 and 11 issue the
+// contractions of one feature half each; elsewhere 10-11 only take part in the register hand-over).
+// The producer warpgroup shrinks to REGS_PRODUCER registers per thread so that the epilogue
 // warpgroups can grow to REGS_EPILOGUE (384 threads x 168 at launch = 128 x 40 + 256 x 232).
 constexpr int EPI_THREADS = 256, WARP_TMA = 8, WARP_MMA = 9, TC_THREADS = 384;
 constexpr int REGS_PRODUCER = 40, REGS_EPILOGUE = 232;
