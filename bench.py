@@ -369,8 +369,7 @@ def main():
 
 # DRAM bytes per launch (read + write) from the ncu captures summarised under profiles/ (same kernels, same workload);
 # an entry is dropped when its kernel changes.
-NCU_TRAFFIC = {("cfg2", "fit_kernel"): 4.39e6, ("cfg2", "tc_kv_kernel"): 75.3e6, ("cfg2", "tc_out_kernel"): 48.4e6,
-               ("cfg2", "tc_stats_kernel"): 71.9e6, ("cfg3", "tc_kv_kernel"): 533.5e6, ("cfg3", "tc_causal_out_kernel"): 626.2e6}
+NCU_TRAFFIC = {("cfg2", "fit_kernel"): 4.39e6, ("cfg2", "tc_kv_kernel"): 74.9e6, ("cfg2", "tc_out_kernel"): 48.8e6}
 
 
 def roofline_for(name, k, w, work, peaks):
