@@ -260,7 +260,10 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       tcgen05_fence_after();
       // thread = feature m: its row of the accumulator is column m of the state [80][256]; a store instruction of
       // the warp covers 32 consecutive features of one state row (128 contiguous bytes).  Rows 65..79 are not written.
+      // Causal use: a chunk's state is only ever read back as a term of a prefix that is itself rounded to bf16,
+      // so it is stored as bf16 (half the bytes of the kernel's largest output).
       float* out = partial + slot * TC_NV * TC_M + hf * 128 + row;
+      __nv_bfloat16* out16 = reinterpret_cast<__nv_bfloat16*>(partial) + slot * TC_NV * TC_M + hf * 128 + row;
       float amax = 0.f;
 #pragma unroll
       for (int c = 0; c < 5; c++) {
@@ -271,7 +274,8 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         for (int j = 0; j < 16; j++) {
           if (c * 16 + j <= TC_DV) {
             amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
-            out[(size_t)(c * 16 + j) * TC_M] = __uint_as_float(a[j]);
+            if (per_tile) out16[(size_t)(c * 16 + j) * TC_M] = __float2bfloat16_rn(__uint_as_float(a[j]));
+            else out[(size_t)(c * 16 + j) * TC_M] = __uint_as_float(a[j]);
           }
         }
       }
@@ -744,7 +748,8 @@ size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
 // Key side: the per-key quadratic term, then the feature / contraction kernel.  crow: [B*H][Lpad] floats,
 // Lpad = ceil(Lk / 128) * 128; partial: [B*H][nsplit][80][256] floats; shifts, pmax: [B*H][nsplit][2], pmax
 // zeroed by the caller.  phik (may be null; causal use): bf16 [B*H][Lpad][256]; with it every 128-key tile
-// is a chunk of its own and partial, shifts, pmax are indexed by tile: [B*H][ceil(Lk / 128)] entries.
+// is a chunk of its own, shifts and pmax are indexed by tile ([B*H][ceil(Lk / 128)] entries) and partial
+// holds bf16 states [B*H][ceil(Lk / 128)][80][256].
 int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                    const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax,
                    __nv_bfloat16* phik) {

@@ -196,7 +196,7 @@ tc_featq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 // ------------------------------------------------------------------------------------------
 // exclusive scan over chunks
 // ------------------------------------------------------------------------------------------
-// state[bh][c]: [80][256] fp32, chunk c's [V | 1]^T phiK with phiK = 2^(exponent - s_c); pmax its largest
+// state[bh][c]: [80][256] bf16, chunk c's [V | 1]^T phiK with phiK = 2^(exponent - s_c); pmax its largest
 // magnitude.  For every chunk c the kernel writes
 //   prefix[bh][c] = alpha_c 2^(-e_c) sum_{c' < c} 2^(s_c' - sigma_c) state[c']   (bf16),
 //   beta[bh][c],
@@ -205,7 +205,7 @@ tc_featq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 constexpr int PFX_SLICES = 10;               // 80 x 256 elements = 10 x 256 threads x 8
 constexpr int PFX_MAXCH = 1024;
 __global__ void __launch_bounds__(256)
-tc_causal_prefix_kernel(const float* __restrict__ state, const float* __restrict__ shifts, const int* __restrict__ pmax,
+tc_causal_prefix_kernel(const __nv_bfloat16* __restrict__ state, const float* __restrict__ shifts, const int* __restrict__ pmax,
                         int nch, __nv_bfloat16* __restrict__ prefix, float* __restrict__ beta) {
   __shared__ float up[PFX_MAXCH], add[PFX_MAXCH], oscale[PFX_MAXCH];
   const int bh = blockIdx.y;
@@ -233,32 +233,32 @@ tc_causal_prefix_kernel(const float* __restrict__ state, const float* __restrict
     }
   }
   __syncthreads();
-  // thread t of slice x owns rows 8x .. 8x+7 of column t
-  const float* sb = state + (size_t)bh * nch * TC_NV * TC_M;
-  __nv_bfloat16* pb = prefix + (size_t)bh * nch * TC_NV * TC_M;
-  float R[8];
+  // thread t of slice x owns columns 2 (t % 128), 2 (t % 128) + 1 of rows 8x + 4 (t / 128) .. + 3: states come in
+  // and prefixes go out as bf16 pairs (4-byte accesses, a warp's access = 128 contiguous bytes)
+  const int cp = threadIdx.x & 127, n0 = blockIdx.x * 8 + (threadIdx.x >> 7) * 4;
+  const uint32_t* sb = reinterpret_cast<const uint32_t*>(state + (size_t)bh * nch * TC_NV * TC_M) + cp;
+  uint32_t* pb = reinterpret_cast<uint32_t*>(prefix + (size_t)bh * nch * TC_NV * TC_M) + cp;
+  float R[4][2];
 #pragma unroll
-  for (int u = 0; u < 8; u++) R[u] = 0.f;
-  // four chunks per trip: their loads are issued together, then the running sums move on
-  for (int c0 = 0; c0 < nch; c0 += 4) {
-    float kv[4][8];
+  for (int u = 0; u < 4; u++) R[u][0] = R[u][1] = 0.f;
+  // eight chunks per trip: their loads are issued together, then the running sums move on
+  for (int c0 = 0; c0 < nch; c0 += 8) {
+    uint32_t kv[8][4];
 #pragma unroll
-    for (int k = 0; k < 4; k++)
+    for (int k = 0; k < 8; k++)
 #pragma unroll
-      for (int u = 0; u < 8; u++) {
-        const int n = blockIdx.x * 8 + u;
-        kv[k][u] = (c0 + k < nch && n <= TC_DV) ? sb[((size_t)(c0 + k) * TC_NV + n) * TC_M + threadIdx.x] : 0.f;
-      }
+      for (int u = 0; u < 4; u++)
+        kv[k][u] = (c0 + k < nch && n0 + u <= TC_DV) ? sb[((size_t)(c0 + k) * TC_NV + n0 + u) * (TC_M / 2)] : 0u;
 #pragma unroll
-    for (int k = 0; k < 4; k++) {
+    for (int k = 0; k < 8; k++) {
       const int c = c0 + k;
       if (c < nch) {
         const float os = oscale[c], upc = up[c], adc = add[c];
 #pragma unroll
-        for (int u = 0; u < 8; u++) {
-          const int n = blockIdx.x * 8 + u;
-          pb[((size_t)c * TC_NV + n) * TC_M + threadIdx.x] = __float2bfloat16_rn(R[u] * os);
-          R[u] = fmaf(R[u], upc, adc * kv[k][u]);
+        for (int u = 0; u < 4; u++) {
+          pb[((size_t)c * TC_NV + n0 + u) * (TC_M / 2)] = pack_bf16(R[u][0] * os, R[u][1] * os);
+          R[u][0] = fmaf(R[u][0], upc, adc * __uint_as_float(kv[k][u] << 16));
+          R[u][1] = fmaf(R[u][1], upc, adc * __uint_as_float(kv[k][u] & 0xffff0000u));
         }
       }
     }
@@ -502,7 +502,7 @@ int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, c
                  const int* flags, void* Y, WsAlloc* ws) {
   const int B = dm->B, H = dm->H, BH = B * H, L = dm->Lq;
   const int nch = (L + TILE - 1) / TILE, Lpad = nch * TILE;
-  float* state = ws->take<float>((size_t)BH * nch * TC_M * TC_NV);
+  __nv_bfloat16* state = ws->take<__nv_bfloat16>((size_t)BH * nch * TC_M * TC_NV);     // chunk states, bf16
   float* shifts = ws->take<float>((size_t)BH * nch * 2);
   int* pmax = ws->take<int>((size_t)BH * nch * 2);
   float* crow = ws->take<float>((size_t)BH * Lpad);
@@ -535,7 +535,7 @@ int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, c
   // key side: chunk states and bf16 key features
   int kper = 0;
   const int ksplit = split(4, &kper);
-  FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, kper, ksplit, crow, state, shifts, pmax, phik16));
+  FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, kper, ksplit, crow, reinterpret_cast<float*>(state), shifts, pmax, phik16));
   int qper = 0;
   const int qsplit = split(4, &qper);
   FS_CUDA_OK(cudaFuncSetAttribute(tc_featq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FqSmem::TOTAL + 1024));
