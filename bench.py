@@ -369,7 +369,9 @@ def main():
 
 # DRAM bytes per launch (read + write) from the ncu captures summarised under profiles/ (same kernels, same workload);
 # an entry is dropped when its kernel changes.
-NCU_TRAFFIC = {("cfg2", "fit_kernel"): 4.39e6, ("cfg2", "tc_kv_kernel"): 74.9e6, ("cfg2", "tc_out_kernel"): 48.8e6}
+NCU_TRAFFIC = {("cfg2", "fit_kernel"): 4.39e6, ("cfg2", "tc_kv_kernel"): 74.9e6, ("cfg2", "tc_out_kernel"): 48.8e6,
+               ("cfg3", "tc_kv_kernel"): 412.4e6, ("cfg3", "tc_causal_out_kernel"): 625.5e6,
+               ("cfg3", "tc_featq_kernel"): 195.5e6, ("cfg3", "tc_causal_prefix_kernel"): 178.2e6}
 
 
 def roofline_for(name, k, w, work, peaks):
@@ -391,7 +393,7 @@ def roofline_for(name, k, w, work, peaks):
     bytes_of = {"stats_kernel": 2 * L * d * es * units, "tc_stats_kernel": 2 * L * d * es * units, "expshift_kernel": 2 * L * M * 4 * units,
                 "rowterm_kernel": L * d * es * units, "groupmax_kernel": L * M * 4 * units,
                 "tc_rowterm_kernel": L * d * es * units,
-                "tc_causal_prefix_kernel": ((L + 127) // 128) * (65 * M * 4 + 80 * M * 2) * units}
+                "tc_causal_prefix_kernel": ((L + 127) // 128) * (65 * M * 2 + 80 * M * 2) * units}
     if name in flops_of and flops_of[name]:
         fl = flops_of[name] * (per_launch if name in ("logits_kernel", "kv_kernel", "out_kernel", "scores_kernel") and
                                k["launches_per_step"] > 1 else 1.0)
