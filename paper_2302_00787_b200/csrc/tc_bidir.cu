@@ -339,6 +339,9 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       }
       // the previous tile's contraction has read the phi half tile and updated the accumulator
       if (it > 0 && !mbar_wait(&misc->phi_free[hf], (it - 1) & 1, abortp, status, false)) { alive = false; break; }
+      // causal use: the previous tile's state leaves now (numbered by its tile index, with its own shift s), not at
+      // the end of its own iteration, where the epilogue would have had to sit out the contraction
+      if (per_tile && it > 0) write_partial((size_t)bh * total_tiles + tile0 + it - 1);
       if (it == 0 || per_tile) {
         s = tm;                      // first tile (causal use: every tile): the shift is the exact maximum
       } else if (tm - s > SHIFT_HEADROOM_LOG2) {
@@ -376,14 +379,11 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       mbar_arrive_warp(&misc->phi_full[hf], lane);
       mbar_arrive_warp(&misc->turn[hf ^ 1], lane);
       cj = cnext;
-      if (per_tile) {                // causal use: the tile's state leaves now, numbered by its tile index
-        if (!mbar_wait(&misc->phi_free[hf], it & 1, abortp, status, false)) { alive = false; break; }
-        write_partial((size_t)bh * total_tiles + tile0 + it);
-      }
     }
-    // write this split's partial [V | 1]^T phi_h (fp32, rows 0..79), its shift and its largest magnitude
-    if (alive && ntiles > 0 && !per_tile && mbar_wait(&misc->phi_free[hf], (ntiles - 1) & 1, abortp, status, false))
-      write_partial((size_t)bh * nsplit + split);
+    // write this split's partial phi_h^T [V | 1] (rows 0..64 of the state), its shift and its largest magnitude
+    // (causal use: the last tile's state)
+    if (alive && ntiles > 0 && mbar_wait(&misc->phi_free[hf], (ntiles - 1) & 1, abortp, status, false))
+      write_partial(per_tile ? (size_t)bh * total_tiles + tile0 + ntiles - 1 : (size_t)bh * nsplit + split);
   }
   tcgen05_fence_before();
   __syncthreads();
