@@ -95,11 +95,11 @@ tc_rowterm_kernel(const __grid_constant__ CUtensorMap tmK, const uint8_t* __rest
         if (!mbar_wait(&misc->t_free[buf], ((it >> 1) & 1) ^ 1, abortp, status)) break;
         tcgen05_fence_after();
         const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
-#pragma unroll 1
+#pragma unroll
         for (int k = 0; k < TC_D / 16; k++)
           mma_bf16(tmem + buf * TC_D, desc_advance(dX, 32 * k), desc_advance(dChi, 32 * k), ID_T, k > 0);
         if (clo) {
-#pragma unroll 1
+#pragma unroll
           for (int k = 0; k < TC_D / 16; k++)
             mma_bf16(tmem + buf * TC_D, desc_advance(dX, 32 * k), desc_advance(dClo, 32 * k), ID_T, 1);
         }

@@ -97,7 +97,9 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // A = [X | E]: block 0 the tile, block 1 the constant tile (leading offset = their distance)
         const uint64_t dA = smem_desc(sX, sOnes - sX, 1024, SWZ_128B);
         const uint64_t dB = smem_desc(sX, TILE_BYTES, 1024, SWZ_128B);
-#pragma unroll 1
+        // unrolled: a step's descriptors are the tile's plus a constant; issued from a rolled loop (index
+        // arithmetic on the dependent chain) an MMA costs its thread noticeably longer
+#pragma unroll
         for (int k = 0; k < TILE / 16; k++)
           mma_bf16(tmem + buf * TC_D, desc_advance(dA, k * 2048), desc_advance(dB, k * 2048), ID, (k > 0 || sub > 0) ? 1 : 0);
         if (sub == ST_FOLD - 1 || it == ntiles - 1) mma_commit(&misc->acc_full[buf]);
