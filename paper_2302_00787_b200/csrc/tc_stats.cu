@@ -16,7 +16,7 @@ using namespace tcl;
 
 namespace {
 
-constexpr int ST_STAGES = 8;                 // ring of token tiles in flight
+constexpr int ST_STAGES = 4;                 // ring of token tiles in flight (two blocks share an SM: eight tiles per SM)
 constexpr int ST_FOLD = 2;                   // tiles summed in one fp32 accumulator before it is folded into fp64
 constexpr int ST_EPI_WARPS = 3;              // rows 0..95 of D; only 0..64 carry data
 constexpr int ST_WARP_TMA = 3, ST_WARP_MMA = 4, ST_THREADS = 160;
@@ -32,7 +32,7 @@ struct StMisc {
 };
 static_assert(sizeof(StMisc) <= 256, "misc block");
 
-__global__ void __launch_bounds__(ST_THREADS, 1)
+__global__ void __launch_bounds__(ST_THREADS, 2)
 tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, int H, int Lq, int Lk,
                 int pool, int Bpool, double qk_scale, int tiles_per_split, double* __restrict__ stats,
                 int* __restrict__ status) {
@@ -186,13 +186,14 @@ int fs_tc_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dims
   const int B = dm->B, H = dm->H, BH = B * H;
   const int Lmax = dm->Lq > dm->Lk ? dm->Lq : dm->Lk;
   const int tiles = (Lmax + TILE - 1) / TILE;
-  // one block per SM: the split of the token range with the fewest (waves x tiles per block)
+  // two blocks per SM (each block has one MMA-issuing thread, and issuing is what bounds a block): the split of
+  // the token range with the fewest (waves x tiles per block)
   int best = 1, best_cost = 0x7fffffff, tps = tiles;
   for (int ns = 1; ns <= tiles; ns++) {
     const int t = (tiles + ns - 1) / ns;
     if ((tiles + t - 1) / t != ns) continue;
     const long long blocks = 2LL * BH * ns;
-    const int waves = (int)((blocks + ctx->sm_count - 1) / ctx->sm_count);
+    const int waves = (int)((blocks + 2 * ctx->sm_count - 1) / (2 * ctx->sm_count));
     const int cost = waves * (t + 6);        // fill, drain and the final atomics cost about six tiles
     if (cost < best_cost) { best_cost = cost; best = ns; tps = t; }
   }
