@@ -163,9 +163,18 @@ int fs_tc_rowterm(fsharp_ctx* ctx, const void* K, const fsharp_dims* dm, const u
   CUtensorMap tmK;
   FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, Lk, dm->d), B, H, Lk, dm->d));
   FS_CUDA_OK(cudaFuncSetAttribute(tc_rowterm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RtSmem::TOTAL + 1024));
+  // The output is indexed by token, so this kernel need not follow the key-side kernel's split: two of its blocks fit
+  // an SM, and a block is bound by its single MMA-issuing thread, so it takes about two blocks per SM.
+  (void)tiles_per_split;
+  (void)nsplit;
+  const int total = (Lk + TILE - 1) / TILE;
+  int ns = (2 * ctx->sm_count) / (B * H);
+  ns = ns < 1 ? 1 : (ns > total ? total : ns);
+  const int tps = (total + ns - 1) / ns;
+  ns = (total + tps - 1) / tps;
   FS_TIME_BEGIN(ctx, FS_K_TC_ROWTERM);
-  tc_rowterm_kernel<<<dim3(nsplit, B * H), RT_THREADS, RtSmem::TOTAL + 1024, ctx->stream>>>(
-      tmK, images, flags, H, dm->pool, Lk, Lpad, tiles_per_split, crow, ctx->d_status);
+  tc_rowterm_kernel<<<dim3(ns, B * H), RT_THREADS, RtSmem::TOTAL + 1024, ctx->stream>>>(
+      tmK, images, flags, H, dm->pool, Lk, Lpad, tps, crow, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;
