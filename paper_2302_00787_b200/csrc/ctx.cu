@@ -157,16 +157,11 @@ const char* fsharp_kernel_name(int id) {
     case FS_K_PAIRS: return "pairs_kernel";
     case FS_K_PAIRVAR_PREP: return "pairvar_prep_kernel";
     case FS_K_PAIRVAR: return "pairvar_kernel";
-    case FS_K_TC_PREP: return "tc_prep_kernel";
     case FS_K_TC_KV: return "tc_kv_kernel";
-    case FS_K_TC_MERGE: return "tc_merge_kernel";
     case FS_K_TC_OUT: return "tc_out_kernel";
-    case FS_K_TC_CAUSAL_STATE: return "tc_causal_state_kernel";
-    case FS_K_TC_CAUSAL_PREFIX: return "tc_causal_prefix_kernel";
-    case FS_K_TC_CAUSAL_OUT: return "tc_causal_out_kernel";
+    case FS_K_TC_CAUSAL: return "tc_causal_kernel";
     case FS_K_TC_STATS: return "tc_stats_kernel";
     case FS_K_TC_ROWTERM: return "tc_rowterm_kernel";
-    case FS_K_TC_FEATQ: return "tc_featq_kernel";
     default: return "";
   }
 }

@@ -1,6 +1,8 @@
 // Per-group precomputation for the feature kernels (Section 4, cost paragraph):
 // W^(k) = Omega B^(k) (row m = (B^(k)T w_m)^T), a_m = w_m^T A w_m, the constant
 // log D - 1/2 log M.
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 #include "tc_common.cuh"
 #include "tc_layout.cuh"
@@ -125,6 +127,7 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
               *reinterpret_cast<__nv_bfloat162*>(img + tcl::IMG_W + off) = __nv_bfloat162(h0, h1);
               *reinterpret_cast<__nv_bfloat162*>(img + tcl::IMG_WLO + off) =
                   __nv_bfloat162(__float2bfloat16_rn(v0 - __bfloat162float(h0)), __float2bfloat16_rn(v1 - __bfloat162float(h1)));
+              *reinterpret_cast<__half2*>(img + tcl::IMG_WH + off) = __floats2half2_rn(v0, v1);
             }
           }
         }

@@ -41,8 +41,8 @@ constexpr int PREFETCH_TILES = 4;   // tiles pulled into L2 ahead of the shared-
 // tensor pipe instead of 128, and every epilogue thread (= one feature) takes part when the state leaves.
 struct KvSmem {
   static constexpr uint32_t X0 = 0, V0 = 2 * TILE_BYTES, ONES = 4 * TILE_BYTES, W = ONES + TILE_BYTES,
-                            WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES, FA2 = PHI + 4 * TILE_BYTES,
-                            MISC = FA2 + TC_M * 4, TOTAL = MISC + 256;
+                            WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES, MISC = PHI + 4 * TILE_BYTES,
+                            TOTAL = MISC + 256;
 };
 static_assert(KvSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 static_assert(KvSmem::PHI % 1024 == 0 && KvSmem::W % 1024 == 0 && KvSmem::ONES % 1024 == 0, "swizzled tiles need 1024-byte alignment");
@@ -58,7 +58,6 @@ struct KvMisc {
   uint32_t tmem_base;
   int abort_flag;
   int tile_max[2][4];     // per half: [0..2] rotating slots of the per-tile maximum
-  int chunk_max[3];       // causal use: rotating slots of the exact maximum of a whole tile
 };
 static_assert(sizeof(KvMisc) <= 256, "misc block");
 
@@ -67,18 +66,12 @@ constexpr int HALF_THREADS = EPI_THREADS / 2;
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-             const __grid_constant__ CUtensorMap tmPhi,
              const uint8_t* __restrict__ images, const float* __restrict__ crow, int H, int pool, int L, int Lpad,
              int tiles_per_split, int nsplit, float* __restrict__ partial, float* __restrict__ shifts,
-             int* __restrict__ pmax, int per_tile, int* __restrict__ status) {
-  // per_tile != 0 (causal use: every 128-key tile is a chunk with a state, a shift and a partial of its
-  // own, numbered by its tile index): the key side's share a2 / 2 of the per-feature term is added to the
-  // logits (the in-chunk scores cannot take it from a merged state), the two feature halves share one
-  // shift, and the tile of features, as the MMA reads it, is also stored through tmPhi, bf16 [B*H][Lpad][256].
+             int* __restrict__ pmax, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   KvMisc* misc = reinterpret_cast<KvMisc*>(sm + KvSmem::MISC);
-  float* fa2 = reinterpret_cast<float*>(sm + KvSmem::FA2);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
   const int g = pool == FSHARP_POOL_PER_BH ? bh : h;
@@ -99,7 +92,6 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       mbar_init(&misc->turn[i], HALF_THREADS / 32);
       for (int j = 0; j < 4; j++) misc->tile_max[i][j] = f2ord(-INFINITY);
     }
-    for (int j = 0; j < 3; j++) misc->chunk_max[j] = f2ord(-INFINITY);
     mbar_init(&misc->logits_full, 1);
     mbar_init(&misc->logits_free, EPI_THREADS / 32);
     mbar_init(&misc->const_bar, 1);
@@ -109,7 +101,6 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   // constant tile written by the block itself: the second 64-row block of [V | 1]^T, whose
   // first row is the 1 and whose other rows are zero
   for (int i = threadIdx.x; i < TILE_BYTES / 16; i += TC_THREADS) reinterpret_cast<uint4*>(sm + KvSmem::ONES)[i] = make_uint4(0, 0, 0, 0);
-  if (per_tile && threadIdx.x < TC_M) fa2[threadIdx.x] = 0.5f * reinterpret_cast<const float*>(img + IMG_A2)[threadIdx.x];
   __syncthreads();
   if (threadIdx.x < TILE)
     *reinterpret_cast<__nv_bfloat16*>(sm + KvSmem::ONES + sw128_offset(threadIdx.x, 0)) = __float2bfloat16(1.f);
@@ -219,23 +210,16 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         const int st = it & 1;
         if (!mbar_wait(&misc->fullV[st], (it >> 1) & 1, abortp, status)) break;
         const uint64_t dV = st ? dVst1 : dVst0;
-        const uint32_t acc0 = (it > 0 && !per_tile) ? 1u : 0u;      // causal use: every tile starts afresh
+        const uint32_t acc0 = it > 0 ? 1u : 0u;
         if (!mbar_wait(&misc->phi_full[hh], it & 1, abortp, status)) break;
         tcgen05_fence_after();
-        if (per_tile) {                 // the half tile also goes out as it is (two 64-feature blocks)
-          tma_store_3d(&tmPhi, sm + KvSmem::PHI + (2 * hh) * TILE_BYTES, (2 * hh) * 64, (tile0 + it) * TILE, bh);
-          tma_store_3d(&tmPhi, sm + KvSmem::PHI + (2 * hh + 1) * TILE_BYTES, (2 * hh + 1) * 64, (tile0 + it) * TILE, bh);
-          bulk_commit();
-        }
 #pragma unroll
         for (int k = 0; k < TILE / 16; k++)
           mma_bf16(tmem + KV_COL_ACC + hh * TC_NV, desc_advance(dPhi, k * 2048), desc_advance(dV, k * 2048), ID_KV,
                    k > 0 ? 1u : acc0);
-        if (per_tile) bulk_wait_read0();         // the store has read the half tile: it may be overwritten
         mma_commit(&misc->phi_free[hh]);
         mma_commit(&misc->emptyV[st]);           // the value tile is free once both halves' contractions have completed
       }
-      if (per_tile) bulk_wait0();
     }
   }
   } else {
@@ -260,10 +244,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       tcgen05_fence_after();
       // thread = feature m: its row of the accumulator is column m of the state [80][256]; a store instruction of
       // the warp covers 32 consecutive features of one state row (128 contiguous bytes).  Rows 65..79 are not written.
-      // Causal use: a chunk's state is only ever read back as a term of a prefix that is itself rounded to bf16,
-      // so it is stored as bf16 (half the bytes of the kernel's largest output).
       float* out = partial + slot * TC_NV * TC_M + hf * 128 + row;
-      __nv_bfloat16* out16 = reinterpret_cast<__nv_bfloat16*>(partial) + slot * TC_NV * TC_M + hf * 128 + row;
       float amax = 0.f;
 #pragma unroll
       for (int c = 0; c < 5; c++) {
@@ -274,8 +255,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         for (int j = 0; j < 16; j++) {
           if (c * 16 + j <= TC_DV) {
             amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
-            if (per_tile) out16[(size_t)(c * 16 + j) * TC_M] = __float2bfloat16_rn(__uint_as_float(a[j]));
-            else out[(size_t)(c * 16 + j) * TC_M] = __uint_as_float(a[j]);
+            out[(size_t)(c * 16 + j) * TC_M] = __uint_as_float(a[j]);
           }
         }
       }
@@ -302,18 +282,8 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       tmem_wait_ld();
       tcgen05_fence_before();
       mbar_arrive_warp(&misc->logits_free, lane);
-      if (per_tile) {
-#pragma unroll
-        for (int i = 0; i < 128; i += 4) {
-          const float4 a4 = *reinterpret_cast<const float4*>(fa2 + hf * 128 + i);
-          v[i] = __float_as_uint(__uint_as_float(v[i]) + a4.x);
-          v[i + 1] = __float_as_uint(__uint_as_float(v[i + 1]) + a4.y);
-          v[i + 2] = __float_as_uint(__uint_as_float(v[i + 2]) + a4.z);
-          v[i + 3] = __float_as_uint(__uint_as_float(v[i + 3]) + a4.w);
-        }
-      }
       const bool valid = (tile0 + it) * TILE + row < L;
-      // Exact maximum of this half of the tile (causal use: of the whole tile), taken BEFORE the exponentials:
+      // Exact maximum of this half of the tile, taken BEFORE the exponentials:
       // it overlaps the contraction of the previous tile, and nothing stands between the last exponential and
       // the arrival that starts this tile's contraction.
       float tm;
@@ -325,25 +295,15 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         float mx = valid ? hm + cj : -INFINITY;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        if (per_tile) {              // one shift for both halves
-          if (lane == 0) atomicMax(&misc->chunk_max[it % 3], f2ord(mx));
-          if (threadIdx.x == 0) misc->chunk_max[(it + 1) % 3] = f2ord(-INFINITY);   // next tile's slot; idle since tile it-2
-          named_bar_sync(3, EPI_THREADS);
-          tm = ord2f(misc->chunk_max[it % 3]);
-        } else {
-          if (lane == 0) atomicMax(&tmax[it % 3], f2ord(mx));
-          if (q == 0 && lane == 0) tmax[(it + 1) % 3] = f2ord(-INFINITY);           // next tile's slot; idle since tile it-2
-          named_bar_sync(1 + hf, HALF_THREADS);
-          tm = ord2f(tmax[it % 3]);
-        }
+        if (lane == 0) atomicMax(&tmax[it % 3], f2ord(mx));
+        if (q == 0 && lane == 0) tmax[(it + 1) % 3] = f2ord(-INFINITY);           // next tile's slot; idle since tile it-2
+        named_bar_sync(1 + hf, HALF_THREADS);
+        tm = ord2f(tmax[it % 3]);
       }
       // the previous tile's contraction has read the phi half tile and updated the accumulator
       if (it > 0 && !mbar_wait(&misc->phi_free[hf], (it - 1) & 1, abortp, status, false)) { alive = false; break; }
-      // causal use: the previous tile's state leaves now (numbered by its tile index, with its own shift s), not at
-      // the end of its own iteration, where the epilogue would have had to sit out the contraction
-      if (per_tile && it > 0) write_partial((size_t)bh * total_tiles + tile0 + it - 1);
-      if (it == 0 || per_tile) {
-        s = tm;                      // first tile (causal use: every tile): the shift is the exact maximum
+      if (it == 0) {
+        s = tm;                      // first tile: the shift is the exact maximum
       } else if (tm - s > SHIFT_HEADROOM_LOG2) {
         // rare (the running maximum grows a handful of times per sequence): the shift moves up to this tile's
         // maximum and the accumulated [V | 1]^T phi_h is brought along
@@ -381,9 +341,8 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       cj = cnext;
     }
     // write this split's partial phi_h^T [V | 1] (rows 0..64 of the state), its shift and its largest magnitude
-    // (causal use: the last tile's state)
     if (alive && ntiles > 0 && mbar_wait(&misc->phi_free[hf], (ntiles - 1) & 1, abortp, status, false))
-      write_partial(per_tile ? (size_t)bh * total_tiles + tile0 + ntiles - 1 : (size_t)bh * nsplit + split);
+      write_partial((size_t)bh * nsplit + split);
   }
   tcgen05_fence_before();
   __syncthreads();
@@ -723,8 +682,6 @@ int pick_split(int units, int tiles, int sms, int max_split, int* tiles_per_spli
 // ------------------------------------------------------------------------------------------
 namespace tchost {
 int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int H, int L, int inner);
-int make_map_kvt(CUtensorMap* map, const void* base, int BH, int bf16);
-int make_map_feat(CUtensorMap* map, const void* base, int BH, int Lpad);
 }  // namespace tchost
 int fs_tc_rowterm(fsharp_ctx* ctx, const void* K, const fsharp_dims* dm, const uint8_t* images, const int* flags, int Lpad,
                   int tiles_per_split, int nsplit, float* crow);
@@ -732,9 +689,7 @@ size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
 int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                 const int* flags, void* Y, WsAlloc* ws);
 int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
-                   const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax,
-                   __nv_bfloat16* phik);
-
+                   const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax);
 
 size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
   const size_t BH = (size_t)dm->B * dm->H;
@@ -747,25 +702,20 @@ size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
 
 // Key side: the per-key quadratic term, then the feature / contraction kernel.  crow: [B*H][Lpad] floats,
 // Lpad = ceil(Lk / 128) * 128; partial: [B*H][nsplit][80][256] floats; shifts, pmax: [B*H][nsplit][2], pmax
-// zeroed by the caller.  phik (may be null; causal use): bf16 [B*H][Lpad][256]; with it every 128-key tile
-// is a chunk of its own, shifts and pmax are indexed by tile ([B*H][ceil(Lk / 128)] entries) and partial
-// holds bf16 states [B*H][ceil(Lk / 128)][80][256].
+// zeroed by the caller.  The quadratic term covers every key; the feature / contraction kernel covers the
+// first nsplit * tiles_per_split tiles (the causal path asks for the segments that have a successor only).
 int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
-                   const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax,
-                   __nv_bfloat16* phik) {
+                   const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax) {
   const int B = dm->B, H = dm->H, Lk = dm->Lk;
   const int Lpad = (Lk + TILE - 1) / TILE * TILE;
   FS_TRY(fs_tc_rowterm(ctx, K, dm, images, flags, Lpad, tiles_per_split, nsplit, crow));
-  CUtensorMap tmK, tmV, tmPhi;
+  CUtensorMap tmK, tmV;
   FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, Lk, dm->d), B, H, Lk, dm->d));
   FS_TRY(tchost::make_map_tokens(&tmV, V, fs_addr(dm->v_stride, H, Lk, dm->dv), B, H, Lk, dm->dv));
-  if (phik != nullptr) FS_TRY(tchost::make_map_feat(&tmPhi, phik, B * H, Lpad));
-  else tmPhi = tmK;                       // not used
   FS_CUDA_OK(cudaFuncSetAttribute(tc_kv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KvSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_KV);
   tc_kv_kernel<<<dim3(nsplit, B * H), TC_THREADS, KvSmem::TOTAL + 1024, ctx->stream>>>(
-      tmK, tmV, tmPhi, images, crow, H, dm->pool, Lk, Lpad, tiles_per_split, nsplit, partial, shifts, pmax,
-      phik != nullptr ? 1 : 0, ctx->d_status);
+      tmK, tmV, images, crow, H, dm->pool, Lk, Lpad, tiles_per_split, nsplit, partial, shifts, pmax, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;
@@ -785,7 +735,7 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * MAX_KEY_SPLIT * 2 * sizeof(int), ctx->stream));
   const int Lpad = ktiles * TILE;
   float* crow = ws->take<float>((size_t)BH * Lpad);
-  FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, tps, nsplit, crow, partial, shifts, pmax, nullptr));
+  FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, tps, nsplit, crow, partial, shifts, pmax));
 
   CUtensorMap tmQ;
   FS_TRY(tchost::make_map_tokens(&tmQ, Q, fs_addr(dm->q_stride, H, Lq, dm->d), B, H, Lq, dm->d));

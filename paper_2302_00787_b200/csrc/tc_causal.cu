@@ -1,16 +1,28 @@
 // Tensor-core path, causal attention (Section 2.2's formula with a lower-triangular mask) for
-// bf16, d = dv = 64, M = 256, chunk = 128 tokens:
+// bf16, d = dv = 64, M = 256.  With P = phi(Q), S = phi(K) (Section 2.1) and tiles of 128 tokens,
 //
-//   Y_c = [ phiQ_c P_c  +  tril(phiQ_c phiK_c^T) [V_c | 1] ]  (numerator | denominator),
-//   P_c = sum over earlier chunks c' of phiK_c'^T [V_c' | 1].
+//   [num | den]_c = P_c T_{c-1} + tril(P_c S_c^T) [V_c | 1],      T_c = T_{c-1} + S_c^T [V_c | 1],
 //
-//   tc_kv_kernel (tc_bidir.cu), every tile a chunk: chunk states and the chunk's bf16 key features
-//   tc_featq_kernel:          bf16 query features, each row shifted by its own maximum
-//   tc_causal_prefix_kernel:  exclusive scan of the chunk states -> bf16 prefixes P_c, every
-//                             chunk brought to a scale of its own that also weighs the in-chunk term
-//   tc_causal_out_kernel:     per chunk  D = phiQ P_c^T, S = phiQ phiK^T (TMEM),
-//                             S masked, scaled, rounded to bf16 into shared memory,
-//                             D += S V, denominator += row sums of S, Y = num / den
+// evaluated by ONE kernel per segment of consecutive tiles: the features of a tile are computed in the
+// kernel and never leave the SM, and the state T is carried from tile to tile in tensor memory.
+//
+//   tc_kv_kernel (tc_bidir.cu)  totals S^T [V | 1] of the segments that have a successor (fp32 partials)
+//   tc_causal_kernel            one block per (segment, batch, head): starts from the sum of the earlier
+//                               segments' totals and walks its tiles
+//
+// Per tile (tensor memory columns in brackets):
+//   logits of the keys, then of the queries, 128 features at a time  X Wh^T         [L: 128 columns]
+//   phi(K) -> bf16 tile in shared memory (the B operand of the scores, the A operand of the state update)
+//   phi(Q) -> bf16, written back over its own logits [L] and read from there as the A operand
+//   [scores | inter-tile output] = phi(Q) [phi(K)^T | bf16(T)]      one MMA stream, N = 208   [S: 128][O: 80]
+//   scores masked (key <= query), rounded to bf16 over their own columns, row sums kept
+//   O[:, :64] += masked scores (from tensor memory) V                                         [O]
+//   T += phi(K)^T [V | 1], 128 features per accumulator                                       [T: 2 x 80]
+//   bf16(T) for the next tile: the accumulators are read back and written to shared memory
+// The token tiles are converted from bf16 to fp16 in shared memory (exact for |x| in [2^-14, 65504]), so the
+// logits need one fp16 image of W (11 significant bits) instead of a bf16 value and its remainder.
+// The keys of a segment share one running shift (raised, with the state rescaled, when a tile's largest
+// exponent exceeds it by the headroom); it cancels between numerator and denominator.
 #include <cuda_fp16.h>
 
 #include "common.cuh"
@@ -22,51 +34,98 @@ using namespace tcl;
 
 namespace {
 
-// ------------------------------------------------------------------------------------------
-// query features
-// ------------------------------------------------------------------------------------------
-constexpr int FQ_STAGES = 3;
-// The feature tile leaves as four 64-feature blocks (16 KB each, one bulk store each) from a ring of six block
-// slots: block j of tile t sits in slot (4 t + j) % 6, so a tile only reuses slots whose stores were issued at least
-// one and a half tiles earlier and the stores of a tile's last two blocks may still be reading when the next is written.
-constexpr int FQ_PHI_SLOTS = 6;
-struct FqSmem {
-  static constexpr uint32_t X0 = 0, W = FQ_STAGES * TILE_BYTES, WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES,
-                            ROWMAX = PHI + FQ_PHI_SLOTS * TILE_BYTES,
-                            AH = ROWMAX + 2 * 2 * TILE * 4, MISC = AH + TC_M * 4, TOTAL = MISC + 256;
+constexpr int WARP_CVT0 = 10;                 // warps 10 and 11 convert the token tiles to fp16
+constexpr int CVT_THREADS = 64;
+// The MMA-issuing thread of this kernel keeps more descriptors alive than those of the other kernels:
+// 128 x 64 + 256 x 216 registers (of the 384 x 168 the block is launched with).
+constexpr int CF_REGS_PRODUCER = 64, CF_REGS_EPILOGUE = 216;
+
+struct CfSmem {
+  // KP: four blocks of 64 features, each [phi(K) 128 keys x 64 | bf16(T) 80 rows x 64], so that one K-major
+  // operand of 208 rows covers both
+  static constexpr uint32_t W1 = 0, W2 = IMG_W_BYTES, X = 2 * IMG_W_BYTES, V = X + TILE_BYTES, ONES = V + TILE_BYTES,
+                            KP = ONES + TILE_BYTES, BLK = TILE_BYTES + KVT_BLOCK_BYTES, ROWMAX = KP + 4 * BLK,
+                            RSUM = ROWMAX + 2 * TILE * 4, FA2 = RSUM + 2 * TILE * 4, MISC = FA2 + TC_M * 4,
+                            TOTAL = MISC + 256;
 };
-struct FqMisc {
-  uint64_t full[FQ_STAGES], empty[FQ_STAGES], logits_full[2], logits_free[2], const_bar;
+static_assert(CfSmem::KP % 1024 == 0 && CfSmem::BLK % 1024 == 0 && CfSmem::X % 1024 == 0, "swizzled tiles need 1024-byte alignment");
+static_assert(CfSmem::TOTAL + 1024 <= 232448, "shared memory budget");
+
+struct CfMisc {
+  uint64_t const_bar, x_full, x_ready, x_free, v_full, v_free, lg_full, lg_free, phik_full[2], phiq_full[2], p_full,
+      s_ready, sm_full, o_ready, o_free, st_ready;
+  // meeting points of the epilogue warps (the two warps of a row quarter; all eight): mbarriers, so that these
+  // waits are bounded like every other
+  uint64_t pair_bar[4], all_bar;
   uint32_t tmem_base;
   int abort_flag;
+  int chunk_max[3];
+  float red[8];
 };
+static_assert(sizeof(CfMisc) <= 256, "misc block");
+
+// tensor memory columns
+constexpr uint32_t CF_L = 0, CF_S = 128, CF_O = 256, CF_T = 336;
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
-tc_featq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmPhi,
-                const uint8_t* __restrict__ images, int H, int pool, int L, int tiles_per_split, int* __restrict__ status) {
+tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                 const __grid_constant__ CUtensorMap tmV, const uint8_t* __restrict__ images,
+                 const float* __restrict__ crow, const float* __restrict__ partial, const float* __restrict__ shifts,
+                 int nsplit1, int H, int pool, int L, int Lpad, int tiles_per_seg,
+                 __nv_bfloat16* __restrict__ Y, TensorAddr ay, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  FqMisc* misc = reinterpret_cast<FqMisc*>(sm + FqSmem::MISC);
-  float* rowmax = reinterpret_cast<float*>(sm + FqSmem::ROWMAX);   // [tile & 1][half][row]
-  float* ah = reinterpret_cast<float*>(sm + FqSmem::AH);           // the query side's share a2 / 2 of the per-feature term
+  CfMisc* misc = reinterpret_cast<CfMisc*>(sm + CfSmem::MISC);
+  float* rowmax = reinterpret_cast<float*>(sm + CfSmem::ROWMAX);   // [half][row]
+  float* rsum = reinterpret_cast<float*>(sm + CfSmem::RSUM);       // [half][row]: row sums of the rounded masked scores
+  float* fa2 = reinterpret_cast<float*>(sm + CfSmem::FA2);         // each side's share a2 / 2 of the per-feature term
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int bh = blockIdx.y, b = bh / H, h = bh % H;
+  const int seg = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
   const int g = pool == FSHARP_POOL_PER_BH ? bh : h;
   const int total_tiles = (L + TILE - 1) / TILE;
-  const int tile0 = blockIdx.x * tiles_per_split;
-  const int ntiles = min(tiles_per_split, total_tiles - tile0);
+  const int tile0 = seg * tiles_per_seg;
+  const int ntiles = min(tiles_per_seg, total_tiles - tile0);
   if (ntiles <= 0) return;                    // uniform over the block, before anything is allocated
-  const uint8_t* img = images + ((size_t)g * 2 + 0) * IMG_BYTES;        // side 1 (queries)
+  const uint8_t* img1 = images + ((size_t)g * 2 + 0) * IMG_BYTES;        // side 1 (queries)
+  const uint8_t* img2 = images + ((size_t)g * 2 + 1) * IMG_BYTES;        // side 2 (keys)
   volatile int* abortp = &misc->abort_flag;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < FQ_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], 1); }
-    for (int i = 0; i < 2; i++) { mbar_init(&misc->logits_full[i], 1); mbar_init(&misc->logits_free[i], EPI_THREADS / 32); }
     mbar_init(&misc->const_bar, 1);
+    mbar_init(&misc->x_full, 1);
+    mbar_init(&misc->x_ready, CVT_THREADS / 32);
+    mbar_init(&misc->x_free, 1);
+    mbar_init(&misc->v_full, 1);
+    mbar_init(&misc->v_free, 1);
+    mbar_init(&misc->lg_full, 1);
+    mbar_init(&misc->lg_free, EPI_THREADS / 32);
+    for (int i = 0; i < 2; i++) {
+      mbar_init(&misc->phik_full[i], EPI_THREADS / 32);
+      mbar_init(&misc->phiq_full[i], EPI_THREADS / 32);
+    }
+    mbar_init(&misc->p_full, EPI_THREADS / 32);
+    mbar_init(&misc->s_ready, 1);
+    mbar_init(&misc->sm_full, EPI_THREADS / 32);
+    mbar_init(&misc->o_ready, 1);
+    mbar_init(&misc->o_free, EPI_THREADS / 32);
+    mbar_init(&misc->st_ready, 1);
+    for (int i = 0; i < 4; i++) mbar_init(&misc->pair_bar[i], 2);
+    mbar_init(&misc->all_bar, EPI_THREADS / 32);
+    for (int j = 0; j < 3; j++) misc->chunk_max[j] = f2ord(-INFINITY);
     misc->abort_flag = 0;
     fence_barrier_init();
   }
-  if (threadIdx.x < TC_M) ah[threadIdx.x] = 0.5f * reinterpret_cast<const float*>(img + IMG_A2)[threadIdx.x];
+  // constants written by the block itself: the second 64-column block of [V | 1] (a one in its first column) and
+  // the zero rows 65..79 of bf16(T) (rows 0..64 are rewritten for every tile)
+  for (int i = threadIdx.x; i < (int)(TILE_BYTES / 16); i += TC_THREADS) reinterpret_cast<uint4*>(sm + CfSmem::ONES)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = threadIdx.x; i < 4 * (int)(KVT_BLOCK_BYTES / 16); i += TC_THREADS)
+    reinterpret_cast<uint4*>(sm + CfSmem::KP + (i / (KVT_BLOCK_BYTES / 16)) * CfSmem::BLK + TILE_BYTES)[i % (KVT_BLOCK_BYTES / 16)] =
+        make_uint4(0, 0, 0, 0);
+  if (threadIdx.x < TC_M) fa2[threadIdx.x] = 0.5f * reinterpret_cast<const float*>(img2 + IMG_A2)[threadIdx.x];
+  __syncthreads();
+  if (threadIdx.x < TILE)
+    *reinterpret_cast<__nv_bfloat16*>(sm + CfSmem::ONES + sw128_offset(threadIdx.x, 0)) = __float2bfloat16(1.f);
+  fence_proxy_async_smem();
   if (warp == WARP_MMA) {
     tmem_alloc(&misc->tmem_base, TMEM_COLS);
     tmem_relinquish();
@@ -77,366 +136,244 @@ tc_featq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const uint32_t tmem = misc->tmem_base;
 
   if (warp >= WARP_TMA) {
-    regs_release<REGS_PRODUCER>();
+    regs_release<CF_REGS_PRODUCER>();
     if (warp == WARP_TMA) {
       if (lane == 0) {
         prefetch_tmap(&tmQ);
+        prefetch_tmap(&tmK);
+        prefetch_tmap(&tmV);
         mbar_expect_tx(&misc->const_bar, 2 * IMG_W_BYTES);
-        bulk_load(sm + FqSmem::W, img + IMG_W, IMG_W_BYTES, &misc->const_bar);
-        bulk_load(sm + FqSmem::WLO, img + IMG_WLO, IMG_W_BYTES, &misc->const_bar);
-        int issued = 0;
-        for (int it = 0; it < ntiles; it++) {
-          const int st = it % FQ_STAGES;
-          if (!mbar_wait(&misc->empty[st], ((it / FQ_STAGES) & 1) ^ 1, abortp, status)) break;
-          mbar_expect_tx(&misc->full[st], TILE_BYTES);
-          tma_load_4d(sm + FqSmem::X0 + st * TILE_BYTES, &tmQ, &misc->full[st], 0, (tile0 + it) * TILE, h, b);
-          issued = it + 1;
+        bulk_load(sm + CfSmem::W1, img1 + IMG_WH, IMG_W_BYTES, &misc->const_bar);
+        bulk_load(sm + CfSmem::W2, img2 + IMG_WH, IMG_W_BYTES, &misc->const_bar);
+        // One token tile in shared memory serves keys and queries in turn: load 2 it is the key tile of tile it
+        // (free once the second half of the key logits has been computed), load 2 it + 1 its query tile.
+        int nx = 0, nv = 0;
+        bool okp = true;
+        for (int it = 0; it < ntiles && okp; it++) {
+          const int tok = (tile0 + it) * TILE;
+          if (nx > 0 && !mbar_wait(&misc->x_free, (nx - 1) & 1, abortp, status)) { okp = false; break; }
+          mbar_expect_tx(&misc->x_full, TILE_BYTES);
+          tma_load_4d(sm + CfSmem::X, &tmK, &misc->x_full, 0, tok, h, b);
+          nx++;
+          if (it + 1 < ntiles) {             // the next tile's operands: into L2 while this one is worked on
+            tma_prefetch_4d(&tmK, 0, tok + TILE, h, b);
+            tma_prefetch_4d(&tmQ, 0, tok + TILE, h, b);
+            tma_prefetch_4d(&tmV, 0, tok + TILE, h, b);
+          }
+          if (nv > 0 && !mbar_wait(&misc->v_free, (nv - 1) & 1, abortp, status)) { okp = false; break; }
+          mbar_expect_tx(&misc->v_full, TILE_BYTES);
+          tma_load_4d(sm + CfSmem::V, &tmV, &misc->v_full, 0, tok, h, b);
+          nv++;
+          if (!mbar_wait(&misc->x_free, (nx - 1) & 1, abortp, status)) { okp = false; break; }
+          mbar_expect_tx(&misc->x_full, TILE_BYTES);
+          tma_load_4d(sm + CfSmem::X, &tmQ, &misc->x_full, 0, tok, h, b);
+          nx++;
         }
         // no copy of this block may still be in flight when it exits
         mbar_wait(&misc->const_bar, 0, abortp, status, false);
-        for (int it = max(0, issued - FQ_STAGES); it < issued; it++)
-          mbar_wait(&misc->full[it % FQ_STAGES], (it / FQ_STAGES) & 1, abortp, status, false);
+        if (nx > 0) mbar_wait(&misc->x_full, (nx - 1) & 1, abortp, status, false);
+        if (nv > 0) mbar_wait(&misc->v_full, (nv - 1) & 1, abortp, status, false);
       }
     } else if (warp == WARP_MMA) {
       if (lane == 0) {
-        constexpr uint32_t ID_LOGITS = idesc_bf16(128, TC_M, 0, 0);
-        const uint64_t dX0 = smem_desc(smem_u32(sm + FqSmem::X0), 16, 1024, SWZ_128B);
-        const uint64_t dW = smem_desc(smem_u32(sm + FqSmem::W), 16, 1024, SWZ_128B);
-        const uint64_t dWlo = smem_desc(smem_u32(sm + FqSmem::WLO), 16, 1024, SWZ_128B);
+        constexpr uint32_t ID_LOGITS = idesc_f16(128, 128, 0, 0);            // X Wh^T, 128 features
+        constexpr uint32_t ID_STATE = idesc_bf16(128, TC_NV, 1, 1);          // phi(K)_h^T [V | 1]
+        constexpr uint32_t ID_SO = idesc_bf16(128, 128 + TC_NV, 0, 0);       // phi(Q) [phi(K)^T | bf16(T)]
+        constexpr uint32_t ID_SV = idesc_bf16(128, TC_DV, 0, 1);             // masked scores x V
+        const uint64_t dX = smem_desc(smem_u32(sm + CfSmem::X), 16, 1024, SWZ_128B);
+        const uint64_t dW1 = smem_desc(smem_u32(sm + CfSmem::W1), 16, 1024, SWZ_128B);
+        const uint64_t dW2 = smem_desc(smem_u32(sm + CfSmem::W2), 16, 1024, SWZ_128B);
+        const uint32_t sV = smem_u32(sm + CfSmem::V), sOnes = smem_u32(sm + CfSmem::ONES);
+        const uint64_t dKP = smem_desc(smem_u32(sm + CfSmem::KP), 16, 1024, SWZ_128B);             // K-major, 208 rows per block
+        const uint64_t dPhiMN = smem_desc(smem_u32(sm + CfSmem::KP), CfSmem::BLK, 1024, SWZ_128B); // features contiguous
+        const uint64_t dV1 = smem_desc(sV, sOnes - sV, 1024, SWZ_128B);                            // [V | 1], value index contiguous
+        auto issue_logits = [&](uint64_t dW, int half) {
+#pragma unroll
+          for (int k = 0; k < TC_D / 16; k++)
+            mma_bf16(tmem + CF_L, desc_advance(dX, 32 * k), desc_advance(dW, half * (IMG_W_BYTES / 2) + 32 * k), ID_LOGITS, k > 0);
+          mma_commit(&misc->lg_full);
+        };
+        int nlg = 0, nxr = 0;                 // logits halves handed over so far, token tiles consumed so far
         bool ok = mbar_wait(&misc->const_bar, 0, abortp, status);
+        if (ok) ok = mbar_wait(&misc->x_ready, nxr & 1, abortp, status);
+        if (ok) {
+          tcgen05_fence_after();
+          issue_logits(dW2, 0);
+        }
         for (int it = 0; ok && it < ntiles; it++) {
-          const int st = it % FQ_STAGES, buf = it & 1;
-          if (!mbar_wait(&misc->full[st], (it / FQ_STAGES) & 1, abortp, status)) break;
-          if (!mbar_wait(&misc->logits_free[buf], ((it >> 1) & 1) ^ 1, abortp, status)) break;
+          // second half of the key logits once the epilogue has taken the first out of tensor memory
+          if (!mbar_wait(&misc->lg_free, nlg & 1, abortp, status)) break;
+          nlg++;
           tcgen05_fence_after();
-          const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
+          issue_logits(dW2, 1);
+          mma_commit(&misc->x_free);
+          nxr++;
+          // query logits
+          if (!mbar_wait(&misc->lg_free, nlg & 1, abortp, status)) break;
+          nlg++;
+          if (!mbar_wait(&misc->x_ready, nxr & 1, abortp, status)) break;
+          tcgen05_fence_after();
+          issue_logits(dW1, 0);
+          if (!mbar_wait(&misc->lg_free, nlg & 1, abortp, status)) break;
+          nlg++;
+          tcgen05_fence_after();
+          issue_logits(dW1, 1);
+          mma_commit(&misc->x_free);
+          nxr++;
+          // state update T_h += phi(K)_h^T [V | 1] (both feature halves were written before the query logits left)
+          if (!mbar_wait(&misc->v_full, it & 1, abortp, status)) break;
+          if (!mbar_wait(&misc->phik_full[0], it & 1, abortp, status)) break;
+          if (!mbar_wait(&misc->phik_full[1], it & 1, abortp, status)) break;
+          tcgen05_fence_after();
+#pragma unroll 1
+          for (int hh = 0; hh < 2; hh++) {
 #pragma unroll
-          for (int k = 0; k < TC_D / 16; k++)
-            mma_bf16(tmem + buf * TC_M, desc_advance(dX, 32 * k), desc_advance(dW, 32 * k), ID_LOGITS, k > 0);
-#pragma unroll
-          for (int k = 0; k < TC_D / 16; k++)
-            mma_bf16(tmem + buf * TC_M, desc_advance(dX, 32 * k), desc_advance(dWlo, 32 * k), ID_LOGITS, 1);
-          mma_commit(&misc->logits_full[buf]);
-          mma_commit(&misc->empty[st]);
-        }
-      }
-    }
-  } else {
-    regs_acquire<REGS_EPILOGUE>();
-    // one query row per thread, 128 of the 256 features; the two threads of a row agree on the row maximum
-    const int q = warp & 3, hf = warp >> 2;
-    const int row = q * 32 + lane;
-    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
-    for (int it = 0; it < ntiles; it++) {
-      const int buf = it & 1;
-      if (!mbar_wait(&misc->logits_full[buf], (it >> 1) & 1, abortp, status, false)) break;
-      __syncwarp();
-      tcgen05_fence_after();
-      uint32_t v[128];
-#pragma unroll
-      for (int c = 0; c < 8; c++) {
-        uint32_t t[16];
-        tmem_ld16(lane_addr + buf * TC_M + hf * 128 + c * 16, t);
-#pragma unroll
-        for (int j = 0; j < 16; j++) v[c * 16 + j] = t[j];
-      }
-      tmem_wait_ld();
-      tcgen05_fence_before();
-      mbar_arrive_warp(&misc->logits_free[buf], lane);
-      float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-      for (int i = 0; i < 128; i += 4) {
-        const float4 a4 = *reinterpret_cast<const float4*>(ah + hf * 128 + i);
-        v[i] = __float_as_uint(__uint_as_float(v[i]) + a4.x);
-        v[i + 1] = __float_as_uint(__uint_as_float(v[i + 1]) + a4.y);
-        v[i + 2] = __float_as_uint(__uint_as_float(v[i + 2]) + a4.z);
-        v[i + 3] = __float_as_uint(__uint_as_float(v[i + 3]) + a4.w);
-      }
-#pragma unroll
-      for (int i = 0; i < 128; i++) mxp[i & 3] = fmaxf(mxp[i & 3], __uint_as_float(v[i]));
-      float mx = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
-      float* rm = rowmax + buf * 2 * TILE;
-      rm[hf * TILE + row] = mx;
-      if (threadIdx.x == 0 && it > 0) bulk_wait_read2();      // all stores but the previous tile's last two have read their slots
-      named_bar_sync(1, EPI_THREADS);
-      mx = fmaxf(mx, rm[(hf ^ 1) * TILE + row]);
-      // the tile goes to shared memory in the layout of an MMA operand and leaves as one TMA store per
-      // 64-feature block
-      const int slot0 = (4 * it + 2 * hf) % FQ_PHI_SLOTS, slot1 = (4 * it + 2 * hf + 1) % FQ_PHI_SLOTS;
-      uint8_t* prow0 = sm + FqSmem::PHI + slot0 * TILE_BYTES + row * 128;
-      uint8_t* prow1 = sm + FqSmem::PHI + slot1 * TILE_BYTES + row * 128;
-#pragma unroll
-      for (int c = 0; c < 16; c++) {
-        uint32_t p[4];
-#pragma unroll
-        for (int j = 0; j < 4; j++)
-          p[j] = pack_bf16(ex2(__uint_as_float(v[c * 8 + 2 * j]) - mx), ex2(__uint_as_float(v[c * 8 + 2 * j + 1]) - mx));
-        *reinterpret_cast<uint4*>((c < 8 ? prow0 : prow1) + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
-      }
-      fence_proxy_async_smem();
-      named_bar_sync(2, EPI_THREADS);
-      if (threadIdx.x == 0) {
-#pragma unroll
-        for (int fb = 0; fb < TC_M / 64; fb++) {
-          tma_store_3d(&tmPhi, sm + FqSmem::PHI + ((4 * it + fb) % FQ_PHI_SLOTS) * TILE_BYTES, fb * 64, (tile0 + it) * TILE, bh);
-          bulk_commit();
-        }
-      }
-    }
-    if (threadIdx.x == 0) bulk_wait0();
-  }
-  tcgen05_fence_before();
-  __syncthreads();
-  if (warp == WARP_MMA) {
-    tcgen05_fence_after();
-    tmem_dealloc(tmem, TMEM_COLS);
-  }
-}
-
-// ------------------------------------------------------------------------------------------
-// exclusive scan over chunks
-// ------------------------------------------------------------------------------------------
-// state[bh][c]: [80][256] bf16, chunk c's [V | 1]^T phiK with phiK = 2^(exponent - s_c); pmax its largest
-// magnitude.  For every chunk c the kernel writes
-//   prefix[bh][c] = alpha_c 2^(-e_c) sum_{c' < c} 2^(s_c' - sigma_c) state[c']   (bf16),
-//   beta[bh][c],
-// where sigma_c = max_{c' < c} s_c', e_c brings the sum to order 2^14, and (alpha_c, beta_c) <= 1 put the
-// prefix term (true scale 2^(sigma_c + e_c)) and the in-chunk term (true scale 2^(s_c)) on one scale.
-constexpr int PFX_SLICES = 10;               // 80 x 256 elements = 10 x 256 threads x 8
-constexpr int PFX_MAXCH = 1024;
-__global__ void __launch_bounds__(256)
-tc_causal_prefix_kernel(const __nv_bfloat16* __restrict__ state, const float* __restrict__ shifts, const int* __restrict__ pmax,
-                        int nch, __nv_bfloat16* __restrict__ prefix, float* __restrict__ beta) {
-  __shared__ float up[PFX_MAXCH], add[PFX_MAXCH], oscale[PFX_MAXCH];
-  const int bh = blockIdx.y;
-  if (threadIdx.x == 0) {
-    float sigma = -INFINITY, bound = 0.f;
-    for (int c = 0; c < nch; c++) {
-      const size_t i2 = ((size_t)bh * nch + c) * 2;
-      const float sc = shifts[i2];            // both halves carry the same shift
-      const float pm = fmaxf(__int_as_float(pmax[i2]), __int_as_float(pmax[i2 + 1]));
-      float os = 0.f, bt = 1.f;
-      if (c > 0 && bound > 0.f && isfinite(bound)) {
-        int ex = 0;
-        frexpf(bound, &ex);
-        const float t_inter = sigma + (float)(ex - 14), tau = fmaxf(t_inter, sc);
-        os = exp2f((float)(14 - ex)) * exp2f(t_inter - tau);
-        bt = exp2f(sc - tau);
-      }
-      oscale[c] = os;
-      if (blockIdx.x == 0) beta[(size_t)bh * nch + c] = bt;
-      const float sn = fmaxf(sigma, sc);
-      up[c] = sigma == -INFINITY ? 0.f : exp2f(sigma - sn);
-      add[c] = exp2f(sc - sn);
-      bound = bound * up[c] + add[c] * pm;
-      sigma = sn;
-    }
-  }
-  __syncthreads();
-  // thread t of slice x owns columns 2 (t % 128), 2 (t % 128) + 1 of rows 8x + 4 (t / 128) .. + 3: states come in
-  // and prefixes go out as bf16 pairs (4-byte accesses, a warp's access = 128 contiguous bytes)
-  const int cp = threadIdx.x & 127, n0 = blockIdx.x * 8 + (threadIdx.x >> 7) * 4;
-  const uint32_t* sb = reinterpret_cast<const uint32_t*>(state + (size_t)bh * nch * TC_NV * TC_M) + cp;
-  uint32_t* pb = reinterpret_cast<uint32_t*>(prefix + (size_t)bh * nch * TC_NV * TC_M) + cp;
-  float R[4][2];
-#pragma unroll
-  for (int u = 0; u < 4; u++) R[u][0] = R[u][1] = 0.f;
-  // eight chunks per trip: their loads are issued together, then the running sums move on
-  for (int c0 = 0; c0 < nch; c0 += 8) {
-    uint32_t kv[8][4];
-#pragma unroll
-    for (int k = 0; k < 8; k++)
-#pragma unroll
-      for (int u = 0; u < 4; u++)
-        kv[k][u] = (c0 + k < nch && n0 + u <= TC_DV) ? sb[((size_t)(c0 + k) * TC_NV + n0 + u) * (TC_M / 2)] : 0u;
-#pragma unroll
-    for (int k = 0; k < 8; k++) {
-      const int c = c0 + k;
-      if (c < nch) {
-        const float os = oscale[c], upc = up[c], adc = add[c];
-#pragma unroll
-        for (int u = 0; u < 4; u++) {
-          pb[((size_t)c * TC_NV + n0 + u) * (TC_M / 2)] = pack_bf16(R[u][0] * os, R[u][1] * os);
-          R[u][0] = fmaf(R[u][0], upc, adc * __uint_as_float(kv[k][u] << 16));
-          R[u][1] = fmaf(R[u][1], upc, adc * __uint_as_float(kv[k][u] & 0xffff0000u));
-        }
-      }
-    }
-  }
-}
-
-// ------------------------------------------------------------------------------------------
-// causal query side
-// ------------------------------------------------------------------------------------------
-struct CoSmem {
-  // PHIK doubles as the masked score tile S (bf16, two 64-key blocks) once the score MMAs have read it
-  static constexpr uint32_t PHIQ = 0, PHIK = 4 * TILE_BYTES, PFX = 8 * TILE_BYTES, V = PFX + KVT_BYTES, STAGE = V + TILE_BYTES,
-                            RSUM = STAGE + (EPI_THREADS / 32) * 2048, MISC = RSUM + 2 * TILE * 4, TOTAL = MISC + 256;
-};
-static_assert(CoSmem::PFX % 1024 == 0 && CoSmem::V % 1024 == 0, "swizzled tiles need 1024-byte alignment");
-static_assert(CoSmem::TOTAL + 1024 <= 232448, "shared memory budget");
-struct CoMisc {
-  uint64_t full, s_ready, s_full, out_done, chunk_free;
-  uint32_t tmem_base;
-  int abort_flag;
-};
-constexpr uint32_t CO_COL_OUT = 0, CO_COL_S = 128, CO_TMEM_COLS = 256;
-constexpr uint32_t CO_CHUNK_BYTES = 8 * TILE_BYTES + KVT_BYTES + TILE_BYTES;
-
-__global__ void __launch_bounds__(TC_THREADS, 1)
-tc_causal_out_kernel(const __grid_constant__ CUtensorMap tmPhiQ, const __grid_constant__ CUtensorMap tmPhiK,
-                     const __grid_constant__ CUtensorMap tmPfx, const __grid_constant__ CUtensorMap tmV,
-                     const float* __restrict__ beta, int H, int L, int nch, int chunks_per_block,
-                     __nv_bfloat16* __restrict__ Y, TensorAddr ay, int* __restrict__ status) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  CoMisc* misc = reinterpret_cast<CoMisc*>(sm + CoSmem::MISC);
-  float* rsum = reinterpret_cast<float*>(sm + CoSmem::RSUM);      // [half][row]: row sums of the rounded masked scores
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int bh = blockIdx.y, b = bh / H, h = bh % H;
-  const int c0 = blockIdx.x * chunks_per_block;
-  const int nmine = min(chunks_per_block, nch - c0);
-  if (nmine <= 0) return;                     // uniform over the block, before anything is allocated
-  volatile int* abortp = &misc->abort_flag;
-
-  if (threadIdx.x == 0) {
-    mbar_init(&misc->full, 1);
-    mbar_init(&misc->s_ready, 1);
-    mbar_init(&misc->s_full, EPI_THREADS / 32);
-    mbar_init(&misc->out_done, 1);
-    mbar_init(&misc->chunk_free, EPI_THREADS / 32);
-    misc->abort_flag = 0;
-    fence_barrier_init();
-  }
-  if (warp == WARP_MMA) {
-    tmem_alloc(&misc->tmem_base, CO_TMEM_COLS);
-    tmem_relinquish();
-  }
-  tcgen05_fence_before();
-  __syncthreads();
-  tcgen05_fence_after();
-  const uint32_t tmem = misc->tmem_base;
-
-  if (warp >= WARP_TMA) {
-    regs_release<REGS_PRODUCER>();
-    if (warp == WARP_TMA) {
-      if (lane == 0) {
-        prefetch_tmap(&tmPhiQ);
-        prefetch_tmap(&tmPhiK);
-        prefetch_tmap(&tmPfx);
-        prefetch_tmap(&tmV);
-        int issued = 0;
-        for (int it = 0; it < nmine; it++) {
-          const int c = c0 + it;
-          if (it > 0 && !mbar_wait(&misc->chunk_free, (it - 1) & 1, abortp, status)) break;
-          mbar_expect_tx(&misc->full, CO_CHUNK_BYTES);
-#pragma unroll
-          for (int fb = 0; fb < TC_M / 64; fb++) {
-            tma_load_3d(sm + CoSmem::PHIQ + fb * TILE_BYTES, &tmPhiQ, &misc->full, fb * 64, c * TILE, bh);
-            tma_load_3d(sm + CoSmem::PHIK + fb * TILE_BYTES, &tmPhiK, &misc->full, fb * 64, c * TILE, bh);
-            tma_load_3d(sm + CoSmem::PFX + fb * KVT_BLOCK_BYTES, &tmPfx, &misc->full, fb * 64, 0, bh * nch + c);
+            for (int k = 0; k < TILE / 16; k++)
+              mma_bf16(tmem + CF_T + hh * TC_NV, desc_advance(dPhiMN, hh * 2 * CfSmem::BLK + k * 2048), desc_advance(dV1, k * 2048),
+                       ID_STATE, 1u);
           }
-          tma_load_4d(sm + CoSmem::V, &tmV, &misc->full, 0, c * TILE, h, b);
-          issued = it + 1;
-          if (it + 1 < nmine) {           // the next chunk's operands: into L2 while this one is worked on
+          mma_commit(&misc->st_ready);
+          // scores and inter-tile output, 64 features (four K steps) at a time
+          if (!mbar_wait(&misc->p_full, it & 1, abortp, status)) break;
+          if (it > 0 && !mbar_wait(&misc->o_free, (it - 1) & 1, abortp, status)) break;
+          bool ok2 = true;
+#pragma unroll 1
+          for (int pr = 0; pr < 2; pr++) {
+            if (!mbar_wait(&misc->phiq_full[pr], it & 1, abortp, status)) { ok2 = false; break; }
+            tcgen05_fence_after();
 #pragma unroll
-            for (int fb = 0; fb < TC_M / 64; fb++) {
-              tma_prefetch_3d(&tmPhiQ, fb * 64, (c + 1) * TILE, bh);
-              tma_prefetch_3d(&tmPhiK, fb * 64, (c + 1) * TILE, bh);
-              tma_prefetch_3d(&tmPfx, fb * 64, 0, bh * nch + c + 1);
+            for (int j = 0; j < 8; j++) {
+              const int fb = 2 * pr + (j >> 2), k = j & 3;
+              mma_bf16_ta(tmem + CF_S, tmem + CF_L + fb * 32 + k * 8, desc_advance(dKP, fb * CfSmem::BLK + 32 * k), ID_SO,
+                          (pr | j) ? 1u : 0u);
             }
-            tma_prefetch_4d(&tmV, 0, (c + 1) * TILE, h, b);
           }
-        }
-        // no copy of this block may still be in flight when it exits
-        if (issued > 0) mbar_wait(&misc->full, (issued - 1) & 1, abortp, status, false);
-      }
-    } else if (warp == WARP_MMA) {
-      if (lane == 0) {
-        constexpr uint32_t ID_INTER = idesc_bf16(128, TC_NV, 0, 0);      // phiQ P^T
-        constexpr uint32_t ID_SCORE = idesc_bf16(128, 128, 0, 0);        // phiQ phiK^T
-        constexpr uint32_t ID_SV = idesc_bf16(128, TC_DV, 0, 1);        // S V (V with the value index contiguous)
-        const uint64_t dQ = smem_desc(smem_u32(sm + CoSmem::PHIQ), 16, 1024, SWZ_128B);
-        const uint64_t dK = smem_desc(smem_u32(sm + CoSmem::PHIK), 16, 1024, SWZ_128B);
-        const uint64_t dP = smem_desc(smem_u32(sm + CoSmem::PFX), 16, 1024, SWZ_128B);
-        const uint64_t dV = smem_desc(smem_u32(sm + CoSmem::V), TILE_BYTES, 1024, SWZ_128B);
-        for (int it = 0; it < nmine; it++) {
-          if (!mbar_wait(&misc->full, it & 1, abortp, status)) break;
-          tcgen05_fence_after();
-#pragma unroll 1
-          for (int fb = 0; fb < TC_M / 64; fb++) {
-#pragma unroll
-            for (int k = 0; k < 4; k++)
-              mma_bf16(tmem + CO_COL_OUT, desc_advance(dQ, fb * TILE_BYTES + 32 * k), desc_advance(dP, fb * KVT_BLOCK_BYTES + 32 * k),
-                       ID_INTER, (fb | k) ? 1u : 0u);
-          }
-#pragma unroll 1
-          for (int fb = 0; fb < TC_M / 64; fb++) {
-#pragma unroll
-            for (int k = 0; k < 4; k++)
-              mma_bf16(tmem + CO_COL_S, desc_advance(dQ, fb * TILE_BYTES + 32 * k), desc_advance(dK, fb * TILE_BYTES + 32 * k),
-                       ID_SCORE, (fb | k) ? 1u : 0u);
-          }
+          if (!ok2) break;
           mma_commit(&misc->s_ready);
-          if (!mbar_wait(&misc->s_full, it & 1, abortp, status)) break;
+          // the next tile's first key logits go ahead of the masked-score product: they only need the columns that
+          // the MMAs above have finished reading by the time they run (the pipe keeps issue order)
+          if (!mbar_wait(&misc->lg_free, nlg & 1, abortp, status)) break;      // (long since: the query logits were taken)
+          nlg++;
+          if (it + 1 < ntiles) {
+            if (!mbar_wait(&misc->x_ready, nxr & 1, abortp, status)) break;
+            tcgen05_fence_after();
+            issue_logits(dW2, 0);
+          }
+          if (!mbar_wait(&misc->sm_full, it & 1, abortp, status)) break;
           tcgen05_fence_after();
-          // S tile: [128 queries x 128 keys] bf16 in the phiK region, two 64-key blocks
-#pragma unroll 2
-          for (int j = 0; j < TILE / 16; j++)
-            mma_bf16(tmem + CO_COL_OUT, desc_advance(dK, (j >> 2) * TILE_BYTES + 32 * (j & 3)), desc_advance(dV, j * 2048), ID_SV, 1u);
-          mma_commit(&misc->out_done);
+#pragma unroll
+          for (int k = 0; k < TILE / 16; k++)
+            mma_bf16_ta(tmem + CF_O, tmem + CF_S + k * 8, desc_advance(dV1, k * 2048), ID_SV, 1u);
+          mma_commit(&misc->o_ready);
+          mma_commit(&misc->v_free);
         }
+      }
+    } else {
+      // ---------------- bf16 -> fp16 of the token tile, in place (16-byte pieces keep their swizzled positions)
+      const int t = (warp - WARP_CVT0) * 32 + lane;
+      for (int n = 0; n < 2 * ntiles; n++) {
+        if (!mbar_wait(&misc->x_full, n & 1, abortp, status, false)) break;
+        uint4* xt = reinterpret_cast<uint4*>(sm + CfSmem::X);
+#pragma unroll 4
+        for (int i = 0; i < (int)(TILE_BYTES / 16) / CVT_THREADS; i++) {
+          uint4 u = xt[t + i * CVT_THREADS];
+          u.x = pack_f16(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
+          u.y = pack_f16(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
+          u.z = pack_f16(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u));
+          u.w = pack_f16(__uint_as_float(u.w << 16), __uint_as_float(u.w & 0xffff0000u));
+          xt[t + i * CVT_THREADS] = u;
+        }
+        fence_proxy_async_smem();
+        mbar_arrive_warp(&misc->x_ready, lane);
       }
     }
   } else {
-    regs_acquire<REGS_EPILOGUE>();
+    regs_acquire<CF_REGS_EPILOGUE>();
+    // ---------------- epilogue warps.  As a token's thread: row = 32 q + lane, feature blocks hf and 2 + hf (64
+    // features each; block hf comes out of the first logits half, block 2 + hf out of the second).  As a
+    // feature's thread (state, bf16(T)): feature m = 128 hf + row, lane `row` of accumulator hf.
     const int q = warp & 3, hf = warp >> 2;
     const int row = q * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+    const int m = hf * 128 + row;
     __nv_bfloat16* Yb = Y + b * ay.sb + h * ay.sh;
-    for (int it = 0; it < nmine; it++) {
-      const int c = c0 + it;
-      const float bt = beta[(size_t)bh * nch + c];
-      if (!mbar_wait(&misc->s_ready, it & 1, abortp, status, false)) break;
-      __syncwarp();
-      tcgen05_fence_after();
-      // this thread's 64 keys of its query row: mask (key <= query), scale, round to bf16
-      float sum = 0.f;
-      uint8_t* srow = sm + CoSmem::PHIK + hf * TILE_BYTES + row * 128;
+    uint8_t* blk0 = sm + CfSmem::KP + hf * CfSmem::BLK;              // phi(K) block hf
+    uint8_t* blk1 = sm + CfSmem::KP + (2 + hf) * CfSmem::BLK;        // phi(K) block 2 + hf
+    uint8_t* pcol = sm + CfSmem::KP + (m >> 6) * CfSmem::BLK + TILE_BYTES;   // bf16(T), block of feature m
+    float s = -INFINITY;                                              // the keys' running shift
+    bool alive = true;
+    int npair = 0, nall = 0;
+    // all threads of the two warps of row quarter q (resp. of all eight warps) have reached this point
+    auto sync_pair = [&]() {
+      mbar_arrive_warp(&misc->pair_bar[q], lane);
+      if (!mbar_wait(&misc->pair_bar[q], npair & 1, abortp, status, false)) alive = false;
+      npair++;
+    };
+    auto sync_all = [&]() {
+      mbar_arrive_warp(&misc->all_bar, lane);
+      if (!mbar_wait(&misc->all_bar, nall & 1, abortp, status, false)) alive = false;
+      nall++;
+    };
+    // ---- the state before this segment: sum of the earlier segments' totals (their own shifts, without the
+    // per-feature term) brought to one shift, with this side's share a2 / 2 of the per-feature term
+    {
+      const int np = seg == 0 ? 0 : min(nsplit1, seg);               // key-side splits are segments
+      float val[TC_NV];
 #pragma unroll
-      for (int cc = 0; cc < 4; cc++) {
-        uint32_t t[16];
-        tmem_ld16(lane_addr + CO_COL_S + hf * 64 + cc * 16, t);
-        tmem_wait_ld();
-        uint32_t p[8];
+      for (int n = 0; n < TC_NV; n++) val[n] = 0.f;
+      if (np > 0) {
+        const float a2h = fa2[m];
+        float wmx = a2h;
 #pragma unroll
-        for (int j = 0; j < 8; j++) {
-          const int k0 = hf * 64 + cc * 16 + 2 * j;
-          const float s0 = k0 <= row ? __uint_as_float(t[2 * j]) * bt : 0.f;
-          const float s1 = k0 + 1 <= row ? __uint_as_float(t[2 * j + 1]) * bt : 0.f;
-          p[j] = pack_bf16(s0, s1);
-          sum += __uint_as_float(p[j] << 16) + __uint_as_float(p[j] & 0xffff0000u);
+        for (int o = 16; o > 0; o >>= 1) wmx = fmaxf(wmx, __shfl_xor_sync(0xffffffffu, wmx, o));
+        if (lane == 0) misc->red[warp] = wmx;
+        sync_all();
+        float a2max = misc->red[0];
+#pragma unroll
+        for (int i = 1; i < EPI_THREADS / 32; i++) a2max = fmaxf(a2max, misc->red[i]);
+        const float* sh = shifts + (size_t)bh * nsplit1 * 2;
+        float smax = -INFINITY;
+        for (int p = 0; p < 2 * np; p++) smax = fmaxf(smax, sh[p]);
+        s = smax + a2max;
+        const float* base = partial + (size_t)bh * nsplit1 * TC_NV * TC_M + m;
+        for (int p = 0; p < np; p++) {
+          const float f = exp2f(sh[2 * p + hf] + a2h - s);
+          const float* bp = base + (size_t)p * TC_NV * TC_M;
+#pragma unroll
+          for (int n = 0; n <= TC_DV; n++) val[n] = fmaf(bp[n * TC_M], f, val[n]);
         }
-        *reinterpret_cast<uint4*>(srow + (((2 * cc) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
-        *reinterpret_cast<uint4*>(srow + (((2 * cc + 1) ^ (row & 7)) << 4)) = make_uint4(p[4], p[5], p[6], p[7]);
       }
-      rsum[hf * TILE + row] = sum;
-      fence_proxy_async_smem();
+#pragma unroll
+      for (int c = 0; c < TC_NV / 16; c++) {
+        uint32_t a[16];
+#pragma unroll
+        for (int j = 0; j < 16; j++) a[j] = __float_as_uint(val[c * 16 + j]);
+        tmem_st16(lane_addr + CF_T + hf * TC_NV + c * 16, a);
+      }
+      tmem_wait_st();
       tcgen05_fence_before();
-      mbar_arrive_warp(&misc->s_full, lane);
-      if (!mbar_wait(&misc->out_done, it & 1, abortp, status, false)) break;
+    }
+    const float* cptr = crow + (size_t)bh * Lpad + (size_t)tile0 * TILE + row;
+    float cj = cptr[0];
+
+    // Y rows of tile j (all its MMAs have completed): 32 of the 64 columns per thread
+    auto write_out = [&](int j) {
       __syncwarp();
       tcgen05_fence_after();
       uint32_t n0[32], d0[16];
-      tmem_ld16(lane_addr + CO_COL_OUT + hf * 32, reinterpret_cast<uint32_t(&)[16]>(n0[0]));
-      tmem_ld16(lane_addr + CO_COL_OUT + hf * 32 + 16, reinterpret_cast<uint32_t(&)[16]>(n0[16]));
-      tmem_ld16(lane_addr + CO_COL_OUT + TC_DV, d0);
+      tmem_ld16(lane_addr + CF_O + hf * 32, reinterpret_cast<uint32_t(&)[16]>(n0[0]));
+      tmem_ld16(lane_addr + CF_O + hf * 32 + 16, reinterpret_cast<uint32_t(&)[16]>(n0[16]));
+      tmem_ld16(lane_addr + CF_O + TC_DV, d0);
       tmem_wait_ld();
+      tcgen05_fence_before();
+      mbar_arrive_warp(&misc->o_free, lane);
       const float den = __uint_as_float(d0[0]) + rsum[row] + rsum[TILE + row];
-      const int64_t r0 = (int64_t)c * TILE + q * 32;                  // first row of this warp
+      const int64_t r0 = (int64_t)(tile0 + j) * TILE + q * 32;       // first row of this warp
       if (r0 + lane < L && (!(den > 0.f) || !isfinite(den))) atomicExch(status, FSHARP_E_NONFINITE);
       const float inv = 1.f / den;
-      uint8_t* stg = sm + CoSmem::STAGE + warp * 2048;
+      // The thread's 64 bytes go through shared memory so that a store instruction of the warp covers 8 rows x 64
+      // contiguous bytes.  The staging area is the part of the phi(K) block that this warp itself writes next.
+      uint8_t* stg = blk0 + q * 4096;
 #pragma unroll
       for (int i = 0; i < 4; i++) {
         uint32_t o[4];
@@ -453,15 +390,225 @@ tc_causal_out_kernel(const __grid_constant__ CUtensorMap tmPhiQ, const __grid_co
         if (r0 + rr < L) *reinterpret_cast<uint4*>(Yb + (r0 + rr) * ay.sl + hf * 32 + cw * 8) = val;
       }
       __syncwarp();
+    };
+
+    int nlg = 0;
+    for (int it = 0; it < ntiles && alive; it++) {
+      const float cnext = it + 1 < ntiles ? cptr[(size_t)(it + 1) * TILE] : 0.f;     // in flight during this tile
+      uint32_t v[128];
+      // ---- key logits, first half
+      if (!mbar_wait(&misc->lg_full, nlg & 1, abortp, status, false)) { alive = false; break; }
+      nlg++;
+      __syncwarp();
+      tcgen05_fence_after();
+#pragma unroll
+      for (int c = 0; c < 4; c++) tmem_ld16(lane_addr + CF_L + hf * 64 + c * 16, reinterpret_cast<uint32_t(&)[16]>(v[c * 16]));
+      tmem_wait_ld();
       tcgen05_fence_before();
-      mbar_arrive_warp(&misc->chunk_free, lane);
+      mbar_arrive_warp(&misc->lg_free, lane);
+      // ---- while the second half is computed: the previous tile's output.  Its state update has completed
+      // (nothing reads the previous phi(K) tile any more), and so has its masked-score product.
+      if (it > 0) {
+        if (!mbar_wait(&misc->st_ready, (it - 1) & 1, abortp, status, false)) { alive = false; break; }
+        if (!mbar_wait(&misc->o_ready, (it - 1) & 1, abortp, status, false)) { alive = false; break; }
+        write_out(it - 1);
+      }
+      // ---- key logits, second half
+      if (!mbar_wait(&misc->lg_full, nlg & 1, abortp, status, false)) { alive = false; break; }
+      nlg++;
+      __syncwarp();
+      tcgen05_fence_after();
+#pragma unroll
+      for (int c = 0; c < 4; c++) tmem_ld16(lane_addr + CF_L + hf * 64 + c * 16, reinterpret_cast<uint32_t(&)[16]>(v[64 + c * 16]));
+      tmem_wait_ld();
+      tcgen05_fence_before();
+      mbar_arrive_warp(&misc->lg_free, lane);
+      const bool valid = (tile0 + it) * TILE + row < L;
+      // ---- exact maximum of the tile's exponents (with the per-feature share), one value for the block
+      float tm;
+      {
+        float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int i = 0; i < 128; i += 4) {
+          const float4 a4 = *reinterpret_cast<const float4*>(fa2 + (i >> 6) * 128 + hf * 64 + (i & 63));
+          v[i] = __float_as_uint(__uint_as_float(v[i]) + a4.x);
+          v[i + 1] = __float_as_uint(__uint_as_float(v[i + 1]) + a4.y);
+          v[i + 2] = __float_as_uint(__uint_as_float(v[i + 2]) + a4.z);
+          v[i + 3] = __float_as_uint(__uint_as_float(v[i + 3]) + a4.w);
+          mxp[0] = fmaxf(mxp[0], __uint_as_float(v[i]));
+          mxp[1] = fmaxf(mxp[1], __uint_as_float(v[i + 1]));
+          mxp[2] = fmaxf(mxp[2], __uint_as_float(v[i + 2]));
+          mxp[3] = fmaxf(mxp[3], __uint_as_float(v[i + 3]));
+        }
+        float mx = valid ? fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])) + cj : -INFINITY;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (lane == 0) atomicMax(&misc->chunk_max[it % 3], f2ord(mx));
+        if (threadIdx.x == 0) misc->chunk_max[(it + 1) % 3] = f2ord(-INFINITY);   // next tile's slot; idle since tile it - 2
+        sync_all();
+        if (!alive) break;
+        tm = ord2f(misc->chunk_max[it % 3]);
+      }
+      if (s == -INFINITY) {
+        s = tm;                      // first keys of the sequence: the state is still zero
+      } else if (tm - s > SHIFT_HEADROOM_LOG2) {
+        // rare: the shift moves up to this tile's maximum and the state with it (the previous tile's update of the
+        // state has completed: st_ready was waited for above)
+        __syncwarp();
+        tcgen05_fence_after();
+        const float f = ex2(s - tm);
+#pragma unroll
+        for (int c = 0; c < TC_NV / 16; c++) {
+          uint32_t a[16];
+          tmem_ld16(lane_addr + CF_T + hf * TC_NV + c * 16, a);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 16; j++) a[j] = __float_as_uint(__uint_as_float(a[j]) * f);
+          tmem_st16(lane_addr + CF_T + hf * TC_NV + c * 16, a);
+        }
+        tmem_wait_st();
+        tcgen05_fence_before();
+        s = tm;
+      }
+      // ---- bf16(T) of the state before this tile: row `row` of accumulator hf = column m of T.  The previous
+      // tile's MMAs that read the old copy have completed (its scores were taken out of tensor memory).
+      {
+        __syncwarp();
+        tcgen05_fence_after();
+#pragma unroll
+        for (int c = 0; c < TC_NV / 16; c++) {
+          uint32_t a[16];
+          tmem_ld16(lane_addr + CF_T + hf * TC_NV + c * 16, a);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 16; j++)
+            if (c * 16 + j <= TC_DV)
+              *reinterpret_cast<__nv_bfloat16*>(pcol + sw128_offset(c * 16 + j, m & 63)) = __float2bfloat16_rn(__uint_as_float(a[j]));
+        }
+        tcgen05_fence_before();
+        fence_proxy_async_smem();
+        mbar_arrive_warp(&misc->p_full, lane);
+      }
+      // ---- phi(K): 2^(exponent - s), bf16, 64 features at a time
+      {
+        const float rc = cj - s;
+#pragma unroll
+        for (int half = 0; half < 2; half++) {
+          uint8_t* prow = (half ? blk1 : blk0) + row * 128;
+#pragma unroll
+          for (int c = 0; c < 8; c++) {
+            uint32_t p[4];
+#pragma unroll
+            for (int j = 0; j < 4; j++)
+              p[j] = pack_bf16(ex2(__uint_as_float(v[half * 64 + c * 8 + 2 * j]) + rc), ex2(__uint_as_float(v[half * 64 + c * 8 + 2 * j + 1]) + rc));
+            if (!valid) p[0] = p[1] = p[2] = p[3] = 0u;
+            *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
+          }
+          fence_proxy_async_smem();
+          mbar_arrive_warp(&misc->phik_full[half], lane);
+        }
+      }
+      // ---- query logits
+      if (!mbar_wait(&misc->lg_full, nlg & 1, abortp, status, false)) { alive = false; break; }
+      nlg++;
+      __syncwarp();
+      tcgen05_fence_after();
+#pragma unroll
+      for (int c = 0; c < 4; c++) tmem_ld16(lane_addr + CF_L + hf * 64 + c * 16, reinterpret_cast<uint32_t(&)[16]>(v[c * 16]));
+      tmem_wait_ld();
+      tcgen05_fence_before();
+      mbar_arrive_warp(&misc->lg_free, lane);
+      if (!mbar_wait(&misc->lg_full, nlg & 1, abortp, status, false)) { alive = false; break; }
+      nlg++;
+      __syncwarp();
+      tcgen05_fence_after();
+#pragma unroll
+      for (int c = 0; c < 4; c++) tmem_ld16(lane_addr + CF_L + hf * 64 + c * 16, reinterpret_cast<uint32_t(&)[16]>(v[64 + c * 16]));
+      tmem_wait_ld();
+      tcgen05_fence_before();
+      mbar_arrive_warp(&misc->lg_free, lane);
+      float mx;
+      {
+        float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int i = 0; i < 128; i += 4) {
+          const float4 a4 = *reinterpret_cast<const float4*>(fa2 + (i >> 6) * 128 + hf * 64 + (i & 63));
+          v[i] = __float_as_uint(__uint_as_float(v[i]) + a4.x);
+          v[i + 1] = __float_as_uint(__uint_as_float(v[i + 1]) + a4.y);
+          v[i + 2] = __float_as_uint(__uint_as_float(v[i + 2]) + a4.z);
+          v[i + 3] = __float_as_uint(__uint_as_float(v[i + 3]) + a4.w);
+          mxp[0] = fmaxf(mxp[0], __uint_as_float(v[i]));
+          mxp[1] = fmaxf(mxp[1], __uint_as_float(v[i + 1]));
+          mxp[2] = fmaxf(mxp[2], __uint_as_float(v[i + 2]));
+          mxp[3] = fmaxf(mxp[3], __uint_as_float(v[i + 3]));
+        }
+        mx = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
+        // the row's other thread sits in warp q of the other warpgroup; after this barrier both have also taken
+        // their logits out of tensor memory, whose columns the features now overwrite
+        rowmax[hf * TILE + row] = mx;
+        sync_pair();
+        if (!alive) break;
+        mx = fmaxf(mx, rowmax[(hf ^ 1) * TILE + row]);
+      }
+      // ---- phi(Q): 2^(exponent - row maximum), bf16 pairs over the logits' columns: block fb at columns 32 fb
+#pragma unroll
+      for (int half = 0; half < 2; half++) {
+        const int fb = 2 * half + hf;
+#pragma unroll
+        for (int c = 0; c < 2; c++) {
+          uint32_t p[16];
+#pragma unroll
+          for (int j = 0; j < 16; j++)
+            p[j] = pack_bf16(ex2(__uint_as_float(v[half * 64 + c * 32 + 2 * j]) - mx), ex2(__uint_as_float(v[half * 64 + c * 32 + 2 * j + 1]) - mx));
+          tmem_st16(lane_addr + CF_L + fb * 32 + c * 16, p);
+        }
+        tmem_wait_st();
+        tcgen05_fence_before();
+        mbar_arrive_warp(&misc->phiq_full[half], lane);
+      }
+      // ---- scores: mask (key <= query), round to bf16 over their own columns, keep the row sums
+      if (!mbar_wait(&misc->s_ready, it & 1, abortp, status, false)) { alive = false; break; }
+      __syncwarp();
+      tcgen05_fence_after();
+      {
+        uint32_t pm[32];
+        float sum = 0.f;
+#pragma unroll
+        for (int cc = 0; cc < 4; cc++) {
+          uint32_t t[16];
+          tmem_ld16(lane_addr + CF_S + hf * 64 + cc * 16, t);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 8; j++) {
+            const int k0 = hf * 64 + cc * 16 + 2 * j;
+            const float s0 = k0 <= row ? __uint_as_float(t[2 * j]) : 0.f;
+            const float s1 = k0 + 1 <= row ? __uint_as_float(t[2 * j + 1]) : 0.f;
+            const uint32_t pk = pack_bf16(s0, s1);
+            pm[cc * 8 + j] = pk;
+            sum += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
+          }
+        }
+        rsum[hf * TILE + row] = sum;
+        // the packed scores of the row's second thread land on columns its first thread reads: both have read
+        sync_pair();
+        if (!alive) break;
+        tmem_st16(lane_addr + CF_S + hf * 32, reinterpret_cast<uint32_t(&)[16]>(pm[0]));
+        tmem_st16(lane_addr + CF_S + hf * 32 + 16, reinterpret_cast<uint32_t(&)[16]>(pm[16]));
+        tmem_wait_st();
+        tcgen05_fence_before();
+        mbar_arrive_warp(&misc->sm_full, lane);
+      }
+      cj = cnext;
     }
+    if (alive && mbar_wait(&misc->st_ready, (ntiles - 1) & 1, abortp, status, false) &&
+        mbar_wait(&misc->o_ready, (ntiles - 1) & 1, abortp, status, false))
+      write_out(ntiles - 1);
   }
   tcgen05_fence_before();
   __syncthreads();
   if (warp == WARP_MMA) {
     tcgen05_fence_after();
-    tmem_dealloc(tmem, CO_TMEM_COLS);
+    tmem_dealloc(tmem, TMEM_COLS);
   }
 }
 
@@ -472,90 +619,77 @@ tc_causal_out_kernel(const __grid_constant__ CUtensorMap tmPhiQ, const __grid_co
 // ------------------------------------------------------------------------------------------
 namespace tchost {
 int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int H, int L, int inner);
-int make_map_kvt(CUtensorMap* map, const void* base, int BH, int bf16);
-int make_map_feat(CUtensorMap* map, const void* base, int BH, int Lpad);
 }  // namespace tchost
+int fs_tc_rowterm(fsharp_ctx* ctx, const void* K, const fsharp_dims* dm, const uint8_t* images, const int* flags, int Lpad,
+                  int tiles_per_split, int nsplit, float* crow);
 int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
-                   const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax,
-                   __nv_bfloat16* phik);
+                   const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax);
 int fs_tc_causal_supported(const fsharp_dims* dm, int chunk);
 size_t fs_tc_causal_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
 int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                  const int* flags, void* Y, WsAlloc* ws);
 
+namespace {
+constexpr int CF_MAX_SEG = 64;
+
+// Segments of equal tile count per (batch, head).  A segment's block walks its tiles one after the other (about 2.2
+// times a key-side tile each); every segment but the last also costs a key-side pass over its tiles.
+int pick_segments(int units, int tiles, int sms, int* tiles_per_seg) {
+  int best = 1, best_per = tiles;
+  double best_cost = 1e300;
+  for (int ns = 1; ns <= tiles && ns <= CF_MAX_SEG; ns++) {
+    const int per = (tiles + ns - 1) / ns;
+    if ((tiles + per - 1) / per != ns) continue;
+    const long long b2 = (long long)units * ns, b1 = (long long)units * (ns - 1);
+    double cost = (double)((b2 + sms - 1) / sms) * (2.2 * per + 3.0);
+    if (ns > 1) cost += (double)((b1 + sms - 1) / sms) * (per + 4.0);
+    if (cost < best_cost) { best_cost = cost; best = ns; best_per = per; }
+  }
+  *tiles_per_seg = best_per;
+  return best;
+}
+}  // namespace
+
+// The mask is applied token by token, so the result does not depend on `chunk`: the kernel always walks 128-token tiles.
 int fs_tc_causal_supported(const fsharp_dims* dm, int chunk) {
-  if (chunk != TILE || dm->Lq != dm->Lk || dm->Lq <= 0) return 0;
-  const int nch = (dm->Lq + TILE - 1) / TILE;
-  return nch <= PFX_MAXCH;
+  (void)chunk;
+  return dm->Lq == dm->Lk && dm->Lq > 0;
 }
 
 size_t fs_tc_causal_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
   (void)ctx;
   const size_t BH = (size_t)dm->B * dm->H, G = fs_groups(dm);
   const size_t nch = (dm->Lk + TILE - 1) / TILE, Lpad = nch * TILE;
-  return ws_round(G * 2 * IMG_BYTES) + ws_round(G * 2 * FLAG_WORDS * 4 + 64) + ws_round(BH * nch * TC_M * TC_NV * 4) +
-         2 * ws_round(BH * nch * 2 * 4) + ws_round(BH * Lpad * 4) + 2 * ws_round(BH * Lpad * TC_M * 2) +
-         ws_round(BH * nch * TC_NV * TC_M * 2) + ws_round(BH * nch * 4);
+  return ws_round(G * 2 * IMG_BYTES) + ws_round(G * 2 * FLAG_WORDS * 4 + 64) + ws_round(BH * CF_MAX_SEG * TC_M * TC_NV * 4) +
+         2 * ws_round(BH * CF_MAX_SEG * 2 * 4) + ws_round(BH * Lpad * 4);
 }
 
 int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                  const int* flags, void* Y, WsAlloc* ws) {
   const int B = dm->B, H = dm->H, BH = B * H, L = dm->Lq;
   const int nch = (L + TILE - 1) / TILE, Lpad = nch * TILE;
-  __nv_bfloat16* state = ws->take<__nv_bfloat16>((size_t)BH * nch * TC_M * TC_NV);     // chunk states, bf16
-  float* shifts = ws->take<float>((size_t)BH * nch * 2);
-  int* pmax = ws->take<int>((size_t)BH * nch * 2);
+  float* partial = ws->take<float>((size_t)BH * CF_MAX_SEG * TC_M * TC_NV);
+  float* shifts = ws->take<float>((size_t)BH * CF_MAX_SEG * 2);
+  int* pmax = ws->take<int>((size_t)BH * CF_MAX_SEG * 2);
   float* crow = ws->take<float>((size_t)BH * Lpad);
-  __nv_bfloat16* phik16 = ws->take<__nv_bfloat16>((size_t)BH * Lpad * TC_M);
-  __nv_bfloat16* phiq16 = ws->take<__nv_bfloat16>((size_t)BH * Lpad * TC_M);
-  __nv_bfloat16* prefix = ws->take<__nv_bfloat16>((size_t)BH * nch * TC_NV * TC_M);
-  float* beta = ws->take<float>((size_t)BH * nch);
-  FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * nch * 2 * sizeof(int), ctx->stream));
-
-  // query features
-  CUtensorMap tmQ, tmPhiQ, tmPhiK, tmPfx, tmV;
+  int per = 0;
+  const int nseg = pick_segments(BH, nch, ctx->sm_count, &per);
+  // key side: the per-key quadratic term of every key, and the totals of the segments that have a successor
+  if (nseg > 1) {
+    FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * (nseg - 1) * 2 * sizeof(int), ctx->stream));
+    FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, per, nseg - 1, crow, partial, shifts, pmax));
+  } else {
+    FS_TRY(fs_tc_rowterm(ctx, K, dm, images, flags, Lpad, per, 1, crow));
+  }
+  CUtensorMap tmQ, tmK, tmV;
   FS_TRY(tchost::make_map_tokens(&tmQ, Q, fs_addr(dm->q_stride, H, L, dm->d), B, H, L, dm->d));
+  FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, L, dm->d), B, H, L, dm->d));
   FS_TRY(tchost::make_map_tokens(&tmV, V, fs_addr(dm->v_stride, H, L, dm->dv), B, H, L, dm->dv));
-  FS_TRY(tchost::make_map_feat(&tmPhiQ, phiq16, BH, Lpad));
-  FS_TRY(tchost::make_map_feat(&tmPhiK, phik16, BH, Lpad));
-  FS_TRY(tchost::make_map_kvt(&tmPfx, prefix, BH * nch, 1));
-  // blocks of equal tile count: (waves of blocks) x (tiles per block + fill and drain)
-  auto split = [&](int overhead, int* per) {
-    int best = 1, best_cost = 0x7fffffff, best_per = nch;
-    for (int ns = 1; ns <= nch; ns++) {
-      const int t = (nch + ns - 1) / ns;
-      if ((nch + t - 1) / t != ns) continue;
-      const long long blocks = (long long)BH * ns;
-      const int cost = (int)((blocks + ctx->sm_count - 1) / ctx->sm_count) * (t + overhead);
-      if (cost < best_cost) { best_cost = cost; best = ns; best_per = t; }
-    }
-    *per = best_per;
-    return best;
-  };
-  // key side: chunk states and bf16 key features
-  int kper = 0;
-  const int ksplit = split(4, &kper);
-  FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, kper, ksplit, crow, reinterpret_cast<float*>(state), shifts, pmax, phik16));
-  int qper = 0;
-  const int qsplit = split(4, &qper);
-  FS_CUDA_OK(cudaFuncSetAttribute(tc_featq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FqSmem::TOTAL + 1024));
-  FS_TIME_BEGIN(ctx, FS_K_TC_FEATQ);
-  tc_featq_kernel<<<dim3(qsplit, BH), TC_THREADS, FqSmem::TOTAL + 1024, ctx->stream>>>(tmQ, tmPhiQ, images, H, dm->pool, L, qper,
-                                                                                       ctx->d_status);
-  FS_TIME_END(ctx);
-  FS_LAUNCH_CHECK(ctx);
-
-  FS_TIME_BEGIN(ctx, FS_K_TC_CAUSAL_PREFIX);
-  tc_causal_prefix_kernel<<<dim3(PFX_SLICES, BH), 256, 0, ctx->stream>>>(state, shifts, pmax, nch, prefix, beta);
-  FS_TIME_END(ctx);
-  FS_LAUNCH_CHECK(ctx);
-
-  int cper = 0;
-  const int csplit = split(2, &cper);
-  FS_CUDA_OK(cudaFuncSetAttribute(tc_causal_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CoSmem::TOTAL + 1024));
-  FS_TIME_BEGIN(ctx, FS_K_TC_CAUSAL_OUT);
-  tc_causal_out_kernel<<<dim3(csplit, BH), TC_THREADS, CoSmem::TOTAL + 1024, ctx->stream>>>(
-      tmPhiQ, tmPhiK, tmPfx, tmV, beta, H, L, nch, cper, (__nv_bfloat16*)Y, fs_addr(dm->y_stride, H, L, dm->dv), ctx->d_status);
+  FS_CUDA_OK(cudaFuncSetAttribute(tc_causal_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CfSmem::TOTAL + 1024));
+  FS_TIME_BEGIN(ctx, FS_K_TC_CAUSAL);
+  tc_causal_kernel<<<dim3(nseg, BH), TC_THREADS, CfSmem::TOTAL + 1024, ctx->stream>>>(
+      tmQ, tmK, tmV, images, crow, partial, shifts, nseg - 1, H, dm->pool, L, Lpad, per, (__nv_bfloat16*)Y,
+      fs_addr(dm->y_stride, H, L, dm->dv), ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;

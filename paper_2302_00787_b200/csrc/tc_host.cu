@@ -56,34 +56,6 @@ int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int
   return r == CUDA_SUCCESS ? FSHARP_OK : FSHARP_E_CUDA;
 }
 
-// kvt [BH, 80, 256] fp16 or bf16 -> 3-D map (feature, row, bh), box 64 x 80 x 1, 128-byte swizzle.
-int make_map_kvt(CUtensorMap* map, const void* base, int BH, int bf16) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return FSHARP_E_CUDA;
-  cuuint64_t dims[3] = {(cuuint64_t)TC_M, (cuuint64_t)TC_NV, (cuuint64_t)BH};
-  cuuint64_t strides[2] = {(cuuint64_t)TC_M * 2, (cuuint64_t)TC_M * TC_NV * 2};
-  cuuint32_t box[3] = {64, (cuuint32_t)TC_NV, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? FSHARP_OK : FSHARP_E_CUDA;
-}
-
-// bf16 features [BH, Lpad, 256] -> 3-D map (feature, token, bh), box 64 x 128 x 1, 128-byte swizzle.
-int make_map_feat(CUtensorMap* map, const void* base, int BH, int Lpad) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return FSHARP_E_CUDA;
-  cuuint64_t dims[3] = {(cuuint64_t)TC_M, (cuuint64_t)Lpad, (cuuint64_t)BH};
-  cuuint64_t strides[2] = {(cuuint64_t)TC_M * 2, (cuuint64_t)TC_M * 2 * (cuuint64_t)Lpad};
-  cuuint32_t box[3] = {64, (cuuint32_t)TILE, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? FSHARP_OK : FSHARP_E_CUDA;
-}
-
 }  // namespace tchost
 
 int fs_tc_supported(const fsharp_dims* dm, int dtype, int causal, int chunk, float qk_scale) {
