@@ -34,8 +34,14 @@ using namespace tcl;
 
 namespace {
 
-constexpr int WARP_CVT0 = 10;                 // warps 10 and 11 convert the token tiles to fp16
+// Warps 0-3 are the producer warpgroup (0: TMA copies, 1: all MMAs, 2 and 3: token tiles to fp16), warps 4-11
+// the epilogue.  The single MMA-issuing warp shares its scheduler with two epilogue warps that always have
+// instructions ready; it sits in the lowest warp slots of the block.
+constexpr int CF_WARP_TMA = 0, CF_WARP_MMA = 1, CF_WARP_CVT0 = 2, CF_PRODUCER_WARPS = 4;
 constexpr int CVT_THREADS = 64;
+// Of every four pairs of exponentials, this many are evaluated on the multiply-add pipe (exp2_poly2), the others
+// by the special-function unit, whose 16 results per clock would otherwise bound the kernel.
+constexpr int CF_POLY_PAIRS = 1;
 // The MMA-issuing thread of this kernel keeps more descriptors alive than those of the other kernels:
 // 128 x 64 + 256 x 216 registers (of the 384 x 168 the block is launched with).
 constexpr int CF_REGS_PRODUCER = 64, CF_REGS_EPILOGUE = 216;
@@ -52,7 +58,7 @@ static_assert(CfSmem::KP % 1024 == 0 && CfSmem::BLK % 1024 == 0 && CfSmem::X % 1
 static_assert(CfSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 
 struct CfMisc {
-  uint64_t const_bar, x_full, x_ready, x_free, v_full, v_free, lg_full, lg_free, phik_full[2], phiq_full[2], p_full,
+  uint64_t const_bar, x_full, x_ready, x_free, v_full, v_free, lg_full, lg_free, phik_full[2], phiq_full[5], p_full,
       s_ready, sm_full, o_ready, o_free, st_ready;
   // meeting points of the epilogue warps (the two warps of a row quarter; all eight): mbarriers, so that these
   // waits are bounded like every other
@@ -60,7 +66,6 @@ struct CfMisc {
   uint32_t tmem_base;
   int abort_flag;
   int chunk_max[3];
-  float red[8];
 };
 static_assert(sizeof(CfMisc) <= 256, "misc block");
 
@@ -78,7 +83,7 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   CfMisc* misc = reinterpret_cast<CfMisc*>(sm + CfSmem::MISC);
   float* rowmax = reinterpret_cast<float*>(sm + CfSmem::ROWMAX);   // [half][row]
   float* rsum = reinterpret_cast<float*>(sm + CfSmem::RSUM);       // [half][row]: row sums of the rounded masked scores
-  float* fa2 = reinterpret_cast<float*>(sm + CfSmem::FA2);         // each side's share a2 / 2 of the per-feature term
+  float* fa2 = reinterpret_cast<float*>(sm + CfSmem::FA2);         // the per-feature term a2 of both sides: it joins the query logits
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int seg = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
   const int g = pool == FSHARP_POOL_PER_BH ? bh : h;
@@ -99,10 +104,8 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     mbar_init(&misc->v_free, 1);
     mbar_init(&misc->lg_full, 1);
     mbar_init(&misc->lg_free, EPI_THREADS / 32);
-    for (int i = 0; i < 2; i++) {
-      mbar_init(&misc->phik_full[i], EPI_THREADS / 32);
-      mbar_init(&misc->phiq_full[i], EPI_THREADS / 32);
-    }
+    for (int i = 0; i < 2; i++) mbar_init(&misc->phik_full[i], EPI_THREADS / 32);
+    for (int i = 0; i < 5; i++) mbar_init(&misc->phiq_full[i], EPI_THREADS / 32);
     mbar_init(&misc->p_full, EPI_THREADS / 32);
     mbar_init(&misc->s_ready, 1);
     mbar_init(&misc->sm_full, EPI_THREADS / 32);
@@ -121,12 +124,12 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   for (int i = threadIdx.x; i < 4 * (int)(KVT_BLOCK_BYTES / 16); i += TC_THREADS)
     reinterpret_cast<uint4*>(sm + CfSmem::KP + (i / (KVT_BLOCK_BYTES / 16)) * CfSmem::BLK + TILE_BYTES)[i % (KVT_BLOCK_BYTES / 16)] =
         make_uint4(0, 0, 0, 0);
-  if (threadIdx.x < TC_M) fa2[threadIdx.x] = 0.5f * reinterpret_cast<const float*>(img2 + IMG_A2)[threadIdx.x];
+  if (threadIdx.x < TC_M) fa2[threadIdx.x] = reinterpret_cast<const float*>(img1 + IMG_A2)[threadIdx.x];
   __syncthreads();
   if (threadIdx.x < TILE)
     *reinterpret_cast<__nv_bfloat16*>(sm + CfSmem::ONES + sw128_offset(threadIdx.x, 0)) = __float2bfloat16(1.f);
   fence_proxy_async_smem();
-  if (warp == WARP_MMA) {
+  if (warp == CF_WARP_MMA) {
     tmem_alloc(&misc->tmem_base, TMEM_COLS);
     tmem_relinquish();
   }
@@ -135,9 +138,9 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   tcgen05_fence_after();
   const uint32_t tmem = misc->tmem_base;
 
-  if (warp >= WARP_TMA) {
+  if (warp < CF_PRODUCER_WARPS) {
     regs_release<CF_REGS_PRODUCER>();
-    if (warp == WARP_TMA) {
+    if (warp == CF_WARP_TMA) {
       if (lane == 0) {
         prefetch_tmap(&tmQ);
         prefetch_tmap(&tmK);
@@ -174,8 +177,10 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (nx > 0) mbar_wait(&misc->x_full, (nx - 1) & 1, abortp, status, false);
         if (nv > 0) mbar_wait(&misc->v_full, (nv - 1) & 1, abortp, status, false);
       }
-    } else if (warp == WARP_MMA) {
-      if (lane == 0) {
+    } else if (warp == CF_WARP_MMA) {
+      // ---------------- all MMAs of the block.  The whole warp walks the schedule (descriptor arithmetic and waits
+      // stay warp-uniform); one elected lane issues the MMAs and their commits.
+      {
         constexpr uint32_t ID_LOGITS = idesc_f16(128, 128, 0, 0);            // X Wh^T, 128 features
         constexpr uint32_t ID_STATE = idesc_bf16(128, TC_NV, 1, 1);          // phi(K)_h^T [V | 1]
         constexpr uint32_t ID_SO = idesc_bf16(128, 128 + TC_NV, 0, 0);       // phi(Q) [phi(K)^T | bf16(T)]
@@ -187,90 +192,116 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const uint64_t dKP = smem_desc(smem_u32(sm + CfSmem::KP), 16, 1024, SWZ_128B);             // K-major, 208 rows per block
         const uint64_t dPhiMN = smem_desc(smem_u32(sm + CfSmem::KP), CfSmem::BLK, 1024, SWZ_128B); // features contiguous
         const uint64_t dV1 = smem_desc(sV, sOnes - sV, 1024, SWZ_128B);                            // [V | 1], value index contiguous
-        auto issue_logits = [&](uint64_t dW, int half) {
+        // low words (start address / 16) and high words of the descriptors; the low words are made opaque once per
+        // tile so that the offsets are added next to each MMA
+        uint32_t xl = (uint32_t)dX, w1l = (uint32_t)dW1, w2l = (uint32_t)dW2, kpl = (uint32_t)dKP, pml = (uint32_t)dPhiMN, v1l = (uint32_t)dV1;
+        const uint32_t xh = (uint32_t)(dX >> 32), wh = (uint32_t)(dW1 >> 32), kph = (uint32_t)(dKP >> 32), pmh = (uint32_t)(dPhiMN >> 32),
+                       v1h = (uint32_t)(dV1 >> 32);
+        auto issue_logits = [&](uint32_t wl, int half) {
+          if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < TC_D / 16; k++)
-            mma_bf16(tmem + CF_L, desc_advance(dX, 32 * k), desc_advance(dW, half * (IMG_W_BYTES / 2) + 32 * k), ID_LOGITS, k > 0);
-          mma_commit(&misc->lg_full);
+            for (int k = 0; k < TC_D / 16; k++)
+              mma_bf16_lh(tmem + CF_L, xl + 2 * k, xh, wl + half * (IMG_W_BYTES / 32) + 2 * k, wh, ID_LOGITS, k > 0);
+            mma_commit(&misc->lg_full);
+          }
+          __syncwarp();
         };
         int nlg = 0, nxr = 0;                 // logits halves handed over so far, token tiles consumed so far
         bool ok = mbar_wait(&misc->const_bar, 0, abortp, status);
         if (ok) ok = mbar_wait(&misc->x_ready, nxr & 1, abortp, status);
+        ok = __all_sync(0xffffffffu, ok);
         if (ok) {
           tcgen05_fence_after();
-          issue_logits(dW2, 0);
+          issue_logits(w2l, 0);
         }
+        // a wait that gave up in one lane ends the schedule for the whole warp
+#define CF_WAIT(bar, par) if (!__all_sync(0xffffffffu, mbar_wait((bar), (par), abortp, status))) break
         for (int it = 0; ok && it < ntiles; it++) {
+          opaque(xl); opaque(w1l); opaque(w2l); opaque(kpl); opaque(pml); opaque(v1l);
           // second half of the key logits once the epilogue has taken the first out of tensor memory
-          if (!mbar_wait(&misc->lg_free, nlg & 1, abortp, status)) break;
+          CF_WAIT(&misc->lg_free, nlg & 1);
           nlg++;
           tcgen05_fence_after();
-          issue_logits(dW2, 1);
-          mma_commit(&misc->x_free);
+          issue_logits(w2l, 1);
+          if (elect_one()) mma_commit(&misc->x_free);
+          __syncwarp();
           nxr++;
           // query logits
-          if (!mbar_wait(&misc->lg_free, nlg & 1, abortp, status)) break;
+          CF_WAIT(&misc->lg_free, nlg & 1);
           nlg++;
-          if (!mbar_wait(&misc->x_ready, nxr & 1, abortp, status)) break;
+          CF_WAIT(&misc->x_ready, nxr & 1);
           tcgen05_fence_after();
-          issue_logits(dW1, 0);
-          if (!mbar_wait(&misc->lg_free, nlg & 1, abortp, status)) break;
+          issue_logits(w1l, 0);
+          CF_WAIT(&misc->lg_free, nlg & 1);
           nlg++;
           tcgen05_fence_after();
-          issue_logits(dW1, 1);
-          mma_commit(&misc->x_free);
+          issue_logits(w1l, 1);
+          if (elect_one()) mma_commit(&misc->x_free);
+          __syncwarp();
           nxr++;
-          // state update T_h += phi(K)_h^T [V | 1] (both feature halves were written before the query logits left)
-          if (!mbar_wait(&misc->v_full, it & 1, abortp, status)) break;
-          if (!mbar_wait(&misc->phik_full[0], it & 1, abortp, status)) break;
-          if (!mbar_wait(&misc->phik_full[1], it & 1, abortp, status)) break;
+          // state update T_h += phi(K)_h^T [V | 1], once the epilogue has taken its bf16 copy of the state BEFORE this
+          // tile (it does so between the two halves of the query logits); runs while it takes the row maxima
+          CF_WAIT(&misc->v_full, it & 1);
+          CF_WAIT(&misc->phik_full[0], it & 1);
+          CF_WAIT(&misc->phik_full[1], it & 1);
+          CF_WAIT(&misc->p_full, it & 1);
           tcgen05_fence_after();
-#pragma unroll 1
-          for (int hh = 0; hh < 2; hh++) {
+          if (elect_one()) {
 #pragma unroll
-            for (int k = 0; k < TILE / 16; k++)
-              mma_bf16(tmem + CF_T + hh * TC_NV, desc_advance(dPhiMN, hh * 2 * CfSmem::BLK + k * 2048), desc_advance(dV1, k * 2048),
-                       ID_STATE, 1u);
-          }
-          mma_commit(&misc->st_ready);
-          // scores and inter-tile output, 64 features (four K steps) at a time
-          if (!mbar_wait(&misc->p_full, it & 1, abortp, status)) break;
-          if (it > 0 && !mbar_wait(&misc->o_free, (it - 1) & 1, abortp, status)) break;
-          bool ok2 = true;
-#pragma unroll 1
-          for (int pr = 0; pr < 2; pr++) {
-            if (!mbar_wait(&misc->phiq_full[pr], it & 1, abortp, status)) { ok2 = false; break; }
-            tcgen05_fence_after();
-#pragma unroll
-            for (int j = 0; j < 8; j++) {
-              const int fb = 2 * pr + (j >> 2), k = j & 3;
-              mma_bf16_ta(tmem + CF_S, tmem + CF_L + fb * 32 + k * 8, desc_advance(dKP, fb * CfSmem::BLK + 32 * k), ID_SO,
-                          (pr | j) ? 1u : 0u);
+            for (int j = 0; j < 2 * (TILE / 16); j++) {
+              const int hh = j >> 3, k = j & 7;
+              mma_bf16_lh(tmem + CF_T + hh * TC_NV, pml + hh * 2 * (CfSmem::BLK / 16) + k * 128, pmh, v1l + k * 128, v1h, ID_STATE, 1u);
             }
+            mma_commit(&misc->st_ready);
+          }
+          __syncwarp();
+          // scores and inter-tile output, 32 features (two K steps) of two blocks at a time
+          if (it > 0) CF_WAIT(&misc->o_free, (it - 1) & 1);
+          bool ok2 = true;
+#pragma unroll
+          for (int qt = 0; qt < 5; qt++) {
+            // hand-over qt < 3: features 32 (qt % 2) .. + 32 of the blocks 2 (qt / 2), 2 (qt / 2) + 1 (two K steps each);
+            // the last 32 features come in two hand-overs of one K step, so that little is left when the exponentials end
+            if (!__all_sync(0xffffffffu, mbar_wait(&misc->phiq_full[qt], it & 1, abortp, status))) { ok2 = false; break; }
+            tcgen05_fence_after();
+            if (elect_one()) {
+#pragma unroll
+              for (int j = 0; j < (qt < 3 ? 4 : 2); j++) {
+                const int fb = qt < 3 ? 2 * (qt >> 1) + (j >> 1) : 2 + j;
+                const int k = qt < 3 ? 2 * (qt & 1) + (j & 1) : qt - 1;
+                mma_bf16_ta_lh(tmem + CF_S, tmem + CF_L + fb * 32 + k * 8, kpl + fb * (CfSmem::BLK / 16) + 2 * k, kph, ID_SO,
+                               (qt | j) ? 1u : 0u);
+              }
+              if (qt == 4) mma_commit(&misc->s_ready);
+            }
+            __syncwarp();
           }
           if (!ok2) break;
-          mma_commit(&misc->s_ready);
           // the next tile's first key logits go ahead of the masked-score product: they only need the columns that
           // the MMAs above have finished reading by the time they run (the pipe keeps issue order)
-          if (!mbar_wait(&misc->lg_free, nlg & 1, abortp, status)) break;      // (long since: the query logits were taken)
+          CF_WAIT(&misc->lg_free, nlg & 1);      // (long since: the query logits were taken)
           nlg++;
           if (it + 1 < ntiles) {
-            if (!mbar_wait(&misc->x_ready, nxr & 1, abortp, status)) break;
+            CF_WAIT(&misc->x_ready, nxr & 1);
             tcgen05_fence_after();
-            issue_logits(dW2, 0);
+            issue_logits(w2l, 0);
           }
-          if (!mbar_wait(&misc->sm_full, it & 1, abortp, status)) break;
+          CF_WAIT(&misc->sm_full, it & 1);
           tcgen05_fence_after();
+          if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < TILE / 16; k++)
-            mma_bf16_ta(tmem + CF_O, tmem + CF_S + k * 8, desc_advance(dV1, k * 2048), ID_SV, 1u);
-          mma_commit(&misc->o_ready);
-          mma_commit(&misc->v_free);
+            for (int k = 0; k < TILE / 16; k++)
+              mma_bf16_ta_lh(tmem + CF_O, tmem + CF_S + k * 8, v1l + k * 128, v1h, ID_SV, 1u);
+            mma_commit(&misc->o_ready);
+            mma_commit(&misc->v_free);
+          }
+          __syncwarp();
         }
+#undef CF_WAIT
       }
     } else {
       // ---------------- bf16 -> fp16 of the token tile, in place (16-byte pieces keep their swizzled positions)
-      const int t = (warp - WARP_CVT0) * 32 + lane;
+      const int t = (warp - CF_WARP_CVT0) * 32 + lane;
       for (int n = 0; n < 2 * ntiles; n++) {
         if (!mbar_wait(&misc->x_full, n & 1, abortp, status, false)) break;
         uint4* xt = reinterpret_cast<uint4*>(sm + CfSmem::X);
@@ -292,14 +323,20 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     // ---------------- epilogue warps.  As a token's thread: row = 32 q + lane, feature blocks hf and 2 + hf (64
     // features each; block hf comes out of the first logits half, block 2 + hf out of the second).  As a
     // feature's thread (state, bf16(T)): feature m = 128 hf + row, lane `row` of accumulator hf.
-    const int q = warp & 3, hf = warp >> 2;
+    const int q = warp & 3, hf = (warp - CF_PRODUCER_WARPS) >> 2;
     const int row = q * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
     const int m = hf * 128 + row;
     __nv_bfloat16* Yb = Y + b * ay.sb + h * ay.sh;
     uint8_t* blk0 = sm + CfSmem::KP + hf * CfSmem::BLK;              // phi(K) block hf
     uint8_t* blk1 = sm + CfSmem::KP + (2 + hf) * CfSmem::BLK;        // phi(K) block 2 + hf
-    uint8_t* pcol = sm + CfSmem::KP + (m >> 6) * CfSmem::BLK + TILE_BYTES;   // bf16(T), block of feature m
+    // bf16(T): column m of T is column m % 64 of the 80-row block of feature block m / 64; row n of a 128-byte-swizzled
+    // block keeps its 16-byte piece p at position p ^ (n % 8): one base address per value of n % 8
+    uint32_t pcol[8];
+#pragma unroll
+    for (int k = 0; k < 8; k++)
+      pcol[k] = smem_u32(sm + CfSmem::KP + (m >> 6) * CfSmem::BLK + TILE_BYTES) + (((((uint32_t)m & 63u) >> 3) ^ (uint32_t)k) << 4) +
+                (((uint32_t)m & 7u) << 1);
     float s = -INFINITY;                                              // the keys' running shift
     bool alive = true;
     int npair = 0, nall = 0;
@@ -314,30 +351,20 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       if (!mbar_wait(&misc->all_bar, nall & 1, abortp, status, false)) alive = false;
       nall++;
     };
-    // ---- the state before this segment: sum of the earlier segments' totals (their own shifts, without the
-    // per-feature term) brought to one shift, with this side's share a2 / 2 of the per-feature term
+    // ---- the state before this segment: sum of the earlier segments' totals, brought to one shift
     {
       const int np = seg == 0 ? 0 : min(nsplit1, seg);               // key-side splits are segments
       float val[TC_NV];
 #pragma unroll
       for (int n = 0; n < TC_NV; n++) val[n] = 0.f;
       if (np > 0) {
-        const float a2h = fa2[m];
-        float wmx = a2h;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) wmx = fmaxf(wmx, __shfl_xor_sync(0xffffffffu, wmx, o));
-        if (lane == 0) misc->red[warp] = wmx;
-        sync_all();
-        float a2max = misc->red[0];
-#pragma unroll
-        for (int i = 1; i < EPI_THREADS / 32; i++) a2max = fmaxf(a2max, misc->red[i]);
         const float* sh = shifts + (size_t)bh * nsplit1 * 2;
         float smax = -INFINITY;
         for (int p = 0; p < 2 * np; p++) smax = fmaxf(smax, sh[p]);
-        s = smax + a2max;
+        s = smax;
         const float* base = partial + (size_t)bh * nsplit1 * TC_NV * TC_M + m;
         for (int p = 0; p < np; p++) {
-          const float f = exp2f(sh[2 * p + hf] + a2h - s);
+          const float f = exp2f(sh[2 * p + hf] - s);
           const float* bp = base + (size_t)p * TC_NV * TC_M;
 #pragma unroll
           for (int n = 0; n <= TC_DV; n++) val[n] = fmaf(bp[n * TC_M], f, val[n]);
@@ -424,27 +451,22 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       tcgen05_fence_before();
       mbar_arrive_warp(&misc->lg_free, lane);
       const bool valid = (tile0 + it) * TILE + row < L;
-      // ---- exact maximum of the tile's exponents (with the per-feature share), one value for the block
+      // ---- exact maximum of the tile's exponents, one value for the block
       float tm;
       {
         float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int i = 0; i < 128; i += 4) {
-          const float4 a4 = *reinterpret_cast<const float4*>(fa2 + (i >> 6) * 128 + hf * 64 + (i & 63));
-          v[i] = __float_as_uint(__uint_as_float(v[i]) + a4.x);
-          v[i + 1] = __float_as_uint(__uint_as_float(v[i + 1]) + a4.y);
-          v[i + 2] = __float_as_uint(__uint_as_float(v[i + 2]) + a4.z);
-          v[i + 3] = __float_as_uint(__uint_as_float(v[i + 3]) + a4.w);
-          mxp[0] = fmaxf(mxp[0], __uint_as_float(v[i]));
-          mxp[1] = fmaxf(mxp[1], __uint_as_float(v[i + 1]));
-          mxp[2] = fmaxf(mxp[2], __uint_as_float(v[i + 2]));
-          mxp[3] = fmaxf(mxp[3], __uint_as_float(v[i + 3]));
+        for (int i = 0; i < 128; i += 8) {
+          mxp[0] = max3(mxp[0], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+          mxp[1] = max3(mxp[1], __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+          mxp[2] = max3(mxp[2], __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+          mxp[3] = max3(mxp[3], __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
         }
         float mx = valid ? fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])) + cj : -INFINITY;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         if (lane == 0) atomicMax(&misc->chunk_max[it % 3], f2ord(mx));
-        if (threadIdx.x == 0) misc->chunk_max[(it + 1) % 3] = f2ord(-INFINITY);   // next tile's slot; idle since tile it - 2
+        if (threadIdx.x == CF_PRODUCER_WARPS * 32) misc->chunk_max[(it + 1) % 3] = f2ord(-INFINITY);   // next tile's slot; idle since tile it - 2
         sync_all();
         if (!alive) break;
         tm = ord2f(misc->chunk_max[it % 3]);
@@ -470,7 +492,48 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         tcgen05_fence_before();
         s = tm;
       }
-      // ---- bf16(T) of the state before this tile: row `row` of accumulator hf = column m of T.  The previous
+      // ---- phi(K): 2^(exponent - s), bf16, 64 features at a time
+      {
+        const float rc = cj - s;
+#pragma unroll
+        for (int half = 0; half < 2; half++) {
+          uint8_t* prow = (half ? blk1 : blk0) + row * 128;
+#pragma unroll
+          for (int c = 0; c < 8; c++) {
+            uint32_t p[4];
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+              uint32_t& e0 = v[half * 64 + c * 8 + 2 * j];
+              uint32_t& e1 = v[half * 64 + c * 8 + 2 * j + 1];
+              add2(e0, e1, rc, rc);
+              if (j < CF_POLY_PAIRS) {
+                exp2_poly2(e0, e1);
+                p[j] = pack_bf16(__uint_as_float(e0), __uint_as_float(e1));
+              } else {
+                p[j] = pack_bf16(ex2(__uint_as_float(e0)), ex2(__uint_as_float(e1)));
+              }
+            }
+            if (!valid) p[0] = p[1] = p[2] = p[3] = 0u;
+            *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
+          }
+          fence_proxy_async_smem();
+          mbar_arrive_warp(&misc->phik_full[half], lane);
+          if (*abortp) { alive = false; goto after_keys; }
+        }
+      }
+    after_keys:
+      if (!alive) break;
+      // ---- query logits
+      if (!mbar_wait(&misc->lg_full, nlg & 1, abortp, status, false)) { alive = false; break; }
+      nlg++;
+      __syncwarp();
+      tcgen05_fence_after();
+#pragma unroll
+      for (int c = 0; c < 4; c++) tmem_ld16(lane_addr + CF_L + hf * 64 + c * 16, reinterpret_cast<uint32_t(&)[16]>(v[c * 16]));
+      tmem_wait_ld();
+      tcgen05_fence_before();
+      mbar_arrive_warp(&misc->lg_free, lane);
+      // ---- while the second half of the query logits is computed: bf16(T) of the state before this tile: row `row` of accumulator hf = column m of T.  The previous
       // tile's MMAs that read the old copy have completed (its scores were taken out of tensor memory).
       {
         __syncwarp();
@@ -482,42 +545,15 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           tmem_wait_ld();
 #pragma unroll
           for (int j = 0; j < 16; j++)
-            if (c * 16 + j <= TC_DV)
-              *reinterpret_cast<__nv_bfloat16*>(pcol + sw128_offset(c * 16 + j, m & 63)) = __float2bfloat16_rn(__uint_as_float(a[j]));
+            if (c * 16 + j <= TC_DV) {
+              const uint16_t hb = __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(a[j])));
+              asm volatile("st.shared.u16 [%0], %1;" ::"r"(pcol[j & 7] + (uint32_t)(c * 16 + j) * 128u), "h"(hb) : "memory");
+            }
         }
         tcgen05_fence_before();
         fence_proxy_async_smem();
         mbar_arrive_warp(&misc->p_full, lane);
       }
-      // ---- phi(K): 2^(exponent - s), bf16, 64 features at a time
-      {
-        const float rc = cj - s;
-#pragma unroll
-        for (int half = 0; half < 2; half++) {
-          uint8_t* prow = (half ? blk1 : blk0) + row * 128;
-#pragma unroll
-          for (int c = 0; c < 8; c++) {
-            uint32_t p[4];
-#pragma unroll
-            for (int j = 0; j < 4; j++)
-              p[j] = pack_bf16(ex2(__uint_as_float(v[half * 64 + c * 8 + 2 * j]) + rc), ex2(__uint_as_float(v[half * 64 + c * 8 + 2 * j + 1]) + rc));
-            if (!valid) p[0] = p[1] = p[2] = p[3] = 0u;
-            *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
-          }
-          fence_proxy_async_smem();
-          mbar_arrive_warp(&misc->phik_full[half], lane);
-        }
-      }
-      // ---- query logits
-      if (!mbar_wait(&misc->lg_full, nlg & 1, abortp, status, false)) { alive = false; break; }
-      nlg++;
-      __syncwarp();
-      tcgen05_fence_after();
-#pragma unroll
-      for (int c = 0; c < 4; c++) tmem_ld16(lane_addr + CF_L + hf * 64 + c * 16, reinterpret_cast<uint32_t(&)[16]>(v[c * 16]));
-      tmem_wait_ld();
-      tcgen05_fence_before();
-      mbar_arrive_warp(&misc->lg_free, lane);
       if (!mbar_wait(&misc->lg_full, nlg & 1, abortp, status, false)) { alive = false; break; }
       nlg++;
       __syncwarp();
@@ -533,14 +569,10 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
         for (int i = 0; i < 128; i += 4) {
           const float4 a4 = *reinterpret_cast<const float4*>(fa2 + (i >> 6) * 128 + hf * 64 + (i & 63));
-          v[i] = __float_as_uint(__uint_as_float(v[i]) + a4.x);
-          v[i + 1] = __float_as_uint(__uint_as_float(v[i + 1]) + a4.y);
-          v[i + 2] = __float_as_uint(__uint_as_float(v[i + 2]) + a4.z);
-          v[i + 3] = __float_as_uint(__uint_as_float(v[i + 3]) + a4.w);
-          mxp[0] = fmaxf(mxp[0], __uint_as_float(v[i]));
-          mxp[1] = fmaxf(mxp[1], __uint_as_float(v[i + 1]));
-          mxp[2] = fmaxf(mxp[2], __uint_as_float(v[i + 2]));
-          mxp[3] = fmaxf(mxp[3], __uint_as_float(v[i + 3]));
+          add2(v[i], v[i + 1], a4.x, a4.y);
+          add2(v[i + 2], v[i + 3], a4.z, a4.w);
+          mxp[(i >> 2) & 1] = max3(mxp[(i >> 2) & 1], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+          mxp[2 + ((i >> 2) & 1)] = max3(mxp[2 + ((i >> 2) & 1)], __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
         }
         mx = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
         // the row's other thread sits in warp q of the other warpgroup; after this barrier both have also taken
@@ -558,14 +590,45 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         for (int c = 0; c < 2; c++) {
           uint32_t p[16];
 #pragma unroll
-          for (int j = 0; j < 16; j++)
-            p[j] = pack_bf16(ex2(__uint_as_float(v[half * 64 + c * 32 + 2 * j]) - mx), ex2(__uint_as_float(v[half * 64 + c * 32 + 2 * j + 1]) - mx));
-          tmem_st16(lane_addr + CF_L + fb * 32 + c * 16, p);
+          for (int j = 0; j < 16; j++) {
+            uint32_t& e0 = v[half * 64 + c * 32 + 2 * j];
+            uint32_t& e1 = v[half * 64 + c * 32 + 2 * j + 1];
+            add2(e0, e1, -mx, -mx);
+            if ((j & 3) < CF_POLY_PAIRS) {
+              exp2_poly2(e0, e1);
+              p[j] = pack_bf16(__uint_as_float(e0), __uint_as_float(e1));
+            } else {
+              p[j] = pack_bf16(ex2(__uint_as_float(e0)), ex2(__uint_as_float(e1)));
+            }
+          }
+          if (half == 1 && c == 1) {
+            // columns of K step 2, then of K step 3
+            uint32_t lo8[8], hi8[8];
+#pragma unroll
+            for (int j = 0; j < 8; j++) { lo8[j] = p[j]; hi8[j] = p[8 + j]; }
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(lane_addr + CF_L + fb * 32 + 16),
+                         "r"(lo8[0]), "r"(lo8[1]), "r"(lo8[2]), "r"(lo8[3]), "r"(lo8[4]), "r"(lo8[5]), "r"(lo8[6]), "r"(lo8[7]) : "memory");
+            tmem_wait_st();
+            tcgen05_fence_before();
+            mbar_arrive_warp(&misc->phiq_full[3], lane);
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(lane_addr + CF_L + fb * 32 + 24),
+                         "r"(hi8[0]), "r"(hi8[1]), "r"(hi8[2]), "r"(hi8[3]), "r"(hi8[4]), "r"(hi8[5]), "r"(hi8[6]), "r"(hi8[7]) : "memory");
+            tmem_wait_st();
+            tcgen05_fence_before();
+            mbar_arrive_warp(&misc->phiq_full[4], lane);
+          } else {
+            tmem_st16(lane_addr + CF_L + fb * 32 + c * 16, p);
+            tmem_wait_st();
+            tcgen05_fence_before();
+            mbar_arrive_warp(&misc->phiq_full[2 * half + c], lane);
+          }
+          // A real branch after every hand-over: without one the instruction scheduler moves the (side-effect-free)
+          // exponentials of the chunks that follow ahead of the hand-over, and all hand-overs bunch at the end.
+          if (*abortp) { alive = false; goto after_queries; }
         }
-        tmem_wait_st();
-        tcgen05_fence_before();
-        mbar_arrive_warp(&misc->phiq_full[half], lane);
       }
+    after_queries:
+      if (!alive) break;
       // ---- scores: mask (key <= query), round to bf16 over their own columns, keep the row sums
       if (!mbar_wait(&misc->s_ready, it & 1, abortp, status, false)) { alive = false; break; }
       __syncwarp();
@@ -606,7 +669,7 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   }
   tcgen05_fence_before();
   __syncthreads();
-  if (warp == WARP_MMA) {
+  if (warp == CF_WARP_MMA) {
     tcgen05_fence_after();
     tmem_dealloc(tmem, TMEM_COLS);
   }

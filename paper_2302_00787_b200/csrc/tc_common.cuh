@@ -214,6 +214,34 @@ __device__ __forceinline__ void mma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, ui
       "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The same two with the descriptors given as (low word + byte offset / 16, high word): the 64-bit values are put
+// together next to the instruction, so a long unrolled schedule keeps one base per operand alive, not one
+// descriptor per MMA.
+__device__ __forceinline__ void mma_bf16_lh(uint32_t d_tmem, uint32_t alo, uint32_t ahi, uint32_t blo, uint32_t bhi, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\tmov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+      "r"(alo), "r"(ahi), "r"(blo), "r"(bhi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_bf16_ta_lh(uint32_t d_tmem, uint32_t a_tmem, uint32_t blo, uint32_t bhi, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\tmov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "r"(blo), "r"(bhi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// The same for sixteen registers: arithmetic on them that follows in the source stays behind this point (the
+// compiler would otherwise move side-effect-free work, e.g. the exponentials of a later chunk, ahead of an
+// earlier chunk's hand-over).
+__device__ __forceinline__ void pin16(uint32_t* r) {
+  asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+               "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]));
+}
+// Keeps the compiler from moving arithmetic on `x` across this point (e.g. out of a loop).
+__device__ __forceinline__ void opaque(uint32_t& x) { asm volatile("" : "+r"(x)); }
 // All MMAs issued so far by this thread arrive on the mbarrier when they have completed.
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -224,6 +252,46 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+// (a, b) += (c, d) as one packed fp32 instruction
+__device__ __forceinline__ void add2(uint32_t& a, uint32_t& b, float c, float d) {
+  asm("{\n\t.reg .b64 x, y;\n\tmov.b64 x, {%0, %1};\n\tmov.b64 y, {%2, %3};\n\tadd.rn.f32x2 x, x, y;\n\tmov.b64 {%0, %1}, x;\n\t}"
+      : "+r"(a), "+r"(b)
+      : "f"(c), "f"(d));
+}
+// (2^a, 2^b) on the multiply-add pipe, leaving the special-function unit to ex2(): with n = floor(x) and
+// f = x - n in [0, 1), 2^x = 2^n p(f), p the cubic of exp2_poly_fit.py (largest relative error 8.6e-5, far below
+// the rounding of a bf16 feature).  x + 1.5 * 2^23 rounded down holds n in its low mantissa bits, which are
+// shifted into the exponent field of p(f).  Arguments below -125 give 2^-125.
+__device__ __forceinline__ void exp2_poly2(uint32_t& a, uint32_t& b) {
+  const float x0 = fmaxf(__uint_as_float(a), -125.f), x1 = fmaxf(__uint_as_float(b), -125.f);
+  uint32_t r0, r1, p0, p1;
+  asm("{\n\t.reg .b64 x, r, n, f, p, c;\n\t"
+      "mov.b64 x, {%4, %5};\n\t"
+      "mov.b64 c, {0x4B400000, 0x4B400000};\n\t"          // 1.5 * 2^23
+      "add.rm.f32x2 r, x, c;\n\t"
+      "mov.b64 c, {0xCB400000, 0xCB400000};\n\t"
+      "add.rn.f32x2 n, r, c;\n\t"                          // n = floor(x), exact
+      "mov.b64 c, {0xBF800000, 0xBF800000};\n\t"
+      "fma.rn.f32x2 f, n, c, x;\n\t"                       // f = x - n
+      "mov.b64 c, {0x3D9DD553, 0x3D9DD553};\n\t"          // c3 = 0.07706704
+      "mov.b64 p, {0x3E691BC5, 0x3E691BC5};\n\t"          // c2 = 0.22764499
+      "fma.rn.f32x2 p, f, c, p;\n\t"
+      "mov.b64 c, {0x3F31F32C, 0x3F31F32C};\n\t"          // c1 = 0.69511676
+      "fma.rn.f32x2 p, p, f, c;\n\t"
+      "mov.b64 c, {0x3F800000, 0x3F800000};\n\t"
+      "fma.rn.f32x2 p, p, f, c;\n\t"
+      "mov.b64 {%0, %1}, r;\n\t"
+      "mov.b64 {%2, %3}, p;\n\t}"
+      : "=r"(r0), "=r"(r1), "=r"(p0), "=r"(p1)
+      : "f"(x0), "f"(x1));
+  a = p0 + (r0 << 23);
+  b = p1 + (r1 << 23);
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
