@@ -50,9 +50,12 @@ struct CfSmem {
   // KP: four blocks of 64 features, each [phi(K) 128 keys x 64 | bf16(T) 80 rows x 64], so that one K-major
   // operand of 208 rows covers both
   static constexpr uint32_t W1 = 0, W2 = IMG_W_BYTES, X = 2 * IMG_W_BYTES, V = X + TILE_BYTES, ONES = V + TILE_BYTES,
-                            KP = ONES + TILE_BYTES, BLK = TILE_BYTES + KVT_BLOCK_BYTES, ROWMAX = KP + 4 * BLK,
-                            RSUM = ROWMAX + 2 * TILE * 4, FA2 = RSUM + 2 * TILE * 4, MISC = FA2 + TC_M * 4,
-                            TOTAL = MISC + 256;
+                            KP = ONES + TILE_BYTES, BLK = TILE_BYTES + KVT_BLOCK_BYTES,
+                            // the row maxima of the query logits and the row sums of the masked scores are never alive together
+                            ROWMAX = KP + 4 * BLK, RSUM = ROWMAX,
+                            // per-feature term as an MMA operand: [256 features x 16] fp16, no swizzle (8 x 16-byte core
+                            // matrices: the two 16-byte K pieces of a row 128 bytes apart, 8-row groups 256 bytes apart)
+                            A2OP = ROWMAX + 2 * TILE * 4, A2OP_BYTES = TC_M * 32, MISC = A2OP + A2OP_BYTES, TOTAL = MISC + 256;
 };
 static_assert(CfSmem::KP % 1024 == 0 && CfSmem::BLK % 1024 == 0 && CfSmem::X % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 static_assert(CfSmem::TOTAL + 1024 <= 232448, "shared memory budget");
@@ -69,8 +72,8 @@ struct CfMisc {
 };
 static_assert(sizeof(CfMisc) <= 256, "misc block");
 
-// tensor memory columns
-constexpr uint32_t CF_L = 0, CF_S = 128, CF_O = 256, CF_T = 336;
+// tensor memory columns; CF_ONE: an A operand of one K step whose first two K elements are 1 (fp16) in every row
+constexpr uint32_t CF_L = 0, CF_S = 128, CF_O = 256, CF_T = 336, CF_ONE = 496;
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -83,7 +86,6 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   CfMisc* misc = reinterpret_cast<CfMisc*>(sm + CfSmem::MISC);
   float* rowmax = reinterpret_cast<float*>(sm + CfSmem::ROWMAX);   // [half][row]
   float* rsum = reinterpret_cast<float*>(sm + CfSmem::RSUM);       // [half][row]: row sums of the rounded masked scores
-  float* fa2 = reinterpret_cast<float*>(sm + CfSmem::FA2);         // the per-feature term a2 of both sides: it joins the query logits
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int seg = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
   const int g = pool == FSHARP_POOL_PER_BH ? bh : h;
@@ -124,7 +126,15 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   for (int i = threadIdx.x; i < 4 * (int)(KVT_BLOCK_BYTES / 16); i += TC_THREADS)
     reinterpret_cast<uint4*>(sm + CfSmem::KP + (i / (KVT_BLOCK_BYTES / 16)) * CfSmem::BLK + TILE_BYTES)[i % (KVT_BLOCK_BYTES / 16)] =
         make_uint4(0, 0, 0, 0);
-  if (threadIdx.x < TC_M) fa2[threadIdx.x] = reinterpret_cast<const float*>(img1 + IMG_A2)[threadIdx.x];
+  // The per-feature term a2 = 2 log2e w^T A w of both sides joins the query logits inside their MMA: one more K step
+  // whose A operand is [1, 1, 0, ...] in every row and whose B operand holds a2 as an fp16 value and its fp16 remainder.
+  if (threadIdx.x < TC_M) {
+    const float a2 = reinterpret_cast<const float*>(img1 + IMG_A2)[threadIdx.x];
+    const __half hi = __float2half_rn(a2), lo = __float2half_rn(a2 - __half2float(hi));
+    uint8_t* rowp = sm + CfSmem::A2OP + (threadIdx.x >> 3) * 256 + (threadIdx.x & 7) * 16;
+    *reinterpret_cast<uint4*>(rowp) = make_uint4((uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16), 0, 0, 0);
+    *reinterpret_cast<uint4*>(rowp + 128) = make_uint4(0, 0, 0, 0);
+  }
   __syncthreads();
   if (threadIdx.x < TILE)
     *reinterpret_cast<__nv_bfloat16*>(sm + CfSmem::ONES + sw128_offset(threadIdx.x, 0)) = __float2bfloat16(1.f);
@@ -197,11 +207,15 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         uint32_t xl = (uint32_t)dX, w1l = (uint32_t)dW1, w2l = (uint32_t)dW2, kpl = (uint32_t)dKP, pml = (uint32_t)dPhiMN, v1l = (uint32_t)dV1;
         const uint32_t xh = (uint32_t)(dX >> 32), wh = (uint32_t)(dW1 >> 32), kph = (uint32_t)(dKP >> 32), pmh = (uint32_t)(dPhiMN >> 32),
                        v1h = (uint32_t)(dV1 >> 32);
-        auto issue_logits = [&](uint32_t wl, int half) {
+        const uint64_t dA2 = smem_desc(smem_u32(sm + CfSmem::A2OP), 128, 256, SWZ_NONE);
+        uint32_t a2l = (uint32_t)dA2;
+        const uint32_t a2h = (uint32_t)(dA2 >> 32);
+        auto issue_logits = [&](uint32_t wl, int half, bool with_a2) {
           if (elect_one()) {
 #pragma unroll
             for (int k = 0; k < TC_D / 16; k++)
               mma_bf16_lh(tmem + CF_L, xl + 2 * k, xh, wl + half * (IMG_W_BYTES / 32) + 2 * k, wh, ID_LOGITS, k > 0);
+            if (with_a2) mma_bf16_ta_lh(tmem + CF_L, tmem + CF_ONE, a2l + half * (128 * 32 / 16), a2h, ID_LOGITS, 1u);
             mma_commit(&misc->lg_full);
           }
           __syncwarp();
@@ -212,17 +226,17 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         ok = __all_sync(0xffffffffu, ok);
         if (ok) {
           tcgen05_fence_after();
-          issue_logits(w2l, 0);
+          issue_logits(w2l, 0, false);
         }
         // a wait that gave up in one lane ends the schedule for the whole warp
 #define CF_WAIT(bar, par) if (!__all_sync(0xffffffffu, mbar_wait((bar), (par), abortp, status))) break
         for (int it = 0; ok && it < ntiles; it++) {
-          opaque(xl); opaque(w1l); opaque(w2l); opaque(kpl); opaque(pml); opaque(v1l);
+          opaque(a2l); opaque(xl); opaque(w1l); opaque(w2l); opaque(kpl); opaque(pml); opaque(v1l);
           // second half of the key logits once the epilogue has taken the first out of tensor memory
           CF_WAIT(&misc->lg_free, nlg & 1);
           nlg++;
           tcgen05_fence_after();
-          issue_logits(w2l, 1);
+          issue_logits(w2l, 1, false);
           if (elect_one()) mma_commit(&misc->x_free);
           __syncwarp();
           nxr++;
@@ -231,11 +245,11 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           nlg++;
           CF_WAIT(&misc->x_ready, nxr & 1);
           tcgen05_fence_after();
-          issue_logits(w1l, 0);
+          issue_logits(w1l, 0, true);
           CF_WAIT(&misc->lg_free, nlg & 1);
           nlg++;
           tcgen05_fence_after();
-          issue_logits(w1l, 1);
+          issue_logits(w1l, 1, true);
           if (elect_one()) mma_commit(&misc->x_free);
           __syncwarp();
           nxr++;
@@ -284,7 +298,7 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           if (it + 1 < ntiles) {
             CF_WAIT(&misc->x_ready, nxr & 1);
             tcgen05_fence_after();
-            issue_logits(w2l, 0);
+            issue_logits(w2l, 0, false);
           }
           CF_WAIT(&misc->sm_full, it & 1);
           tcgen05_fence_after();
@@ -376,6 +390,10 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
         for (int j = 0; j < 16; j++) a[j] = __float_as_uint(val[c * 16 + j]);
         tmem_st16(lane_addr + CF_T + hf * TC_NV + c * 16, a);
+      }
+      if (hf == 0) {
+        asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %2, %2, %2, %2, %2, %2};" ::"r"(lane_addr + CF_ONE),
+                     "r"(0x3C003C00u), "r"(0u) : "memory");
       }
       tmem_wait_st();
       tcgen05_fence_before();
@@ -567,12 +585,11 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       {
         float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int i = 0; i < 128; i += 4) {
-          const float4 a4 = *reinterpret_cast<const float4*>(fa2 + (i >> 6) * 128 + hf * 64 + (i & 63));
-          add2(v[i], v[i + 1], a4.x, a4.y);
-          add2(v[i + 2], v[i + 3], a4.z, a4.w);
-          mxp[(i >> 2) & 1] = max3(mxp[(i >> 2) & 1], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
-          mxp[2 + ((i >> 2) & 1)] = max3(mxp[2 + ((i >> 2) & 1)], __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+        for (int i = 0; i < 128; i += 8) {
+          mxp[0] = max3(mxp[0], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+          mxp[1] = max3(mxp[1], __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+          mxp[2] = max3(mxp[2], __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+          mxp[3] = max3(mxp[3], __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
         }
         mx = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
         // the row's other thread sits in warp q of the other warpgroup; after this barrier both have also taken
