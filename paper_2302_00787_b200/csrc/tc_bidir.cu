@@ -360,29 +360,39 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 // phi(Q) with this state in fp16, whose exponent range is narrow, and what a feature contributes to
 // an output is phi(Q)_m times the size of column m of the state.  So every column m is brought to
 // order one by a power of two 2^-e_m, and g_m = e_m + a2_m - max a2 (the per-feature term w^T A w
-// of both sides rides along) is added to the query logits BEFORE the row maximum is taken: a query
+// of both sides rides along) joins the query logits BEFORE the row maximum is taken: a query
 // feature near 1 is then one that matters, and what underflows in either operand is negligible by
-// construction.
-constexpr int OUT_STAGES = 2;
+// construction.  g joins the logits inside their MMA, as one more K step whose A operand is
+// [1, 1, 0, ...] in every row (tensor memory) and whose B operand holds g as an fp16 value and its
+// fp16 remainder.  The query tile is converted from bf16 to fp16 in shared memory (exact for |x| in
+// [2^-14, 65504]), so the logits need one fp16 image of W instead of a bf16 value and its remainder.
+constexpr int OUT_STAGES = 3;
+constexpr int WARP_OUT_MMA2 = WARP_MMA + 1, WARP_OUT_CVT = WARP_MMA + 2;
+// Of every four pairs of exponentials, this many run on the multiply-add pipe (exp2_poly2).
+constexpr int OUT_POLY_PAIRS = 1;
 struct OutSmem {
-  static constexpr uint32_t X0 = 0, W = OUT_STAGES * TILE_BYTES, WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES,
-                            KVT = PHI + 4 * TILE_BYTES, ROWMAX = KVT + KVT_BYTES,
-                            STAGE = ROWMAX + 3 * 2 * TILE * 4,          // 2 KB per epilogue warp: output rows on their way out
-                            GQ = STAGE + (EPI_THREADS / 32) * 2048,     // the merge's per-feature exponents g_m
-                            MISC = GQ + TC_M * 4, TOTAL = MISC + 256;
+  // PHI also serves the merge (shifts and their factors) and, 2 KB per epilogue warp inside the rows that warp
+  // itself writes next, the output rows on their way out
+  static constexpr uint32_t X0 = 0, WH = OUT_STAGES * TILE_BYTES, PHI = WH + IMG_W_BYTES, KVT = PHI + 4 * TILE_BYTES,
+                            ROWMAX = KVT + KVT_BYTES,
+                            // g as an MMA operand: [256 features x 16] fp16, no swizzle (the two 16-byte K pieces of a
+                            // row 128 bytes apart, 8-row groups 256 bytes apart)
+                            GOP = ROWMAX + 2 * 2 * TILE * 4, GOP_BYTES = TC_M * 32, MISC = GOP + GOP_BYTES, TOTAL = MISC + 256;
 };
-static_assert(OutSmem::PHI % 1024 == 0 && OutSmem::KVT % 1024 == 0 && OutSmem::W % 1024 == 0, "alignment");
+static_assert(OutSmem::PHI % 1024 == 0 && OutSmem::KVT % 1024 == 0 && OutSmem::WH % 1024 == 0, "alignment");
 static_assert(OutSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 
 struct OutMisc {
-  // phi_full[f]: the 64-feature block f of the phi tile is written (the 128 threads of its half arrive)
-  uint64_t full[OUT_STAGES], empty[OUT_STAGES], logits_full, logits_free, phi_full[TC_M / 64], phi_free, const_bar;
-
+  // full: the tile has landed; conv: it has been converted to fp16; phi_full[f]: the 64-feature block f of the phi
+  // tile is written (the four warps of its half arrive); g_ready: the merge has written its operands
+  uint64_t full[OUT_STAGES], conv[OUT_STAGES], empty[OUT_STAGES], logits_full, logits_free, phi_full[TC_M / 64], phi_free, const_bar,
+      g_ready;
   uint32_t tmem_base;
   int abort_flag;
 };
-// TMEM columns: logits, then [num | den]
-constexpr uint32_t OUT_COL_LOGITS = 0, OUT_COL_OUT = 256;
+static_assert(sizeof(OutMisc) <= 256, "misc block");
+// TMEM columns: logits, then [num | den], then the A operand of the g step
+constexpr uint32_t OUT_COL_LOGITS = 0, OUT_COL_OUT = 256, OUT_COL_ONE = 496;
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict__ images,
@@ -392,8 +402,7 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   OutMisc* misc = reinterpret_cast<OutMisc*>(sm + OutSmem::MISC);
-  float* rowmax = reinterpret_cast<float*>(sm + OutSmem::ROWMAX);   // [tile % 3][half][row]
-  float* gs = reinterpret_cast<float*>(sm + OutSmem::GQ);
+  float* rowmax = reinterpret_cast<float*>(sm + OutSmem::ROWMAX);   // [tile % 2][half][row]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
   const int g = pool == FSHARP_POOL_PER_BH ? bh : h;
@@ -404,12 +413,13 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
   volatile int* abortp = &misc->abort_flag;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < OUT_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], 1); }
+    for (int i = 0; i < OUT_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->conv[i], 1); mbar_init(&misc->empty[i], 1); }
     mbar_init(&misc->logits_full, 1);
     mbar_init(&misc->logits_free, EPI_THREADS / 32);
     for (int i = 0; i < TC_M / 64; i++) mbar_init(&misc->phi_full[i], EPI_THREADS / 64);
     mbar_init(&misc->phi_free, 1);
     mbar_init(&misc->const_bar, 1);
+    mbar_init(&misc->g_ready, EPI_THREADS / 32);
     misc->abort_flag = 0;
     fence_barrier_init();
   }
@@ -427,9 +437,8 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
   if (warp == WARP_TMA) {
     if (lane == 0) {
       prefetch_tmap(&tmQ);
-      mbar_expect_tx(&misc->const_bar, 2 * IMG_W_BYTES);
-      bulk_load(sm + OutSmem::W, img + IMG_W, IMG_W_BYTES, &misc->const_bar);
-      bulk_load(sm + OutSmem::WLO, img + IMG_WLO, IMG_W_BYTES, &misc->const_bar);
+      mbar_expect_tx(&misc->const_bar, IMG_W_BYTES);
+      bulk_load(sm + OutSmem::WH, img + IMG_WH, IMG_W_BYTES, &misc->const_bar);
       for (int it = 0; it < min(ntiles, PREFETCH_TILES); it++) tma_prefetch_4d(&tmQ, 0, (tile0 + it) * TILE, h, b);
       int issued = 0;
       for (int it = 0; it < ntiles; it++) {
@@ -444,66 +453,89 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
       for (int it = max(0, issued - OUT_STAGES); it < issued; it++)
         mbar_wait(&misc->full[it % OUT_STAGES], (it / OUT_STAGES) & 1, abortp, status, false);
     }
+  } else if (warp == WARP_OUT_CVT) {
+    // ---------------- bf16 -> fp16 of the query tile, in place (16-byte pieces keep their swizzled positions)
+    for (int it = 0; it < ntiles; it++) {
+      const int st = it % OUT_STAGES;
+      if (!mbar_wait(&misc->full[st], (it / OUT_STAGES) & 1, abortp, status, false)) break;
+      uint4* xt = reinterpret_cast<uint4*>(sm + OutSmem::X0 + st * TILE_BYTES);
+#pragma unroll 4
+      for (int i = 0; i < (int)(TILE_BYTES / 16) / 32; i++) {
+        uint4 u = xt[lane + i * 32];
+        u.x = pack_f16(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
+        u.y = pack_f16(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
+        u.z = pack_f16(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u));
+        u.w = pack_f16(__uint_as_float(u.w << 16), __uint_as_float(u.w & 0xffff0000u));
+        xt[lane + i * 32] = u;
+      }
+      fence_proxy_async_smem();
+      mbar_arrive_warp(&misc->conv[st], lane);
+    }
   } else if (warp == WARP_MMA) {
-    // ---------------- logits MMAs (the two warps after this one issue the contractions, a feature half each)
-    if (lane == 0) {
-      constexpr uint32_t ID_LOGITS = idesc_bf16(128, TC_M, 0, 0);
-      const uint64_t dX0 = smem_desc(smem_u32(sm + OutSmem::X0), 16, 1024, SWZ_128B);
-      const uint64_t dW = smem_desc(smem_u32(sm + OutSmem::W), 16, 1024, SWZ_128B);
-      const uint64_t dWlo = smem_desc(smem_u32(sm + OutSmem::WLO), 16, 1024, SWZ_128B);
-      auto issue_logits = [&](int st) {
-        const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
+    // ---------------- logits MMAs: the whole warp walks the schedule, one elected lane issues
+    constexpr uint32_t ID_LOGITS = idesc_f16(128, TC_M, 0, 0);
+    const uint64_t dX0 = smem_desc(smem_u32(sm + OutSmem::X0), 16, 1024, SWZ_128B);
+    const uint64_t dW = smem_desc(smem_u32(sm + OutSmem::WH), 16, 1024, SWZ_128B);
+    const uint64_t dG = smem_desc(smem_u32(sm + OutSmem::GOP), 128, 256, SWZ_NONE);
+    uint32_t xl = (uint32_t)dX0, wl = (uint32_t)dW, gl = (uint32_t)dG;
+    const uint32_t xh = (uint32_t)(dX0 >> 32), wh = (uint32_t)(dW >> 32), gh = (uint32_t)(dG >> 32);
+    auto issue_logits = [&](int st) {
+      if (elect_one()) {
 #pragma unroll
         for (int k = 0; k < TC_D / 16; k++)
-          mma_bf16(tmem + OUT_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dW, 32 * k), ID_LOGITS, k > 0);
-#pragma unroll
-        for (int k = 0; k < TC_D / 16; k++)
-          mma_bf16(tmem + OUT_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dWlo, 32 * k), ID_LOGITS, 1);
+          mma_bf16_lh(tmem + OUT_COL_LOGITS, xl + st * (TILE_BYTES / 16) + 2 * k, xh, wl + 2 * k, wh, ID_LOGITS, k > 0);
+        mma_bf16_ta_lh(tmem + OUT_COL_LOGITS, tmem + OUT_COL_ONE, gl, gh, ID_LOGITS, 1u);
         mma_commit(&misc->logits_full);
         mma_commit(&misc->empty[st]);
-      };
-      bool ok = mbar_wait(&misc->const_bar, 0, abortp, status);
-      if (ok && ntiles > 0) ok = mbar_wait(&misc->full[0], 0, abortp, status);
-      if (ok && ntiles > 0) {
-        tcgen05_fence_after();
-        issue_logits(0);
       }
-      for (int it = 0; ok && it + 1 < ntiles; it++) {
-        const int sn = (it + 1) % OUT_STAGES;
-        if (!mbar_wait(&misc->full[sn], ((it + 1) / OUT_STAGES) & 1, abortp, status)) break;
-        if (!mbar_wait(&misc->logits_free, it & 1, abortp, status)) break;
-        // The tensor pipe runs MMAs in the order they were issued: the last contraction steps of tile it - 1, which
-        // the epilogue is about to wait for, go before the next tile's logits, which nobody needs for a whole tile.
-        if (it > 0 && !mbar_wait(&misc->phi_free, (it - 1) & 1, abortp, status)) break;
-        tcgen05_fence_after();
-        issue_logits(sn);
+      __syncwarp();
+    };
+#define OUT_WAIT(bar, par) if (!__all_sync(0xffffffffu, mbar_wait((bar), (par), abortp, status))) break
+    for (int it = 0; it < ntiles; it++) {
+      const int st = it % OUT_STAGES;
+      opaque(xl); opaque(wl); opaque(gl);
+      if (it == 0) {
+        OUT_WAIT(&misc->const_bar, 0);
+        OUT_WAIT(&misc->g_ready, 0);
       }
+      OUT_WAIT(&misc->conv[st], (it / OUT_STAGES) & 1);
+      if (it > 0) OUT_WAIT(&misc->logits_free, (it - 1) & 1);
+      // The tensor pipe runs MMAs in the order they were issued: the last contraction steps of tile it - 2, which
+      // the epilogue is about to wait for, go before the next tile's logits, which nobody needs for a whole tile.
+      if (it > 1) OUT_WAIT(&misc->phi_free, (it - 2) & 1);
+      tcgen05_fence_after();
+      issue_logits(st);
     }
-  } else if (warp == WARP_MMA + 1) {
+#undef OUT_WAIT
+  } else if (warp == WARP_OUT_MMA2) {
     // ---------------- contraction: every 64-feature block of phi is contracted as soon as it is written, first
     // blocks of both halves first, so only the last block's MMAs are left when the exponentials end.  One
     // accumulator [num | den] for all 256 features (the two threads of a row agree on the row's shift).
-    if (lane == 0) {
-      constexpr uint32_t ID_OUT = idesc_f16(128, TC_NV, 0, 0);      // fp16: phi(Q) <= 1 and a state of order one per feature
-      const uint64_t dPhi = smem_desc(smem_u32(sm + OutSmem::PHI), 16, 1024, SWZ_128B);
-      const uint64_t dKvt = smem_desc(smem_u32(sm + OutSmem::KVT), 16, 1024, SWZ_128B);
-      bool ok = true;
-      for (int it = 0; ok && it < ntiles; it++) {
-        // An epilogue thread arrives on its half's first block only after it has read the previous tile's output
-        // row, so the accumulator may be overwritten once the first blocks of BOTH halves are in.
-        if (!mbar_wait(&misc->phi_full[0], it & 1, abortp, status)) break;
-        if (!mbar_wait(&misc->phi_full[2], it & 1, abortp, status)) break;
+    constexpr uint32_t ID_OUT = idesc_f16(128, TC_NV, 0, 0);      // fp16: phi(Q) <= 1 and a state of order one per feature
+    const uint64_t dPhi = smem_desc(smem_u32(sm + OutSmem::PHI), 16, 1024, SWZ_128B);
+    const uint64_t dKvt = smem_desc(smem_u32(sm + OutSmem::KVT), 16, 1024, SWZ_128B);
+    uint32_t pl = (uint32_t)dPhi, kl = (uint32_t)dKvt;
+    const uint32_t ph = (uint32_t)(dPhi >> 32), kh = (uint32_t)(dKvt >> 32);
+    bool ok = true;
+    for (int it = 0; ok && it < ntiles; it++) {
+      opaque(pl); opaque(kl);
+      // An epilogue thread arrives on its half's first block only after it has read the previous tile's output
+      // row, so the accumulator may be overwritten once the first blocks of BOTH halves are in.
+      if (!__all_sync(0xffffffffu, mbar_wait(&misc->phi_full[0], it & 1, abortp, status))) break;
+      if (!__all_sync(0xffffffffu, mbar_wait(&misc->phi_full[2], it & 1, abortp, status))) break;
 #pragma unroll
-        for (int o = 0; o < TC_M / 64; o++) {
-          const int fb = ((o & 1) << 1) | (o >> 1);      // 0, 2, 1, 3
-          if (o >= 2 && !mbar_wait(&misc->phi_full[fb], it & 1, abortp, status)) { ok = false; break; }
-          tcgen05_fence_after();
+      for (int o = 0; o < TC_M / 64; o++) {
+        const int fb = ((o & 1) << 1) | (o >> 1);      // 0, 2, 1, 3
+        if (o >= 2 && !__all_sync(0xffffffffu, mbar_wait(&misc->phi_full[fb], it & 1, abortp, status))) { ok = false; break; }
+        tcgen05_fence_after();
+        if (elect_one()) {
 #pragma unroll
           for (int k = 0; k < 4; k++)
-            mma_bf16(tmem + OUT_COL_OUT, desc_advance(dPhi, fb * TILE_BYTES + 32 * k),
-                     desc_advance(dKvt, fb * KVT_BLOCK_BYTES + 32 * k), ID_OUT, (o > 0 || k > 0) ? 1u : 0u);
+            mma_bf16_lh(tmem + OUT_COL_OUT, pl + fb * (TILE_BYTES / 16) + 2 * k, ph, kl + fb * (KVT_BLOCK_BYTES / 16) + 2 * k, kh, ID_OUT,
+                        (o > 0 || k > 0) ? 1u : 0u);
+          if (o == TC_M / 64 - 1) mma_commit(&misc->phi_free);
         }
-        if (ok) mma_commit(&misc->phi_free);
+        __syncwarp();
       }
     }
   }
@@ -522,7 +554,7 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
       // merge (see above); thread = feature m, whose half (m / 128) is also the thread's half below, so the
       // arrivals that release a 64-feature block to the MMA warp cover the writers of that block of the state
       const int m = threadIdx.x, hh = m >> 7;
-      float* sft = reinterpret_cast<float*>(sm + OutSmem::STAGE);        // shifts, then their factors (the stage is idle)
+      float* sft = reinterpret_cast<float*>(sm + OutSmem::PHI);          // shifts, then their factors (the phi tile is idle)
       float* red = sft + 2 * MAX_KEY_SPLIT;
       const float a2m = reinterpret_cast<const float*>(img + IMG_A2)[m];
       float wmx = a2m;
@@ -558,8 +590,24 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
 #pragma unroll
       for (int n = 0; n < TC_NV; n++)
         *reinterpret_cast<__half*>(kcol + sw128_offset(n, m & 63)) = __float2half_rn(n <= TC_DV ? val[n <= TC_DV ? n : 0] * sc : 0.f);
-      gs[m] = (float)ex + a2m - a2max;
-      named_bar_sync(1, EPI_THREADS);
+      // g_m as an fp16 value and its fp16 remainder: K elements 0 and 1 of row m of the operand
+      {
+        const float gm = (float)ex + a2m - a2max;
+        const __half hi = __float2half_rn(gm), lo = __float2half_rn(gm - __half2float(hi));
+        uint8_t* rowp = sm + OutSmem::GOP + (m >> 3) * 256 + (m & 7) * 16;
+        *reinterpret_cast<uint4*>(rowp) = make_uint4((uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16), 0, 0, 0);
+        *reinterpret_cast<uint4*>(rowp + 128) = make_uint4(0, 0, 0, 0);
+      }
+      // the A operand of that step: 1, 1, 0, ... (fp16) in every row
+      if (hf == 0) {
+        asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %2, %2, %2, %2, %2, %2};" ::"r"(lane_addr + OUT_COL_ONE),
+                     "r"(0x3C003C00u), "r"(0u) : "memory");
+        tmem_wait_st();
+      }
+      named_bar_sync(1, EPI_THREADS);          // the shifts' factors have been read: the phi tile may be written
+      fence_proxy_async_smem();
+      tcgen05_fence_before();
+      mbar_arrive_warp(&misc->g_ready, lane);
     }
     // Y rows of tile j (its contraction has completed): 32 of the 64 columns per thread
     auto write_out = [&](int j) {
@@ -576,9 +624,9 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
       if (r0 + lane < L && (!(den > 0.f) || !isfinite(den))) atomicExch(status, FSHARP_E_NONFINITE);
       float inv;                       // outputs are rounded to bf16: the approximate reciprocal (1 ulp) is exact enough
       asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(den));
-      // The thread's 64 bytes go through shared memory so that a store instruction of the warp
-      // covers 8 rows x 64 contiguous bytes instead of 32 rows x 16 bytes.
-      uint8_t* stg = sm + OutSmem::STAGE + warp * 2048;
+      // The thread's 64 bytes go through shared memory so that a store instruction of the warp covers 8 rows x 64
+      // contiguous bytes.  The staging area lies inside the rows of the phi tile that this warp itself writes next.
+      uint8_t* stg = sm + OutSmem::PHI + hf * 2 * TILE_BYTES + q * 4096;
 #pragma unroll
       for (int i = 0; i < 4; i++) {
         uint32_t o[4];
@@ -594,6 +642,7 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
         const uint4 val = *reinterpret_cast<const uint4*>(stg + rr * 64 + ((c ^ ((rr >> 1) & 3)) << 4));
         if (r0 + rr < L) *reinterpret_cast<uint4*>(Yb + (r0 + rr) * ay.sl + hf * 32 + c * 8) = val;
       }
+      __syncwarp();
     };
     for (int it = 0; it < ntiles && alive; it++) {
       if (!mbar_wait(&misc->logits_full, it & 1, abortp, status, false)) { alive = false; break; }
@@ -601,27 +650,19 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
       tcgen05_fence_after();
       uint32_t v[128];
 #pragma unroll
-      for (int c = 0; c < 8; c++) {
-        uint32_t t[16];
-        tmem_ld16(lane_addr + OUT_COL_LOGITS + hf * 128 + c * 16, t);
-#pragma unroll
-        for (int j = 0; j < 16; j++) v[c * 16 + j] = t[j];
-      }
+      for (int c = 0; c < 8; c++) tmem_ld16(lane_addr + OUT_COL_LOGITS + hf * 128 + c * 16, reinterpret_cast<uint32_t(&)[16]>(v[c * 16]));
       tmem_wait_ld();
       tcgen05_fence_before();
       mbar_arrive_warp(&misc->logits_free, lane);
-      // the exponent of feature m's column of the state, and w^T A w of both sides, join the logit
-#pragma unroll
-      for (int i = 0; i < 128; i += 4) {
-        const float4 g4 = *reinterpret_cast<const float4*>(gs + hf * 128 + i);
-        v[i] = __float_as_uint(__uint_as_float(v[i]) + g4.x);
-        v[i + 1] = __float_as_uint(__uint_as_float(v[i + 1]) + g4.y);
-        v[i + 2] = __float_as_uint(__uint_as_float(v[i + 2]) + g4.z);
-        v[i + 3] = __float_as_uint(__uint_as_float(v[i + 3]) + g4.w);
-      }
+      // (the exponent of feature m's column of the state and w^T A w of both sides are already in the logits)
       float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int i = 0; i < 128; i++) mxp[i & 3] = fmaxf(mxp[i & 3], __uint_as_float(v[i]));
+      for (int i = 0; i < 128; i += 8) {
+        mxp[0] = max3(mxp[0], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+        mxp[1] = max3(mxp[1], __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+        mxp[2] = max3(mxp[2], __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+        mxp[3] = max3(mxp[3], __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+      }
       float mx = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
       // the other half of the row: its thread sits in warp q of the other warpgroup (slots rotate over two tiles:
       // a slot is rewritten only after both warps have passed the next tile's barrier)
@@ -638,13 +679,25 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
       for (int c = 0; c < 16; c++) {
         uint32_t p[4];
 #pragma unroll
-        for (int j = 0; j < 4; j++)
-          p[j] = pack_f16(ex2(__uint_as_float(v[c * 8 + 2 * j]) - mx), ex2(__uint_as_float(v[c * 8 + 2 * j + 1]) - mx));
+        for (int j = 0; j < 4; j++) {
+          uint32_t& e0 = v[c * 8 + 2 * j];
+          uint32_t& e1 = v[c * 8 + 2 * j + 1];
+          add2(e0, e1, -mx, -mx);
+          if (j < OUT_POLY_PAIRS) {
+            exp2_poly2(e0, e1);
+            p[j] = pack_f16(__uint_as_float(e0), __uint_as_float(e1));
+          } else {
+            p[j] = pack_f16(ex2(__uint_as_float(e0)), ex2(__uint_as_float(e1)));
+          }
+        }
         *reinterpret_cast<uint4*>(prow + (c >> 3) * TILE_BYTES + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
         if ((c & 7) == 7) {                     // a 64-feature block of this half is complete
           fence_proxy_async_smem();
           tcgen05_fence_before();
           mbar_arrive_warp(&misc->phi_full[hf * 2 + (c >> 3)], lane);
+          // a real branch after the hand-over: the instruction scheduler would otherwise move the (side-effect-free)
+          // exponentials of the second block ahead of it
+          if (*abortp) { alive = false; break; }
         }
       }
     }
