@@ -39,10 +39,12 @@ constexpr int PREFETCH_TILES = 4;   // tiles pulled into L2 ahead of the shared-
 // The accumulator of half h is acc_h = phi_h^T [V | 1] (128 feature lanes x 80 columns: the phi half
 // tile is the M-side operand, [V | 1] the N = 80 side), so a contraction step costs 80 columns of the
 // tensor pipe instead of 128, and every epilogue thread (= one feature) takes part when the state leaves.
+constexpr int KV_KSTAGES = 3;       // key tiles in flight (TMA, conversion to fp16, logits MMA)
+constexpr bool KV_TURNS = false;    // the two feature halves take turns at the exponentials
+constexpr int KV_POLY_PAIRS = 1;    // of every four pairs of exponentials, this many run on the multiply-add pipe
 struct KvSmem {
-  static constexpr uint32_t X0 = 0, V0 = 2 * TILE_BYTES, ONES = 4 * TILE_BYTES, W = ONES + TILE_BYTES,
-                            WLO = W + IMG_W_BYTES, PHI = WLO + IMG_W_BYTES, MISC = PHI + 4 * TILE_BYTES,
-                            TOTAL = MISC + 256;
+  static constexpr uint32_t X0 = 0, V0 = KV_KSTAGES * TILE_BYTES, ONES = V0 + 2 * TILE_BYTES, W = ONES + TILE_BYTES,
+                            PHI = W + IMG_W_BYTES, MISC = PHI + 4 * TILE_BYTES, TOTAL = MISC + 256;
 };
 static_assert(KvSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 static_assert(KvSmem::PHI % 1024 == 0 && KvSmem::W % 1024 == 0 && KvSmem::ONES % 1024 == 0, "swizzled tiles need 1024-byte alignment");
@@ -50,7 +52,8 @@ static_assert(KvSmem::PHI % 1024 == 0 && KvSmem::W % 1024 == 0 && KvSmem::ONES %
 struct KvMisc {
   // key and value tiles have barriers of their own: a key tile is free again once the logits MMA that read it
   // has completed, long before the contraction that reads the value tile of the same stage
-  uint64_t fullK[2], emptyK[2], fullV[2], emptyV[2], logits_full, logits_free, phi_full[2], phi_free[2], const_bar;
+  uint64_t fullK[KV_KSTAGES], convK[KV_KSTAGES], emptyK[KV_KSTAGES], fullV[2], emptyV[2], logits_full, logits_free, phi_full[2],
+      phi_free[2], const_bar;
   // turn[h]: half h may run its exponentials.  The halves take turns (each arrives on the other's barrier when its
   // exponentials are done), so one half has the exponential unit to itself while the other half's contraction
   // runs on the tensor cores and its warps load and scan the next tile's logits.
@@ -82,9 +85,12 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   volatile int* abortp = &misc->abort_flag;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 2; i++) {
+    for (int i = 0; i < KV_KSTAGES; i++) {
       mbar_init(&misc->fullK[i], 1);
+      mbar_init(&misc->convK[i], 1);
       mbar_init(&misc->emptyK[i], 1);
+    }
+    for (int i = 0; i < 2; i++) {
       mbar_init(&misc->fullV[i], 1);
       mbar_init(&misc->emptyV[i], 2);
       mbar_init(&misc->phi_full[i], HALF_THREADS / 32);
@@ -120,17 +126,16 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     if (lane == 0) {
       prefetch_tmap(&tmK);
       prefetch_tmap(&tmV);
-      mbar_expect_tx(&misc->const_bar, 2 * IMG_W_BYTES);
-      bulk_load(sm + KvSmem::W, img + IMG_W, IMG_W_BYTES, &misc->const_bar);
-      bulk_load(sm + KvSmem::WLO, img + IMG_WLO, IMG_W_BYTES, &misc->const_bar);
-      // the shared-memory ring is only two tiles deep; tiles further ahead are pulled into L2
+      mbar_expect_tx(&misc->const_bar, IMG_W_BYTES);
+      bulk_load(sm + KvSmem::W, img + IMG_WH, IMG_W_BYTES, &misc->const_bar);
+      // tiles ahead of the shared-memory ring are pulled into L2
       for (int it = 0; it < min(ntiles, PREFETCH_TILES); it++) {
         tma_prefetch_4d(&tmK, 0, (tile0 + it) * TILE, h, b);
         tma_prefetch_4d(&tmV, 0, (tile0 + it) * TILE, h, b);
       }
-      // Key tile `it` is loaded as soon as the logits MMA of tile it - 2 has completed; the value tile follows one
-      // iteration behind (its stage is held until the contraction of tile it - 2 has completed, which is later
-      // than the logits MMA of tile it - 1).  So the next tile's logits never wait for a value tile.
+      // Key tile `it` is loaded as soon as the logits MMA of tile it - 3 has completed; the value tile follows one
+      // iteration behind (its stage is held until the contraction of tile it - 2 has completed).  So the next
+      // tile's logits never wait for a value tile.
       int issuedK = 0, issuedV = 0;
       auto load_v = [&](int j) {
         const int sj = j & 1;
@@ -142,12 +147,12 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       };
       bool okp = true;
       for (int it = 0; it < ntiles && okp; it++) {
-        const int st = it & 1;
+        const int st = it % KV_KSTAGES;
         if (it + PREFETCH_TILES < ntiles) {
           tma_prefetch_4d(&tmK, 0, (tile0 + it + PREFETCH_TILES) * TILE, h, b);
           tma_prefetch_4d(&tmV, 0, (tile0 + it + PREFETCH_TILES) * TILE, h, b);
         }
-        if (!mbar_wait(&misc->emptyK[st], ((it >> 1) & 1) ^ 1, abortp, status)) { okp = false; break; }
+        if (!mbar_wait(&misc->emptyK[st], ((it / KV_KSTAGES) & 1) ^ 1, abortp, status)) { okp = false; break; }
         mbar_expect_tx(&misc->fullK[st], TILE_BYTES);
         tma_load_4d(sm + KvSmem::X0 + st * TILE_BYTES, &tmK, &misc->fullK[st], 0, (tile0 + it) * TILE, h, b);
         issuedK = it + 1;
@@ -156,69 +161,86 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       if (okp && ntiles > 0) load_v(ntiles - 1);
       // no copy of this block may still be in flight when it exits
       mbar_wait(&misc->const_bar, 0, abortp, status, false);
-      for (int it = max(0, issuedK - 2); it < issuedK; it++) mbar_wait(&misc->fullK[it & 1], (it >> 1) & 1, abortp, status, false);
+      for (int it = max(0, issuedK - KV_KSTAGES); it < issuedK; it++)
+        mbar_wait(&misc->fullK[it % KV_KSTAGES], (it / KV_KSTAGES) & 1, abortp, status, false);
       for (int it = max(0, issuedV - 2); it < issuedV; it++) mbar_wait(&misc->fullV[it & 1], (it >> 1) & 1, abortp, status, false);
     }
+  } else if (warp == WARP_MMA + 2) {
+    // ---------------- bf16 -> fp16 of the key tile, in place (16-byte pieces keep their swizzled positions): the
+    // logits then need one fp16 image of W (11 significant bits) instead of a bf16 value and its remainder
+    for (int it = 0; it < ntiles; it++) {
+      const int st = it % KV_KSTAGES;
+      if (!mbar_wait(&misc->fullK[st], (it / KV_KSTAGES) & 1, abortp, status, false)) break;
+      uint4* xt = reinterpret_cast<uint4*>(sm + KvSmem::X0 + st * TILE_BYTES);
+#pragma unroll 4
+      for (int i = 0; i < (int)(TILE_BYTES / 16) / 32; i++) {
+        uint4 u = xt[lane + i * 32];
+        u.x = pack_f16(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
+        u.y = pack_f16(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
+        u.z = pack_f16(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u));
+        u.w = pack_f16(__uint_as_float(u.w << 16), __uint_as_float(u.w & 0xffff0000u));
+        xt[lane + i * 32] = u;
+      }
+      fence_proxy_async_smem();
+      mbar_arrive_warp(&misc->convK[st], lane);
+    }
   } else if (warp == WARP_MMA) {
-    // ---------------- logits MMAs.  Issuing an MMA costs its thread about a hundred cycles (descriptor arithmetic
-    // and the moves into uniform registers, on a scheduler shared with two epilogue warps), so the three MMA
-    // streams of a tile have an issuing warp each: this one the logits, the next two a feature half each.
-    if (lane == 0) {
-      constexpr uint32_t ID_LOGITS = idesc_bf16(128, TC_M, 0, 0);
-      // descriptors are built once; inside the loops each MMA costs one add per operand
-      const uint64_t dX0 = smem_desc(smem_u32(sm + KvSmem::X0), 16, 1024, SWZ_128B);
-      const uint64_t dW = smem_desc(smem_u32(sm + KvSmem::W), 16, 1024, SWZ_128B);
-      const uint64_t dWlo = smem_desc(smem_u32(sm + KvSmem::WLO), 16, 1024, SWZ_128B);
-      auto issue_logits = [&](int st) {
-        const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
+    // ---------------- logits MMAs: the whole warp walks the schedule (descriptor arithmetic and waits stay
+    // warp-uniform), one elected lane issues
+    constexpr uint32_t ID_LOGITS = idesc_f16(128, TC_M, 0, 0);
+    const uint64_t dX0 = smem_desc(smem_u32(sm + KvSmem::X0), 16, 1024, SWZ_128B);
+    const uint64_t dW = smem_desc(smem_u32(sm + KvSmem::W), 16, 1024, SWZ_128B);
+    uint32_t xl = (uint32_t)dX0, wl = (uint32_t)dW;
+    const uint32_t xh = (uint32_t)(dX0 >> 32), wh = (uint32_t)(dW >> 32);
+    for (int it = 0; it < ntiles; it++) {
+      const int st = it % KV_KSTAGES;
+      opaque(xl); opaque(wl);
+      if (it == 0 && !__all_sync(0xffffffffu, mbar_wait(&misc->const_bar, 0, abortp, status))) break;
+      if (!__all_sync(0xffffffffu, mbar_wait(&misc->convK[st], (it / KV_KSTAGES) & 1, abortp, status))) break;
+      if (it > 0 && !__all_sync(0xffffffffu, mbar_wait(&misc->logits_free, (it - 1) & 1, abortp, status))) break;
+      tcgen05_fence_after();
+      if (elect_one()) {
 #pragma unroll
         for (int k = 0; k < TC_D / 16; k++)
-          mma_bf16(tmem + KV_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dW, 32 * k), ID_LOGITS, k > 0);
-#pragma unroll
-        for (int k = 0; k < TC_D / 16; k++)
-          mma_bf16(tmem + KV_COL_LOGITS, desc_advance(dX, 32 * k), desc_advance(dWlo, 32 * k), ID_LOGITS, 1);
+          mma_bf16_lh(tmem + KV_COL_LOGITS, xl + st * (TILE_BYTES / 16) + 2 * k, xh, wl + 2 * k, wh, ID_LOGITS, k > 0);
         mma_commit(&misc->logits_full);
         mma_commit(&misc->emptyK[st]);
-      };
-      bool ok = mbar_wait(&misc->const_bar, 0, abortp, status);
-      if (ok && ntiles > 0) ok = mbar_wait(&misc->fullK[0], 0, abortp, status);
-      if (ok && ntiles > 0) {
-        tcgen05_fence_after();
-        issue_logits(0);
       }
-      for (int it = 0; ok && it + 1 < ntiles; it++) {
-        const int sn = (it + 1) & 1;
-        if (!mbar_wait(&misc->fullK[sn], ((it + 1) >> 1) & 1, abortp, status)) break;
-        if (!mbar_wait(&misc->logits_free, it & 1, abortp, status)) break;
-        tcgen05_fence_after();
-        issue_logits(sn);
-      }
+      __syncwarp();
     }
   } else {
-    // ---------------- contraction of feature half hh = warp - (WARP_MMA + 1)
-    if (lane == 0) {
-      const int hh = warp - (WARP_MMA + 1);
-      constexpr uint32_t ID_KV = idesc_bf16(128, TC_NV, 1, 1);     // phi_h^T [V | 1]
-      const uint32_t sV0 = smem_u32(sm + KvSmem::V0), sOnes = smem_u32(sm + KvSmem::ONES);
-      // phi half hh as the operand whose 128 features (M) are the contiguous index: two 64-feature blocks
-      const uint64_t dPhi = smem_desc(smem_u32(sm + KvSmem::PHI) + hh * 2 * TILE_BYTES, TILE_BYTES, 1024, SWZ_128B);
-      // [V | 1] with the value index (N = 80) contiguous: block 0 = the V tile of the stage, block 1 = the ones
-      // tile, of which the first 16 columns are read
-      const uint64_t dVst0 = smem_desc(sV0, sOnes - sV0, 1024, SWZ_128B);
-      const uint64_t dVst1 = smem_desc(sV0 + TILE_BYTES, sOnes - sV0 - TILE_BYTES, 1024, SWZ_128B);
-      for (int it = 0; it < ntiles; it++) {
-        const int st = it & 1;
-        if (!mbar_wait(&misc->fullV[st], (it >> 1) & 1, abortp, status)) break;
-        const uint64_t dV = st ? dVst1 : dVst0;
-        const uint32_t acc0 = it > 0 ? 1u : 0u;
-        if (!mbar_wait(&misc->phi_full[hh], it & 1, abortp, status)) break;
-        tcgen05_fence_after();
+    // ---------------- contractions of both feature halves (the halves take turns, half 0 first, so one static order
+    // serves both): phi_h^T [V | 1]
+    constexpr uint32_t ID_KV = idesc_bf16(128, TC_NV, 1, 1);
+    const uint32_t sV0 = smem_u32(sm + KvSmem::V0), sOnes = smem_u32(sm + KvSmem::ONES);
+    // phi half hh as the operand whose 128 features (M) are the contiguous index: two 64-feature blocks
+    const uint64_t dPhi = smem_desc(smem_u32(sm + KvSmem::PHI), TILE_BYTES, 1024, SWZ_128B);
+    // [V | 1] with the value index (N = 80) contiguous: block 0 = the V tile of the stage, block 1 = the ones
+    // tile, of which the first 16 columns are read
+    const uint64_t dVst0 = smem_desc(sV0, sOnes - sV0, 1024, SWZ_128B);
+    const uint64_t dVst1 = smem_desc(sV0 + TILE_BYTES, sOnes - sV0 - TILE_BYTES, 1024, SWZ_128B);
+    uint32_t pl = (uint32_t)dPhi, v0l = (uint32_t)dVst0, v1l = (uint32_t)dVst1;
+    const uint32_t ph = (uint32_t)(dPhi >> 32), v0h = (uint32_t)(dVst0 >> 32), v1h = (uint32_t)(dVst1 >> 32);
+    bool ok = true;
+    for (int it = 0; ok && it < ntiles; it++) {
+      const int st = it & 1;
+      opaque(pl); opaque(v0l); opaque(v1l);
+      if (!__all_sync(0xffffffffu, mbar_wait(&misc->fullV[st], (it >> 1) & 1, abortp, status))) break;
+      const uint32_t vl = st ? v1l : v0l, vh = st ? v1h : v0h;
+      const uint32_t acc0 = it > 0 ? 1u : 0u;
 #pragma unroll
-        for (int k = 0; k < TILE / 16; k++)
-          mma_bf16(tmem + KV_COL_ACC + hh * TC_NV, desc_advance(dPhi, k * 2048), desc_advance(dV, k * 2048), ID_KV,
-                   k > 0 ? 1u : acc0);
-        mma_commit(&misc->phi_free[hh]);
-        mma_commit(&misc->emptyV[st]);           // the value tile is free once both halves' contractions have completed
+      for (int hh = 0; hh < 2; hh++) {
+        if (!__all_sync(0xffffffffu, mbar_wait(&misc->phi_full[hh], it & 1, abortp, status))) { ok = false; break; }
+        tcgen05_fence_after();
+        if (elect_one()) {
+#pragma unroll
+          for (int k = 0; k < TILE / 16; k++)
+            mma_bf16_lh(tmem + KV_COL_ACC + hh * TC_NV, pl + hh * 2 * (TILE_BYTES / 16) + k * 128, ph, vl + k * 128, vh, ID_KV,
+                        k > 0 ? 1u : acc0);
+          mma_commit(&misc->phi_free[hh]);
+          mma_commit(&misc->emptyV[st]);           // the value tile is free once both halves' contractions have completed
+        }
+        __syncwarp();
       }
     }
   }
@@ -237,7 +259,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     float s = 0.f;
     float cj = ntiles > 0 ? cptr[0] : 0.f;
     bool alive = true;
-    if (hf == 1) mbar_arrive_warp(&misc->turn[0], lane);     // half 0 goes first
+    if (KV_TURNS && hf == 1) mbar_arrive_warp(&misc->turn[0], lane);     // half 0 goes first
     // accumulator of this half -> partial `slot` (the contraction that feeds it has completed)
     auto write_partial = [&](size_t slot) {
       __syncwarp();
@@ -290,7 +312,12 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       {
         float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int i = 0; i < 128; i++) mxp[i & 3] = fmaxf(mxp[i & 3], __uint_as_float(v[i]));
+        for (int i = 0; i < 128; i += 8) {
+          mxp[0] = max3(mxp[0], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+          mxp[1] = max3(mxp[1], __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+          mxp[2] = max3(mxp[2], __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+          mxp[3] = max3(mxp[3], __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+        }
         const float hm = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
         float mx = valid ? hm + cj : -INFINITY;
 #pragma unroll
@@ -324,20 +351,29 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       }
       uint8_t* prow = sm + KvSmem::PHI + hf * 2 * TILE_BYTES + row * 128;
       const float rc = cj - s;
-      if (!mbar_wait(&misc->turn[hf], it & 1, abortp, status, false)) { alive = false; break; }
+      if (KV_TURNS && !mbar_wait(&misc->turn[hf], it & 1, abortp, status, false)) { alive = false; break; }
 #pragma unroll
       for (int c = 0; c < 16; c++) {
         uint32_t p[4];
 #pragma unroll
-        for (int j = 0; j < 4; j++)
-          p[j] = pack_bf16(ex2(__uint_as_float(v[c * 8 + 2 * j]) + rc), ex2(__uint_as_float(v[c * 8 + 2 * j + 1]) + rc));
+        for (int j = 0; j < 4; j++) {
+          uint32_t& e0 = v[c * 8 + 2 * j];
+          uint32_t& e1 = v[c * 8 + 2 * j + 1];
+          add2(e0, e1, rc, rc);
+          if (j < KV_POLY_PAIRS) {
+            exp2_poly2(e0, e1);
+            p[j] = pack_bf16(__uint_as_float(e0), __uint_as_float(e1));
+          } else {
+            p[j] = pack_bf16(ex2(__uint_as_float(e0)), ex2(__uint_as_float(e1)));
+          }
+        }
         if (!valid) p[0] = p[1] = p[2] = p[3] = 0u;
         *reinterpret_cast<uint4*>(prow + (c >> 3) * TILE_BYTES + (((c & 7) ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
       }
       fence_proxy_async_smem();
       tcgen05_fence_before();
       mbar_arrive_warp(&misc->phi_full[hf], lane);
-      mbar_arrive_warp(&misc->turn[hf ^ 1], lane);
+      if (KV_TURNS) mbar_arrive_warp(&misc->turn[hf ^ 1], lane);
       cj = cnext;
     }
     // write this split's partial phi_h^T [V | 1] (rows 0..64 of the state), its shift and its largest magnitude

@@ -30,6 +30,12 @@ def _worker(rank, world, port, out):
                       LOCAL_RANK=str(rank))
     dist.init_process_group("gloo", rank=rank, world_size=world)
     r, lr, w = sharding.env_rank_world()
+    import bench                                  # the benchmark's own rank set-up, as torchrun would start it
+    assert bench.rank_setup(2) == (r, lr, w) == (rank, rank, world)
+
+    class A:
+        gpus, impl = 2, "native"
+    assert bench.relaunch_if_needed(A) is False   # already under a launcher: no second one is started
     units = sharding.unit_partition(48, r, w)
     # each rank "times" its own share; the job's time is the slowest rank, its work the sum
     t = sharding.max_over_ranks(1.0 + 0.5 * r)
@@ -55,3 +61,24 @@ def test_two_gloo_ranks_share_units_and_reduce_time():
         assert p.exitcode == 0
     assert res[0][1] + res[1][1] == list(range(48))
     assert all(abs(t - 1.5) < 1e-12 and n == 48.0 for _, _, t, n in res)
+
+
+def test_bench_starts_its_own_ranks_only_when_asked(monkeypatch):
+    """`python bench.py --gpus N` outside a launcher re-executes itself under torch.distributed.run with N
+    ranks on 127.0.0.1; with one GPU, under a launcher, or for the CPU reference arm it does not."""
+    import bench
+
+    class A:
+        gpus, impl = 1, "native"
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    assert bench.relaunch_if_needed(A) is False
+    A.gpus, A.impl = 4, "reference"
+    assert bench.relaunch_if_needed(A) is False
+    A.impl = "native"
+    seen = {}
+    monkeypatch.setattr(bench.subprocess, "call", lambda cmd: seen.setdefault("cmd", cmd) and 0)
+    with pytest.raises(SystemExit):
+        bench.relaunch_if_needed(A)
+    cmd = seen["cmd"]
+    assert "torch.distributed.run" in cmd and "--nproc-per-node=4" in cmd and "127.0.0.1" in cmd
+    assert bench.rank_setup(1) == (0, 0, 1)
