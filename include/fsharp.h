@@ -171,7 +171,9 @@ int fsharp_featurize(fsharp_ctx* ctx, const void* X, const float* Omega, const d
  * that first call before any stream capture begins.  All calls share the one array and
  * it keeps whatever the last call left in it; each call writes every word it later reads,
  * so stale contents are harmless, but two calls whose kernels may overlap on the GPU
- * (different streams, or different host threads) race on it: serialise them. */
+ * (different streams, or different host threads) race on it: serialise them.
+ * The work is launched on the CURRENT device: make the device that holds X current before the call.
+ * With device_status == NULL a non-finite value met on the device is not reported anywhere. */
 size_t fsharp_static_scratch_bytes(void);
 int fsharp_featurize_static(void* stream, const void* X, const float* Omega, const double* params,
                             int side, const fsharp_dims* dims, int dtype, float qk_scale, int stab,

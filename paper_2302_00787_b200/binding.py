@@ -281,11 +281,26 @@ def fsharp_featurize_static(X, Omega, params, side, phi, logscale=None, pool=POO
     M = Omega.shape[-2]
     ohs = Omega.stride(0) if Omega.dim() == 3 else 0
     dm = make_dims(B, H, L, L, d, d, M, pool, q=X, k=X, omega_head_stride=ohs)
+
+    # the kernels write through these pointers unchecked: refuse anything they would overrun
+    def need(t, name, dtype, shape):
+        if t.device != X.device or t.dtype != dtype or tuple(t.shape) != shape or not t.is_contiguous():
+            raise ValueError(f"{name}: expected a contiguous {dtype} tensor of shape {shape} on {X.device}")
+    need(phi, "phi", torch.float32, (B, H, L, M))
+    if stab == STAB_ROW:
+        if logscale is not None:
+            need(logscale, "logscale", torch.float32, (B, H, L))
+    elif stab == STAB_GROUP:
+        if logscale is not None:
+            need(logscale, "logscale", torch.float32, (B, H))
+    if device_status is not None:
+        need(device_status, "device_status", torch.int32, (1,))
     sp = stream.cuda_stream if stream is not None else torch.cuda.current_stream(X.device).cuda_stream
-    return lib.fsharp_featurize_static(
-        C.c_void_p(sp), X.data_ptr(), Omega.data_ptr(), params.data_ptr(), side, C.byref(dm), _dtype_code(X),
-        qk_scale, stab, phi.data_ptr(), logscale.data_ptr() if logscale is not None else None,
-        device_status.data_ptr() if device_status is not None else None)
+    with torch.cuda.device(X.device):          # the entry point launches on the current device
+        return lib.fsharp_featurize_static(
+            C.c_void_p(sp), X.data_ptr(), Omega.data_ptr(), params.data_ptr(), side, C.byref(dm), _dtype_code(X),
+            qk_scale, stab, phi.data_ptr(), logscale.data_ptr() if logscale is not None else None,
+            device_status.data_ptr() if device_status is not None else None)
 
 
 def unpack_params(blob: torch.Tensor, d: int):

@@ -119,6 +119,8 @@ int fsharp_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, 
     use_tc = fs_tc_supported(dims, dtype, causal, chunk, qk_scale) != 0;
     if (!use_tc && ctx->impl == FSHARP_IMPL_TENSOR) return FSHARP_E_SHAPE;
   }
+  // the fp32 path indexes (batch, head, chunk) through a grid z coordinate: refuse before anything is launched
+  if (!use_tc && causal && (int64_t)dims->B * dims->H * (dims->Lq / chunk) > 65535) return FSHARP_E_SHAPE;
   const size_t need = ws_round(prep_f * 4) + (use_tc ? fs_tc_attend_scratch_bytes(ctx, dims, causal, chunk)
                                                      : fs_simt_attend_scratch_bytes(dims, causal, chunk));
   FS_TRY(fs_ws_reserve(ctx, need));

@@ -370,6 +370,7 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
     int nsl = (4 * ctx->sm_count + BH - 1) / BH;
     int maxsl = (Lk + 255) / 256;
     if (nsl > maxsl) nsl = maxsl;
+    if (nsl > 65535 / BH) nsl = 65535 / BH;          // the (unit, slice) index is a grid z coordinate
     if (nsl < 1) nsl = 1;
     int slen = (Lk + nsl - 1) / nsl;
     nsl = (Lk + slen - 1) / slen;

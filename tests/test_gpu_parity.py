@@ -424,6 +424,11 @@ def test_error_codes(ctx):
     flat = torch.empty(64 * 16 + 1, device="cuda")[1:].view(1, 1, 64, 16)
     assert code(lambda: ctx.fsharp_stats(flat, flat)) == -3                                       # misaligned
     assert code(lambda: ctx.fsharp_attend(dQ, dK[:, :, :0], dV[:, :, :0], dOm, pr)) == -2         # no keys
+    # fp32 causal: (batch, head, chunk) is a grid coordinate of at most 65535; refused as a shape, before any launch
+    wide = dQ[:, :1, :1].expand(1, 1024, 4096, 16)
+    n0 = ctx.launch_count()
+    assert code(lambda: ctx.fsharp_attend(wide, wide, wide, dOm, pr, causal=True, chunk=64)) == -2
+    assert ctx.launch_count() == n0
     lib = fb.load_library()
     assert lib.fsharp_fit_params(ctx._h, None, 1, 16, 4, 0.0, pr.data_ptr()) == -1
     assert lib.fsharp_fit_params(ctx._h, pr.data_ptr(), 1, 16, 9, 0.0, pr.data_ptr()) == -1

@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import favor_sharp as fs
 from paper_2302_00787_b200 import binding as fb
 from paper_2302_00787_b200 import workloads as wl
 
@@ -20,7 +21,7 @@ def _inputs(w):
     Q, K, V = wl.make_qkv(w)
     Om = wl.make_omega(w)
     td = torch.bfloat16 if w.dtype == "bf16" else torch.float32
-    return torch.from_numpy(Q).cuda().to(td), torch.from_numpy(K).cuda().to(td), torch.from_numpy(Om).cuda()
+    return (Q, K, Om), (torch.from_numpy(Q).cuda().to(td), torch.from_numpy(K).cuda().to(td), torch.from_numpy(Om).cuda())
 
 
 def test_static_scratch_entry_point_matches_featurize_twice_in_a_row():
@@ -28,7 +29,7 @@ def test_static_scratch_entry_point_matches_featurize_twice_in_a_row():
     cases = [(wl.WORKLOADS["cfg2"].scaled(B=1, H=2, L=300), 1, fb.STAB_ROW),
              (wl.WORKLOADS["cfg3"].scaled(B=1, H=2, L=256), 2, fb.STAB_GROUP)]
     for call, (w, side, stab) in enumerate(cases):   # two calls in a row on the shared scratch, different problems
-        dQ, dK, dOm = _inputs(w)
+        (Q, K, Om), (dQ, dK, dOm) = _inputs(w)
         X = dQ if side == 1 else dK
         st = ctx.fsharp_stats(dQ, dK)
         pr = ctx.fsharp_fit_params(st, w.d, w.variant)
@@ -51,6 +52,15 @@ def test_static_scratch_entry_point_matches_featurize_twice_in_a_row():
         big = ref > 1e-30
         assert np.max(np.abs(got[big] / ref[big] - 1)) < 2e-4
         assert np.max(np.abs(ls.cpu().numpy() - ref_ls.cpu().numpy())) < 1e-4
+        # and against the fp64 checker itself, not only against the library's other entry point: the features of
+        # one (batch, head) from the definition (Section 4 with Section 2.1's M^-1/2), on the same parameter blob
+        p = fb.unpack_params(pr.cpu().numpy()[1], w.d)
+        Xh = (Q if side == 1 else K)[0, 1]
+        logf = fs.derf_log_features(Xh, Om, p["A"], p[f"B{side}"], p[f"C{side}"], p["logD"])
+        shift = ls.cpu().numpy().astype(np.float64)[0, 1]
+        expect = np.exp(logf - (shift[:, None] if stab == fb.STAB_ROW else shift))
+        big = expect > 1e-30
+        assert np.max(np.abs(got[0, 1][big] / expect[big] - 1)) < 2e-4
     ctx.close()
 
 
@@ -65,3 +75,10 @@ def test_static_scratch_entry_point_refuses_what_does_not_fit():
     assert fb.fsharp_featurize_static(X, Om, pr, 1, phi, ls) == -10
     assert "scratch" in fb.strerror(-10)
     assert fb.fsharp_featurize_static(X, Om, pr, 3, phi, ls) == -1          # bad side
+    # the binding refuses outputs that the kernels would overrun
+    with pytest.raises(ValueError):
+        fb.fsharp_featurize_static(X, Om, pr, 1, phi[..., :512], ls)
+    with pytest.raises(ValueError):
+        fb.fsharp_featurize_static(X, Om, pr, 1, phi.double(), ls)
+    with pytest.raises(ValueError):
+        fb.fsharp_featurize_static(X, Om, pr, 1, phi, ls[:, :8], stab=fb.STAB_ROW)
