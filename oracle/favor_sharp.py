@@ -359,3 +359,17 @@ def pair_closed_form_variance(X, Y, p, M):
     X = np.asarray(X, F64)
     Y = np.asarray(Y, F64)
     return np.array([derf_variance(X[i], Y[i], p) for i in range(X.shape[0])]) / M
+
+
+def pair_pooled_relative_variance(est, X, Y, var_cf):
+    """The two pooled numbers of the variance study (Section 5.1), for one parameterisation:
+    mean over pairs of (sample variance of Khat over the R feature draws) / K^2, and
+    mean over pairs of (Theorem 4.1's variance / M) / K^2, with K = exp(x^T y) (Section 2.1, alpha = 0).
+    est: (R, npairs) estimates, one row per draw; var_cf: (npairs,) from pair_closed_form_variance.
+    The sample variance is the unbiased one (divisor R - 1)."""
+    est = np.asarray(est, F64)
+    X = np.asarray(X, F64)
+    Y = np.asarray(Y, F64)
+    K2 = np.exp(2.0 * np.sum(X * Y, axis=1))
+    emp = est.var(axis=0, ddof=1) / K2
+    return float(emp.mean()), float((np.asarray(var_cf, F64) / K2).mean())

@@ -157,6 +157,32 @@ def test_empirical_variance_matches_closed_form():
         assert abs(est.mean() / np.exp(x[0] @ y[0]) - 1) < 4 * np.sqrt(cf / R) / np.exp(x[0] @ y[0])
 
 
+def test_pooled_relative_variances_agree_on_small_norm_iid_draws():
+    """Pooled over pairs, the empirical relative variance over R draws of M iid omegas agrees with the pooled
+    closed form (Theorem 4.1 / M) -- small norms and small d, where the summands have light tails -- and the
+    pooled numbers equal their definitions written out pair by pair."""
+    rng = np.random.default_rng(44)
+    d, M, R, npairs = 4, 8, 100000, 16
+    X, Y = toy_sets(rng, npairs, d, shift=0.1, scale=0.3)
+    Om = rng.standard_normal((R * M, d))            # R independent draws of M iid omegas, side by side
+    for variant in ("posrf", "gerf", "aderf", "sderf"):
+        p = fs.fit_params(X, Y, variant)
+        P, S = fs.features_pair(X, Y, Om, p)         # scaled by (R M)^-1/2: undo, then average each draw's M features
+        est = (P * S * (R * M)).reshape(npairs, R, M).mean(axis=2).T
+        cf = fs.pair_closed_form_variance(X, Y, p, M)
+        emp_pooled, cf_pooled = fs.pair_pooled_relative_variance(est, X, Y, cf)
+        assert abs(emp_pooled / cf_pooled - 1) < 0.05, variant
+        # definitions, one pair at a time
+        e2 = c2 = 0.0
+        for i in range(npairs):
+            K = np.exp(X[i] @ Y[i])
+            m = est[:, i].sum() / R
+            e2 += ((est[:, i] - m) ** 2).sum() / (R - 1) / K ** 2
+            c2 += cf[i] / K ** 2
+        assert abs(emp_pooled - e2 / npairs) < 1e-12 * abs(emp_pooled)
+        assert abs(cf_pooled - c2 / npairs) < 1e-12 * abs(cf_pooled)
+
+
 # ------------------------------------------------------------------ fits
 def thm41_residuals(p):
     d = p["A"].shape[0]
