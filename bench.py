@@ -244,6 +244,84 @@ def kernel_flops(name, w, work):
     return None
 
 
+def run_pairs(args):
+    """The variance-study batch (--workload cfg4): for each of the four parameterisations, R draws of estimates for
+    every pair, the closed-form variances and the two pooled relative variances.  One line, in pairs/s."""
+    import torch
+    from paper_2302_00787_b200 import binding as fb
+    from paper_2302_00787_b200 import workloads as wl
+    pw = wl.PAIR_WORKLOADS[args.workload]
+    dev = torch.device("cuda", 0)
+    X, Y = wl.make_pairs(pw.npairs, pw.d, pw.seed)
+    Om = wl.make_pair_omegas(pw)
+    dX, dY, dOm = (torch.from_numpy(a).to(dev) for a in (X, Y, Om))
+    ctx = fb.Context(0)
+    st = ctx.fsharp_stats(dX.view(1, 1, pw.npairs, pw.d), dY.view(1, 1, pw.npairs, pw.d))
+    prs = [ctx.fsharp_fit_params(st, pw.d, v) for v in pw.variants]
+    est = torch.empty(pw.R, pw.npairs, dtype=torch.float32, device=dev)
+    pooled = {}
+
+    def step():
+        for v, pr in zip(pw.variants, prs):
+            pooled[v] = ctx.fsharp_pair_estimate(dX, dY, dOm, pr, want_pooled=True, est=est)[2]
+
+    steps, warm = max(1, min(args.steps, 10)), 3
+    for _ in range(warm):
+        step()
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    sampler = ClockSampler(physical_index(0))
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0 = ctx.launch_count()
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    launches = ctx.launch_count() - n0
+    ctx.set_timing(True)
+    step()
+    kern = ctx.read_timing()
+    ctx.set_timing(False)
+    sampler.stop_flag = True
+    sampler.join(timeout=2)
+    nv = len(pw.variants)
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+    flops = nv * pw.R * pw.npairs * 2 * (2 * pw.M * pw.d)            # both sides' w^T B x per pair, draw and variant
+    peak = 128 * 2 * sm_count * 1965e6 / 1e12                           # fp32: 128 multiply-adds per clock and SM
+    t_k = kern["pairs_kernel"][0] / kern["pairs_kernel"][1] * 1e-3
+    out = {"metric": "kernel estimates for (x, y) pairs with empirical and closed-form variance", "value": pw.npairs / (ms * 1e-3),
+           "unit": "pairs/s", "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+           "config": {"workload": f"{pw.name}: {pw.npairs} pairs, d {pw.d}, M {pw.M} orthogonal features, R {pw.R} draws, "
+                                  f"parameterisations {', '.join(pw.variants)} (a step covers all of them)"},
+           "clocks": sampler.result(), "gpu_launches": launches,
+           "roofline": {"kernel": "pairs_kernel", "bound": "alu", "achieved": flops / nv / t_k / 1e12, "peak": peak, "unit": "TFLOP/s",
+                        "frac": flops / nv / t_k / 1e12 / peak, "traffic": None,
+                        "peak_source": "128 fp32 multiply-adds per clock and SM x SMs x 1965 MHz"},
+           "kernels": {k: {"ms_per_launch": v[0] / v[1], "launches_per_step": v[1]} for k, v in kern.items()},
+           "pooled_relative_variance": {v: {"empirical": float(pooled[v][0]), "closed_form": float(pooled[v][1])} for v in pw.variants}}
+    if not args.no_cpu_baseline:
+        from oracle import favor_sharp as fs
+        n = 4096
+        pr0 = fb.unpack_params(prs[0].cpu().numpy()[0], pw.d)
+        t0 = time.perf_counter()
+        for r in range(2):
+            fs.pair_estimate(X[:n], Y[:n], Om[r], pr0)
+        t_est = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        fs.pair_closed_form_variance(X[:256], Y[:256], pr0, pw.M)
+        t_var = time.perf_counter() - t0
+        # scaled to one step: every pair gets R draws of estimates and one closed-form variance per parameterisation
+        per_est, per_var = t_est / (2 * n), t_var / 256
+        out["cpu_baseline"] = {"value": 1.0 / (nv * (pw.R * per_est + per_var)), "unit": "pairs/s", "cores": cpu_threads(), "kind": "oracle",
+                               "sample": f"{n} pairs x 2 draws of estimates and 256 closed-form variances of one parameterisation, "
+                                         "scaled to all draws and parameterisations"}
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -259,6 +337,9 @@ def main():
     ap.add_argument("--kernel-impl", default="auto", choices=["auto", "simt", "tensor"])
     args = ap.parse_args()
 
+    if args.workload == "cfg4":
+        run_pairs(args)
+        return
     ws = workload_list(args.workload)
     if args.impl == "reference":
         run_reference(args, ws)

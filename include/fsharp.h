@@ -198,10 +198,14 @@ int fsharp_forward_host(fsharp_ctx* ctx, const void* Q, const void* K, const voi
 /* Kernel estimates for npairs (x_p, y_p) pairs (Section 2.1: Khat = sum_m P_pm S_pm)
  * with R independent feature draws: X, Y float32 [npairs, d]; Omega float32
  * [R, M, d]; params: one group; est: float32 [R, npairs].  If var_cf is not NULL it
- * receives, per pair, Theorem 4.1's variance divided by M (needs a diagonal A). */
+ * receives, per pair, Theorem 4.1's variance divided by M (needs a diagonal A).
+ * If pooled is not NULL (device, 2 doubles; needs var_cf) it receives the two pooled numbers of
+ * the variance study (Section 5.1) for this parameterisation: the mean over pairs of the unbiased
+ * sample variance of the R estimates over K^2, and the mean over pairs of var_cf over K^2, with
+ * K = exp(x^T y). */
 int fsharp_pair_estimate(fsharp_ctx* ctx, const float* X, const float* Y, const float* Omega,
                          const double* params, int64_t npairs, int d, int M, int R,
-                         float* est, double* var_cf);
+                         float* est, double* var_cf, double* pooled);
 
 #ifdef __cplusplus
 }

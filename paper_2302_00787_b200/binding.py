@@ -72,7 +72,7 @@ def load_library() -> C.CDLL:
         "fsharp_featurize": (i32, [vp, vp, vp, vp, i32, dims_p, i32, f32, i32, vp, vp]),
         "fsharp_attend": (i32, [vp, vp, vp, vp, vp, vp, dims_p, i32, i32, i32, f32, vp]),
         "fsharp_forward_host": (i32, [vp, vp, vp, vp, vp, dims_p, i32, i32, i32, i32, f32, vp]),
-        "fsharp_pair_estimate": (i32, [vp, vp, vp, vp, vp, i64, i32, i32, i32, vp, vp]),
+        "fsharp_pair_estimate": (i32, [vp, vp, vp, vp, vp, i64, i32, i32, i32, vp, vp, vp]),
         "fsharp_set_timing": (i32, [vp, i32]),
         "fsharp_read_timing": (i32, [vp, i32, C.POINTER(C.c_float), C.POINTER(i32)]),
         "fsharp_kernel_name": (C.c_char_p, [i32]),
@@ -255,15 +255,20 @@ class Context:
                                             out.data_ptr()), "fsharp_forward_host")
         return out
 
-    def fsharp_pair_estimate(self, X, Y, Omega, params, want_variance=True):
+    def fsharp_pair_estimate(self, X, Y, Omega, params, want_variance=True, want_pooled=False, est=None):
+        """Returns (est [R, npairs], var_cf [npairs] or None) and, with want_pooled, a third item: a float64
+        tensor [2] = (pooled empirical, pooled closed-form) relative variance."""
         npairs, d = X.shape
         R, M = Omega.shape[0], Omega.shape[1]
-        est = torch.empty(R, npairs, dtype=torch.float32, device=X.device)
-        var = torch.empty(npairs, dtype=torch.float64, device=X.device) if want_variance else None
+        if est is None:
+            est = torch.empty(R, npairs, dtype=torch.float32, device=X.device)
+        var = torch.empty(npairs, dtype=torch.float64, device=X.device) if (want_variance or want_pooled) else None
+        pooled = torch.empty(2, dtype=torch.float64, device=X.device) if want_pooled else None
         _check(self.lib.fsharp_pair_estimate(self._h, X.data_ptr(), Y.data_ptr(), Omega.data_ptr(),
                                              params.data_ptr(), npairs, d, M, R, est.data_ptr(),
-                                             var.data_ptr() if var is not None else None), "fsharp_pair_estimate")
-        return est, var
+                                             var.data_ptr() if var is not None else None,
+                                             pooled.data_ptr() if pooled is not None else None), "fsharp_pair_estimate")
+        return (est, var, pooled) if want_pooled else (est, var)
 
 
 def static_scratch_bytes() -> int:

@@ -202,14 +202,15 @@ int fsharp_forward_host(fsharp_ctx* ctx, const void* Q, const void* K, const voi
 }
 
 int fsharp_pair_estimate(fsharp_ctx* ctx, const float* X, const float* Y, const float* Omega, const double* params,
-                         int64_t npairs, int d, int M, int R, float* est, double* var_cf) {
+                         int64_t npairs, int d, int M, int R, float* est, double* var_cf, double* pooled) {
   if (!ctx || !Omega || !params) return FSHARP_E_BADARG;
+  if (pooled && !var_cf) return FSHARP_E_BADARG;
   if (npairs < 0 || !dim_ok(d) || M <= 0 || M % 16 != 0 || M > 1024 || R <= 0 || R > 65535) return FSHARP_E_SHAPE;
   if (npairs > 0 && (!X || !Y || !est)) return FSHARP_E_BADARG;
   FS_CUDA_OK(cudaSetDevice(ctx->device));
   FS_TRY(fs_ws_reserve(ctx, fs_pairs_scratch_bytes(d, M, R)));
   WsAlloc ws{ctx->ws, 0};
-  return fs_run_pairs(ctx, X, Y, Omega, params, npairs, d, M, R, est, var_cf, &ws);
+  return fs_run_pairs(ctx, X, Y, Omega, params, npairs, d, M, R, est, var_cf, pooled, &ws);
 }
 
 }  // extern "C"

@@ -48,7 +48,7 @@ enum { PS_BIAS = 0, PS_CSCALAR = 3, PS_CGAMMA = 4 };
 // Kernel ids for the optional per-kernel timing (fsharp_set_timing / fsharp_read_timing).
 enum {
   FS_K_STATS = 1, FS_K_FIT, FS_K_PREP, FS_K_ROWTERM, FS_K_LOGITS, FS_K_GROUPMAX, FS_K_EXPSHIFT, FS_K_KV,
-  FS_K_PREFIX, FS_K_SCORES, FS_K_OUT, FS_K_PAIRS, FS_K_PAIRVAR_PREP, FS_K_PAIRVAR,
+  FS_K_PREFIX, FS_K_SCORES, FS_K_OUT, FS_K_PAIRS, FS_K_PAIRVAR_PREP, FS_K_PAIRVAR, FS_K_PAIRPOOL,
   FS_K_TC_KV, FS_K_TC_OUT, FS_K_TC_CAUSAL, FS_K_TC_STATS, FS_K_TC_ROWTERM,
   FS_K_COUNT
 };
@@ -170,5 +170,5 @@ int fs_simt_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V,
                    WsAlloc* ws);
 size_t fs_simt_attend_scratch_bytes(const fsharp_dims* dm, int causal, int chunk);
 int fs_run_pairs(fsharp_ctx* ctx, const float* X, const float* Y, const float* Omega, const double* params,
-                 int64_t npairs, int d, int M, int R, float* est, double* var_cf, WsAlloc* ws);
+                 int64_t npairs, int d, int M, int R, float* est, double* var_cf, double* pooled, WsAlloc* ws);
 size_t fs_pairs_scratch_bytes(int d, int M, int R);

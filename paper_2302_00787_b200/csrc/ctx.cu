@@ -157,6 +157,7 @@ const char* fsharp_kernel_name(int id) {
     case FS_K_PAIRS: return "pairs_kernel";
     case FS_K_PAIRVAR_PREP: return "pairvar_prep_kernel";
     case FS_K_PAIRVAR: return "pairvar_kernel";
+    case FS_K_PAIRPOOL: return "pairpool_kernel";
     case FS_K_TC_KV: return "tc_kv_kernel";
     case FS_K_TC_OUT: return "tc_out_kernel";
     case FS_K_TC_CAUSAL: return "tc_causal_kernel";

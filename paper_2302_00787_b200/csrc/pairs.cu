@@ -146,6 +146,52 @@ pairvar_kernel(const float* __restrict__ X, const float* __restrict__ Y, int64_t
   }
 }
 
+// Pooled relative variances (Section 5.1), one warp per pair: the unbiased sample variance of the R estimates and
+// the closed-form variance, both over K^2 = exp(2 x^T y), averaged over the pairs.  pooled[0] += empirical / np,
+// pooled[1] += closed form / np (fp64 atomics; pooled is zero on entry).
+__global__ void __launch_bounds__(NTH)
+pairpool_kernel(const float* __restrict__ X, const float* __restrict__ Y, int64_t np, int d, int R,
+                const float* __restrict__ est, const double* __restrict__ var, double* __restrict__ pooled) {
+  __shared__ double red[2][NTH / 32];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int64_t warp = (int64_t)blockIdx.x * (NTH / 32) + wib;
+  const int64_t nwarps = (int64_t)gridDim.x * (NTH / 32);
+  double acc_e = 0.0, acc_c = 0.0;                    // lane 0's running sums over this warp's pairs
+  for (int64_t p = warp; p < np; p += nwarps) {
+    const float* x = X + p * d;
+    const float* y = Y + p * d;
+    double xy = 0.0, s1 = 0.0;
+    for (int j = lane; j < d; j += 32) xy += (double)x[j] * (double)y[j];
+    for (int r = lane; r < R; r += 32) s1 += (double)est[(int64_t)r * np + p];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      xy += __shfl_xor_sync(0xffffffffu, xy, o);
+      s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+    }
+    const double mean = s1 / (double)R;
+    double s2 = 0.0;
+    for (int r = lane; r < R; r += 32) {
+      const double dv = (double)est[(int64_t)r * np + p] - mean;
+      s2 = fma(dv, dv, s2);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+    if (lane == 0) {
+      const double ik2 = exp(-2.0 * xy);
+      acc_e += (R > 1 ? s2 / (double)(R - 1) : 0.0) * ik2;
+      acc_c += var[p] * ik2;
+    }
+  }
+  if (lane == 0) { red[0][wib] = acc_e; red[1][wib] = acc_c; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double e = 0.0, c = 0.0;
+    for (int i = 0; i < NTH / 32; i++) { e += red[0][i]; c += red[1][i]; }
+    atomicAdd(&pooled[0], e / (double)np);
+    atomicAdd(&pooled[1], c / (double)np);
+  }
+}
+
 }  // namespace
 
 size_t fs_pairs_scratch_bytes(int d, int M, int R) {
@@ -154,7 +200,7 @@ size_t fs_pairs_scratch_bytes(int d, int M, int R) {
 }
 
 int fs_run_pairs(fsharp_ctx* ctx, const float* X, const float* Y, const float* Omega, const double* params,
-                 int64_t npairs, int d, int M, int R, float* est, double* var_cf, WsAlloc* ws) {
+                 int64_t npairs, int d, int M, int R, float* est, double* var_cf, double* pooled, WsAlloc* ws) {
   float* prep = ws->take<float>((size_t)R * 2 * PrepLayout{d, M}.total());
   double* ev = ws->take<double>(3 * (size_t)d * d + 1);
   // one "group" per draw, all reading the same parameter blob
@@ -177,6 +223,13 @@ int fs_run_pairs(fsharp_ctx* ctx, const float* X, const float* Y, const float* O
     pairvar_kernel<<<(unsigned)blocks, NTH, 0, ctx->stream>>>(X, Y, npairs, d, M, ev, var_cf);
     FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
+    if (pooled) {
+      FS_CUDA_OK(cudaMemsetAsync(pooled, 0, 2 * sizeof(double), ctx->stream));
+      FS_TIME_BEGIN(ctx, FS_K_PAIRPOOL);
+      pairpool_kernel<<<(unsigned)blocks, NTH, 0, ctx->stream>>>(X, Y, npairs, d, R, est, var_cf, pooled);
+      FS_TIME_END(ctx);
+      FS_LAUNCH_CHECK(ctx);
+    }
   }
   return FSHARP_OK;
 }

@@ -134,3 +134,29 @@ def make_pairs(npairs: int, d: int = 64, seed: int = 4000):
     X *= np.float32(2.0) / np.linalg.norm(X, axis=1, keepdims=True).astype(np.float32)
     Y *= np.float32(2.0) / np.linalg.norm(Y, axis=1, keepdims=True).astype(np.float32)
     return X, Y
+
+
+@dataclass(frozen=True)
+class PairWorkload:
+    """The variance-study batch: npairs (x, y) pairs, R independent draws of M orthogonal features shared by
+    all pairs, one parameter fit per variant over all the x's and y's."""
+    name: str
+    npairs: int
+    d: int
+    M: int
+    R: int
+    variants: tuple
+    seed: int = 4000
+
+    def scaled(self, **kw) -> "PairWorkload":
+        return replace(self, **kw)
+
+
+PAIR_WORKLOADS = {
+    "cfg4": PairWorkload("cfg4", 2 ** 20, 64, 64, 32, ("aderf", "sderf", "gerf", "posrf")),
+}
+
+
+def make_pair_omegas(pw: PairWorkload) -> np.ndarray:
+    """(R, M, d): draw r is an orthogonal block of its own (seed + r)."""
+    return np.stack([orthogonal_omega(pw.M, pw.d, pw.seed + r) for r in range(pw.R)])

@@ -474,6 +474,41 @@ def test_pair_estimates_and_closed_form_variance(ctx, variant):
 
 
 # ------------------------------------------------------------------ several steps in flight
+def test_variance_study_batch_many_pairs_many_draws(ctx):
+    """The variance-study batch at 2^16 pairs and 32 draws (a multi-wave grid for the estimates, the grid-stride
+    loops of the per-pair variance and of the pooling): estimates on sampled pairs for every draw, closed-form
+    variances on sampled pairs, and the two pooled relative variances, against the checker."""
+    pw = wl.PAIR_WORKLOADS["cfg4"].scaled(npairs=2 ** 16)
+    X, Y = wl.make_pairs(pw.npairs, pw.d, pw.seed)
+    Om = wl.make_pair_omegas(pw)
+    dX, dY, dOm = dev(X), dev(Y), dev(Om)
+    st = ctx.fsharp_stats(dX.view(1, 1, pw.npairs, pw.d), dY.view(1, 1, pw.npairs, pw.d))
+    rng = np.random.default_rng(5)
+    sel = np.unique(np.concatenate([rng.integers(0, pw.npairs, 500), np.arange(pw.npairs - 70, pw.npairs), [0, 63, 64]]))
+    dXs, dYs = dev(X[sel]), dev(Y[sel])
+    for variant in pw.variants:
+        pr = ctx.fsharp_fit_params(st, pw.d, variant)
+        est, var, pooled = ctx.fsharp_pair_estimate(dX, dY, dOm, pr, want_pooled=True)
+        assert ctx.status() == 0
+        p = fb.unpack_params(pr.cpu().numpy()[0], pw.d)
+        ref = np.stack([fs.pair_estimate(X[sel], Y[sel], Om[r], p) for r in range(pw.R)])
+        assert np.max(np.abs(host(est)[:, sel] / ref - 1)) < 1e-4, variant
+        vsel = sel[::4]
+        refv = fs.pair_closed_form_variance(X[vsel], Y[vsel], p, pw.M)
+        assert np.max(np.abs(var.cpu().numpy()[vsel] / refv - 1)) < 1e-8, variant
+        # pooled numbers of the full batch: the reduction over all pairs of the per-pair quantities just checked
+        K2 = torch.exp(2.0 * (dX.double() * dY.double()).sum(dim=1))
+        emp_full = (est.double().var(dim=0, unbiased=True) / K2).mean().item()
+        cf_full = (var / K2).mean().item()
+        assert abs(pooled[0].item() / emp_full - 1) < 1e-9 and abs(pooled[1].item() / cf_full - 1) < 1e-9, variant
+        # and on the sampled pairs alone, where the checker computes both numbers itself
+        est_s, var_s, pooled_s = ctx.fsharp_pair_estimate(dXs, dYs, dOm, pr, want_pooled=True)
+        emp_ref, cf_ref = fs.pair_pooled_relative_variance(ref, X[sel], Y[sel], fs.pair_closed_form_variance(X[sel], Y[sel], p, pw.M))
+        assert abs(pooled_s[0].item() / emp_ref - 1) < 1e-3, variant      # fp32 estimates: their variance to 1e-3
+        assert abs(pooled_s[1].item() / cf_ref - 1) < 1e-8, variant
+    assert ctx.status() == 0
+
+
 @pytest.mark.parametrize("name", ["cfg2", "cfg3"])
 def test_contexts_on_separate_streams_overlap_without_interference(ctx, name):
     """Three contexts, each with a stream, scratch block and outputs of its own, run whole steps
