@@ -373,3 +373,24 @@ def pair_pooled_relative_variance(est, X, Y, var_cf):
     K2 = np.exp(2.0 * np.sum(X * Y, axis=1))
     emp = est.var(axis=0, ddof=1) / K2
     return float(emp.mean()), float((np.asarray(var_cf, F64) / K2).mean())
+
+
+# --------------------------------------------------------------------------
+# The unnormalised operator (Section 2.1), scaled softmax kernel K^(alpha)
+# --------------------------------------------------------------------------
+def kernel_matrix_exact(X, Y, alpha):
+    """K^(alpha)(x, y) = exp(alpha |x|^2 + x^T y + alpha |y|^2) (Section 2.1) for all pairs: (Lx, Ly)."""
+    X = np.asarray(X, F64)
+    Y = np.asarray(Y, F64)
+    return np.exp(alpha * np.sum(X * X, axis=1)[:, None] + X @ Y.T + alpha * np.sum(Y * Y, axis=1)[None, :])
+
+
+def kernel_apply(X, Y, Cmat, Omega, p, alpha):
+    """Khat^(alpha)(X, Y) C with Khat = P S^T (Section 2.1), P and S built from fhat = exp(alpha |x|^2) f
+    (Section 2.3), evaluated in the O(L M n) order P (S^T C)."""
+    X = np.asarray(X, F64)
+    Y = np.asarray(Y, F64)
+    P, S = features_pair(X, Y, Omega, p)
+    P = P * np.exp(alpha * np.sum(X * X, axis=1))[:, None]
+    S = S * np.exp(alpha * np.sum(Y * Y, axis=1))[:, None]
+    return P @ (S.T @ np.asarray(Cmat, F64))

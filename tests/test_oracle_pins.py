@@ -183,6 +183,33 @@ def test_pooled_relative_variances_agree_on_small_norm_iid_draws():
         assert abs(cf_pooled - c2 / npairs) < 1e-12 * abs(cf_pooled)
 
 
+def test_unnormalised_operator_converges_to_the_exact_kernel_matrix():
+    """Khat^(alpha) C approaches K^(alpha) C as M grows, at rate M^-1/2, for the softmax (alpha = 0) and the
+    Gaussian kernel (alpha = -1/2); the exact Gaussian kernel matrix is exp(-|x - y|^2 / 2); and the result equals
+    the explicit L x L form."""
+    rng = np.random.default_rng(90)
+    d, L, n = 4, 24, 3
+    X, Y = toy_sets(rng, L, d, shift=0.1, scale=0.4)
+    Cm = rng.standard_normal((L, n))
+    D2 = ((X[:, None, :] - Y[None, :, :]) ** 2).sum(axis=2)
+    assert np.abs(fs.kernel_matrix_exact(X, Y, -0.5) - np.exp(-0.5 * D2)).max() < 1e-14
+    assert np.abs(fs.kernel_matrix_exact(X, Y, 0.0) - np.exp(X @ Y.T)).max() < 1e-14
+    for variant in ("posrf", "sderf", "aderf"):
+        p = fs.fit_params(X, Y, variant)
+        for alpha in (0.0, -0.5):
+            exact = fs.kernel_matrix_exact(X, Y, alpha) @ Cm
+            errs = []
+            for M in (64, 4096, 262144):
+                Om = rng.standard_normal((M, d))
+                got = fs.kernel_apply(X, Y, Cm, Om, p, alpha)
+                errs.append(np.abs(got - exact).max() / np.abs(exact).max())
+                if M == 64:                                   # explicit form: every entry of Khat, then the product
+                    P, S = fs.features_pair(X, Y, Om, p)
+                    Kh = (P @ S.T) * fs.kernel_matrix_exact(X, Y, alpha) / np.exp(X @ Y.T)
+                    assert np.abs(got - Kh @ Cm).max() < 1e-12 * np.abs(got).max()
+            assert errs[2] < 0.02 and errs[2] < errs[0] / 8, (variant, alpha, errs)
+
+
 # ------------------------------------------------------------------ fits
 def thm41_residuals(p):
     d = p["A"].shape[0]
