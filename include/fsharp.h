@@ -14,6 +14,7 @@
  *   fsharp_featurize      P or S for given parameters
  *   fsharp_attend         Y, bidirectional or causal (lower-triangular mask)
  *   fsharp_pair_estimate  Khat(x, y) for pairs, with Theorem 4.1's variance
+ *   fsharp_kernel_apply   the unnormalised operator Khat^(alpha) C (softmax and Gaussian kernels)
  *
  * Conventions common to every call
  *   - All data pointers are DEVICE pointers owned by the caller unless the
@@ -186,6 +187,17 @@ int fsharp_featurize_static(void* stream, const void* X, const float* Omega, con
 int fsharp_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V,
                   const float* Omega, const double* params, const fsharp_dims* dims,
                   int dtype, int causal, int chunk, float qk_scale, void* Y);
+
+/* The unnormalised operator of Section 2.1: out = Khat^(alpha)(X, Y) C, the O(L M n) evaluation P (S^T C) of
+ * K^(alpha)(x, y) = exp(alpha |x|^2 + x^T y + alpha |y|^2) applied to a matrix C, with the features
+ * fhat = exp(alpha |x|^2) f of Section 2.3 (alpha = 0: softmax kernel; alpha = -1/2: Gaussian kernel).
+ * X [B,H,Lq,d] (q_stride), Y [B,H,Lk,d] (k_stride), C [B,H,Lk,dv] (v_stride), out [B,H,Lq,dv] (y_stride), all of
+ * type `dtype`; Omega and params as for fsharp_attend.  Nothing is normalised, so out carries the scale of the
+ * kernel values (bf16 keeps the range, at 8 bits of precision).  Runs on the fp32 kernels for every shape.
+ * Lk = 0 is refused (FSHARP_E_SHAPE). */
+int fsharp_kernel_apply(fsharp_ctx* ctx, const void* X, const void* Y, const void* C, const float* Omega,
+                        const double* params, double alpha, const fsharp_dims* dims, int dtype, float qk_scale,
+                        void* out);
 
 /* The whole path on HOST buffers: copies Q, K, V (dense [B,H,L,*], type `dtype`)
  * to the device, runs stats -> fit -> attend, copies Y back and waits for it.

@@ -23,7 +23,7 @@ EXPORTS = [
     "fsharp_launch_count", "fsharp_workspace_bytes", "fsharp_strerror", "fsharp_stats_doubles",
     "fsharp_params_doubles", "fsharp_stats", "fsharp_fit_params", "fsharp_featurize", "fsharp_attend",
     "fsharp_forward_host", "fsharp_pair_estimate", "fsharp_set_timing", "fsharp_read_timing",
-    "fsharp_kernel_name", "fsharp_static_scratch_bytes", "fsharp_featurize_static",
+    "fsharp_kernel_name", "fsharp_static_scratch_bytes", "fsharp_featurize_static", "fsharp_kernel_apply",
 ]
 
 
@@ -71,6 +71,7 @@ def load_library() -> C.CDLL:
         "fsharp_fit_params": (i32, [vp, vp, i32, i32, i32, f64, vp]),
         "fsharp_featurize": (i32, [vp, vp, vp, vp, i32, dims_p, i32, f32, i32, vp, vp]),
         "fsharp_attend": (i32, [vp, vp, vp, vp, vp, vp, dims_p, i32, i32, i32, f32, vp]),
+        "fsharp_kernel_apply": (i32, [vp, vp, vp, vp, vp, vp, f64, dims_p, i32, f32, vp]),
         "fsharp_forward_host": (i32, [vp, vp, vp, vp, vp, dims_p, i32, i32, i32, i32, f32, vp]),
         "fsharp_pair_estimate": (i32, [vp, vp, vp, vp, vp, i64, i32, i32, i32, vp, vp, vp]),
         "fsharp_set_timing": (i32, [vp, i32]),
@@ -235,6 +236,19 @@ class Context:
         _check(self.lib.fsharp_attend(self._h, Q.data_ptr(), K.data_ptr(), V.data_ptr(), Omega.data_ptr(),
                                       params.data_ptr(), C.byref(dm), _dtype_code(Q), int(bool(causal)), chunk,
                                       qk_scale, out.data_ptr()), "fsharp_attend")
+        return out
+
+    def fsharp_kernel_apply(self, X, Y, Cmat, Omega, params, alpha=0.0, pool=POOL_PER_BH, qk_scale=1.0, out=None):
+        B, H, Lq, d = X.shape
+        Lk, dv = Y.shape[2], Cmat.shape[3]
+        M = Omega.shape[-2]
+        ohs = Omega.stride(0) if Omega.dim() == 3 else 0
+        if out is None:
+            out = torch.empty(B, H, Lq, dv, dtype=X.dtype, device=X.device)
+        dm = make_dims(B, H, Lq, Lk, d, dv, M, pool, q=X, k=Y, v=Cmat, y=out, omega_head_stride=ohs)
+        _check(self.lib.fsharp_kernel_apply(self._h, X.data_ptr(), Y.data_ptr(), Cmat.data_ptr(), Omega.data_ptr(),
+                                            params.data_ptr(), float(alpha), C.byref(dm), _dtype_code(X), qk_scale,
+                                            out.data_ptr()), "fsharp_kernel_apply")
         return out
 
     def fsharp_forward_host(self, Q, K, V, Omega, variant, causal=False, chunk=0, pool=POOL_PER_BH,

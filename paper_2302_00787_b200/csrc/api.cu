@@ -139,6 +139,32 @@ int fsharp_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, 
   return fs_simt_attend(ctx, Q, K, V, dims, dtype, causal, chunk, qk_scale, prep, Y, &ws);
 }
 
+int fsharp_kernel_apply(fsharp_ctx* ctx, const void* X, const void* Y, const void* Cmat, const float* Omega,
+                        const double* params, double alpha, const fsharp_dims* dims, int dtype, float qk_scale, void* out) {
+  if (!ctx || !Omega || !params) return FSHARP_E_BADARG;
+  FS_TRY(check_dims(dims, true));
+  if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
+  if (!isfinite(alpha)) return FSHARP_E_BADARG;
+  if (dims->B * dims->H == 0 || dims->Lq == 0) return FSHARP_OK;
+  if (dims->Lk == 0) return FSHARP_E_SHAPE;
+  FS_TRY(check_ptr(X, dtype, dims->q_stride));
+  FS_TRY(check_ptr(out, dtype, dims->y_stride));
+  FS_TRY(check_ptr(Y, dtype, dims->k_stride));
+  FS_TRY(check_ptr(Cmat, dtype, dims->v_stride));
+  FS_CUDA_OK(cudaSetDevice(ctx->device));
+  const int G = fs_groups(dims);
+  const size_t prep_f = (size_t)G * 2 * PrepLayout{dims->d, dims->M}.total();
+  const size_t np = (size_t)G * ParamsLayout{dims->d}.total();
+  FS_TRY(fs_ws_reserve(ctx, ws_round(prep_f * 4) + ws_round(np * 8) + fs_simt_attend_scratch_bytes(dims, 0, 0)));
+  WsAlloc ws{ctx->ws, 0};
+  float* prep = ws.take<float>(prep_f);
+  double* shifted = ws.take<double>(np);
+  FS_TRY(fs_shift_c(ctx, params, shifted, G, dims->d, alpha));
+  FS_TRY(fs_run_prep(ctx, Omega, dims->omega_head_stride, shifted, (int64_t)ParamsLayout{dims->d}.total(), G, dims->H,
+                     dims->pool, dims->d, dims->M, prep));
+  return fs_simt_kernel_apply(ctx, X, Y, Cmat, dims, dtype, qk_scale, prep, out, &ws);
+}
+
 int fsharp_forward_host(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const float* Omega,
                         const fsharp_dims* dims, int dtype, int variant, int causal, int chunk, float qk_scale,
                         void* Y) {

@@ -245,7 +245,10 @@ template <typename T>
 __global__ void __launch_bounds__(NTH)
 out_kernel(const float* __restrict__ phiQ, const float* __restrict__ KV, const float* __restrict__ sc,
            const T* __restrict__ V, TensorAddr av, T* __restrict__ Y, TensorAddr ay, int H, int L, int M, int dv,
-           int causal, int C, int nchunks, int* __restrict__ status) {
+           int causal, int C, int nchunks, const float* __restrict__ lsq, const float* __restrict__ lsk,
+           int* __restrict__ status) {
+  // lsq != nullptr: the unnormalised operator Khat C of Section 2.1 is wanted: row i of the numerator times
+  // exp(lsq[i] + lsk[bh]), the shifts that the feature kernels took out of phi(Q) and phi(K)
   __shared__ Tiles sm;
   __shared__ float den[TM];
   const int bh = blockIdx.z, b = bh / H, h = bh % H;
@@ -293,8 +296,13 @@ out_kernel(const float* __restrict__ phiQ, const float* __restrict__ KV, const f
     int r = ty + 16 * i;
     if (i0 + r >= L) continue;
     float dn = den[r];
-    if (!(dn > 0.f) || !isfinite(dn)) bad = true;
-    float inv = 1.f / dn;
+    float inv;
+    if (lsq != nullptr) {
+      inv = expf(lsq[(int64_t)bh * L + i0 + r] + lsk[bh]);
+    } else {
+      if (!(dn > 0.f) || !isfinite(dn)) bad = true;
+      inv = 1.f / dn;
+    }
 #pragma unroll
     for (int j = 0; j < 4; j++) {
       int n = n0 + tx + 16 * j;
@@ -350,7 +358,7 @@ int featurize_t(fsharp_ctx* ctx, const void* X, TensorAddr ax, int B, int H, int
 
 template <typename T>
 int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, int causal,
-             int chunk, float qk_scale, const float* prep, void* Y, WsAlloc* ws) {
+             int chunk, float qk_scale, const float* prep, void* Y, WsAlloc* ws, bool unnormalised) {
   const int B = dm->B, H = dm->H, BH = B * H, Lq = dm->Lq, Lk = dm->Lk, d = dm->d, dv = dm->dv, M = dm->M;
   const int N = dv + 1;
   TensorAddr aq = fs_addr(dm->q_stride, H, Lq, d), ak = fs_addr(dm->k_stride, H, Lk, d);
@@ -359,10 +367,12 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
   float* phiK = ws->take<float>((size_t)BH * Lk * M);
   float* rowc = ws->take<float>((size_t)BH * (Lq > Lk ? Lq : Lk));
   unsigned* gmax = ws->take<unsigned>((size_t)BH);
+  float* lsq = unnormalised ? ws->take<float>((size_t)BH * Lq) : nullptr;
+  float* lsk = unnormalised ? ws->take<float>((size_t)BH) : nullptr;
   FS_TRY(featurize_t<T>(ctx, K, ak, B, H, Lk, d, M, dm->pool, prep, 2, qk_scale, FSHARP_STAB_GROUP, rowc, gmax,
-                        phiK, nullptr));
+                        phiK, lsk));
   FS_TRY(featurize_t<T>(ctx, Q, aq, B, H, Lq, d, M, dm->pool, prep, 1, qk_scale, FSHARP_STAB_ROW, rowc, gmax,
-                        phiQ, nullptr));
+                        phiQ, lsq));
   dim3 gout((Lq + TM - 1) / TM, (dv + TN - 1) / TN, BH);
   if (!causal) {
     float* KV = ws->take<float>((size_t)BH * M * N);
@@ -381,7 +391,7 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
     FS_LAUNCH_CHECK(ctx);
     FS_TIME_BEGIN(ctx, FS_K_OUT);
     out_kernel<T><<<gout, NTH, 0, ctx->stream>>>(phiQ, KV, nullptr, (const T*)V, av, (T*)Y, ay, H, Lq, M, dv, 0, 0,
-                                                1, ctx->d_status);
+                                                1, lsq, lsk, ctx->d_status);
     FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
   } else {
@@ -404,7 +414,7 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
     FS_LAUNCH_CHECK(ctx);
     FS_TIME_BEGIN(ctx, FS_K_OUT);
     out_kernel<T><<<gout, NTH, 0, ctx->stream>>>(phiQ, st, sc, (const T*)V, av, (T*)Y, ay, H, Lq, M, dv, 1, C, nch,
-                                                ctx->d_status);
+                                                nullptr, nullptr, ctx->d_status);
     FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
   }
@@ -427,7 +437,7 @@ size_t fs_simt_attend_scratch_bytes(const fsharp_dims* dm, int causal, int chunk
   const size_t BH = (size_t)dm->B * dm->H, N = dm->dv + 1;
   const size_t Lmax = dm->Lq > dm->Lk ? dm->Lq : dm->Lk;
   size_t b = ws_round(BH * dm->Lq * dm->M * 4) + ws_round(BH * dm->Lk * dm->M * 4) + ws_round(BH * Lmax * 4) +
-             ws_round(BH * 4);
+             ws_round(BH * 4) + ws_round(BH * dm->Lq * 4) + ws_round(BH * 4);     // (the last two: the shifts of the unnormalised mode)
   if (!causal) {
     b += ws_round(BH * dm->M * N * 4);
   } else {
@@ -439,6 +449,36 @@ size_t fs_simt_attend_scratch_bytes(const fsharp_dims* dm, int causal, int chunk
 
 int fs_simt_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm,
                    int dtype, int causal, int chunk, float qk_scale, const float* prep, void* Y, WsAlloc* ws) {
-  if (dtype == FSHARP_F32) return attend_t<float>(ctx, Q, K, V, dm, causal, chunk, qk_scale, prep, Y, ws);
-  return attend_t<__nv_bfloat16>(ctx, Q, K, V, dm, causal, chunk, qk_scale, prep, Y, ws);
+  if (dtype == FSHARP_F32) return attend_t<float>(ctx, Q, K, V, dm, causal, chunk, qk_scale, prep, Y, ws, false);
+  return attend_t<__nv_bfloat16>(ctx, Q, K, V, dm, causal, chunk, qk_scale, prep, Y, ws, false);
+}
+
+// The unnormalised operator Khat C (Section 2.1): the bidirectional pipeline with the shifts carried to the output.
+int fs_simt_kernel_apply(fsharp_ctx* ctx, const void* X, const void* Yset, const void* Cmat, const fsharp_dims* dm,
+                         int dtype, float qk_scale, const float* prep, void* out, WsAlloc* ws) {
+  if (dtype == FSHARP_F32) return attend_t<float>(ctx, X, Yset, Cmat, dm, 0, 0, qk_scale, prep, out, ws, true);
+  return attend_t<__nv_bfloat16>(ctx, X, Yset, Cmat, dm, 0, 0, qk_scale, prep, out, ws, true);
+}
+
+// params_out = params with alpha added to the diagonals of C1 and C2: exp(alpha |x|^2) f(w, x) is the DERF with
+// C + alpha I (Section 2.3's reduction of K^(alpha) to K^(0)).
+namespace {
+__global__ void shift_c_kernel(const double* __restrict__ params, double* __restrict__ out, int d, double alpha, size_t total) {
+  const size_t g = blockIdx.x;
+  ParamsLayout pl{d};
+  for (size_t e = threadIdx.x; e < total; e += blockDim.x) {
+    double v = params[g * total + e];
+    if (e >= pl.C(1) && e < pl.tail()) {
+      const size_t r = (e - pl.C(1)) % pl.dd();
+      if (r / d == r % d) v += alpha;
+    }
+    out[g * total + e] = v;
+  }
+}
+}  // namespace
+int fs_shift_c(fsharp_ctx* ctx, const double* params, double* out, int G, int d, double alpha) {
+  if (G == 0) return FSHARP_OK;
+  shift_c_kernel<<<G, 256, 0, ctx->stream>>>(params, out, d, alpha, ParamsLayout{d}.total());
+  FS_LAUNCH_CHECK(ctx);
+  return FSHARP_OK;
 }

@@ -474,6 +474,30 @@ def test_pair_estimates_and_closed_form_variance(ctx, variant):
 
 
 # ------------------------------------------------------------------ several steps in flight
+@pytest.mark.parametrize("alpha", [0.0, -0.5])
+@pytest.mark.parametrize("w", [W["cfg1"], W["cfg2"].scaled(B=1, H=2, L=300), W["cfg3b"].scaled(B=2, H=1, L=200)],
+                         ids=lambda w: f"{w.name}-{w.variant}")
+def test_unnormalised_operator_matches_definition(ctx, w, alpha):
+    """Khat^(alpha) C of Sections 2.1 / 2.3 (alpha = 0: softmax kernel, alpha = -1/2: Gaussian kernel) against the
+    checker on the same Omega and the same parameter blob, relative to the largest output of the (batch, head);
+    the sets X and Y have different sizes."""
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    _, pr = gpu_fit(ctx, dQ, dK, w.d, w.variant)
+    Lq = w.L - 37
+    out = ctx.fsharp_kernel_apply(dQ[:, :, :Lq].contiguous(), dK, dV, dOm, pr, alpha=alpha)
+    assert ctx.status() == 0
+    out = host(out)
+    prh = pr.cpu().numpy()
+    for b in range(w.B):
+        for h in range(w.H):
+            p = fb.unpack_params(prh[b * w.H + h], w.d)
+            ref = fs.kernel_apply(Q[b, h, :Lq], K[b, h], V[b, h], Om, p, alpha)
+            assert rel_err(out[b, h], ref) < TOL[w.dtype], (b, h)
+    with pytest.raises(fb.FsharpError) as ei:
+        ctx.fsharp_kernel_apply(dQ, dK[:, :, :0], dV[:, :, :0], dOm, pr, alpha=alpha)
+    assert ei.value.code == -2
+
+
 def test_variance_study_batch_many_pairs_many_draws(ctx):
     """The variance-study batch at 2^16 pairs and 32 draws (a multi-wave grid for the estimates, the grid-stride
     loops of the per-pair variance and of the pooling): estimates on sampled pairs for every draw, closed-form
