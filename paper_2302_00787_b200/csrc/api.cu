@@ -9,6 +9,10 @@ int fs_tc_supported(const fsharp_dims* dm, int dtype, int causal, int chunk, flo
 size_t fs_tc_attend_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm, int causal, int chunk);
 int fs_tc_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, int causal,
                  int chunk, const uint8_t* images, const int* flags, void* Y, WsAlloc* ws);
+int fs_tc_featurize_supported(const fsharp_dims* dm, int dtype, int stab);
+size_t fs_tc_featurize_scratch_bytes(const fsharp_dims* dm, int side);
+int fs_tc_featurize(fsharp_ctx* ctx, const void* X, const fsharp_dims* dm, int side, int stab, const float* prep,
+                    const uint8_t* images, const int* flags, float* phi, float* logscale, WsAlloc* ws);
 
 namespace {
 
@@ -81,6 +85,22 @@ int fsharp_featurize(fsharp_ctx* ctx, const void* X, const float* Omega, const d
   FS_CUDA_OK(cudaSetDevice(ctx->device));
   const int G = fs_groups(dims);
   const size_t prep_f = (size_t)G * 2 * PrepLayout{dims->d, dims->M}.total();
+  // tensor-core kernel (bf16, d = 64, M = 256, row shift or none, dense phi), unless the fp32 kernels are forced
+  bool use_tc = false;
+  if (ctx->impl != FSHARP_IMPL_SIMT) {
+    use_tc = fs_tc_featurize_supported(dims, dtype, stab) != 0;
+    if (!use_tc && ctx->impl == FSHARP_IMPL_TENSOR) return FSHARP_E_SHAPE;
+  }
+  if (use_tc) {
+    FS_TRY(fs_ws_reserve(ctx, ws_round(prep_f * 4) + fs_tc_featurize_scratch_bytes(dims, side)));
+    WsAlloc wst{ctx->ws, 0};
+    float* prep_t = wst.take<float>(prep_f);
+    uint8_t* images = wst.take<uint8_t>((size_t)G * 2 * tcl::IMG_BYTES);
+    int* flags = wst.take<int>((size_t)G * 2 * tcl::FLAG_WORDS + 16);
+    FS_TRY(fs_run_prep_images(ctx, Omega, dims->omega_head_stride, params, (int64_t)ParamsLayout{dims->d}.total(), G,
+                              dims->H, dims->pool, dims->d, dims->M, prep_t, qk_scale, images, flags));
+    return fs_tc_featurize(ctx, X, dims, side, stab, prep_t, images, flags, phi, logscale, &wst);
+  }
   const size_t need = ws_round(prep_f * 4) + ws_round((size_t)dims->B * dims->H * L * 4) +
                       ws_round((size_t)dims->B * dims->H * 4);
   FS_TRY(fs_ws_reserve(ctx, need));

@@ -49,7 +49,7 @@ enum { PS_BIAS = 0, PS_CSCALAR = 3, PS_CGAMMA = 4 };
 enum {
   FS_K_STATS = 1, FS_K_FIT, FS_K_PREP, FS_K_ROWTERM, FS_K_LOGITS, FS_K_GROUPMAX, FS_K_EXPSHIFT, FS_K_KV,
   FS_K_PREFIX, FS_K_SCORES, FS_K_OUT, FS_K_PAIRS, FS_K_PAIRVAR_PREP, FS_K_PAIRVAR, FS_K_PAIRPOOL,
-  FS_K_TC_KV, FS_K_TC_OUT, FS_K_TC_CAUSAL, FS_K_TC_STATS, FS_K_TC_ROWTERM,
+  FS_K_TC_KV, FS_K_TC_OUT, FS_K_TC_CAUSAL, FS_K_TC_STATS, FS_K_TC_ROWTERM, FS_K_TC_FEAT,
   FS_K_COUNT
 };
 constexpr int FS_TIMING_SLOTS = 4096;

@@ -163,6 +163,7 @@ const char* fsharp_kernel_name(int id) {
     case FS_K_TC_CAUSAL: return "tc_causal_kernel";
     case FS_K_TC_STATS: return "tc_stats_kernel";
     case FS_K_TC_ROWTERM: return "tc_rowterm_kernel";
+    case FS_K_TC_FEAT: return "tc_feat_kernel";
     default: return "";
   }
 }

@@ -31,7 +31,7 @@ static_assert(sizeof(RtMisc) <= 256, "misc block");
 
 __global__ void __launch_bounds__(RT_THREADS)
 tc_rowterm_kernel(const __grid_constant__ CUtensorMap tmK, const uint8_t* __restrict__ images,
-                  const int* __restrict__ img_flags, int H, int pool, int L, int Lpad, int tiles_per_split,
+                  const int* __restrict__ img_flags, int side, int H, int pool, int L, int Lpad, int tiles_per_split,
                   float* __restrict__ crow, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -43,8 +43,8 @@ tc_rowterm_kernel(const __grid_constant__ CUtensorMap tmK, const uint8_t* __rest
   const int tile0 = blockIdx.x * tiles_per_split;
   const int ntiles = min(tiles_per_split, total_tiles - tile0);
   if (ntiles <= 0) return;                    // uniform over the block, before anything is allocated
-  const uint8_t* img = images + ((size_t)g * 2 + 1) * IMG_BYTES;        // side 2 (keys)
-  const bool clo = (img_flags[((size_t)g * 2 + 1) * FLAG_WORDS] & FLAG_C_LO) != 0;
+  const uint8_t* img = images + ((size_t)g * 2 + (side - 1)) * IMG_BYTES;        // side 1: queries (C1), side 2: keys (C2)
+  const bool clo = (img_flags[((size_t)g * 2 + (side - 1)) * FLAG_WORDS] & FLAG_C_LO) != 0;
   volatile int* abortp = &misc->abort_flag;
 
   if (threadIdx.x == 0) {
@@ -156,26 +156,32 @@ namespace tchost {
 int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int H, int L, int inner);
 }
 
-// crow: [B*H][Lpad] floats with Lpad = ceil(Lk / 128) * 128; rows at and beyond Lk come out as zero.
-int fs_tc_rowterm(fsharp_ctx* ctx, const void* K, const fsharp_dims* dm, const uint8_t* images, const int* flags, int Lpad,
-                  int tiles_per_split, int nsplit, float* crow) {
-  const int B = dm->B, H = dm->H, Lk = dm->Lk;
-  CUtensorMap tmK;
-  FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, Lk, dm->d), B, H, Lk, dm->d));
+// crow: [B*H][Lpad] floats with Lpad = ceil(L / 128) * 128; rows at and beyond L come out as zero.  side 1: X is the
+// query tensor (q_stride, Lq) and C1 is used; side 2: the key tensor (k_stride, Lk) and C2.
+int fs_tc_rowterm_side(fsharp_ctx* ctx, const void* X, const fsharp_dims* dm, int side, const uint8_t* images, const int* flags,
+                       int Lpad, float* crow) {
+  const int B = dm->B, H = dm->H, L = side == 1 ? dm->Lq : dm->Lk;
+  CUtensorMap tmX;
+  FS_TRY(tchost::make_map_tokens(&tmX, X, fs_addr(side == 1 ? dm->q_stride : dm->k_stride, H, L, dm->d), B, H, L, dm->d));
   FS_CUDA_OK(cudaFuncSetAttribute(tc_rowterm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RtSmem::TOTAL + 1024));
-  // The output is indexed by token, so this kernel need not follow the key-side kernel's split: two of its blocks fit
-  // an SM, and a block is bound by its single MMA-issuing thread, so it takes about two blocks per SM.
-  (void)tiles_per_split;
-  (void)nsplit;
-  const int total = (Lk + TILE - 1) / TILE;
+  // The output is indexed by token, so this kernel has a split of its own: two of its blocks fit an SM, and a block
+  // is bound by its single MMA-issuing thread, so it takes about two blocks per SM.
+  const int total = (L + TILE - 1) / TILE;
   int ns = (2 * ctx->sm_count) / (B * H);
   ns = ns < 1 ? 1 : (ns > total ? total : ns);
   const int tps = (total + ns - 1) / ns;
   ns = (total + tps - 1) / tps;
   FS_TIME_BEGIN(ctx, FS_K_TC_ROWTERM);
   tc_rowterm_kernel<<<dim3(ns, B * H), RT_THREADS, RtSmem::TOTAL + 1024, ctx->stream>>>(
-      tmK, images, flags, H, dm->pool, Lk, Lpad, tps, crow, ctx->d_status);
+      tmX, images, flags, side, H, dm->pool, L, Lpad, tps, crow, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;
+}
+
+int fs_tc_rowterm(fsharp_ctx* ctx, const void* K, const fsharp_dims* dm, const uint8_t* images, const int* flags, int Lpad,
+                  int tiles_per_split, int nsplit, float* crow) {
+  (void)tiles_per_split;
+  (void)nsplit;
+  return fs_tc_rowterm_side(ctx, K, dm, 2, images, flags, Lpad, crow);
 }

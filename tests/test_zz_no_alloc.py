@@ -33,7 +33,9 @@ def test_static_scratch_entry_point_matches_featurize_twice_in_a_row():
         X = dQ if side == 1 else dK
         st = ctx.fsharp_stats(dQ, dK)
         pr = ctx.fsharp_fit_params(st, w.d, w.variant)
+        ctx.set_impl(fb.IMPL_SIMT)          # the entry point under test runs the fp32 kernels: compare like with like
         ref_phi, ref_ls = ctx.fsharp_featurize(X, dOm, pr, side, stab=stab)
+        ctx.set_impl(fb.IMPL_AUTO)
         assert ctx.status() == 0
         phi = torch.full_like(ref_phi, float("nan"))
         ls = torch.full_like(ref_ls, float("nan"))
