@@ -57,7 +57,8 @@ enum {
   FSHARP_E_NONFINITE = -7,  /* NaN or Inf met on the device */
   FSHARP_E_TIMEOUT = -8,    /* a bounded device-side wait expired */
   FSHARP_E_CUDA = -9,       /* a CUDA runtime or driver call failed */
-  FSHARP_E_LIMIT = -10      /* problem needs more than the fixed scratch of fsharp_featurize_static */
+  FSHARP_E_LIMIT = -10,     /* problem needs more than the fixed scratch of fsharp_featurize_static */
+  FSHARP_E_INTERNAL = -11   /* an index check of the debug build (-DFSHARP_DEBUG) failed on the device */
 };
 
 enum { FSHARP_F32 = 0, FSHARP_BF16 = 1 };
@@ -106,6 +107,10 @@ int64_t fsharp_launch_count(const fsharp_ctx* ctx);
 int fsharp_set_timing(fsharp_ctx* ctx, int on);
 int fsharp_read_timing(fsharp_ctx* ctx, int cap, float* total_ms, int* launches);
 const char* fsharp_kernel_name(int id);
+/* Self-test of the bounded device-side waits (no counterpart in the paper): launches a one-warp kernel that waits, with
+ * a limit of `limit_us` microseconds (1 .. 100000), on a barrier that nothing ever completes.  The wait gives up,
+ * the kernel returns, and the next fsharp_status() reports FSHARP_E_TIMEOUT; the context stays usable. */
+int fsharp_selftest_bounded_wait(fsharp_ctx* ctx, int limit_us);
 /* Bytes of scratch the context currently holds. */
 size_t fsharp_workspace_bytes(const fsharp_ctx* ctx);
 const char* fsharp_strerror(int code);

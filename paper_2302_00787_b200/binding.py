@@ -10,7 +10,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "lib", "libfsharp.so")
+# FSHARP_LIB selects another build of the library (the debug build with index checks: lib/libfsharp_debug.so)
+LIB_PATH = os.environ.get("FSHARP_LIB") or os.path.join(_HERE, "lib", "libfsharp.so")
 
 FSHARP_F32, FSHARP_BF16 = 0, 1
 VARIANTS = {"posrf": 0, "gerf": 1, "saderf": 2, "aderf": 3, "sderf": 4}
@@ -24,6 +25,7 @@ EXPORTS = [
     "fsharp_params_doubles", "fsharp_stats", "fsharp_fit_params", "fsharp_featurize", "fsharp_attend",
     "fsharp_forward_host", "fsharp_pair_estimate", "fsharp_set_timing", "fsharp_read_timing",
     "fsharp_kernel_name", "fsharp_static_scratch_bytes", "fsharp_featurize_static", "fsharp_kernel_apply",
+    "fsharp_selftest_bounded_wait",
 ]
 
 
@@ -75,6 +77,7 @@ def load_library() -> C.CDLL:
         "fsharp_forward_host": (i32, [vp, vp, vp, vp, vp, dims_p, i32, i32, i32, i32, f32, vp]),
         "fsharp_pair_estimate": (i32, [vp, vp, vp, vp, vp, i64, i32, i32, i32, vp, vp, vp]),
         "fsharp_set_timing": (i32, [vp, i32]),
+        "fsharp_selftest_bounded_wait": (i32, [vp, i32]),
         "fsharp_read_timing": (i32, [vp, i32, C.POINTER(C.c_float), C.POINTER(i32)]),
         "fsharp_kernel_name": (C.c_char_p, [i32]),
         "fsharp_static_scratch_bytes": (C.c_size_t, []),
@@ -171,6 +174,9 @@ class Context:
 
     def workspace_bytes(self) -> int:
         return self.lib.fsharp_workspace_bytes(self._h)
+
+    def selftest_bounded_wait(self, limit_us: int = 1000):
+        _check(self.lib.fsharp_selftest_bounded_wait(self._h, limit_us), "fsharp_selftest_bounded_wait")
 
     def set_timing(self, on: bool):
         _check(self.lib.fsharp_set_timing(self._h, int(on)), "fsharp_set_timing")

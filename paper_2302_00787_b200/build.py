@@ -30,7 +30,23 @@ def _newer(path: str, deps: list[str]) -> bool:
     return all(os.path.getmtime(d) <= t for d in deps)
 
 
-def build(verbose: bool = False, force: bool = False) -> str:
+LIB_DEBUG = os.path.join(LIB_DIR, "libfsharp_debug.so")
+
+
+def build(verbose: bool = False, force: bool = False, debug: bool = False) -> str:
+    """debug=True builds lib/libfsharp_debug.so with -DFSHARP_DEBUG: the tensor-core kernels then check their tile,
+    shared-memory and tensor-memory indices and latch FSHARP_E_INTERNAL when one is out of range."""
+    global OBJ, LIB
+    obj_keep, lib_keep = OBJ, LIB
+    if debug:
+        OBJ, LIB = OBJ + "_debug", LIB_DEBUG
+    try:
+        return _build(verbose, force, ["-DFSHARP_DEBUG"] if debug else [])
+    finally:
+        OBJ, LIB = obj_keep, lib_keep
+
+
+def _build(verbose: bool, force: bool, extra: list) -> str:
     os.makedirs(OBJ, exist_ok=True)
     os.makedirs(LIB_DIR, exist_ok=True)
     nvcc = _nvcc()
@@ -45,7 +61,7 @@ def build(verbose: bool = False, force: bool = False) -> str:
         o = os.path.join(OBJ, src[:-3] + ".o")
         objs.append(o)
         if force or not _newer(o, [s] + headers):
-            cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
+            cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
             jobs.append(cmd)
 
     def run(cmd):
@@ -64,4 +80,4 @@ def build(verbose: bool = False, force: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv))
+    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv, debug="--debug" in sys.argv))

@@ -108,6 +108,7 @@ const char* fsharp_strerror(int code) {
     case FSHARP_E_TIMEOUT: return "bounded device-side wait expired";
     case FSHARP_E_CUDA: return "CUDA call failed";
     case FSHARP_E_LIMIT: return "problem exceeds the fixed scratch of the no-allocation entry point";
+    case FSHARP_E_INTERNAL: return "index check of the debug build failed on the device";
     default: return "unknown error";
   }
 }

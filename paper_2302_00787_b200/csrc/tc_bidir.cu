@@ -289,6 +289,9 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       tcgen05_fence_before();
     };
     for (int it = 0; it < ntiles && alive; it++) {
+      FS_DBG(tile0 + it < total_tiles && (size_t)tile0 * TILE + (size_t)(it + 1) * TILE <= (size_t)Lpad, status);
+      FS_DBG(KV_COL_ACC + hf * TC_NV + TC_NV <= TMEM_COLS && row < TILE, status);
+      FS_DBG(KvSmem::PHI + hf * 2 * TILE_BYTES + TILE_BYTES + row * 128 + 128 <= KvSmem::MISC, status);
       const float cnext = it + 1 < ntiles ? cptr[(size_t)(it + 1) * TILE] : 0.f;     // in flight during this tile
       if (!mbar_wait(&misc->logits_full, it & 1, abortp, status, false)) { alive = false; break; }
       __syncwarp();
@@ -681,6 +684,8 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
       __syncwarp();
     };
     for (int it = 0; it < ntiles && alive; it++) {
+      FS_DBG(tile0 + it < total_tiles && OUT_COL_OUT + TC_NV <= OUT_COL_ONE && OUT_COL_ONE + 8 <= TMEM_COLS, status);
+      FS_DBG(OutSmem::PHI + hf * 2 * TILE_BYTES + TILE_BYTES + row * 128 + 128 <= OutSmem::KVT && row < TILE, status);
       if (!mbar_wait(&misc->logits_full, it & 1, abortp, status, false)) { alive = false; break; }
       __syncwarp();
       tcgen05_fence_after();

@@ -439,6 +439,10 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
     int nlg = 0;
     for (int it = 0; it < ntiles && alive; it++) {
+      FS_DBG(tile0 + it < total_tiles && (size_t)tile0 * TILE + (size_t)(it + 1) * TILE <= (size_t)Lpad, status);
+      FS_DBG(CF_T + hf * TC_NV + TC_NV <= CF_ONE && CF_ONE + 8 <= TMEM_COLS && CF_L + 2 * 64 <= CF_S, status);
+      FS_DBG(pcol[7] + (uint32_t)TC_DV * 128u + 2u <= smem_u32(sm) + CfSmem::KP + 4 * CfSmem::BLK, status);
+      FS_DBG(blk1 + row * 128 + 128 <= sm + CfSmem::KP + 4 * CfSmem::BLK && row < TILE, status);
       const float cnext = it + 1 < ntiles ? cptr[(size_t)(it + 1) * TILE] : 0.f;     // in flight during this tile
       uint32_t v[128];
       // ---- key logits, first half

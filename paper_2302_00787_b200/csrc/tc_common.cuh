@@ -59,14 +59,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;
 
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          bool honor_abort = true) {
+                                          bool honor_abort = true, long long limit_cycles = WAIT_LIMIT_CYCLES) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 255u) == 0u) {
       if (honor_abort && *abort_flag) return false;
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      if (clock64() - t0 > limit_cycles) {
         *abort_flag = 1;
         atomicExch(status, -8 /* FSHARP_E_TIMEOUT */);
         return false;
@@ -75,6 +75,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   }
   return true;
 }
+
+// Index checks of the debug build (-DFSHARP_DEBUG; the memory checker is not available on every machine): a failed
+// check latches FSHARP_E_INTERNAL in the status word and the access still happens only if it is in range of the
+// block's own shared memory / tensor memory (the callers clamp); nothing traps.
+#ifdef FSHARP_DEBUG
+#define FS_DBG(cond, status) do { if (!(cond)) atomicExch((status), -11 /* FSHARP_E_INTERNAL */); } while (0)
+#else
+#define FS_DBG(cond, status) ((void)0)
+#endif
 
 // ---------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }

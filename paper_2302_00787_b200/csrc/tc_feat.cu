@@ -156,6 +156,8 @@ tc_feat_kernel(const __grid_constant__ CUtensorMap tmX, const uint8_t* __restric
     const float* cptr = crow + (size_t)bh * Lpad + (size_t)tile0 * TILE + row;
     float* phib = phi + (size_t)bh * L * TC_M;
     for (int it = 0; it < ntiles; it++) {
+      FS_DBG(tile0 + it < total_tiles && (size_t)tile0 * TILE + (size_t)(it + 1) * TILE <= (size_t)Lpad && row < TILE, status);
+      FS_DBG(FT_COL_LOGITS + TC_M <= FT_COL_ONE && FT_COL_ONE + 8 <= TMEM_COLS, status);
       const float ci = cptr[(size_t)it * TILE];
       if (!mbar_wait(&misc->logits_full, it & 1, abortp, status, false)) break;
       __syncwarp();

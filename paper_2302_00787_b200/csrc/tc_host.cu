@@ -79,3 +79,35 @@ int fs_tc_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, c
   if (causal) return fs_tc_causal(ctx, Q, K, V, dm, images, flags, Y, ws);
   return fs_tc_bidir(ctx, Q, K, V, dm, images, flags, Y, ws);
 }
+
+// ------------------------------------------------------------------------------------------
+// self-test of the bounded waits
+// ------------------------------------------------------------------------------------------
+namespace {
+__global__ void __launch_bounds__(32)
+bounded_wait_selftest_kernel(long long limit_cycles, int* __restrict__ status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    tc::mbar_init(&bar, 1);
+    abort_flag = 0;
+    tc::fence_barrier_init();
+  }
+  __syncwarp();
+  // nothing ever arrives on `bar`: the wait runs into its limit, latches FSHARP_E_TIMEOUT and returns false
+  const bool ok = tc::mbar_wait(&bar, 0, &abort_flag, status, false, limit_cycles);
+  if (ok) atomicExch(status, FSHARP_E_INTERNAL);       // (a wait that returned true here would be a bug of mbar_wait)
+}
+}  // namespace
+
+extern "C" int fsharp_selftest_bounded_wait(fsharp_ctx* ctx, int limit_us) {
+  if (!ctx) return FSHARP_E_BADARG;
+  if (limit_us < 1 || limit_us > 100000) return FSHARP_E_BADARG;
+  FS_CUDA_OK(cudaSetDevice(ctx->device));
+  int khz = 0;
+  FS_CUDA_OK(cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, ctx->device));
+  const long long cycles = (long long)limit_us * (long long)(khz > 0 ? khz : 1965000) / 1000;
+  bounded_wait_selftest_kernel<<<1, 32, 0, ctx->stream>>>(cycles, ctx->d_status);
+  FS_LAUNCH_CHECK(ctx);
+  return FSHARP_OK;
+}

@@ -510,6 +510,54 @@ def test_unnormalised_operator_matches_definition(ctx, w, alpha):
     assert ei.value.code == -2
 
 
+def test_bounded_wait_runs_out_and_the_context_stays_usable(ctx):
+    """Every device-side wait is bounded.  The self-test kernel waits 2 ms on a barrier that nothing completes: the
+    wait gives up, the kernel returns, the status word reports the time-out, and the next call works."""
+    w = W["cfg3"].scaled(B=1, H=1, L=256)
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    _, pr = gpu_fit(ctx, dQ, dK, w.d, w.variant)
+    ctx.selftest_bounded_wait(2000)
+    assert ctx.status() == -8                     # FSHARP_E_TIMEOUT, latched once ...
+    assert ctx.status() == 0                      # ... and cleared by the read
+    Y = host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=True, chunk=128))
+    assert ctx.status() == 0
+    ref = oracle_unit(Q, K, V, Om, pr.cpu().numpy()[0], w.d, 0, 0, True)
+    assert rel_err(Y[0, 0], ref) < TOL["bf16"]
+    with pytest.raises(fb.FsharpError):
+        ctx.selftest_bounded_wait(0)
+
+
+def test_debug_build_index_checks_stay_silent():
+    """The build with -DFSHARP_DEBUG checks tile, shared-memory and tensor-memory indices inside the tensor-core
+    kernels and latches an error instead of faulting.  Run small cases of every tensor-core kernel through it in a
+    process of its own (another build of the same library): no check fires and the results are finite."""
+    import subprocess, sys, os
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    lib = os.path.join(root, "paper_2302_00787_b200", "lib", "libfsharp_debug.so")
+    if not os.path.exists(lib):
+        from paper_2302_00787_b200 import build as b
+        b.build(debug=True)
+    script = """
+import torch
+from paper_2302_00787_b200 import binding as fb, workloads as wl
+assert fb.LIB_PATH.endswith('libfsharp_debug.so')
+ctx = fb.Context(0)
+for w in (wl.WORKLOADS['cfg2'].scaled(B=2, H=2, L=300), wl.WORKLOADS['cfg3'].scaled(B=1, H=3, L=1024),
+          wl.WORKLOADS['cfg3b'].scaled(B=1, H=2, L=640), wl.WORKLOADS['cfg3'].scaled(B=1, H=150, L=640)):
+    Q, K, V = wl.make_qkv(w); Om = wl.make_omega(w)
+    dQ, dK, dV = (torch.from_numpy(a).cuda().to(torch.bfloat16) for a in (Q, K, V)); dOm = torch.from_numpy(Om).cuda()
+    st = ctx.fsharp_stats(dQ, dK); pr = ctx.fsharp_fit_params(st, w.d, w.variant)
+    Y = ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=w.causal, chunk=w.chunk)
+    phi, ls = ctx.fsharp_featurize(dK, dOm, pr, 2, stab=fb.STAB_ROW)
+    assert ctx.status() == 0, w
+    assert torch.isfinite(Y.float()).all() and torch.isfinite(phi).all()
+print('debug build ok')
+"""
+    env = dict(os.environ, FSHARP_LIB=lib, PYTHONPATH=root)
+    r = subprocess.run([sys.executable, "-c", script], env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and "debug build ok" in r.stdout, r.stdout + r.stderr
+
+
 def test_variance_study_batch_many_pairs_many_draws(ctx):
     """The variance-study batch at 2^16 pairs and 32 draws (a multi-wave grid for the estimates, the grid-stride
     loops of the per-pair variance and of the pooling): estimates on sampled pairs for every draw, closed-form
