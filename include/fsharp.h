@@ -90,8 +90,10 @@ typedef struct {
 int fsharp_create(fsharp_ctx** out, int device, void* stream);
 int fsharp_destroy(fsharp_ctx* ctx);
 int fsharp_set_stream(fsharp_ctx* ctx, void* stream);
-/* Forces a kernel family for fsharp_attend (FSHARP_IMPL_*).  AUTO picks the
- * tensor-core path when the shape allows it (bf16, d = dv in {64, 128}). */
+/* Forces a kernel family for fsharp_attend and fsharp_featurize (FSHARP_IMPL_*).  AUTO picks the
+ * tensor-core kernels when the shape allows it: bf16, d = dv = 64, M = 256 (attend, bidirectional or causal with
+ * Lq == Lk; featurize with a row shift or none); everything else runs on the fp32 kernels.  TENSOR refuses
+ * (FSHARP_E_SHAPE) what the tensor-core kernels do not cover. */
 int fsharp_set_impl(fsharp_ctx* ctx, int impl);
 /* Synchronises the stream, then returns the latched device status in *code
  * (0 or a negative FSHARP_E_*), and clears it. */
@@ -140,9 +142,14 @@ int fsharp_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dim
 /* Closed-form minimisers of the shifted log-variance objective (Section 3.1):
  * PosRF and GERF (Section 2.3 / 3.1), SADERF (Section 4.3), ADERF (Theorem 4.2),
  * SDERF (Theorem 4.3), all through Lemma A.1's scalar map.  The symmetric
- * eigenproblems are solved on the device by a cyclic Jacobi method in fp64, one
- * thread block per group.  ADERF uses eig(M1) and eig(L1^1/2 Q1^T M2 Q1 L1^1/2),
- * whose eigenvectors and eigenvalues are U and Sigma^2 of the theorem's SVD.
+ * eigenproblems are solved on the device in fp64, one thread block per group
+ * (d <= 64: tridiagonalisation, Sturm multisection and twisted-factorisation vectors,
+ * confirmed by a cyclic Jacobi solver; d = 128: the Jacobi solver).  ADERF factors
+ * M1 = L L^T (Cholesky) and solves one eigenproblem, of L^T M2 L: its eigenvectors
+ * and eigenvalues are U and Sigma^2 of the theorem's SVD for the factor L^T of M1
+ * (any factor F with F^T F = M1 gives the same B1, B2).  The literal B is "one of
+ * the solutions" of the theorems (eigenvector signs and rotations inside equal
+ * eigenvalues are free); there is no second, canonical form of the parameters.
  * ridge >= 0 adds ridge * tr(M)/d * I to M1 and M2 first (0 = the paper's formulas).
  * stats: device, G groups.  params: device, G * fsharp_params_doubles(d). */
 int fsharp_fit_params(fsharp_ctx* ctx, const double* stats, int G, int d, int variant,

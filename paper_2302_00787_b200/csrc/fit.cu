@@ -1,5 +1,9 @@
-// Closed-form parameter fits (Section 3.1, Section 4.3, Theorems 4.2 and 4.3, Lemma A.1)
-// with an fp64 cyclic Jacobi eigensolver, one thread block per parameter group.
+// Closed-form parameter fits (Section 3.1, Section 4.3, Theorems 4.2 and 4.3, Lemma A.1), fp64, one thread block
+// per parameter group.  Symmetric eigenproblems, d <= 64: Householder tridiagonalisation, Sturm-count multisection,
+// one vector per eigenvalue from the twisted factorisation, reflectors applied back, one symmetric orthogonalisation;
+// a cyclic Jacobi solver then confirms convergence (or completes it).  d = 128: the Jacobi solver alone.
+// ADERF factors M1 by Cholesky (M1 = L L^T) and solves ONE eigenproblem, of L^T M2 L (Theorem 4.2's U and Sigma^2
+// for the factor L^T of M1).
 #include "common.cuh"
 
 namespace {

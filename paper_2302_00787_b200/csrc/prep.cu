@@ -11,7 +11,8 @@ namespace {
 
 constexpr int PREP_THREADS = 256;
 constexpr int PREP_MB = 64;                   // features per block
-constexpr int PREP_LDO = PREP_MB + 4;         // row stride of the transposed Omega chunk (keeps 16-byte alignment)
+constexpr int PREP_LDO = PREP_MB + 1;         // row stride of the transposed Omega chunk: odd, so that the transposing stores
+                                              // (32 consecutive rows, one column) fall into 32 different banks
 
 // One block = one (group, role, chunk of 64 features) with role 0, 1: W of side 1, 2; role 2: a (the same for both
 // sides, written for both); role 3: C, the scalars and the flags of side blockIdx.z + 1.  Omega's chunk
@@ -90,8 +91,8 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
       for (int v = 0; v < NC; v++) acc[u][v] = 0.f;
 #pragma unroll 4
     for (int i = 0; i < d; i++) {
-      const float4 a4 = *reinterpret_cast<const float4*>(Ot + i * PREP_LDO + 4 * ty);
-      const float a[4] = {a4.x, a4.y, a4.z, a4.w};
+      const float* ap = Ot + i * PREP_LDO + 4 * ty;       // (two addresses per warp: broadcast reads)
+      const float a[4] = {ap[0], ap[1], ap[2], ap[3]};
       float b[NC];
       if (NC >= 4) {
 #pragma unroll
@@ -150,9 +151,11 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
     }
     return;
   }
-  // C = gamma I exactly?
+  // C = gamma I exactly?  The operand images (row j, column i = C[i][j], 128-byte swizzle) are put together in shared
+  // memory and leave in 16-byte pieces: element-wise stores of a transposed 2-byte layout would touch a sector each.
   int cscalar = 1, lo_nonzero = 0;
   const double gamma = Cm[0];
+  uint8_t* simg = reinterpret_cast<uint8_t*>(stage);             // [hi image | lo image], IMG_C_BYTES each (d = 64 only)
   for (int e0 = tid; e0 < d * d; e0 += 8 * PREP_THREADS) {
     double cv[8];
 #pragma unroll
@@ -169,16 +172,21 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
       if (i == j ? (cv[q] != gamma) : (cv[q] != 0.0)) cscalar = 0;
       if (images != nullptr) {
         // log2e * qk_scale^2 * C[i][j] goes to row j, column i of the MMA operand
-        uint8_t* img = images + ((size_t)g * 2 + (side - 1)) * tcl::IMG_BYTES;
         const float v = (float)cv[q] * (FS_LOG2E * qk_scale * qk_scale);
         const __nv_bfloat16 hi = __float2bfloat16_rn(v), lo = __float2bfloat16_rn(v - __bfloat162float(hi));
         if (__bfloat162float(lo) != 0.f) lo_nonzero = 1;
-        *reinterpret_cast<__nv_bfloat16*>(img + tcl::IMG_CHI + tc::sw128_offset(j, i)) = hi;
-        *reinterpret_cast<__nv_bfloat16*>(img + tcl::IMG_CLO + tc::sw128_offset(j, i)) = lo;
+        *reinterpret_cast<__nv_bfloat16*>(simg + tc::sw128_offset(j, i)) = hi;
+        *reinterpret_cast<__nv_bfloat16*>(simg + tcl::IMG_C_BYTES + tc::sw128_offset(j, i)) = lo;
       }
     }
   }
   lo_nonzero = __syncthreads_or(lo_nonzero);
+  if (images != nullptr) {
+    // the two images are adjacent in the operand image block as well (IMG_CLO = IMG_CHI + IMG_C_BYTES)
+    uint4* dst = reinterpret_cast<uint4*>(images + ((size_t)g * 2 + (side - 1)) * tcl::IMG_BYTES + tcl::IMG_CHI);
+    const uint4* src = reinterpret_cast<const uint4*>(simg);
+    for (int e = tid; e < (int)(2 * tcl::IMG_C_BYTES / 16); e += PREP_THREADS) dst[e] = src[e];
+  }
   redi[tid] = cscalar;
   __syncthreads();
   for (int s = PREP_THREADS / 2; s > 0; s >>= 1) {
