@@ -539,9 +539,9 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
       }
       OUT_WAIT(&misc->conv[st], (it / OUT_STAGES) & 1);
       if (it > 0) OUT_WAIT(&misc->logits_free, (it - 1) & 1);
-      // The tensor pipe runs MMAs in the order they were issued: the last contraction steps of tile it - 2, which
-      // the epilogue is about to wait for, go before the next tile's logits, which nobody needs for a whole tile.
-      if (it > 1) OUT_WAIT(&misc->phi_free, (it - 2) & 1);
+      // (Every barrier this warp waits on is one whose next phase cannot complete before this warp has moved on: a
+      // wait by parity on a barrier that may run two phases ahead of its waiter would never end.  phi_free is such
+      // a barrier for this warp, so the logits are not ordered behind the contraction of an earlier tile.)
       tcgen05_fence_after();
       issue_logits(st);
     }
