@@ -15,8 +15,8 @@
 //   phi(K) -> bf16 tile in shared memory (the B operand of the scores, the A operand of the state update)
 //   phi(Q) -> bf16, written back over its own logits [L] and read from there as the A operand
 //   [scores | inter-tile output] = phi(Q) [phi(K)^T | bf16(T)]      one MMA stream, N = 208   [S: 128][O: 80]
-//   scores masked (key <= query), rounded to bf16 over their own columns, row sums kept
-//   O[:, :64] += masked scores (from tensor memory) V                                         [O]
+//   scores masked (key <= query), rounded to bf16 over their own columns
+//   O += masked scores (from tensor memory) [V | 1]: column 64 collects the denominators       [O]
 //   T += phi(K)^T [V | 1], 128 features per accumulator                                       [T: 2 x 80]
 //   bf16(T) for the next tile: the accumulators are read back and written to shared memory
 // The token tiles are converted from bf16 to fp16 in shared memory (exact for |x| in [2^-14, 65504]), so the
@@ -34,11 +34,11 @@ using namespace tcl;
 
 namespace {
 
-// Warps 0-3 are the producer warpgroup (0: TMA copies, 1: all MMAs, 2 and 3: token tiles to fp16), warps 4-11
-// the epilogue.  The single MMA-issuing warp shares its scheduler with two epilogue warps that always have
-// instructions ready; it sits in the lowest warp slots of the block.
+// Warps 0-3 are the producer warpgroup (0: TMA copies, 1: all MMAs; 0, 2 and 3: token tiles to fp16), warps 4-11
+// the epilogue.  Every scheduler thus carries one producer warp and two epilogue warps: the epilogue warps of a
+// tile meet at barriers several times per tile, so the slowest scheduler sets the pace.
 constexpr int CF_WARP_TMA = 0, CF_WARP_MMA = 1, CF_WARP_CVT0 = 2, CF_PRODUCER_WARPS = 4;
-constexpr int CVT_THREADS = 64;
+constexpr int CVT_THREADS = 96;       // warps 0, 2 and 3 (each shares its scheduler with two epilogue warps; so does the MMA warp)
 // Of every four pairs of exponentials, this many are evaluated on the multiply-add pipe (exp2_poly2), the others
 // by the special-function unit, whose 16 results per clock would otherwise bound the kernel.
 constexpr int CF_POLY_PAIRS = 1;
@@ -51,8 +51,8 @@ struct CfSmem {
   // operand of 208 rows covers both
   static constexpr uint32_t W1 = 0, W2 = IMG_W_BYTES, X = 2 * IMG_W_BYTES, V = X + TILE_BYTES, ONES = V + TILE_BYTES,
                             KP = ONES + TILE_BYTES, BLK = TILE_BYTES + KVT_BLOCK_BYTES,
-                            // the row maxima of the query logits and the row sums of the masked scores are never alive together
-                            ROWMAX = KP + 4 * BLK, RSUM = ROWMAX,
+                            // row maxima of the query logits, exchanged between the two threads of a row: [2][128] floats
+                            ROWMAX = KP + 4 * BLK,
                             // per-feature term as an MMA operand: [256 features x 16] fp16, no swizzle (8 x 16-byte core
                             // matrices: the two 16-byte K pieces of a row 128 bytes apart, 8-row groups 256 bytes apart)
                             A2OP = ROWMAX + 2 * TILE * 4, A2OP_BYTES = TC_M * 32, MISC = A2OP + A2OP_BYTES, TOTAL = MISC + 256;
@@ -62,7 +62,8 @@ static_assert(CfSmem::TOTAL + 1024 <= 232448, "shared memory budget");
 
 struct CfMisc {
   uint64_t const_bar, x_full, x_ready, x_free, v_full, v_free, lg_full, lg_free, phik_full[2], phiq_full[5], p_full,
-      s_ready, sm_full, o_ready, o_free, st_ready;
+      s_ready, sm_full, o_ready, o_free, st_ready,
+      stage_free;   // the output rows staged in the token tile have been read by their copies to global memory
   // meeting points of the epilogue warps (the two warps of a row quarter; all eight): mbarriers, so that these
   // waits are bounded like every other
   uint64_t pair_bar[4], all_bar;
@@ -77,15 +78,14 @@ constexpr uint32_t CF_L = 0, CF_S = 128, CF_O = 256, CF_T = 336, CF_ONE = 496;
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                 const __grid_constant__ CUtensorMap tmV, const uint8_t* __restrict__ images,
+                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmY,
+                 const uint8_t* __restrict__ images,
                  const float* __restrict__ crow, const float* __restrict__ partial, const float* __restrict__ shifts,
-                 int nsplit1, int H, int pool, int L, int Lpad, int tiles_per_seg,
-                 __nv_bfloat16* __restrict__ Y, TensorAddr ay, int* __restrict__ status) {
+                 int nsplit1, int H, int pool, int L, int Lpad, int tiles_per_seg, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   CfMisc* misc = reinterpret_cast<CfMisc*>(sm + CfSmem::MISC);
   float* rowmax = reinterpret_cast<float*>(sm + CfSmem::ROWMAX);   // [half][row]
-  float* rsum = reinterpret_cast<float*>(sm + CfSmem::RSUM);       // [half][row]: row sums of the rounded masked scores
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int seg = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
   const int g = pool == FSHARP_POOL_PER_BH ? bh : h;
@@ -114,6 +114,7 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     mbar_init(&misc->o_ready, 1);
     mbar_init(&misc->o_free, EPI_THREADS / 32);
     mbar_init(&misc->st_ready, 1);
+    mbar_init(&misc->stage_free, EPI_THREADS / 32);
     for (int i = 0; i < 4; i++) mbar_init(&misc->pair_bar[i], 2);
     mbar_init(&misc->all_bar, EPI_THREADS / 32);
     for (int j = 0; j < 3; j++) misc->chunk_max[j] = f2ord(-INFINITY);
@@ -150,39 +151,69 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
   if (warp < CF_PRODUCER_WARPS) {
     regs_release<CF_REGS_PRODUCER>();
+    // bf16 -> fp16 of token tile n, in place (16-byte pieces keep their swizzled positions); t: 0 .. CVT_THREADS - 1
+    auto convert_tile = [&](int n, int t) -> bool {
+      if (!__all_sync(0xffffffffu, mbar_wait(&misc->x_full, n & 1, abortp, status, false))) return false;    // warp-uniform
+      uint4* xt = reinterpret_cast<uint4*>(sm + CfSmem::X);
+#pragma unroll 4
+      for (int i = t; i < (int)(TILE_BYTES / 16); i += CVT_THREADS) {
+        uint4 u = xt[i];
+        u.x = pack_f16(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
+        u.y = pack_f16(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
+        u.z = pack_f16(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u));
+        u.w = pack_f16(__uint_as_float(u.w << 16), __uint_as_float(u.w & 0xffff0000u));
+        xt[i] = u;
+      }
+      fence_proxy_async_smem();
+      mbar_arrive_warp(&misc->x_ready, lane);
+      return true;
+    };
     if (warp == CF_WARP_TMA) {
+      // The whole warp walks the schedule (it also converts a third of every token tile); lane 0 issues the copies.
       if (lane == 0) {
         prefetch_tmap(&tmQ);
         prefetch_tmap(&tmK);
         prefetch_tmap(&tmV);
+        prefetch_tmap(&tmY);
         mbar_expect_tx(&misc->const_bar, 2 * IMG_W_BYTES);
         bulk_load(sm + CfSmem::W1, img1 + IMG_WH, IMG_W_BYTES, &misc->const_bar);
         bulk_load(sm + CfSmem::W2, img2 + IMG_WH, IMG_W_BYTES, &misc->const_bar);
-        // One token tile in shared memory serves keys and queries in turn: load 2 it is the key tile of tile it
-        // (free once the second half of the key logits has been computed), load 2 it + 1 its query tile.
-        int nx = 0, nv = 0;
-        bool okp = true;
-        for (int it = 0; it < ntiles && okp; it++) {
-          const int tok = (tile0 + it) * TILE;
-          if (nx > 0 && !mbar_wait(&misc->x_free, (nx - 1) & 1, abortp, status)) { okp = false; break; }
+      }
+      // One token tile in shared memory serves keys and queries in turn: load 2 it is the key tile of tile it
+      // (free once the second half of the key logits has been computed), load 2 it + 1 its query tile.
+      int nx = 0, nv = 0;
+      for (int it = 0; it < ntiles; it++) {
+        const int tok = (tile0 + it) * TILE;
+        if (nx > 0 && !__all_sync(0xffffffffu, mbar_wait(&misc->x_free, (nx - 1) & 1, abortp, status))) break;
+        // (between its query logits and this load the token tile staged the output rows of tile it - 2)
+        if (it >= 2 && !__all_sync(0xffffffffu, mbar_wait(&misc->stage_free, (it - 2) & 1, abortp, status))) break;
+        if (lane == 0) {
           mbar_expect_tx(&misc->x_full, TILE_BYTES);
           tma_load_4d(sm + CfSmem::X, &tmK, &misc->x_full, 0, tok, h, b);
-          nx++;
           if (it + 1 < ntiles) {             // the next tile's operands: into L2 while this one is worked on
             tma_prefetch_4d(&tmK, 0, tok + TILE, h, b);
             tma_prefetch_4d(&tmQ, 0, tok + TILE, h, b);
             tma_prefetch_4d(&tmV, 0, tok + TILE, h, b);
           }
-          if (nv > 0 && !mbar_wait(&misc->v_free, (nv - 1) & 1, abortp, status)) { okp = false; break; }
+        }
+        nx++;
+        if (!convert_tile(nx - 1, lane)) break;
+        if (nv > 0 && !__all_sync(0xffffffffu, mbar_wait(&misc->v_free, (nv - 1) & 1, abortp, status))) break;
+        if (lane == 0) {
           mbar_expect_tx(&misc->v_full, TILE_BYTES);
           tma_load_4d(sm + CfSmem::V, &tmV, &misc->v_full, 0, tok, h, b);
-          nv++;
-          if (!mbar_wait(&misc->x_free, (nx - 1) & 1, abortp, status)) { okp = false; break; }
+        }
+        nv++;
+        if (!__all_sync(0xffffffffu, mbar_wait(&misc->x_free, (nx - 1) & 1, abortp, status))) break;
+        if (lane == 0) {
           mbar_expect_tx(&misc->x_full, TILE_BYTES);
           tma_load_4d(sm + CfSmem::X, &tmQ, &misc->x_full, 0, tok, h, b);
-          nx++;
         }
-        // no copy of this block may still be in flight when it exits
+        nx++;
+        if (!convert_tile(nx - 1, lane)) break;
+      }
+      // no copy of this block may still be in flight when it exits
+      if (lane == 0) {
         mbar_wait(&misc->const_bar, 0, abortp, status, false);
         if (nx > 0) mbar_wait(&misc->x_full, (nx - 1) & 1, abortp, status, false);
         if (nv > 0) mbar_wait(&misc->v_full, (nv - 1) & 1, abortp, status, false);
@@ -194,7 +225,7 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         constexpr uint32_t ID_LOGITS = idesc_f16(128, 128, 0, 0);            // X Wh^T, 128 features
         constexpr uint32_t ID_STATE = idesc_bf16(128, TC_NV, 1, 1);          // phi(K)_h^T [V | 1]
         constexpr uint32_t ID_SO = idesc_bf16(128, 128 + TC_NV, 0, 0);       // phi(Q) [phi(K)^T | bf16(T)]
-        constexpr uint32_t ID_SV = idesc_bf16(128, TC_DV, 0, 1);             // masked scores x V
+        constexpr uint32_t ID_SV = idesc_bf16(128, TC_NV, 0, 1);             // masked scores x [V | 1]: the ones column adds the row sums
         const uint64_t dX = smem_desc(smem_u32(sm + CfSmem::X), 16, 1024, SWZ_128B);
         const uint64_t dW1 = smem_desc(smem_u32(sm + CfSmem::W1), 16, 1024, SWZ_128B);
         const uint64_t dW2 = smem_desc(smem_u32(sm + CfSmem::W2), 16, 1024, SWZ_128B);
@@ -314,23 +345,10 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #undef CF_WAIT
       }
     } else {
-      // ---------------- bf16 -> fp16 of the token tile, in place (16-byte pieces keep their swizzled positions)
-      const int t = (warp - CF_WARP_CVT0) * 32 + lane;
-      for (int n = 0; n < 2 * ntiles; n++) {
-        if (!mbar_wait(&misc->x_full, n & 1, abortp, status, false)) break;
-        uint4* xt = reinterpret_cast<uint4*>(sm + CfSmem::X);
-#pragma unroll 4
-        for (int i = 0; i < (int)(TILE_BYTES / 16) / CVT_THREADS; i++) {
-          uint4 u = xt[t + i * CVT_THREADS];
-          u.x = pack_f16(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
-          u.y = pack_f16(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
-          u.z = pack_f16(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u));
-          u.w = pack_f16(__uint_as_float(u.w << 16), __uint_as_float(u.w & 0xffff0000u));
-          xt[t + i * CVT_THREADS] = u;
-        }
-        fence_proxy_async_smem();
-        mbar_arrive_warp(&misc->x_ready, lane);
-      }
+      // ---------------- bf16 -> fp16 of the token tiles, with the copying warp
+      const int t = (warp - CF_WARP_CVT0 + 1) * 32 + lane;
+      for (int n = 0; n < 2 * ntiles; n++)
+        if (!convert_tile(n, t)) break;
     }
   } else {
     regs_acquire<CF_REGS_EPILOGUE>();
@@ -341,7 +359,6 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int row = q * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
     const int m = hf * 128 + row;
-    __nv_bfloat16* Yb = Y + b * ay.sb + h * ay.sh;
     uint8_t* blk0 = sm + CfSmem::KP + hf * CfSmem::BLK;              // phi(K) block hf
     uint8_t* blk1 = sm + CfSmem::KP + (2 + hf) * CfSmem::BLK;        // phi(K) block 2 + hf
     // bf16(T): column m of T is column m % 64 of the 80-row block of feature block m / 64; row n of a 128-byte-swizzled
@@ -401,24 +418,24 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const float* cptr = crow + (size_t)bh * Lpad + (size_t)tile0 * TILE + row;
     float cj = cptr[0];
 
-    // Y rows of tile j (all its MMAs have completed): 32 of the 64 columns per thread
+    // Y rows of tile j (all its MMAs have completed): 32 of the 64 columns per thread.  A warp's 32 rows x 64 bytes are
+    // staged in its eighth of the token tile (idle between the query logits of a tile and the next tile's keys) with
+    // the 64-byte swizzle and leave as one TMA store, which also drops the rows past the end of the sequence.
     auto write_out = [&](int j) {
       __syncwarp();
       tcgen05_fence_after();
-      uint32_t n0[32], d0[16];
+      uint32_t n0[32], d0[8];
       tmem_ld16(lane_addr + CF_O + hf * 32, reinterpret_cast<uint32_t(&)[16]>(n0[0]));
       tmem_ld16(lane_addr + CF_O + hf * 32 + 16, reinterpret_cast<uint32_t(&)[16]>(n0[16]));
-      tmem_ld16(lane_addr + CF_O + TC_DV, d0);
+      tmem_ld8(lane_addr + CF_O + TC_DV, d0);
       tmem_wait_ld();
       tcgen05_fence_before();
       mbar_arrive_warp(&misc->o_free, lane);
-      const float den = __uint_as_float(d0[0]) + rsum[row] + rsum[TILE + row];
-      const int64_t r0 = (int64_t)(tile0 + j) * TILE + q * 32;       // first row of this warp
+      const float den = __uint_as_float(d0[0]);
+      const int r0 = (tile0 + j) * TILE + q * 32;                    // first row of this warp
       if (r0 + lane < L && (!(den > 0.f) || !isfinite(den))) atomicExch(status, FSHARP_E_NONFINITE);
       const float inv = 1.f / den;
-      // The thread's 64 bytes go through shared memory so that a store instruction of the warp covers 8 rows x 64
-      // contiguous bytes.  The staging area is the part of the phi(K) block that this warp itself writes next.
-      uint8_t* stg = blk0 + q * 4096;
+      uint8_t* stg = sm + CfSmem::X + (warp - CF_PRODUCER_WARPS) * 2048;
 #pragma unroll
       for (int i = 0; i < 4; i++) {
         uint32_t o[4];
@@ -427,14 +444,12 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           o[e] = pack_bf16(inv * __uint_as_float(n0[8 * i + 2 * e]), inv * __uint_as_float(n0[8 * i + 2 * e + 1]));
         *reinterpret_cast<uint4*>(stg + lane * 64 + ((i ^ ((lane >> 1) & 3)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
       }
+      fence_proxy_async_smem();
       __syncwarp();
-#pragma unroll
-      for (int i = 0; i < 4; i++) {
-        const int rr = (lane >> 2) + 8 * i, cw = lane & 3;
-        const uint4 val = *reinterpret_cast<const uint4*>(stg + rr * 64 + ((cw ^ ((rr >> 1) & 3)) << 4));
-        if (r0 + rr < L) *reinterpret_cast<uint4*>(Yb + (r0 + rr) * ay.sl + hf * 32 + cw * 8) = val;
+      if (lane == 0) {
+        tma_store_4d(&tmY, stg, hf * 32, r0, h, b);
+        bulk_commit();
       }
-      __syncwarp();
     };
 
     int nlg = 0;
@@ -455,13 +470,17 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       tmem_wait_ld();
       tcgen05_fence_before();
       mbar_arrive_warp(&misc->lg_free, lane);
-      // ---- while the second half is computed: the previous tile's output.  Its state update has completed
-      // (nothing reads the previous phi(K) tile any more), and so has its masked-score product.
-      if (it > 0) {
-        if (!mbar_wait(&misc->st_ready, (it - 1) & 1, abortp, status, false)) { alive = false; break; }
-        if (!mbar_wait(&misc->o_ready, (it - 1) & 1, abortp, status, false)) { alive = false; break; }
-        write_out(it - 1);
+      // ---- while the second half is computed: the maximum of the first
+      float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int i = 0; i < 64; i += 8) {
+        mxp[0] = max3(mxp[0], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+        mxp[1] = max3(mxp[1], __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+        mxp[2] = max3(mxp[2], __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+        mxp[3] = max3(mxp[3], __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
       }
+      // the previous tile's state update has completed: nothing reads the previous phi(K) tile any more
+      if (it > 0 && !mbar_wait(&misc->st_ready, (it - 1) & 1, abortp, status, false)) { alive = false; break; }
       // ---- key logits, second half
       if (!mbar_wait(&misc->lg_full, nlg & 1, abortp, status, false)) { alive = false; break; }
       nlg++;
@@ -476,9 +495,8 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       // ---- exact maximum of the tile's exponents, one value for the block
       float tm;
       {
-        float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int i = 0; i < 128; i += 8) {
+        for (int i = 64; i < 128; i += 8) {
           mxp[0] = max3(mxp[0], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
           mxp[1] = max3(mxp[1], __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
           mxp[2] = max3(mxp[2], __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
@@ -514,7 +532,8 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         tcgen05_fence_before();
         s = tm;
       }
-      // ---- phi(K): 2^(exponent - s), bf16, 64 features at a time
+      // ---- phi(K): 2^(exponent - s), bf16, 64 features at a time.  Rows past the end of the sequence (last tile only)
+      // are not zeroed: the mask removes their scores, and the state after the last tile is not used.
       {
         const float rc = cj - s;
 #pragma unroll
@@ -535,7 +554,6 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 p[j] = pack_bf16(ex2(__uint_as_float(e0)), ex2(__uint_as_float(e1)));
               }
             }
-            if (!valid) p[0] = p[1] = p[2] = p[3] = 0u;
             *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
           }
           fence_proxy_async_smem();
@@ -585,6 +603,12 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       tmem_wait_ld();
       tcgen05_fence_before();
       mbar_arrive_warp(&misc->lg_free, lane);
+      // ---- the previous tile's output: its masked-score product has long completed (the scores of this tile wait for
+      // it), and the query logits just taken were the last readers of the token tile
+      if (it > 0) {
+        if (!mbar_wait(&misc->o_ready, (it - 1) & 1, abortp, status, false)) { alive = false; break; }
+        write_out(it - 1);
+      }
       float mx;
       {
         float mxp[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -602,6 +626,10 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         sync_pair();
         if (!alive) break;
         mx = fmaxf(mx, rowmax[(hf ^ 1) * TILE + row]);
+      }
+      if (it > 0) {                    // the staged rows have been read: the token tile may take the next keys
+        if (lane == 0) bulk_wait_read0();
+        mbar_arrive_warp(&misc->stage_free, lane);
       }
       // ---- phi(Q): 2^(exponent - row maximum), bf16 pairs over the logits' columns: block fb at columns 32 fb
 #pragma unroll
@@ -650,29 +678,27 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
     after_queries:
       if (!alive) break;
-      // ---- scores: mask (key <= query), round to bf16 over their own columns, keep the row sums
+      // ---- scores: mask (key <= query) and round to bf16 over their own columns (their row sums come out of the
+      // product with [V | 1])
       if (!mbar_wait(&misc->s_ready, it & 1, abortp, status, false)) { alive = false; break; }
       __syncwarp();
       tcgen05_fence_after();
       {
         uint32_t pm[32];
-        float sum = 0.f;
 #pragma unroll
-        for (int cc = 0; cc < 4; cc++) {
-          uint32_t t[16];
-          tmem_ld16(lane_addr + CF_S + hf * 64 + cc * 16, t);
+        for (int cc = 0; cc < 2; cc++) {
+          uint32_t t[32];
+          tmem_ld16(lane_addr + CF_S + hf * 64 + cc * 32, reinterpret_cast<uint32_t(&)[16]>(t[0]));
+          tmem_ld16(lane_addr + CF_S + hf * 64 + cc * 32 + 16, reinterpret_cast<uint32_t(&)[16]>(t[16]));
           tmem_wait_ld();
 #pragma unroll
-          for (int j = 0; j < 8; j++) {
-            const int k0 = hf * 64 + cc * 16 + 2 * j;
+          for (int j = 0; j < 16; j++) {
+            const int k0 = hf * 64 + cc * 32 + 2 * j;
             const float s0 = k0 <= row ? __uint_as_float(t[2 * j]) : 0.f;
             const float s1 = k0 + 1 <= row ? __uint_as_float(t[2 * j + 1]) : 0.f;
-            const uint32_t pk = pack_bf16(s0, s1);
-            pm[cc * 8 + j] = pk;
-            sum += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
+            pm[cc * 16 + j] = pack_bf16(s0, s1);
           }
         }
-        rsum[hf * TILE + row] = sum;
         // the packed scores of the row's second thread land on columns its first thread reads: both have read
         sync_pair();
         if (!alive) break;
@@ -685,8 +711,10 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       cj = cnext;
     }
     if (alive && mbar_wait(&misc->st_ready, (ntiles - 1) & 1, abortp, status, false) &&
-        mbar_wait(&misc->o_ready, (ntiles - 1) & 1, abortp, status, false))
+        mbar_wait(&misc->o_ready, (ntiles - 1) & 1, abortp, status, false)) {
       write_out(ntiles - 1);
+      if (lane == 0) bulk_wait0();                 // the block's shared memory outlives its copies
+    }
   }
   tcgen05_fence_before();
   __syncthreads();
@@ -703,6 +731,7 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 // ------------------------------------------------------------------------------------------
 namespace tchost {
 int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int H, int L, int inner);
+int make_map_out(CUtensorMap* map, void* base, TensorAddr a, int B, int H, int L, int inner);
 }  // namespace tchost
 int fs_tc_rowterm(fsharp_ctx* ctx, const void* K, const fsharp_dims* dm, const uint8_t* images, const int* flags, int Lpad,
                   int tiles_per_split, int nsplit, float* crow);
@@ -765,15 +794,15 @@ int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, c
   } else {
     FS_TRY(fs_tc_rowterm(ctx, K, dm, images, flags, Lpad, per, 1, crow));
   }
-  CUtensorMap tmQ, tmK, tmV;
+  CUtensorMap tmQ, tmK, tmV, tmY;
   FS_TRY(tchost::make_map_tokens(&tmQ, Q, fs_addr(dm->q_stride, H, L, dm->d), B, H, L, dm->d));
   FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, L, dm->d), B, H, L, dm->d));
   FS_TRY(tchost::make_map_tokens(&tmV, V, fs_addr(dm->v_stride, H, L, dm->dv), B, H, L, dm->dv));
+  FS_TRY(tchost::make_map_out(&tmY, Y, fs_addr(dm->y_stride, H, L, dm->dv), B, H, L, dm->dv));
   FS_CUDA_OK(cudaFuncSetAttribute(tc_causal_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CfSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_CAUSAL);
   tc_causal_kernel<<<dim3(nseg, BH), TC_THREADS, CfSmem::TOTAL + 1024, ctx->stream>>>(
-      tmQ, tmK, tmV, images, crow, partial, shifts, nseg - 1, H, dm->pool, L, Lpad, per, (__nv_bfloat16*)Y,
-      fs_addr(dm->y_stride, H, L, dm->dv), ctx->d_status);
+      tmQ, tmK, tmV, tmY, images, crow, partial, shifts, nseg - 1, H, dm->pool, L, Lpad, per, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;

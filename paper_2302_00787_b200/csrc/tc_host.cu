@@ -56,6 +56,21 @@ int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int
   return r == CUDA_SUCCESS ? FSHARP_OK : FSHARP_E_CUDA;
 }
 
+// Output rows as TMA store tiles: 32 rows x 32 values (64 bytes), staged in shared memory with the 64-byte swizzle.
+int make_map_out(CUtensorMap* map, void* base, TensorAddr a, int B, int H, int L, int inner) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return FSHARP_E_CUDA;
+  cuuint64_t dims[4] = {(cuuint64_t)inner, (cuuint64_t)L, (cuuint64_t)H, (cuuint64_t)B};
+  cuuint64_t strides[3] = {(cuuint64_t)a.sl * 2, (cuuint64_t)a.sh * 2, (cuuint64_t)a.sb * 2};
+  if (H == 1 && strides[1] == 0) strides[1] = strides[0] * (cuuint64_t)L;
+  if (B == 1 && strides[2] == 0) strides[2] = strides[1] * (cuuint64_t)H;
+  cuuint32_t box[4] = {32, 32, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? FSHARP_OK : FSHARP_E_CUDA;
+}
+
 }  // namespace tchost
 
 int fs_tc_supported(const fsharp_dims* dm, int dtype, int causal, int chunk, float qk_scale) {
