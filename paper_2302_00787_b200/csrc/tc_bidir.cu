@@ -87,7 +87,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   if (threadIdx.x == 0) {
     for (int i = 0; i < KV_KSTAGES; i++) {
       mbar_init(&misc->fullK[i], 1);
-      mbar_init(&misc->convK[i], 1);
+      mbar_init(&misc->convK[i], 2);
       mbar_init(&misc->emptyK[i], 1);
     }
     for (int i = 0; i < 2; i++) {
@@ -122,7 +122,28 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 
   if (warp >= WARP_TMA) {
   regs_release<REGS_PRODUCER>();
+  // bf16 -> fp16 of key tile `it`, in place (16-byte pieces keep their swizzled positions): the logits then need one
+  // fp16 image of W (11 significant bits) instead of a bf16 value and its remainder.  Half a tile per call, by the
+  // converting warp (part 0) and the copying warp (part 1), which sit on different schedulers.
+  auto convert_half = [&](int it, int part) -> bool {
+    const int st = it % KV_KSTAGES;
+    if (!__all_sync(0xffffffffu, mbar_wait(&misc->fullK[st], (it / KV_KSTAGES) & 1, abortp, status, false))) return false;
+    uint4* xt = reinterpret_cast<uint4*>(sm + KvSmem::X0 + st * TILE_BYTES) + part * (int)(TILE_BYTES / 32);
+#pragma unroll 4
+    for (int i = 0; i < (int)(TILE_BYTES / 32) / 32; i++) {
+      uint4 u = xt[lane + i * 32];
+      u.x = pack_f16(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
+      u.y = pack_f16(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
+      u.z = pack_f16(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u));
+      u.w = pack_f16(__uint_as_float(u.w << 16), __uint_as_float(u.w & 0xffff0000u));
+      xt[lane + i * 32] = u;
+    }
+    fence_proxy_async_smem();
+    mbar_arrive_warp(&misc->convK[st], lane);
+    return true;
+  };
   if (warp == WARP_TMA) {
+    // The whole warp walks the schedule; lane 0 issues the copies.
     if (lane == 0) {
       prefetch_tmap(&tmK);
       prefetch_tmap(&tmV);
@@ -133,57 +154,53 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         tma_prefetch_4d(&tmK, 0, (tile0 + it) * TILE, h, b);
         tma_prefetch_4d(&tmV, 0, (tile0 + it) * TILE, h, b);
       }
-      // Key tile `it` is loaded as soon as the logits MMA of tile it - 3 has completed; the value tile follows one
-      // iteration behind (its stage is held until the contraction of tile it - 2 has completed).  So the next
-      // tile's logits never wait for a value tile.
-      int issuedK = 0, issuedV = 0;
-      auto load_v = [&](int j) {
-        const int sj = j & 1;
-        if (!mbar_wait(&misc->emptyV[sj], ((j >> 1) & 1) ^ 1, abortp, status)) return false;
+    }
+    // Key tile `it` is loaded as soon as the logits MMA of tile it - 3 has completed; the warp then converts its half
+    // of key tile it - 1, which has landed meanwhile; the value tile follows one iteration behind (its stage is held
+    // until the contraction of tile it - 2 has completed).  So the next tile's logits never wait for a value tile.
+    int issuedK = 0, issuedV = 0;
+    auto load_v = [&](int j) {
+      const int sj = j & 1;
+      if (!__all_sync(0xffffffffu, mbar_wait(&misc->emptyV[sj], ((j >> 1) & 1) ^ 1, abortp, status))) return false;
+      if (lane == 0) {
         mbar_expect_tx(&misc->fullV[sj], TILE_BYTES);
         tma_load_4d(sm + KvSmem::V0 + sj * TILE_BYTES, &tmV, &misc->fullV[sj], 0, (tile0 + j) * TILE, h, b);
-        issuedV = j + 1;
-        return true;
-      };
-      bool okp = true;
-      for (int it = 0; it < ntiles && okp; it++) {
-        const int st = it % KV_KSTAGES;
+      }
+      issuedV = j + 1;
+      return true;
+    };
+    bool okp = true;
+    for (int it = 0; it < ntiles && okp; it++) {
+      const int st = it % KV_KSTAGES;
+      if (!__all_sync(0xffffffffu, mbar_wait(&misc->emptyK[st], ((it / KV_KSTAGES) & 1) ^ 1, abortp, status))) { okp = false; break; }
+      if (lane == 0) {
         if (it + PREFETCH_TILES < ntiles) {
           tma_prefetch_4d(&tmK, 0, (tile0 + it + PREFETCH_TILES) * TILE, h, b);
           tma_prefetch_4d(&tmV, 0, (tile0 + it + PREFETCH_TILES) * TILE, h, b);
         }
-        if (!mbar_wait(&misc->emptyK[st], ((it / KV_KSTAGES) & 1) ^ 1, abortp, status)) { okp = false; break; }
         mbar_expect_tx(&misc->fullK[st], TILE_BYTES);
         tma_load_4d(sm + KvSmem::X0 + st * TILE_BYTES, &tmK, &misc->fullK[st], 0, (tile0 + it) * TILE, h, b);
-        issuedK = it + 1;
-        if (it >= 1) okp = load_v(it - 1);
       }
-      if (okp && ntiles > 0) load_v(ntiles - 1);
-      // no copy of this block may still be in flight when it exits
+      issuedK = it + 1;
+      if (it >= 1) {
+        okp = convert_half(it - 1, 1);
+        if (okp) okp = load_v(it - 1);
+      }
+    }
+    if (okp && ntiles > 0) {
+      okp = convert_half(ntiles - 1, 1);
+      if (okp) load_v(ntiles - 1);
+    }
+    // no copy of this block may still be in flight when it exits
+    if (lane == 0) {
       mbar_wait(&misc->const_bar, 0, abortp, status, false);
       for (int it = max(0, issuedK - KV_KSTAGES); it < issuedK; it++)
         mbar_wait(&misc->fullK[it % KV_KSTAGES], (it / KV_KSTAGES) & 1, abortp, status, false);
       for (int it = max(0, issuedV - 2); it < issuedV; it++) mbar_wait(&misc->fullV[it & 1], (it >> 1) & 1, abortp, status, false);
     }
   } else if (warp == WARP_MMA + 2) {
-    // ---------------- bf16 -> fp16 of the key tile, in place (16-byte pieces keep their swizzled positions): the
-    // logits then need one fp16 image of W (11 significant bits) instead of a bf16 value and its remainder
-    for (int it = 0; it < ntiles; it++) {
-      const int st = it % KV_KSTAGES;
-      if (!mbar_wait(&misc->fullK[st], (it / KV_KSTAGES) & 1, abortp, status, false)) break;
-      uint4* xt = reinterpret_cast<uint4*>(sm + KvSmem::X0 + st * TILE_BYTES);
-#pragma unroll 4
-      for (int i = 0; i < (int)(TILE_BYTES / 16) / 32; i++) {
-        uint4 u = xt[lane + i * 32];
-        u.x = pack_f16(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
-        u.y = pack_f16(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
-        u.z = pack_f16(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u));
-        u.w = pack_f16(__uint_as_float(u.w << 16), __uint_as_float(u.w & 0xffff0000u));
-        xt[lane + i * 32] = u;
-      }
-      fence_proxy_async_smem();
-      mbar_arrive_warp(&misc->convK[st], lane);
-    }
+    for (int it = 0; it < ntiles; it++)
+      if (!convert_half(it, 0)) break;
   } else if (warp == WARP_MMA) {
     // ---------------- logits MMAs: the whole warp walks the schedule (descriptor arithmetic and waits stay
     // warp-uniform), one elected lane issues
@@ -323,9 +340,8 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         }
         const float hm = fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3]));
         float mx = valid ? hm + cj : -INFINITY;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        if (lane == 0) atomicMax(&tmax[it % 3], f2ord(mx));
+        const int wm = __reduce_max_sync(0xffffffffu, f2ord(mx));       // one instruction for the warp's maximum
+        if (lane == 0) atomicMax(&tmax[it % 3], wm);
         if (q == 0 && lane == 0) tmax[(it + 1) % 3] = f2ord(-INFINITY);           // next tile's slot; idle since tile it-2
         named_bar_sync(1 + hf, HALF_THREADS);
         tm = ord2f(tmax[it % 3]);
@@ -452,7 +468,7 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
   volatile int* abortp = &misc->abort_flag;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < OUT_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->conv[i], 1); mbar_init(&misc->empty[i], 1); }
+    for (int i = 0; i < OUT_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->conv[i], 2); mbar_init(&misc->empty[i], 1); }
     mbar_init(&misc->logits_full, 1);
     mbar_init(&misc->logits_free, EPI_THREADS / 32);
     for (int i = 0; i < TC_M / 64; i++) mbar_init(&misc->phi_full[i], EPI_THREADS / 64);
@@ -473,43 +489,57 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
 
   if (warp >= WARP_TMA) {
   regs_release<REGS_PRODUCER>();
+  // bf16 -> fp16 of query tile `it`, in place (16-byte pieces keep their swizzled positions): half a tile per call,
+  // by the converting warp (part 0) and the copying warp (part 1), which sit on different schedulers
+  auto convert_half = [&](int it, int part) -> bool {
+    const int st = it % OUT_STAGES;
+    if (!__all_sync(0xffffffffu, mbar_wait(&misc->full[st], (it / OUT_STAGES) & 1, abortp, status, false))) return false;
+    uint4* xt = reinterpret_cast<uint4*>(sm + OutSmem::X0 + st * TILE_BYTES) + part * (int)(TILE_BYTES / 32);
+#pragma unroll 4
+    for (int i = 0; i < (int)(TILE_BYTES / 32) / 32; i++) {
+      uint4 u = xt[lane + i * 32];
+      u.x = pack_f16(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
+      u.y = pack_f16(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
+      u.z = pack_f16(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u));
+      u.w = pack_f16(__uint_as_float(u.w << 16), __uint_as_float(u.w & 0xffff0000u));
+      xt[lane + i * 32] = u;
+    }
+    fence_proxy_async_smem();
+    mbar_arrive_warp(&misc->conv[st], lane);
+    return true;
+  };
   if (warp == WARP_TMA) {
+    // The whole warp walks the schedule; lane 0 issues the copies.  After the copy of tile it has been issued the
+    // warp converts its half of tile it - 1, which has landed meanwhile.
     if (lane == 0) {
       prefetch_tmap(&tmQ);
       mbar_expect_tx(&misc->const_bar, IMG_W_BYTES);
       bulk_load(sm + OutSmem::WH, img + IMG_WH, IMG_W_BYTES, &misc->const_bar);
       for (int it = 0; it < min(ntiles, PREFETCH_TILES); it++) tma_prefetch_4d(&tmQ, 0, (tile0 + it) * TILE, h, b);
-      int issued = 0;
-      for (int it = 0; it < ntiles; it++) {
-        const int st = it % OUT_STAGES;
+    }
+    int issued = 0;
+    bool okp = true;
+    for (int it = 0; it < ntiles; it++) {
+      const int st = it % OUT_STAGES;
+      if (!__all_sync(0xffffffffu, mbar_wait(&misc->empty[st], ((it / OUT_STAGES) & 1) ^ 1, abortp, status))) { okp = false; break; }
+      if (lane == 0) {
         if (it + PREFETCH_TILES < ntiles) tma_prefetch_4d(&tmQ, 0, (tile0 + it + PREFETCH_TILES) * TILE, h, b);
-        if (!mbar_wait(&misc->empty[st], ((it / OUT_STAGES) & 1) ^ 1, abortp, status)) break;
         mbar_expect_tx(&misc->full[st], TILE_BYTES);
         tma_load_4d(sm + OutSmem::X0 + st * TILE_BYTES, &tmQ, &misc->full[st], 0, (tile0 + it) * TILE, h, b);
-        issued = it + 1;
       }
+      issued = it + 1;
+      if (it > 0 && !convert_half(it - 1, 1)) { okp = false; break; }
+    }
+    if (okp && ntiles > 0) convert_half(ntiles - 1, 1);
+    // no copy of this block may still be in flight when it exits
+    if (lane == 0) {
       mbar_wait(&misc->const_bar, 0, abortp, status, false);
       for (int it = max(0, issued - OUT_STAGES); it < issued; it++)
         mbar_wait(&misc->full[it % OUT_STAGES], (it / OUT_STAGES) & 1, abortp, status, false);
     }
   } else if (warp == WARP_OUT_CVT) {
-    // ---------------- bf16 -> fp16 of the query tile, in place (16-byte pieces keep their swizzled positions)
-    for (int it = 0; it < ntiles; it++) {
-      const int st = it % OUT_STAGES;
-      if (!mbar_wait(&misc->full[st], (it / OUT_STAGES) & 1, abortp, status, false)) break;
-      uint4* xt = reinterpret_cast<uint4*>(sm + OutSmem::X0 + st * TILE_BYTES);
-#pragma unroll 4
-      for (int i = 0; i < (int)(TILE_BYTES / 16) / 32; i++) {
-        uint4 u = xt[lane + i * 32];
-        u.x = pack_f16(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
-        u.y = pack_f16(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
-        u.z = pack_f16(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u));
-        u.w = pack_f16(__uint_as_float(u.w << 16), __uint_as_float(u.w & 0xffff0000u));
-        xt[lane + i * 32] = u;
-      }
-      fence_proxy_async_smem();
-      mbar_arrive_warp(&misc->conv[st], lane);
-    }
+    for (int it = 0; it < ntiles; it++)
+      if (!convert_half(it, 0)) break;
   } else if (warp == WARP_MMA) {
     // ---------------- logits MMAs: the whole warp walks the schedule, one elected lane issues
     constexpr uint32_t ID_LOGITS = idesc_f16(128, TC_M, 0, 0);

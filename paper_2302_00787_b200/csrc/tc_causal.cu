@@ -503,9 +503,8 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           mxp[3] = max3(mxp[3], __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
         }
         float mx = valid ? fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])) + cj : -INFINITY;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        if (lane == 0) atomicMax(&misc->chunk_max[it % 3], f2ord(mx));
+        const int wm = __reduce_max_sync(0xffffffffu, f2ord(mx));       // one instruction for the warp's maximum
+        if (lane == 0) atomicMax(&misc->chunk_max[it % 3], wm);
         if (threadIdx.x == CF_PRODUCER_WARPS * 32) misc->chunk_max[(it + 1) % 3] = f2ord(-INFINITY);   // next tile's slot; idle since tile it - 2
         sync_all();
         if (!alive) break;
