@@ -41,7 +41,7 @@ constexpr int PREFETCH_TILES = 4;   // tiles pulled into L2 ahead of the shared-
 // tensor pipe instead of 128, and every epilogue thread (= one feature) takes part when the state leaves.
 constexpr int KV_KSTAGES = 3;       // key tiles in flight (TMA, conversion to fp16, logits MMA)
 constexpr bool KV_TURNS = false;    // the two feature halves take turns at the exponentials
-constexpr int KV_POLY_PAIRS = 1;    // of every four pairs of exponentials, this many run on the multiply-add pipe
+constexpr int KV_POLY_PAIRS = 2;    // of every four pairs of exponentials, this many run on the multiply-add pipe (measured: 1 and 3 are slower)
 struct KvSmem {
   static constexpr uint32_t X0 = 0, V0 = KV_KSTAGES * TILE_BYTES, ONES = V0 + 2 * TILE_BYTES, W = ONES + TILE_BYTES,
                             PHI = W + IMG_W_BYTES, MISC = PHI + 4 * TILE_BYTES, TOTAL = MISC + 256;

@@ -41,7 +41,7 @@ constexpr int CF_WARP_TMA = 0, CF_WARP_MMA = 1, CF_WARP_CVT0 = 2, CF_PRODUCER_WA
 constexpr int CVT_THREADS = 96;       // warps 0, 2 and 3 (each shares its scheduler with two epilogue warps; so does the MMA warp)
 // Of every four pairs of exponentials, this many are evaluated on the multiply-add pipe (exp2_poly2), the others
 // by the special-function unit, whose 16 results per clock would otherwise bound the kernel.
-constexpr int CF_POLY_PAIRS = 1;
+constexpr int CF_POLY_PAIRS_K = 1, CF_POLY_PAIRS_Q = 1;     // key features, query features (2 for either is slower here)
 // The MMA-issuing thread of this kernel keeps more descriptors alive than those of the other kernels:
 // 128 x 64 + 256 x 216 registers (of the 384 x 168 the block is launched with).
 constexpr int CF_REGS_PRODUCER = 64, CF_REGS_EPILOGUE = 216;
@@ -546,7 +546,7 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
               uint32_t& e0 = v[half * 64 + c * 8 + 2 * j];
               uint32_t& e1 = v[half * 64 + c * 8 + 2 * j + 1];
               add2(e0, e1, rc, rc);
-              if (j < CF_POLY_PAIRS) {
+              if (j < CF_POLY_PAIRS_K) {
                 exp2_poly2(e0, e1);
                 p[j] = pack_bf16(__uint_as_float(e0), __uint_as_float(e1));
               } else {
@@ -642,7 +642,7 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             uint32_t& e0 = v[half * 64 + c * 32 + 2 * j];
             uint32_t& e1 = v[half * 64 + c * 32 + 2 * j + 1];
             add2(e0, e1, -mx, -mx);
-            if ((j & 3) < CF_POLY_PAIRS) {
+            if ((j & 3) < CF_POLY_PAIRS_Q) {
               exp2_poly2(e0, e1);
               p[j] = pack_bf16(__uint_as_float(e0), __uint_as_float(e1));
             } else {
