@@ -114,22 +114,18 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
       const int m = m0 + 4 * ty + u;
       if (pass == 0) {
         if (m < M) {
+          // (the fp32 copy serves the fp32 kernels only; the tensor-core path reads the operand image)
+          if (images == nullptr) {
 #pragma unroll
-          for (int v = 0; v < NC; v++) W[(size_t)m * d + NC * tx + v] = acc[u][v];
-          if (images != nullptr) {
-            // log2e * qk_scale * W as a bf16 value and its bf16 remainder, two neighbours per store
+            for (int v = 0; v < NC; v++) W[(size_t)m * d + NC * tx + v] = acc[u][v];
+          } else {
+            // log2e * qk_scale * W rounded to fp16, two neighbours per store
             uint8_t* img = images + ((size_t)g * 2 + (side - 1)) * tcl::IMG_BYTES;
             const float sw = FS_LOG2E * qk_scale;
 #pragma unroll
-            for (int v = 0; v + 1 < NC; v += 2) {
-              const float v0 = acc[u][v] * sw, v1 = acc[u][v + 1] * sw;
-              const __nv_bfloat16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
-              const uint32_t off = tc::sw128_offset(m, NC * tx + v);
-              *reinterpret_cast<__nv_bfloat162*>(img + tcl::IMG_W + off) = __nv_bfloat162(h0, h1);
-              *reinterpret_cast<__nv_bfloat162*>(img + tcl::IMG_WLO + off) =
-                  __nv_bfloat162(__float2bfloat16_rn(v0 - __bfloat162float(h0)), __float2bfloat16_rn(v1 - __bfloat162float(h1)));
-              *reinterpret_cast<__half2*>(img + tcl::IMG_WH + off) = __floats2half2_rn(v0, v1);
-            }
+            for (int v = 0; v + 1 < NC; v += 2)
+              *reinterpret_cast<__half2*>(img + tcl::IMG_WH + tc::sw128_offset(m, NC * tx + v)) =
+                  __floats2half2_rn(acc[u][v] * sw, acc[u][v + 1] * sw);
           }
         }
       } else {
@@ -168,7 +164,7 @@ prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const do
       const int e = e0 + q * PREP_THREADS;
       if (e >= d * d) continue;
       const int i = e / d, j = e % d;
-      Cf[e] = (float)cv[q];
+      if (images == nullptr) Cf[e] = (float)cv[q];
       if (i == j ? (cv[q] != gamma) : (cv[q] != 0.0)) cscalar = 0;
       if (images != nullptr) {
         // log2e * qk_scale^2 * C[i][j] goes to row j, column i of the MMA operand

@@ -18,17 +18,15 @@ constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t TILE_BYTES = 16384;          // 128 rows x 128 bytes
 
 // Per (group, side) operand image, already in the shared-memory layouts the MMAs read:
-//   W     [256 features x 64]  K-major, 128-byte swizzle, bf16(log2e * qk_scale * W)
-//   Wlo   [256 features x 64]  the bf16 remainder of the same matrix (W is used as hi + lo: a single
-//                              bf16 rounding of W alone costs ~0.4% per feature)
+//   Wh    [256 features x 64]  K-major, 128-byte swizzle, fp16(log2e * qk_scale * W): rounded once to 11
+//                              significant bits (the token tiles are converted to fp16 as well, so one
+//                              operand serves where a bf16 value and its remainder would be needed)
 //   Chi   [64 x 64]            K-major, 128-byte swizzle, bf16 of log2e * qk_scale^2 * C (row n, col k = C[k][n])
 //   Clo   [64 x 64]            the bf16 remainder of the same matrix
 //   a2    [256] fp32           2 log2e w_m^T A w_m: the factor 2^a2 of feature m (it appears once in
 //                              phi(Q) and once in phi(K)) is applied to row m of S^T [V | 1] by the merge
-//   Wh    [256 features x 64]  the same matrix as W, rounded once to fp16 (11 significant bits: one operand
-//                              instead of hi + lo where the token tile is converted to fp16 as well)
-constexpr uint32_t IMG_W = 0, IMG_W_BYTES = 32768, IMG_WLO = 32768, IMG_CHI = 65536, IMG_C_BYTES = 8192, IMG_CLO = 73728,
-                   IMG_A2 = 81920, IMG_A2_BYTES = 1024, IMG_WH = 82944, IMG_BYTES = 115712;
+constexpr uint32_t IMG_WH = 0, IMG_W_BYTES = 32768, IMG_CHI = 32768, IMG_C_BYTES = 8192, IMG_CLO = 40960, IMG_A2 = 49152,
+                   IMG_A2_BYTES = 1024, IMG_BYTES = 50176;
 // S^T [V | 1] transposed, fp16: 4 blocks of [80 rows x 64 features], 128-byte swizzle
 constexpr uint32_t KVT_BLOCK_BYTES = 10240, KVT_BYTES = 40960;
 
