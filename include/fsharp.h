@@ -15,6 +15,8 @@
  *   fsharp_attend         Y, bidirectional or causal (lower-triangular mask)
  *   fsharp_pair_estimate  Khat(x, y) for pairs, with Theorem 4.1's variance
  *   fsharp_kernel_apply   the unnormalised operator Khat^(alpha) C (softmax and Gaussian kernels)
+ *   fsharp_attend_key_state, fsharp_attend_with_state   the same Y with the keys of a sequence spread over
+ *                         several calls or devices (key-side sums of disjoint key ranges add)
  *
  * Conventions common to every call
  *   - All data pointers are DEVICE pointers owned by the caller unless the
@@ -199,6 +201,35 @@ int fsharp_featurize_static(void* stream, const void* X, const float* Omega, con
 int fsharp_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V,
                   const float* Omega, const double* params, const fsharp_dims* dims,
                   int dtype, int causal, int chunk, float qk_scale, void* Y);
+
+/* Sequence-parallel attention.  In Section 2.2's formula the numerator phi(Q) (phi(K)^T V) and the normaliser
+ * phi(Q) (phi(K)^T 1) are sums over keys, so the key-side sums S^T [V | 1] of disjoint key ranges add: the keys of
+ * one (batch, head) may be spread over several calls, contexts or devices, each of which reduces its range to a
+ * "key state", and any holder of all the states of the keys a query may see can finish the query's row.
+ * Tensor-core kernels only: dtype FSHARP_BF16, d = dv = 64, M = 256 (anything else: FSHARP_E_SHAPE); all calls that
+ * take part must be given the same Omega and params.
+ *
+ * fsharp_key_state_splits   ns >= 1, the number of pieces a key-state call cuts its key range into (a function of
+ *                           dims->B, H, Lk and the device's SM count), or a negative error code.
+ * fsharp_attend_key_state   state  [B*H][ns][80][256] fp32 (device, 16-byte aligned): rows 0..64 of piece p are
+ *                           sum_j phi(k_j) [v_j | 1]^T over the keys j of piece p, every feature half (128
+ *                           features) scaled by 2^-shift; shifts [B*H][ns][2] fp32 (device): those shifts (log2).
+ *                           K, V, strides and Lk as in fsharp_attend; Lq and the query strides are ignored.
+ * fsharp_attend_with_state  states [B*H][n_states][80][256], shifts [B*H][n_states][2] (device): key states in the
+ *                           layout above, concatenated along the piece index in any order.
+ *                           causal = 0: Y = attention of Q over exactly the keys behind the states (n_states >= 1;
+ *                           K and V are not read and may be null).
+ *                           causal = 1: the keys behind the states precede every token of this call (n_states may
+ *                           be 0); Y = causal attention of Q over those keys and, with the lower-triangular mask,
+ *                           over K, V (Lq == Lk, any length).
+ *                           n_states > 64 (causal = 0): FSHARP_E_LIMIT.
+ * All pointers are device pointers; the calls are asynchronous on the context's stream like fsharp_attend. */
+int fsharp_key_state_splits(fsharp_ctx* ctx, const fsharp_dims* dims);
+int fsharp_attend_key_state(fsharp_ctx* ctx, const void* K, const void* V, const float* Omega, const double* params,
+                            const fsharp_dims* dims, int dtype, float qk_scale, float* state, float* shifts);
+int fsharp_attend_with_state(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const float* Omega,
+                             const double* params, const fsharp_dims* dims, int dtype, int causal, float qk_scale,
+                             const float* states, const float* shifts, int n_states, void* Y);
 
 /* The unnormalised operator of Section 2.1: out = Khat^(alpha)(X, Y) C, the O(L M n) evaluation P (S^T C) of
  * K^(alpha)(x, y) = exp(alpha |x|^2 + x^T y + alpha |y|^2) applied to a matrix C, with the features

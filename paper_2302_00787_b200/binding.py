@@ -25,6 +25,7 @@ EXPORTS = [
     "fsharp_params_doubles", "fsharp_stats", "fsharp_fit_params", "fsharp_featurize", "fsharp_attend",
     "fsharp_forward_host", "fsharp_pair_estimate", "fsharp_set_timing", "fsharp_read_timing",
     "fsharp_kernel_name", "fsharp_static_scratch_bytes", "fsharp_featurize_static", "fsharp_kernel_apply",
+    "fsharp_key_state_splits", "fsharp_attend_key_state", "fsharp_attend_with_state",
     "fsharp_selftest_bounded_wait",
 ]
 
@@ -74,6 +75,9 @@ def load_library() -> C.CDLL:
         "fsharp_featurize": (i32, [vp, vp, vp, vp, i32, dims_p, i32, f32, i32, vp, vp]),
         "fsharp_attend": (i32, [vp, vp, vp, vp, vp, vp, dims_p, i32, i32, i32, f32, vp]),
         "fsharp_kernel_apply": (i32, [vp, vp, vp, vp, vp, vp, f64, dims_p, i32, f32, vp]),
+        "fsharp_key_state_splits": (i32, [vp, dims_p]),
+        "fsharp_attend_key_state": (i32, [vp, vp, vp, vp, vp, dims_p, i32, f32, vp, vp]),
+        "fsharp_attend_with_state": (i32, [vp, vp, vp, vp, vp, vp, dims_p, i32, i32, f32, vp, vp, i32, vp]),
         "fsharp_forward_host": (i32, [vp, vp, vp, vp, vp, dims_p, i32, i32, i32, i32, f32, vp]),
         "fsharp_pair_estimate": (i32, [vp, vp, vp, vp, vp, i64, i32, i32, i32, vp, vp, vp]),
         "fsharp_set_timing": (i32, [vp, i32]),
@@ -242,6 +246,48 @@ class Context:
         _check(self.lib.fsharp_attend(self._h, Q.data_ptr(), K.data_ptr(), V.data_ptr(), Omega.data_ptr(),
                                       params.data_ptr(), C.byref(dm), _dtype_code(Q), int(bool(causal)), chunk,
                                       qk_scale, out.data_ptr()), "fsharp_attend")
+        return out
+
+    def fsharp_attend_key_state(self, K, V, Omega, params, pool=POOL_PER_BH, qk_scale=1.0):
+        """Key-side sums of this call's keys: (state [B*H, ns, 80, 256] fp32, shifts [B*H, ns, 2] fp32)."""
+        B, H, Lk, d = K.shape
+        dv, M = V.shape[3], Omega.shape[-2]
+        ohs = Omega.stride(0) if Omega.dim() == 3 else 0
+        dm = make_dims(B, H, Lk, Lk, d, dv, M, pool, q=K, k=K, v=V, omega_head_stride=ohs)
+        ns = self.lib.fsharp_key_state_splits(self._h, C.byref(dm))
+        _check(min(ns, 0), "fsharp_key_state_splits")
+        state = torch.empty(B * H, ns, 80, 256, dtype=torch.float32, device=K.device)
+        shifts = torch.empty(B * H, ns, 2, dtype=torch.float32, device=K.device)
+        _check(self.lib.fsharp_attend_key_state(self._h, K.data_ptr(), V.data_ptr(), Omega.data_ptr(), params.data_ptr(),
+                                                C.byref(dm), _dtype_code(K), qk_scale, state.data_ptr(),
+                                                shifts.data_ptr()), "fsharp_attend_key_state")
+        return state, shifts
+
+    def fsharp_attend_with_state(self, Q, K, V, Omega, params, states, shifts, causal=False, pool=POOL_PER_BH,
+                                 qk_scale=1.0, out=None):
+        """Attention of Q over the keys behind `states` (and, causal, over K, V under the mask).  states
+        [B*H, n, 80, 256] and shifts [B*H, n, 2] fp32 contiguous, or None (causal only: nothing precedes)."""
+        B, H, Lq, d = Q.shape
+        M = Omega.shape[-2]
+        ohs = Omega.stride(0) if Omega.dim() == 3 else 0
+        n = 0 if states is None else states.shape[1]
+        if n:
+            if not (states.is_contiguous() and shifts.is_contiguous() and states.dtype == torch.float32
+                    and shifts.dtype == torch.float32 and tuple(states.shape) == (B * H, n, 80, 256)
+                    and tuple(shifts.shape) == (B * H, n, 2)):
+                raise ValueError("states / shifts: contiguous fp32 [B*H, n, 80, 256] / [B*H, n, 2]")
+        dv = V.shape[3] if V is not None else 64
+        if out is None:
+            out = torch.empty(B, H, Lq, dv, dtype=Q.dtype, device=Q.device)
+        if causal:
+            dm = make_dims(B, H, Lq, K.shape[2], d, dv, M, pool, q=Q, k=K, v=V, y=out, omega_head_stride=ohs)
+        else:
+            dm = make_dims(B, H, Lq, Lq, d, dv, M, pool, q=Q, k=Q, v=out, y=out, omega_head_stride=ohs)
+        _check(self.lib.fsharp_attend_with_state(
+            self._h, Q.data_ptr(), K.data_ptr() if causal else None, V.data_ptr() if causal else None, Omega.data_ptr(),
+            params.data_ptr(), C.byref(dm), _dtype_code(Q), int(bool(causal)), qk_scale,
+            states.data_ptr() if n else None, shifts.data_ptr() if n else None, n, out.data_ptr()),
+            "fsharp_attend_with_state")
         return out
 
     def fsharp_kernel_apply(self, X, Y, Cmat, Omega, params, alpha=0.0, pool=POOL_PER_BH, qk_scale=1.0, out=None):

@@ -10,6 +10,15 @@ size_t fs_tc_attend_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm, 
 int fs_tc_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, int causal,
                  int chunk, const uint8_t* images, const int* flags, void* Y, WsAlloc* ws);
 int fs_tc_featurize_supported(const fsharp_dims* dm, int dtype, int stab);
+int fs_tc_key_state_splits(const fsharp_ctx* ctx, const fsharp_dims* dm, int* tiles_per_split);
+size_t fs_tc_key_state_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
+int fs_tc_key_state(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
+                    const int* flags, float* state, float* shifts, WsAlloc* ws);
+int fs_tc_query_side(fsharp_ctx* ctx, const void* Q, const fsharp_dims* dm, const uint8_t* images, const float* partial,
+                     const float* shifts, int nsplit, void* Y);
+size_t fs_tc_causal_prefix_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm, int nprefix);
+int fs_tc_causal_prefix(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
+                        const int* flags, const float* pre_state, const float* pre_shifts, int nprefix, void* Y, WsAlloc* ws);
 size_t fs_tc_featurize_scratch_bytes(const fsharp_dims* dm, int side);
 int fs_tc_featurize(fsharp_ctx* ctx, const void* X, const fsharp_dims* dm, int side, int stab, const float* prep,
                     const uint8_t* images, const int* flags, float* phi, float* logscale, WsAlloc* ws);
@@ -157,6 +166,76 @@ int fsharp_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, 
   FS_TRY(fs_run_prep(ctx, Omega, dims->omega_head_stride, params, (int64_t)ParamsLayout{dims->d}.total(), G,
                      dims->H, dims->pool, dims->d, dims->M, prep));
   return fs_simt_attend(ctx, Q, K, V, dims, dtype, causal, chunk, qk_scale, prep, Y, &ws);
+}
+
+int fsharp_key_state_splits(fsharp_ctx* ctx, const fsharp_dims* dims) {
+  if (!ctx) return FSHARP_E_BADARG;
+  FS_TRY(check_dims(dims, true));
+  if (dims->B * dims->H == 0 || dims->Lk <= 0) return FSHARP_E_SHAPE;
+  return fs_tc_key_state_splits(ctx, dims, nullptr);
+}
+
+int fsharp_attend_key_state(fsharp_ctx* ctx, const void* K, const void* V, const float* Omega, const double* params,
+                            const fsharp_dims* dims, int dtype, float qk_scale, float* state, float* shifts) {
+  if (!ctx || !Omega || !params || !state || !shifts) return FSHARP_E_BADARG;
+  FS_TRY(check_dims(dims, true));
+  if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
+  if (dims->B * dims->H == 0 || dims->Lk <= 0) return FSHARP_E_SHAPE;
+  // the tensor-core kernels only (bf16, d = dv = 64, M = 256): the state is their key-side sum
+  fsharp_dims kd = *dims;
+  kd.Lq = kd.Lk;
+  for (int i = 0; i < 3; i++) kd.q_stride[i] = kd.k_stride[i];
+  if (!fs_tc_supported(&kd, dtype, 0, 0, qk_scale)) return FSHARP_E_SHAPE;
+  FS_TRY(check_ptr(K, dtype, dims->k_stride));
+  FS_TRY(check_ptr(V, dtype, dims->v_stride));
+  if (reinterpret_cast<uintptr_t>(state) % 16 != 0 || reinterpret_cast<uintptr_t>(shifts) % 8 != 0) return FSHARP_E_ALIGN;
+  FS_CUDA_OK(cudaSetDevice(ctx->device));
+  const int G = fs_groups(dims);
+  const size_t prep_f = (size_t)G * 2 * PrepLayout{dims->d, dims->M}.total();
+  FS_TRY(fs_ws_reserve(ctx, ws_round(prep_f * 4) + fs_tc_key_state_scratch_bytes(ctx, &kd)));
+  WsAlloc ws{ctx->ws, 0};
+  float* prep = ws.take<float>(prep_f);
+  uint8_t* images = ws.take<uint8_t>((size_t)G * 2 * tcl::IMG_BYTES);
+  int* flags = ws.take<int>((size_t)G * 2 * tcl::FLAG_WORDS + 16);
+  FS_TRY(fs_run_prep_images(ctx, Omega, dims->omega_head_stride, params, (int64_t)ParamsLayout{dims->d}.total(), G,
+                            dims->H, dims->pool, dims->d, dims->M, prep, qk_scale, images, flags));
+  return fs_tc_key_state(ctx, K, V, &kd, images, flags, state, shifts, &ws);
+}
+
+int fsharp_attend_with_state(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const float* Omega,
+                             const double* params, const fsharp_dims* dims, int dtype, int causal, float qk_scale,
+                             const float* states, const float* shifts, int n_states, void* Y) {
+  if (!ctx || !Omega || !params) return FSHARP_E_BADARG;
+  FS_TRY(check_dims(dims, true));
+  if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
+  if (n_states < 0 || (n_states > 0 && (!states || !shifts))) return FSHARP_E_BADARG;
+  if (causal ? dims->Lq != dims->Lk : n_states == 0) return FSHARP_E_SHAPE;   // bidirectional: every key is behind a state
+  if (dims->B * dims->H == 0 || dims->Lq == 0) return FSHARP_OK;
+  fsharp_dims qd = *dims;
+  if (!causal) {                       // K and V are not read: the query tensor stands in for the shape checks
+    qd.Lk = qd.Lq;
+    for (int i = 0; i < 3; i++) qd.k_stride[i] = qd.v_stride[i] = qd.q_stride[i];
+  }
+  if (!fs_tc_supported(&qd, dtype, causal, 128, qk_scale)) return FSHARP_E_SHAPE;
+  FS_TRY(check_ptr(Q, dtype, dims->q_stride));
+  FS_TRY(check_ptr(Y, dtype, dims->y_stride));
+  if (causal) {
+    FS_TRY(check_ptr(K, dtype, dims->k_stride));
+    FS_TRY(check_ptr(V, dtype, dims->v_stride));
+  }
+  FS_CUDA_OK(cudaSetDevice(ctx->device));
+  const int G = fs_groups(dims);
+  const size_t prep_f = (size_t)G * 2 * PrepLayout{dims->d, dims->M}.total();
+  const size_t img_bytes = ws_round((size_t)G * 2 * tcl::IMG_BYTES) + ws_round((size_t)G * 2 * tcl::FLAG_WORDS * 4 + 64);
+  FS_TRY(fs_ws_reserve(ctx, ws_round(prep_f * 4) + img_bytes + (causal ? fs_tc_causal_prefix_scratch_bytes(ctx, &qd, n_states) : 0)));
+  WsAlloc ws{ctx->ws, 0};
+  float* prep = ws.take<float>(prep_f);
+  uint8_t* images = ws.take<uint8_t>((size_t)G * 2 * tcl::IMG_BYTES);
+  int* flags = ws.take<int>((size_t)G * 2 * tcl::FLAG_WORDS + 16);
+  FS_TRY(fs_run_prep_images(ctx, Omega, dims->omega_head_stride, params, (int64_t)ParamsLayout{dims->d}.total(), G,
+                            dims->H, dims->pool, dims->d, dims->M, prep, qk_scale, images, flags));
+  if (causal) return fs_tc_causal_prefix(ctx, Q, K, V, &qd, images, flags, states, shifts, n_states, Y, &ws);
+  return fs_tc_query_side(ctx, Q, &qd, images, states, shifts, n_states, Y);
 }
 
 int fsharp_kernel_apply(fsharp_ctx* ctx, const void* X, const void* Y, const void* Cmat, const float* Omega,

@@ -814,6 +814,41 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
                 const int* flags, void* Y, WsAlloc* ws);
 int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                    const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax);
+int fs_tc_query_side(fsharp_ctx* ctx, const void* Q, const fsharp_dims* dm, const uint8_t* images, const float* partial,
+                     const float* shifts, int nsplit, void* Y);
+int fs_tc_key_state_splits(const fsharp_ctx* ctx, const fsharp_dims* dm, int* tiles_per_split);
+size_t fs_tc_key_state_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
+int fs_tc_key_state(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
+                    const int* flags, float* state, float* shifts, WsAlloc* ws);
+
+// The key range of a key-state call is cut into at most this many pieces (each is one [80][256] block to hand on).
+constexpr int MAX_STATE_SPLIT = 8;
+
+int fs_tc_key_state_splits(const fsharp_ctx* ctx, const fsharp_dims* dm, int* tiles_per_split) {
+  int tps = 0;
+  const int ns = pick_split(dm->B * dm->H, (dm->Lk + TILE - 1) / TILE, ctx->sm_count, MAX_STATE_SPLIT, &tps);
+  if (tiles_per_split) *tiles_per_split = tps;
+  return ns;
+}
+
+size_t fs_tc_key_state_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
+  (void)ctx;
+  const size_t BH = (size_t)dm->B * dm->H, G = fs_groups(dm);
+  return ws_round(G * 2 * IMG_BYTES) + ws_round(G * 2 * FLAG_WORDS * 4 + 64) + ws_round(BH * MAX_STATE_SPLIT * 2 * 4) +
+         ws_round(BH * (size_t)((dm->Lk + TILE - 1) / TILE) * TILE * 4);
+}
+
+// Key side alone, over all keys of the call: state [B*H][ns][80][256], shifts [B*H][ns][2] with ns = fs_tc_key_state_splits.
+int fs_tc_key_state(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
+                    const int* flags, float* state, float* shifts, WsAlloc* ws) {
+  const int BH = dm->B * dm->H;
+  int tps = 0;
+  const int ns = fs_tc_key_state_splits(ctx, dm, &tps);
+  int* pmax = ws->take<int>((size_t)BH * MAX_STATE_SPLIT * 2);
+  FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * MAX_STATE_SPLIT * 2 * sizeof(int), ctx->stream));
+  float* crow = ws->take<float>((size_t)BH * ((dm->Lk + TILE - 1) / TILE) * TILE);
+  return fs_tc_key_side(ctx, K, V, dm, images, flags, tps, ns, crow, state, shifts, pmax);
+}
 
 size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
   const size_t BH = (size_t)dm->B * dm->H;
@@ -861,6 +896,15 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   float* crow = ws->take<float>((size_t)BH * Lpad);
   FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, tps, nsplit, crow, partial, shifts, pmax));
 
+  return fs_tc_query_side(ctx, Q, dm, images, partial, shifts, nsplit, Y);
+}
+
+// Query side alone: partial [B*H][nsplit][80][256], shifts [B*H][nsplit][2] are key-side sums of disjoint key ranges
+// (of this call's key side, or handed in by the caller).
+int fs_tc_query_side(fsharp_ctx* ctx, const void* Q, const fsharp_dims* dm, const uint8_t* images, const float* partial,
+                     const float* shifts, int nsplit, void* Y) {
+  const int B = dm->B, H = dm->H, BH = B * H, Lq = dm->Lq;
+  if (nsplit < 1 || nsplit > MAX_KEY_SPLIT) return FSHARP_E_LIMIT;
   CUtensorMap tmQ;
   FS_TRY(tchost::make_map_tokens(&tmQ, Q, fs_addr(dm->q_stride, H, Lq, dm->d), B, H, Lq, dm->d));
   FS_CUDA_OK(cudaFuncSetAttribute(tc_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)OutSmem::TOTAL + 1024));

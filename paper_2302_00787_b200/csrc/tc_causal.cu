@@ -81,7 +81,7 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmY,
                  const uint8_t* __restrict__ images,
                  const float* __restrict__ crow, const float* __restrict__ partial, const float* __restrict__ shifts,
-                 int nsplit1, int H, int pool, int L, int Lpad, int tiles_per_seg, int* __restrict__ status) {
+                 int nsplit1, int nprefix, int H, int pool, int L, int Lpad, int tiles_per_seg, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   CfMisc* misc = reinterpret_cast<CfMisc*>(sm + CfSmem::MISC);
@@ -384,7 +384,8 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     };
     // ---- the state before this segment: sum of the earlier segments' totals, brought to one shift
     {
-      const int np = seg == 0 ? 0 : min(nsplit1, seg);               // key-side splits are segments
+      // key-side splits are segments; the first nprefix totals belong to keys that precede the whole sequence
+      const int np = min(nsplit1, nprefix + seg);
       float val[TC_NV];
 #pragma unroll
       for (int n = 0; n < TC_NV; n++) val[n] = 0.f;
@@ -740,6 +741,9 @@ int fs_tc_causal_supported(const fsharp_dims* dm, int chunk);
 size_t fs_tc_causal_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
 int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                  const int* flags, void* Y, WsAlloc* ws);
+size_t fs_tc_causal_prefix_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm, int nprefix);
+int fs_tc_causal_prefix(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
+                        const int* flags, const float* pre_state, const float* pre_shifts, int nprefix, void* Y, WsAlloc* ws);
 
 namespace {
 constexpr int CF_MAX_SEG = 64;
@@ -778,6 +782,19 @@ size_t fs_tc_causal_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) 
 
 int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                  const int* flags, void* Y, WsAlloc* ws) {
+  return fs_tc_causal_prefix(ctx, Q, K, V, dm, images, flags, nullptr, nullptr, 0, Y, ws);
+}
+
+size_t fs_tc_causal_prefix_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm, int nprefix) {
+  const size_t BH = (size_t)dm->B * dm->H;
+  return fs_tc_causal_scratch_bytes(ctx, dm) + ws_round(BH * (size_t)(nprefix + CF_MAX_SEG) * TC_M * TC_NV * 4) +
+         ws_round(BH * (size_t)(nprefix + CF_MAX_SEG) * 2 * 4);
+}
+
+// pre_state [B*H][nprefix][80][256], pre_shifts [B*H][nprefix][2]: key-side sums (in the layout of the key-side kernel's
+// partials) of keys that precede every token of this call; nprefix = 0: none.
+int fs_tc_causal_prefix(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
+                        const int* flags, const float* pre_state, const float* pre_shifts, int nprefix, void* Y, WsAlloc* ws) {
   const int B = dm->B, H = dm->H, BH = B * H, L = dm->Lq;
   const int nch = (L + TILE - 1) / TILE, Lpad = nch * TILE;
   float* partial = ws->take<float>((size_t)BH * CF_MAX_SEG * TC_M * TC_NV);
@@ -793,6 +810,24 @@ int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, c
   } else {
     FS_TRY(fs_tc_rowterm(ctx, K, dm, images, flags, Lpad, per, 1, crow));
   }
+  int ntot = nseg - 1;
+  if (nprefix > 0) {
+    // one list per (batch, head): the totals that precede the sequence, then those of this call's segments
+    ntot = nprefix + nseg - 1;
+    float* all = ws->take<float>((size_t)BH * ntot * TC_M * TC_NV);
+    float* allsh = ws->take<float>((size_t)BH * ntot * 2);
+    const size_t one = (size_t)TC_M * TC_NV * sizeof(float), onesh = 2 * sizeof(float);
+    FS_CUDA_OK(cudaMemcpy2DAsync(all, ntot * one, pre_state, nprefix * one, nprefix * one, BH, cudaMemcpyDeviceToDevice, ctx->stream));
+    FS_CUDA_OK(cudaMemcpy2DAsync(allsh, ntot * onesh, pre_shifts, nprefix * onesh, nprefix * onesh, BH, cudaMemcpyDeviceToDevice, ctx->stream));
+    if (nseg > 1) {
+      FS_CUDA_OK(cudaMemcpy2DAsync(all + (size_t)nprefix * TC_M * TC_NV, ntot * one, partial, (nseg - 1) * one, (nseg - 1) * one, BH,
+                                   cudaMemcpyDeviceToDevice, ctx->stream));
+      FS_CUDA_OK(cudaMemcpy2DAsync(allsh + (size_t)nprefix * 2, ntot * onesh, shifts, (nseg - 1) * onesh, (nseg - 1) * onesh, BH,
+                                   cudaMemcpyDeviceToDevice, ctx->stream));
+    }
+    partial = all;
+    shifts = allsh;
+  }
   CUtensorMap tmQ, tmK, tmV, tmY;
   FS_TRY(tchost::make_map_tokens(&tmQ, Q, fs_addr(dm->q_stride, H, L, dm->d), B, H, L, dm->d));
   FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, L, dm->d), B, H, L, dm->d));
@@ -801,7 +836,7 @@ int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, c
   FS_CUDA_OK(cudaFuncSetAttribute(tc_causal_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CfSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_CAUSAL);
   tc_causal_kernel<<<dim3(nseg, BH), TC_THREADS, CfSmem::TOTAL + 1024, ctx->stream>>>(
-      tmQ, tmK, tmV, tmY, images, crow, partial, shifts, nseg - 1, H, dm->pool, L, Lpad, per, ctx->d_status);
+      tmQ, tmK, tmV, tmY, images, crow, partial, shifts, ntot, nprefix, H, dm->pool, L, Lpad, per, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;

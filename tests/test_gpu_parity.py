@@ -354,6 +354,68 @@ def test_causal_tensor_core_path_scales_across_chunks(ctx, ramp):
     assert np.abs(Y[:, :, 0] - V[:, :, 0]).max() < 1e-2          # the first query sees only the first key
 
 
+@pytest.mark.gpu
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("slices", [(512, 512, 512), (600, 424, 512), (1280,), (130, 1150)])
+def test_sequence_parallel_key_states(ctx, causal, slices):
+    """Sequence parallelism (the token axis cut into contiguous slices, one per rank): every slice's keys are reduced
+    to a key state, the states are handed round, and every slice's queries are finished from the states they may see.
+    The ranks are emulated one after the other on this device (their kernels do not wait on one another); the result
+    must match the definition on the whole sequence, and the single call on the whole sequence."""
+    from paper_2302_00787_b200 import sharding
+    L = sum(slices)
+    w = W["cfg3"].scaled(B=1, H=3, L=L, variant="aderf")
+    Q, K, V = wl.make_qkv(w)
+    Om = wl.make_omega(w)
+    t = np.arange(L, dtype=np.float64) / L
+    K = wl.bf16_round(K * (1.0 + 1.5 * t)[None, None, :, None])       # the slices' shifts differ
+    dQ, dK, dV, dOm = dev(Q, "bf16"), dev(K, "bf16"), dev(V, "bf16"), dev(Om)
+    # per-slice statistics combined with the slice lengths as weights = statistics of the whole sequence
+    off = np.concatenate([[0], np.cumsum(slices)])
+    cut = lambda x, r: x[:, :, off[r]:off[r + 1]].contiguous()
+    st_all = ctx.fsharp_stats(dQ, dK)
+    st = sum(ctx.fsharp_stats(cut(dQ, r), cut(dK, r)) * float(n) for r, n in enumerate(slices)) / float(L)
+    assert float((st - st_all).abs().max()) <= 2e-6 * float(st_all.abs().max())    # (fp32 products per tile, fp64 sums)
+    pr = ctx.fsharp_fit_params(st, w.d, w.variant)
+    gathered = [ctx.fsharp_attend_key_state(cut(dK, r), cut(dV, r), dOm, pr) for r in range(len(slices))]
+    Y = torch.empty(w.B, w.H, L, w.dv, dtype=dQ.dtype, device="cuda")
+    for r in range(len(slices)):
+        states, shifts = sharding.select_states(gathered, r, causal)
+        Y[:, :, off[r]:off[r + 1]] = ctx.fsharp_attend_with_state(cut(dQ, r), cut(dK, r), cut(dV, r), dOm, pr, states, shifts,
+                                                                  causal=causal)
+    assert ctx.status() == 0
+    Y1 = host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=causal, chunk=128)) if L % 128 == 0 else None
+    Y = host(Y)
+    prh = pr.cpu().numpy()
+    for h in range(w.H):
+        ref = oracle_unit(Q, K, V, Om, prh[h], w.d, 0, h, causal)
+        assert rel_err(Y[0, h], ref) < TOL["bf16"], h
+        if Y1 is not None:
+            assert rel_err(Y[0, h], Y1[0, h]) < TOL["bf16"], h
+
+
+@pytest.mark.gpu
+def test_sequence_parallel_argument_checks(ctx):
+    w = W["cfg3"].scaled(B=1, H=1, L=256, variant="sderf")
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    _, pr = gpu_fit(ctx, dQ, dK, w.d, w.variant)
+    state, shifts = ctx.fsharp_attend_key_state(dK, dV, dOm, pr)
+    assert state.shape[0] == 1 and state.shape[2:] == (80, 256) and shifts.shape == (1, state.shape[1], 2)
+    with pytest.raises(fb.FsharpError) as e:            # bidirectional: every key must be behind a state
+        ctx.fsharp_attend_with_state(dQ, dK, dV, dOm, pr, None, None, causal=False)
+    assert e.value.code == -2
+    with pytest.raises(fb.FsharpError) as e:            # the tensor-core kernels' shape only
+        ctx.fsharp_attend_key_state(dK.float(), dV.float(), dOm, pr)
+    assert e.value.code == -2
+    with pytest.raises(ValueError):
+        ctx.fsharp_attend_with_state(dQ, dK, dV, dOm, pr, state[:, :, :40], shifts, causal=True)
+    # causal with nothing before it is the plain causal call
+    Y0 = host(ctx.fsharp_attend_with_state(dQ, dK, dV, dOm, pr, None, None, causal=True))
+    Y1 = host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=True, chunk=128))
+    assert np.array_equal(Y0, Y1)
+    assert ctx.status() == 0
+
+
 def test_attend_strided_layout_per_head_omega_and_pooling(ctx):
     w = W["cfg2"].scaled(B=2, H=3, L=256)
     (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
