@@ -19,6 +19,8 @@
 //   O += masked scores (from tensor memory) [V | 1]: column 64 collects the denominators       [O]
 //   T += phi(K)^T [V | 1], 128 features per accumulator                                       [T: 2 x 80]
 //   bf16(T) for the next tile: the accumulators are read back and written to shared memory
+//   Y rows of the previous tile: [O] normalised, staged in the idle token tile, one TMA store per warp
+// A block may also start from handed-in totals of keys that precede its whole sequence (sequence parallelism).
 // The token tiles are converted from bf16 to fp16 in shared memory (exact for |x| in [2^-14, 65504]), so the
 // logits need one fp16 image of W (11 significant bits) instead of a bf16 value and its remainder.
 // The keys of a segment share one running shift (raised, with the state rescaled, when a tile's largest
