@@ -75,3 +75,27 @@ def test_long_sequence_causal_sampled_parity(ctx):
     host_in, dev_in, pr, Y = run_full(ctx, w)
     assert torch.isfinite(Y.float()).all()
     check_sampled(w, host_in, pr, Y, [(0, 0), (0, 9)], 12, 5)
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_long_sequence_tensor_core_path_sampled_parity(ctx, causal):
+    """Few, long sequences on the tensor-core kernels: L = 65536, d = 64, M = 256, 2 heads (512 tiles per head: the causal
+    state is carried through 512 tiles in fp32 tensor memory, the key-side sums through many splits), as one call and
+    as four slices of the token axis finished from handed-on key states (the ranks of the sequence-parallel form, run
+    one after the other on this device)."""
+    from paper_2302_00787_b200 import sharding
+    w = wl.WORKLOADS["cfg3"].scaled(B=1, H=2, L=65536, causal=causal)
+    host_in, (dQ, dK, dV, dOm), pr, Y = run_full(ctx, w)
+    assert torch.isfinite(Y.float()).all()
+    check_sampled(w, host_in, pr, Y, [(0, 0), (0, 1)], 12, 7)
+    R = 4
+    n = w.L // R
+    cut = lambda x, r: x[:, :, r * n:(r + 1) * n].contiguous()
+    gathered = [ctx.fsharp_attend_key_state(cut(dK, r), cut(dV, r), dOm, pr) for r in range(R)]
+    Ys = torch.empty_like(Y)
+    for r in range(R):
+        states, shifts = sharding.select_states(gathered, r, causal)
+        Ys[:, :, r * n:(r + 1) * n] = ctx.fsharp_attend_with_state(cut(dQ, r), cut(dK, r), cut(dV, r), dOm, pr, states, shifts,
+                                                                   causal=causal)
+    assert ctx.status() == 0
+    check_sampled(w, host_in, pr, Ys, [(0, 1)], 12, 9)
