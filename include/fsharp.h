@@ -59,7 +59,8 @@ enum {
   FSHARP_E_NONFINITE = -7,  /* NaN or Inf met on the device */
   FSHARP_E_TIMEOUT = -8,    /* a bounded device-side wait expired */
   FSHARP_E_CUDA = -9,       /* a CUDA runtime or driver call failed */
-  FSHARP_E_LIMIT = -10,     /* problem needs more than the fixed scratch of fsharp_featurize_static */
+  FSHARP_E_LIMIT = -10,     /* problem needs more than the fixed scratch of fsharp_featurize_static, or more key
+                             * states than one query-side launch merges */
   FSHARP_E_INTERNAL = -11   /* an index check of the debug build (-DFSHARP_DEBUG) failed on the device */
 };
 

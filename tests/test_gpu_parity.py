@@ -412,6 +412,23 @@ def test_sequence_parallel_argument_checks(ctx):
     assert e.value.code == -2
     with pytest.raises(ValueError):
         ctx.fsharp_attend_with_state(dQ, dK, dV, dOm, pr, state[:, :, :40], shifts, causal=True)
+    many = state[:, :1].expand(1, 65, 80, 256).contiguous()                      # more states than one launch merges
+    with pytest.raises(fb.FsharpError) as e:
+        ctx.fsharp_attend_with_state(dQ, None, None, dOm, pr, many, shifts[:, :1].expand(1, 65, 2).contiguous(), causal=False)
+    assert e.value.code == -10
+    # the same states twice = every key counted twice: numerator and normaliser double, the output does not change
+    twice = (torch.cat([state, state], dim=1).contiguous(), torch.cat([shifts, shifts], dim=1).contiguous())
+    Ya = host(ctx.fsharp_attend_with_state(dQ, None, None, dOm, pr, state, shifts, causal=False))
+    Yb = host(ctx.fsharp_attend_with_state(dQ, None, None, dOm, pr, twice[0], twice[1], causal=False))
+    assert np.abs(Ya - Yb).max() <= 2.0 ** -7 * np.abs(Ya).max()
+    assert rel_err(Ya, host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr))) < TOL["bf16"]
+    # strided tensors ([B, L, H, d] storage) and one parameter group per head
+    tr = lambda t: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    st_h = ctx.fsharp_stats(dQ, dK, pool=fb.POOL_PER_HEAD)
+    pr_h = ctx.fsharp_fit_params(st_h, w.d, w.variant)
+    s2, h2 = ctx.fsharp_attend_key_state(tr(dK), tr(dV), dOm, pr_h, pool=fb.POOL_PER_HEAD)
+    Yc = host(ctx.fsharp_attend_with_state(tr(dQ), None, None, dOm, pr_h, s2, h2, causal=False, pool=fb.POOL_PER_HEAD))
+    assert rel_err(Yc, host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr_h, pool=fb.POOL_PER_HEAD))) < TOL["bf16"]
     # causal with nothing before it is the plain causal call
     Y0 = host(ctx.fsharp_attend_with_state(dQ, dK, dV, dOm, pr, None, None, causal=True))
     Y1 = host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=True, chunk=128))
