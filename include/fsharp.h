@@ -246,7 +246,9 @@ int fsharp_kernel_apply(fsharp_ctx* ctx, const void* X, const void* Y, const voi
 /* The whole path on HOST buffers: copies Q, K, V (dense [B,H,L,*], type `dtype`)
  * to the device, runs stats -> fit -> attend, copies Y back and waits for it.
  * Q, K, V, Y: host memory (pinned memory makes the copies asynchronous).
- * Omega: host float32 [M, d].  dims' strides are ignored (dense). */
+ * Omega: host float32 [M, d].  dims' strides are ignored (dense).
+ * With one parameter group per (batch, head) the batch elements go through one after the other: the upload of one, the
+ * path on the one before and the download of the one before that overlap (three streams owned by the context). */
 int fsharp_forward_host(fsharp_ctx* ctx, const void* Q, const void* K, const void* V,
                         const float* Omega, const fsharp_dims* dims, int dtype, int variant,
                         int causal, int chunk, float qk_scale, void* Y);

@@ -306,22 +306,46 @@ int fsharp_forward_host(fsharp_ctx* ctx, const void* Q, const void* K, const voi
   double* dP = ws.take<double>(nparams / 8);
   if (!ctx->copy_stream) {
     FS_CUDA_OK(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+    FS_CUDA_OK(cudaStreamCreateWithFlags(&ctx->down_stream, cudaStreamNonBlocking));
     FS_CUDA_OK(cudaEventCreateWithFlags(&ctx->ev_inputs, cudaEventDisableTiming));
     FS_CUDA_OK(cudaEventCreateWithFlags(&ctx->ev_v, cudaEventDisableTiming));
   }
-  // Q, K and Omega go up first; V follows on a stream of its own while statistics and fit run
-  FS_CUDA_OK(cudaMemcpyAsync(dQ, Q, nq, cudaMemcpyHostToDevice, ctx->stream));
-  FS_CUDA_OK(cudaMemcpyAsync(dK, K, nk, cudaMemcpyHostToDevice, ctx->stream));
-  FS_CUDA_OK(cudaMemcpyAsync(dO, Omega, no, cudaMemcpyHostToDevice, ctx->stream));
+  // With one parameter group per (batch, head) the batch elements are independent all the way: element b's inputs go up
+  // on the upload stream while element b - 1 runs on the context's stream and element b - 2's rows come down on the
+  // download stream.  (An event may be recorded again while an earlier wait on it is pending: a wait refers to the
+  // record that preceded it.)  Pooled groups (one per head over the whole batch) make one piece of the whole batch.
+  const int pieces = dd.pool == FSHARP_POOL_PER_BH ? dd.B : 1;
+  fsharp_dims dp = dd;
+  dp.B = dd.B / pieces;
+  const size_t f = (size_t)pieces;
+  const int Gp = G / pieces;
+  // the uploads start when the stream's earlier work (which may still read the staging buffers) has finished
   FS_CUDA_OK(cudaEventRecord(ctx->ev_inputs, ctx->stream));
   FS_CUDA_OK(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_inputs, 0));
-  FS_CUDA_OK(cudaMemcpyAsync(dV, V, nv, cudaMemcpyHostToDevice, ctx->copy_stream));
-  FS_CUDA_OK(cudaEventRecord(ctx->ev_v, ctx->copy_stream));
-  FS_TRY(fsharp_stats(ctx, dQ, dK, &dd, dtype, qk_scale, dS));
-  FS_TRY(fsharp_fit_params(ctx, dS, G, dd.d, variant, 0.0, dP));
-  FS_CUDA_OK(cudaStreamWaitEvent(ctx->stream, ctx->ev_v, 0));
-  FS_TRY(fsharp_attend(ctx, dQ, dK, dV, dO, dP, &dd, dtype, causal, chunk, qk_scale, dY));
-  FS_CUDA_OK(cudaMemcpyAsync(Y, dY, ny, cudaMemcpyDeviceToHost, ctx->stream));
+  FS_CUDA_OK(cudaStreamWaitEvent(ctx->down_stream, ctx->ev_inputs, 0));
+  FS_CUDA_OK(cudaMemcpyAsync(dO, Omega, no, cudaMemcpyHostToDevice, ctx->copy_stream));
+  for (int p = 0; p < pieces; p++) {
+    const char* hQ = static_cast<const char*>(Q) + p * (nq / f);
+    const char* hK = static_cast<const char*>(K) + p * (nk / f);
+    const char* hV = static_cast<const char*>(V) + p * (nv / f);
+    char *pQ = dQ + p * (nq / f), *pK = dK + p * (nk / f), *pV = dV + p * (nv / f), *pY = dY + p * (ny / f);
+    double* pS = dS + (size_t)p * Gp * StatsLayout{dd.d}.total();
+    double* pP = dP + (size_t)p * Gp * ParamsLayout{dd.d}.total();
+    FS_CUDA_OK(cudaMemcpyAsync(pQ, hQ, nq / f, cudaMemcpyHostToDevice, ctx->copy_stream));
+    FS_CUDA_OK(cudaMemcpyAsync(pK, hK, nk / f, cudaMemcpyHostToDevice, ctx->copy_stream));
+    FS_CUDA_OK(cudaEventRecord(ctx->ev_inputs, ctx->copy_stream));
+    FS_CUDA_OK(cudaMemcpyAsync(pV, hV, nv / f, cudaMemcpyHostToDevice, ctx->copy_stream));
+    FS_CUDA_OK(cudaEventRecord(ctx->ev_v, ctx->copy_stream));
+    FS_CUDA_OK(cudaStreamWaitEvent(ctx->stream, ctx->ev_inputs, 0));
+    FS_TRY(fsharp_stats(ctx, pQ, pK, &dp, dtype, qk_scale, pS));
+    FS_TRY(fsharp_fit_params(ctx, pS, Gp, dd.d, variant, 0.0, pP));
+    FS_CUDA_OK(cudaStreamWaitEvent(ctx->stream, ctx->ev_v, 0));
+    FS_TRY(fsharp_attend(ctx, pQ, pK, pV, dO, pP, &dp, dtype, causal, chunk, qk_scale, pY));
+    FS_CUDA_OK(cudaEventRecord(ctx->ev_v, ctx->stream));
+    FS_CUDA_OK(cudaStreamWaitEvent(ctx->down_stream, ctx->ev_v, 0));
+    FS_CUDA_OK(cudaMemcpyAsync(static_cast<char*>(Y) + p * (ny / f), pY, ny / f, cudaMemcpyDeviceToHost, ctx->down_stream));
+  }
+  FS_CUDA_OK(cudaStreamSynchronize(ctx->down_stream));
   FS_CUDA_OK(cudaStreamSynchronize(ctx->stream));
   return FSHARP_OK;
 }

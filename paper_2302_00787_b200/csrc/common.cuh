@@ -68,8 +68,9 @@ struct fsharp_ctx {
   int t_used;
   cudaEvent_t* t_ev;  // 2 * FS_TIMING_SLOTS, created on first use
   int* t_tag;
-  // second stream and two events of fsharp_forward_host (V is uploaded while statistics and fit run); created on first use
-  cudaStream_t copy_stream;
+  // the two copy streams and events of fsharp_forward_host (uploads, downloads and the path overlap batch element by
+  // batch element); created on first use
+  cudaStream_t copy_stream, down_stream;
   cudaEvent_t ev_inputs, ev_v;
 };
 

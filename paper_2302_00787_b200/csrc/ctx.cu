@@ -29,6 +29,7 @@ int fsharp_create(fsharp_ctx** out, int device, void* stream) {
   c->t_ev = nullptr;
   c->t_tag = nullptr;
   c->copy_stream = nullptr;
+  c->down_stream = nullptr;
   c->ev_inputs = nullptr;
   c->ev_v = nullptr;
   cudaDeviceProp prop;
@@ -57,6 +58,8 @@ int fsharp_destroy(fsharp_ctx* ctx) {
   if (ctx->copy_stream) {
     cudaStreamSynchronize(ctx->copy_stream);
     cudaStreamDestroy(ctx->copy_stream);
+    cudaStreamSynchronize(ctx->down_stream);
+    cudaStreamDestroy(ctx->down_stream);
     cudaEventDestroy(ctx->ev_inputs);
     cudaEventDestroy(ctx->ev_v);
   }

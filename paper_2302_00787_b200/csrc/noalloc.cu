@@ -99,6 +99,7 @@ extern "C" int fsharp_featurize_static(void* stream, const void* X, const float*
   ctx.t_ev = nullptr;
   ctx.t_tag = nullptr;
   ctx.copy_stream = nullptr;
+  ctx.down_stream = nullptr;
   ctx.ev_inputs = nullptr;
   ctx.ev_v = nullptr;
 
