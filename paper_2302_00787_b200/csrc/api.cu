@@ -55,6 +55,7 @@ extern "C" {
 
 int fsharp_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dims* dims, int dtype,
                  float qk_scale, double* stats) {
+  FS_RANGE("fsharp_stats");
   if (!ctx) return FSHARP_E_BADARG;
   FS_TRY(check_dims(dims, false));
   if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
@@ -68,6 +69,7 @@ int fsharp_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dim
 
 int fsharp_fit_params(fsharp_ctx* ctx, const double* stats, int G, int d, int variant, double ridge,
                       double* params) {
+  FS_RANGE("fsharp_fit_params");
   if (!ctx || !stats || !params) return FSHARP_E_BADARG;
   if (G < 0 || !dim_ok(d)) return FSHARP_E_SHAPE;
   if (variant < FSHARP_POSRF || variant > FSHARP_SDERF) return FSHARP_E_BADARG;
@@ -81,6 +83,7 @@ int fsharp_fit_params(fsharp_ctx* ctx, const double* stats, int G, int d, int va
 
 int fsharp_featurize(fsharp_ctx* ctx, const void* X, const float* Omega, const double* params, int side,
                      const fsharp_dims* dims, int dtype, float qk_scale, int stab, float* phi, float* logscale) {
+  FS_RANGE("fsharp_featurize");
   if (!ctx || !Omega || !params || !phi) return FSHARP_E_BADARG;
   FS_TRY(check_dims(dims, false));
   if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
@@ -126,6 +129,7 @@ int fsharp_featurize(fsharp_ctx* ctx, const void* X, const float* Omega, const d
 int fsharp_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const float* Omega,
                   const double* params, const fsharp_dims* dims, int dtype, int causal, int chunk, float qk_scale,
                   void* Y) {
+  FS_RANGE("fsharp_attend");
   if (!ctx || !Omega || !params) return FSHARP_E_BADARG;
   FS_TRY(check_dims(dims, true));
   if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
@@ -177,6 +181,7 @@ int fsharp_key_state_splits(fsharp_ctx* ctx, const fsharp_dims* dims) {
 
 int fsharp_attend_key_state(fsharp_ctx* ctx, const void* K, const void* V, const float* Omega, const double* params,
                             const fsharp_dims* dims, int dtype, float qk_scale, float* state, float* shifts) {
+  FS_RANGE("fsharp_attend_key_state");
   if (!ctx || !Omega || !params || !state || !shifts) return FSHARP_E_BADARG;
   FS_TRY(check_dims(dims, true));
   if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
@@ -205,6 +210,7 @@ int fsharp_attend_key_state(fsharp_ctx* ctx, const void* K, const void* V, const
 int fsharp_attend_with_state(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const float* Omega,
                              const double* params, const fsharp_dims* dims, int dtype, int causal, float qk_scale,
                              const float* states, const float* shifts, int n_states, void* Y) {
+  FS_RANGE("fsharp_attend_with_state");
   if (!ctx || !Omega || !params) return FSHARP_E_BADARG;
   FS_TRY(check_dims(dims, true));
   if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
@@ -240,6 +246,7 @@ int fsharp_attend_with_state(fsharp_ctx* ctx, const void* Q, const void* K, cons
 
 int fsharp_kernel_apply(fsharp_ctx* ctx, const void* X, const void* Y, const void* Cmat, const float* Omega,
                         const double* params, double alpha, const fsharp_dims* dims, int dtype, float qk_scale, void* out) {
+  FS_RANGE("fsharp_kernel_apply");
   if (!ctx || !Omega || !params) return FSHARP_E_BADARG;
   FS_TRY(check_dims(dims, true));
   if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
@@ -267,6 +274,7 @@ int fsharp_kernel_apply(fsharp_ctx* ctx, const void* X, const void* Y, const voi
 int fsharp_forward_host(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const float* Omega,
                         const fsharp_dims* dims, int dtype, int variant, int causal, int chunk, float qk_scale,
                         void* Y) {
+  FS_RANGE("fsharp_forward_host");
   if (!ctx || !Q || !K || !V || !Omega || !Y) return FSHARP_E_BADARG;
   FS_TRY(check_dims(dims, true));
   if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
@@ -352,6 +360,7 @@ int fsharp_forward_host(fsharp_ctx* ctx, const void* Q, const void* K, const voi
 
 int fsharp_pair_estimate(fsharp_ctx* ctx, const float* X, const float* Y, const float* Omega, const double* params,
                          int64_t npairs, int d, int M, int R, float* est, double* var_cf, double* pooled) {
+  FS_RANGE("fsharp_pair_estimate");
   if (!ctx || !Omega || !params) return FSHARP_E_BADARG;
   if (pooled && !var_cf) return FSHARP_E_BADARG;
   if (npairs < 0 || !dim_ok(d) || M <= 0 || M % 16 != 0 || M > 1024 || R <= 0 || R > 65535) return FSHARP_E_SHAPE;

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <stddef.h>
@@ -73,6 +74,15 @@ struct fsharp_ctx {
   cudaStream_t copy_stream, down_stream;
   cudaEvent_t ev_inputs, ev_v;
 };
+
+// NVTX range of a host-side stage (a no-op unless a tool that listens to NVTX is attached)
+struct FsRange {
+  explicit FsRange(const char* name) { nvtxRangePushA(name); }
+  ~FsRange() { nvtxRangePop(); }
+  FsRange(const FsRange&) = delete;
+  FsRange& operator=(const FsRange&) = delete;
+};
+#define FS_RANGE(name) FsRange fs_range_guard_(name)
 
 void fs_time_begin(fsharp_ctx* ctx, int tag);
 void fs_time_end(fsharp_ctx* ctx);

@@ -212,6 +212,7 @@ int fs_run_prep(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_stride, 
 int fs_run_prep_images(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_stride, const double* params,
                        int64_t params_stride, int G, int H, int pool, int d, int M, float* prep, float qk_scale,
                        uint8_t* images, int* flags) {
+  FS_RANGE("operand images");
   if (G == 0) return FSHARP_OK;
   if (images != nullptr && (d != tcl::TC_D || M != tcl::TC_M)) return FSHARP_E_SHAPE;
   const int nchunks = (M + PREP_MB - 1) / PREP_MB;

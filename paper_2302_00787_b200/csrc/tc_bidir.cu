@@ -865,6 +865,7 @@ size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
 // first nsplit * tiles_per_split tiles (the causal path asks for the segments that have a successor only).
 int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                    const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax) {
+  FS_RANGE("key side");
   const int B = dm->B, H = dm->H, Lk = dm->Lk;
   const int Lpad = (Lk + TILE - 1) / TILE * TILE;
   FS_TRY(fs_tc_rowterm(ctx, K, dm, images, flags, Lpad, tiles_per_split, nsplit, crow));
@@ -903,6 +904,7 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
 // (of this call's key side, or handed in by the caller).
 int fs_tc_query_side(fsharp_ctx* ctx, const void* Q, const fsharp_dims* dm, const uint8_t* images, const float* partial,
                      const float* shifts, int nsplit, void* Y) {
+  FS_RANGE("query side");
   const int B = dm->B, H = dm->H, BH = B * H, Lq = dm->Lq;
   if (nsplit < 1 || nsplit > MAX_KEY_SPLIT) return FSHARP_E_LIMIT;
   CUtensorMap tmQ;

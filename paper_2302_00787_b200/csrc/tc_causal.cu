@@ -797,6 +797,7 @@ size_t fs_tc_causal_prefix_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dim
 // partials) of keys that precede every token of this call; nprefix = 0: none.
 int fs_tc_causal_prefix(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                         const int* flags, const float* pre_state, const float* pre_shifts, int nprefix, void* Y, WsAlloc* ws) {
+  FS_RANGE("causal segments");
   const int B = dm->B, H = dm->H, BH = B * H, L = dm->Lq;
   const int nch = (L + TILE - 1) / TILE, Lpad = nch * TILE;
   float* partial = ws->take<float>((size_t)BH * CF_MAX_SEG * TC_M * TC_NV);
