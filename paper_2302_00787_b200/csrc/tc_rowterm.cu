@@ -83,28 +83,31 @@ tc_rowterm_kernel(const __grid_constant__ CUtensorMap tmK, const uint8_t* __rest
         mbar_wait(&misc->full[it % RT_STAGES], (it / RT_STAGES) & 1, abortp, status, false);
     }
   } else if (warp == RT_WARP_MMA) {
-    if (lane == 0) {
-      constexpr uint32_t ID_T = idesc_bf16(128, TC_D, 0, 0);
-      const uint64_t dX0 = smem_desc(smem_u32(sm + RtSmem::X0), 16, 1024, SWZ_128B);
-      const uint64_t dChi = smem_desc(smem_u32(sm + RtSmem::CHI), 16, 1024, SWZ_128B);
-      const uint64_t dClo = smem_desc(smem_u32(sm + RtSmem::CLO), 16, 1024, SWZ_128B);
-      bool ok = mbar_wait(&misc->const_bar, 0, abortp, status);
-      for (int it = 0; ok && it < ntiles; it++) {
-        const int st = it % RT_STAGES, buf = it & 1;
-        if (!mbar_wait(&misc->full[st], (it / RT_STAGES) & 1, abortp, status)) break;
-        if (!mbar_wait(&misc->t_free[buf], ((it >> 1) & 1) ^ 1, abortp, status)) break;
-        tcgen05_fence_after();
-        const uint64_t dX = desc_advance(dX0, st * TILE_BYTES);
+    // The whole warp walks the schedule (waits and descriptor arithmetic stay warp-uniform); one elected lane issues.
+    constexpr uint32_t ID_T = idesc_bf16(128, TC_D, 0, 0);
+    const uint64_t dX0 = smem_desc(smem_u32(sm + RtSmem::X0), 16, 1024, SWZ_128B);
+    const uint64_t dChi = smem_desc(smem_u32(sm + RtSmem::CHI), 16, 1024, SWZ_128B);
+    const uint64_t dClo = smem_desc(smem_u32(sm + RtSmem::CLO), 16, 1024, SWZ_128B);
+    uint32_t xl0 = (uint32_t)dX0, chl = (uint32_t)dChi, cll = (uint32_t)dClo;
+    const uint32_t xh = (uint32_t)(dX0 >> 32), ch = (uint32_t)(dChi >> 32);
+    bool ok = __all_sync(0xffffffffu, mbar_wait(&misc->const_bar, 0, abortp, status));
+    for (int it = 0; ok && it < ntiles; it++) {
+      const int st = it % RT_STAGES, buf = it & 1;
+      if (!__all_sync(0xffffffffu, mbar_wait(&misc->full[st], (it / RT_STAGES) & 1, abortp, status))) break;
+      if (!__all_sync(0xffffffffu, mbar_wait(&misc->t_free[buf], ((it >> 1) & 1) ^ 1, abortp, status))) break;
+      tcgen05_fence_after();
+      opaque(xl0); opaque(chl); opaque(cll);
+      const uint32_t xl = xl0 + st * (TILE_BYTES / 16);
+      if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < TC_D / 16; k++)
-          mma_bf16(tmem + buf * TC_D, desc_advance(dX, 32 * k), desc_advance(dChi, 32 * k), ID_T, k > 0);
+        for (int k = 0; k < TC_D / 16; k++) mma_bf16_lh(tmem + buf * TC_D, xl + 2 * k, xh, chl + 2 * k, ch, ID_T, k > 0 ? 1u : 0u);
         if (clo) {
 #pragma unroll
-          for (int k = 0; k < TC_D / 16; k++)
-            mma_bf16(tmem + buf * TC_D, desc_advance(dX, 32 * k), desc_advance(dClo, 32 * k), ID_T, 1);
+          for (int k = 0; k < TC_D / 16; k++) mma_bf16_lh(tmem + buf * TC_D, xl + 2 * k, xh, cll + 2 * k, ch, ID_T, 1u);
         }
         mma_commit(&misc->t_full[buf]);
       }
+      __syncwarp();
     }
   } else {
     // epilogue: one key row per thread

@@ -85,26 +85,31 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         mbar_wait(&misc->full[it % ST_STAGES], (it / ST_STAGES) & 1, abortp, status, false);
     }
   } else if (warp == ST_WARP_MMA) {
-    if (lane == 0) {
-      constexpr uint32_t ID = idesc_bf16(128, TC_D, 1, 1);      // both operands MN-major (feature index contiguous)
-      const uint32_t sX0 = smem_u32(sm + StSmem::X0), sOnes = smem_u32(sm + StSmem::ONES);
-      for (int it = 0; it < ntiles; it++) {
-        const int st = it % ST_STAGES, grp = it / ST_FOLD, buf = grp & 1, sub = it % ST_FOLD;
-        if (!mbar_wait(&misc->full[st], (it / ST_STAGES) & 1, abortp, status)) break;
-        if (sub == 0 && !mbar_wait(&misc->acc_free[buf], ((grp >> 1) & 1) ^ 1, abortp, status)) break;
-        tcgen05_fence_after();
-        const uint32_t sX = sX0 + st * TILE_BYTES;
-        // A = [X | E]: block 0 the tile, block 1 the constant tile (leading offset = their distance)
-        const uint64_t dA = smem_desc(sX, sOnes - sX, 1024, SWZ_128B);
-        const uint64_t dB = smem_desc(sX, TILE_BYTES, 1024, SWZ_128B);
-        // unrolled: a step's descriptors are the tile's plus a constant; issued from a rolled loop (index
-        // arithmetic on the dependent chain) an MMA costs its thread noticeably longer
+    // The whole warp walks the schedule (waits and descriptor arithmetic stay warp-uniform); one elected lane issues.
+    // An MMA issued by a single lane of a diverged warp costs its thread two to three times as long.
+    constexpr uint32_t ID = idesc_bf16(128, TC_D, 1, 1);      // both operands MN-major (feature index contiguous)
+    const uint32_t sX0 = smem_u32(sm + StSmem::X0), sOnes = smem_u32(sm + StSmem::ONES);
+    for (int it = 0; it < ntiles; it++) {
+      const int st = it % ST_STAGES, grp = it / ST_FOLD, buf = grp & 1, sub = it % ST_FOLD;
+      if (!__all_sync(0xffffffffu, mbar_wait(&misc->full[st], (it / ST_STAGES) & 1, abortp, status))) break;
+      if (sub == 0 && !__all_sync(0xffffffffu, mbar_wait(&misc->acc_free[buf], ((grp >> 1) & 1) ^ 1, abortp, status))) break;
+      tcgen05_fence_after();
+      const uint32_t sX = sX0 + st * TILE_BYTES;
+      // A = [X | E]: block 0 the tile, block 1 the constant tile (leading offset = their distance); a step's
+      // descriptors are the tile's plus a constant in the low word (start address / 16)
+      const uint64_t dA = smem_desc(sX, sOnes - sX, 1024, SWZ_128B);
+      const uint64_t dB = smem_desc(sX, TILE_BYTES, 1024, SWZ_128B);
+      uint32_t al = (uint32_t)dA, bl = (uint32_t)dB;
+      const uint32_t ah = (uint32_t)(dA >> 32), bh = (uint32_t)(dB >> 32);
+      opaque(al); opaque(bl);
+      if (elect_one()) {
 #pragma unroll
         for (int k = 0; k < TILE / 16; k++)
-          mma_bf16(tmem + buf * TC_D, desc_advance(dA, k * 2048), desc_advance(dB, k * 2048), ID, (k > 0 || sub > 0) ? 1 : 0);
+          mma_bf16_lh(tmem + buf * TC_D, al + k * 128, ah, bl + k * 128, bh, ID, (k > 0 || sub > 0) ? 1u : 0u);
         if (sub == ST_FOLD - 1 || it == ntiles - 1) mma_commit(&misc->acc_full[buf]);
         mma_commit(&misc->empty[st]);
       }
+      __syncwarp();
     }
   } else {
     // epilogue: thread = row of D (rows 0..63 Gram, row 64 column sums), 64 columns

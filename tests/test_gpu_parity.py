@@ -393,8 +393,8 @@ def test_sequence_parallel_key_states(ctx, causal, slices):
     for h in range(w.H):
         ref = oracle_unit(Q, K, V, Om, prh[h], w.d, 0, h, causal)
         assert rel_err(Y[0, h], ref) < TOL["bf16"], h
-        if Y1 is not None:
-            assert rel_err(Y[0, h], Y1[0, h]) < TOL["bf16"], h
+        if Y1 is not None:                   # two results that are each within the tolerance of the definition
+            assert rel_err(Y[0, h], Y1[0, h]) < 2 * TOL["bf16"], h
 
 
 @pytest.mark.gpu
@@ -421,14 +421,14 @@ def test_sequence_parallel_argument_checks(ctx):
     Ya = host(ctx.fsharp_attend_with_state(dQ, None, None, dOm, pr, state, shifts, causal=False))
     Yb = host(ctx.fsharp_attend_with_state(dQ, None, None, dOm, pr, twice[0], twice[1], causal=False))
     assert np.abs(Ya - Yb).max() <= 2.0 ** -7 * np.abs(Ya).max()
-    assert rel_err(Ya, host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr))) < TOL["bf16"]
+    assert rel_err(Ya, host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr))) < 2 * TOL["bf16"]
     # strided tensors ([B, L, H, d] storage) and one parameter group per head
     tr = lambda t: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
     st_h = ctx.fsharp_stats(dQ, dK, pool=fb.POOL_PER_HEAD)
     pr_h = ctx.fsharp_fit_params(st_h, w.d, w.variant)
     s2, h2 = ctx.fsharp_attend_key_state(tr(dK), tr(dV), dOm, pr_h, pool=fb.POOL_PER_HEAD)
     Yc = host(ctx.fsharp_attend_with_state(tr(dQ), None, None, dOm, pr_h, s2, h2, causal=False, pool=fb.POOL_PER_HEAD))
-    assert rel_err(Yc, host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr_h, pool=fb.POOL_PER_HEAD))) < TOL["bf16"]
+    assert rel_err(Yc, host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr_h, pool=fb.POOL_PER_HEAD))) < 2 * TOL["bf16"]
     # causal with nothing before it is the plain causal call
     Y0 = host(ctx.fsharp_attend_with_state(dQ, dK, dV, dOm, pr, None, None, causal=True))
     Y1 = host(ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=True, chunk=128))
