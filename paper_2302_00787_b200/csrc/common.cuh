@@ -84,6 +84,32 @@ struct FsRange {
 };
 #define FS_RANGE(name) FsRange fs_range_guard_(name)
 
+// Programmatic dependent launch: a kernel launched with fs_launch_chained may be scheduled while the kernel before it
+// in the stream is still draining; it must not touch global memory before fs_grid_dependency_wait() (which returns
+// when that kernel has completed and its writes are visible), and it lets ITS successor be scheduled only after that
+// wait, so everything older than its predecessor is complete as well.  Launched the ordinary way both calls do nothing.
+#ifdef __CUDACC__
+__device__ __forceinline__ void fs_grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t fs_launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                     Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 void fs_time_begin(fsharp_ctx* ctx, int tag);
 void fs_time_end(fsharp_ctx* ctx);
 #define FS_TIME_BEGIN(ctx, tag) do { if ((ctx)->timing) fs_time_begin((ctx), (tag)); } while (0)

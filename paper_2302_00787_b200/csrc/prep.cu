@@ -24,6 +24,7 @@ __global__ void __launch_bounds__(PREP_THREADS)
 prep_kernel(const float* __restrict__ Omega, int64_t omega_head_stride, const double* __restrict__ params,
             int64_t params_stride, int H, int pool, int M, float* __restrict__ prep, float qk_scale,
             uint8_t* __restrict__ images, int* __restrict__ img_flags) {
+  fs_grid_dependency_wait();
   // images != nullptr (d = 64, M = 256 only): the tensor-core path's operand images of this (group, side)
   // are written as well, in the layouts of tc_layout.cuh
   constexpr int d = D, NC = D / 16;
@@ -222,7 +223,7 @@ int fs_run_prep_images(fsharp_ctx* ctx, const float* Omega, int64_t omega_head_s
   do {                                                                                                               \
     FS_CUDA_OK(cudaFuncSetAttribute(prep_kernel<DD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));        \
     FS_TIME_BEGIN(ctx, FS_K_PREP);                                                                                    \
-    prep_kernel<DD><<<grid, PREP_THREADS, smem, ctx->stream>>>(Omega, omega_head_stride, params, params_stride, H,   \
+    (void)fs_launch_chained(prep_kernel<DD>, grid, dim3(PREP_THREADS), smem, ctx->stream, Omega, omega_head_stride, params, params_stride, H,   \
                                                                pool, M, prep, qk_scale, images, flags);              \
   } while (0)
   switch (d) {

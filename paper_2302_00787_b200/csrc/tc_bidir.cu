@@ -72,6 +72,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
              const uint8_t* __restrict__ images, const float* __restrict__ crow, int H, int pool, int L, int Lpad,
              int tiles_per_split, int nsplit, float* __restrict__ partial, float* __restrict__ shifts,
              int* __restrict__ pmax, int* __restrict__ status) {
+  fs_grid_dependency_wait();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   KvMisc* misc = reinterpret_cast<KvMisc*>(sm + KvSmem::MISC);
@@ -454,6 +455,7 @@ tc_out_kernel(const __grid_constant__ CUtensorMap tmQ, const uint8_t* __restrict
               const float* __restrict__ partial, const float* __restrict__ shifts, int nsplit, int H, int pool, int L,
               int tiles_per_split,
               __nv_bfloat16* __restrict__ Y, TensorAddr ay, int* __restrict__ status) {
+  fs_grid_dependency_wait();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   OutMisc* misc = reinterpret_cast<OutMisc*>(sm + OutSmem::MISC);
@@ -874,7 +876,7 @@ int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_d
   FS_TRY(tchost::make_map_tokens(&tmV, V, fs_addr(dm->v_stride, H, Lk, dm->dv), B, H, Lk, dm->dv));
   FS_CUDA_OK(cudaFuncSetAttribute(tc_kv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KvSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_KV);
-  tc_kv_kernel<<<dim3(nsplit, B * H), TC_THREADS, KvSmem::TOTAL + 1024, ctx->stream>>>(
+  (void)fs_launch_chained(tc_kv_kernel, dim3(nsplit, B * H), dim3(TC_THREADS), KvSmem::TOTAL + 1024, ctx->stream,
       tmK, tmV, images, crow, H, dm->pool, Lk, Lpad, tiles_per_split, nsplit, partial, shifts, pmax, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
@@ -914,7 +916,7 @@ int fs_tc_query_side(fsharp_ctx* ctx, const void* Q, const fsharp_dims* dm, cons
   int qtps = 0;
   int qsplit = pick_split(BH, qtiles, ctx->sm_count, 1 << 20, &qtps);
   FS_TIME_BEGIN(ctx, FS_K_TC_OUT);
-  tc_out_kernel<<<dim3(qsplit, BH), TC_THREADS, OutSmem::TOTAL + 1024, ctx->stream>>>(
+  (void)fs_launch_chained(tc_out_kernel, dim3(qsplit, BH), dim3(TC_THREADS), OutSmem::TOTAL + 1024, ctx->stream,
       tmQ, images, partial, shifts, nsplit, H, dm->pool, Lq, qtps, (__nv_bfloat16*)Y, fs_addr(dm->y_stride, H, Lq, dm->dv), ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);

@@ -84,6 +84,7 @@ tc_causal_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                  const uint8_t* __restrict__ images,
                  const float* __restrict__ crow, const float* __restrict__ partial, const float* __restrict__ shifts,
                  int nsplit1, int nprefix, int H, int pool, int L, int Lpad, int tiles_per_seg, int* __restrict__ status) {
+  fs_grid_dependency_wait();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   CfMisc* misc = reinterpret_cast<CfMisc*>(sm + CfSmem::MISC);
@@ -838,7 +839,7 @@ int fs_tc_causal_prefix(fsharp_ctx* ctx, const void* Q, const void* K, const voi
   FS_TRY(tchost::make_map_out(&tmY, Y, fs_addr(dm->y_stride, H, L, dm->dv), B, H, L, dm->dv));
   FS_CUDA_OK(cudaFuncSetAttribute(tc_causal_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CfSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_CAUSAL);
-  tc_causal_kernel<<<dim3(nseg, BH), TC_THREADS, CfSmem::TOTAL + 1024, ctx->stream>>>(
+  (void)fs_launch_chained(tc_causal_kernel, dim3(nseg, BH), dim3(TC_THREADS), CfSmem::TOTAL + 1024, ctx->stream,
       tmQ, tmK, tmV, tmY, images, crow, partial, shifts, ntot, nprefix, H, dm->pool, L, Lpad, per, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);

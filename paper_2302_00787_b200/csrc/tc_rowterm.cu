@@ -33,6 +33,7 @@ __global__ void __launch_bounds__(RT_THREADS)
 tc_rowterm_kernel(const __grid_constant__ CUtensorMap tmK, const uint8_t* __restrict__ images,
                   const int* __restrict__ img_flags, int side, int H, int pool, int L, int Lpad, int tiles_per_split,
                   float* __restrict__ crow, int* __restrict__ status) {
+  fs_grid_dependency_wait();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   RtMisc* misc = reinterpret_cast<RtMisc*>(sm + RtSmem::MISC);
@@ -175,7 +176,7 @@ int fs_tc_rowterm_side(fsharp_ctx* ctx, const void* X, const fsharp_dims* dm, in
   const int tps = (total + ns - 1) / ns;
   ns = (total + tps - 1) / tps;
   FS_TIME_BEGIN(ctx, FS_K_TC_ROWTERM);
-  tc_rowterm_kernel<<<dim3(ns, B * H), RT_THREADS, RtSmem::TOTAL + 1024, ctx->stream>>>(
+  (void)fs_launch_chained(tc_rowterm_kernel, dim3(ns, B * H), dim3(RT_THREADS), RtSmem::TOTAL + 1024, ctx->stream,
       tmX, images, flags, side, H, dm->pool, L, Lpad, tps, crow, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
