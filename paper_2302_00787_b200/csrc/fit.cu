@@ -915,6 +915,7 @@ struct FitArgs {
 
 template <bool V_IN_SMEM>
 __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(FitArgs a) {
+  fs_grid_dependency_wait();
   extern __shared__ __align__(16) double sm[];
   const int d = a.d, tid = threadIdx.x, g = blockIdx.x;
   const int lda = d + 1;
@@ -1363,8 +1364,8 @@ int fs_run_fit(fsharp_ctx* ctx, const double* stats, int G, int d, int variant, 
   if (a.v_in_smem) FS_CUDA_OK(cudaFuncSetAttribute(fit_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   else FS_CUDA_OK(cudaFuncSetAttribute(fit_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   FS_TIME_BEGIN(ctx, FS_K_FIT);
-  if (a.v_in_smem) fit_kernel<true><<<G, FIT_THREADS, smem, ctx->stream>>>(a);
-  else fit_kernel<false><<<G, FIT_THREADS, smem, ctx->stream>>>(a);
+  if (a.v_in_smem) (void)fs_launch_chained(fit_kernel<true>, dim3(G), dim3(FIT_THREADS), smem, ctx->stream, a);
+  else (void)fs_launch_chained(fit_kernel<false>, dim3(G), dim3(FIT_THREADS), smem, ctx->stream, a);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;

@@ -36,6 +36,7 @@ __global__ void __launch_bounds__(ST_THREADS, 2)
 tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, int H, int Lq, int Lk,
                 int pool, int Bpool, double qk_scale, int tiles_per_split, double* __restrict__ stats,
                 int* __restrict__ status) {
+  fs_grid_dependency_wait();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   StMisc* misc = reinterpret_cast<StMisc*>(sm + StSmem::MISC);
@@ -208,7 +209,7 @@ int fs_tc_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dims
   FS_CUDA_OK(cudaFuncSetAttribute(tc_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)StSmem::TOTAL + 1024));
   const int Bpool = dm->pool == FSHARP_POOL_PER_BH ? 1 : B;
   FS_TIME_BEGIN(ctx, FS_K_TC_STATS);
-  tc_stats_kernel<<<dim3(best, BH, 2), ST_THREADS, StSmem::TOTAL + 1024, ctx->stream>>>(
+  (void)fs_launch_chained(tc_stats_kernel, dim3(best, BH, 2), dim3(ST_THREADS), StSmem::TOTAL + 1024, ctx->stream,
       tmQ, tmK, H, dm->Lq, dm->Lk, dm->pool, Bpool, (double)qk_scale, tps, stats, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
