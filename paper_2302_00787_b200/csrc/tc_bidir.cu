@@ -71,7 +71,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
              const uint8_t* __restrict__ images, const float* __restrict__ crow, int H, int pool, int L, int Lpad,
              int tiles_per_split, int nsplit, float* __restrict__ partial, float* __restrict__ shifts,
-             int* __restrict__ pmax, int* __restrict__ status) {
+             int* __restrict__ status) {
   fs_grid_dependency_wait();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -285,7 +285,6 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       // thread = feature m: its row of the accumulator is column m of the state [80][256]; a store instruction of
       // the warp covers 32 consecutive features of one state row (128 contiguous bytes).  Rows 65..79 are not written.
       float* out = partial + slot * TC_NV * TC_M + hf * 128 + row;
-      float amax = 0.f;
 #pragma unroll
       for (int c = 0; c < 5; c++) {
         uint32_t a[16];
@@ -293,16 +292,9 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         tmem_wait_ld();
 #pragma unroll
         for (int j = 0; j < 16; j++) {
-          if (c * 16 + j <= TC_DV) {
-            amax = fmaxf(amax, fabsf(__uint_as_float(a[j])));
-            out[(size_t)(c * 16 + j) * TC_M] = __uint_as_float(a[j]);
-          }
+          if (c * 16 + j <= TC_DV) out[(size_t)(c * 16 + j) * TC_M] = __uint_as_float(a[j]);
         }
       }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-      // non-negative floats order like their bit patterns
-      if (lane == 0) atomicMax(&pmax[slot * 2 + hf], __float_as_int(amax));
       if (q == 0 && lane == 0) shifts[slot * 2 + hf] = s;
       tcgen05_fence_before();
     };
@@ -396,7 +388,7 @@ tc_kv_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       if (KV_TURNS) mbar_arrive_warp(&misc->turn[hf ^ 1], lane);
       cj = cnext;
     }
-    // write this split's partial phi_h^T [V | 1] (rows 0..64 of the state), its shift and its largest magnitude
+    // write this split's partial phi_h^T [V | 1] (rows 0..64 of the state) and its shift
     if (alive && ntiles > 0 && mbar_wait(&misc->phi_free[hf], (ntiles - 1) & 1, abortp, status, false))
       write_partial((size_t)bh * nsplit + split);
   }
@@ -815,7 +807,7 @@ size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
 int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
                 const int* flags, void* Y, WsAlloc* ws);
 int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
-                   const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax);
+                   const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts);
 int fs_tc_query_side(fsharp_ctx* ctx, const void* Q, const fsharp_dims* dm, const uint8_t* images, const float* partial,
                      const float* shifts, int nsplit, void* Y);
 int fs_tc_key_state_splits(const fsharp_ctx* ctx, const fsharp_dims* dm, int* tiles_per_split);
@@ -846,10 +838,8 @@ int fs_tc_key_state(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_
   const int BH = dm->B * dm->H;
   int tps = 0;
   const int ns = fs_tc_key_state_splits(ctx, dm, &tps);
-  int* pmax = ws->take<int>((size_t)BH * MAX_STATE_SPLIT * 2);
-  FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * MAX_STATE_SPLIT * 2 * sizeof(int), ctx->stream));
   float* crow = ws->take<float>((size_t)BH * ((dm->Lk + TILE - 1) / TILE) * TILE);
-  return fs_tc_key_side(ctx, K, V, dm, images, flags, tps, ns, crow, state, shifts, pmax);
+  return fs_tc_key_side(ctx, K, V, dm, images, flags, tps, ns, crow, state, shifts);
 }
 
 size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
@@ -862,11 +852,11 @@ size_t fs_tc_bidir_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm) {
 }
 
 // Key side: the per-key quadratic term, then the feature / contraction kernel.  crow: [B*H][Lpad] floats,
-// Lpad = ceil(Lk / 128) * 128; partial: [B*H][nsplit][80][256] floats; shifts, pmax: [B*H][nsplit][2], pmax
-// zeroed by the caller.  The quadratic term covers every key; the feature / contraction kernel covers the
+// Lpad = ceil(Lk / 128) * 128; partial: [B*H][nsplit][80][256] floats; shifts: [B*H][nsplit][2].
+// The quadratic term covers every key; the feature / contraction kernel covers the
 // first nsplit * tiles_per_split tiles (the causal path asks for the segments that have a successor only).
 int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
-                   const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax) {
+                   const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts) {
   FS_RANGE("key side");
   const int B = dm->B, H = dm->H, Lk = dm->Lk;
   const int Lpad = (Lk + TILE - 1) / TILE * TILE;
@@ -877,7 +867,7 @@ int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_d
   FS_CUDA_OK(cudaFuncSetAttribute(tc_kv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KvSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_KV);
   (void)fs_launch_chained(tc_kv_kernel, dim3(nsplit, B * H), dim3(TC_THREADS), KvSmem::TOTAL + 1024, ctx->stream,
-      tmK, tmV, images, crow, H, dm->pool, Lk, Lpad, tiles_per_split, nsplit, partial, shifts, pmax, ctx->d_status);
+      tmK, tmV, images, crow, H, dm->pool, Lk, Lpad, tiles_per_split, nsplit, partial, shifts, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;
@@ -893,11 +883,9 @@ int fs_tc_bidir(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, co
   int nsplit = pick_split(BH, ktiles, ctx->sm_count, MAX_KEY_SPLIT, &tps);
   float* partial = ws->take<float>((size_t)BH * MAX_KEY_SPLIT * TC_M * TC_NV);
   float* shifts = ws->take<float>((size_t)BH * MAX_KEY_SPLIT * 2);
-  int* pmax = ws->take<int>((size_t)BH * MAX_KEY_SPLIT * 2);
-  FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * MAX_KEY_SPLIT * 2 * sizeof(int), ctx->stream));
   const int Lpad = ktiles * TILE;
   float* crow = ws->take<float>((size_t)BH * Lpad);
-  FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, tps, nsplit, crow, partial, shifts, pmax));
+  FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, tps, nsplit, crow, partial, shifts));
 
   return fs_tc_query_side(ctx, Q, dm, images, partial, shifts, nsplit, Y);
 }

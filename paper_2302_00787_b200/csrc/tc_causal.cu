@@ -739,7 +739,7 @@ int make_map_out(CUtensorMap* map, void* base, TensorAddr a, int B, int H, int L
 int fs_tc_rowterm(fsharp_ctx* ctx, const void* K, const fsharp_dims* dm, const uint8_t* images, const int* flags, int Lpad,
                   int tiles_per_split, int nsplit, float* crow);
 int fs_tc_key_side(fsharp_ctx* ctx, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
-                   const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts, int* pmax);
+                   const int* flags, int tiles_per_split, int nsplit, float* crow, float* partial, float* shifts);
 int fs_tc_causal_supported(const fsharp_dims* dm, int chunk);
 size_t fs_tc_causal_scratch_bytes(const fsharp_ctx* ctx, const fsharp_dims* dm);
 int fs_tc_causal(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm, const uint8_t* images,
@@ -803,14 +803,12 @@ int fs_tc_causal_prefix(fsharp_ctx* ctx, const void* Q, const void* K, const voi
   const int nch = (L + TILE - 1) / TILE, Lpad = nch * TILE;
   float* partial = ws->take<float>((size_t)BH * CF_MAX_SEG * TC_M * TC_NV);
   float* shifts = ws->take<float>((size_t)BH * CF_MAX_SEG * 2);
-  int* pmax = ws->take<int>((size_t)BH * CF_MAX_SEG * 2);
   float* crow = ws->take<float>((size_t)BH * Lpad);
   int per = 0;
   const int nseg = pick_segments(BH, nch, ctx->sm_count, &per);
   // key side: the per-key quadratic term of every key, and the totals of the segments that have a successor
   if (nseg > 1) {
-    FS_CUDA_OK(cudaMemsetAsync(pmax, 0, (size_t)BH * (nseg - 1) * 2 * sizeof(int), ctx->stream));
-    FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, per, nseg - 1, crow, partial, shifts, pmax));
+    FS_TRY(fs_tc_key_side(ctx, K, V, dm, images, flags, per, nseg - 1, crow, partial, shifts));
   } else {
     FS_TRY(fs_tc_rowterm(ctx, K, dm, images, flags, Lpad, per, 1, crow));
   }
