@@ -236,8 +236,8 @@ class Runner:
 
 # DRAM bytes per launch (read + write) from the ncu captures summarised under profiles/ (same kernels, same
 # workload); an entry is dropped when its kernel changes.
-NCU_TRAFFIC = {("cfg3", "tc_causal_kernel"): 196.3e6,      # 162.2 MB read + 34.0 MB written (Y stays partly in L2)
-               ("cfg3b", "tc_kv_kernel"): 109.3e6, ("cfg3b", "tc_out_kernel"): 69.1e6}
+NCU_TRAFFIC = {("cfg3", "tc_causal_kernel"): 192.3e6,      # 162.2 MB read + 30.1 MB written (Y stays partly in L2)
+               ("cfg3b", "tc_kv_kernel"): 111.5e6, ("cfg3b", "tc_out_kernel"): 69.1e6}
 
 
 def kernel_flops(name, w, work):
