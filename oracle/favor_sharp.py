@@ -346,6 +346,49 @@ def favor_sharp_attention(Q, K, V, Omega, p, causal=False, qk_scale=1.0, rows=No
 
 
 # --------------------------------------------------------------------------
+# Backward pass (Section 5.3 trains Transformers through this attention): the
+# vector-Jacobian product of favor_sharp_attention with the parameters held fixed
+# --------------------------------------------------------------------------
+def favor_sharp_attention_vjp(Q, K, V, dY, Omega, p, causal=False, qk_scale=1.0):
+    """(dQ, dK, dV) = gradient of sum(dY * favor_sharp_attention(Q, K, V, ...)) for one
+    (batch, head), Omega and the parameters p being constants.  The chain rule on the
+    explicit L x L form of Section 2.2, step by step:
+
+      Khat = P S^T (lower triangle when causal), den = Khat 1, Y = Khat V / den
+      dNum = dY / den,  dden_i = -sum_c dY_ic Y_ic / den_i
+      dKhat_ij = dNum_i . V_j + dden_i   (same mask),   dV = Khat^T dNum
+      dP = dKhat S,  dS = dKhat^T P;  through the exponential: dlogP = dP * P, dlogS = dS * S
+      log feature (Section 4): w^T B x + x^T C x + terms without x, so
+      dx_i = sum_m dlog_im B^T w_m + (C + C^T) x_i sum_m dlog_im,  dQ = qk_scale dx.
+    """
+    X = qk_scale * np.asarray(Q, F64)
+    Yk = qk_scale * np.asarray(K, F64)
+    V = np.asarray(V, F64)
+    dY = np.asarray(dY, F64)
+    Om = np.asarray(Omega, F64)
+    P = derf_features(X, Om, p["A"], p["B1"], p["C1"], p["logD"])
+    S = derf_features(Yk, Om, p["A"], p["B2"], p["C2"], p["logD"])
+    Khat = P @ S.T
+    if causal:
+        Khat = np.tril(Khat)
+    den = Khat.sum(axis=1, keepdims=True)
+    Yout = (Khat @ V) / den
+    dNum = dY / den
+    dden = -np.sum(dY * Yout, axis=1, keepdims=True) / den
+    dKhat = dNum @ V.T + dden
+    if causal:
+        dKhat = np.tril(dKhat)
+    dV = Khat.T @ dNum
+    dlogP = (dKhat @ S) * P
+    dlogS = (dKhat.T @ P) * S
+    C1 = np.asarray(p["C1"], F64)
+    C2 = np.asarray(p["C2"], F64)
+    dX = dlogP @ (Om @ np.asarray(p["B1"], F64)) + dlogP.sum(axis=1, keepdims=True) * (X @ (C1 + C1.T))
+    dYk = dlogS @ (Om @ np.asarray(p["B2"], F64)) + dlogS.sum(axis=1, keepdims=True) * (Yk @ (C2 + C2.T))
+    return qk_scale * dX, qk_scale * dYk, dV
+
+
+# --------------------------------------------------------------------------
 # Kernel estimation for pairs (Section 2.1 estimator, Section 5.1 setting)
 # --------------------------------------------------------------------------
 def pair_estimate(X, Y, Omega, p):

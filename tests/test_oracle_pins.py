@@ -461,3 +461,65 @@ def test_sderf_variance_gain_on_heterogeneous_sets():
     g = fs.fit_params(X, Y, "gerf")["objective"]
     s = fs.fit_params(X, Y, "sderf")["objective"]
     assert s < g - 0.5
+
+
+# ------------------------------------------------------------------ backward pass
+def _vjp_case(seed, causal, L=11, d=4, M=8, dv=3):
+    rng = np.random.default_rng(seed)
+    p = random_valid_derf(rng, d)
+    # a C that is not symmetric, so that (C + C^T) is told apart from 2 C
+    p["C1"] = p["C1"] + 0.05 * rng.standard_normal((d, d))
+    p["C2"] = p["C2"] + 0.05 * rng.standard_normal((d, d))
+    Om = rng.standard_normal((M, d))
+    Q = 0.6 * rng.standard_normal((L, d))
+    K = 0.6 * rng.standard_normal((L, d))
+    V = rng.standard_normal((L, dv))
+    dY = rng.standard_normal((L, dv))
+    return Q, K, V, dY, Om, p
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_attention_vjp_matches_central_differences(causal):
+    """The gradient formulas against the numerical derivative of the (pinned) forward function."""
+    Q, K, V, dY, Om, p = _vjp_case(31, causal)
+    qk = 0.8
+    dQ, dK, dV = fs.favor_sharp_attention_vjp(Q, K, V, dY, Om, p, causal=causal, qk_scale=qk)
+
+    def loss(q, k, v):
+        return float(np.sum(dY * fs.favor_sharp_attention(q, k, v, Om, p, causal=causal, qk_scale=qk)))
+
+    h = 1e-5
+    for arr, grad, which in ((Q, dQ, 0), (K, dK, 1), (V, dV, 2)):
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            a_p = arr.copy(); a_p[idx] += h
+            a_m = arr.copy(); a_m[idx] -= h
+            args_p = [Q, K, V]; args_p[which] = a_p
+            args_m = [Q, K, V]; args_m[which] = a_m
+            num[idx] = (loss(*args_p) - loss(*args_m)) / (2 * h)
+        assert np.max(np.abs(num - grad)) <= 2e-7 * max(1.0, np.max(np.abs(grad)))
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_attention_vjp_closed_form_properties(causal):
+    """Y(V + 1 c^T) = Y + 1 c^T, so the column sums of dV equal those of dY; Y does not move when all
+    queries (or all keys) are featurised with a common extra factor, which the x^T C x term of the
+    queries is per row: dQ is the same with C1 replaced by any other matrix."""
+    Q, K, V, dY, Om, p = _vjp_case(32, causal)
+    dQ, dK, dV = fs.favor_sharp_attention_vjp(Q, K, V, dY, Om, p, causal=causal)
+    assert np.allclose(dV.sum(axis=0), dY.sum(axis=0), rtol=1e-10, atol=1e-12)
+    p2 = dict(p); p2["C1"] = np.zeros_like(p["C1"])
+    dQ2, dK2, dV2 = fs.favor_sharp_attention_vjp(Q, K, V, dY, Om, p2, causal=causal)
+    assert np.allclose(dQ, dQ2, rtol=1e-9, atol=1e-12)
+    assert np.allclose(dK, dK2, rtol=1e-9, atol=1e-12) and np.allclose(dV, dV2, rtol=1e-9, atol=1e-12)
+
+
+def test_causal_attention_vjp_sees_no_future():
+    """A cotangent on row i alone: no gradient reaches keys or values after i, nor any other query."""
+    Q, K, V, dY, Om, p = _vjp_case(33, True)
+    i = 6
+    dY1 = np.zeros_like(dY); dY1[i] = dY[i]
+    dQ, dK, dV = fs.favor_sharp_attention_vjp(Q, K, V, dY1, Om, p, causal=True)
+    assert np.all(dK[i + 1:] == 0) and np.all(dV[i + 1:] == 0)
+    assert np.all(np.delete(dQ, i, axis=0) == 0)
+    assert np.any(dK[: i + 1] != 0) and np.any(dV[: i + 1] != 0) and np.any(dQ[i] != 0)
