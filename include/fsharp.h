@@ -13,6 +13,7 @@
  *   fsharp_fit_params     closed-form optimal A, B, C, D per parameter group
  *   fsharp_featurize      P or S for given parameters
  *   fsharp_attend         Y, bidirectional or causal (lower-triangular mask)
+ *   fsharp_attend_backward  dQ, dK, dV for a cotangent dY of that Y
  *   fsharp_pair_estimate  Khat(x, y) for pairs, with Theorem 4.1's variance
  *   fsharp_kernel_apply   the unnormalised operator Khat^(alpha) C (softmax and Gaussian kernels)
  *   fsharp_attend_key_state, fsharp_attend_with_state   the same Y with the keys of a sequence spread over
@@ -202,6 +203,22 @@ int fsharp_featurize_static(void* stream, const void* X, const float* Omega, con
 int fsharp_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V,
                   const float* Omega, const double* params, const fsharp_dims* dims,
                   int dtype, int causal, int chunk, float qk_scale, void* Y);
+
+/* Backward pass of fsharp_attend (Section 5.3 trains Transformers through the attention of Section 2.2): with
+ * Y = fsharp_attend(Q, K, V) and a cotangent dY [B,H,Lq,dv] (y_stride), writes the gradients of sum(dY * Y):
+ * dQ [B,H,Lq,d] (q_stride), dK [B,H,Lk,d] (k_stride), dV [B,H,Lk,dv] (v_stride), all of type `dtype`.  Omega and the
+ * fitted parameters are constants of the differentiation (no gradient flows through the statistics or the fit).
+ * With [num | den]_i = P_i KV_i, G_i = [dY_i / den_i | -(dY_i . Y_i) / den_i] and R_j the sum of P_i G_i^T over the
+ * queries i that see key j:  dlogP_i = (G_i KV_i^T) * P_i,  dlogS_j = ([V_j | 1] R_j^T) * S_j,  dV_j = S_j R_j[:, :dv],
+ * and, the exponent of Section 4's feature being w^T B x + x^T C x + terms without x,
+ * dx = dlog (Omega B) + rowsum(dlog) (C + C^T) x, dQ = qk_scale dx (likewise dK).  causal, chunk, qk_scale and the
+ * argument checks are those of fsharp_attend; Q, K, V are read again (nothing is kept from the forward call).
+ * fp32 kernels for every shape and both dtypes (bf16 tensors are widened on load, gradients rounded on store).
+ * All pointers are device pointers, 16-byte aligned; asynchronous on the context's stream.  A normaliser that is
+ * zero or not finite, or a gradient that is not finite, latches FSHARP_E_NONFINITE in the status word. */
+int fsharp_attend_backward(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const void* dY,
+                           const float* Omega, const double* params, const fsharp_dims* dims, int dtype, int causal,
+                           int chunk, float qk_scale, void* dQ, void* dK, void* dV);
 
 /* Sequence-parallel attention.  In Section 2.2's formula the numerator phi(Q) (phi(K)^T V) and the normaliser
  * phi(Q) (phi(K)^T 1) are sums over keys, so the key-side sums S^T [V | 1] of disjoint key ranges add: the keys of

@@ -25,7 +25,7 @@ EXPORTS = [
     "fsharp_params_doubles", "fsharp_stats", "fsharp_fit_params", "fsharp_featurize", "fsharp_attend",
     "fsharp_forward_host", "fsharp_pair_estimate", "fsharp_set_timing", "fsharp_read_timing",
     "fsharp_kernel_name", "fsharp_static_scratch_bytes", "fsharp_featurize_static", "fsharp_kernel_apply",
-    "fsharp_key_state_splits", "fsharp_attend_key_state", "fsharp_attend_with_state",
+    "fsharp_key_state_splits", "fsharp_attend_key_state", "fsharp_attend_with_state", "fsharp_attend_backward",
     "fsharp_selftest_bounded_wait",
 ]
 
@@ -75,6 +75,7 @@ def load_library() -> C.CDLL:
         "fsharp_featurize": (i32, [vp, vp, vp, vp, i32, dims_p, i32, f32, i32, vp, vp]),
         "fsharp_attend": (i32, [vp, vp, vp, vp, vp, vp, dims_p, i32, i32, i32, f32, vp]),
         "fsharp_kernel_apply": (i32, [vp, vp, vp, vp, vp, vp, f64, dims_p, i32, f32, vp]),
+        "fsharp_attend_backward": (i32, [vp, vp, vp, vp, vp, vp, vp, dims_p, i32, i32, i32, f32, vp, vp, vp]),
         "fsharp_key_state_splits": (i32, [vp, dims_p]),
         "fsharp_attend_key_state": (i32, [vp, vp, vp, vp, vp, dims_p, i32, f32, vp, vp]),
         "fsharp_attend_with_state": (i32, [vp, vp, vp, vp, vp, vp, dims_p, i32, i32, f32, vp, vp, i32, vp]),
@@ -247,6 +248,21 @@ class Context:
                                       params.data_ptr(), C.byref(dm), _dtype_code(Q), int(bool(causal)), chunk,
                                       qk_scale, out.data_ptr()), "fsharp_attend")
         return out
+
+    def fsharp_attend_backward(self, Q, K, V, dY, Omega, params, causal=False, chunk=0, pool=POOL_PER_BH,
+                               qk_scale=1.0):
+        """(dQ, dK, dV) for the cotangent dY of fsharp_attend's Y; each gradient has its tensor's shape and strides."""
+        B, H, Lq, d = Q.shape
+        Lk, dv = K.shape[2], V.shape[3]
+        M = Omega.shape[-2]
+        ohs = Omega.stride(0) if Omega.dim() == 3 else 0
+        dQ, dK, dV = (torch.empty_strided(t.shape, t.stride(), dtype=t.dtype, device=t.device) for t in (Q, K, V))
+        dm = make_dims(B, H, Lq, Lk, d, dv, M, pool, q=Q, k=K, v=V, y=dY, omega_head_stride=ohs)
+        _check(self.lib.fsharp_attend_backward(self._h, Q.data_ptr(), K.data_ptr(), V.data_ptr(), dY.data_ptr(),
+                                               Omega.data_ptr(), params.data_ptr(), C.byref(dm), _dtype_code(Q),
+                                               int(bool(causal)), chunk, qk_scale, dQ.data_ptr(), dK.data_ptr(),
+                                               dV.data_ptr()), "fsharp_attend_backward")
+        return dQ, dK, dV
 
     def fsharp_attend_key_state(self, K, V, Omega, params, pool=POOL_PER_BH, qk_scale=1.0):
         """Key-side sums of this call's keys: (state [B*H, ns, 80, 256] fp32, shifts [B*H, ns, 2] fp32)."""

@@ -172,6 +172,40 @@ int fsharp_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, 
   return fs_simt_attend(ctx, Q, K, V, dims, dtype, causal, chunk, qk_scale, prep, Y, &ws);
 }
 
+int fsharp_attend_backward(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const void* dY,
+                           const float* Omega, const double* params, const fsharp_dims* dims, int dtype, int causal,
+                           int chunk, float qk_scale, void* dQ, void* dK, void* dV) {
+  FS_RANGE("fsharp_attend_backward");
+  if (!ctx || !Omega || !params) return FSHARP_E_BADARG;
+  FS_TRY(check_dims(dims, true));
+  if (!dtype_ok(dtype)) return FSHARP_E_DTYPE;
+  if (causal) {
+    if (dims->Lq != dims->Lk) return FSHARP_E_SHAPE;
+    if (chunk != 64 && chunk != 128 && chunk != 256) return FSHARP_E_SHAPE;
+    if (dims->Lq % chunk != 0) return FSHARP_E_SHAPE;
+  }
+  if (dims->B * dims->H == 0 || (dims->Lq == 0 && dims->Lk == 0)) return FSHARP_OK;
+  if (dims->Lk == 0 || dims->Lq == 0) return FSHARP_E_SHAPE;   // no key: no normaliser; no query: nothing to differentiate
+  FS_TRY(check_ptr(Q, dtype, dims->q_stride));
+  FS_TRY(check_ptr(K, dtype, dims->k_stride));
+  FS_TRY(check_ptr(V, dtype, dims->v_stride));
+  FS_TRY(check_ptr(dY, dtype, dims->y_stride));
+  FS_TRY(check_ptr(dQ, dtype, dims->q_stride));
+  FS_TRY(check_ptr(dK, dtype, dims->k_stride));
+  FS_TRY(check_ptr(dV, dtype, dims->v_stride));
+  // (batch, head, chunk) is a grid z coordinate
+  if (causal && (int64_t)dims->B * dims->H * (dims->Lq / chunk) > 65535) return FSHARP_E_SHAPE;
+  FS_CUDA_OK(cudaSetDevice(ctx->device));
+  const int G = fs_groups(dims);
+  const size_t prep_f = (size_t)G * 2 * PrepLayout{dims->d, dims->M}.total();
+  FS_TRY(fs_ws_reserve(ctx, ws_round(prep_f * 4) + fs_backward_scratch_bytes(dims, causal, chunk)));
+  WsAlloc ws{ctx->ws, 0};
+  float* prep = ws.take<float>(prep_f);
+  FS_TRY(fs_run_prep(ctx, Omega, dims->omega_head_stride, params, (int64_t)ParamsLayout{dims->d}.total(), G,
+                     dims->H, dims->pool, dims->d, dims->M, prep));
+  return fs_backward(ctx, Q, K, V, dY, dims, dtype, causal, chunk, qk_scale, prep, dQ, dK, dV, &ws);
+}
+
 int fsharp_key_state_splits(fsharp_ctx* ctx, const fsharp_dims* dims) {
   if (!ctx) return FSHARP_E_BADARG;
   FS_TRY(check_dims(dims, true));

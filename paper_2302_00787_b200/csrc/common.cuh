@@ -208,6 +208,10 @@ int fs_simt_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V,
 size_t fs_simt_attend_scratch_bytes(const fsharp_dims* dm, int causal, int chunk);
 int fs_simt_kernel_apply(fsharp_ctx* ctx, const void* X, const void* Yset, const void* Cmat, const fsharp_dims* dm,
                          int dtype, float qk_scale, const float* prep, void* out, WsAlloc* ws);
+size_t fs_backward_scratch_bytes(const fsharp_dims* dm, int causal, int chunk);
+int fs_backward(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const void* dY, const fsharp_dims* dm,
+                int dtype, int causal, int chunk, float qk_scale, const float* prep, void* dQ, void* dK, void* dV,
+                WsAlloc* ws);
 int fs_shift_c(fsharp_ctx* ctx, const double* params, double* out, int G, int d, double alpha);
 int fs_run_pairs(fsharp_ctx* ctx, const float* X, const float* Y, const float* Omega, const double* params,
                  int64_t npairs, int d, int M, int R, float* est, double* var_cf, double* pooled, WsAlloc* ws);
