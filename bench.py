@@ -234,6 +234,52 @@ class Runner:
         return hQ, hK, hV, hOm, hY
 
 
+def backward_flops(w):
+    """Multiply-adds x 2 of the backward pass as the kernels issue them (Section 2.2 differentiated; the header of
+    csrc/backward.cu lists the products): features of both sides, the two key- / query-side sums, numerators and
+    normalisers, the gradients of the features, dV, and the two products back to Q and K; causal adds the masked
+    blocks of each chunk (half of a full block each)."""
+    L, d, dv, M, N = w.L, w.d, w.dv, w.M, w.dv + 1
+    per = 2 * (2 * L * M * d) + 2 * (2 * L * M * N) + 3 * (2 * L * M * N) + 2 * L * M * dv + 2 * (2 * L * M * d + 2 * L * d * d)
+    if w.causal:
+        C = w.chunk
+        per += L * C * (M + N) + L * C * (N + 2 * M + dv)
+    return float(per * w.B * w.H)
+
+
+def backward_leg(runners, sm_count, sm_mhz):
+    """fsharp_attend_backward on the bench workloads: CUDA-event time of the call (its kernels run on the fp32 cores),
+    against the fp32 multiply-add peak: SMs x 128 lanes x 2 flops x the SM clock seen under load."""
+    import torch
+    res = {}
+    peak = sm_count * 128 * 2 * sm_mhz * 1e6 / 1e12
+    for r in runners:
+        w = r.w
+        dQ, dK, dV = r.sets[0]
+        g = torch.Generator(device=dQ.device).manual_seed(w.seed + 99)
+        dY = torch.randn(w.B, w.H, w.L, w.dv, generator=g, device=dQ.device, dtype=torch.float32).to(r.td)
+        call = lambda: r.ctx.fsharp_attend_backward(dQ, dK, dV, dY, r.dOm, r.pr, causal=w.causal, chunk=w.chunk)
+        for _ in range(2):
+            call()
+        torch.cuda.synchronize()
+        n = 3
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            grads = call()
+        e1.record()
+        torch.cuda.synchronize()
+        assert r.ctx.status() == 0
+        ms = e0.elapsed_time(e1) / n
+        fl = backward_flops(w)
+        res[w.name] = {"ms": ms, "tokens_per_s": w.B * w.L / (ms * 1e-3), "gflop": fl / 1e9,
+                       "roofline": {"bound": "alu", "achieved": fl / (ms * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
+                                    "frac": fl / (ms * 1e-3) / 1e12 / peak},
+                       "finite": bool(all(torch.isfinite(t.float()).all().item() for t in grads))}
+        del grads, dY
+    return res
+
+
 # DRAM bytes per launch (read + write) from the ncu captures summarised under profiles/ (same kernels, same
 # workload); an entry is dropped when its kernel changes.
 NCU_TRAFFIC = {("cfg3", "tc_causal_kernel"): 192.3e6,      # 162.2 MB read + 30.1 MB written (Y stays partly in L2)
@@ -342,6 +388,8 @@ def main():
     ap.add_argument("--cpu-baseline-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--backward", action="store_true",
+                    help="also time fsharp_attend_backward on the workloads (fp32 kernels; a few GB of scratch)")
     ap.add_argument("--fit-per-workload", action="store_true",
                     help="one fit launch per workload instead of one launch over the groups of all workloads of a step")
     ap.add_argument("--kernel-impl", default="auto", choices=["auto", "simt", "tensor"])
@@ -575,6 +623,9 @@ def main():
                       "ms": fk[0] / fk[1] if fk else None,
                       "note": "one launch fits the groups of all workloads of the step (one block per group); every "
                               "workload's ms_per_step_alone includes a fit launch of its own"}
+    if args.backward and world == 1:
+        clk = out["clocks"].get("sm_mhz") or out["clocks"].get("sm_max_mhz") or 1965
+        out["backward"] = backward_leg(runners, torch.cuda.get_device_properties(dev).multi_processor_count, float(clk))
     if e2e is not None:
         e2e_ms, n_e2e, h2d, d2h = e2e
         out["e2e"] = {"value": tokens_per_step * n_e2e / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,

@@ -99,3 +99,30 @@ def test_long_sequence_tensor_core_path_sampled_parity(ctx, causal):
                                                                    causal=causal)
     assert ctx.status() == 0
     check_sampled(w, host_in, pr, Ys, [(0, 1)], 12, 9)
+
+
+@pytest.mark.parametrize("name,unit", [("cfg3b", (1, 4)), ("cfg3", (2, 7))])
+def test_full_size_backward_parity(ctx, name, unit):
+    """fsharp_attend_backward on the whole benchmark workload; the checker differentiates one (batch, head) unit
+    (all of its 8192 rows, through the explicit L x L form) and every row of dQ, dK, dV of that unit is compared."""
+    w = wl.WORKLOADS[name]
+    Q, K, V = wl.make_qkv(w)
+    Om = wl.make_omega(w)
+    dY = wl.bf16_round(np.random.default_rng(17).standard_normal((w.B, w.H, w.L, w.dv), dtype=np.float32))
+    dQ, dK, dV, ddY = (torch.from_numpy(a).cuda().to(torch.bfloat16) for a in (Q, K, V, dY))
+    dOm = torch.from_numpy(Om).cuda()
+    st = ctx.fsharp_stats(dQ, dK)
+    pr = ctx.fsharp_fit_params(st, w.d, w.variant)
+    grads = ctx.fsharp_attend_backward(dQ, dK, dV, ddY, dOm, pr, causal=w.causal, chunk=w.chunk)
+    assert ctx.status() == 0
+    assert all(torch.isfinite(g.float()).all() for g in grads)
+    b, h = unit
+    p = fb.unpack_params(pr.cpu().numpy()[b * w.H + h], w.d)
+    ref = fs.favor_sharp_attention_vjp(Q[b, h], K[b, h], V[b, h], dY[b, h], Om, p, causal=w.causal)
+    for name_, got, want in zip(("dQ", "dK", "dV"), grads, ref):
+        err = np.abs(host(got[b, h]) - want).max() / np.abs(want).max()
+        assert err < TOL["bf16"], (name_, err)
+    # the column sums of dV equal those of dY (Y moves with V by the same constant), unit by unit
+    s_dv = grads[2].float().sum(dim=2)
+    s_dy = ddY.float().sum(dim=2)
+    assert (s_dv - s_dy).abs().max().item() < 2e-2 * s_dy.abs().max().item()
