@@ -84,7 +84,7 @@ tc_rowterm_kernel(const __grid_constant__ CUtensorMap tmK, const uint8_t* __rest
         mbar_wait(&misc->full[it % RT_STAGES], (it / RT_STAGES) & 1, abortp, status, false);
     }
   } else if (warp == RT_WARP_MMA) {
-    // The whole warp walks the schedule (waits and descriptor arithmetic stay warp-uniform); one elected lane issues.
+    // The whole warp walks the schedule (waits and descriptor arithmetic stay warp-uniform); lane 0 issues.
     constexpr uint32_t ID_T = idesc_bf16(128, TC_D, 0, 0);
     const uint64_t dX0 = smem_desc(smem_u32(sm + RtSmem::X0), 16, 1024, SWZ_128B);
     const uint64_t dChi = smem_desc(smem_u32(sm + RtSmem::CHI), 16, 1024, SWZ_128B);
@@ -99,7 +99,8 @@ tc_rowterm_kernel(const __grid_constant__ CUtensorMap tmK, const uint8_t* __rest
       tcgen05_fence_after();
       opaque(xl0); opaque(chl); opaque(cll);
       const uint32_t xl = xl0 + st * (TILE_BYTES / 16);
-      if (elect_one()) {
+      // (a fixed lane, not an elected one: with two of these blocks on an SM the elected form gave wrong products now and then)
+      if (lane == 0) {
 #pragma unroll
         for (int k = 0; k < TC_D / 16; k++) mma_bf16_lh(tmem + buf * TC_D, xl + 2 * k, xh, chl + 2 * k, ch, ID_T, k > 0 ? 1u : 0u);
         if (clo) {

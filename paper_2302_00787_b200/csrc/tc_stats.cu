@@ -86,7 +86,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         mbar_wait(&misc->full[it % ST_STAGES], (it / ST_STAGES) & 1, abortp, status, false);
     }
   } else if (warp == ST_WARP_MMA) {
-    // The whole warp walks the schedule (waits and descriptor arithmetic stay warp-uniform); one elected lane issues.
+    // The whole warp walks the schedule (waits and descriptor arithmetic stay warp-uniform); lane 0 issues.
     // An MMA issued by a single lane of a diverged warp costs its thread two to three times as long.
     constexpr uint32_t ID = idesc_bf16(128, TC_D, 1, 1);      // both operands MN-major (feature index contiguous)
     const uint32_t sX0 = smem_u32(sm + StSmem::X0), sOnes = smem_u32(sm + StSmem::ONES);
@@ -103,7 +103,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       uint32_t al = (uint32_t)dA, bl = (uint32_t)dB;
       const uint32_t ah = (uint32_t)(dA >> 32), bh = (uint32_t)(dB >> 32);
       opaque(al); opaque(bl);
-      if (elect_one()) {
+      // (a fixed lane, not an elected one: with two of these blocks on an SM the elected form gave wrong products now and then)
+      if (lane == 0) {
 #pragma unroll
         for (int k = 0; k < TILE / 16; k++)
           mma_bf16_lh(tmem + buf * TC_D, al + k * 128, ah, bl + k * 128, bh, ID, (k > 0 || sub > 0) ? 1u : 0u);
