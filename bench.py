@@ -282,8 +282,8 @@ def backward_leg(runners, sm_count, sm_mhz):
 
 # DRAM bytes per launch (read + write) from the ncu captures summarised under profiles/ (same kernels, same
 # workload); an entry is dropped when its kernel changes.
-NCU_TRAFFIC = {("cfg3", "tc_causal_kernel"): 192.3e6,      # 162.2 MB read + 30.1 MB written (Y stays partly in L2)
-               ("cfg3b", "tc_kv_kernel"): 111.5e6, ("cfg3b", "tc_out_kernel"): 69.1e6}
+NCU_TRAFFIC = {("cfg3", "tc_causal_kernel"): 194.3e6,      # 162.3 MB read + 32.1 MB written (Y stays partly in L2)
+               ("cfg3b", "tc_kv_kernel"): 108.4e6, ("cfg3b", "tc_out_kernel"): 70.5e6}
 
 
 def kernel_flops(name, w, work):
