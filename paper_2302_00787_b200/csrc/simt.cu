@@ -330,11 +330,16 @@ int featurize_t(fsharp_ctx* ctx, const void* X, TensorAddr ax, int B, int H, int
     FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
   }
-  FS_TIME_BEGIN(ctx, FS_K_LOGITS);
-  logits_kernel<T><<<dim3((L + TM - 1) / TM, (M + TN - 1) / TN, BH), NTH, 0, ctx->stream>>>(
-      (const T*)X, ax, H, L, d, M, pool, side, prep, qk_scale, rowc, phi);
-  FS_TIME_END(ctx);
-  FS_LAUNCH_CHECK(ctx);
+  // bf16 tokens with d = 128 (no fused attention kernel takes them): the exponents' product on the tensor cores
+  if (ctx->impl != FSHARP_IMPL_SIMT && fs_tc_logits128_supported(X, sizeof(T) == 2 ? FSHARP_BF16 : FSHARP_F32, ax, L, d, M)) {
+    FS_TRY(fs_tc_logits128(ctx, X, ax, B, H, L, M, pool, prep, side, qk_scale, rowc, phi));
+  } else {
+    FS_TIME_BEGIN(ctx, FS_K_LOGITS);
+    logits_kernel<T><<<dim3((L + TM - 1) / TM, (M + TN - 1) / TN, BH), NTH, 0, ctx->stream>>>(
+        (const T*)X, ax, H, L, d, M, pool, side, prep, qk_scale, rowc, phi);
+    FS_TIME_END(ctx);
+    FS_LAUNCH_CHECK(ctx);
+  }
   {
     int gx = (L + 7) / 8;
     if (gx > 4 * ctx->sm_count) gx = 4 * ctx->sm_count;

@@ -245,6 +245,37 @@ def test_featurize_matches_definition(ctx, w, stab, impl):
         ctx.set_impl(fb.IMPL_AUTO)
 
 
+def test_exponents_tensor_core_kernel_d128(ctx):
+    """bf16 tokens with d = 128 take the tensor-core kernel for the exponents' product (W as a bf16 value and its
+    remainder): a ragged tail, three feature blocks, [B, L, H, d] storage, parameters pooled per head, a query / key
+    scale; element by element against the definition, and against the fp32 kernels."""
+    w = W["cfg5"].scaled(B=2, H=3, L=300, M=384, outlier_frac=0.05)
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    s = 0.9
+    st = ctx.fsharp_stats(dQ, dK, pool=fb.POOL_PER_HEAD, qk_scale=s)
+    pr = ctx.fsharp_fit_params(st, w.d, "aderf")
+    prh = pr.cpu().numpy()
+    tr = lambda t: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    for side, X, dX in ((1, Q, tr(dQ)), (2, K, tr(dK))):
+        phi, ls = ctx.fsharp_featurize(dX, dOm, pr, side, pool=fb.POOL_PER_HEAD, qk_scale=s, stab=fb.STAB_ROW)
+        ctx.set_impl(fb.IMPL_SIMT)
+        try:
+            phi32, ls32 = ctx.fsharp_featurize(dX, dOm, pr, side, pool=fb.POOL_PER_HEAD, qk_scale=s, stab=fb.STAB_ROW)
+        finally:
+            ctx.set_impl(fb.IMPL_AUTO)
+        assert ctx.status() == 0
+        assert (ls - ls32).abs().max().item() < 2e-4 and (phi - phi32).abs().max().item() < 2e-4
+        phi, ls = host(phi), host(ls)
+        for b in range(w.B):
+            for h in range(w.H):
+                p = fb.unpack_params(prh[h], w.d)
+                ref = fs.derf_log_features(s * X[b, h], Om, p["A"], p[f"B{side}"], p[f"C{side}"], p["logD"])
+                expect = np.exp(ref - ls[b, h][:, None])
+                big = expect > 1e-30
+                assert np.max(np.abs(phi[b, h][big] / expect[big] - 1)) < 2e-4
+                assert np.max(np.abs(ls[b, h] - ref.max(axis=1))) < 2e-4 * max(1.0, np.abs(ref).max())
+
+
 # ------------------------------------------------------------------ attend
 @pytest.mark.parametrize("w", small_cases(), ids=lambda w: f"{w.name}-L{w.L}-{w.variant}")
 @pytest.mark.parametrize("impl", [fb.IMPL_SIMT, fb.IMPL_AUTO])
