@@ -7,6 +7,9 @@
 // are exact in fp32; the fp32 sums of ST_FOLD tiles at a time are folded into fp64 registers (the fold, 64
 // conversions and additions per thread, is what a tile's arrival rate from HBM has to cover), and the
 // blocks of one group are combined with fp64 atomics.  The kernel is bound by the HBM read of Q and K.
+// d = 128 (WIDE): the Gram matrix is four 64 x 64 blocks G_ab = X_a^T X_b over the column halves a, b of the tokens; a
+// block of the grid computes one of them from the two 64-column panels of a token tile, D = [X_a | E]^T X_b (row 64:
+// the column sums of X_b, kept when a = b).
 #include "common.cuh"
 #include "tc_common.cuh"
 #include "tc_layout.cuh"
@@ -22,9 +25,13 @@ constexpr int ST_EPI_WARPS = 3;              // rows 0..95 of D; only 0..64 carr
 constexpr int ST_WARP_TMA = 3, ST_WARP_MMA = 4, ST_THREADS = 160;
 constexpr uint32_t ST_TMEM_COLS = 128;       // two accumulators of 64 columns
 
-struct StSmem {
-  static constexpr uint32_t X0 = 0, ONES = ST_STAGES * TILE_BYTES, MISC = ONES + TILE_BYTES, TOTAL = MISC + 256;
+template <bool WIDE>
+struct StSmemT {
+  static constexpr uint32_t STAGE = (WIDE ? 2u : 1u) * TILE_BYTES;     // WIDE: panel a, then panel b
+  static constexpr int NST = WIDE ? 2 : ST_STAGES;                    // (two blocks of either kind fit an SM)
+  static constexpr uint32_t X0 = 0, ONES = NST * STAGE, MISC = ONES + TILE_BYTES, TOTAL = MISC + 256;
 };
+using StSmem = StSmemT<false>;
 struct StMisc {
   uint64_t full[ST_STAGES], empty[ST_STAGES], acc_full[2], acc_free[2];
   uint32_t tmem_base;
@@ -32,16 +39,22 @@ struct StMisc {
 };
 static_assert(sizeof(StMisc) <= 256, "misc block");
 
+template <bool WIDE>
 __global__ void __launch_bounds__(ST_THREADS, 2)
 tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, int H, int Lq, int Lk,
                 int pool, int Bpool, double qk_scale, int tiles_per_split, double* __restrict__ stats,
                 int* __restrict__ status) {
+  using StSmem = StSmemT<WIDE>;
+  constexpr int DD = WIDE ? 2 * TC_D : TC_D;          // head dimension
+  constexpr int NST = StSmem::NST;
   fs_grid_dependency_wait();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   StMisc* misc = reinterpret_cast<StMisc*>(sm + StSmem::MISC);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int side = blockIdx.z, bh = blockIdx.y, b = bh / H, h = bh % H;
+  // WIDE: blockIdx.z = 4 side + 2 a + b, the column halves of the A and the B operand
+  const int side = WIDE ? blockIdx.z >> 2 : blockIdx.z, ha = WIDE ? (blockIdx.z >> 1) & 1 : 0, hb = WIDE ? blockIdx.z & 1 : 0;
+  const int bh = blockIdx.y, b = bh / H, h = bh % H;
   const int L = side ? Lk : Lq;
   const CUtensorMap* tm = side ? &tmK : &tmQ;
   const int total_tiles = (L + TILE - 1) / TILE;
@@ -51,7 +64,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   volatile int* abortp = &misc->abort_flag;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < ST_STAGES; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], 1); }
+    for (int i = 0; i < NST; i++) { mbar_init(&misc->full[i], 1); mbar_init(&misc->empty[i], 1); }
     for (int i = 0; i < 2; i++) { mbar_init(&misc->acc_full[i], 1); mbar_init(&misc->acc_free[i], ST_EPI_WARPS); }
     misc->abort_flag = 0;
     fence_barrier_init();
@@ -75,15 +88,16 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       prefetch_tmap(tm);
       int issued = 0;
       for (int it = 0; it < ntiles; it++) {
-        const int st = it % ST_STAGES;
-        if (!mbar_wait(&misc->empty[st], ((it / ST_STAGES) & 1) ^ 1, abortp, status)) break;
-        mbar_expect_tx(&misc->full[st], TILE_BYTES);
-        tma_load_4d(sm + StSmem::X0 + st * TILE_BYTES, tm, &misc->full[st], 0, (tile0 + it) * TILE, h, b);
+        const int st = it % NST;
+        if (!mbar_wait(&misc->empty[st], ((it / NST) & 1) ^ 1, abortp, status)) break;
+        mbar_expect_tx(&misc->full[st], StSmem::STAGE);
+        tma_load_4d(sm + StSmem::X0 + st * StSmem::STAGE, tm, &misc->full[st], 64 * ha, (tile0 + it) * TILE, h, b);
+        if (WIDE) tma_load_4d(sm + StSmem::X0 + st * StSmem::STAGE + TILE_BYTES, tm, &misc->full[st], 64 * hb, (tile0 + it) * TILE, h, b);
         issued = it + 1;
       }
       // no copy of this block may still be in flight when it exits
-      for (int it = max(0, issued - ST_STAGES); it < issued; it++)
-        mbar_wait(&misc->full[it % ST_STAGES], (it / ST_STAGES) & 1, abortp, status, false);
+      for (int it = max(0, issued - NST); it < issued; it++)
+        mbar_wait(&misc->full[it % NST], (it / NST) & 1, abortp, status, false);
     }
   } else if (warp == ST_WARP_MMA) {
     // The whole warp walks the schedule (waits and descriptor arithmetic stay warp-uniform); lane 0 issues.
@@ -91,15 +105,15 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     constexpr uint32_t ID = idesc_bf16(128, TC_D, 1, 1);      // both operands MN-major (feature index contiguous)
     const uint32_t sX0 = smem_u32(sm + StSmem::X0), sOnes = smem_u32(sm + StSmem::ONES);
     for (int it = 0; it < ntiles; it++) {
-      const int st = it % ST_STAGES, grp = it / ST_FOLD, buf = grp & 1, sub = it % ST_FOLD;
-      if (!__all_sync(0xffffffffu, mbar_wait(&misc->full[st], (it / ST_STAGES) & 1, abortp, status))) break;
+      const int st = it % NST, grp = it / ST_FOLD, buf = grp & 1, sub = it % ST_FOLD;
+      if (!__all_sync(0xffffffffu, mbar_wait(&misc->full[st], (it / NST) & 1, abortp, status))) break;
       if (sub == 0 && !__all_sync(0xffffffffu, mbar_wait(&misc->acc_free[buf], ((grp >> 1) & 1) ^ 1, abortp, status))) break;
       tcgen05_fence_after();
-      const uint32_t sX = sX0 + st * TILE_BYTES;
+      const uint32_t sX = sX0 + st * StSmem::STAGE, sXb = WIDE ? sX + TILE_BYTES : sX;
       // A = [X | E]: block 0 the tile, block 1 the constant tile (leading offset = their distance); a step's
       // descriptors are the tile's plus a constant in the low word (start address / 16)
       const uint64_t dA = smem_desc(sX, sOnes - sX, 1024, SWZ_128B);
-      const uint64_t dB = smem_desc(sX, TILE_BYTES, 1024, SWZ_128B);
+      const uint64_t dB = smem_desc(sXb, TILE_BYTES, 1024, SWZ_128B);
       uint32_t al = (uint32_t)dA, bl = (uint32_t)dB;
       const uint32_t ah = (uint32_t)(dA >> 32), bh = (uint32_t)(dB >> 32);
       opaque(al); opaque(bl);
@@ -141,20 +155,21 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (alive && row <= TC_D) {
       const int g = pool == FSHARP_POOL_PER_BH ? bh : h;
       const double inv = 1.0 / ((double)L * (double)Bpool);
-      StatsLayout sl{TC_D};
+      StatsLayout sl{DD};
       double* out = stats + (size_t)g * sl.total();
       bool bad = false;
       if (row < TC_D) {
         // the Gram matrix is symmetric: row `row` is stored as column `row`, so a warp's atomics coalesce
-        double* Mo = out + sl.M(side + 1);
+        // (entry (64 a + row, 64 b + j) of the matrix goes to row 64 b + j, column 64 a + row)
+        double* Mo = out + sl.M(side + 1) + (size_t)(TC_D * hb) * DD + TC_D * ha;
         const double f = inv * qk_scale * qk_scale;
 #pragma unroll
         for (int j = 0; j < TC_D; j++) {
           if (!isfinite(acc[j])) bad = true;
-          atomicAdd(&Mo[(size_t)j * TC_D + row], acc[j] * f);
+          atomicAdd(&Mo[(size_t)j * DD + row], acc[j] * f);
         }
-      } else {
-        double* mu = out + sl.mu(side + 4);
+      } else if (ha == hb) {
+        double* mu = out + sl.mu(side + 4) + TC_D * hb;
         const double f = inv * qk_scale;
 #pragma unroll
         for (int j = 0; j < TC_D; j++) {
@@ -184,7 +199,7 @@ int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int
 }
 
 int fs_tc_stats_supported(const void* Q, const void* K, const fsharp_dims* dm, int dtype) {
-  if (dtype != FSHARP_BF16 || dm->d != TC_D || dm->Lq <= 0 || dm->Lk <= 0) return 0;
+  if (dtype != FSHARP_BF16 || (dm->d != TC_D && dm->d != 2 * TC_D) || dm->Lq <= 0 || dm->Lk <= 0) return 0;
   return aligned16(Q, fs_addr(dm->q_stride, dm->H, dm->Lq, dm->d)) && aligned16(K, fs_addr(dm->k_stride, dm->H, dm->Lk, dm->d));
 }
 
@@ -193,13 +208,14 @@ int fs_tc_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dims
   const int B = dm->B, H = dm->H, BH = B * H;
   const int Lmax = dm->Lq > dm->Lk ? dm->Lq : dm->Lk;
   const int tiles = (Lmax + TILE - 1) / TILE;
+  const bool wide = dm->d == 2 * TC_D;
   // two blocks per SM (each block has one MMA-issuing thread, and issuing is what bounds a block): the split of
   // the token range with the fewest (waves x tiles per block)
   int best = 1, best_cost = 0x7fffffff, tps = tiles;
   for (int ns = 1; ns <= tiles; ns++) {
     const int t = (tiles + ns - 1) / ns;
     if ((tiles + t - 1) / t != ns) continue;
-    const long long blocks = 2LL * BH * ns;
+    const long long blocks = (wide ? 8LL : 2LL) * BH * ns;
     const int waves = (int)((blocks + 2 * ctx->sm_count - 1) / (2 * ctx->sm_count));
     const int cost = waves * (t + 6);        // fill, drain and the final atomics cost about six tiles
     if (cost < best_cost) { best_cost = cost; best = ns; tps = t; }
@@ -207,12 +223,20 @@ int fs_tc_stats(fsharp_ctx* ctx, const void* Q, const void* K, const fsharp_dims
   CUtensorMap tmQ, tmK;
   FS_TRY(tchost::make_map_tokens(&tmQ, Q, fs_addr(dm->q_stride, H, dm->Lq, dm->d), B, H, dm->Lq, dm->d));
   FS_TRY(tchost::make_map_tokens(&tmK, K, fs_addr(dm->k_stride, H, dm->Lk, dm->d), B, H, dm->Lk, dm->d));
-  FS_CUDA_OK(cudaFuncSetAttribute(tc_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)StSmem::TOTAL + 1024));
   const int Bpool = dm->pool == FSHARP_POOL_PER_BH ? 1 : B;
-  FS_TIME_BEGIN(ctx, FS_K_TC_STATS);
-  (void)fs_launch_chained(tc_stats_kernel, dim3(best, BH, 2), dim3(ST_THREADS), StSmem::TOTAL + 1024, ctx->stream,
-      tmQ, tmK, H, dm->Lq, dm->Lk, dm->pool, Bpool, (double)qk_scale, tps, stats, ctx->d_status);
-  FS_TIME_END(ctx);
+  if (wide) {
+    FS_CUDA_OK(cudaFuncSetAttribute(tc_stats_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)StSmemT<true>::TOTAL + 1024));
+    FS_TIME_BEGIN(ctx, FS_K_TC_STATS);
+    (void)fs_launch_chained(tc_stats_kernel<true>, dim3(best, BH, 8), dim3(ST_THREADS), StSmemT<true>::TOTAL + 1024, ctx->stream,
+        tmQ, tmK, H, dm->Lq, dm->Lk, dm->pool, Bpool, (double)qk_scale, tps, stats, ctx->d_status);
+    FS_TIME_END(ctx);
+  } else {
+    FS_CUDA_OK(cudaFuncSetAttribute(tc_stats_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)StSmem::TOTAL + 1024));
+    FS_TIME_BEGIN(ctx, FS_K_TC_STATS);
+    (void)fs_launch_chained(tc_stats_kernel<false>, dim3(best, BH, 2), dim3(ST_THREADS), StSmem::TOTAL + 1024, ctx->stream,
+        tmQ, tmK, H, dm->Lq, dm->Lk, dm->pool, Bpool, (double)qk_scale, tps, stats, ctx->d_status);
+    FS_TIME_END(ctx);
+  }
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;
 }

@@ -69,10 +69,11 @@ def test_stats_pooled_over_batch_and_strided(ctx):
     assert np.abs(st2 - st).max() < 1e-12
 
 
-def test_stats_tensor_core_path_matches_simt_and_definition(ctx):
-    """bf16, d = 64 takes the tensor-core Gram kernel: several tiles, a ragged tail, unequal
-    query and key lengths, pooled and per-(batch, head) groups, and a query/key scale."""
-    w = W["cfg2"].scaled(B=2, H=3, L=1000)
+@pytest.mark.parametrize("name", ["cfg2", "cfg5"])
+def test_stats_tensor_core_path_matches_simt_and_definition(ctx, name):
+    """bf16, d = 64 and d = 128 (four 64 x 64 blocks over the column halves) take the tensor-core Gram kernel: several
+    tiles, a ragged tail, unequal query and key lengths, pooled and per-(batch, head) groups, and a query/key scale."""
+    w = W[name].scaled(B=2, H=3, L=1000)
     (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
     dKs, Ks = dK[:, :, :333], K[:, :, :333]
     for pool in (fb.POOL_PER_BH, fb.POOL_PER_HEAD):
