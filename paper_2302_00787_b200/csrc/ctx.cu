@@ -169,6 +169,7 @@ const char* fsharp_kernel_name(int id) {
     case FS_K_TC_ROWTERM: return "tc_rowterm_kernel";
     case FS_K_TC_FEAT: return "tc_feat_kernel";
     case FS_K_TC_LOGITS128: return "tc_logits128_kernel";
+    case FS_K_TC_SCORES128: return "tc_scores128_kernel";
     default: return "";
   }
 }

@@ -121,7 +121,7 @@ groupmax_kernel(const float* __restrict__ phi, int64_t per_bh, unsigned* __restr
 // shift: the row's largest exponent (ROW), the (batch, head)'s largest exponent (GROUP), or 0.
 __global__ void __launch_bounds__(NTH)
 expshift_kernel(float* __restrict__ phi, int L, int M, int stab, const unsigned* __restrict__ gmax,
-                float* __restrict__ logscale, int* __restrict__ status) {
+                float* __restrict__ logscale, __nv_bfloat16* __restrict__ phi16, int* __restrict__ status) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int bh = blockIdx.y;
   const float gshift = stab == FSHARP_STAB_GROUP ? ord2f(gmax[bh]) : 0.f;
@@ -141,7 +141,9 @@ expshift_kernel(float* __restrict__ phi, int L, int M, int stab, const unsigned*
     for (int m = lane; m < M; m += 32) {
       float e = row[m];
       if (!isfinite(e)) bad = true;
-      row[m] = expf(e - s);
+      const float f = expf(e - s);
+      row[m] = f;
+      if (phi16) phi16[((int64_t)bh * L + i) * M + m] = __float2bfloat16_rn(f);     // (a copy for the tensor-core score kernel)
     }
     if (bad) atomicExch(status, FSHARP_E_NONFINITE);
     if (logscale && lane == 0) {
@@ -315,7 +317,7 @@ out_kernel(const float* __restrict__ phiQ, const float* __restrict__ KV, const f
 template <typename T>
 int featurize_t(fsharp_ctx* ctx, const void* X, TensorAddr ax, int B, int H, int L, int d, int M, int pool,
                 const float* prep, int side, float qk_scale, int stab, float* rowc, unsigned* gmax, float* phi,
-                float* logscale) {
+                float* logscale, __nv_bfloat16* phi16 = nullptr) {
   const int BH = B * H;
   if (BH == 0 || L == 0) return FSHARP_OK;
   {
@@ -354,7 +356,7 @@ int featurize_t(fsharp_ctx* ctx, const void* X, TensorAddr ax, int B, int H, int
       FS_LAUNCH_CHECK(ctx);
     }
     FS_TIME_BEGIN(ctx, FS_K_EXPSHIFT);
-    expshift_kernel<<<dim3(gx, BH), NTH, 0, ctx->stream>>>(phi, L, M, stab, gmax, logscale, ctx->d_status);
+    expshift_kernel<<<dim3(gx, BH), NTH, 0, ctx->stream>>>(phi, L, M, stab, gmax, logscale, phi16, ctx->d_status);
     FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
   }
@@ -374,10 +376,15 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
   unsigned* gmax = ws->take<unsigned>((size_t)BH);
   float* lsq = unnormalised ? ws->take<float>((size_t)BH * Lq) : nullptr;
   float* lsk = unnormalised ? ws->take<float>((size_t)BH) : nullptr;
+  // causal, bf16 tensors: the in-chunk scores come from the tensor cores, from bf16 copies of the features
+  const bool tc_scores = causal && !unnormalised && sizeof(T) == 2 && ctx->impl != FSHARP_IMPL_SIMT &&
+                         fs_tc_scores128_supported(M, chunk);
+  __nv_bfloat16* phiQ16 = tc_scores ? ws->take<__nv_bfloat16>((size_t)BH * Lq * M) : nullptr;
+  __nv_bfloat16* phiK16 = tc_scores ? ws->take<__nv_bfloat16>((size_t)BH * Lk * M) : nullptr;
   FS_TRY(featurize_t<T>(ctx, K, ak, B, H, Lk, d, M, dm->pool, prep, 2, qk_scale, FSHARP_STAB_GROUP, rowc, gmax,
-                        phiK, lsk));
+                        phiK, lsk, phiK16));
   FS_TRY(featurize_t<T>(ctx, Q, aq, B, H, Lq, d, M, dm->pool, prep, 1, qk_scale, FSHARP_STAB_ROW, rowc, gmax,
-                        phiQ, lsq));
+                        phiQ, lsq, phiQ16));
   dim3 gout((Lq + TM - 1) / TM, (dv + TN - 1) / TN, BH);
   if (!causal) {
     float* KV = ws->take<float>((size_t)BH * M * N);
@@ -413,10 +420,14 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
     prefix_kernel<<<dim3((unsigned)((elems + NTH - 1) / NTH), BH), NTH, 0, ctx->stream>>>(st, nch, elems);
     FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
-    FS_TIME_BEGIN(ctx, FS_K_SCORES);
-    scores_kernel<<<dim3(C / TM, C / TN, BH * nch), NTH, 0, ctx->stream>>>(phiQ, phiK, Lq, M, C, nch, sc);
-    FS_TIME_END(ctx);
-    FS_LAUNCH_CHECK(ctx);
+    if (tc_scores) {
+      FS_TRY(fs_tc_scores128(ctx, phiQ16, phiK16, BH, Lq, M, C, sc));
+    } else {
+      FS_TIME_BEGIN(ctx, FS_K_SCORES);
+      scores_kernel<<<dim3(C / TM, C / TN, BH * nch), NTH, 0, ctx->stream>>>(phiQ, phiK, Lq, M, C, nch, sc);
+      FS_TIME_END(ctx);
+      FS_LAUNCH_CHECK(ctx);
+    }
     FS_TIME_BEGIN(ctx, FS_K_OUT);
     out_kernel<T><<<gout, NTH, 0, ctx->stream>>>(phiQ, st, sc, (const T*)V, av, (T*)Y, ay, H, Lq, M, dv, 1, C, nch,
                                                 nullptr, nullptr, ctx->d_status);
@@ -448,6 +459,7 @@ size_t fs_simt_attend_scratch_bytes(const fsharp_dims* dm, int causal, int chunk
   } else {
     size_t nch = chunk > 0 ? dm->Lq / chunk : 0;
     b += ws_round(BH * nch * dm->M * N * 4) + ws_round(BH * nch * (size_t)chunk * chunk * 4);
+    b += ws_round(BH * dm->Lq * dm->M * 2) + ws_round(BH * dm->Lk * dm->M * 2);      // bf16 copies of the features
   }
   return b;
 }
