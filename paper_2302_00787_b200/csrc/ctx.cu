@@ -170,6 +170,7 @@ const char* fsharp_kernel_name(int id) {
     case FS_K_TC_FEAT: return "tc_feat_kernel";
     case FS_K_TC_LOGITS128: return "tc_logits128_kernel";
     case FS_K_TC_SCORES128: return "tc_scores128_kernel";
+    case FS_K_TC_KV128: return "tc_kv128_kernel";
     default: return "";
   }
 }

@@ -248,7 +248,8 @@ __global__ void __launch_bounds__(NTH)
 out_kernel(const float* __restrict__ phiQ, const float* __restrict__ KV, const float* __restrict__ sc,
            const T* __restrict__ V, TensorAddr av, T* __restrict__ Y, TensorAddr ay, int H, int L, int M, int dv,
            int causal, int C, int nchunks, const float* __restrict__ lsq, const float* __restrict__ lsk,
-           int* __restrict__ status) {
+           int st_t, int* __restrict__ status) {
+  // st_t != 0: the states are stored column index first, [dv + 1][M] (the tensor-core key-side kernel writes them so)
   // lsq != nullptr: the unnormalised operator Khat C of Section 2.1 is wanted: row i of the numerator times
   // exp(lsq[i] + lsk[bh]), the shifts that the feature kernels took out of phi(Q) and phi(K)
   __shared__ Tiles sm;
@@ -269,7 +270,7 @@ out_kernel(const float* __restrict__ phiQ, const float* __restrict__ KV, const f
     int r = tid >> 2, part = tid & 3;
     float s = 0.f;
     if (i0 + r < L) {
-      for (int m = part; m < M; m += 4) s = fmaf(PQ[(int64_t)(i0 + r) * M + m], S[(int64_t)m * N + dv], s);
+      for (int m = part; m < M; m += 4) s = fmaf(PQ[(int64_t)(i0 + r) * M + m], st_t ? S[(int64_t)dv * M + m] : S[(int64_t)m * N + dv], s);
       if (causal)
         for (int j = part; j < C; j += 4) s += SC[(int64_t)(ic + r) * C + j];
     }
@@ -279,9 +280,14 @@ out_kernel(const float* __restrict__ phiQ, const float* __restrict__ KV, const f
   }
   __syncthreads();
   float acc[4][4] = {};
-  tile_gemm<true, false>(
-      acc, M, [&](int r, int k) { return (i0 + r < L) ? PQ[(int64_t)(i0 + r) * M + k] : 0.f; },
-      [&](int k, int c) { return (n0 + c < dv) ? S[(int64_t)k * N + n0 + c] : 0.f; }, sm);
+  if (st_t)
+    tile_gemm<true, true>(
+        acc, M, [&](int r, int k) { return (i0 + r < L) ? PQ[(int64_t)(i0 + r) * M + k] : 0.f; },
+        [&](int k, int c) { return (n0 + c < dv) ? S[(int64_t)(n0 + c) * M + k] : 0.f; }, sm);
+  else
+    tile_gemm<true, false>(
+        acc, M, [&](int r, int k) { return (i0 + r < L) ? PQ[(int64_t)(i0 + r) * M + k] : 0.f; },
+        [&](int k, int c) { return (n0 + c < dv) ? S[(int64_t)k * N + n0 + c] : 0.f; }, sm);
   if (causal) {
     const int jmax = min(C, ic + TM);   // columns beyond the tile's last row are masked to zero
     tile_gemm<true, false>(
@@ -403,18 +409,24 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
     FS_LAUNCH_CHECK(ctx);
     FS_TIME_BEGIN(ctx, FS_K_OUT);
     out_kernel<T><<<gout, NTH, 0, ctx->stream>>>(phiQ, KV, nullptr, (const T*)V, av, (T*)Y, ay, H, Lq, M, dv, 0, 0,
-                                                1, lsq, lsk, ctx->d_status);
+                                                1, lsq, lsk, 0, ctx->d_status);
     FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
   } else {
     const int C = chunk, nch = Lq / C;
     float* st = ws->take<float>((size_t)BH * nch * M * N);
     float* sc = ws->take<float>((size_t)BH * nch * C * C);
-    FS_TIME_BEGIN(ctx, FS_K_KV);
-    kv_kernel<T><<<dim3((M + TM - 1) / TM, (N + TN - 1) / TN, BH * nch), NTH, 0, ctx->stream>>>(
-        phiK, (const T*)V, av, H, Lk, M, dv, C, nch, 1, st);
-    FS_TIME_END(ctx);
-    FS_LAUNCH_CHECK(ctx);
+    // (with the bf16 copy of phi(K) at hand: the per-chunk sums on the tensor cores, stored column index first)
+    const bool tc_kv = tc_scores && fs_tc_kv128_supported(V, av, dv, M, C);
+    if (tc_kv) {
+      FS_TRY(fs_tc_kv128(ctx, phiK16, V, av, B, H, Lk, M, C, st));
+    } else {
+      FS_TIME_BEGIN(ctx, FS_K_KV);
+      kv_kernel<T><<<dim3((M + TM - 1) / TM, (N + TN - 1) / TN, BH * nch), NTH, 0, ctx->stream>>>(
+          phiK, (const T*)V, av, H, Lk, M, dv, C, nch, 1, st);
+      FS_TIME_END(ctx);
+      FS_LAUNCH_CHECK(ctx);
+    }
     int64_t elems = (int64_t)M * N;
     FS_TIME_BEGIN(ctx, FS_K_PREFIX);
     prefix_kernel<<<dim3((unsigned)((elems + NTH - 1) / NTH), BH), NTH, 0, ctx->stream>>>(st, nch, elems);
@@ -430,7 +442,7 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
     }
     FS_TIME_BEGIN(ctx, FS_K_OUT);
     out_kernel<T><<<gout, NTH, 0, ctx->stream>>>(phiQ, st, sc, (const T*)V, av, (T*)Y, ay, H, Lq, M, dv, 1, C, nch,
-                                                nullptr, nullptr, ctx->d_status);
+                                                nullptr, nullptr, tc_kv ? 1 : 0, ctx->d_status);
     FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
   }
