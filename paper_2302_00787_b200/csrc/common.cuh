@@ -50,7 +50,7 @@ enum { PS_BIAS = 0, PS_CSCALAR = 3, PS_CGAMMA = 4 };
 enum {
   FS_K_STATS = 1, FS_K_FIT, FS_K_PREP, FS_K_ROWTERM, FS_K_LOGITS, FS_K_GROUPMAX, FS_K_EXPSHIFT, FS_K_KV,
   FS_K_PREFIX, FS_K_SCORES, FS_K_OUT, FS_K_PAIRS, FS_K_PAIRVAR_PREP, FS_K_PAIRVAR, FS_K_PAIRPOOL,
-  FS_K_TC_KV, FS_K_TC_OUT, FS_K_TC_CAUSAL, FS_K_TC_STATS, FS_K_TC_ROWTERM, FS_K_TC_FEAT, FS_K_TC_LOGITS128, FS_K_TC_SCORES128, FS_K_TC_KV128,
+  FS_K_TC_KV, FS_K_TC_OUT, FS_K_TC_CAUSAL, FS_K_TC_STATS, FS_K_TC_ROWTERM, FS_K_TC_FEAT, FS_K_TC_LOGITS128, FS_K_TC_SCORES128, FS_K_TC_KV128, FS_K_TC_OUT128,
   FS_K_COUNT
 };
 constexpr int FS_TIMING_SLOTS = 4096;
@@ -208,10 +208,14 @@ int fs_tc_logits128(fsharp_ctx* ctx, const void* X, TensorAddr ax, int B, int H,
                     int side, float qk_scale, const float* rowc, float* phi);
 // Masked in-chunk scores from bf16 feature matrices [BH][L][M] on the tensor cores (tc_scores128.cu); sc [BH * L / C][C][C] fp32.
 int fs_tc_scores128_supported(int M, int C);
-int fs_tc_scores128(fsharp_ctx* ctx, const void* phiQ16, const void* phiK16, int BH, int L, int M, int C, float* sc);
+int fs_tc_scores128(fsharp_ctx* ctx, const void* phiQ16, const void* phiK16, int BH, int L, int M, int C, float* sc, void* sc16);
 // Per-chunk key-side sums from the bf16 copy of phi(K) on the tensor cores (tc_kv128.cu); st [BH * L / C][129][M] fp32.
 int fs_tc_kv128_supported(const void* V, TensorAddr av, int dv, int M, int C);
 int fs_tc_kv128(fsharp_ctx* ctx, const void* phiK16, const void* V, TensorAddr av, int B, int H, int L, int M, int C, float* st);
+// Query side of the causal chunked form from bf16 copies of phi(Q), the running sums and the scores (tc_out128.cu).
+int fs_tc_out128_supported(const void* Y, TensorAddr ay);
+int fs_tc_out128(fsharp_ctx* ctx, const void* phiQ16, const void* st16, const void* sc16, const void* V, TensorAddr av, void* Y,
+                 TensorAddr ay, int B, int H, int L, int M, int C);
 int fs_simt_attend(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const fsharp_dims* dm,
                    int dtype, int causal, int chunk, float qk_scale, const float* prep, void* Y,
                    WsAlloc* ws);

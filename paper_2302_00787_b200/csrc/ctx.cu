@@ -171,6 +171,7 @@ const char* fsharp_kernel_name(int id) {
     case FS_K_TC_LOGITS128: return "tc_logits128_kernel";
     case FS_K_TC_SCORES128: return "tc_scores128_kernel";
     case FS_K_TC_KV128: return "tc_kv128_kernel";
+    case FS_K_TC_OUT128: return "tc_out128_kernel";
     default: return "";
   }
 }

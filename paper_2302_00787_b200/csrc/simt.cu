@@ -195,7 +195,7 @@ kv_kernel(const float* __restrict__ phiK, const T* __restrict__ V, TensorAddr av
 
 // ---- exclusive prefix over chunks of the per-chunk S^T [V | 1] ---------------------------
 __global__ void __launch_bounds__(NTH)
-prefix_kernel(float* __restrict__ st, int nchunks, int64_t elems) {
+prefix_kernel(float* __restrict__ st, int nchunks, int64_t elems, __nv_bfloat16* __restrict__ st16) {
   const int bh = blockIdx.y;
   float* base = st + (int64_t)bh * nchunks * elems;
   for (int64_t e = blockIdx.x * (int64_t)NTH + threadIdx.x; e < elems; e += (int64_t)gridDim.x * NTH) {
@@ -207,7 +207,10 @@ prefix_kernel(float* __restrict__ st, int nchunks, int64_t elems) {
       for (int u = 0; u < 8; u++) v[u] = c0 + u < nchunks ? base[(c0 + u) * elems + e] : 0.f;
 #pragma unroll
       for (int u = 0; u < 8; u++) {
-        if (c0 + u < nchunks) base[(c0 + u) * elems + e] = run;
+        if (c0 + u < nchunks) {
+          base[(c0 + u) * elems + e] = run;
+          if (st16) st16[((int64_t)bh * nchunks + c0 + u) * elems + e] = __float2bfloat16_rn(run);   // (for the tensor-core query side)
+        }
         run += v[u];
       }
     }
@@ -418,6 +421,10 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
     float* sc = ws->take<float>((size_t)BH * nch * C * C);
     // (with the bf16 copy of phi(K) at hand: the per-chunk sums on the tensor cores, stored column index first)
     const bool tc_kv = tc_scores && fs_tc_kv128_supported(V, av, dv, M, C);
+    // ... and then the query side as well, from bf16 copies of the running sums and of the scores
+    const bool tc_out = tc_kv && fs_tc_out128_supported(Y, ay);
+    __nv_bfloat16* st16 = tc_out ? ws->take<__nv_bfloat16>((size_t)BH * nch * M * N) : nullptr;
+    __nv_bfloat16* sc16 = tc_out ? ws->take<__nv_bfloat16>((size_t)BH * nch * C * C) : nullptr;
     if (tc_kv) {
       FS_TRY(fs_tc_kv128(ctx, phiK16, V, av, B, H, Lk, M, C, st));
     } else {
@@ -429,22 +436,26 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
     }
     int64_t elems = (int64_t)M * N;
     FS_TIME_BEGIN(ctx, FS_K_PREFIX);
-    prefix_kernel<<<dim3((unsigned)((elems + NTH - 1) / NTH), BH), NTH, 0, ctx->stream>>>(st, nch, elems);
+    prefix_kernel<<<dim3((unsigned)((elems + NTH - 1) / NTH), BH), NTH, 0, ctx->stream>>>(st, nch, elems, st16);
     FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
     if (tc_scores) {
-      FS_TRY(fs_tc_scores128(ctx, phiQ16, phiK16, BH, Lq, M, C, sc));
+      FS_TRY(fs_tc_scores128(ctx, phiQ16, phiK16, BH, Lq, M, C, tc_out ? nullptr : sc, sc16));
     } else {
       FS_TIME_BEGIN(ctx, FS_K_SCORES);
       scores_kernel<<<dim3(C / TM, C / TN, BH * nch), NTH, 0, ctx->stream>>>(phiQ, phiK, Lq, M, C, nch, sc);
       FS_TIME_END(ctx);
       FS_LAUNCH_CHECK(ctx);
     }
-    FS_TIME_BEGIN(ctx, FS_K_OUT);
-    out_kernel<T><<<gout, NTH, 0, ctx->stream>>>(phiQ, st, sc, (const T*)V, av, (T*)Y, ay, H, Lq, M, dv, 1, C, nch,
-                                                nullptr, nullptr, tc_kv ? 1 : 0, ctx->d_status);
-    FS_TIME_END(ctx);
-    FS_LAUNCH_CHECK(ctx);
+    if (tc_out) {
+      FS_TRY(fs_tc_out128(ctx, phiQ16, st16, sc16, V, av, Y, ay, B, H, Lq, M, C));
+    } else {
+      FS_TIME_BEGIN(ctx, FS_K_OUT);
+      out_kernel<T><<<gout, NTH, 0, ctx->stream>>>(phiQ, st, sc, (const T*)V, av, (T*)Y, ay, H, Lq, M, dv, 1, C, nch,
+                                                  nullptr, nullptr, tc_kv ? 1 : 0, ctx->d_status);
+      FS_TIME_END(ctx);
+      FS_LAUNCH_CHECK(ctx);
+    }
   }
   return FSHARP_OK;
 }
@@ -472,6 +483,7 @@ size_t fs_simt_attend_scratch_bytes(const fsharp_dims* dm, int causal, int chunk
     size_t nch = chunk > 0 ? dm->Lq / chunk : 0;
     b += ws_round(BH * nch * dm->M * N * 4) + ws_round(BH * nch * (size_t)chunk * chunk * 4);
     b += ws_round(BH * dm->Lq * dm->M * 2) + ws_round(BH * dm->Lk * dm->M * 2);      // bf16 copies of the features
+    b += ws_round(BH * nch * dm->M * N * 2) + ws_round(BH * nch * (size_t)chunk * chunk * 2);   // ... of the running sums and the scores
   }
   return b;
 }

@@ -40,7 +40,13 @@ namespace tchost {
 
 // [B, H, L, inner] bf16 tensor with element strides a -> 4-D map (inner, token, head, batch),
 // box 64 x 128 x 1 x 1, 128-byte swizzle; rows beyond L read as zero.
+int make_map_rows(CUtensorMap* map, const void* base, TensorAddr a, int B, int H, int L, int inner, int box_rows);
 int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int H, int L, int inner) {
+  return make_map_rows(map, base, a, B, H, L, inner, TILE);
+}
+
+// The same with a box of 64 x box_rows (box_rows a multiple of 8, at most 256).
+int make_map_rows(CUtensorMap* map, const void* base, TensorAddr a, int B, int H, int L, int inner, int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return FSHARP_E_CUDA;
   cuuint64_t dims[4] = {(cuuint64_t)inner, (cuuint64_t)L, (cuuint64_t)H, (cuuint64_t)B};
@@ -48,7 +54,7 @@ int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int
   // a dimension of size one may carry any stride; give it a legal one
   if (H == 1 && strides[1] == 0) strides[1] = strides[0] * (cuuint64_t)L;
   if (B == 1 && strides[2] == 0) strides[2] = strides[1] * (cuuint64_t)H;
-  cuuint32_t box[4] = {64, (cuuint32_t)TILE, 1, 1};
+  cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,

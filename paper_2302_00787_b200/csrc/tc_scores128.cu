@@ -5,7 +5,7 @@
 // One block = one 128 x 128 tile of a chunk's C x C score block.  Tiles above the diagonal are all zero and are only
 // written.  The feature index is the contraction: 64 features of both token tiles per TMA stage (two panels with the
 // 128-byte swizzle), four MMAs of N = 128 per stage into one accumulator in tensor memory; the epilogue masks the
-// diagonal tile and writes fp32 rows.
+// diagonal tile and writes the rows (fp32, bf16, or both).
 #include "common.cuh"
 #include "tc_common.cuh"
 #include "tc_layout.cuh"
@@ -32,7 +32,8 @@ static_assert(sizeof(ScMisc) <= 256, "misc block");
 
 __global__ void __launch_bounds__(SC_THREADS, 2)
 tc_scores128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, float* __restrict__ sc,
-                    int M, int C, int nch, int* __restrict__ status) {
+                    __nv_bfloat16* __restrict__ sc16, int M, int C, int nch, int* __restrict__ status) {
+  // sc (fp32) and sc16 (bf16): either may be null
   fs_grid_dependency_wait();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -40,10 +41,15 @@ tc_scores128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nt = C / TILE, ti = blockIdx.x / nt, tj = blockIdx.x % nt;
   const int c = blockIdx.y, bh = blockIdx.z;
-  float* S = sc + ((size_t)bh * nch + c) * C * C + (size_t)ti * TILE * C + (size_t)tj * TILE;
+  const size_t toff = ((size_t)bh * nch + c) * C * C + (size_t)ti * TILE * C + (size_t)tj * TILE;
+  float* S = sc + toff;
+  __nv_bfloat16* S16 = sc16 + toff;
   if (tj > ti) {                               // above the diagonal: zeros (uniform over the block)
-    for (int e = threadIdx.x; e < TILE * (TILE / 4); e += SC_THREADS)
-      *reinterpret_cast<float4*>(S + (size_t)(e / (TILE / 4)) * C + 4 * (e % (TILE / 4))) = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int e = threadIdx.x; e < TILE * (TILE / 4); e += SC_THREADS) {
+      const size_t o = (size_t)(e / (TILE / 4)) * C + 4 * (e % (TILE / 4));
+      if (sc) *reinterpret_cast<float4*>(S + o) = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (sc16) *reinterpret_cast<uint2*>(S16 + o) = make_uint2(0u, 0u);
+    }
     return;
   }
   const int nk = M / 64;
@@ -113,18 +119,26 @@ tc_scores128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       __syncwarp();
       tcgen05_fence_after();
       float* out = S + (size_t)row * C;
+      __nv_bfloat16* out16 = S16 + (size_t)row * C;
       const int last = ti == tj ? row : TILE;          // columns up to `last` (inclusive) are kept
 #pragma unroll
       for (int cc = 0; cc < TILE / 16; cc++) {
         uint32_t t[16];
         tmem_ld16(lane_addr + cc * 16, t);
         tmem_wait_ld();
+        float v[16];
 #pragma unroll
-        for (int j = 0; j < 4; j++) {
-          const int c0 = cc * 16 + 4 * j;
-          *reinterpret_cast<float4*>(out + c0) =
-              make_float4(c0 <= last ? __uint_as_float(t[4 * j]) : 0.f, c0 + 1 <= last ? __uint_as_float(t[4 * j + 1]) : 0.f,
-                          c0 + 2 <= last ? __uint_as_float(t[4 * j + 2]) : 0.f, c0 + 3 <= last ? __uint_as_float(t[4 * j + 3]) : 0.f);
+        for (int j = 0; j < 16; j++) v[j] = cc * 16 + j <= last ? __uint_as_float(t[j]) : 0.f;
+        if (sc) {
+#pragma unroll
+          for (int j = 0; j < 4; j++) *reinterpret_cast<float4*>(out + cc * 16 + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        }
+        if (sc16) {
+          uint32_t o[8];
+#pragma unroll
+          for (int j = 0; j < 8; j++) o[j] = pack_bf16(v[2 * j], v[2 * j + 1]);
+          *reinterpret_cast<uint4*>(out16 + cc * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+          *reinterpret_cast<uint4*>(out16 + cc * 16 + 8) = make_uint4(o[4], o[5], o[6], o[7]);
         }
       }
       tcgen05_fence_before();
@@ -147,8 +161,8 @@ int make_map_tokens(CUtensorMap* map, const void* base, TensorAddr a, int B, int
 // bf16 feature matrices, M a multiple of 64, chunks of 128 or 256 tokens
 int fs_tc_scores128_supported(int M, int C) { return M % 64 == 0 && M >= 64 && (C == 128 || C == 256); }
 
-// phiQ16, phiK16: [BH][L][M] bf16 (L a multiple of C); sc: [BH * L / C][C][C] fp32
-int fs_tc_scores128(fsharp_ctx* ctx, const void* phiQ16, const void* phiK16, int BH, int L, int M, int C, float* sc) {
+// phiQ16, phiK16: [BH][L][M] bf16 (L a multiple of C); sc (fp32) and sc16 (bf16): [BH * L / C][C][C], either may be null
+int fs_tc_scores128(fsharp_ctx* ctx, const void* phiQ16, const void* phiK16, int BH, int L, int M, int C, float* sc, void* sc16) {
   const int nch = L / C, nt = C / TILE;
   CUtensorMap tmQ, tmK;
   TensorAddr a{(int64_t)BH * L * M, (int64_t)L * M, (int64_t)M};
@@ -156,7 +170,7 @@ int fs_tc_scores128(fsharp_ctx* ctx, const void* phiQ16, const void* phiK16, int
   FS_TRY(tchost::make_map_tokens(&tmK, phiK16, a, 1, BH, L, M));
   FS_CUDA_OK(cudaFuncSetAttribute(tc_scores128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScSmem::TOTAL + 1024));
   FS_TIME_BEGIN(ctx, FS_K_TC_SCORES128);
-  tc_scores128_kernel<<<dim3(nt * nt, nch, BH), SC_THREADS, ScSmem::TOTAL + 1024, ctx->stream>>>(tmQ, tmK, sc, M, C, nch, ctx->d_status);
+  tc_scores128_kernel<<<dim3(nt * nt, nch, BH), SC_THREADS, ScSmem::TOTAL + 1024, ctx->stream>>>(tmQ, tmK, sc, (__nv_bfloat16*)sc16, M, C, nch, ctx->d_status);
   FS_TIME_END(ctx);
   FS_LAUNCH_CHECK(ctx);
   return FSHARP_OK;
