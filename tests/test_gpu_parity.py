@@ -488,6 +488,41 @@ def test_attend_strided_layout_per_head_omega_and_pooling(ctx):
             assert rel_err(Y[b, h], ref) < TOL["bf16"]
 
 
+@pytest.mark.parametrize("chunk,M", [(128, 256), (256, 384), (64, 512)])
+def test_causal_d128_chain_of_tensor_core_kernels(ctx, chunk, M):
+    """bf16, d = dv = 128 has no fused kernel: exponents, in-chunk scores, per-chunk key-side sums and the query side
+    each run on the tensor cores (chunk 64 leaves the last three to the fp32 kernels).  [B, L, H, *] storage,
+    per-head Omega, parameters pooled per head, several chunks, a query / key scale; against the definition, unit by
+    unit, and against the fp32 kernels."""
+    w = W["cfg5"].scaled(B=2, H=2, L=768, M=M, chunk=chunk, outlier_frac=0.05)
+    (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
+    OmH = np.stack([wl.orthogonal_omega(w.M, w.d, 31 + h) for h in range(w.H)])
+    s = 0.95
+    st = ctx.fsharp_stats(dQ, dK, pool=fb.POOL_PER_HEAD, qk_scale=s)
+    pr = ctx.fsharp_fit_params(st, w.d, "sderf")
+    tr = lambda t: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    out = torch.empty(w.B, w.L, w.H, w.dv, dtype=dQ.dtype, device="cuda").permute(0, 2, 1, 3)
+    n0 = ctx.launch_count()
+    Y = ctx.fsharp_attend(tr(dQ), tr(dK), tr(dV), dev(OmH), pr, causal=True, chunk=chunk, pool=fb.POOL_PER_HEAD, qk_scale=s, out=out)
+    launches = ctx.launch_count() - n0
+    ctx.set_impl(fb.IMPL_SIMT)
+    try:
+        Y32 = ctx.fsharp_attend(tr(dQ), tr(dK), tr(dV), dev(OmH), pr, causal=True, chunk=chunk, pool=fb.POOL_PER_HEAD, qk_scale=s)
+    finally:
+        ctx.set_impl(fb.IMPL_AUTO)
+    assert ctx.status() == 0 and launches == 12        # prep; 4 + 3 feature kernels; sums, scan, scores, query side
+    Y, Y32 = host(Y), host(Y32)
+    prh = pr.cpu().numpy()
+    for b in range(w.B):
+        for h in range(w.H):
+            p = fb.unpack_params(prh[h], w.d)
+            ref = fs.favor_sharp_attention(Q[b, h], K[b, h], V[b, h], OmH[h], p, causal=True, qk_scale=s)
+            assert rel_err(Y[b, h], ref) < TOL["bf16"], (b, h, rel_err(Y[b, h], ref))
+            assert rel_err(Y32[b, h], ref) < TOL["bf16"]
+            assert rel_err(Y[b, h], Y32[b, h]) < TOL["bf16"]
+    assert np.abs(Y[:, :, 0] - V[:, :, 0]).max() < 1e-2        # the first token attends to itself only
+
+
 def test_qk_scale_is_applied(ctx):
     w = W["cfg1"]
     (Q, K, V, Om), (dQ, dK, dV, dOm) = upload(w)
