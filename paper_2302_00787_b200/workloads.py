@@ -56,6 +56,9 @@ WORKLOADS = {
                       seed=3000),
     "cfg5": Workload("cfg5", 1, 16, 65536, 128, 128, 512, "bf16", "sderf", True, 256, "orthogonal",
                      outlier_frac=0.05, outlier_scale=3.0, seed=5000),
+    # cfg5 at a quarter of its length: small enough for a profiler capture, inputs still larger than L2
+    "cfg5m": Workload("cfg5m", 1, 16, 16384, 128, 128, 512, "bf16", "sderf", True, 256, "orthogonal",
+                      outlier_frac=0.05, outlier_scale=3.0, seed=5000),
     # cfg5's few, long sequences (1 x 16 heads x 65536 tokens, x3 outlier tokens) at the head size of cfg2 / cfg3
     "cfg5s": Workload("cfg5s", 1, 16, 65536, 64, 64, 256, "bf16", "sderf", True, 128, "orthogonal",
                       outlier_frac=0.05, outlier_scale=3.0, seed=5500),
