@@ -121,7 +121,8 @@ groupmax_kernel(const float* __restrict__ phi, int64_t per_bh, unsigned* __restr
 // shift: the row's largest exponent (ROW), the (batch, head)'s largest exponent (GROUP), or 0.
 __global__ void __launch_bounds__(NTH)
 expshift_kernel(float* __restrict__ phi, int L, int M, int stab, const unsigned* __restrict__ gmax,
-                float* __restrict__ logscale, __nv_bfloat16* __restrict__ phi16, int* __restrict__ status) {
+                float* __restrict__ logscale, __nv_bfloat16* __restrict__ phi16, int keep32, int* __restrict__ status) {
+  // keep32 == 0 (only with phi16): the fp32 features have no reader, only the bf16 copy is written
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int bh = blockIdx.y;
   const float gshift = stab == FSHARP_STAB_GROUP ? ord2f(gmax[bh]) : 0.f;
@@ -142,7 +143,7 @@ expshift_kernel(float* __restrict__ phi, int L, int M, int stab, const unsigned*
       float e = row[m];
       if (!isfinite(e)) bad = true;
       const float f = expf(e - s);
-      row[m] = f;
+      if (keep32) row[m] = f;
       if (phi16) phi16[((int64_t)bh * L + i) * M + m] = __float2bfloat16_rn(f);     // (a copy for the tensor-core score kernel)
     }
     if (bad) atomicExch(status, FSHARP_E_NONFINITE);
@@ -326,7 +327,7 @@ out_kernel(const float* __restrict__ phiQ, const float* __restrict__ KV, const f
 template <typename T>
 int featurize_t(fsharp_ctx* ctx, const void* X, TensorAddr ax, int B, int H, int L, int d, int M, int pool,
                 const float* prep, int side, float qk_scale, int stab, float* rowc, unsigned* gmax, float* phi,
-                float* logscale, __nv_bfloat16* phi16 = nullptr) {
+                float* logscale, __nv_bfloat16* phi16 = nullptr, bool keep32 = true) {
   const int BH = B * H;
   if (BH == 0 || L == 0) return FSHARP_OK;
   {
@@ -365,7 +366,7 @@ int featurize_t(fsharp_ctx* ctx, const void* X, TensorAddr ax, int B, int H, int
       FS_LAUNCH_CHECK(ctx);
     }
     FS_TIME_BEGIN(ctx, FS_K_EXPSHIFT);
-    expshift_kernel<<<dim3(gx, BH), NTH, 0, ctx->stream>>>(phi, L, M, stab, gmax, logscale, phi16, ctx->d_status);
+    expshift_kernel<<<dim3(gx, BH), NTH, 0, ctx->stream>>>(phi, L, M, stab, gmax, logscale, phi16, (keep32 || !phi16) ? 1 : 0, ctx->d_status);
     FS_TIME_END(ctx);
     FS_LAUNCH_CHECK(ctx);
   }
@@ -388,12 +389,16 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
   // causal, bf16 tensors: the in-chunk scores come from the tensor cores, from bf16 copies of the features
   const bool tc_scores = causal && !unnormalised && sizeof(T) == 2 && ctx->impl != FSHARP_IMPL_SIMT &&
                          fs_tc_scores128_supported(M, chunk);
+  // (with the bf16 copy of phi(K) at hand: the per-chunk sums on the tensor cores, stored column index first; and then
+  // the query side as well, from bf16 copies of the running sums and of the scores)
+  const bool tc_kv = tc_scores && fs_tc_kv128_supported(V, av, dv, M, chunk);
+  const bool tc_out = tc_kv && fs_tc_out128_supported(Y, ay);
   __nv_bfloat16* phiQ16 = tc_scores ? ws->take<__nv_bfloat16>((size_t)BH * Lq * M) : nullptr;
   __nv_bfloat16* phiK16 = tc_scores ? ws->take<__nv_bfloat16>((size_t)BH * Lk * M) : nullptr;
   FS_TRY(featurize_t<T>(ctx, K, ak, B, H, Lk, d, M, dm->pool, prep, 2, qk_scale, FSHARP_STAB_GROUP, rowc, gmax,
-                        phiK, lsk, phiK16));
+                        phiK, lsk, phiK16, !tc_kv));
   FS_TRY(featurize_t<T>(ctx, Q, aq, B, H, Lq, d, M, dm->pool, prep, 1, qk_scale, FSHARP_STAB_ROW, rowc, gmax,
-                        phiQ, lsq, phiQ16));
+                        phiQ, lsq, phiQ16, !tc_out));
   dim3 gout((Lq + TM - 1) / TM, (dv + TN - 1) / TN, BH);
   if (!causal) {
     float* KV = ws->take<float>((size_t)BH * M * N);
@@ -419,10 +424,6 @@ int attend_t(fsharp_ctx* ctx, const void* Q, const void* K, const void* V, const
     const int C = chunk, nch = Lq / C;
     float* st = ws->take<float>((size_t)BH * nch * M * N);
     float* sc = ws->take<float>((size_t)BH * nch * C * C);
-    // (with the bf16 copy of phi(K) at hand: the per-chunk sums on the tensor cores, stored column index first)
-    const bool tc_kv = tc_scores && fs_tc_kv128_supported(V, av, dv, M, C);
-    // ... and then the query side as well, from bf16 copies of the running sums and of the scores
-    const bool tc_out = tc_kv && fs_tc_out128_supported(Y, ay);
     __nv_bfloat16* st16 = tc_out ? ws->take<__nv_bfloat16>((size_t)BH * nch * M * N) : nullptr;
     __nv_bfloat16* sc16 = tc_out ? ws->take<__nv_bfloat16>((size_t)BH * nch * C * C) : nullptr;
     if (tc_kv) {
