@@ -96,8 +96,11 @@ int fsharp_destroy(fsharp_ctx* ctx);
 int fsharp_set_stream(fsharp_ctx* ctx, void* stream);
 /* Forces a kernel family for fsharp_attend and fsharp_featurize (FSHARP_IMPL_*).  AUTO picks the
  * tensor-core kernels when the shape allows it: bf16, d = dv = 64, M = 256 (attend, bidirectional or causal with
- * Lq == Lk; featurize with a row shift or none); everything else runs on the fp32 kernels.  TENSOR refuses
- * (FSHARP_E_SHAPE) what the tensor-core kernels do not cover. */
+ * Lq == Lk; featurize with a row shift or none).  bf16 tensors with d = 128 have no fused kernel: under AUTO their
+ * statistics, the exponents' product and, for causal attention with dv = 128, M a multiple of 128 and chunk 128 or 256,
+ * the in-chunk scores, the per-chunk key-side sums and the query side run as separate tensor-core kernels, the rest
+ * (shift and exponential, scan over chunks) on the fp32 kernels.  Everything else runs on the fp32 kernels.  TENSOR
+ * refuses (FSHARP_E_SHAPE) what the fused tensor-core kernels do not cover; SIMT forces the fp32 kernels throughout. */
 int fsharp_set_impl(fsharp_ctx* ctx, int impl);
 /* Synchronises the stream, then returns the latched device status in *code
  * (0 or a negative FSHARP_E_*), and clears it. */
