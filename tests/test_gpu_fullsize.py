@@ -128,7 +128,7 @@ def test_full_size_backward_parity(ctx, name, unit):
     assert (s_dv - s_dy).abs().max().item() < 2e-2 * s_dy.abs().max().item()
 
 
-@pytest.mark.parametrize("name", ["cfg3", "cfg3b"])
+@pytest.mark.parametrize("name", ["cfg3", "cfg3b", "cfg5m"])
 def test_repeated_calls_agree_bit_for_bit(ctx, name):
     """Nothing on the attention path of these workloads adds across blocks with atomics, so a call repeated on the same
     inputs must give the same bits: 200 calls against the first (a kernel whose result depends on timing shows up
@@ -138,10 +138,12 @@ def test_repeated_calls_agree_bit_for_bit(ctx, name):
     host_in, (dQ, dK, dV, dOm), pr, Y = run_full(ctx, w)
     Y0 = Y.clone()
     differ = 0
-    for _ in range(200):
+    for _ in range(200 if w.d == 64 else 60):
         ctx.fsharp_attend(dQ, dK, dV, dOm, pr, causal=w.causal, chunk=w.chunk, out=Y)
         differ += int(not torch.equal(Y, Y0))
     assert differ == 0
+    if w.d != 64:           # (the chain of kernels for d = 128: its exponents come out of fsharp_attend's own kernels)
+        return
     phi0, ls0 = ctx.fsharp_featurize(dK, dOm, pr, side=2, stab=fb.STAB_ROW)
     for _ in range(10):
         phi, ls = ctx.fsharp_featurize(dK, dOm, pr, side=2, stab=fb.STAB_ROW)
